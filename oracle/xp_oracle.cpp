@@ -1,0 +1,328 @@
+// CPU ORACLE -- TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, single-threaded statement of what the repair search computes.
+// Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
+// build or call this file; the product path never does, and it shares no code
+// with the CUDA library.
+//
+// What it computes (Section 4.4, Algorithm 3: the CreateSMTQuery / SynthesisCode
+// steps).  The paper enumerates one constraint per concrete index of the snippet
+// and asks a solver to fill the sketch's missing expressions so that all of them
+// hold.  Here that question is answered by its definition over a bounded grammar:
+//
+//   for every size k = 1..K and every derivation tree e of the start symbol with
+//   exactly k nodes, taken in canonical order,
+//       match(e)  <=>  for every domain point p:
+//                      e(p) is defined, ctx(e(p), p) is defined and equals spec(p)
+//   cand_count[k]  = number of trees of size k
+//   match_count[k] = number of matching trees of size k
+//   least          = the matching tree with the smallest (size, rank)
+//
+// Readings the paper leaves open (it prints no grammar, order or arithmetic):
+//   * size = number of tree nodes (each leaf 1, each operator 1);
+//   * canonical order within (nonterminal, size): by production in the order the
+//     grammar lists them; for a binary production by left size ascending, then
+//     left subtree rank, then right subtree rank (fastest); a size-1 tree's rank
+//     is the position of its leaf production among the nonterminal's leaves;
+//   * values are int64 with wrap-around; '/' truncates toward zero, '%' takes the
+//     dividend's sign; INT64_MIN / -1 = INT64_MIN and INT64_MIN % -1 = 0;
+//   * a zero divisor anywhere in a tree (or in the context, or in the spec) at a
+//     point makes the candidate fail at that point, with no short-circuiting;
+//   * comparison and logic operators (context / spec only) yield 0 or 1 and
+//     evaluate both operands.
+//
+// Parity against the paper itself is unpinned: it prints no instance, query or
+// solution for this step (its constraint figure is not available).  The functions
+// below are pinned by the tests against closed-form counts, hand-derived match
+// sets, a separate brute force over materialised trees, and invariants.
+
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <string>
+#include <vector>
+
+typedef uint64_t u64;
+typedef int64_t i64;
+
+enum { XO_MAX_SIZE = 15 };
+enum { OP_ADD = 0, OP_SUB, OP_MUL, OP_DIV, OP_MOD, OP_LT, OP_LE, OP_EQ, OP_NE, OP_MIN, OP_MAX, OP_AND, OP_OR, OP_COUNT };
+enum { K_VAR = 0, K_CONST = 1, K_HOLE = 2, K_OP = 3 };
+enum { P_VAR = 0, P_CONST = 1, P_BIN = 2 };
+
+extern "C" {
+
+struct xo_prod { int32_t lhs, kind, var, op, left, right; i64 value; };
+struct xo_instr { int32_t kind, arg; i64 value; };
+
+struct xo_grammar {
+    int32_t n_vars;
+    const i64* lo;                 // inclusive lower bounds
+    const i64* hi;                 // exclusive upper bounds
+    const char* const* var_names;
+    int32_t n_nt;
+    int32_t n_prods;
+    const xo_prod* prods;
+};
+
+struct xo_problem {
+    xo_grammar g;
+    i64 n_points;
+    const int32_t* coords;         // null: the full box of the variable ranges, first variable slowest
+    i64 n_first;                   // optional: point indices checked before the rest (any order is allowed:
+    const i64* first_points;       //   mismatch and invalidity are not told apart, so the order is free)
+    int32_t start_nt, max_size;
+    int32_t ctx_len;  const xo_instr* ctx;         // 0 = identity
+    int32_t spec_len; const xo_instr* spec_expr;   // used when spec_table is null
+    const i64* spec_table;                          // n_points values
+    const u64* rank_begin;         // optional windows per size [max_size+1]; null = everything
+    const u64* rank_end;
+};
+
+struct xo_result {
+    u64 cand_count[XO_MAX_SIZE + 1];
+    u64 match_count[XO_MAX_SIZE + 1];
+    int32_t solved, least_size;
+    u64 least_rank;
+    u64 evals;                     // candidate-point evaluations carried out
+    char least_text[1024];
+};
+
+}  // extern "C"
+
+namespace {
+
+// ---- arithmetic (C semantics on int64, zero divisors reported) ---------------
+
+bool apply_op(int op, i64 a, i64 b, i64& out) {
+    switch (op) {
+        case OP_ADD: out = (i64)((u64)a + (u64)b); return true;
+        case OP_SUB: out = (i64)((u64)a - (u64)b); return true;
+        case OP_MUL: out = (i64)((u64)a * (u64)b); return true;
+        case OP_DIV:
+            if (b == 0) return false;
+            out = (b == -1) ? (i64)(0 - (u64)a) : a / b;
+            return true;
+        case OP_MOD:
+            if (b == 0) return false;
+            out = (b == -1) ? 0 : a % b;
+            return true;
+        case OP_LT: out = a < b; return true;
+        case OP_LE: out = a <= b; return true;
+        case OP_EQ: out = a == b; return true;
+        case OP_NE: out = a != b; return true;
+        case OP_MIN: out = a < b ? a : b; return true;
+        case OP_MAX: out = a > b ? a : b; return true;
+        case OP_AND: out = (a != 0) && (b != 0); return true;
+        case OP_OR: out = (a != 0) || (b != 0); return true;
+    }
+    return false;
+}
+
+const char* const OP_TEXT[OP_COUNT] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
+
+// Postfix evaluation of a context or spec expression at one point.
+bool eval_code(const xo_instr* code, int n, const i64* pt, i64 hole, i64& out) {
+    i64 st[64];
+    int sp = 0;
+    for (int i = 0; i < n; ++i) {
+        const xo_instr& c = code[i];
+        if (c.kind == K_VAR) st[sp++] = pt[c.arg];
+        else if (c.kind == K_CONST) st[sp++] = c.value;
+        else if (c.kind == K_HOLE) st[sp++] = hole;
+        else {
+            i64 b = st[--sp], a = st[--sp], r;
+            if (!apply_op(c.arg, a, b, r)) return false;
+            st[sp++] = r;
+        }
+        if (sp >= 63) return false;
+    }
+    if (sp != 1) return false;
+    out = st[0];
+    return true;
+}
+
+// ---- grammar, counts -------------------------------------------------------------
+
+struct Node { const xo_prod* p; Node* l; Node* r; };
+
+struct Gram {
+    const xo_grammar* g;
+    std::vector<std::vector<const xo_prod*>> of;          // productions per nonterminal, in order
+    std::vector<std::vector<u64>> cnt;                     // cnt[nt][size]
+    bool overflow = false;
+
+    Gram(const xo_grammar* g_, int max_size) : g(g_) {
+        of.resize(g->n_nt);
+        for (int i = 0; i < g->n_prods; ++i) of[g->prods[i].lhs].push_back(&g->prods[i]);
+        cnt.assign(g->n_nt, std::vector<u64>(max_size + 1, 0));
+        for (int s = 1; s <= max_size; ++s)
+            for (int nt = 0; nt < g->n_nt; ++nt) {
+                unsigned __int128 c = 0;
+                for (const xo_prod* p : of[nt]) {
+                    if (p->kind != P_BIN) { if (s == 1) c += 1; }
+                    else for (int a = 1; a <= s - 2; ++a)
+                        c += (unsigned __int128)cnt[p->left][a] * cnt[p->right][s - 1 - a];
+                    if (c >> 63) { overflow = true; c = 0; }
+                }
+                cnt[nt][s] = (u64)c;
+            }
+    }
+};
+
+typedef std::function<void()> Fn;
+
+// Calls k() once for every tree of (nt, size) whose rank lies in [lo, hi), in
+// canonical order, with `out` pointing at the tree.
+void gen(const Gram& G, int nt, int size, u64 lo, u64 hi, Node*& out, const Fn& k) {
+    u64 base = 0;
+    for (const xo_prod* p : G.of[nt]) {
+        if (p->kind != P_BIN) {
+            if (size == 1) {
+                if (base >= lo && base < hi) { Node n{p, nullptr, nullptr}; out = &n; k(); }
+                ++base;
+            }
+            continue;
+        }
+        for (int a = 1; a <= size - 2; ++a) {
+            const int b = size - 1 - a;
+            const u64 cl = G.cnt[p->left][a], cr = G.cnt[p->right][b];
+            const u64 block = cl * cr;
+            if (block == 0) continue;
+            if (base + block <= lo || base >= hi) { base += block; continue; }
+            const u64 wlo = lo > base ? lo - base : 0;                     // window inside this block
+            const u64 whi = (hi - base < block) ? hi - base : block;
+            Node n{p, nullptr, nullptr};
+            out = &n;
+            u64 l = wlo / cr;                                              // rank of the current left subtree
+            gen(G, p->left, a, wlo / cr, (whi + cr - 1) / cr, n.l, [&]() {
+                const u64 row = l * cr;
+                const u64 rlo = wlo > row ? wlo - row : 0;
+                const u64 rhi = (whi - row < cr) ? whi - row : cr;
+                gen(G, p->right, b, rlo, rhi, n.r, [&]() { out = &n; k(); });
+                ++l;
+            });
+            base += block;
+        }
+    }
+}
+
+bool eval_tree(const Node* n, const i64* pt, i64& out) {
+    if (n->p->kind == P_VAR) { out = pt[n->p->var]; return true; }
+    if (n->p->kind == P_CONST) { out = n->p->value; return true; }
+    i64 a, b;
+    const bool va = eval_tree(n->l, pt, a);
+    const bool vb = eval_tree(n->r, pt, b);
+    if (!va || !vb) return false;
+    return apply_op(n->p->op, a, b, out);
+}
+
+void tree_text(const xo_grammar* g, const Node* n, std::string& s) {
+    if (n->p->kind == P_VAR) { s += g->var_names ? g->var_names[n->p->var] : ("v" + std::to_string(n->p->var)); return; }
+    if (n->p->kind == P_CONST) { s += std::to_string((long long)n->p->value); return; }
+    s += "("; tree_text(g, n->l, s); s += OP_TEXT[n->p->op]; tree_text(g, n->r, s); s += ")";
+}
+
+}  // namespace
+
+extern "C" {
+
+// Number of derivation trees per size for nonterminal nt; returns 1 if a count reaches 2^63.
+int xo_counts(const xo_grammar* g, int nt, int max_size, u64* out) {
+    Gram G(g, max_size);
+    for (int s = 0; s <= max_size; ++s) out[s] = G.cnt[nt][s];
+    return G.overflow ? 1 : 0;
+}
+
+// Texts of the trees of (nt, size) with rank in [begin, end), one per line.
+// Returns the number of bytes needed (including the final NUL).
+i64 xo_list(const xo_grammar* g, int nt, int size, u64 begin, u64 end, char* buf, i64 buflen) {
+    Gram G(g, size);
+    std::string all;
+    Node* root = nullptr;
+    if (end > G.cnt[nt][size]) end = G.cnt[nt][size];
+    gen(G, nt, size, begin, end, root, [&]() { tree_text(g, root, all); all += "\n"; });
+    if ((i64)all.size() + 1 <= buflen) memcpy(buf, all.c_str(), all.size() + 1);
+    return (i64)all.size() + 1;
+}
+
+// Value of a postfix expression at one point (returns 0 when a divisor is zero).
+int xo_eval_code(const xo_instr* code, int n, const i64* pt, i64 hole, i64* out) {
+    return eval_code(code, n, pt, hole, *out) ? 1 : 0;
+}
+
+// The repair search for one hole.  Returns 0, or 1 on a malformed problem.
+int xo_repair(const xo_problem* P, xo_result* R) {
+    memset(R, 0, sizeof(*R));
+    const xo_grammar* g = &P->g;
+    const int K = P->max_size;
+    if (K < 1 || K > XO_MAX_SIZE || g->n_vars > 16) return 1;
+    Gram G(g, K);
+    if (G.overflow) return 1;
+    const int nv = g->n_vars;
+    const i64 np = P->n_points;
+
+    // Every domain point and the spec's value there.
+    std::vector<i64> pts((size_t)np * (nv ? nv : 1));
+    for (i64 p = 0; p < np; ++p) {
+        if (P->coords) for (int d = 0; d < nv; ++d) pts[p * nv + d] = P->coords[p * nv + d];
+        else {
+            i64 rem = p;
+            for (int d = nv - 1; d >= 0; --d) {
+                const i64 ext = g->hi[d] - g->lo[d];
+                pts[p * nv + d] = g->lo[d] + rem % ext;
+                rem /= ext;
+            }
+        }
+    }
+    std::vector<i64> spec(np);
+    std::vector<char> spec_ok(np, 1);
+    for (i64 p = 0; p < np; ++p) {
+        if (P->spec_table) spec[p] = P->spec_table[p];
+        else spec_ok[p] = eval_code(P->spec_expr, P->spec_len, &pts[p * nv], 0, spec[p]);
+    }
+    // Order in which points are tried: the caller's "first" points, then all of them.
+    std::vector<i64> order;
+    for (i64 i = 0; i < P->n_first; ++i) order.push_back(P->first_points[i]);
+    for (i64 p = 0; p < np; ++p) order.push_back(p);
+
+    for (int k = 1; k <= K; ++k) {
+        R->cand_count[k] = G.cnt[P->start_nt][k];
+        u64 lo = 0, hi = R->cand_count[k];
+        if (P->rank_begin) {
+            lo = P->rank_begin[k];
+            if (P->rank_end[k] < hi) hi = P->rank_end[k];
+        }
+        if (lo >= hi) continue;
+        Node* root = nullptr;
+        u64 rank = lo;
+        gen(G, P->start_nt, k, lo, hi, root, [&]() {
+            bool ok = true;
+            for (i64 p : order) {
+                ++R->evals;
+                const i64* pt = &pts[p * nv];
+                i64 h, v;
+                ok = spec_ok[p] && eval_tree(root, pt, h);
+                if (ok) {
+                    if (P->ctx_len == 0) v = h;
+                    else ok = eval_code(P->ctx, P->ctx_len, pt, h, v);
+                }
+                ok = ok && v == spec[p];
+                if (!ok) break;
+            }
+            if (ok) {
+                ++R->match_count[k];
+                if (!R->solved) {
+                    R->solved = 1; R->least_size = k; R->least_rank = rank;
+                    std::string s; tree_text(g, root, s);
+                    snprintf(R->least_text, sizeof(R->least_text), "%s", s.c_str());
+                }
+            }
+            ++rank;
+        });
+    }
+    return 0;
+}
+
+}  // extern "C"
