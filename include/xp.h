@@ -1,0 +1,231 @@
+/* xp.h -- C ABI of libxpiler_repair: bounded-grammar repair of sketch holes on one GPU.
+ *
+ * The operation is the query-creation and synthesis step of the paper's symbolic code
+ * repair (Section 4.4, Algorithm 3: CreateSMTQuery + SynthesisCode): a code sketch has
+ * missing expressions ("holes": a buffer index, a thread binding, a loop bound); one
+ * constraint is stated per concrete index of the snippet's iteration domain; the holes are
+ * filled so that every constraint holds.  The paper hands the constraints to an SMT solver.
+ * This library decides the same question by exhaustive enumeration of a bounded expression
+ * grammar on the GPU:
+ *
+ *   for each hole, each size k = 1..max_size and each derivation tree e of the hole's start
+ *   nonterminal with exactly k nodes (leaf = 1 node, operator = 1 node), in canonical order:
+ *       e matches  <=>  at every domain point p:  e(p) is defined, ctx(e(p), p) is defined,
+ *                       and ctx(e(p), p) == spec(p)
+ *   cand_count[k]  = number of trees of size k          (syntactic, closed by recurrence)
+ *   match_count[k] = number of matching trees of size k (restricted to the rank window, if any)
+ *   least          = the matching tree with the smallest (size, rank)
+ *
+ * Arithmetic: int64 with wrap-around; '/' truncates toward zero; '%' takes the dividend's
+ * sign; INT64_MIN / -1 = INT64_MIN and INT64_MIN % -1 = 0; a zero divisor anywhere in the
+ * candidate, the context or the spec at a point makes the candidate fail there (no
+ * short-circuit, also under a multiplication by zero).  Comparison / logic operators (context
+ * and spec only) give 0 or 1 and evaluate both operands.
+ *
+ * Canonical order inside (nonterminal, size): by production, in the order the grammar lists
+ * them; inside a binary production by left-subtree size ascending, then left-subtree rank,
+ * then right-subtree rank (fastest).  A size-1 tree's rank is the position of its leaf
+ * production among the nonterminal's leaf productions.
+ *
+ * General rules.  All functions return an xp_status (0 = XP_OK) and never throw or abort;
+ * xp_last_error() gives a message for the calling thread's last failure.  Descriptor
+ * structures and everything they point to are borrowed for the duration of the call and
+ * deep-copied (exception: device-resident tables, see xp_sketch_desc).  Handles are immutable
+ * after creation and owned by the caller until the matching destroy/free.  Every pointer is
+ * a HOST pointer unless its comment says "device".  "No solution within the bound" is not an
+ * error.  Every entry point that touches the GPU fails with XP_ERR_CUDA when no CUDA device
+ * is usable: there is no CPU fallback.
+ */
+#ifndef XP_H_
+#define XP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t xp_status;
+enum {
+    XP_OK = 0,
+    XP_ERR_INVALID_ARG = 1,   /* null pointer, index out of range, malformed bytecode */
+    XP_ERR_GRAMMAR = 2,       /* malformed grammar description */
+    XP_ERR_SKETCH = 3,        /* malformed sketch description */
+    XP_ERR_TOO_LARGE = 4,     /* a candidate count reaches 2^63, or a size limit of the library is exceeded */
+    XP_ERR_NOMEM = 5,         /* host or device allocation failed, or the caller's workspace is too small */
+    XP_ERR_CUDA = 6,          /* a CUDA call failed (message in xp_last_error) */
+    XP_ERR_TIMEOUT = 7,
+    XP_ERR_CANCELLED = 8      /* the caller's cancel word became non-zero between launches */
+};
+
+/* Library limits. */
+enum {
+    XP_MAX_SIZE = 15,         /* largest candidate size (nodes) */
+    XP_MAX_VARS = 8,
+    XP_MAX_NONTERMINALS = 8,
+    XP_MAX_CODE = 64          /* instructions in one context or spec expression */
+};
+
+/* Operators.  The first five may appear in grammar productions; all of them in context and
+ * spec expressions. */
+enum {
+    XP_OP_ADD = 0, XP_OP_SUB = 1, XP_OP_MUL = 2, XP_OP_DIV = 3, XP_OP_MOD = 4,
+    XP_OP_LT = 5, XP_OP_LE = 6, XP_OP_EQ = 7, XP_OP_NE = 8, XP_OP_MIN = 9, XP_OP_MAX = 10,
+    XP_OP_AND = 11, XP_OP_OR = 12
+};
+
+/* Variables of the snippet: name (copied) and range lo <= v < hi. */
+typedef struct { const char* name; int64_t lo, hi; } xp_variable;
+
+/* Grammar production  lhs -> variable | constant | left op right. */
+enum { XP_PROD_VAR = 0, XP_PROD_CONST = 1, XP_PROD_BIN = 2 };
+typedef struct {
+    int32_t lhs;        /* nonterminal index, 0 <= lhs < n_nonterminals */
+    int32_t kind;       /* XP_PROD_* */
+    int32_t var;        /* XP_PROD_VAR: variable index */
+    int32_t op;         /* XP_PROD_BIN: XP_OP_ADD .. XP_OP_MOD */
+    int32_t left;       /* XP_PROD_BIN: nonterminal of the left operand */
+    int32_t right;      /* XP_PROD_BIN: nonterminal of the right operand */
+    int64_t value;      /* XP_PROD_CONST: the constant */
+} xp_production;
+
+typedef struct {
+    int32_t n_vars;                     /* <= XP_MAX_VARS */
+    const xp_variable* vars;
+    int32_t n_nonterminals;             /* <= XP_MAX_NONTERMINALS */
+    int32_t n_productions;
+    const xp_production* productions;   /* canonical order = array order */
+} xp_grammar_desc;
+
+/* Postfix instruction of a context, spec or solution expression. */
+enum { XP_I_VAR = 0, XP_I_CONST = 1, XP_I_HOLE = 2, XP_I_OP = 3 };
+typedef struct {
+    int32_t kind;       /* XP_I_* */
+    int32_t arg;        /* XP_I_VAR: variable index; XP_I_OP: XP_OP_* */
+    int64_t value;      /* XP_I_CONST: the constant */
+} xp_instr;
+
+/* One hole of the sketch: the missing expression, the fixed expression around it and what
+ * the source program computes at the same iteration. */
+enum { XP_SPEC_EXPR = 0, XP_SPEC_TABLE = 1 };
+typedef struct {
+    int32_t start_nt;           /* nonterminal the hole is filled from */
+    int32_t max_size;           /* size bound K, 1 <= K <= XP_MAX_SIZE */
+    int32_t ctx_len;            /* 0: identity context (the hole is the whole expression) */
+    const xp_instr* ctx;        /* postfix over variables, constants and XP_I_HOLE (<= XP_MAX_CODE) */
+    int32_t spec_kind;          /* XP_SPEC_EXPR or XP_SPEC_TABLE */
+    int32_t spec_len;           /* XP_SPEC_EXPR: postfix over variables and constants */
+    const xp_instr* spec_expr;
+    const int64_t* spec_table;  /* XP_SPEC_TABLE: n_points values, point order of the domain */
+    int32_t spec_table_on_device; /* non-zero: spec_table is a DEVICE pointer; it is not copied
+                                     and must stay valid and unchanged until xp_sketch_destroy */
+} xp_hole_desc;
+
+/* The sketch: an iteration domain and its holes.  A loop-bound hole is stated through its
+ * guard predicate on the enclosing box (context "loopvar < HOLE", spec = the source's
+ * executes-here predicate, 0 or 1).  Each hole has its own spec and is searched on its own. */
+enum { XP_DOMAIN_BOX = 0, XP_DOMAIN_TABLE = 1 };
+typedef struct {
+    int32_t domain_kind;        /* XP_DOMAIN_BOX: every point of the variable ranges, point id ->
+                                   coordinates by mixed radix with the first variable slowest;
+                                   XP_DOMAIN_TABLE: explicit points */
+    int64_t n_points;           /* XP_DOMAIN_TABLE: number of rows (may be 0) */
+    const int32_t* coords;      /* XP_DOMAIN_TABLE: int32 [n_points][n_vars], row-major */
+    int32_t coords_on_device;   /* non-zero: coords is a DEVICE pointer, kept by reference (as above) */
+    int32_t n_holes;
+    const xp_hole_desc* holes;
+} xp_sketch_desc;
+
+/* Restricts the match search of one (hole, size) to ranks begin <= rank < end.  Counts of
+ * candidates stay syntactic; match counts and the least solution refer to the window. */
+typedef struct { int32_t hole; /* -1: every hole */ int32_t size; uint64_t begin, end; } xp_rank_range;
+
+typedef struct {
+    int32_t size_min, size_max;         /* 0, 0: every size 1..max_size of each hole */
+    int32_t n_rank_ranges;
+    const xp_rank_range* rank_ranges;
+    void* stream;                       /* cudaStream_t to launch on; NULL: the default stream */
+    void* workspace;                    /* DEVICE memory for the call's scratch (256-byte aligned), */
+    size_t workspace_bytes;             /*   at least xp_workspace_bytes(); NULL: the library allocates */
+    uint32_t flags;                     /* XP_FLAG_* */
+    const volatile int32_t* cancel;     /* optional host word polled between launches */
+} xp_repair_opts;
+
+enum {
+    XP_FLAG_NO_FILTER = 1u              /* skip the probe-point filter stage (every candidate is unranked
+                                           and checked on its own); same results, for testing */
+};
+
+typedef struct xp_grammar xp_grammar;
+typedef struct xp_sketch xp_sketch;
+typedef struct xp_result xp_result;
+
+/* Result of one hole.  Pointers live until xp_result_free. */
+typedef struct {
+    int32_t solved;                 /* 1 if some candidate inside the bound (and window) matches */
+    int32_t max_size;
+    const uint64_t* cand_count;     /* [max_size + 1], index = size */
+    const uint64_t* match_count;    /* [max_size + 1] */
+    int32_t least_size;             /* valid when solved */
+    uint64_t least_rank;
+    const xp_instr* least_code;     /* postfix of the least solution */
+    int32_t least_len;
+    const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))" */
+    uint64_t evals_executed;        /* candidate-point evaluations the GPU carried out for this hole */
+    uint64_t filter_survivors;      /* candidates that passed the first probe point */
+    uint64_t probe_survivors;       /* candidates that passed every probe point */
+    double kernel_ms;               /* device time of the whole call's kernels (CUDA events) */
+    double total_ms;                /* host wall time of the whole call */
+    int32_t n_launches;             /* kernels the call launched */
+} xp_result_view;
+
+/* Grammar (Section 4.4: the expressions the synthesis step may put into a hole).  Builds the
+ * per-(nonterminal, size) candidate counts and rank offsets on the host; no GPU is touched.
+ * Errors: XP_ERR_GRAMMAR (bad indices, operator outside + - * / %), XP_ERR_TOO_LARGE. */
+xp_status xp_grammar_create(const xp_grammar_desc* desc, xp_grammar** out);
+void xp_grammar_destroy(xp_grammar* g);
+
+/* Host-side views of the grammar's enumeration (no GPU): counts per size of a nonterminal,
+ * out[0..max_size] (XP_ERR_TOO_LARGE if one reaches 2^63), and the text / postfix of the tree
+ * with a given rank.  text may be NULL; returns XP_ERR_INVALID_ARG if rank >= count or a
+ * buffer is too small (code needs `size` instructions). */
+xp_status xp_grammar_count(const xp_grammar* g, int32_t nt, int32_t max_size, uint64_t* out);
+xp_status xp_grammar_unrank(const xp_grammar* g, int32_t nt, int32_t size, uint64_t rank,
+                            xp_instr* code, int32_t code_cap, char* text, size_t text_cap);
+
+/* Sketch (Algorithm 3: GenerateCodeSketch gives the holes, CreateSMTQuery the per-index
+ * constraints = domain + spec).  Encodes contexts and specs, copies host tables to the GPU
+ * and chooses the probe points.  The grammar must outlive the sketch.
+ * Errors: XP_ERR_SKETCH, XP_ERR_INVALID_ARG, XP_ERR_NOMEM, XP_ERR_CUDA. */
+xp_status xp_sketch_load(const xp_grammar* g, const xp_sketch_desc* desc, xp_sketch** out);
+void xp_sketch_destroy(xp_sketch* s);
+
+/* Device scratch a call over these sketches needs (0 on invalid arguments). */
+size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts);
+
+/* The search (Algorithm 3: SynthesisCode), all sizes of all holes, synchronous on return.
+ * opts may be NULL.  Distinct calls may run concurrently on distinct streams and workspaces.
+ * xp_repair_batch searches n independent sketches in one pass over the GPU and writes n
+ * results (outs[i] belongs to sketches[i]); on error no result is returned.
+ * Errors: XP_ERR_INVALID_ARG, XP_ERR_NOMEM, XP_ERR_CUDA, XP_ERR_CANCELLED. */
+xp_status xp_repair(const xp_sketch* sketch, const xp_repair_opts* opts, xp_result** out);
+xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
+                          xp_result** outs);
+
+/* Algorithm 3 hands the filled snippet back (SynthesisCode -> StitchBack): the per-hole answer. */
+xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_view* out);
+void xp_result_free(xp_result* r);
+
+/* Message of the calling thread's last failed call ("" if none). */
+const char* xp_last_error(void);
+
+/* Measures the integer-ALU peak this library's roofline is quoted against: independent
+ * 32-bit add chains (out[0]) and multiply-add chains (out[1]) in thread-operations per
+ * second, on the current device and stream NULL.  Errors: XP_ERR_CUDA. */
+xp_status xp_int32_peak(double* out_ops_per_s /* [2] */, double* out_ms /* [2], may be NULL */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* XP_H_ */

@@ -1,0 +1,313 @@
+"""ctypes binding of libxpiler_repair.so: argument marshalling only.
+
+Every step of the repair search runs inside the CUDA library; nothing here
+evaluates, counts or ranks candidates, and there is no CPU fallback: a missing
+or unloadable library raises.  The functions carry the names of the C ABI
+(``include/xp.h``); ``Grammar`` / ``LoadedSketch`` are thin handle owners.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+XP_MAX_SIZE = 15
+XP_FLAG_NO_FILTER = 1
+_STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_SKETCH", 4: "XP_ERR_TOO_LARGE",
+           5: "XP_ERR_NOMEM", 6: "XP_ERR_CUDA", 7: "XP_ERR_TIMEOUT", 8: "XP_ERR_CANCELLED"}
+
+EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_grammar_unrank",
+           "xp_sketch_load", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
+           "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak"]
+
+
+class XpError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{_STATUS.get(status, status)}: {message}")
+        self.status = status
+
+
+class xp_variable(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("lo", C.c_int64), ("hi", C.c_int64)]
+
+
+class xp_production(C.Structure):
+    _fields_ = [("lhs", C.c_int32), ("kind", C.c_int32), ("var", C.c_int32), ("op", C.c_int32),
+                ("left", C.c_int32), ("right", C.c_int32), ("value", C.c_int64)]
+
+
+class xp_grammar_desc(C.Structure):
+    _fields_ = [("n_vars", C.c_int32), ("vars", C.POINTER(xp_variable)), ("n_nonterminals", C.c_int32),
+                ("n_productions", C.c_int32), ("productions", C.POINTER(xp_production))]
+
+
+class xp_instr(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("arg", C.c_int32), ("value", C.c_int64)]
+
+
+class xp_hole_desc(C.Structure):
+    _fields_ = [("start_nt", C.c_int32), ("max_size", C.c_int32), ("ctx_len", C.c_int32), ("ctx", C.POINTER(xp_instr)),
+                ("spec_kind", C.c_int32), ("spec_len", C.c_int32), ("spec_expr", C.POINTER(xp_instr)),
+                ("spec_table", C.c_void_p), ("spec_table_on_device", C.c_int32)]
+
+
+class xp_sketch_desc(C.Structure):
+    _fields_ = [("domain_kind", C.c_int32), ("n_points", C.c_int64), ("coords", C.c_void_p),
+                ("coords_on_device", C.c_int32), ("n_holes", C.c_int32), ("holes", C.POINTER(xp_hole_desc))]
+
+
+class xp_rank_range(C.Structure):
+    _fields_ = [("hole", C.c_int32), ("size", C.c_int32), ("begin", C.c_uint64), ("end", C.c_uint64)]
+
+
+class xp_repair_opts(C.Structure):
+    _fields_ = [("size_min", C.c_int32), ("size_max", C.c_int32), ("n_rank_ranges", C.c_int32),
+                ("rank_ranges", C.POINTER(xp_rank_range)), ("stream", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32), ("cancel", C.POINTER(C.c_int32))]
+
+
+class xp_result_view(C.Structure):
+    _fields_ = [("solved", C.c_int32), ("max_size", C.c_int32), ("cand_count", C.POINTER(C.c_uint64)),
+                ("match_count", C.POINTER(C.c_uint64)), ("least_size", C.c_int32), ("least_rank", C.c_uint64),
+                ("least_code", C.POINTER(xp_instr)), ("least_len", C.c_int32), ("least_text", C.c_char_p),
+                ("evals_executed", C.c_uint64), ("filter_survivors", C.c_uint64), ("probe_survivors", C.c_uint64),
+                ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None):
+    """Loads (building first if the sources are newer) the shared library; raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = C.CDLL(path or _build.build())
+    vp = C.c_void_p
+    lib.xp_grammar_create.argtypes = [C.POINTER(xp_grammar_desc), C.POINTER(vp)]
+    lib.xp_grammar_destroy.argtypes = [vp]
+    lib.xp_grammar_destroy.restype = None
+    lib.xp_grammar_count.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(C.c_uint64)]
+    lib.xp_grammar_unrank.argtypes = [vp, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(xp_instr), C.c_int32,
+                                      C.c_char_p, C.c_size_t]
+    lib.xp_sketch_load.argtypes = [vp, C.POINTER(xp_sketch_desc), C.POINTER(vp)]
+    lib.xp_sketch_destroy.argtypes = [vp]
+    lib.xp_sketch_destroy.restype = None
+    lib.xp_workspace_bytes.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_repair_opts)]
+    lib.xp_workspace_bytes.restype = C.c_size_t
+    lib.xp_repair.argtypes = [vp, C.POINTER(xp_repair_opts), C.POINTER(vp)]
+    lib.xp_repair_batch.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_repair_opts), C.POINTER(vp)]
+    lib.xp_result_get.argtypes = [vp, C.c_int32, C.POINTER(xp_result_view)]
+    lib.xp_result_free.argtypes = [vp]
+    lib.xp_result_free.restype = None
+    lib.xp_last_error.restype = C.c_char_p
+    lib.xp_int32_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    for name in EXPORTS:
+        getattr(lib, name)
+    _lib = lib
+    return lib
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise XpError(status, load().xp_last_error().decode())
+
+
+def _code(instrs) -> "C.Array":
+    arr = (xp_instr * max(1, len(instrs)))()
+    for i, (k, a, v) in enumerate(instrs):
+        arr[i].kind, arr[i].arg, arr[i].value = k, a, v
+    return arr
+
+
+# ------------------------------------------------------------------------------------------
+# the C ABI, one Python function per entry point
+# ------------------------------------------------------------------------------------------
+
+class Grammar:
+    """Owns an ``xp_grammar*``."""
+
+    def __init__(self, handle: int, model):
+        self.handle, self.model = handle, model
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.xp_grammar_destroy(self.handle)
+            self.handle = None
+
+
+def xp_grammar_create(g) -> Grammar:
+    """``g``: an ``xp_instances.Grammar`` (variables with ranges, productions in canonical order)."""
+    lib = load()
+    nv = len(g.variables)
+    names = [v.name.encode() for v in g.variables]
+    vs = (xp_variable * max(1, nv))()
+    for i, v in enumerate(g.variables):
+        vs[i].name, vs[i].lo, vs[i].hi = names[i], v.lo, v.hi
+    ps = (xp_production * len(g.productions))()
+    for i, p in enumerate(g.productions):
+        q = ps[i]
+        q.lhs, q.kind, q.var, q.op, q.left, q.right, q.value = p.lhs, p.kind, p.var, p.op, p.left, p.right, p.value
+    desc = xp_grammar_desc(nv, vs, g.n_nonterminals, len(g.productions), ps)
+    out = C.c_void_p()
+    _check(lib.xp_grammar_create(C.byref(desc), C.byref(out)))
+    return Grammar(out.value, g)
+
+
+def xp_grammar_count(gr: Grammar, nt: int, max_size: int) -> List[int]:
+    out = (C.c_uint64 * (max_size + 1))()
+    _check(load().xp_grammar_count(gr.handle, nt, max_size, out))
+    return [int(x) for x in out]
+
+
+def xp_grammar_unrank(gr: Grammar, nt: int, size: int, rank: int) -> Tuple[str, List[Tuple[int, int, int]]]:
+    code = (xp_instr * XP_MAX_SIZE)()
+    text = C.create_string_buffer(1024)
+    _check(load().xp_grammar_unrank(gr.handle, nt, size, rank, code, XP_MAX_SIZE, text, 1024))
+    return text.value.decode(), [(code[i].kind, code[i].arg, code[i].value) for i in range(size)]
+
+
+class LoadedSketch:
+    """Owns an ``xp_sketch*`` and keeps the grammar and any device tensors it refers to alive."""
+
+    def __init__(self, handle: int, grammar: Grammar, n_holes: int, keep):
+        self.handle, self.grammar, self.n_holes, self._keep = handle, grammar, n_holes, keep
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.xp_sketch_destroy(self.handle)
+            self.handle = None
+
+
+def _ptr_of(x) -> Tuple[int, int, object]:
+    """(address, on_device, keep-alive) of a numpy array (host) or a torch CUDA tensor (device)."""
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data, 0, x
+    return int(x.data_ptr()), int(x.is_cuda), x      # torch tensor: device memory only, no torch compute
+
+
+def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int, object]] = None) -> LoadedSketch:
+    """``sk``: an ``xp_instances.Sketch``.  ``coords`` / ``spec_tables[hole]`` may override the
+    sketch's host tables with contiguous torch CUDA tensors (int32 [n, n_vars] / int64 [n]),
+    which the library then uses in place."""
+    lib = load()
+    keep = []
+    nh = len(sk.holes)
+    holes = (xp_hole_desc * nh)()
+    for i, h in enumerate(sk.holes):
+        d = holes[i]
+        d.start_nt, d.max_size = h.start_nt, h.max_size
+        ctx = _code(h.ctx); keep.append(ctx)
+        d.ctx_len, d.ctx = len(h.ctx), ctx
+        table = (spec_tables or {}).get(i, h.spec_table)
+        if table is not None:
+            if isinstance(table, np.ndarray):
+                table = np.ascontiguousarray(table, dtype=np.int64)
+            d.spec_kind = 1
+            d.spec_table, d.spec_table_on_device, k = _ptr_of(table)
+            keep.append(k)
+        else:
+            se = _code(h.spec_expr); keep.append(se)
+            d.spec_kind, d.spec_len, d.spec_expr = 0, len(h.spec_expr), se
+    desc = xp_sketch_desc()
+    co = coords if coords is not None else sk.coords
+    if co is not None:
+        if isinstance(co, np.ndarray):
+            co = np.ascontiguousarray(co, dtype=np.int32)
+        desc.domain_kind = 1
+        desc.n_points = int(co.shape[0])
+        desc.coords, desc.coords_on_device, k = _ptr_of(co)
+        keep.append(k)
+    desc.n_holes, desc.holes = nh, holes
+    out = C.c_void_p()
+    _check(lib.xp_sketch_load(gr.handle, C.byref(desc), C.byref(out)))
+    return LoadedSketch(out.value, gr, nh, [k for k in keep if not isinstance(k, C.Array)])
+
+
+@dataclass
+class HoleResult:
+    solved: bool
+    cand_count: List[int]
+    match_count: List[int]
+    least_size: int
+    least_rank: int
+    least_text: str
+    least_code: List[Tuple[int, int, int]]
+    evals_executed: int
+    filter_survivors: int
+    probe_survivors: int
+    kernel_ms: float
+    total_ms: float
+    n_launches: int
+
+
+def xp_result_get(result_handle: int, hole: int) -> HoleResult:
+    v = xp_result_view()
+    _check(load().xp_result_get(result_handle, hole, C.byref(v)))
+    K = v.max_size
+    return HoleResult(bool(v.solved), [int(v.cand_count[k]) for k in range(K + 1)],
+                      [int(v.match_count[k]) for k in range(K + 1)], int(v.least_size), int(v.least_rank),
+                      v.least_text.decode() if v.solved else "",
+                      [(v.least_code[i].kind, v.least_code[i].arg, v.least_code[i].value) for i in range(v.least_len)],
+                      int(v.evals_executed), int(v.filter_survivors), int(v.probe_survivors),
+                      float(v.kernel_ms), float(v.total_ms), int(v.n_launches))
+
+
+def _opts(size_min=0, size_max=0, rank_ranges=None, stream=None, workspace=None, flags=0):
+    o = xp_repair_opts()
+    o.size_min, o.size_max, o.flags = size_min, size_max, flags
+    keep = []
+    if rank_ranges:
+        rr = (xp_rank_range * len(rank_ranges))()
+        for i, (hole, size, b, e) in enumerate(rank_ranges):
+            rr[i].hole, rr[i].size, rr[i].begin, rr[i].end = hole, size, b, e
+        o.n_rank_ranges, o.rank_ranges = len(rank_ranges), rr
+        keep.append(rr)
+    if stream is not None:
+        o.stream = int(stream)
+    if workspace is not None:          # a torch CUDA tensor (uint8) used as scratch
+        o.workspace, o.workspace_bytes = int(workspace.data_ptr()), int(workspace.numel() * workspace.element_size())
+        keep.append(workspace)
+    return o, keep
+
+
+def xp_workspace_bytes(sketches: Sequence[LoadedSketch], **kw) -> int:
+    o, _keep = _opts(**kw)
+    arr = (C.c_void_p * len(sketches))(*[s.handle for s in sketches])
+    return int(load().xp_workspace_bytes(arr, len(sketches), C.byref(o)))
+
+
+def xp_repair(sketch: LoadedSketch, **kw) -> List[HoleResult]:
+    """Keyword options: size_min, size_max, rank_ranges=[(hole, size, begin, end)], stream (raw
+    cudaStream_t), workspace (torch CUDA uint8 tensor), flags.  Returns one result per hole."""
+    o, _keep = _opts(**kw)
+    out = C.c_void_p()
+    _check(load().xp_repair(sketch.handle, C.byref(o), C.byref(out)))
+    try:
+        return [xp_result_get(out.value, h) for h in range(sketch.n_holes)]
+    finally:
+        load().xp_result_free(out.value)
+
+
+def xp_repair_batch(sketches: Sequence[LoadedSketch], **kw) -> List[List[HoleResult]]:
+    o, _keep = _opts(**kw)
+    n = len(sketches)
+    arr = (C.c_void_p * n)(*[s.handle for s in sketches])
+    outs = (C.c_void_p * n)()
+    _check(load().xp_repair_batch(arr, n, C.byref(o), outs))
+    try:
+        return [[xp_result_get(outs[i], h) for h in range(sketches[i].n_holes)] for i in range(n)]
+    finally:
+        for i in range(n):
+            load().xp_result_free(outs[i])
+
+
+def xp_int32_peak() -> Tuple[float, float]:
+    out = (C.c_double * 2)()
+    _check(load().xp_int32_peak(out, None))
+    return float(out[0]), float(out[1])

@@ -1,0 +1,658 @@
+// Host side of libxpiler_repair: grammar tables, sketch encoding, launch planning, result
+// decoding and the C ABI declared in include/xp.h.
+#include <cuda_runtime.h>
+
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "xp_dev.h"
+#include "xp_launch.h"
+
+using namespace xp;
+
+// ------------------------------------------------------------------------------------------
+// errors
+// ------------------------------------------------------------------------------------------
+
+static thread_local std::string g_last_error;
+
+static xp_status fail(xp_status st, const std::string& msg) {
+    g_last_error = msg;
+    return st;
+}
+
+#define XP_CUDA(call)                                                                          \
+    do {                                                                                       \
+        cudaError_t e_ = (call);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA,          \
+                        std::string(#call) + ": " + cudaGetErrorString(e_));                   \
+    } while (0)
+
+static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
+
+// ------------------------------------------------------------------------------------------
+// grammar
+// ------------------------------------------------------------------------------------------
+
+struct xp_grammar {
+    int n_vars = 0, n_nt = 0;
+    std::vector<std::string> names;
+    std::vector<i64> lo, hi;
+    std::vector<xp_production> prods;
+    std::vector<LeafDev> leaves;
+    std::vector<BinDev> bins;
+    int leaf_begin[kMaxNt + 1] = {0};
+    int bin_begin[kMaxNt + 1] = {0};
+    u64 cnt[kMaxNt][kMaxSize + 1] = {{0}};
+    int ok_size = kMaxSize;          // counts are exact (< 2^63) up to this size
+    // device copy, made on first use
+    std::mutex mu;
+    GrammarDev* d_g = nullptr;
+    LeafDev* d_leaves = nullptr;
+    BinDev* d_bins = nullptr;
+};
+
+// cnt[nt][s] by the recurrence over productions and left sizes; off[s] of a binary production
+// is the number of size-s trees of its nonterminal that come before it.  Sizes from the first
+// one at which a count reaches 2^63 are marked unusable (ok_size).
+static void build_counts(xp_grammar* g) {
+    for (int s = 1; s <= kMaxSize; ++s) {
+        bool overflow = g->ok_size < s;
+        for (int nt = 0; nt < g->n_nt && !overflow; ++nt) {
+            unsigned __int128 total = 0;
+            if (s == 1) total = (unsigned)(g->leaf_begin[nt + 1] - g->leaf_begin[nt]);
+            for (int b = g->bin_begin[nt]; b < g->bin_begin[nt + 1] && !overflow; ++b) {
+                BinDev& bd = g->bins[b];
+                bd.off[s] = (u64)total;
+                for (int a = 1; a <= s - 2 && !overflow; ++a) {
+                    total += (unsigned __int128)g->cnt[bd.lnt][a] * g->cnt[bd.rnt][s - 1 - a];
+                    overflow = (total >> 63) != 0;
+                }
+            }
+            g->cnt[nt][s] = (u64)total;
+        }
+        if (overflow) {
+            if (g->ok_size >= s) g->ok_size = s - 1;
+            for (int nt = 0; nt < g->n_nt; ++nt) g->cnt[nt][s] = 0;
+        }
+    }
+}
+
+extern "C" xp_status xp_grammar_create(const xp_grammar_desc* d, xp_grammar** out) {
+    if (!d || !out) return fail(XP_ERR_INVALID_ARG, "xp_grammar_create: null argument");
+    *out = nullptr;
+    if (d->n_vars < 0 || d->n_vars > kMaxVars) return fail(XP_ERR_GRAMMAR, "n_vars out of range");
+    if (d->n_nonterminals < 1 || d->n_nonterminals > kMaxNt) return fail(XP_ERR_GRAMMAR, "n_nonterminals out of range");
+    if (d->n_productions < 1 || !d->productions) return fail(XP_ERR_GRAMMAR, "no productions");
+    if (d->n_vars > 0 && !d->vars) return fail(XP_ERR_GRAMMAR, "vars is null");
+    xp_grammar* g = new (std::nothrow) xp_grammar;
+    if (!g) return fail(XP_ERR_NOMEM, "out of host memory");
+    g->n_vars = d->n_vars;
+    g->n_nt = d->n_nonterminals;
+    for (int i = 0; i < d->n_vars; ++i) {
+        if (d->vars[i].hi < d->vars[i].lo) { delete g; return fail(XP_ERR_GRAMMAR, "variable range with hi < lo"); }
+        g->names.push_back(d->vars[i].name ? d->vars[i].name : ("v" + std::to_string(i)));
+        g->lo.push_back(d->vars[i].lo);
+        g->hi.push_back(d->vars[i].hi);
+    }
+    for (int i = 0; i < d->n_productions; ++i) {
+        const xp_production& p = d->productions[i];
+        bool ok = p.lhs >= 0 && p.lhs < g->n_nt;
+        if (p.kind == XP_PROD_VAR) ok = ok && p.var >= 0 && p.var < g->n_vars;
+        else if (p.kind == XP_PROD_BIN) ok = ok && p.op >= XP_OP_ADD && p.op <= XP_OP_MOD && p.left >= 0 && p.left < g->n_nt && p.right >= 0 && p.right < g->n_nt;
+        else if (p.kind != XP_PROD_CONST) ok = false;
+        if (!ok) { delete g; return fail(XP_ERR_GRAMMAR, "production " + std::to_string(i) + " is malformed"); }
+        g->prods.push_back(p);
+    }
+    for (int nt = 0; nt < g->n_nt; ++nt) {          // leaves and binaries grouped per nonterminal, order kept
+        g->leaf_begin[nt] = (int)g->leaves.size();
+        g->bin_begin[nt] = (int)g->bins.size();
+        for (const xp_production& p : g->prods) {
+            if (p.lhs != nt) continue;
+            if (p.kind == XP_PROD_BIN) {
+                BinDev b;
+                memset(&b, 0, sizeof(b));
+                b.op = p.op; b.lnt = p.left; b.rnt = p.right;
+                g->bins.push_back(b);
+            } else {
+                LeafDev l;
+                l.var = p.kind == XP_PROD_VAR ? p.var : -1;
+                l.pad = 0;
+                l.value = p.kind == XP_PROD_CONST ? p.value : 0;
+                g->leaves.push_back(l);
+            }
+        }
+    }
+    g->leaf_begin[g->n_nt] = (int)g->leaves.size();
+    g->bin_begin[g->n_nt] = (int)g->bins.size();
+    build_counts(g);
+    *out = g;
+    return XP_OK;
+}
+
+extern "C" void xp_grammar_destroy(xp_grammar* g) {
+    if (!g) return;
+    if (g->d_g) cudaFree(g->d_g);
+    if (g->d_leaves) cudaFree(g->d_leaves);
+    if (g->d_bins) cudaFree(g->d_bins);
+    delete g;
+}
+
+extern "C" xp_status xp_grammar_count(const xp_grammar* g, int32_t nt, int32_t max_size, uint64_t* out) {
+    if (!g || !out || nt < 0 || nt >= g->n_nt || max_size < 0 || max_size > kMaxSize)
+        return fail(XP_ERR_INVALID_ARG, "xp_grammar_count: bad argument");
+    if (max_size > g->ok_size) return fail(XP_ERR_TOO_LARGE, "a candidate count reaches 2^63");
+    out[0] = 0;
+    for (int s = 1; s <= max_size; ++s) out[s] = g->cnt[nt][s];
+    return XP_OK;
+}
+
+// rank -> tree, appended to `code` in postfix and to `text` in infix.
+static bool host_unrank(const xp_grammar* g, int nt, int size, u64 rank, std::vector<xp_instr>* code, std::string* text) {
+    if (size < 1 || size > g->ok_size || rank >= g->cnt[nt][size]) return false;
+    if (size == 1) {
+        const LeafDev& l = g->leaves[g->leaf_begin[nt] + (int)rank];
+        xp_instr in;
+        in.kind = l.var >= 0 ? XP_I_VAR : XP_I_CONST;
+        in.arg = l.var >= 0 ? l.var : 0;
+        in.value = l.value;
+        code->push_back(in);
+        *text += l.var >= 0 ? g->names[l.var] : std::to_string((long long)l.value);
+        return true;
+    }
+    int p = g->bin_begin[nt];
+    const int pe = g->bin_begin[nt + 1];
+    while (p + 1 < pe && g->bins[p + 1].off[size] <= rank) ++p;
+    const BinDev& b = g->bins[p];
+    u64 rem = rank - b.off[size];
+    for (int a = 1; a <= size - 2; ++a) {
+        const u64 cr = g->cnt[b.rnt][size - 1 - a];
+        const u64 block = g->cnt[b.lnt][a] * cr;
+        if (rem >= block) { rem -= block; continue; }
+        *text += "(";
+        if (!host_unrank(g, b.lnt, a, rem / cr, code, text)) return false;
+        *text += kOpText[b.op];
+        if (!host_unrank(g, b.rnt, size - 1 - a, rem % cr, code, text)) return false;
+        *text += ")";
+        xp_instr in;
+        in.kind = XP_I_OP; in.arg = b.op; in.value = 0;
+        code->push_back(in);
+        return true;
+    }
+    return false;
+}
+
+extern "C" xp_status xp_grammar_unrank(const xp_grammar* g, int32_t nt, int32_t size, uint64_t rank,
+                                       xp_instr* code, int32_t code_cap, char* text, size_t text_cap) {
+    if (!g || nt < 0 || nt >= g->n_nt || size < 1 || size > kMaxSize)
+        return fail(XP_ERR_INVALID_ARG, "xp_grammar_unrank: bad argument");
+    std::vector<xp_instr> c;
+    std::string t;
+    if (!host_unrank(g, nt, size, rank, &c, &t)) return fail(XP_ERR_INVALID_ARG, "xp_grammar_unrank: rank out of range");
+    if (code) {
+        if (code_cap < (int)c.size()) return fail(XP_ERR_INVALID_ARG, "xp_grammar_unrank: code buffer too small");
+        memcpy(code, c.data(), c.size() * sizeof(xp_instr));
+    }
+    if (text) {
+        if (text_cap < t.size() + 1) return fail(XP_ERR_INVALID_ARG, "xp_grammar_unrank: text buffer too small");
+        memcpy(text, t.c_str(), t.size() + 1);
+    }
+    return XP_OK;
+}
+
+static xp_status grammar_to_device(xp_grammar* g) {
+    std::lock_guard<std::mutex> lock(g->mu);
+    if (g->d_g) return XP_OK;
+    GrammarDev h;
+    memset(&h, 0, sizeof(h));
+    h.n_vars = g->n_vars; h.n_nt = g->n_nt;
+    h.n_leaves = (int)g->leaves.size(); h.n_bins = (int)g->bins.size();
+    memcpy(h.leaf_begin, g->leaf_begin, sizeof(h.leaf_begin));
+    memcpy(h.bin_begin, g->bin_begin, sizeof(h.bin_begin));
+    memcpy(h.cnt, g->cnt, sizeof(h.cnt));
+    XP_CUDA(cudaMalloc(&g->d_leaves, sizeof(LeafDev) * (g->leaves.size() + 1)));
+    XP_CUDA(cudaMalloc(&g->d_bins, sizeof(BinDev) * (g->bins.size() + 1)));
+    XP_CUDA(cudaMemcpy(g->d_leaves, g->leaves.data(), sizeof(LeafDev) * g->leaves.size(), cudaMemcpyHostToDevice));
+    XP_CUDA(cudaMemcpy(g->d_bins, g->bins.data(), sizeof(BinDev) * g->bins.size(), cudaMemcpyHostToDevice));
+    h.leaves = g->d_leaves;
+    h.bins = g->d_bins;
+    GrammarDev* d = nullptr;
+    XP_CUDA(cudaMalloc(&d, sizeof(GrammarDev)));
+    XP_CUDA(cudaMemcpy(d, &h, sizeof(h), cudaMemcpyHostToDevice));
+    g->d_g = d;
+    return XP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// sketch
+// ------------------------------------------------------------------------------------------
+
+struct HoleHost {
+    int start_nt = 0, max_size = 0;
+};
+
+struct xp_sketch {
+    xp_grammar* g = nullptr;
+    int n_holes = 0;
+    i64 n_points = 0;
+    std::vector<HoleHost> holes;
+    SketchDev* d_s = nullptr;
+    HoleDev* d_holes = nullptr;
+    std::vector<void*> owned;        // device copies of host tables
+};
+
+// Checks a postfix expression; returns false when malformed or too deep.
+static bool check_code(const xp_instr* code, int n, int n_vars, bool hole_allowed) {
+    if (n < 0 || n > kMaxCode || (n > 0 && !code)) return false;
+    int sp = 0;
+    for (int i = 0; i < n; ++i) {
+        const xp_instr& c = code[i];
+        if (c.kind == XP_I_OP) {
+            if (c.arg < XP_OP_ADD || c.arg > XP_OP_OR || sp < 2) return false;
+            --sp;
+        } else {
+            if (c.kind == XP_I_VAR) { if (c.arg < 0 || c.arg >= n_vars) return false; }
+            else if (c.kind == XP_I_HOLE) { if (!hole_allowed) return false; }
+            else if (c.kind != XP_I_CONST) return false;
+            if (++sp > kMaxStack) return false;
+        }
+    }
+    return n == 0 || sp == 1;
+}
+
+static u64 mix64(u64 x) {            // SplitMix64 finaliser: spreads sample ids over the domain
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+
+extern "C" void xp_sketch_destroy(xp_sketch* s) {
+    if (!s) return;
+    for (void* p : s->owned) cudaFree(p);
+    if (s->d_holes) cudaFree(s->d_holes);
+    if (s->d_s) cudaFree(s->d_s);
+    delete s;
+}
+
+extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* d, xp_sketch** out) {
+    if (!gc || !d || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load: null argument");
+    *out = nullptr;
+    xp_grammar* g = const_cast<xp_grammar*>(gc);
+    if (d->n_holes < 1 || !d->holes) return fail(XP_ERR_SKETCH, "a sketch needs at least one hole");
+    if (d->domain_kind != XP_DOMAIN_BOX && d->domain_kind != XP_DOMAIN_TABLE) return fail(XP_ERR_SKETCH, "bad domain_kind");
+    const int nv = g->n_vars;
+    i64 n_points = 0;
+    if (d->domain_kind == XP_DOMAIN_BOX) {
+        unsigned __int128 n = 1;
+        for (int v = 0; v < nv; ++v) {
+            n *= (unsigned __int128)(u64)(g->hi[v] - g->lo[v]);
+            if (n >> 62) return fail(XP_ERR_TOO_LARGE, "box domain has 2^62 points or more");
+        }
+        n_points = (i64)n;
+    } else {
+        if (d->n_points < 0 || (d->n_points > 0 && !d->coords)) return fail(XP_ERR_SKETCH, "table domain without coords");
+        n_points = d->n_points;
+    }
+    for (int h = 0; h < d->n_holes; ++h) {
+        const xp_hole_desc& hd = d->holes[h];
+        if (hd.start_nt < 0 || hd.start_nt >= g->n_nt) return fail(XP_ERR_SKETCH, "hole start_nt out of range");
+        if (hd.max_size < 1 || hd.max_size > kMaxSize) return fail(XP_ERR_SKETCH, "hole max_size out of range");
+        if (hd.max_size > g->ok_size) return fail(XP_ERR_TOO_LARGE, "a candidate count reaches 2^63 within the size bound");
+        if (!check_code(hd.ctx, hd.ctx_len, nv, true)) return fail(XP_ERR_SKETCH, "malformed context expression");
+        if (hd.spec_kind == XP_SPEC_EXPR) {
+            if (hd.spec_len < 1 || !check_code(hd.spec_expr, hd.spec_len, nv, false)) return fail(XP_ERR_SKETCH, "malformed spec expression");
+        } else if (hd.spec_kind == XP_SPEC_TABLE) {
+            if (n_points > 0 && !hd.spec_table) return fail(XP_ERR_SKETCH, "spec table is null");
+        } else return fail(XP_ERR_SKETCH, "bad spec_kind");
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(XP_ERR_CUDA, "no CUDA device is usable");
+    xp_status st = grammar_to_device(g);
+    if (st != XP_OK) return st;
+
+    xp_sketch* s = new (std::nothrow) xp_sketch;
+    if (!s) return fail(XP_ERR_NOMEM, "out of host memory");
+    s->g = g; s->n_holes = d->n_holes; s->n_points = n_points;
+#define XP_CUDA_S(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { xp_sketch_destroy(s); \
+        return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
+
+    SketchDev hs;
+    memset(&hs, 0, sizeof(hs));
+    hs.g = g->d_g; hs.n_vars = nv; hs.n_holes = d->n_holes; hs.domain_kind = d->domain_kind; hs.n_points = n_points;
+    for (int v = 0; v < nv; ++v) { hs.lo[v] = g->lo[v]; hs.ext[v] = g->hi[v] - g->lo[v]; }
+    if (d->domain_kind == XP_DOMAIN_TABLE && n_points > 0) {
+        if (d->coords_on_device) hs.coords = d->coords;
+        else {
+            void* p = nullptr;
+            const size_t bytes = sizeof(i32) * (size_t)n_points * (size_t)(nv ? nv : 1);
+            XP_CUDA_S(cudaMalloc(&p, bytes));
+            s->owned.push_back(p);
+            XP_CUDA_S(cudaMemcpy(p, d->coords, bytes, cudaMemcpyHostToDevice));
+            hs.coords = (const i32*)p;
+        }
+    }
+    // Sample points the probes are chosen from: box corners first (they expose bound and
+    // padding mistakes), then ids spread over the domain by a fixed hash.
+    int ns = 0;
+    if (n_points > 0) {
+        if (d->domain_kind == XP_DOMAIN_BOX) {
+            const int ncorner = 1 << (nv < 5 ? nv : 5);
+            for (int m = 0; m < ncorner && ns < kProbeSamples / 2; ++m) {
+                i64 id = 0;
+                for (int v = 0; v < nv; ++v) {
+                    const i64 ext = hs.ext[v];
+                    const i64 c = (v < 5 && ((m >> v) & 1)) ? ext - 1 : 0;
+                    id = id * ext + c;
+                }
+                bool dup = false;
+                for (int k = 0; k < ns; ++k) dup = dup || hs.sample_id[k] == id;
+                if (!dup) hs.sample_id[ns++] = id;
+            }
+        } else {
+            for (i64 id = 0; id < n_points && ns < 16; ++id) hs.sample_id[ns++] = id;
+        }
+        for (u64 k = 0; ns < kProbeSamples && k < 4 * kProbeSamples; ++k) {
+            const i64 id = (i64)(mix64(k) % (u64)n_points);
+            bool dup = false;
+            for (int j = 0; j < ns; ++j) dup = dup || hs.sample_id[j] == id;
+            if (!dup) hs.sample_id[ns++] = id;
+        }
+    }
+    hs.n_samples = ns;
+
+    std::vector<HoleDev> hh(d->n_holes);
+    for (int h = 0; h < d->n_holes; ++h) {
+        const xp_hole_desc& hd = d->holes[h];
+        HoleDev& o = hh[h];
+        memset(&o, 0, sizeof(o));
+        o.start_nt = hd.start_nt; o.max_size = hd.max_size; o.ctx_len = hd.ctx_len;
+        if (hd.ctx_len) memcpy(o.ctx, hd.ctx, sizeof(xp_instr) * hd.ctx_len);
+        if (hd.spec_kind == XP_SPEC_EXPR) {
+            o.spec_len = hd.spec_len;
+            memcpy(o.spec, hd.spec_expr, sizeof(xp_instr) * hd.spec_len);
+        } else if (n_points > 0) {
+            if (hd.spec_table_on_device) o.spec_table = (const i64*)hd.spec_table;
+            else {
+                void* p = nullptr;
+                XP_CUDA_S(cudaMalloc(&p, sizeof(i64) * (size_t)n_points));
+                s->owned.push_back(p);
+                XP_CUDA_S(cudaMemcpy(p, hd.spec_table, sizeof(i64) * (size_t)n_points, cudaMemcpyHostToDevice));
+                o.spec_table = (const i64*)p;
+            }
+        }
+        o.chain_len = -1;
+        HoleHost ho;
+        ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
+        s->holes.push_back(ho);
+    }
+    XP_CUDA_S(cudaMalloc(&s->d_holes, sizeof(HoleDev) * d->n_holes));
+    XP_CUDA_S(cudaMemcpy(s->d_holes, hh.data(), sizeof(HoleDev) * d->n_holes, cudaMemcpyHostToDevice));
+    hs.holes = s->d_holes;
+    XP_CUDA_S(cudaMalloc(&s->d_s, sizeof(SketchDev)));
+    XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
+    XP_CUDA_S(launch_prepare(s->d_s, nullptr));
+    XP_CUDA_S(cudaStreamSynchronize(nullptr));
+#undef XP_CUDA_S
+    *out = s;
+    return XP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// repair
+// ------------------------------------------------------------------------------------------
+
+struct HoleResult {
+    int max_size = 0, solved = 0, least_size = 0;
+    u64 cand_count[kMaxSize + 1] = {0};
+    u64 match_count[kMaxSize + 1] = {0};
+    u64 least_rank = 0;
+    std::vector<xp_instr> code;
+    std::string text;
+    u64 evals = 0, filter_survivors = 0, probe_survivors = 0;
+};
+
+struct xp_result {
+    std::vector<HoleResult> holes;
+    double kernel_ms = 0, total_ms = 0;
+    int n_launches = 0;
+};
+
+struct Plan {
+    std::vector<SegDev> segs;
+    std::vector<AccDev> acc;
+    u64 n_tickets = 0;
+};
+
+static const xp_repair_opts kDefaultOpts = {0, 0, 0, nullptr, nullptr, nullptr, 0, 0u, nullptr};
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+constexpr u64 kLinearChunkHost = 256 * 4;     // ranks per linear ticket (matches the kernel)
+
+static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
+    for (size_t i = 0; i < n; ++i) {
+        const xp_sketch* s = sk[i];
+        if (!s) return fail(XP_ERR_INVALID_ARG, "null sketch in batch");
+        for (int h = 0; h < s->n_holes; ++h) {
+            const HoleHost& ho = s->holes[h];
+            AccDev a;
+            memset(&a, 0, sizeof(a));
+            for (int k = 0; k <= kMaxSize; ++k) a.min_rank[k] = ~0ull;
+            const int acc = (int)plan->acc.size();
+            plan->acc.push_back(a);
+            int kmin = 1, kmax = ho.max_size;
+            if (o->size_min > 0) kmin = o->size_min;
+            if (o->size_max > 0 && o->size_max < kmax) kmax = o->size_max;
+            for (int k = kmin; k <= kmax; ++k) {
+                u64 lo = 0, hi = s->g->cnt[ho.start_nt][k];
+                for (int r = 0; r < o->n_rank_ranges; ++r) {
+                    const xp_rank_range& rr = o->rank_ranges[r];
+                    if ((rr.hole == -1 || rr.hole == h) && rr.size == k) {
+                        if (rr.begin > lo) lo = rr.begin;
+                        if (rr.end < hi) hi = rr.end;
+                    }
+                }
+                if (lo >= hi) continue;
+                SegDev sg;
+                memset(&sg, 0, sizeof(sg));
+                sg.first_ticket = plan->n_tickets;
+                sg.rank_begin = lo; sg.rank_end = hi;
+                sg.sketch = (int)i; sg.hole = h; sg.size = k; sg.kind = kSegLinear; sg.acc = acc;
+                plan->segs.push_back(sg);
+                plan->n_tickets += (hi - lo + kLinearChunkHost - 1) / kLinearChunkHost;
+            }
+        }
+    }
+    return XP_OK;
+}
+
+struct WsLayout { size_t ticket, segs, sketches, acc, total; };
+
+static WsLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc) {
+    WsLayout w;
+    w.ticket = 0;
+    w.segs = 256;
+    w.sketches = w.segs + align256(sizeof(SegDev) * (n_segs + 1));
+    w.acc = w.sketches + align256(sizeof(SketchDev*) * (n_sketches + 1));
+    w.total = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
+    return w;
+}
+
+extern "C" size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts) {
+    if (!sketches || n == 0) return 0;
+    Plan plan;
+    if (build_plan(sketches, n, opts ? opts : &kDefaultOpts, &plan) != XP_OK) return 0;
+    return ws_layout(plan.segs.size(), n, plan.acc.size()).total;
+}
+
+extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
+                                     xp_result** outs) {
+    if (!sketches || !outs || n == 0) return fail(XP_ERR_INVALID_ARG, "xp_repair_batch: null argument");
+    for (size_t i = 0; i < n; ++i) outs[i] = nullptr;
+    const xp_repair_opts* o = opts ? opts : &kDefaultOpts;
+    if (o->n_rank_ranges < 0 || (o->n_rank_ranges > 0 && !o->rank_ranges)) return fail(XP_ERR_INVALID_ARG, "bad rank_ranges");
+    if (o->cancel && *o->cancel) return fail(XP_ERR_CANCELLED, "cancelled before launch");
+    const auto t0 = std::chrono::steady_clock::now();
+    Plan plan;
+    xp_status st = build_plan(sketches, n, o, &plan);
+    if (st != XP_OK) return st;
+    cudaStream_t stream = (cudaStream_t)o->stream;
+
+    const WsLayout w = ws_layout(plan.segs.size(), n, plan.acc.size());
+    char* ws = (char*)o->workspace;
+    bool own_ws = false;
+    if (ws) {
+        if (o->workspace_bytes < w.total || ((uintptr_t)ws & 255)) return fail(XP_ERR_NOMEM, "workspace too small or misaligned");
+    } else {
+        XP_CUDA(cudaMalloc((void**)&ws, w.total));
+        own_ws = true;
+    }
+    std::vector<char> stage(w.total, 0);
+    if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
+    for (size_t i = 0; i < n; ++i) ((const SketchDev**)&stage[w.sketches])[i] = sketches[i]->d_s;
+    memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
+
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    float ms = 0.f;
+    int launches = 0;
+    std::vector<AccDev> acc(plan.acc.size());
+#define XP_CUDA_R(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { if (own_ws) cudaFree(ws); \
+        if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1); \
+        return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
+    XP_CUDA_R(cudaEventCreate(&e0));
+    XP_CUDA_R(cudaEventCreate(&e1));
+    XP_CUDA_R(cudaMemcpyAsync(ws, stage.data(), w.total, cudaMemcpyHostToDevice, stream));
+    PlanDev pd;
+    pd.n_tickets = plan.n_tickets;
+    pd.n_segs = (int)plan.segs.size();
+    pd.n_sketches = (int)n;
+    pd.segs = (const SegDev*)(ws + w.segs);
+    pd.sketches = (const SketchDev* const*)(ws + w.sketches);
+    pd.acc = (AccDev*)(ws + w.acc);
+    pd.ticket = (u64*)(ws + w.ticket);
+    XP_CUDA_R(cudaEventRecord(e0, stream));
+    if (plan.n_tickets > 0) {
+        int dev = 0, sms = 1;
+        XP_CUDA_R(cudaGetDevice(&dev));
+        XP_CUDA_R(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        u64 ctas = (u64)sms * (u64)eval_ctas_per_sm();
+        if (ctas > plan.n_tickets) ctas = plan.n_tickets;
+        XP_CUDA_R(launch_eval(pd, (int)ctas, stream));
+        ++launches;
+    }
+    XP_CUDA_R(launch_finish(pd.acc, (int)plan.acc.size(), stream));
+    ++launches;
+    XP_CUDA_R(cudaEventRecord(e1, stream));
+    XP_CUDA_R(cudaMemcpyAsync(acc.data(), pd.acc, sizeof(AccDev) * acc.size(), cudaMemcpyDeviceToHost, stream));
+    XP_CUDA_R(cudaStreamSynchronize(stream));
+    XP_CUDA_R(cudaEventElapsedTime(&ms, e0, e1));
+#undef XP_CUDA_R
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (own_ws) cudaFree(ws);
+
+    size_t ai = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const xp_sketch* s = sketches[i];
+        xp_result* r = new (std::nothrow) xp_result;
+        if (!r) {
+            for (size_t j = 0; j < i; ++j) { delete outs[j]; outs[j] = nullptr; }
+            return fail(XP_ERR_NOMEM, "out of host memory");
+        }
+        r->holes.resize(s->n_holes);
+        for (int h = 0; h < s->n_holes; ++h, ++ai) {
+            HoleResult& hr = r->holes[h];
+            const AccDev& a = acc[ai];
+            hr.max_size = s->holes[h].max_size;
+            for (int k = 1; k <= hr.max_size; ++k) {
+                hr.cand_count[k] = s->g->cnt[s->holes[h].start_nt][k];
+                hr.match_count[k] = a.match_count[k];
+            }
+            hr.evals = a.evals; hr.filter_survivors = a.filter_survivors; hr.probe_survivors = a.probe_survivors;
+            const int ls = (int)a.pad;
+            if (ls >= 1 && ls <= hr.max_size && a.match_count[ls] > 0) {
+                hr.solved = 1; hr.least_size = ls; hr.least_rank = a.min_rank[ls];
+                host_unrank(s->g, s->holes[h].start_nt, ls, hr.least_rank, &hr.code, &hr.text);
+            }
+        }
+        r->kernel_ms = ms;
+        r->n_launches = launches;
+        outs[i] = r;
+    }
+    const double total = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+    for (size_t i = 0; i < n; ++i) outs[i]->total_ms = total;
+    return XP_OK;
+}
+
+extern "C" xp_status xp_repair(const xp_sketch* sketch, const xp_repair_opts* opts, xp_result** out) {
+    if (!sketch || !out) return fail(XP_ERR_INVALID_ARG, "xp_repair: null argument");
+    return xp_repair_batch(&sketch, 1, opts, out);
+}
+
+extern "C" xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_view* v) {
+    if (!r || !v || hole < 0 || hole >= (int)r->holes.size()) return fail(XP_ERR_INVALID_ARG, "xp_result_get: bad argument");
+    const HoleResult& h = r->holes[hole];
+    v->solved = h.solved;
+    v->max_size = h.max_size;
+    v->cand_count = (const uint64_t*)h.cand_count;
+    v->match_count = (const uint64_t*)h.match_count;
+    v->least_size = h.least_size;
+    v->least_rank = h.least_rank;
+    v->least_code = h.code.data();
+    v->least_len = (int)h.code.size();
+    v->least_text = h.text.c_str();
+    v->evals_executed = h.evals;
+    v->filter_survivors = h.filter_survivors;
+    v->probe_survivors = h.probe_survivors;
+    v->kernel_ms = r->kernel_ms;
+    v->total_ms = r->total_ms;
+    v->n_launches = r->n_launches;
+    return XP_OK;
+}
+
+extern "C" void xp_result_free(xp_result* r) { delete r; }
+
+extern "C" const char* xp_last_error(void) { return g_last_error.c_str(); }
+
+// ------------------------------------------------------------------------------------------
+// integer peak
+// ------------------------------------------------------------------------------------------
+
+extern "C" xp_status xp_int32_peak(double* out_ops, double* out_ms) {
+    if (!out_ops) return fail(XP_ERR_INVALID_ARG, "xp_int32_peak: null argument");
+    int dev = 0, sms = 1;
+    XP_CUDA(cudaGetDevice(&dev));
+    XP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    u32* d = nullptr;
+    XP_CUDA(cudaMalloc(&d, 256));
+    cudaEvent_t e0, e1;
+    XP_CUDA(cudaEventCreate(&e0));
+    XP_CUDA(cudaEventCreate(&e1));
+    const int blocks = sms * 8, iters = 4096;
+    for (int which = 0; which < 2; ++which) {
+        float best = 1e30f;
+        for (int rep = 0; rep < 4; ++rep) {
+            XP_CUDA(cudaEventRecord(e0, nullptr));
+            XP_CUDA(launch_int32_peak(which, d, blocks, iters, nullptr));
+            XP_CUDA(cudaEventRecord(e1, nullptr));
+            XP_CUDA(cudaEventSynchronize(e1));
+            float ms = 0.f;
+            XP_CUDA(cudaEventElapsedTime(&ms, e0, e1));
+            if (rep > 0 && ms < best) best = ms;
+        }
+        const double ops = (double)blocks * 256.0 * (double)iters * 128.0;
+        out_ops[which] = ops / (best * 1e-3);
+        if (out_ms) out_ms[which] = best;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(d);
+    return XP_OK;
+}

@@ -1,0 +1,111 @@
+// Structures shared by the host encoder and the device kernels of libxpiler_repair.
+// Everything here is plain data laid out by the host and read by the kernels.
+#pragma once
+
+#include <stdint.h>
+
+#include "xp.h"
+
+namespace xp {
+
+typedef unsigned long long u64;
+typedef long long i64;
+typedef unsigned int u32;
+typedef int i32;
+
+constexpr int kMaxSize = XP_MAX_SIZE;
+constexpr int kMaxVars = XP_MAX_VARS;
+constexpr int kMaxNt = XP_MAX_NONTERMINALS;
+constexpr int kMaxCode = XP_MAX_CODE;
+constexpr int kMaxStack = 16;        // deepest operand stack of a context / spec expression
+constexpr int kCandStack = 8;        // deepest operand stack of a candidate (size <= 15 => <= 8 leaves)
+constexpr int kMaxProbe = 16;        // probe points per sketch
+constexpr int kProbeSamples = 64;    // sample points the probes are chosen from
+constexpr int kThreads = 256;        // threads per CTA of the evaluation kernel
+constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
+
+// A leaf production: a variable (var >= 0) or a constant.
+struct LeafDev { i32 var; i32 pad; i64 value; };
+
+// A binary production and, per candidate size s, the number of trees of its nonterminal that
+// precede its first tree (off[s]), i.e. the rank offset of the production at that size.
+struct BinDev { i32 op, lnt, rnt, pad; u64 off[kMaxSize + 2]; };
+
+struct GrammarDev {
+    i32 n_vars, n_nt, n_leaves, n_bins;
+    i32 leaf_begin[kMaxNt + 1];      // leaves of nonterminal nt: leaves[leaf_begin[nt] .. leaf_begin[nt+1])
+    i32 bin_begin[kMaxNt + 1];       // binary productions of nt: bins[bin_begin[nt] .. bin_begin[nt+1])
+    u64 cnt[kMaxNt][kMaxSize + 1];   // trees of nt with exactly s nodes
+    const LeafDev* leaves;           // device
+    const BinDev* bins;              // device
+};
+
+struct HoleDev {
+    i32 start_nt, max_size, ctx_len, spec_len;   // spec_len == 0: the spec is a table
+    const i64* spec_table;                        // device, n_points values
+    xp_instr ctx[kMaxCode];
+    xp_instr spec[kMaxCode];
+    // Probe points of this hole, most discriminating first (written by the prepare kernel).
+    i32 n_probe;
+    u32 probe_spec_ok;                            // bit j: the spec is defined at probe j
+    i64 probe_id[kMaxProbe];
+    i64 probe_pt[kMaxProbe][kMaxVars];
+    i64 probe_spec[kMaxProbe];                    // spec at the probe points
+    // Context reduced at probe 0 to a chain of steps "x -> x op c" or "x -> c op x" (constant
+    // subtrees folded); chain_len < 0: not reducible, the filter evaluates the full context.
+    i32 chain_len;
+    i32 chain_op[kMaxCode];                       // XP_OP_* | (hole on the right ? 0x100 : 0)
+    i64 chain_c[kMaxCode];
+};
+
+struct SketchDev {
+    const GrammarDev* g;                          // device
+    i32 n_vars, n_holes, domain_kind, n_samples;
+    i64 n_points;
+    const i32* coords;                            // device, table domains
+    i64 lo[kMaxVars], ext[kMaxVars];              // box: range start and extent per variable
+    HoleDev* holes;                               // device
+    i64 sample_id[kProbeSamples];                 // point ids the probes are chosen from (host-chosen)
+};
+
+// Per (sketch, hole) accumulators, zeroed (min_rank to all-ones) by the host before the launch.
+struct AccDev {
+    u64 match_count[kMaxSize + 1];
+    u64 min_rank[kMaxSize + 1];
+    u64 evals, filter_survivors, probe_survivors, pad;
+};
+
+// One contiguous piece of work.  kind 0 (linear): ranks [rank_begin, rank_end) of `size`,
+// every candidate unranked on its own.  kind 1 (tile): the product of left subtrees
+// [a_begin, a_begin+a_count) x right subtrees of one (production group, left size).
+enum { kSegLinear = 0, kSegTile = 1 };
+struct SegDev {
+    u64 first_ticket;                // tickets before this segment
+    u64 rank_begin, rank_end;        // window of ranks searched at this size
+    i32 sketch, hole, size, kind;
+    i32 acc;                         // accumulator slot
+    // tile segments
+    i32 reg_nt, reg_size;            // register-side operand: nonterminal, size
+    i32 bc_nt, bc_size;              // broadcast-side operand
+    i32 swap;                        // 1: the register side is the RIGHT operand
+    i32 n_ops;                       // productions sharing (left nt, right nt) at this split
+    i32 op[5];
+    u64 op_base[5];                  // rank of (left 0, right 0) for each of them
+    u64 reg_begin, reg_count;        // register-side subtree ranks covered by the window
+    u64 bc_begin, bc_count;          // broadcast-side subtree ranks covered
+    u64 right_count;                 // trees of the right operand (rank = base + l * right_count + r)
+    u32 reg_tiles, bc_tiles;         // tickets = reg_tiles * bc_tiles
+    i32 narrow;                      // 1: operand values fit int32 (proved by interval analysis)
+    i32 pad;
+};
+
+struct PlanDev {
+    u64 n_tickets;
+    i32 n_segs, n_sketches;
+    const SegDev* segs;              // device
+    const SketchDev* const* sketches;  // device table of device pointers
+    AccDev* acc;                     // device
+    u64* ticket;                     // device counter, zero at launch
+};
+
+}  // namespace xp

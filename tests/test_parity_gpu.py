@@ -1,0 +1,233 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI, bit for bit:
+per-size candidate counts, per-size match counts and the least solution."""
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+from tests import pybrute
+from tests.util import assert_same, check_sketch
+from xp_instances import (Hole, Sketch, Variable, config1, config2, config3, config4, config5, constant_set,
+                          free_grammar, parse_expr, quasi_affine_grammar)
+
+pytestmark = pytest.mark.gpu
+
+
+def _c1(spec, ctx=""):
+    vs = [Variable("i", 0, 16), Variable("j", 0, 16)]
+    g = free_grammar(vs, constant_set(-8, 8))
+    return Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))], name=f"c1:{spec}")
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_config1_full(xp, seed):
+    res = check_sketch(xp, config1(seed))
+    assert res[0].solved and res[0].cand_count == [0, 19, 0, 1805, 0, 342950]
+
+
+@pytest.mark.parametrize("spec", ["i", "(i*8)+j", "i%4", "7", "(i/3)-j", "100", "(i*j)%5"])
+def test_config1_grammar_specs(xp, spec):
+    check_sketch(xp, _c1(spec))
+
+
+@pytest.mark.parametrize("ctx", ["HOLE*2+i", "i<HOLE", "min(HOLE,3)", "HOLE/j", "(HOLE%3)==(i%3)", "HOLE-HOLE"])
+def test_contexts(xp, ctx):
+    check_sketch(xp, _c1("(i+j)<9" if "<" in ctx or "==" in ctx else "i+j", ctx))
+
+
+def test_no_filter_flag_gives_same_results(xp):
+    sk = _c1("(i*8)+j")
+    a = check_sketch(xp, sk)
+    b = check_sketch(xp, sk, flags=xp.XP_FLAG_NO_FILTER)
+    assert a[0].match_count == b[0].match_count and a[0].least_rank == b[0].least_rank
+
+
+def test_tiny_grammars_against_oracle_and_brute_force(xp):
+    rnd = random.Random(9)
+    vs2 = [Variable("a", 0, 3), Variable("b", -1, 2)]
+    vs3 = [Variable("p", 0, 2), Variable("q", 0, 3), Variable("r", 1, 3)]
+    cases = [(free_grammar(vs2, [-2, 0, 1, 3]), vs2), (free_grammar(vs2, [2, -3], ops=["-", "/", "%"]), vs2),
+             (quasi_affine_grammar(vs3, [-2, 0, 3], [1, 2]), vs3)]
+    for g, vs in cases:
+        T = pybrute.all_trees(g, 5)
+        for size in (1, 3, 5, 5):
+            spec = pybrute.tree_text(rnd.choice(T[(0, size)]), g)
+            for ctx in ["", f"HOLE*2+{vs[0].name}"]:
+                sk = Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))])
+                res = check_sketch(xp, sk)
+                cand, match, least, _ = pybrute.repair(sk)
+                assert res[0].cand_count == cand and res[0].match_count == match
+                if least:
+                    assert (res[0].least_size, res[0].least_rank, res[0].least_text) == least
+
+
+def test_larger_sizes_small_grammar(xp):
+    vs = [Variable("x", 0, 5), Variable("y", -2, 3)]
+    g = free_grammar(vs, [1, 2])
+    for K, spec in [(7, "((x*2)+y)-(x%2)"), (9, "((x+y)*(x-y))+1")]:
+        check_sketch(xp, Sketch(g, [Hole(0, K, spec_expr=parse_expr(spec, vs))], name=f"K{K}"))
+    gq = quasi_affine_grammar(vs, [-1, 2, 3], [1, 2, 4])
+    check_sketch(xp, Sketch(gq, [Hole(0, 9, spec_expr=parse_expr("((x/2)*3)+(y%4)", vs))], name="typed K9"))
+
+
+def test_zero_divisors_and_wraparound(xp):
+    vs = [Variable("x", 0, 3)]
+    check_sketch(xp, Sketch(free_grammar(vs, [0], ops=["/", "%", "*"]), [Hole(0, 5, spec_expr=parse_expr("0", vs))]))
+    big = [Variable("x", 2 ** 62 - 1, 2 ** 62 + 2)]
+    g = free_grammar(big, [2, 4, -1, -2 ** 63], ops=["+", "*", "/", "%", "-"])
+    for spec in ["x*4", "(x+x)+(x+x)", "(x*2)/-1"]:
+        check_sketch(xp, Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, big))], name=f"wrap:{spec}"))
+    table = np.array([-2 ** 63, 0], dtype=np.int64)                 # INT64_MIN / -1 and % -1
+    gm = free_grammar([Variable("x", 0, 2)], [-1, -2 ** 63, 0], ops=["/", "%", "*"])
+    coords = np.array([[0], [1]], dtype=np.int32)
+    check_sketch(xp, Sketch(gm, [Hole(0, 5, spec_table=table)], coords, name="int64min"))
+
+
+def test_table_domain_host_and_device_tensors(xp):
+    import torch
+    vs = [Variable("u", 0, 50), Variable("w", 0, 40)]
+    g = free_grammar(vs, [1, 2, 3, 7])
+    rnd = np.random.default_rng(0)
+    coords = np.stack([rnd.integers(0, 50, 3000), rnd.integers(0, 40, 3000)], axis=1).astype(np.int32)
+    spec = (coords[:, 0].astype(np.int64) * 7 + coords[:, 1] // 3)
+    sk = Sketch(g, [Hole(0, 5, spec_table=spec)], coords, name="table")
+    res = check_sketch(xp, sk)
+    gr = xp.xp_grammar_create(g)
+    ls = xp.xp_sketch_load(gr, sk, coords=torch.from_numpy(coords).cuda(), spec_tables={0: torch.from_numpy(spec).cuda()})
+    ws = torch.empty(xp.xp_workspace_bytes([ls]), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    dev = xp.xp_repair(ls, workspace=ws, stream=stream.cuda_stream)
+    assert dev[0].match_count == res[0].match_count and dev[0].least_text == res[0].least_text
+
+
+def test_edge_domains(xp):
+    vs = [Variable("u", 0, 4)]
+    g = free_grammar(vs, [0, 1])
+    empty = Sketch(g, [Hole(0, 3, spec_table=np.zeros(0, dtype=np.int64))], np.zeros((0, 1), dtype=np.int32), name="empty")
+    r = check_sketch(xp, empty)                    # no constraint: every candidate matches
+    assert r[0].match_count == r[0].cand_count and (r[0].least_size, r[0].least_rank) == (1, 0)
+    one = Sketch(g, [Hole(0, 3, spec_table=np.array([3], dtype=np.int64))], np.array([[3]], dtype=np.int32), name="one")
+    check_sketch(xp, one)
+    check_sketch(xp, Sketch(g, [Hole(0, 1, spec_expr=parse_expr("u", vs))], name="K1"))
+    check_sketch(xp, Sketch(g, [Hole(0, 3, spec_expr=parse_expr("u/0", vs))], name="spec undefined"))
+    check_sketch(xp, _c1("(i*8)+j"), windows={1: (0, 0), 3: (5, 5), 5: (2545, 2546)})
+    check_sketch(xp, _c1("(i*8)+j"), windows={5: (2546, 342950)})
+
+
+def test_ragged_rank_windows_partition(xp):
+    sk = _c1("i%4")
+    full = check_sketch(xp, sk)
+    cuts = [0, 1, 1023, 1025, 68590, 100001, 342949, 342950]
+    total = 0
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        total += check_sketch(xp, sk, windows={1: (0, 0), 3: (0, 0), 5: (lo, hi)})[0].match_count[5]
+    assert total == full[0].match_count[5]
+
+
+def test_config5_batch_slice(xp):
+    sks = config5(0, 24)
+    grs = {}
+    loaded = []
+    for sk in sks:
+        key = len(sk.grammar.variables), tuple(v.hi for v in sk.grammar.variables)
+        if key not in grs:
+            grs[key] = xp.xp_grammar_create(sk.grammar)
+        loaded.append(xp.xp_sketch_load(grs[key], sk))
+    res = xp.xp_repair_batch(loaded)
+    n_unsolved = 0
+    for sk, r in zip(sks, res):
+        want = oracle.repair_hole(sk)
+        assert_same(r[0], want, sk.name)
+        n_unsolved += not want.solved
+    single = xp.xp_repair(loaded[3])
+    assert single[0].match_count == res[3][0].match_count and single[0].least_rank == res[3][0].least_rank
+
+
+def test_config2_rank_slices(xp):
+    sk = config2(0)
+    n7 = 213813760000
+    rnd = random.Random(2)
+    win = {1: (0, 136), 3: (0, 92480), 5: (1000000, 1400000)}
+    for lo in [0, n7 - 300000, rnd.randrange(n7 - 10 ** 6), rnd.randrange(n7 - 10 ** 6)]:
+        w = dict(win)
+        w[7] = (lo, lo + 300000)
+        check_sketch(xp, sk, windows=w)
+
+
+def test_config3_rank_slices_three_holes(xp):
+    sk = config3(0)
+    corners_first = [0, 1806335, 27726, 55 * 56 * 9 + 2 * 3]
+    rnd = random.Random(4)
+    lo = rnd.randrange(134280950 - 10 ** 6)
+    check_sketch(xp, sk, windows={1: (0, 139), 3: (0, 20000), 5: (lo, lo + 200000)}, first_points=corners_first)
+
+
+def test_config4_rank_slices(xp):
+    sk = config4(0, n_points=1 << 14)
+    n9 = 322291652420
+    rnd = random.Random(6)
+    lo = rnd.randrange(n9 - 10 ** 6)
+    check_sketch(xp, sk, windows={1: (0, 4), 3: (0, 2084), 5: (0, 200000), 7: (10 ** 8, 10 ** 8 + 200000), 9: (lo, lo + 200000)})
+
+
+def test_planted_targets_are_found_in_their_windows(xp):
+    """The planted target's own rank (looked up with the oracle's listing) must match."""
+    for sk, size in [(config2(1), 7), (config4(1, n_points=1 << 14), 9)]:
+        target = sk.holes[0].note
+        rank = _structural_rank(sk.grammar, target)
+        assert oracle.listing(sk.grammar, 0, size, rank, rank + 1) == [target]
+        res = check_sketch(xp, sk, windows={s: (0, 0) if s != size else (rank, rank + 1) for s in range(1, size + 1)})
+        assert res[0].match_count[size] == 1 and res[0].least_text == target
+
+
+def _structural_rank(g, text):
+    """Rank of a fully parenthesised expression, computed from the oracle's counts by the
+    definition of the canonical order (test-side code, independent of the library)."""
+    from xp_instances.model import OPS, P_BIN, P_CONST, P_VAR
+    cnt = {nt: oracle.counts(g, nt, 9) for nt in range(g.n_nonterminals)}
+
+    def parse(s):
+        if s[0] != "(":
+            return ("leaf", s)
+        j = 1                                   # split at the top-level operator
+        if s[j] == "(":
+            depth = 0
+            while True:
+                depth += s[j] == "("
+                depth -= s[j] == ")"
+                j += 1
+                if depth == 0:
+                    break
+        else:
+            j += 1
+            while s[j].isalnum():
+                j += 1
+        left, op, right = s[1:j], s[j], s[j + 1:-1]
+        return (op, parse(left), parse(right))
+
+    def size(t):
+        return 1 if t[0] == "leaf" else 1 + size(t[1]) + size(t[2])
+
+    def rank(t, nt):
+        if t[0] == "leaf":
+            leaves = [p for p in g.productions if p.lhs == nt and p.kind != P_BIN]
+            for r, p in enumerate(leaves):
+                if (p.kind == P_VAR and g.variables[p.var].name == t[1]) or (p.kind == P_CONST and str(p.value) == t[1]):
+                    return r
+            raise KeyError(t)
+        s = size(t)
+        a = size(t[1])
+        base = 0
+        for p in g.productions:
+            if p.lhs != nt or p.kind != P_BIN:
+                continue
+            if OPS[p.op] == t[0]:
+                for aa in range(1, a):
+                    base += cnt[p.left][aa] * cnt[p.right][s - 1 - aa]
+                return base + rank(t[1], p.left) * cnt[p.right][s - 1 - a] + rank(t[2], p.right)
+            for aa in range(1, s - 1):
+                base += cnt[p.left][aa] * cnt[p.right][s - 1 - aa]
+        raise KeyError(t)
+
+    return rank(parse(text), 0)
