@@ -153,8 +153,10 @@ typedef struct {
 } xp_repair_opts;
 
 enum {
-    XP_FLAG_NO_FILTER = 1u              /* skip the probe-point filter stage (every candidate is unranked
+    XP_FLAG_NO_FILTER = 1u,             /* skip the probe-point filter stage (every candidate is unranked
                                            and checked on its own); same results, for testing */
+    XP_FLAG_ALWAYS_FILTER = 2u          /* use the filter stage also for rank windows too small to gain
+                                           from it; same results, for testing */
 };
 
 typedef struct xp_grammar xp_grammar;

@@ -18,6 +18,7 @@ from . import build as _build
 
 XP_MAX_SIZE = 15
 XP_FLAG_NO_FILTER = 1
+XP_FLAG_ALWAYS_FILTER = 2
 _STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_SKETCH", 4: "XP_ERR_TOO_LARGE",
            5: "XP_ERR_NOMEM", 6: "XP_ERR_CUDA", 7: "XP_ERR_TIMEOUT", 8: "XP_ERR_CANCELLED"}
 

@@ -235,6 +235,7 @@ static xp_status grammar_to_device(xp_grammar* g) {
 
 struct HoleHost {
     int start_nt = 0, max_size = 0;
+    bool filter_ok = false;          // the probe filter applies (probe 0 exists, context affine there)
 };
 
 struct xp_sketch {
@@ -387,7 +388,6 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
                 o.spec_table = (const i64*)p;
             }
         }
-        o.chain_len = -1;
         HoleHost ho;
         ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
         s->holes.push_back(ho);
@@ -398,7 +398,8 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     XP_CUDA_S(cudaMalloc(&s->d_s, sizeof(SketchDev)));
     XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
     XP_CUDA_S(launch_prepare(s->d_s, nullptr));
-    XP_CUDA_S(cudaStreamSynchronize(nullptr));
+    XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
+    for (int h = 0; h < d->n_holes; ++h) s->holes[h].filter_ok = hh[h].n_probe > 0 && hh[h].aff_ok != 0;
 #undef XP_CUDA_S
     *out = s;
     return XP_OK;
@@ -434,7 +435,73 @@ static const xp_repair_opts kDefaultOpts = {0, 0, 0, nullptr, nullptr, nullptr, 
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-constexpr u64 kLinearChunkHost = 256 * 4;     // ranks per linear ticket (matches the kernel)
+static void add_linear(Plan* plan, int sketch, int hole, int acc, int k, u64 lo, u64 hi) {
+    SegDev sg;
+    memset(&sg, 0, sizeof(sg));
+    sg.first_ticket = plan->n_tickets;
+    sg.rank_begin = lo; sg.rank_end = hi;
+    sg.sketch = sketch; sg.hole = hole; sg.size = k; sg.kind = kSegLinear; sg.acc = acc;
+    plan->segs.push_back(sg);
+    plan->n_tickets += (hi - lo + (u64)kLinearChunk - 1) / (u64)kLinearChunk;
+}
+
+// Tile segments of (start nonterminal, size k) restricted to ranks [lo, hi): one per
+// (left size, group of productions with the same operand nonterminals and the same rows).
+static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int hole, int acc, int k, u64 lo, u64 hi) {
+    const size_t first_seg = plan->segs.size();
+    for (int b = g->bin_begin[nt]; b < g->bin_begin[nt + 1]; ++b) {
+        const BinDev& bd = g->bins[b];
+        u64 base = bd.off[k];
+        for (int a = 1; a <= k - 2; ++a) {
+            const u64 cl = g->cnt[bd.lnt][a], cr = g->cnt[bd.rnt][k - 1 - a];
+            const u64 block = cl * cr;
+            if (block == 0) continue;
+            const u64 this_base = base;
+            base += block;
+            if (this_base + block <= lo || this_base >= hi) continue;
+            const u64 wlo = lo > this_base ? lo - this_base : 0;
+            const u64 whi = hi - this_base < block ? hi - this_base : block;
+            const u64 l0 = wlo / cr, l1 = (whi + cr - 1) / cr;
+            const bool reg_left = (l1 - l0) >= cr;
+            SegDev* sg = nullptr;
+            for (size_t i = first_seg; i < plan->segs.size() && !sg; ++i) {       // an open group this production fits in
+                SegDev& c = plan->segs[i];
+                const int c_lnt = c.swap ? c.bc_nt : c.reg_nt, c_rnt = c.swap ? c.reg_nt : c.bc_nt;
+                const int c_a = c.swap ? c.bc_size : c.reg_size;
+                const u64 c_l0 = c.swap ? c.bc_begin : c.reg_begin, c_l1 = c_l0 + (c.swap ? c.bc_count : c.reg_count);
+                bool has_op = false;
+                for (int o = 0; o < c.n_ops; ++o) has_op = has_op || c.op[o] == bd.op;
+                if (c_lnt == bd.lnt && c_rnt == bd.rnt && c_a == a && c_l0 == l0 && c_l1 == l1 && !has_op && c.n_ops < 5) sg = &c;
+            }
+            if (!sg) {
+                SegDev n;
+                memset(&n, 0, sizeof(n));
+                n.rank_begin = lo; n.rank_end = hi;
+                n.sketch = sketch; n.hole = hole; n.size = k; n.kind = kSegTile; n.acc = acc;
+                n.swap = reg_left ? 0 : 1;
+                n.reg_nt = reg_left ? bd.lnt : bd.rnt;  n.reg_size = reg_left ? a : k - 1 - a;
+                n.bc_nt = reg_left ? bd.rnt : bd.lnt;   n.bc_size = reg_left ? k - 1 - a : a;
+                n.reg_begin = reg_left ? l0 : 0;        n.reg_count = reg_left ? l1 - l0 : cr;
+                n.bc_begin = reg_left ? 0 : l0;         n.bc_count = reg_left ? cr : l1 - l0;
+                n.right_count = cr;
+                n.reg_tiles = (u32)((n.reg_count + kRegTile - 1) / kRegTile);
+                n.bc_tiles = (u32)((n.bc_count + kBcTile - 1) / kBcTile);
+                plan->segs.push_back(n);
+                sg = &plan->segs.back();
+            }
+            sg->op[sg->n_ops] = bd.op;
+            sg->op_base[sg->n_ops] = this_base;
+            sg->n_ops += 1;
+            if (bd.op == XP_OP_DIV || bd.op == XP_OP_MOD) sg->has_div = 1;
+        }
+    }
+    for (size_t i = first_seg; i < plan->segs.size(); ++i) {
+        plan->segs[i].first_ticket = plan->n_tickets;
+        plan->n_tickets += (u64)plan->segs[i].reg_tiles * plan->segs[i].bc_tiles;
+    }
+}
+
+constexpr u64 kTileMinRanks = 4096;          // smaller windows are searched rank by rank
 
 static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
     for (size_t i = 0; i < n; ++i) {
@@ -460,13 +527,11 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
                     }
                 }
                 if (lo >= hi) continue;
-                SegDev sg;
-                memset(&sg, 0, sizeof(sg));
-                sg.first_ticket = plan->n_tickets;
-                sg.rank_begin = lo; sg.rank_end = hi;
-                sg.sketch = (int)i; sg.hole = h; sg.size = k; sg.kind = kSegLinear; sg.acc = acc;
-                plan->segs.push_back(sg);
-                plan->n_tickets += (hi - lo + kLinearChunkHost - 1) / kLinearChunkHost;
+                const bool forced = (o->flags & XP_FLAG_ALWAYS_FILTER) != 0;
+                const bool tiles = k >= 3 && ho.filter_ok && !(o->flags & XP_FLAG_NO_FILTER) &&
+                                   (forced || hi - lo >= kTileMinRanks);
+                if (tiles) add_tiles(plan, s->g, ho.start_nt, (int)i, h, acc, k, lo, hi);
+                else add_linear(plan, (int)i, h, acc, k, lo, hi);
             }
         }
     }

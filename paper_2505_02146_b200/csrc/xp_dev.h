@@ -22,6 +22,10 @@ constexpr int kCandStack = 8;        // deepest operand stack of a candidate (si
 constexpr int kMaxProbe = 16;        // probe points per sketch
 constexpr int kProbeSamples = 64;    // sample points the probes are chosen from
 constexpr int kThreads = 256;        // threads per CTA of the evaluation kernel
+constexpr int kLinearChunk = kThreads * 4;   // ranks per linear ticket
+constexpr int kNA = 8;                // tile tickets: register-side operands per thread
+constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
+constexpr int kBcTile = 1024;         // broadcast-side operands per tile
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 
 // A leaf production: a variable (var >= 0) or a constant.
@@ -51,11 +55,11 @@ struct HoleDev {
     i64 probe_id[kMaxProbe];
     i64 probe_pt[kMaxProbe][kMaxVars];
     i64 probe_spec[kMaxProbe];                    // spec at the probe points
-    // Context reduced at probe 0 to a chain of steps "x -> x op c" or "x -> c op x" (constant
-    // subtrees folded); chain_len < 0: not reducible, the filter evaluates the full context.
-    i32 chain_len;
-    i32 chain_op[kMaxCode];                       // XP_OP_* | (hole on the right ? 0x100 : 0)
-    i64 chain_c[kMaxCode];
+    // Context at probe 0 as an affine map of the hole value, ctx(h) = aff_A * h + aff_B in
+    // wrap-around arithmetic (possible when the hole only passes through + - * with
+    // hole-free operands); aff_ok == 0: not of that form, the probe filter is not used.
+    i32 aff_ok, pad1;
+    u64 aff_A, aff_B;
 };
 
 struct SketchDev {
@@ -95,7 +99,7 @@ struct SegDev {
     u64 bc_begin, bc_count;          // broadcast-side subtree ranks covered
     u64 right_count;                 // trees of the right operand (rank = base + l * right_count + r)
     u32 reg_tiles, bc_tiles;         // tickets = reg_tiles * bc_tiles
-    i32 narrow;                      // 1: operand values fit int32 (proved by interval analysis)
+    i32 has_div;                     // some production of the group is / or %
     i32 pad;
 };
 
