@@ -20,6 +20,44 @@ namespace xp {
 // prepare
 // ------------------------------------------------------------------------------------------
 
+// Context of a hole at one point as an affine map of the hole value (wrap-around ring
+// arithmetic): walks the postfix code with entries "A*h + B".  Fails when the hole meets an
+// operator other than + - *, or itself under *, or when a hole-free operand divides by zero.
+__device__ bool ctx_affine(const HoleDev* hole, const i64* pt, u64& A, u64& B) {
+    if (hole->ctx_len == 0) { A = 1; B = 0; return true; }
+    u64 sa[kMaxStack], sb[kMaxStack];
+    int sp = 0;
+    u32 has = 0;                                        // bit i: stack entry i contains the hole
+    for (int i = 0; i < hole->ctx_len; ++i) {
+        const xp_instr c = hole->ctx[i];
+        if (c.kind != XP_I_OP) {
+            sa[sp] = c.kind == XP_I_HOLE ? 1ull : 0ull;
+            sb[sp] = c.kind == XP_I_VAR ? (u64)pt[c.arg] : (c.kind == XP_I_CONST ? (u64)c.value : 0ull);
+            has = (has & ~(1u << sp)) | ((c.kind == XP_I_HOLE ? 1u : 0u) << sp);
+            ++sp;
+            continue;
+        }
+        --sp;
+        const bool hy = (has >> sp) & 1, hx = (has >> (sp - 1)) & 1;
+        const u64 xa = sa[sp - 1], xb = sb[sp - 1], ya = sa[sp], yb = sb[sp];
+        if (!hx && !hy) {
+            i64 r;
+            if (!apply_op(c.arg, (i64)xb, (i64)yb, r)) return false;
+            sb[sp - 1] = (u64)r;
+            continue;
+        }
+        if (c.arg == XP_OP_ADD) { sa[sp - 1] = xa + ya; sb[sp - 1] = xb + yb; }
+        else if (c.arg == XP_OP_SUB) { sa[sp - 1] = xa - ya; sb[sp - 1] = xb - yb; }
+        else if (c.arg == XP_OP_MUL && !(hx && hy)) {
+            if (hx) { sa[sp - 1] = xa * yb; sb[sp - 1] = xb * yb; }
+            else { sa[sp - 1] = ya * xb; sb[sp - 1] = yb * xb; }
+        } else return false;
+        has |= 1u << (sp - 1);
+    }
+    A = sa[0]; B = sb[0];
+    return true;
+}
+
 // One CTA of kProbeSamples threads per sketch.  Thread t evaluates sample point t; thread 0
 // then orders each hole's probes: the sample with the largest |spec| + sum |coordinate|
 // first (large, distinct operand values make coincidental matches rare), the rest in sample
@@ -72,7 +110,10 @@ __global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
             }
             hole->n_probe = n;
             hole->probe_spec_ok = okmask;
-            hole->chain_len = -1;
+            u64 A = 0, B = 0;
+            hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
+            hole->aff_A = A;
+            hole->aff_B = B;
         }
     }
 }
@@ -81,9 +122,11 @@ __global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
 // eval
 // ------------------------------------------------------------------------------------------
 
-constexpr int kLinearPerThread = 4;                       // ranks per thread per linear ticket
-constexpr int kLinearChunk = kThreads * kLinearPerThread; // ranks per linear ticket
+constexpr int kLinearPerThread = kLinearChunk / kThreads; // ranks per thread per linear ticket
 constexpr int kMaxSurvivors = kLinearChunk;
+constexpr int kQueueCap = 4096;                           // filter hits waiting for the exact probe check
+constexpr int kChunkB = 32;                               // broadcast operands between block-wide queue checks
+static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
 
 struct EvalShared {
     u64 ticket;
@@ -101,11 +144,21 @@ struct EvalShared {
     u64 min_rank[kMaxSize + 1];
     u64 filter_survivors, probe_survivors;
     u64 warp_evals[kThreads / 32];
+    // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
+    // dropped), the reciprocal of each as a divisor, and the queue of filter hits
+    u32 bc_n;
+    u32 q_n, q_overflow;
+    i32 tile_wide;               // some operand of the tile does not fit int32
+    i64 bc_val[kBcTile];
+    u32 bc_mag[kBcTile];
+    unsigned short bc_idx[kBcTile];
+    unsigned char bc_sh[kBcTile];
+    u32 queue[kQueueCap];        // reg index | broadcast slot << 11 | op index << 21
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
 // Counts are sums and ranks are minima, so the order of flushes cannot change the result.
-__device__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64& my_evals) {
+__device__ __noinline__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64& my_evals) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     u64 e = my_evals;
     for (int o = 16; o > 0; o >>= 1) e += __shfl_down_sync(0xffffffffu, e, o);
@@ -134,7 +187,7 @@ __device__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64& my_evals) {
 }
 
 // Stage 2: exact check of one candidate on the hole's probe points, first failure ends it.
-__device__ __forceinline__ bool probe_check(const GrammarDev* g, const HoleDev* hole, const u32* code, int n,
+__device__ __noinline__ bool probe_check(const GrammarDev* g, const HoleDev* hole, const u32* code, int n,
                                             u64& my_evals) {
     const int np = hole->n_probe;
     for (int j = 0; j < np; ++j) {
@@ -149,7 +202,7 @@ __device__ __forceinline__ bool probe_check(const GrammarDev* g, const HoleDev* 
 
 // Stage 3: the whole CTA checks one candidate on every domain point, kThreads points at a
 // time; a failing point anywhere ends the scan at the next block-wide vote.
-__device__ void verify_survivors(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64& my_evals) {
+__device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64& my_evals) {
     const GrammarDev* g = sk->g;
     const u32 ns = sh.n_surv;
     for (u32 i = 0; i < ns; ++i) {
@@ -205,7 +258,7 @@ __device__ void verify_survivors(EvalShared& sh, const SketchDev* sk, const Hole
 }
 
 // A linear ticket: kLinearChunk consecutive ranks, each unranked and checked on its own.
-__device__ void linear_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
+__device__ __noinline__ void linear_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     const u64 first = seg.rank_begin + local * (u64)kLinearChunk;
@@ -223,6 +276,292 @@ __device__ void linear_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev
     __syncthreads();
     if (threadIdx.x == 0) { sh.filter_survivors += sh.n_surv; sh.probe_survivors += sh.n_surv; }
     verify_survivors(sh, sk, hole, seg.size, my_evals);
+}
+
+
+// ------------------------------------------------------------------------------------------
+// stage 1: probe-point filter over a product of operand tiles
+// ------------------------------------------------------------------------------------------
+//
+// A tile ticket covers candidates  L op R  for one group of productions and one left size:
+// kRegTile subtrees of one operand (kNA per thread, in registers) times up to kBcTile subtrees
+// of the other (in shared memory, read as warp-wide broadcasts).  Each operand subtree is
+// unranked and evaluated ONCE at probe 0; a candidate then costs one operation and one
+// comparison.  Everything the filter lets through is re-checked exactly (stage 2), so the
+// filter only has to be a necessary condition:
+//   * operands that fit int32 are combined in 32-bit arithmetic and compared with the low
+//     32 bits of the target (+ - * commute with reduction mod 2^32; / and % of int32 operands
+//     are exact);
+//   * an affine context  A*h + B  is folded into the operands (ring operators) or applied to
+//     the quotient / remainder;
+//   * division by a broadcast operand uses a precomputed reciprocal: for 1 <= d < 2^31,
+//     s = ceil(log2 d), m = floor(2^(31+s) / d) + 1 < 2^32, and floor(n / d) = (n * m) >> (31+s)
+//     for every 0 <= n < 2^31.
+
+__device__ __forceinline__ void reciprocal_u31(u32 d, u32& m, u32& s) {
+    s = d <= 1 ? 0u : 32u - (u32)__clz((int)(d - 1));
+    m = (u32)((1ull << (31 + s)) / d) + 1u;
+}
+
+__device__ __forceinline__ u32 div_u31(u32 n, u32 m, u32 s) { return (u32)(((u64)n * m) >> (31 + s)); }
+
+__device__ __forceinline__ u32 abs_u32(i32 x) { return x < 0 ? 0u - (u32)x : (u32)x; }
+
+// Truncating signed quotient of int32 operands whose magnitudes are below 2^31, through the
+// reciprocal (m, s) of |d|.
+__device__ __forceinline__ i32 quot_i32(i32 n, i32 d, u32 m, u32 s) {
+    const u32 q = div_u31(abs_u32(n), m, s);
+    const i32 sg = (n ^ d) >> 31;
+    return ((i32)q ^ sg) - sg;
+}
+
+__device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, u32 opi) {
+    const u32 at = atomicAdd(&sh.q_n, 1u);
+    if (at < (u32)kQueueCap) sh.queue[at] = reg_idx | (slot << 11) | (opi << 21);
+    else sh.q_overflow = 1u;
+}
+
+// Value of the subtree (nt, size, rank) at the hole's probe 0; false when a divisor is zero.
+__device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank, i64& v) {
+    if (size == 1) {
+        const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)rank];
+        v = lf.var >= 0 ? hole->probe_pt[0][lf.var] : lf.value;
+        return true;
+    }
+    u32 code[kMaxSize];
+    const int n = unrank(g, nt, size, rank, code);
+    return eval_cand(code, n, g->leaves, hole->probe_pt[0], v);
+}
+
+// Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
+// aA[j] = A * a[j]; tp = low 32 bits of (target - B).  MASK: bit0 +, bit1 -, bit2 *.
+template <u32 MASK, bool SWAP>
+__device__ __forceinline__ void ring_chunk32(EvalShared& sh, const u32 (&aA)[kNA], u32 alive,
+                                             u32 A, u32 tp, int s0, int s1, const u32 (&opi)[5]) {
+    for (int s = s0; s < s1; ++s) {
+        const u32 b = (u32)sh.bc_val[s];
+        const u32 bA = b * A;
+        bool hit = false;
+#pragma unroll
+        for (int j = 0; j < kNA; ++j) {
+            if (MASK & 1u) hit |= (aA[j] + bA) == tp;
+            if (MASK & 2u) hit |= (SWAP ? bA - aA[j] : aA[j] - bA) == tp;
+            if (MASK & 4u) hit |= (aA[j] * b) == tp;
+        }
+        if (__any_sync(0xffffffffu, hit)) {
+#pragma unroll
+            for (int j = 0; j < kNA; ++j) {
+                if (!((alive >> j) & 1u)) continue;
+                const u32 idx = (u32)j * kThreads + threadIdx.x;
+                if ((MASK & 1u) && (aA[j] + bA) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_ADD]);
+                if ((MASK & 2u) && (SWAP ? bA - aA[j] : aA[j] - bA) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_SUB]);
+                if ((MASK & 4u) && (aA[j] * b) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_MUL]);
+            }
+        }
+    }
+}
+
+// / and % on int32-exact operands.  MASK: bit0 /, bit1 %.  SWAP = false: register operand
+// divided by the broadcast one (reciprocal from shared memory); SWAP = true: the broadcast
+// operand divided by the register one (reciprocals am/as in registers).
+template <u32 MASK, bool SWAP, bool HAS_A>
+__device__ __forceinline__ void div_chunk32(EvalShared& sh, const u32 (&a)[kNA], const u32 (&am)[kNA], const u32 (&as)[kNA],
+                                            u32 alive, u32 A, u32 tp, int s0, int s1, const u32 (&opi)[5]) {
+    for (int s = s0; s < s1; ++s) {
+        const i32 b = (i32)(u32)sh.bc_val[s];
+        if (!SWAP && b == 0) continue;
+        const u32 bm = sh.bc_mag[s], bs = sh.bc_sh[s];
+        u32 hits = 0;
+#pragma unroll
+        for (int j = 0; j < kNA; ++j) {
+            const i32 aj = (i32)a[j];
+            const i32 n = SWAP ? b : aj, d = SWAP ? aj : b;
+            const i32 q = quot_i32(n, d, SWAP ? am[j] : bm, SWAP ? as[j] : bs);
+            u32 vq = (u32)q, vr = (u32)n - (u32)q * (u32)d;
+            if (HAS_A) { vq *= A; vr *= A; }
+            if ((MASK & 1u) && vq == tp) hits |= 1u << (2 * j);
+            if ((MASK & 2u) && vr == tp) hits |= 2u << (2 * j);
+        }
+        // register operands that are invalid, or (SWAP) zero divisors, are dropped here
+        if (__any_sync(0xffffffffu, hits != 0)) {
+#pragma unroll
+            for (int j = 0; j < kNA; ++j) {
+                if (!((alive >> j) & 1u) || (SWAP && a[j] == 0u)) continue;
+                const u32 idx = (u32)j * kThreads + threadIdx.x;
+                if ((hits >> (2 * j)) & 1u) push_hit(sh, idx, (u32)s, opi[XP_OP_DIV]);
+                if ((hits >> (2 * j)) & 2u) push_hit(sh, idx, (u32)s, opi[XP_OP_MOD]);
+            }
+        }
+    }
+}
+
+// Any operator on int64 operands (tiles with an operand outside int32): exact, slow, rare.
+__device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive, bool swap, u64 A, u64 tq,
+                                        int s0, int s1, int n_ops, const i32* ops) {
+    for (int s = s0; s < s1; ++s) {
+        const i64 b = sh.bc_val[s];
+        for (int j = 0; j < kNA; ++j) {
+            if (!((alive >> j) & 1u)) continue;
+            for (int o = 0; o < n_ops; ++o) {
+                i64 v;
+                if (!apply_op(ops[o], swap ? b : a[j], swap ? a[j] : b, v)) continue;
+                if ((u64)v * A == tq) push_hit(sh, (u32)j * kThreads + threadIdx.x, (u32)s, (u32)o);
+            }
+        }
+    }
+}
+
+// Stage 2 over the queue: every filter hit is rebuilt as a full candidate, checked exactly on
+// the probe points (lane = candidate), and the survivors go through the whole-domain check.
+__device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
+                                         u64 bc_first, u64& my_evals) {
+    const SegDev& seg = sh.seg;
+    const GrammarDev* g = sk->g;
+    __syncthreads();
+    const u32 nq = sh.q_n < (u32)kQueueCap ? sh.q_n : (u32)kQueueCap;
+    for (u32 base = 0; base < nq; base += kMaxSurvivors) {
+        for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
+            const u32 e = sh.queue[i];
+            const u64 rr = reg_first + (e & 2047u);
+            const u64 br = bc_first + sh.bc_idx[(e >> 11) & 1023u];
+            const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
+            const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
+            if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
+            u32 code[kMaxSize];
+            const int n = unrank(g, hole->start_nt, seg.size, rank, code);
+            if (probe_check(g, hole, code, n, my_evals)) {
+                const u32 slot = atomicAdd(&sh.n_surv, 1u);
+                sh.surv_rank[slot] = rank;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) sh.probe_survivors += sh.n_surv;
+        verify_survivors(sh, sk, hole, seg.size, my_evals);
+    }
+    if (threadIdx.x == 0) { sh.filter_survivors += nq; sh.q_n = 0; }
+    __syncthreads();
+}
+
+template <bool SWAP>
+__device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
+                                          u64 bc_first, int n_reg, i64* a64, u32 alive, u64& my_evals) {
+    const SegDev& seg = sh.seg;
+    const int nb = (int)sh.bc_n;
+    const bool tile_wide = sh.tile_wide != 0;
+    const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
+    u32 opi[5] = {0, 0, 0, 0, 0};
+    u32 mask = 0;
+    for (int o = 0; o < seg.n_ops; ++o) { opi[seg.op[o]] = (u32)o; mask |= 1u << seg.op[o]; }
+
+    u32 a[kNA], aA[kNA], am[kNA], as[kNA];
+    const u32 A = (u32)A64, tp = (u32)tq;
+#pragma unroll
+    for (int j = 0; j < kNA; ++j) {
+        a[j] = (u32)a64[j];
+        aA[j] = a[j] * A;
+        am[j] = 0; as[j] = 0;
+        if (SWAP && !tile_wide && (mask & 24u) && a[j] != 0u) reciprocal_u31(abs_u32((i32)a[j]), am[j], as[j]);
+    }
+
+    // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
+    auto run = [&](int s0, int s1, u32 alv) {
+        if (tile_wide) {
+            wide_chunk(sh, a64, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
+            return;
+        }
+        switch (mask & 7u) {
+#define XP_RING(M) case M: ring_chunk32<M, SWAP>(sh, aA, alv, A, tp, s0, s1, opi); break;
+            XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
+#undef XP_RING
+            default: break;
+        }
+        switch (((mask >> 3) & 3u) | (A != 1u ? 4u : 0u)) {
+#define XP_DIV(C, M, HA) case C: div_chunk32<M, SWAP, HA>(sh, a, am, as, alv, A, tp, s0, s1, opi); break;
+            XP_DIV(1u, 1u, false) XP_DIV(2u, 2u, false) XP_DIV(3u, 3u, false)
+            XP_DIV(5u, 1u, true) XP_DIV(6u, 2u, true) XP_DIV(7u, 3u, true)
+#undef XP_DIV
+            default: break;
+        }
+    };
+
+    u32 q_start = 0;                                    // queue length when the current chunk began
+    for (int s0 = 0; s0 < nb; s0 += kChunkB) {
+        const int s1 = s0 + kChunkB < nb ? s0 + kChunkB : nb;
+        run(s0, s1, alive);
+        __syncthreads();
+        const u32 qn = sh.q_n;
+        const bool overflow = sh.q_overflow != 0;
+        __syncthreads();
+        if (overflow) {
+            // More hits than the queue holds (a spec that most candidates satisfy at probe 0).
+            // Forget this chunk's hits, empty the queue, and redo the chunk one broadcast slot
+            // and one register operand at a time: at most kThreads * 5 hits per step.
+            if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
+            drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+            for (int s = s0; s < s1; ++s)
+                for (int j = 0; j < kNA; ++j) {
+                    run(s, s + 1, alive & (1u << j));
+                    drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                }
+            q_start = 0;
+        } else if (qn > (u32)(kQueueCap / 2)) {
+            drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+            q_start = 0;
+        } else {
+            q_start = qn;
+        }
+    }
+    drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+    (void)n_reg;
+}
+
+__device__ __noinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
+    const SegDev& seg = sh.seg;
+    const GrammarDev* g = sk->g;
+    if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
+    const u64 reg_tile = local / seg.bc_tiles, bc_tile = local % seg.bc_tiles;
+    const u64 reg_first = seg.reg_begin + reg_tile * (u64)kRegTile;
+    const u64 bc_first = seg.bc_begin + bc_tile * (u64)kBcTile;
+    const u64 reg_left = seg.reg_begin + seg.reg_count - reg_first;
+    const u64 bc_left = seg.bc_begin + seg.bc_count - bc_first;
+    const int n_reg = reg_left < (u64)kRegTile ? (int)reg_left : kRegTile;
+    const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
+    const bool swap = seg.swap != 0;
+
+    if (threadIdx.x == 0) { sh.bc_n = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
+    __syncthreads();
+
+    // operand values at probe 0
+    bool wide = false;
+    for (int i = threadIdx.x; i < n_bc; i += kThreads) {
+        i64 v;
+        if (!operand_value(g, hole, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
+        const u32 slot = atomicAdd(&sh.bc_n, 1u);
+        sh.bc_val[slot] = v;
+        sh.bc_idx[slot] = (unsigned short)i;
+        const bool fits = v > -(1ll << 31) && v < (1ll << 31);
+        wide |= !fits;
+        u32 m = 0, s = 0;
+        if (fits && v != 0 && seg.has_div && !swap) reciprocal_u31(abs_u32((i32)v), m, s);
+        sh.bc_mag[slot] = m;
+        sh.bc_sh[slot] = (unsigned char)s;
+    }
+    i64 a64[kNA];
+    u32 alive = 0;
+    for (int j = 0; j < kNA; ++j) {
+        const int idx = j * kThreads + threadIdx.x;
+        i64 v = 0;
+        if (idx < n_reg && operand_value(g, hole, seg.reg_nt, seg.reg_size, reg_first + idx, v)) {
+            alive |= 1u << j;
+            wide |= !(v > -(1ll << 31) && v < (1ll << 31));
+        } else v = 0;
+        a64[j] = v;
+    }
+    if (wide) sh.tile_wide = 1;
+    __syncthreads();
+    if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
+    if (swap) tile_body<true>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+    else tile_body<false>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
 }
 
 __global__ void __launch_bounds__(kThreads) eval_kernel(const PlanDev plan) {
@@ -255,7 +594,8 @@ __global__ void __launch_bounds__(kThreads) eval_kernel(const PlanDev plan) {
         const SketchDev* sk = plan.sketches[sh.seg.sketch];
         const HoleDev* hole = &sk->holes[sh.seg.hole];
         const u64 local = t - sh.seg.first_ticket;
-        linear_ticket(sh, sk, hole, local, my_evals);
+        if (sh.seg.kind == kSegTile) tile_ticket(sh, sk, hole, local, my_evals);
+        else linear_ticket(sh, sk, hole, local, my_evals);
         __syncthreads();
     }
     flush_acc(sh, plan, my_evals);
