@@ -13,6 +13,10 @@ from xp_instances import (Hole, Sketch, Variable, config1, config2, config3, con
 
 pytestmark = pytest.mark.gpu
 
+# 0: the library's own choice of path per rank window; 1: every candidate unranked on its own;
+# 2: the probe filter over operand tiles wherever it is legal, however small the window.
+PATHS = [0, 1, 2]
+
 
 def _c1(spec, ctx=""):
     vs = [Variable("i", 0, 16), Variable("j", 0, 16)]
@@ -26,21 +30,33 @@ def test_config1_full(xp, seed):
     assert res[0].solved and res[0].cand_count == [0, 19, 0, 1805, 0, 342950]
 
 
-@pytest.mark.parametrize("spec", ["i", "(i*8)+j", "i%4", "7", "(i/3)-j", "100", "(i*j)%5"])
-def test_config1_grammar_specs(xp, spec):
-    check_sketch(xp, _c1(spec))
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("spec", ["i", "(i*8)+j", "i%4", "7", "(i/3)-j", "100", "(i*j)%5", "0", "j-j"])
+def test_config1_grammar_specs(xp, spec, flags):
+    check_sketch(xp, _c1(spec), flags=flags)
 
 
 @pytest.mark.parametrize("ctx", ["HOLE*2+i", "i<HOLE", "min(HOLE,3)", "HOLE/j", "(HOLE%3)==(i%3)", "HOLE-HOLE"])
-def test_contexts(xp, ctx):
-    check_sketch(xp, _c1("(i+j)<9" if "<" in ctx or "==" in ctx else "i+j", ctx))
+@pytest.mark.parametrize("flags", PATHS)
+def test_contexts(xp, ctx, flags):
+    check_sketch(xp, _c1("(i+j)<9" if "<" in ctx or "==" in ctx else "i+j", ctx), flags=flags)
 
 
-def test_no_filter_flag_gives_same_results(xp):
+@pytest.mark.parametrize("ctx,spec", [("(HOLE*3)+(i*16)", "((i+j)*3)+(i*16)"), ("j-(HOLE*-5)", "j+(i*40)"),
+                                       ("(2*HOLE)-(HOLE*3)", "0-(i%5)"), ("HOLE*0", "0"), ("(i*j)+7", "(i*j)+7")])
+def test_affine_contexts_through_the_filter(xp, ctx, spec):
+    for flags in PATHS:
+        check_sketch(xp, _c1(spec, ctx), flags=flags)
+
+
+def test_path_flags_change_work_not_results(xp):
     sk = _c1("(i*8)+j")
     a = check_sketch(xp, sk)
     b = check_sketch(xp, sk, flags=xp.XP_FLAG_NO_FILTER)
-    assert a[0].match_count == b[0].match_count and a[0].least_rank == b[0].least_rank
+    c = check_sketch(xp, sk, flags=xp.XP_FLAG_ALWAYS_FILTER)
+    assert a[0].match_count == b[0].match_count == c[0].match_count and a[0].least_rank == b[0].least_rank == c[0].least_rank
+    assert b[0].filter_survivors == b[0].probe_survivors          # no filter stage: nothing is dropped before the probes
+    assert c[0].filter_survivors < sum(c[0].cand_count)           # the filter drops candidates at probe 0
 
 
 def test_tiny_grammars_against_oracle_and_brute_force(xp):
@@ -56,6 +72,9 @@ def test_tiny_grammars_against_oracle_and_brute_force(xp):
             for ctx in ["", f"HOLE*2+{vs[0].name}"]:
                 sk = Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))])
                 res = check_sketch(xp, sk)
+                for flags in (1, 2):
+                    other = check_sketch(xp, sk, flags=flags)
+                    assert other[0].match_count == res[0].match_count
                 cand, match, least, _ = pybrute.repair(sk)
                 assert res[0].cand_count == cand and res[0].match_count == match
                 if least:
@@ -66,22 +85,33 @@ def test_larger_sizes_small_grammar(xp):
     vs = [Variable("x", 0, 5), Variable("y", -2, 3)]
     g = free_grammar(vs, [1, 2])
     for K, spec in [(7, "((x*2)+y)-(x%2)"), (9, "((x+y)*(x-y))+1")]:
-        check_sketch(xp, Sketch(g, [Hole(0, K, spec_expr=parse_expr(spec, vs))], name=f"K{K}"))
+        for flags in (0, 2):
+            check_sketch(xp, Sketch(g, [Hole(0, K, spec_expr=parse_expr(spec, vs))], name=f"K{K}"), flags=flags)
     gq = quasi_affine_grammar(vs, [-1, 2, 3], [1, 2, 4])
-    check_sketch(xp, Sketch(gq, [Hole(0, 9, spec_expr=parse_expr("((x/2)*3)+(y%4)", vs))], name="typed K9"))
+    for flags in (0, 2):
+        check_sketch(xp, Sketch(gq, [Hole(0, 9, spec_expr=parse_expr("((x/2)*3)+(y%4)", vs))], name="typed K9"), flags=flags)
 
 
 def test_zero_divisors_and_wraparound(xp):
     vs = [Variable("x", 0, 3)]
-    check_sketch(xp, Sketch(free_grammar(vs, [0], ops=["/", "%", "*"]), [Hole(0, 5, spec_expr=parse_expr("0", vs))]))
+    for flags in PATHS:
+        check_sketch(xp, Sketch(free_grammar(vs, [0], ops=["/", "%", "*"]), [Hole(0, 5, spec_expr=parse_expr("0", vs))]), flags=flags)
     big = [Variable("x", 2 ** 62 - 1, 2 ** 62 + 2)]
     g = free_grammar(big, [2, 4, -1, -2 ** 63], ops=["+", "*", "/", "%", "-"])
     for spec in ["x*4", "(x+x)+(x+x)", "(x*2)/-1"]:
-        check_sketch(xp, Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, big))], name=f"wrap:{spec}"))
+        for flags in PATHS:
+            check_sketch(xp, Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, big))], name=f"wrap:{spec}"), flags=flags)
     table = np.array([-2 ** 63, 0], dtype=np.int64)                 # INT64_MIN / -1 and % -1
     gm = free_grammar([Variable("x", 0, 2)], [-1, -2 ** 63, 0], ops=["/", "%", "*"])
     coords = np.array([[0], [1]], dtype=np.int32)
-    check_sketch(xp, Sketch(gm, [Hole(0, 5, spec_table=table)], coords, name="int64min"))
+    for flags in PATHS:
+        check_sketch(xp, Sketch(gm, [Hole(0, 5, spec_table=table)], coords, name="int64min"), flags=flags)
+    # operands around the int32 boundary: tiles mix 32-bit and 64-bit operand values
+    edge = [Variable("x", 2 ** 31 - 3, 2 ** 31 + 2)]
+    ge = free_grammar(edge, [1, 2, -1, 2 ** 31, -2 ** 31], ops=["+", "-", "*", "/", "%"])
+    for spec in ["x-2147483648", "(x*2)/2", "x%-2147483648"]:
+        for flags in (0, 2):
+            check_sketch(xp, Sketch(ge, [Hole(0, 5, spec_expr=parse_expr(spec, edge))], name=f"edge32:{spec}"), flags=flags)
 
 
 def test_table_domain_host_and_device_tensors(xp):
