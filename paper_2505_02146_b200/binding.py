@@ -77,7 +77,7 @@ class xp_result_view(C.Structure):
                 ("match_count", C.POINTER(C.c_uint64)), ("least_size", C.c_int32), ("least_rank", C.c_uint64),
                 ("least_code", C.POINTER(xp_instr)), ("least_len", C.c_int32), ("least_text", C.c_char_p),
                 ("evals_executed", C.c_uint64), ("filter_survivors", C.c_uint64), ("probe_survivors", C.c_uint64),
-                ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
+                ("nominal_ops", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
 
 
 _lib = None
@@ -242,6 +242,7 @@ class HoleResult:
     evals_executed: int
     filter_survivors: int
     probe_survivors: int
+    nominal_ops: int
     kernel_ms: float
     total_ms: float
     n_launches: int
@@ -256,7 +257,7 @@ def xp_result_get(result_handle: int, hole: int) -> HoleResult:
                       v.least_text.decode() if v.solved else "",
                       [(v.least_code[i].kind, v.least_code[i].arg, v.least_code[i].value) for i in range(v.least_len)],
                       int(v.evals_executed), int(v.filter_survivors), int(v.probe_survivors),
-                      float(v.kernel_ms), float(v.total_ms), int(v.n_launches))
+                      int(v.nominal_ops), float(v.kernel_ms), float(v.total_ms), int(v.n_launches))
 
 
 def _opts(size_min=0, size_max=0, rank_ranges=None, stream=None, workspace=None, flags=0):

@@ -416,7 +416,7 @@ struct HoleResult {
     u64 least_rank = 0;
     std::vector<xp_instr> code;
     std::string text;
-    u64 evals = 0, filter_survivors = 0, probe_survivors = 0;
+    u64 evals = 0, filter_survivors = 0, probe_survivors = 0, nominal_ops = 0;
 };
 
 struct xp_result {
@@ -428,6 +428,7 @@ struct xp_result {
 struct Plan {
     std::vector<SegDev> segs;
     std::vector<AccDev> acc;
+    std::vector<u64> nominal_ops;    // per accumulator: cost-model operations of the filter stage
     u64 n_tickets = 0;
 };
 
@@ -496,8 +497,19 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
         }
     }
     for (size_t i = first_seg; i < plan->segs.size(); ++i) {
-        plan->segs[i].first_ticket = plan->n_tickets;
-        plan->n_tickets += (u64)plan->segs[i].reg_tiles * plan->segs[i].bc_tiles;
+        SegDev& c = plan->segs[i];
+        c.first_ticket = plan->n_tickets;
+        plan->n_tickets += (u64)c.reg_tiles * c.bc_tiles;
+        // cost model: operation + comparison per evaluation; / and % share one reciprocal division
+        u64 per_pair = 0;
+        bool div = false, mod = false;
+        for (int o = 0; o < c.n_ops; ++o) {
+            if (c.op[o] == XP_OP_DIV) div = true;
+            else if (c.op[o] == XP_OP_MOD) mod = true;
+            else per_pair += 2;
+        }
+        if (div || mod) per_pair += 7 + (div ? 1 : 0) + (mod ? 2 : 0);
+        plan->nominal_ops[acc] += c.reg_count * c.bc_count * per_pair;
     }
 }
 
@@ -514,6 +526,7 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
             for (int k = 0; k <= kMaxSize; ++k) a.min_rank[k] = ~0ull;
             const int acc = (int)plan->acc.size();
             plan->acc.push_back(a);
+            plan->nominal_ops.push_back(0);
             int kmin = 1, kmax = ho.max_size;
             if (o->size_min > 0) kmin = o->size_min;
             if (o->size_max > 0 && o->size_max < kmax) kmax = o->size_max;
@@ -641,6 +654,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
                 hr.match_count[k] = a.match_count[k];
             }
             hr.evals = a.evals; hr.filter_survivors = a.filter_survivors; hr.probe_survivors = a.probe_survivors;
+            hr.nominal_ops = plan.nominal_ops[ai];
             const int ls = (int)a.pad;
             if (ls >= 1 && ls <= hr.max_size && a.match_count[ls] > 0) {
                 hr.solved = 1; hr.least_size = ls; hr.least_rank = a.min_rank[ls];
@@ -676,6 +690,7 @@ extern "C" xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_v
     v->evals_executed = h.evals;
     v->filter_survivors = h.filter_survivors;
     v->probe_survivors = h.probe_survivors;
+    v->nominal_ops = h.nominal_ops;
     v->kernel_ms = r->kernel_ms;
     v->total_ms = r->total_ms;
     v->n_launches = r->n_launches;
