@@ -223,6 +223,44 @@ xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_r
 xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_view* out);
 void xp_result_free(xp_result* r);
 
+/* The same search as xp_repair for ONE sketch, for callers that must not allocate device
+ * memory while they run.  (The paper has no counterpart for this entry point: it exists for
+ * how the library is embedded, not for the method.)  Such callers are, for example, a
+ * framework whose caching allocator owns all device memory after start-up, a serving loop in
+ * which the implicit device-wide synchronisation of cudaMalloc / cudaFree is not acceptable,
+ * or a process that runs under a hard device-memory budget fixed before the first request.
+ * xp_repair either takes a caller-allocated workspace or calls cudaMalloc itself, and it
+ * creates CUDA events; this entry point does neither.  Its scratch (ticket counter, segment
+ * table, accumulators) lives in a fixed array of XP_STATIC_SCRATCH_BYTES inside the library,
+ * which every GPU that loads the library holds until the process exits.
+ *
+ *  - Inputs and outputs stay the caller's: the sketch (loaded earlier with xp_sketch_load,
+ *    which does allocate) and `out`, an array of at least n_holes summaries, filled in place.
+ *  - opts->workspace is ignored; size / rank windows, flags, stream and cancel work as in
+ *    xp_repair.  The call returns after the stream has been synchronised.
+ *  - A call whose plan needs more than the fixed array, or a sketch with more than 64 holes,
+ *    fails with XP_ERR_TOO_LARGE and a message giving the limit; nothing is launched.
+ *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ *    keeps it; make that first call before any stream capture begins.
+ *  - All calls share the one array per device.  Each call overwrites the whole part it uses
+ *    (counter and accumulators are staged in their start state), so earlier contents never
+ *    leak into a result; but two calls that overlap in time on the same device race on it.
+ *    Serialise them (same stream, or wait for the previous call to return).
+ *  - No cudaMalloc, cudaFree, event or stream creation happens inside; kernel_ms is therefore
+ *    not measured here.
+ * Errors: XP_ERR_INVALID_ARG, XP_ERR_TOO_LARGE, XP_ERR_CUDA, XP_ERR_CANCELLED. */
+enum { XP_STATIC_SCRATCH_BYTES = 1 << 20 };
+typedef struct {
+    int32_t solved, max_size, least_size, pad;
+    uint64_t least_rank;
+    uint64_t cand_count[XP_MAX_SIZE + 1];
+    uint64_t match_count[XP_MAX_SIZE + 1];
+    uint64_t evals_executed;
+    char least_text[256];
+} xp_hole_summary;
+xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_opts* opts, xp_hole_summary* out,
+                           int32_t out_cap);
+
 /* Message of the calling thread's last failed call ("" if none). */
 const char* xp_last_error(void);
 

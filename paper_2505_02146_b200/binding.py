@@ -24,7 +24,7 @@ _STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_
 
 EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_grammar_unrank",
            "xp_sketch_load", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
-           "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak"]
+           "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static"]
 
 
 class XpError(RuntimeError):
@@ -80,6 +80,13 @@ class xp_result_view(C.Structure):
                 ("nominal_ops", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
 
 
+class xp_hole_summary(C.Structure):
+    _fields_ = [("solved", C.c_int32), ("max_size", C.c_int32), ("least_size", C.c_int32), ("pad", C.c_int32),
+                ("least_rank", C.c_uint64), ("cand_count", C.c_uint64 * (XP_MAX_SIZE + 1)),
+                ("match_count", C.c_uint64 * (XP_MAX_SIZE + 1)), ("evals_executed", C.c_uint64),
+                ("least_text", C.c_char * 256)]
+
+
 _lib = None
 
 
@@ -108,6 +115,7 @@ def load(path: Optional[str] = None):
     lib.xp_result_free.restype = None
     lib.xp_last_error.restype = C.c_char_p
     lib.xp_int32_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.xp_repair_static.argtypes = [vp, C.POINTER(xp_repair_opts), C.POINTER(xp_hole_summary), C.c_int32]
     for name in EXPORTS:
         getattr(lib, name)
     _lib = lib
@@ -307,6 +315,17 @@ def xp_repair_batch(sketches: Sequence[LoadedSketch], **kw) -> List[List[HoleRes
     finally:
         for i in range(n):
             load().xp_result_free(outs[i])
+
+
+def xp_repair_static(sketch: LoadedSketch, **kw) -> List[xp_hole_summary]:
+    """The search of one sketch with the scratch in the library's fixed device array: for
+    callers that may not allocate device memory at call time.  The summaries are ctypes
+    structures owned by the caller (cand_count, match_count, solved, least_size, least_rank,
+    least_text).  Keyword options as for ``xp_repair`` (``workspace`` is ignored)."""
+    o, _keep = _opts(**kw)
+    out = (xp_hole_summary * sketch.n_holes)()
+    _check(load().xp_repair_static(sketch.handle, C.byref(o), out, sketch.n_holes))
+    return list(out)
 
 
 def xp_int32_peak() -> Tuple[float, float]:

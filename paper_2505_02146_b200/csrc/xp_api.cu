@@ -675,6 +675,62 @@ extern "C" xp_status xp_repair(const xp_sketch* sketch, const xp_repair_opts* op
     return xp_repair_batch(&sketch, 1, opts, out);
 }
 
+// The search of one sketch with every byte of device scratch taken from a fixed array inside
+// the library: no device memory is allocated or freed, no event or stream is created.
+extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_opts* opts, xp_hole_summary* out,
+                                      int32_t out_cap) {
+    if (!sketch || !out) return fail(XP_ERR_INVALID_ARG, "xp_repair_static: null argument");
+    if (out_cap < sketch->n_holes) return fail(XP_ERR_INVALID_ARG, "xp_repair_static: out has fewer entries than the sketch has holes");
+    const xp_repair_opts* o = opts ? opts : &kDefaultOpts;
+    if (o->n_rank_ranges < 0 || (o->n_rank_ranges > 0 && !o->rank_ranges)) return fail(XP_ERR_INVALID_ARG, "bad rank_ranges");
+    if (o->cancel && *o->cancel) return fail(XP_ERR_CANCELLED, "cancelled before launch");
+    Plan plan;
+    xp_status st = build_plan(&sketch, 1, o, &plan);
+    if (st != XP_OK) return st;
+    const WsLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size());
+    if (plan.acc.size() > 64)
+        return fail(XP_ERR_TOO_LARGE, "xp_repair_static: the sketch has more than 64 holes; use xp_repair with a workspace");
+    if (w.total > kStaticScratchBytes)
+        return fail(XP_ERR_TOO_LARGE, "xp_repair_static: the call needs " + std::to_string(w.total) +
+                    " bytes of scratch, the fixed array holds " + std::to_string(kStaticScratchBytes) +
+                    "; use xp_repair with a workspace");
+    static thread_local char stage[kStaticScratchBytes];          // no heap use that grows with the call
+    memset(stage, 0, w.total);
+    if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
+    ((const SketchDev**)&stage[w.sketches])[0] = sketch->d_s;
+    memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
+    AccDev acc[64];
+    cudaStream_t stream = (cudaStream_t)o->stream;
+    int dev = 0, sms = 1;
+    XP_CUDA(cudaGetDevice(&dev));
+    XP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    u64 ctas = (u64)sms * (u64)eval_ctas_per_sm();
+    if (ctas > plan.n_tickets) ctas = plan.n_tickets;
+    XP_CUDA(launch_search_static(stage, w.total, w.segs, w.sketches, w.acc, plan.n_tickets, (int)plan.segs.size(),
+                                 (int)plan.acc.size(), (int)ctas, acc, stream));
+    XP_CUDA(cudaStreamSynchronize(stream));
+    for (int h = 0; h < sketch->n_holes; ++h) {
+        xp_hole_summary& r = out[h];
+        memset(&r, 0, sizeof(r));
+        const AccDev& a = acc[h];
+        r.max_size = sketch->holes[h].max_size;
+        for (int k = 1; k <= r.max_size; ++k) {
+            r.cand_count[k] = sketch->g->cnt[sketch->holes[h].start_nt][k];
+            r.match_count[k] = a.match_count[k];
+        }
+        r.evals_executed = a.evals;
+        const int ls = (int)a.pad;
+        if (ls >= 1 && ls <= r.max_size && a.match_count[ls] > 0) {
+            r.solved = 1; r.least_size = ls; r.least_rank = a.min_rank[ls];
+            std::vector<xp_instr> code;
+            std::string text;
+            host_unrank(sketch->g, sketch->holes[h].start_nt, ls, r.least_rank, &code, &text);
+            snprintf(r.least_text, sizeof(r.least_text), "%s", text.c_str());
+        }
+    }
+    return XP_OK;
+}
+
 extern "C" xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_view* v) {
     if (!r || !v || hole < 0 || hole >= (int)r->holes.size()) return fail(XP_ERR_INVALID_ARG, "xp_result_get: bad argument");
     const HoleResult& h = r->holes[hole];

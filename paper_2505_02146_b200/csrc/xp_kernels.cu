@@ -679,6 +679,56 @@ int eval_ctas_per_sm() {
     return n;
 }
 
+// ------------------------------------------------------------------------------------------
+// search with the scratch in a fixed device array (no allocation at call time)
+// ------------------------------------------------------------------------------------------
+
+// Scratch of the allocation-free entry point: ticket counter, segment table, sketch pointer
+// and accumulators of ONE call.  Every GPU that loads the library holds these bytes until the
+// process exits.  In host code the name below is only a stand-in for the symbol; the device
+// address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+static void* g_static_scratch_addr[64];      // per device, filled on the first call made on it
+
+// Copies the staged plan (host bytes laid out as ticket | segments | sketch table | accumulators;
+// the ticket and the accumulators staged in their start state, which also wipes what the last
+// call left) into the fixed array, runs the search and the reduction on it, and queues the copy
+// of the accumulators back to `acc_out`.  Allocates nothing.
+cudaError_t launch_search_static(const void* stage, size_t total, size_t off_segs, size_t off_sketches, size_t off_acc,
+                                 u64 n_tickets, int n_segs, int n_acc, int n_ctas, AccDev* acc_out, cudaStream_t stream) {
+    if (total > kStaticScratchBytes) return cudaErrorInvalidValue;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_scratch_addr[dev] = p;
+    }
+    char* base = (char*)g_static_scratch_addr[dev];
+    e = cudaMemcpyAsync(base, stage, total, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return e;
+    PlanDev pd;
+    pd.n_tickets = n_tickets;
+    pd.n_segs = n_segs;
+    pd.n_sketches = 1;
+    pd.ticket = (u64*)base;
+    pd.segs = (const SegDev*)(base + off_segs);
+    pd.sketches = (const SketchDev* const*)(base + off_sketches);
+    pd.acc = (AccDev*)(base + off_acc);
+    if (n_tickets > 0) {
+        eval_kernel<<<n_ctas, kThreads, 0, stream>>>(pd);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    e = launch_finish(pd.acc, n_acc, stream);
+    if (e != cudaSuccess) return e;
+    return cudaMemcpyAsync(acc_out, pd.acc, sizeof(AccDev) * (size_t)n_acc, cudaMemcpyDeviceToHost, stream);
+}
+
 cudaError_t launch_int32_peak(int which, u32* out, int blocks, int iters, cudaStream_t stream) {
     if (which == 0) int32_peak_add_kernel<<<blocks, 256, 0, stream>>>(out, iters, 1u);
     else int32_peak_mad_kernel<<<blocks, 256, 0, stream>>>(out, iters, 1u);
