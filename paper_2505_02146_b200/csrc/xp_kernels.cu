@@ -128,6 +128,10 @@ constexpr int kQueueCap = 4096;                           // filter hits waiting
 constexpr int kChunkB = 32;                               // broadcast operands between block-wide queue checks
 static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
 
+// A broadcast-side operand of a tile: its value at probe 0 (lo/hi words), the reciprocal
+// multiplier of |value| as a divisor, and meta = index inside the tile | reciprocal shift << 16.
+struct __align__(16) BcEntry { u32 lo, hi, mag, meta; };
+
 struct EvalShared {
     u64 ticket;
     SegDev seg;
@@ -149,10 +153,7 @@ struct EvalShared {
     u32 bc_n;
     u32 q_n, q_overflow;
     i32 tile_wide;               // some operand of the tile does not fit int32
-    i64 bc_val[kBcTile];
-    u32 bc_mag[kBcTile];
-    unsigned short bc_idx[kBcTile];
-    unsigned char bc_sh[kBcTile];
+    BcEntry bc[kBcTile];
     u32 queue[kQueueCap];        // reg index | broadcast slot << 11 | op index << 21
 };
 
@@ -333,63 +334,105 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
     return eval_cand(code, n, g->leaves, hole->probe_pt[0], v);
 }
 
+// The register-side operands of a tile as the 32-bit loops use them.
+struct RegOps {
+    u32 aA[kNA];     // A * value (the affine context's factor folded in)
+    u32 ua[kNA];     // |value|
+    u32 sa[kNA];     // value >> 31 (all ones when negative)
+    u32 am[kNA];     // SWAP: reciprocal multiplier of |value| as a divisor (0 when |value| <= 1)
+    u32 ash[kNA];    // SWAP: reciprocal shift - 1
+    u32 ac[kNA];     // SWAP: all ones when |value| == 1 (the quotient is the dividend)
+    u32 alive;       // bit j: operand j exists and is valid at probe 0
+};
+
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
-// aA[j] = A * a[j]; tp = low 32 bits of (target - B).  MASK: bit0 +, bit1 -, bit2 *.
+// tp = low 32 bits of (target - B).  MASK: bit0 +, bit1 -, bit2 *.  Per broadcast operand b
+// the comparisons are brought to the register operand's side once:
+//   A*(a + b) == tp  <=>  A*a == tp - A*b;    A*(a - b) == tp  <=>  A*a == tp + A*b;
+//   A*(b - a) == tp  <=>  A*a == A*b - tp;    A*(a * b) == tp  <=>  (A*a) * b == tp.
 template <u32 MASK, bool SWAP>
-__device__ __forceinline__ void ring_chunk32(EvalShared& sh, const u32 (&aA)[kNA], u32 alive,
-                                             u32 A, u32 tp, int s0, int s1, const u32 (&opi)[5]) {
+__device__ __forceinline__ void ring_chunk32(EvalShared& sh, const RegOps& R, u32 alive, u32 A, u32 tp, int s0, int s1,
+                                             const u32 (&opi)[5]) {
     for (int s = s0; s < s1; ++s) {
-        const u32 b = (u32)sh.bc_val[s];
+        const u32 b = sh.bc[s].lo;
         const u32 bA = b * A;
+        const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
         bool hit = false;
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
-            if (MASK & 1u) hit |= (aA[j] + bA) == tp;
-            if (MASK & 2u) hit |= (SWAP ? bA - aA[j] : aA[j] - bA) == tp;
-            if (MASK & 4u) hit |= (aA[j] * b) == tp;
+            if (MASK & 1u) hit |= R.aA[j] == t_add;
+            if (MASK & 2u) hit |= R.aA[j] == t_sub;
+            if (MASK & 4u) hit |= R.aA[j] * b == tp;
         }
         if (__any_sync(0xffffffffu, hit)) {
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
                 if (!((alive >> j) & 1u)) continue;
                 const u32 idx = (u32)j * kThreads + threadIdx.x;
-                if ((MASK & 1u) && (aA[j] + bA) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_ADD]);
-                if ((MASK & 2u) && (SWAP ? bA - aA[j] : aA[j] - bA) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_SUB]);
-                if ((MASK & 4u) && (aA[j] * b) == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_MUL]);
+                if ((MASK & 1u) && R.aA[j] == t_add) push_hit(sh, idx, (u32)s, opi[XP_OP_ADD]);
+                if ((MASK & 2u) && R.aA[j] == t_sub) push_hit(sh, idx, (u32)s, opi[XP_OP_SUB]);
+                if ((MASK & 4u) && R.aA[j] * b == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_MUL]);
             }
         }
     }
 }
 
-// / and % on int32-exact operands.  MASK: bit0 /, bit1 %.  SWAP = false: register operand
-// divided by the broadcast one (reciprocal from shared memory); SWAP = true: the broadcast
-// operand divided by the register one (reciprocals am/as in registers).
-template <u32 MASK, bool SWAP, bool HAS_A>
-__device__ __forceinline__ void div_chunk32(EvalShared& sh, const u32 (&a)[kNA], const u32 (&am)[kNA], const u32 (&as)[kNA],
-                                            u32 alive, u32 A, u32 tp, int s0, int s1, const u32 (&opi)[5]) {
+// / and % on int32-exact operands.  MASK: bit0 /, bit1 %.
+// SWAP = false: register operand / broadcast operand (reciprocal from shared memory);
+// SWAP = true: broadcast operand / register operand (reciprocals in registers).
+// SIGNED = false (context factor A == 1): only magnitudes are compared, |quotient| or
+// |remainder| against |target| (tabs) -- still a necessary condition, and the signs are settled
+// by the exact check.  SIGNED = true: signed results times A against tp.
+template <u32 MASK, bool SWAP, bool SIGNED>
+__device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32 alive, u32 A, u32 tp, u32 tabs,
+                                            int s0, int s1, const u32 (&opi)[5]) {
     for (int s = s0; s < s1; ++s) {
-        const i32 b = (i32)(u32)sh.bc_val[s];
-        if (!SWAP && b == 0) continue;
-        const u32 bm = sh.bc_mag[s], bs = sh.bc_sh[s];
-        u32 hits = 0;
+        const BcEntry e = sh.bc[s];
+        const u32 ub = abs_u32((i32)e.lo);
+        const u32 sb = (u32)((i32)e.lo >> 31);
+        if (!SWAP && ub == 0u) continue;                              // zero divisor: invalid
+        const u32 bm = e.mag, bsh = (e.meta >> 16) - 1u;
+        const bool unit = !SWAP && ub == 1u;
+        // magnitudes of quotient and remainder for register operand j
+        auto qr = [&](int j, u32& qu, u32& ru) {
+            if (SWAP) {
+                qu = (__umulhi(ub, R.am[j]) >> R.ash[j]) + (ub & R.ac[j]);
+                ru = ub - qu * R.ua[j];
+            } else {
+                qu = unit ? R.ua[j] : (__umulhi(R.ua[j], bm) >> bsh);
+                ru = R.ua[j] - qu * ub;
+            }
+        };
+        auto test = [&](int j, bool& hq, bool& hr) {
+            u32 qu, ru;
+            qr(j, qu, ru);
+            if (SIGNED) {
+                const u32 sq = R.sa[j] ^ sb, sr = SWAP ? sb : R.sa[j];       // signs of quotient / remainder
+                hq = (((qu ^ sq) - sq) * A) == tp;
+                hr = (((ru ^ sr) - sr) * A) == tp;
+            } else {
+                hq = qu == tabs;
+                hr = ru == tabs;
+            }
+        };
+        bool hit = false;
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
-            const i32 aj = (i32)a[j];
-            const i32 n = SWAP ? b : aj, d = SWAP ? aj : b;
-            const i32 q = quot_i32(n, d, SWAP ? am[j] : bm, SWAP ? as[j] : bs);
-            u32 vq = (u32)q, vr = (u32)n - (u32)q * (u32)d;
-            if (HAS_A) { vq *= A; vr *= A; }
-            if ((MASK & 1u) && vq == tp) hits |= 1u << (2 * j);
-            if ((MASK & 2u) && vr == tp) hits |= 2u << (2 * j);
+            bool hq, hr;
+            test(j, hq, hr);
+            if (MASK & 1u) hit |= hq;
+            if (MASK & 2u) hit |= hr;
         }
-        // register operands that are invalid, or (SWAP) zero divisors, are dropped here
-        if (__any_sync(0xffffffffu, hits != 0)) {
+        if (__any_sync(0xffffffffu, hit)) {
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
-                if (!((alive >> j) & 1u) || (SWAP && a[j] == 0u)) continue;
+                // register operands that are invalid, or (SWAP) zero divisors, are dropped here
+                if (!((alive >> j) & 1u) || (SWAP && R.ua[j] == 0u)) continue;
+                bool hq, hr;
+                test(j, hq, hr);
                 const u32 idx = (u32)j * kThreads + threadIdx.x;
-                if ((hits >> (2 * j)) & 1u) push_hit(sh, idx, (u32)s, opi[XP_OP_DIV]);
-                if ((hits >> (2 * j)) & 2u) push_hit(sh, idx, (u32)s, opi[XP_OP_MOD]);
+                if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, opi[XP_OP_DIV]);
+                if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, opi[XP_OP_MOD]);
             }
         }
     }
@@ -399,7 +442,7 @@ __device__ __forceinline__ void div_chunk32(EvalShared& sh, const u32 (&a)[kNA],
 __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive, bool swap, u64 A, u64 tq,
                                         int s0, int s1, int n_ops, const i32* ops) {
     for (int s = s0; s < s1; ++s) {
-        const i64 b = sh.bc_val[s];
+        const i64 b = (i64)(((u64)sh.bc[s].hi << 32) | sh.bc[s].lo);
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
             for (int o = 0; o < n_ops; ++o) {
@@ -423,7 +466,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, co
         for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
             const u32 e = sh.queue[i];
             const u64 rr = reg_first + (e & 2047u);
-            const u64 br = bc_first + sh.bc_idx[(e >> 11) & 1023u];
+            const u64 br = bc_first + (sh.bc[(e >> 11) & 1023u].meta & 0xffffu);
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
             const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
             if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
@@ -453,14 +496,25 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     u32 mask = 0;
     for (int o = 0; o < seg.n_ops; ++o) { opi[seg.op[o]] = (u32)o; mask |= 1u << seg.op[o]; }
 
-    u32 a[kNA], aA[kNA], am[kNA], as[kNA];
     const u32 A = (u32)A64, tp = (u32)tq;
+    // With A == 1 a quotient or remainder of int32 operands can only equal a target of
+    // magnitude below 2^31; its magnitude is what the unsigned loops compare with.
+    const i64 T = (i64)tq;
+    const bool t_small = T > -(1ll << 31) && T < (1ll << 31);
+    const u32 tabs = (u32)(T < 0 ? -T : T);
+    RegOps R;
+    R.alive = alive;
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
-        a[j] = (u32)a64[j];
-        aA[j] = a[j] * A;
-        am[j] = 0; as[j] = 0;
-        if (SWAP && !tile_wide && (mask & 24u) && a[j] != 0u) reciprocal_u31(abs_u32((i32)a[j]), am[j], as[j]);
+        const i32 v = (i32)a64[j];
+        R.aA[j] = (u32)v * A;
+        R.ua[j] = abs_u32(v);
+        R.sa[j] = (u32)(v >> 31);
+        R.am[j] = 0; R.ash[j] = 0; R.ac[j] = 0;
+        if (SWAP && !tile_wide && (mask & 24u)) {
+            if (R.ua[j] == 1u) R.ac[j] = 0xffffffffu;
+            else if (R.ua[j] > 1u) { u32 m, sft; reciprocal_u31(R.ua[j], m, sft); R.am[j] = m; R.ash[j] = sft - 1u; }
+        }
     }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
@@ -470,13 +524,14 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_chunk32<M, SWAP>(sh, aA, alv, A, tp, s0, s1, opi); break;
+#define XP_RING(M) case M: ring_chunk32<M, SWAP>(sh, R, alv, A, tp, s0, s1, opi); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
         }
+        if (A == 1u && !t_small) return;                 // no int32 quotient or remainder can be the target
         switch (((mask >> 3) & 3u) | (A != 1u ? 4u : 0u)) {
-#define XP_DIV(C, M, HA) case C: div_chunk32<M, SWAP, HA>(sh, a, am, as, alv, A, tp, s0, s1, opi); break;
+#define XP_DIV(C, M, SG) case C: div_chunk32<M, SWAP, SG>(sh, R, alv, A, tp, tabs, s0, s1, opi); break;
             XP_DIV(1u, 1u, false) XP_DIV(2u, 2u, false) XP_DIV(3u, 3u, false)
             XP_DIV(5u, 1u, true) XP_DIV(6u, 2u, true) XP_DIV(7u, 3u, true)
 #undef XP_DIV
@@ -515,7 +570,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     (void)n_reg;
 }
 
-__device__ __noinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
+__device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
@@ -537,14 +592,13 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, co
         i64 v;
         if (!operand_value(g, hole, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
         const u32 slot = atomicAdd(&sh.bc_n, 1u);
-        sh.bc_val[slot] = v;
-        sh.bc_idx[slot] = (unsigned short)i;
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
         u32 m = 0, s = 0;
         if (fits && v != 0 && seg.has_div && !swap) reciprocal_u31(abs_u32((i32)v), m, s);
-        sh.bc_mag[slot] = m;
-        sh.bc_sh[slot] = (unsigned char)s;
+        BcEntry e;
+        e.lo = (u32)(u64)v; e.hi = (u32)((u64)v >> 32); e.mag = m; e.meta = (u32)i | (s << 16);
+        sh.bc[slot] = e;
     }
     i64 a64[kNA];
     u32 alive = 0;
@@ -564,7 +618,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, co
     else tile_body<false>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
 }
 
-__global__ void __launch_bounds__(kThreads) eval_kernel(const PlanDev plan) {
+__global__ void __launch_bounds__(kThreads, 2) eval_kernel(const PlanDev plan) {
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
