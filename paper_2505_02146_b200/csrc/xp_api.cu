@@ -400,6 +400,40 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     XP_CUDA_S(launch_prepare(s->d_s, nullptr));
     XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
     for (int h = 0; h < d->n_holes; ++h) s->holes[h].filter_ok = hh[h].n_probe > 0 && hh[h].aff_ok != 0;
+    // Subtree-value tables at probe 0 for the holes that use the filter: sizes 1, 2, ... while
+    // every nonterminal has at most kTabMaxEntries trees of that size, and never the sizes that
+    // only occur as whole candidates (operands have at most max_size - 2 nodes).
+    for (int h = 0; h < d->n_holes; ++h) {
+        if (!s->holes[h].filter_ok) continue;
+        HoleDev& o = hh[h];
+        u64 total = 0;
+        int tmax = 0;
+        for (int k = 1; k <= o.max_size - 2; ++k) {
+            u64 at_size = 0;
+            bool fits = true;
+            for (int nt = 0; nt < g->n_nt; ++nt) { fits = fits && g->cnt[nt][k] <= kTabMaxEntries; at_size += g->cnt[nt][k]; }
+            if (!fits) break;
+            for (int nt = 0; nt < g->n_nt; ++nt) { o.tab_off[nt][k] = total; total += g->cnt[nt][k]; }
+            tmax = k;
+        }
+        if (tmax == 0 || total == 0) continue;
+        void* pv = nullptr;
+        void* pk = nullptr;
+        XP_CUDA_S(cudaMalloc(&pv, sizeof(i64) * total));
+        s->owned.push_back(pv);
+        XP_CUDA_S(cudaMalloc(&pk, total));
+        s->owned.push_back(pk);
+        o.tab_val = (i64*)pv;
+        o.tab_ok = (unsigned char*)pk;
+        o.tab_max_size = tmax;
+        XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &o, sizeof(HoleDev), cudaMemcpyHostToDevice));
+        for (int k = 1; k <= tmax; ++k) {
+            u64 at_size = 0;
+            for (int nt = 0; nt < g->n_nt; ++nt) at_size += g->cnt[nt][k];
+            XP_CUDA_S(launch_subvalues(s->d_s, h, k, at_size, nullptr));
+        }
+    }
+    XP_CUDA_S(cudaStreamSynchronize(nullptr));
 #undef XP_CUDA_S
     *out = s;
     return XP_OK;

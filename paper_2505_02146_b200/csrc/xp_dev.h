@@ -26,6 +26,7 @@ constexpr int kLinearChunk = kThreads * 4;   // ranks per linear ticket
 constexpr int kNA = 8;                // tile tickets: register-side operands per thread
 constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
 constexpr int kBcTile = 1024;         // broadcast-side operands per tile
+constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 
 // A leaf production: a variable (var >= 0) or a constant.
@@ -60,6 +61,14 @@ struct HoleDev {
     // hole-free operands); aff_ok == 0: not of that form, the probe filter is not used.
     i32 aff_ok, pad1;
     u64 aff_A, aff_B;
+    // Values at probe 0 of every subtree of the small sizes 1..tab_max_size, by (nonterminal,
+    // size, rank): tab_val[tab_off[nt][size] + rank], with tab_ok telling whether the subtree
+    // is defined there (no zero divisor).  Built bottom-up once per sketch; operands of the
+    // filter stage are looked up here instead of being unranked again in every tile.
+    i32 tab_max_size, pad2;
+    u64 tab_off[kMaxNt][kMaxSize + 1];
+    i64* tab_val;                                 // device
+    unsigned char* tab_ok;                        // device
 };
 
 struct SketchDev {

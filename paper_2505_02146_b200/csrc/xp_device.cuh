@@ -77,6 +77,26 @@ __device__ __noinline__ int unrank(const GrammarDev* __restrict__ g, int nt, int
     return n;
 }
 
+// One level of unranking: the root production and the operand subtrees (sizes and ranks) of
+// the tree of (nt, size >= 3) with the given rank.
+__device__ __forceinline__ void unrank_root(const GrammarDev* __restrict__ g, int nt, int size, u64 rank,
+                                            int& op, int& lnt, int& rnt, int& a, u64& l, u64& r) {
+    int p = g->bin_begin[nt];
+    const int pe = g->bin_begin[nt + 1];
+    while (p + 1 < pe && g->bins[p + 1].off[size] <= rank) ++p;
+    const BinDev* bp = &g->bins[p];
+    u64 rem = rank - bp->off[size];
+    op = bp->op; lnt = bp->lnt; rnt = bp->rnt;
+    u64 cr;
+    for (a = 1;; ++a) {
+        cr = g->cnt[rnt][size - 1 - a];
+        const u64 block = g->cnt[lnt][a] * cr;
+        if (rem < block || a == size - 2) break;
+        rem -= block;
+    }
+    divmod_u64(rem, cr, l, r);
+}
+
 // Value of a candidate (postfix code over the grammar's leaves) at one point.
 __device__ __forceinline__ bool eval_cand(const u32* code, int n, const LeafDev* __restrict__ leaves,
                                           const i64* pt, i64& out) {

@@ -323,15 +323,61 @@ __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, 
 }
 
 // Value of the subtree (nt, size, rank) at the hole's probe 0; false when a divisor is zero.
+// Small sizes come from the hole's subtree-value tables; a larger subtree whose operands are
+// both in the tables costs one level of unranking; anything else is unranked in full.
 __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank, i64& v) {
+    const int tmax = hole->tab_max_size;
+    if (size <= tmax) {
+        const u64 at = hole->tab_off[nt][size] + rank;
+        v = hole->tab_val[at];
+        return hole->tab_ok[at] != 0;
+    }
     if (size == 1) {
         const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)rank];
         v = lf.var >= 0 ? hole->probe_pt[0][lf.var] : lf.value;
         return true;
     }
+    if (tmax >= 1) {
+        int op, lnt, rnt, a;
+        u64 l, r;
+        unrank_root(g, nt, size, rank, op, lnt, rnt, a, l, r);
+        if (a <= tmax && size - 1 - a <= tmax) {
+            const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;
+            if (!hole->tab_ok[la] || !hole->tab_ok[ra]) return false;
+            return apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
+        }
+    }
     u32 code[kMaxSize];
     const int n = unrank(g, nt, size, rank, code);
     return eval_cand(code, n, g->leaves, hole->probe_pt[0], v);
+}
+
+// Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
+// rank); the operands' values come from the smaller sizes built by earlier launches.
+__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size) {
+    const GrammarDev* g = sk->g;
+    HoleDev* hole = &sk->holes[hole_index];
+    u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int nt = 0; nt < g->n_nt; ++nt) {
+        const u64 c = g->cnt[nt][size];
+        if (idx >= c) { idx -= c; continue; }
+        i64 v = 0;
+        bool ok = true;
+        if (size == 1) {
+            const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)idx];
+            v = lf.var >= 0 ? hole->probe_pt[0][lf.var] : lf.value;
+        } else {
+            int op, lnt, rnt, a;
+            u64 l, r;
+            unrank_root(g, nt, size, idx, op, lnt, rnt, a, l, r);
+            const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;
+            ok = hole->tab_ok[la] && hole->tab_ok[ra] && apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
+        }
+        const u64 at = hole->tab_off[nt][size] + idx;
+        hole->tab_val[at] = v;
+        hole->tab_ok[at] = ok ? 1 : 0;
+        return;
+    }
 }
 
 // The register-side operands of a tile as the 32-bit loops use them.
@@ -712,6 +758,12 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream) {
     prepare_kernel<<<1, kProbeSamples, 0, stream>>>(s);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, u64 n_entries, cudaStream_t stream) {
+    if (n_entries == 0) return cudaSuccess;
+    subvalue_kernel<<<(unsigned)((n_entries + 255) / 256), 256, 0, stream>>>(s, hole_index, size);
     return cudaGetLastError();
 }
 

@@ -8,6 +8,7 @@
 namespace xp {
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream);
+cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, u64 n_entries, cudaStream_t stream);
 cudaError_t launch_eval(const PlanDev& plan, int n_ctas, cudaStream_t stream);
 cudaError_t launch_finish(AccDev* acc, int n_acc, cudaStream_t stream);
 int eval_ctas_per_sm();
