@@ -352,6 +352,64 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
     return eval_cand(code, n, g->leaves, hole->probe_pt[0], v);
 }
 
+// Values at probe 0 of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
+// returns the mask of those that are defined there and sets `wide` if one does not fit int32.
+// A subtree above the table sizes whose operands are in the tables is unranked one level for
+// the first rank only; the following ranks advance the operand ranks like an odometer (right
+// operand fastest), so the left operand's value is fetched once per run.
+__device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank,
+                                              int n, i64* out, bool& wide) {
+    u32 alive = 0;
+    const int tmax = hole->tab_max_size;
+    for (int j = 0; j < kNA; ++j) out[j] = 0;
+    if (n <= 0) return 0;
+    if (size > tmax && tmax >= 1 && size >= 3) {
+        int op, lnt, rnt, a;
+        u64 l, r;
+        unrank_root(g, nt, size, rank, op, lnt, rnt, a, l, r);
+        bool tables = a <= tmax && size - 1 - a <= tmax;
+        int j = 0;
+        while (tables && j < n) {
+            const u64 cl = g->cnt[lnt][a], cr = g->cnt[rnt][size - 1 - a];
+            const u64 lbase = hole->tab_off[lnt][a], rbase = hole->tab_off[rnt][size - 1 - a];
+            for (; j < n && l < cl; ++l, r = 0) {
+                const bool lok = hole->tab_ok[lbase + l] != 0;
+                const i64 lv = hole->tab_val[lbase + l];
+                for (; j < n && r < cr; ++r, ++j) {
+                    i64 v;
+                    if (lok && hole->tab_ok[rbase + r] && apply_op(op, lv, hole->tab_val[rbase + r], v)) {
+                        out[j] = v;
+                        alive |= 1u << j;
+                        wide |= !(v > -(1ll << 31) && v < (1ll << 31));
+                    }
+                }
+                if (j == n) break;
+            }
+            if (j < n) {                                  // ran off this (production, left size) block
+                unrank_root(g, nt, size, rank + j, op, lnt, rnt, a, l, r);
+                tables = a <= tmax && size - 1 - a <= tmax;
+            }
+        }
+        if (j == n) return alive;
+        for (; j < n; ++j) {
+            i64 v;
+            if (operand_value(g, hole, nt, size, rank + j, v)) {
+                out[j] = v; alive |= 1u << j;
+                wide |= !(v > -(1ll << 31) && v < (1ll << 31));
+            }
+        }
+        return alive;
+    }
+    for (int j = 0; j < n; ++j) {
+        i64 v;
+        if (operand_value(g, hole, nt, size, rank + j, v)) {
+            out[j] = v; alive |= 1u << j;
+            wide |= !(v > -(1ll << 31) && v < (1ll << 31));
+        }
+    }
+    return alive;
+}
+
 // Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
 // rank); the operands' values come from the smaller sizes built by earlier launches.
 __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size) {
@@ -384,7 +442,7 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int 
 struct RegOps {
     u32 aA[kNA];     // A * value (the affine context's factor folded in)
     u32 ua[kNA];     // |value|
-    u32 sa[kNA];     // value >> 31 (all ones when negative)
+    u32 neg;         // bit j: value j is negative
     u32 am[kNA];     // SWAP: reciprocal multiplier of |value| as a divisor (0 when |value| <= 1)
     u32 ash[kNA];    // SWAP: reciprocal shift - 1
     u32 ac[kNA];     // SWAP: all ones when |value| == 1 (the quotient is the dividend)
@@ -403,18 +461,19 @@ __device__ __forceinline__ void ring_chunk32(EvalShared& sh, const RegOps& R, u3
         const u32 b = sh.bc[s].lo;
         const u32 bA = b * A;
         const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
-        bool hit = false;
+        bool h0 = false, h1 = false, h2 = false, h3 = false;          // independent chains of comparisons
 #pragma unroll
-        for (int j = 0; j < kNA; ++j) {
-            if (MASK & 1u) hit |= R.aA[j] == t_add;
-            if (MASK & 2u) hit |= R.aA[j] == t_sub;
-            if (MASK & 4u) hit |= R.aA[j] * b == tp;
+        for (int j = 0; j < kNA; j += 2) {
+            if (MASK & 1u) { h0 |= R.aA[j] == t_add; h1 |= R.aA[j + 1] == t_add; }
+            if (MASK & 2u) { h2 |= R.aA[j] == t_sub; h3 |= R.aA[j + 1] == t_sub; }
+            if (MASK & 4u) { h0 |= R.aA[j] * b == tp; h3 |= R.aA[j + 1] * b == tp; }
         }
+        const bool hit = h0 | h1 | h2 | h3;
         if (__any_sync(0xffffffffu, hit)) {
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
                 if (!((alive >> j) & 1u)) continue;
-                const u32 idx = (u32)j * kThreads + threadIdx.x;
+                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
                 if ((MASK & 1u) && R.aA[j] == t_add) push_hit(sh, idx, (u32)s, opi[XP_OP_ADD]);
                 if ((MASK & 2u) && R.aA[j] == t_sub) push_hit(sh, idx, (u32)s, opi[XP_OP_SUB]);
                 if ((MASK & 4u) && R.aA[j] * b == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_MUL]);
@@ -438,22 +497,22 @@ __device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32
         const u32 sb = (u32)((i32)e.lo >> 31);
         if (!SWAP && ub == 0u) continue;                              // zero divisor: invalid
         const u32 bm = e.mag, bsh = (e.meta >> 16) - 1u;
-        const bool unit = !SWAP && ub == 1u;
-        // magnitudes of quotient and remainder for register operand j
-        auto qr = [&](int j, u32& qu, u32& ru) {
+        // magnitudes of quotient and remainder for register operand j; UNIT: the divisor is +-1
+        auto test = [&](int j, bool unit, bool& hq, bool& hr) {
+            u32 qu, ru;
             if (SWAP) {
                 qu = (__umulhi(ub, R.am[j]) >> R.ash[j]) + (ub & R.ac[j]);
                 ru = ub - qu * R.ua[j];
+            } else if (unit) {
+                qu = R.ua[j];
+                ru = 0u;
             } else {
-                qu = unit ? R.ua[j] : (__umulhi(R.ua[j], bm) >> bsh);
+                qu = __umulhi(R.ua[j], bm) >> bsh;
                 ru = R.ua[j] - qu * ub;
             }
-        };
-        auto test = [&](int j, bool& hq, bool& hr) {
-            u32 qu, ru;
-            qr(j, qu, ru);
             if (SIGNED) {
-                const u32 sq = R.sa[j] ^ sb, sr = SWAP ? sb : R.sa[j];       // signs of quotient / remainder
+                const u32 sa = (u32)((i32)(R.neg << (31 - j)) >> 31);
+                const u32 sq = sa ^ sb, sr = SWAP ? sb : sa;          // signs of quotient / remainder
                 hq = (((qu ^ sq) - sq) * A) == tp;
                 hr = (((ru ^ sr) - sr) * A) == tp;
             } else {
@@ -461,22 +520,34 @@ __device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32
                 hr = ru == tabs;
             }
         };
-        bool hit = false;
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+        if (!SWAP && ub == 1u) {
 #pragma unroll
-        for (int j = 0; j < kNA; ++j) {
-            bool hq, hr;
-            test(j, hq, hr);
-            if (MASK & 1u) hit |= hq;
-            if (MASK & 2u) hit |= hr;
+            for (int j = 0; j < kNA; j += 2) {
+                bool q0, r0, q1, r1;
+                test(j, true, q0, r0);
+                test(j + 1, true, q1, r1);
+                if (MASK & 1u) { h0 |= q0; h1 |= q1; }
+                if (MASK & 2u) { h2 |= r0; h3 |= r1; }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kNA; j += 2) {
+                bool q0, r0, q1, r1;
+                test(j, false, q0, r0);
+                test(j + 1, false, q1, r1);
+                if (MASK & 1u) { h0 |= q0; h1 |= q1; }
+                if (MASK & 2u) { h2 |= r0; h3 |= r1; }
+            }
         }
-        if (__any_sync(0xffffffffu, hit)) {
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
                 // register operands that are invalid, or (SWAP) zero divisors, are dropped here
                 if (!((alive >> j) & 1u) || (SWAP && R.ua[j] == 0u)) continue;
                 bool hq, hr;
-                test(j, hq, hr);
-                const u32 idx = (u32)j * kThreads + threadIdx.x;
+                test(j, !SWAP && ub == 1u, hq, hr);
+                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
                 if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, opi[XP_OP_DIV]);
                 if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, opi[XP_OP_MOD]);
             }
@@ -494,7 +565,7 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive,
             for (int o = 0; o < n_ops; ++o) {
                 i64 v;
                 if (!apply_op(ops[o], swap ? b : a[j], swap ? a[j] : b, v)) continue;
-                if ((u64)v * A == tq) push_hit(sh, (u32)j * kThreads + threadIdx.x, (u32)s, (u32)o);
+                if ((u64)v * A == tq) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
             }
         }
     }
@@ -550,12 +621,13 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     const u32 tabs = (u32)(T < 0 ? -T : T);
     RegOps R;
     R.alive = alive;
+    R.neg = 0;
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
         const i32 v = (i32)a64[j];
         R.aA[j] = (u32)v * A;
         R.ua[j] = abs_u32(v);
-        R.sa[j] = (u32)(v >> 31);
+        if (v < 0) R.neg |= 1u << j;
         R.am[j] = 0; R.ash[j] = 0; R.ac[j] = 0;
         if (SWAP && !tile_wide && (mask & 24u)) {
             if (R.ua[j] == 1u) R.ac[j] = 0xffffffffu;
@@ -647,16 +719,9 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
         sh.bc[slot] = e;
     }
     i64 a64[kNA];
-    u32 alive = 0;
-    for (int j = 0; j < kNA; ++j) {
-        const int idx = j * kThreads + threadIdx.x;
-        i64 v = 0;
-        if (idx < n_reg && operand_value(g, hole, seg.reg_nt, seg.reg_size, reg_first + idx, v)) {
-            alive |= 1u << j;
-            wide |= !(v > -(1ll << 31) && v < (1ll << 31));
-        } else v = 0;
-        a64[j] = v;
-    }
+    const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
+    const u32 alive = fill_reg_operands(g, hole, seg.reg_nt, seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+                                        mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide);
     if (wide) sh.tile_wide = 1;
     __syncthreads();
     if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
@@ -664,7 +729,10 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
     else tile_body<false>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
 }
 
-__global__ void __launch_bounds__(kThreads, 2) eval_kernel(const PlanDev plan) {
+#ifndef XP_MIN_CTAS
+#define XP_MIN_CTAS 3
+#endif
+__global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanDev plan) {
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
