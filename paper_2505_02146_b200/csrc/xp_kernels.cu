@@ -449,14 +449,21 @@ struct RegOps {
     u32 alive;       // bit j: operand j exists and is valid at probe 0
 };
 
+// The two loops below are separate (not inlined) functions on purpose: each copies just the
+// operand arrays it needs from the tile's RegOps into registers and runs with a small live
+// set, instead of sharing one large frame with the rest of the kernel.
+// `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
+
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
 // tp = low 32 bits of (target - B).  MASK: bit0 +, bit1 -, bit2 *.  Per broadcast operand b
 // the comparisons are brought to the register operand's side once:
 //   A*(a + b) == tp  <=>  A*a == tp - A*b;    A*(a - b) == tp  <=>  A*a == tp + A*b;
 //   A*(b - a) == tp  <=>  A*a == A*b - tp;    A*(a * b) == tp  <=>  (A*a) * b == tp.
 template <u32 MASK, bool SWAP>
-__device__ __forceinline__ void ring_chunk32(EvalShared& sh, const RegOps& R, u32 alive, u32 A, u32 tp, int s0, int s1,
-                                             const u32 (&opi)[5]) {
+__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, int s0, int s1, u32 opip) {
+    u32 aA[kNA];
+#pragma unroll
+    for (int j = 0; j < kNA; ++j) aA[j] = Rm->aA[j];
     for (int s = s0; s < s1; ++s) {
         const u32 b = sh.bc[s].lo;
         const u32 bA = b * A;
@@ -464,19 +471,18 @@ __device__ __forceinline__ void ring_chunk32(EvalShared& sh, const RegOps& R, u3
         bool h0 = false, h1 = false, h2 = false, h3 = false;          // independent chains of comparisons
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
-            if (MASK & 1u) { h0 |= R.aA[j] == t_add; h1 |= R.aA[j + 1] == t_add; }
-            if (MASK & 2u) { h2 |= R.aA[j] == t_sub; h3 |= R.aA[j + 1] == t_sub; }
-            if (MASK & 4u) { h0 |= R.aA[j] * b == tp; h3 |= R.aA[j + 1] * b == tp; }
+            if (MASK & 1u) { h0 |= aA[j] == t_add; h1 |= aA[j + 1] == t_add; }
+            if (MASK & 2u) { h2 |= aA[j] == t_sub; h3 |= aA[j + 1] == t_sub; }
+            if (MASK & 4u) { h0 |= aA[j] * b == tp; h3 |= aA[j + 1] * b == tp; }
         }
-        const bool hit = h0 | h1 | h2 | h3;
-        if (__any_sync(0xffffffffu, hit)) {
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
                 if (!((alive >> j) & 1u)) continue;
                 const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-                if ((MASK & 1u) && R.aA[j] == t_add) push_hit(sh, idx, (u32)s, opi[XP_OP_ADD]);
-                if ((MASK & 2u) && R.aA[j] == t_sub) push_hit(sh, idx, (u32)s, opi[XP_OP_SUB]);
-                if ((MASK & 4u) && R.aA[j] * b == tp) push_hit(sh, idx, (u32)s, opi[XP_OP_MUL]);
+                if ((MASK & 1u) && aA[j] == t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
+                if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
+                if ((MASK & 4u) && aA[j] * b == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
             }
         }
     }
@@ -489,29 +495,36 @@ __device__ __forceinline__ void ring_chunk32(EvalShared& sh, const RegOps& R, u3
 // |remainder| against |target| (tabs) -- still a necessary condition, and the signs are settled
 // by the exact check.  SIGNED = true: signed results times A against tp.
 template <u32 MASK, bool SWAP, bool SIGNED>
-__device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32 alive, u32 A, u32 tp, u32 tabs,
-                                            int s0, int s1, const u32 (&opi)[5]) {
+__device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, u32 tabs,
+                                      int s0, int s1, u32 opip) {
+    u32 ua[kNA], am[kNA], ash[kNA], ac[kNA];
+#pragma unroll
+    for (int j = 0; j < kNA; ++j) {
+        ua[j] = Rm->ua[j];
+        if (SWAP) { am[j] = Rm->am[j]; ash[j] = Rm->ash[j]; ac[j] = Rm->ac[j]; }
+    }
+    const u32 neg = Rm->neg;
     for (int s = s0; s < s1; ++s) {
         const BcEntry e = sh.bc[s];
         const u32 ub = abs_u32((i32)e.lo);
         const u32 sb = (u32)((i32)e.lo >> 31);
         if (!SWAP && ub == 0u) continue;                              // zero divisor: invalid
         const u32 bm = e.mag, bsh = (e.meta >> 16) - 1u;
-        // magnitudes of quotient and remainder for register operand j; UNIT: the divisor is +-1
+        // magnitudes of quotient and remainder for register operand j; unit: the divisor is +-1
         auto test = [&](int j, bool unit, bool& hq, bool& hr) {
             u32 qu, ru;
             if (SWAP) {
-                qu = (__umulhi(ub, R.am[j]) >> R.ash[j]) + (ub & R.ac[j]);
-                ru = ub - qu * R.ua[j];
+                qu = (__umulhi(ub, am[j]) >> ash[j]) + (ub & ac[j]);
+                ru = ub - qu * ua[j];
             } else if (unit) {
-                qu = R.ua[j];
+                qu = ua[j];
                 ru = 0u;
             } else {
-                qu = __umulhi(R.ua[j], bm) >> bsh;
-                ru = R.ua[j] - qu * ub;
+                qu = __umulhi(ua[j], bm) >> bsh;
+                ru = ua[j] - qu * ub;
             }
             if (SIGNED) {
-                const u32 sa = (u32)((i32)(R.neg << (31 - j)) >> 31);
+                const u32 sa = (u32)((i32)(neg << (31 - j)) >> 31);
                 const u32 sq = sa ^ sb, sr = SWAP ? sb : sa;          // signs of quotient / remainder
                 hq = (((qu ^ sq) - sq) * A) == tp;
                 hr = (((ru ^ sr) - sr) * A) == tp;
@@ -521,7 +534,8 @@ __device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32
             }
         };
         bool h0 = false, h1 = false, h2 = false, h3 = false;
-        if (!SWAP && ub == 1u) {
+        const bool unit = !SWAP && ub == 1u;
+        if (unit) {
 #pragma unroll
             for (int j = 0; j < kNA; j += 2) {
                 bool q0, r0, q1, r1;
@@ -544,12 +558,12 @@ __device__ __forceinline__ void div_chunk32(EvalShared& sh, const RegOps& R, u32
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
                 // register operands that are invalid, or (SWAP) zero divisors, are dropped here
-                if (!((alive >> j) & 1u) || (SWAP && R.ua[j] == 0u)) continue;
+                if (!((alive >> j) & 1u) || (SWAP && ua[j] == 0u)) continue;
                 bool hq, hr;
-                test(j, !SWAP && ub == 1u, hq, hr);
+                test(j, unit, hq, hr);
                 const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-                if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, opi[XP_OP_DIV]);
-                if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, opi[XP_OP_MOD]);
+                if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
+                if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
             }
         }
     }
@@ -609,9 +623,8 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     const int nb = (int)sh.bc_n;
     const bool tile_wide = sh.tile_wide != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
-    u32 opi[5] = {0, 0, 0, 0, 0};
-    u32 mask = 0;
-    for (int o = 0; o < seg.n_ops; ++o) { opi[seg.op[o]] = (u32)o; mask |= 1u << seg.op[o]; }
+    u32 opip = 0, mask = 0;
+    for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * seg.op[o]); mask |= 1u << seg.op[o]; }
 
     const u32 A = (u32)A64, tp = (u32)tq;
     // With A == 1 a quotient or remainder of int32 operands can only equal a target of
@@ -642,14 +655,14 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_chunk32<M, SWAP>(sh, R, alv, A, tp, s0, s1, opi); break;
+#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, A, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
         }
         if (A == 1u && !t_small) return;                 // no int32 quotient or remainder can be the target
         switch (((mask >> 3) & 3u) | (A != 1u ? 4u : 0u)) {
-#define XP_DIV(C, M, SG) case C: div_chunk32<M, SWAP, SG>(sh, R, alv, A, tp, tabs, s0, s1, opi); break;
+#define XP_DIV(C, M, SG) case C: div_pass<M, SWAP, SG>(sh, &R, alv, A, tp, tabs, s0, s1, opip); break;
             XP_DIV(1u, 1u, false) XP_DIV(2u, 2u, false) XP_DIV(3u, 3u, false)
             XP_DIV(5u, 1u, true) XP_DIV(6u, 2u, true) XP_DIV(7u, 3u, true)
 #undef XP_DIV
