@@ -150,7 +150,7 @@ struct EvalShared {
     u64 warp_evals[kThreads / 32];
     // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
     // dropped), the reciprocal of each as a divisor, and the queue of filter hits
-    u32 bc_n;
+    u32 bc_n, bc_nspecial;       // general operands fill slots from 0 up, those of magnitude <= 1 from the top down
     u32 q_n, q_overflow;
     i32 tile_wide;               // some operand of the tile does not fit int32
     BcEntry bc[kBcTile];
@@ -464,27 +464,45 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     u32 aA[kNA];
 #pragma unroll
     for (int j = 0; j < kNA; ++j) aA[j] = Rm->aA[j];
-    for (int s = s0; s < s1; ++s) {
+    // comparisons of all register operands with broadcast operand s, OR-ed into four chains
+    auto scan = [&](int s, bool& h0, bool& h1, bool& h2, bool& h3) {
         const u32 b = sh.bc[s].lo;
         const u32 bA = b * A;
         const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
-        bool h0 = false, h1 = false, h2 = false, h3 = false;          // independent chains of comparisons
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
             if (MASK & 1u) { h0 |= aA[j] == t_add; h1 |= aA[j + 1] == t_add; }
             if (MASK & 2u) { h2 |= aA[j] == t_sub; h3 |= aA[j + 1] == t_sub; }
             if (MASK & 4u) { h0 |= aA[j] * b == tp; h3 |= aA[j + 1] * b == tp; }
         }
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
+    };
+    // the rare path: which candidates of broadcast operand s hit
+    auto resolve = [&](int s) {
+        const u32 b = sh.bc[s].lo;
+        const u32 bA = b * A;
+        const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
 #pragma unroll
-            for (int j = 0; j < kNA; ++j) {
-                if (!((alive >> j) & 1u)) continue;
-                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-                if ((MASK & 1u) && aA[j] == t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
-                if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
-                if ((MASK & 4u) && aA[j] * b == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
-            }
+        for (int j = 0; j < kNA; ++j) {
+            if (!((alive >> j) & 1u)) continue;
+            const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
+            if ((MASK & 1u) && aA[j] == t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
+            if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
+            if ((MASK & 4u) && aA[j] * b == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
         }
+    };
+    int s = s0;
+    for (; s + 4 <= s1; s += 4) {                       // one warp vote per four broadcast operands
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+        scan(s, h0, h1, h2, h3);
+        scan(s + 1, h0, h1, h2, h3);
+        scan(s + 2, h0, h1, h2, h3);
+        scan(s + 3, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(s); resolve(s + 1); resolve(s + 2); resolve(s + 3); }
+    }
+    for (; s < s1; ++s) {
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+        scan(s, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(s);
     }
 }
 
@@ -494,7 +512,9 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
 // SIGNED = false (context factor A == 1): only magnitudes are compared, |quotient| or
 // |remainder| against |target| (tabs) -- still a necessary condition, and the signs are settled
 // by the exact check.  SIGNED = true: signed results times A against tp.
-template <u32 MASK, bool SWAP, bool SIGNED>
+// SPECIAL (only without SWAP): the slots hold the divisors 0 and +-1, which the reciprocal
+// form does not cover: 0 is skipped (invalid), +-1 gives |quotient| = |dividend|, remainder 0.
+template <u32 MASK, bool SWAP, bool SIGNED, bool SPECIAL>
 __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, u32 tabs,
                                       int s0, int s1, u32 opip) {
     u32 ua[kNA], am[kNA], ash[kNA], ac[kNA];
@@ -504,68 +524,67 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
         if (SWAP) { am[j] = Rm->am[j]; ash[j] = Rm->ash[j]; ac[j] = Rm->ac[j]; }
     }
     const u32 neg = Rm->neg;
-    for (int s = s0; s < s1; ++s) {
-        const BcEntry e = sh.bc[s];
+    // hits of register operand j against broadcast entry e (quotient, remainder)
+    auto test = [&](const BcEntry& e, int j, bool& hq, bool& hr) {
         const u32 ub = abs_u32((i32)e.lo);
-        const u32 sb = (u32)((i32)e.lo >> 31);
-        if (!SWAP && ub == 0u) continue;                              // zero divisor: invalid
-        const u32 bm = e.mag, bsh = (e.meta >> 16) - 1u;
-        // magnitudes of quotient and remainder for register operand j; unit: the divisor is +-1
-        auto test = [&](int j, bool unit, bool& hq, bool& hr) {
-            u32 qu, ru;
-            if (SWAP) {
-                qu = (__umulhi(ub, am[j]) >> ash[j]) + (ub & ac[j]);
-                ru = ub - qu * ua[j];
-            } else if (unit) {
-                qu = ua[j];
-                ru = 0u;
-            } else {
-                qu = __umulhi(ua[j], bm) >> bsh;
-                ru = ua[j] - qu * ub;
-            }
-            if (SIGNED) {
-                const u32 sa = (u32)((i32)(neg << (31 - j)) >> 31);
-                const u32 sq = sa ^ sb, sr = SWAP ? sb : sa;          // signs of quotient / remainder
-                hq = (((qu ^ sq) - sq) * A) == tp;
-                hr = (((ru ^ sr) - sr) * A) == tp;
-            } else {
-                hq = qu == tabs;
-                hr = ru == tabs;
-            }
-        };
-        bool h0 = false, h1 = false, h2 = false, h3 = false;
-        const bool unit = !SWAP && ub == 1u;
-        if (unit) {
-#pragma unroll
-            for (int j = 0; j < kNA; j += 2) {
-                bool q0, r0, q1, r1;
-                test(j, true, q0, r0);
-                test(j + 1, true, q1, r1);
-                if (MASK & 1u) { h0 |= q0; h1 |= q1; }
-                if (MASK & 2u) { h2 |= r0; h3 |= r1; }
-            }
+        u32 qu, ru;
+        if (SWAP) {
+            qu = (__umulhi(ub, am[j]) >> ash[j]) + (ub & ac[j]);
+            ru = ub - qu * ua[j];
+        } else if (SPECIAL) {
+            qu = ua[j];
+            ru = 0u;
         } else {
-#pragma unroll
-            for (int j = 0; j < kNA; j += 2) {
-                bool q0, r0, q1, r1;
-                test(j, false, q0, r0);
-                test(j + 1, false, q1, r1);
-                if (MASK & 1u) { h0 |= q0; h1 |= q1; }
-                if (MASK & 2u) { h2 |= r0; h3 |= r1; }
-            }
+            qu = __umulhi(ua[j], e.mag) >> ((e.meta >> 16) - 1u);
+            ru = ua[j] - qu * ub;
         }
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
-#pragma unroll
-            for (int j = 0; j < kNA; ++j) {
-                // register operands that are invalid, or (SWAP) zero divisors, are dropped here
-                if (!((alive >> j) & 1u) || (SWAP && ua[j] == 0u)) continue;
-                bool hq, hr;
-                test(j, unit, hq, hr);
-                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-                if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
-                if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
-            }
+        if (SIGNED) {
+            const u32 sb = (u32)((i32)e.lo >> 31);
+            const u32 sa = (u32)((i32)(neg << (31 - j)) >> 31);
+            const u32 sq = sa ^ sb, sr = SWAP ? sb : sa;              // signs of quotient / remainder
+            hq = (((qu ^ sq) - sq) * A) == tp;
+            hr = (((ru ^ sr) - sr) * A) == tp;
+        } else {
+            hq = qu == tabs;
+            hr = ru == tabs;
         }
+    };
+    auto scan = [&](const BcEntry& e, bool& h0, bool& h1, bool& h2, bool& h3) {
+#pragma unroll
+        for (int j = 0; j < kNA; j += 2) {
+            bool q0, r0, q1, r1;
+            test(e, j, q0, r0);
+            test(e, j + 1, q1, r1);
+            if (MASK & 1u) { h0 |= q0; h1 |= q1; }
+            if (MASK & 2u) { h2 |= r0; h3 |= r1; }
+        }
+    };
+    auto resolve = [&](const BcEntry& e, int s) {
+        if (SPECIAL && e.lo == 0u) return;
+#pragma unroll
+        for (int j = 0; j < kNA; ++j) {
+            // register operands that are invalid, or (SWAP) zero divisors, are dropped here
+            if (!((alive >> j) & 1u) || (SWAP && ua[j] == 0u)) continue;
+            bool hq, hr;
+            test(e, j, hq, hr);
+            const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
+            if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
+            if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
+        }
+    };
+    int s = s0;
+    for (; s + 2 <= s1; s += 2) {                       // one warp vote per two broadcast operands
+        const BcEntry e0 = sh.bc[s], e1 = sh.bc[s + 1];
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+        scan(e0, h0, h1, h2, h3);
+        scan(e1, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(e0, s); resolve(e1, s + 1); }
+    }
+    for (; s < s1; ++s) {
+        const BcEntry e0 = sh.bc[s];
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+        scan(e0, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(e0, s);
     }
 }
 
@@ -649,7 +668,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
-    auto run = [&](int s0, int s1, u32 alv) {
+    auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide) {
             wide_chunk(sh, a64, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
             return;
@@ -662,7 +681,8 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
         }
         if (A == 1u && !t_small) return;                 // no int32 quotient or remainder can be the target
         switch (((mask >> 3) & 3u) | (A != 1u ? 4u : 0u)) {
-#define XP_DIV(C, M, SG) case C: div_pass<M, SWAP, SG>(sh, &R, alv, A, tp, tabs, s0, s1, opip); break;
+#define XP_DIV(C, M, SG) case C: if (special && !SWAP) div_pass<M, SWAP, SG, true>(sh, &R, alv, A, tp, tabs, s0, s1, opip); \
+                         else div_pass<M, SWAP, SG, false>(sh, &R, alv, A, tp, tabs, s0, s1, opip); break;
             XP_DIV(1u, 1u, false) XP_DIV(2u, 2u, false) XP_DIV(3u, 3u, false)
             XP_DIV(5u, 1u, true) XP_DIV(6u, 2u, true) XP_DIV(7u, 3u, true)
 #undef XP_DIV
@@ -670,31 +690,37 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
         }
     };
 
+    // The broadcast operands sit in two runs of slots: the general ones from slot 0 up, the
+    // ones of magnitude <= 1 (special as divisors) from the last slot down.
+    const int n_special = (int)sh.bc_nspecial;
     u32 q_start = 0;                                    // queue length when the current chunk began
-    for (int s0 = 0; s0 < nb; s0 += kChunkB) {
-        const int s1 = s0 + kChunkB < nb ? s0 + kChunkB : nb;
-        run(s0, s1, alive);
-        __syncthreads();
-        const u32 qn = sh.q_n;
-        const bool overflow = sh.q_overflow != 0;
-        __syncthreads();
-        if (overflow) {
-            // More hits than the queue holds (a spec that most candidates satisfy at probe 0).
-            // Forget this chunk's hits, empty the queue, and redo the chunk one broadcast slot
-            // and one register operand at a time: at most kThreads * 5 hits per step.
-            if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
-            drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
-            for (int s = s0; s < s1; ++s)
-                for (int j = 0; j < kNA; ++j) {
-                    run(s, s + 1, alive & (1u << j));
-                    drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
-                }
-            q_start = 0;
-        } else if (qn > (u32)(kQueueCap / 2)) {
-            drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
-            q_start = 0;
-        } else {
-            q_start = qn;
+    for (int part = 0; part < 2; ++part) {
+        const int lo = part == 0 ? 0 : kBcTile - n_special, hi = part == 0 ? nb : kBcTile;
+        for (int s0 = lo; s0 < hi; s0 += kChunkB) {
+            const int s1 = s0 + kChunkB < hi ? s0 + kChunkB : hi;
+            run(s0, s1, alive, part == 1);
+            __syncthreads();
+            const u32 qn = sh.q_n;
+            const bool overflow = sh.q_overflow != 0;
+            __syncthreads();
+            if (overflow) {
+                // More hits than the queue holds (a spec that most candidates satisfy at probe 0).
+                // Forget this chunk's hits, empty the queue, and redo the chunk one broadcast slot
+                // and one register operand at a time: at most kThreads * 5 hits per step.
+                if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
+                drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                for (int s = s0; s < s1; ++s)
+                    for (int j = 0; j < kNA; ++j) {
+                        run(s, s + 1, alive & (1u << j), part == 1);
+                        drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                    }
+                q_start = 0;
+            } else if (qn > (u32)(kQueueCap / 2)) {
+                drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                q_start = 0;
+            } else {
+                q_start = qn;
+            }
         }
     }
     drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
@@ -714,7 +740,7 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
     const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
     const bool swap = seg.swap != 0;
 
-    if (threadIdx.x == 0) { sh.bc_n = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
+    if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
     __syncthreads();
 
     // operand values at probe 0
@@ -722,7 +748,8 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
     for (int i = threadIdx.x; i < n_bc; i += kThreads) {
         i64 v;
         if (!operand_value(g, hole, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
-        const u32 slot = atomicAdd(&sh.bc_n, 1u);
+        const bool special = v >= -1 && v <= 1;
+        const u32 slot = special ? (u32)kBcTile - 1u - atomicAdd(&sh.bc_nspecial, 1u) : atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
         u32 m = 0, s = 0;
