@@ -103,6 +103,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4"],
+                    help="profiling aid: time another config's instance instead (the bench line is config2's)")
     ap.add_argument("--window", type=int, default=0,
                     help="profiling aid: search only the first WINDOW ranks of size 7 (a small case of the same kernel)")
     args = ap.parse_args()
@@ -112,7 +114,7 @@ def main():
 
     import torch
     import paper_2505_02146_b200 as xp
-    from xp_instances import config2
+    from xp_instances import config2, config3, config4
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -126,7 +128,7 @@ def main():
     xp.load()
 
     # Independent problems shard with no data-path exchange: rank r searches the instance of seed r.
-    sk = config2(rank)
+    sk = {"config2": config2, "config3": config3, "config4": config4}[args.workload](rank)
     gr = xp.xp_grammar_create(sk.grammar)
     ls = xp.xp_sketch_load(gr, sk)
     stream = torch.cuda.current_stream()
@@ -200,7 +202,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
         "ms_per_step": dev_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD if not args.window else WORKLOAD + f"_first_{args.window}_ranks_of_size7",
+        "config": {"workload": (WORKLOAD if args.workload == "config2" else args.workload) +
+                               (f"_first_{args.window}_ranks_of_size7" if args.window else ""),
                    "candidates_per_step": cand, "domain_points": sk.n_points,
                    "nominal_evals_per_step": cand * sk.n_points, "l2": "flushed between steps (256 MiB write)",
                    "time_to_solution_ms": res.total_ms, "kernel_ms_per_step": kern_ms / args.steps,
@@ -215,7 +218,7 @@ def main():
                      "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
                      "model": "operation + comparison per candidate-point evaluation (see DESIGN.md)"},
     }
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.workload == "config2":
         e, dt, sample = oracle_sample(0, ORACLE_SAMPLE_RANKS)
         out["cpu_baseline"] = {"value": e / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                                "seconds": dt, "host_cores_present": os.cpu_count()}
