@@ -25,7 +25,7 @@ constexpr int kThreads = 256;        // threads per CTA of the evaluation kernel
 constexpr int kLinearChunk = kThreads * 4;   // ranks per linear ticket
 constexpr int kNA = 8;                // tile tickets: register-side operands per thread
 constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
-constexpr int kBcTile = 1024;         // broadcast-side operands per tile
+constexpr int kBcTile = 512;          // broadcast-side operands per tile
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 

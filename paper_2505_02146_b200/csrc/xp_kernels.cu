@@ -124,13 +124,23 @@ __global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
 
 constexpr int kLinearPerThread = kLinearChunk / kThreads; // ranks per thread per linear ticket
 constexpr int kMaxSurvivors = kLinearChunk;
-constexpr int kQueueCap = 4096;                           // filter hits waiting for the exact probe check
-constexpr int kChunkB = 32;                               // broadcast operands between block-wide queue checks
+constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check
+constexpr int kChunkB = 128;                              // broadcast operands between block-wide queue checks
 static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
+static_assert(kThreads * 5 <= kQueueCap / 2, "one replay step must fit the free half of the queue");
 
-// A broadcast-side operand of a tile: its value at probe 0 (lo/hi words), the reciprocal
-// multiplier of |value| as a divisor, and meta = index inside the tile | reciprocal shift << 16.
-struct __align__(16) BcEntry { u32 lo, hi, mag, meta; };
+// A broadcast-side operand of a tile, as three 16-byte records so that each loop fetches what
+// it needs with one shared-memory load.  All per-operand arithmetic that does not depend on
+// the register operand is done once, when the tile is filled:
+//   BcRing: the values a register operand (times A) must equal for + and -, and the mask and
+//           value for *:  (A*a) * b == tp (mod 2^32)  <=>  ((A*a) & mask) == tm, where
+//           b = 2^k * o (o odd), mask = 2^(32-k) - 1, tm = (tp >> k) * o^-1 & mask, provided the
+//           low k bits of tp are zero (else tm lies outside the mask and nothing matches);
+//   BcDiv:  magnitudes for / and %, see div_pass;
+//   BcMeta: the value itself, and meta = index inside the tile | ctz(|value|) << 16.
+struct __align__(16) BcRing { u32 t_add, t_sub, mul_mask, mul_tm; };
+struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
+struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
 struct EvalShared {
     u64 ticket;
@@ -153,7 +163,9 @@ struct EvalShared {
     u32 bc_n, bc_nspecial;       // general operands fill slots from 0 up, those of magnitude <= 1 from the top down
     u32 q_n, q_overflow;
     i32 tile_wide;               // some operand of the tile does not fit int32
-    BcEntry bc[kBcTile];
+    BcRing bc_ring[kBcTile];
+    BcDiv bc_div[kBcTile];
+    BcMeta bc_meta[kBcTile];
     u32 queue[kQueueCap];        // reg index | broadcast slot << 11 | op index << 21
 };
 
@@ -295,26 +307,11 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const SketchDev* sk, 
 //     are exact);
 //   * an affine context  A*h + B  is folded into the operands (ring operators) or applied to
 //     the quotient / remainder;
-//   * division by a broadcast operand uses a precomputed reciprocal: for 1 <= d < 2^31,
-//     s = ceil(log2 d), m = floor(2^(31+s) / d) + 1 < 2^32, and floor(n / d) = (n * m) >> (31+s)
-//     for every 0 <= n < 2^31.
-
-__device__ __forceinline__ void reciprocal_u31(u32 d, u32& m, u32& s) {
-    s = d <= 1 ? 0u : 32u - (u32)__clz((int)(d - 1));
-    m = (u32)((1ull << (31 + s)) / d) + 1u;
-}
-
-__device__ __forceinline__ u32 div_u31(u32 n, u32 m, u32 s) { return (u32)(((u64)n * m) >> (31 + s)); }
+//   * everything that depends on one operand only is computed when the tile is filled, so a
+//     candidate costs one comparison for + and -, a mask and a comparison for *, and for / and %
+//     a range test and a divisibility test on magnitudes (see ring_pass and div_pass).
 
 __device__ __forceinline__ u32 abs_u32(i32 x) { return x < 0 ? 0u - (u32)x : (u32)x; }
-
-// Truncating signed quotient of int32 operands whose magnitudes are below 2^31, through the
-// reciprocal (m, s) of |d|.
-__device__ __forceinline__ i32 quot_i32(i32 n, i32 d, u32 m, u32 s) {
-    const u32 q = div_u31(abs_u32(n), m, s);
-    const i32 sg = (n ^ d) >> 31;
-    return ((i32)q ^ sg) - sg;
-}
 
 __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, u32 opi) {
     const u32 at = atomicAdd(&sh.q_n, 1u);
@@ -438,153 +435,172 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int 
     }
 }
 
+// Inverse of an odd number modulo 2^32 (Newton: each step doubles the number of correct bits).
+__device__ __forceinline__ u32 inv_odd(u32 o) {
+    u32 x = o;                       // correct to 3 bits
+    x *= 2u - o * x; x *= 2u - o * x; x *= 2u - o * x; x *= 2u - o * x;
+    return x;
+}
+
+__device__ __forceinline__ u32 rotr32(u32 x, u32 k) { return __funnelshift_r(x, x, k); }
+
 // The register-side operands of a tile as the 32-bit loops use them.
 struct RegOps {
     u32 aA[kNA];     // A * value (the affine context's factor folded in)
     u32 ua[kNA];     // |value|
     u32 neg;         // bit j: value j is negative
-    u32 am[kNA];     // SWAP: reciprocal multiplier of |value| as a divisor (0 when |value| <= 1)
-    u32 ash[kNA];    // SWAP: reciprocal shift - 1
-    u32 ac[kNA];     // SWAP: all ones when |value| == 1 (the quotient is the dividend)
+    // register operand as DIVISOR (SWAP), magnitudes only:
+    u32 low[kNA];    // tabs * |value| (0x80000000 when that is 2^31 or more: never matches)
+    u32 inv[kNA];    // inverse mod 2^32 of the odd part of |value|
+    u32 kk[kNA];     // number of trailing zero bits of |value|
+    u32 cc[kNA];     // floor((2^32-1) / |value|), or 0 when the remainder tabs is impossible
     u32 alive;       // bit j: operand j exists and is valid at probe 0
 };
 
-// The two loops below are separate (not inlined) functions on purpose: each copies just the
+// The loops below are separate (not inlined) functions on purpose: each copies just the
 // operand arrays it needs from the tile's RegOps into registers and runs with a small live
 // set, instead of sharing one large frame with the rest of the kernel.
 // `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
 
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
-// tp = low 32 bits of (target - B).  MASK: bit0 +, bit1 -, bit2 *.  Per broadcast operand b
-// the comparisons are brought to the register operand's side once:
+// MASK: bit0 +, bit1 -, bit2 *.  The comparisons were brought to the register operand's side
+// when the tile was filled (tp = low 32 bits of target - B):
 //   A*(a + b) == tp  <=>  A*a == tp - A*b;    A*(a - b) == tp  <=>  A*a == tp + A*b;
-//   A*(b - a) == tp  <=>  A*a == A*b - tp;    A*(a * b) == tp  <=>  (A*a) * b == tp.
-template <u32 MASK, bool SWAP>
-__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, int s0, int s1, u32 opip) {
+//   A*(b - a) == tp  <=>  A*a == A*b - tp;    A*(a * b) == tp  <=>  ((A*a) & mask) == tm.
+template <u32 MASK>
+__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, int s0, int s1, u32 opip) {
     u32 aA[kNA];
 #pragma unroll
     for (int j = 0; j < kNA; ++j) aA[j] = Rm->aA[j];
-    // comparisons of all register operands with broadcast operand s, OR-ed into four chains
-    auto scan = [&](int s, bool& h0, bool& h1, bool& h2, bool& h3) {
-        const u32 b = sh.bc[s].lo;
-        const u32 bA = b * A;
-        const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
+    auto scan = [&](const BcRing& e, bool& h0, bool& h1, bool& h2, bool& h3) {
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
-            if (MASK & 1u) { h0 |= aA[j] == t_add; h1 |= aA[j + 1] == t_add; }
-            if (MASK & 2u) { h2 |= aA[j] == t_sub; h3 |= aA[j + 1] == t_sub; }
-            if (MASK & 4u) { h0 |= aA[j] * b == tp; h3 |= aA[j + 1] * b == tp; }
+            if (MASK & 1u) { h0 |= aA[j] == e.t_add; h1 |= aA[j + 1] == e.t_add; }
+            if (MASK & 2u) { h2 |= aA[j] == e.t_sub; h3 |= aA[j + 1] == e.t_sub; }
+            if (MASK & 4u) { h1 |= (aA[j] & e.mul_mask) == e.mul_tm; h2 |= (aA[j + 1] & e.mul_mask) == e.mul_tm; }
         }
     };
-    // the rare path: which candidates of broadcast operand s hit
-    auto resolve = [&](int s) {
-        const u32 b = sh.bc[s].lo;
-        const u32 bA = b * A;
-        const u32 t_add = tp - bA, t_sub = SWAP ? bA - tp : tp + bA;
+    auto resolve = [&](int s) {                          // the rare path: which candidates hit
+        const BcRing e = sh.bc_ring[s];
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
             const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-            if ((MASK & 1u) && aA[j] == t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
-            if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
-            if ((MASK & 4u) && aA[j] * b == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
+            if ((MASK & 1u) && aA[j] == e.t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
+            if ((MASK & 2u) && aA[j] == e.t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
+            if ((MASK & 4u) && (aA[j] & e.mul_mask) == e.mul_tm) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
         }
     };
     int s = s0;
     for (; s + 4 <= s1; s += 4) {                       // one warp vote per four broadcast operands
-        bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(s, h0, h1, h2, h3);
-        scan(s + 1, h0, h1, h2, h3);
-        scan(s + 2, h0, h1, h2, h3);
-        scan(s + 3, h0, h1, h2, h3);
+        const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
+        bool h0 = false, h1 = false, h2 = false, h3 = false;      // independent chains of comparisons
+        scan(e0, h0, h1, h2, h3);
+        scan(e1, h0, h1, h2, h3);
+        scan(e2, h0, h1, h2, h3);
+        scan(e3, h0, h1, h2, h3);
         if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(s); resolve(s + 1); resolve(s + 2); resolve(s + 3); }
     }
     for (; s < s1; ++s) {
+        const BcRing e0 = sh.bc_ring[s];
         bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(s, h0, h1, h2, h3);
+        scan(e0, h0, h1, h2, h3);
         if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(s);
     }
 }
 
-// / and % on int32-exact operands.  MASK: bit0 /, bit1 %.
-// SWAP = false: register operand / broadcast operand (reciprocal from shared memory);
-// SWAP = true: broadcast operand / register operand (reciprocals in registers).
-// SIGNED = false (context factor A == 1): only magnitudes are compared, |quotient| or
-// |remainder| against |target| (tabs) -- still a necessary condition, and the signs are settled
-// by the exact check.  SIGNED = true: signed results times A against tp.
-// SPECIAL (only without SWAP): the slots hold the divisors 0 and +-1, which the reciprocal
-// form does not cover: 0 is skipped (invalid), +-1 gives |quotient| = |dividend|, remainder 0.
-template <u32 MASK, bool SWAP, bool SIGNED, bool SPECIAL>
-__device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, u32 tabs,
-                                      int s0, int s1, u32 opip) {
-    u32 ua[kNA], am[kNA], ash[kNA], ac[kNA];
+// / and % on int32-exact operands with the context factor A == 1.  MASK: bit0 /, bit1 %.
+// Only magnitudes are compared (|quotient| or |remainder| against tabs = |target|): still a
+// necessary condition, the signs are settled by the exact check.  With n the dividend's and d
+// the divisor's magnitude:
+//   floor(n / d) == tabs  <=>  n - tabs*d < d            (unsigned; tabs*d precomputed)
+//   n mod d == tabs       <=>  d divides n - tabs (and tabs < d, n >= tabs); for d = 2^k * o,
+//                              d | x  <=>  rotr(x * o^-1, k) <= floor((2^32-1) / d).
+// SWAP = false: register operand / broadcast operand; SWAP = true: broadcast / register.
+// SPECIAL (without SWAP only): the slots hold the divisors 0 and +-1: 0 is skipped (invalid),
+// +-1 gives |quotient| = |dividend| and remainder 0.
+template <u32 MASK, bool SWAP, bool SPECIAL>
+__device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tabs, int s0, int s1, u32 opip) {
+    u32 ua[kNA], xa[kNA], low[kNA], inv[kNA], kk[kNA], cc[kNA];
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
         ua[j] = Rm->ua[j];
-        if (SWAP) { am[j] = Rm->am[j]; ash[j] = Rm->ash[j]; ac[j] = Rm->ac[j]; }
+        xa[j] = ua[j] >= tabs ? ua[j] - tabs : 1u;      // 1 is a multiple of no divisor >= 2
+        if (SWAP) { low[j] = Rm->low[j]; inv[j] = Rm->inv[j]; kk[j] = Rm->kk[j]; cc[j] = Rm->cc[j]; }
     }
-    const u32 neg = Rm->neg;
     // hits of register operand j against broadcast entry e (quotient, remainder)
-    auto test = [&](const BcEntry& e, int j, bool& hq, bool& hr) {
-        const u32 ub = abs_u32((i32)e.lo);
-        u32 qu, ru;
-        if (SWAP) {
-            qu = (__umulhi(ub, am[j]) >> ash[j]) + (ub & ac[j]);
-            ru = ub - qu * ua[j];
+    auto test = [&](const BcDiv& e, u32 ek, int j, bool& hq, bool& hr) {
+        if (SWAP) {                 // e.ub: dividend magnitude; e.low: dividend - tabs (or 1)
+            hq = (e.ub - low[j]) < ua[j];
+            hr = rotr32(e.low * inv[j], kk[j]) <= cc[j];
         } else if (SPECIAL) {
-            qu = ua[j];
-            ru = 0u;
-        } else {
-            qu = __umulhi(ua[j], e.mag) >> ((e.meta >> 16) - 1u);
-            ru = ua[j] - qu * ub;
-        }
-        if (SIGNED) {
-            const u32 sb = (u32)((i32)e.lo >> 31);
-            const u32 sa = (u32)((i32)(neg << (31 - j)) >> 31);
-            const u32 sq = sa ^ sb, sr = SWAP ? sb : sa;              // signs of quotient / remainder
-            hq = (((qu ^ sq) - sq) * A) == tp;
-            hr = (((ru ^ sr) - sr) * A) == tp;
-        } else {
-            hq = qu == tabs;
-            hr = ru == tabs;
+            hq = e.ub == 1u && ua[j] == tabs;
+            hr = e.ub == 1u && tabs == 0u;
+        } else {                    // e.low: tabs * divisor (or never); e.ub: divisor magnitude
+            hq = (ua[j] - e.low) < e.ub;
+            hr = rotr32(xa[j] * e.inv, ek) <= e.cmax;
         }
     };
-    auto scan = [&](const BcEntry& e, bool& h0, bool& h1, bool& h2, bool& h3) {
+    auto scan = [&](const BcDiv& e, u32 ek, bool& h0, bool& h1, bool& h2, bool& h3) {
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
             bool q0, r0, q1, r1;
-            test(e, j, q0, r0);
-            test(e, j + 1, q1, r1);
+            test(e, ek, j, q0, r0);
+            test(e, ek, j + 1, q1, r1);
             if (MASK & 1u) { h0 |= q0; h1 |= q1; }
             if (MASK & 2u) { h2 |= r0; h3 |= r1; }
         }
     };
-    auto resolve = [&](const BcEntry& e, int s) {
-        if (SPECIAL && e.lo == 0u) return;
+    auto resolve = [&](const BcDiv& e, u32 ek, int s) {
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
             // register operands that are invalid, or (SWAP) zero divisors, are dropped here
             if (!((alive >> j) & 1u) || (SWAP && ua[j] == 0u)) continue;
             bool hq, hr;
-            test(e, j, hq, hr);
+            test(e, ek, j, hq, hr);
             const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
             if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
             if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
         }
     };
+    const bool need_k = !SWAP && !SPECIAL && (MASK & 2u);
     int s = s0;
     for (; s + 2 <= s1; s += 2) {                       // one warp vote per two broadcast operands
-        const BcEntry e0 = sh.bc[s], e1 = sh.bc[s + 1];
+        const BcDiv e0 = sh.bc_div[s], e1 = sh.bc_div[s + 1];
+        const u32 k0 = need_k ? sh.bc_meta[s].meta >> 16 : 0u, k1 = need_k ? sh.bc_meta[s + 1].meta >> 16 : 0u;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(e0, h0, h1, h2, h3);
-        scan(e1, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(e0, s); resolve(e1, s + 1); }
+        scan(e0, k0, h0, h1, h2, h3);
+        scan(e1, k1, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(e0, k0, s); resolve(e1, k1, s + 1); }
     }
     for (; s < s1; ++s) {
-        const BcEntry e0 = sh.bc[s];
+        const BcDiv e0 = sh.bc_div[s];
+        const u32 k0 = need_k ? sh.bc_meta[s].meta >> 16 : 0u;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(e0, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(e0, s);
+        scan(e0, k0, h0, h1, h2, h3);
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(e0, k0, s);
+    }
+}
+
+// / and % on int32-exact operands under a context factor A != 1: signed results times A are
+// compared with tp.  Plain 32-bit division; this form only serves sketches whose hole sits
+// under a multiplication (small searches).
+template <bool SWAP>
+__device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegOps* Rm, u32 alive, u32 mask, u32 A, u32 tp,
+                                             int s0, int s1, u32 opip) {
+    for (int s = s0; s < s1; ++s) {
+        const i32 b = (i32)sh.bc_meta[s].lo;
+        for (int j = 0; j < kNA; ++j) {
+            if (!((alive >> j) & 1u)) continue;
+            const i32 a = ((Rm->neg >> j) & 1u) ? (i32)(0u - Rm->ua[j]) : (i32)Rm->ua[j];
+            const i32 n = SWAP ? b : a, d = SWAP ? a : b;
+            if (d == 0) continue;
+            const i32 q = n / d;                         // magnitudes are below 2^31: no overflow case
+            const u32 r = (u32)n - (u32)q * (u32)d;
+            const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
+            if ((mask & 8u) && (u32)q * A == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
+            if ((mask & 16u) && r * A == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
+        }
     }
 }
 
@@ -592,7 +608,7 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
 __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive, bool swap, u64 A, u64 tq,
                                         int s0, int s1, int n_ops, const i32* ops) {
     for (int s = s0; s < s1; ++s) {
-        const i64 b = (i64)(((u64)sh.bc[s].hi << 32) | sh.bc[s].lo);
+        const i64 b = (i64)(((u64)sh.bc_meta[s].hi << 32) | sh.bc_meta[s].lo);
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
             for (int o = 0; o < n_ops; ++o) {
@@ -616,7 +632,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, co
         for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
             const u32 e = sh.queue[i];
             const u64 rr = reg_first + (e & 2047u);
-            const u64 br = bc_first + (sh.bc[(e >> 11) & 1023u].meta & 0xffffu);
+            const u64 br = bc_first + (sh.bc_meta[(e >> 11) & 1023u].meta & 0xffffu);
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
             const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
             if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
@@ -654,16 +670,20 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
     RegOps R;
     R.alive = alive;
     R.neg = 0;
-#pragma unroll
     for (int j = 0; j < kNA; ++j) {
         const i32 v = (i32)a64[j];
+        const u32 ua = abs_u32(v);
         R.aA[j] = (u32)v * A;
-        R.ua[j] = abs_u32(v);
+        R.ua[j] = ua;
         if (v < 0) R.neg |= 1u << j;
-        R.am[j] = 0; R.ash[j] = 0; R.ac[j] = 0;
-        if (SWAP && !tile_wide && (mask & 24u)) {
-            if (R.ua[j] == 1u) R.ac[j] = 0xffffffffu;
-            else if (R.ua[j] > 1u) { u32 m, sft; reciprocal_u31(R.ua[j], m, sft); R.am[j] = m; R.ash[j] = sft - 1u; }
+        R.low[j] = 0x80000000u; R.inv[j] = 1u; R.kk[j] = 0u; R.cc[j] = 0u;
+        if (SWAP && !tile_wide && (mask & 24u) && A == 1u && ua != 0u) {
+            const u64 lw = (u64)tabs * ua;
+            if (lw < (1ull << 31)) R.low[j] = (u32)lw;
+            const u32 k = (u32)__ffs((int)ua) - 1u;
+            R.kk[j] = k;
+            R.inv[j] = inv_odd(ua >> k);
+            R.cc[j] = tabs < ua ? 0xffffffffu / ua : 0u;
         }
     }
 
@@ -674,17 +694,18 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, A, tp, s0, s1, opip); break;
+#define XP_RING(M) case M: ring_pass<M>(sh, &R, alv, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
         }
-        if (A == 1u && !t_small) return;                 // no int32 quotient or remainder can be the target
-        switch (((mask >> 3) & 3u) | (A != 1u ? 4u : 0u)) {
-#define XP_DIV(C, M, SG) case C: if (special && !SWAP) div_pass<M, SWAP, SG, true>(sh, &R, alv, A, tp, tabs, s0, s1, opip); \
-                         else div_pass<M, SWAP, SG, false>(sh, &R, alv, A, tp, tabs, s0, s1, opip); break;
-            XP_DIV(1u, 1u, false) XP_DIV(2u, 2u, false) XP_DIV(3u, 3u, false)
-            XP_DIV(5u, 1u, true) XP_DIV(6u, 2u, true) XP_DIV(7u, 3u, true)
+        if (!(mask & 24u)) return;
+        if (A != 1u) { div_pass_signed<SWAP>(sh, &R, alv, mask, A, tp, s0, s1, opip); return; }
+        if (!t_small) return;                            // no int32 quotient or remainder can be the target
+        switch ((mask >> 3) & 3u) {
+#define XP_DIV(M) case M: if (special && !SWAP) div_pass<M, SWAP, true>(sh, &R, alv, tabs, s0, s1, opip); \
+                          else div_pass<M, SWAP, false>(sh, &R, alv, tabs, s0, s1, opip); break;
+            XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
 #undef XP_DIV
             default: break;
         }
@@ -743,7 +764,11 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
     if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
     __syncthreads();
 
-    // operand values at probe 0
+    // operand values at probe 0, with everything the loops need that depends on them alone
+    const u32 fA = (u32)hole->aff_A;
+    const u64 ftq = (u64)hole->probe_spec[0] - hole->aff_B;
+    const u32 ftp = (u32)ftq;
+    const u32 ftabs = (u32)((i64)ftq < 0 ? 0ull - ftq : ftq);
     bool wide = false;
     for (int i = threadIdx.x; i < n_bc; i += kThreads) {
         i64 v;
@@ -752,11 +777,35 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
         const u32 slot = special ? (u32)kBcTile - 1u - atomicAdd(&sh.bc_nspecial, 1u) : atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
-        u32 m = 0, s = 0;
-        if (fits && v != 0 && seg.has_div && !swap) reciprocal_u31(abs_u32((i32)v), m, s);
-        BcEntry e;
-        e.lo = (u32)(u64)v; e.hi = (u32)((u64)v >> 32); e.mag = m; e.meta = (u32)i | (s << 16);
-        sh.bc[slot] = e;
+        const u32 b = (u32)(u64)v, ub = abs_u32((i32)v);
+        const u32 k = ub ? (u32)__ffs((int)ub) - 1u : 0u;
+        const u32 io = ub ? inv_odd(ub >> k) : 1u;          // inverse of the odd part of |v|
+        BcMeta m;
+        m.lo = b; m.hi = (u32)((u64)v >> 32); m.meta = (u32)i | (k << 16); m.pad = 0;
+        sh.bc_meta[slot] = m;
+        // + and -: the value A*a must have; *: mask and value of A*a's low bits
+        BcRing r;
+        const u32 bA = b * fA;
+        r.t_add = ftp - bA;
+        r.t_sub = swap ? bA - ftp : ftp + bA;
+        if (ub == 0u) { r.mul_mask = 0u; r.mul_tm = ftp == 0u ? 0u : 1u; }
+        else {
+            r.mul_mask = 0xffffffffu >> k;
+            const bool feasible = k == 0u || (ftp << (32u - k)) == 0u;
+            const u32 io_signed = (i32)b < 0 ? 0u - io : io;  // b = 2^k * (+-o)
+            r.mul_tm = feasible ? ((ftp >> k) * io_signed) & r.mul_mask : 0xffffffffu;
+        }
+        sh.bc_ring[slot] = r;
+        // / and %: this operand as divisor (not swap) or as dividend (swap)
+        BcDiv d;
+        d.ub = ub; d.inv = io;
+        if (swap) { d.low = ub >= ftabs ? ub - ftabs : 1u; d.cmax = 0u; }
+        else {
+            const u64 lw = (u64)ftabs * ub;
+            d.low = lw < (1ull << 31) ? (u32)lw : 0x80000000u;
+            d.cmax = (ub != 0u && ftabs < ub) ? 0xffffffffu / ub : 0u;
+        }
+        sh.bc_div[slot] = d;
     }
     i64 a64[kNA];
     const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
