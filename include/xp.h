@@ -230,8 +230,8 @@ void xp_result_free(xp_result* r);
  * which the implicit device-wide synchronisation of cudaMalloc / cudaFree is not acceptable,
  * or a process that runs under a hard device-memory budget fixed before the first request.
  * xp_repair either takes a caller-allocated workspace or calls cudaMalloc itself, and it
- * creates CUDA events; this entry point does neither.  Its scratch (ticket counter, segment
- * table, accumulators) lives in a fixed array of XP_STATIC_SCRATCH_BYTES inside the library,
+ * creates CUDA events; this entry point does neither.  Its scratch (counters, segment table,
+ * accumulators, survivor queue) lives in a fixed array of XP_STATIC_SCRATCH_BYTES inside the library,
  * which every GPU that loads the library holds until the process exits.
  *
  *  - Inputs and outputs stay the caller's: the sketch (loaded earlier with xp_sketch_load,

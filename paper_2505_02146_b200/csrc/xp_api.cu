@@ -585,23 +585,33 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
     return XP_OK;
 }
 
-struct WsLayout { size_t ticket, segs, sketches, acc, total; };
+constexpr u32 kSurvCap = 65536;              // survivor queue entries of a call with its own workspace
+constexpr u32 kSurvCapStatic = 8192;         // ... of a call on the library's fixed scratch
 
-static WsLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc) {
-    WsLayout w;
-    w.ticket = 0;
+static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap) {
+    SearchLayout w;
     w.segs = 256;
     w.sketches = w.segs + align256(sizeof(SegDev) * (n_segs + 1));
     w.acc = w.sketches + align256(sizeof(SketchDev*) * (n_sketches + 1));
-    w.total = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
+    w.head = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
+    w.surv = w.head;
+    w.total = w.surv + align256(sizeof(SurvDev) * (size_t)surv_cap);
+    w.surv_cap = surv_cap;
     return w;
+}
+
+// Chunks of the whole-domain check that the largest domain among the sketches needs.
+static u32 max_chunks_of(const xp_sketch* const* sk, size_t n) {
+    i64 most = 0;
+    for (size_t i = 0; i < n; ++i) most = sk[i]->n_points > most ? sk[i]->n_points : most;
+    return (u32)((most + kVerifyChunk - 1) / kVerifyChunk);
 }
 
 extern "C" size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts) {
     if (!sketches || n == 0) return 0;
     Plan plan;
     if (build_plan(sketches, n, opts ? opts : &kDefaultOpts, &plan) != XP_OK) return 0;
-    return ws_layout(plan.segs.size(), n, plan.acc.size()).total;
+    return ws_layout(plan.segs.size(), n, plan.acc.size(), kSurvCap).total;
 }
 
 extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
@@ -617,7 +627,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
-    const WsLayout w = ws_layout(plan.segs.size(), n, plan.acc.size());
+    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), kSurvCap);
     char* ws = (char*)o->workspace;
     bool own_ws = false;
     if (ws) {
@@ -626,7 +636,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
         XP_CUDA(cudaMalloc((void**)&ws, w.total));
         own_ws = true;
     }
-    std::vector<char> stage(w.total, 0);
+    std::vector<char> stage(w.head, 0);
     if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
     for (size_t i = 0; i < n; ++i) ((const SketchDev**)&stage[w.sketches])[i] = sketches[i]->d_s;
     memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
@@ -640,29 +650,12 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
     XP_CUDA_R(cudaEventCreate(&e0));
     XP_CUDA_R(cudaEventCreate(&e1));
-    XP_CUDA_R(cudaMemcpyAsync(ws, stage.data(), w.total, cudaMemcpyHostToDevice, stream));
-    PlanDev pd;
-    pd.n_tickets = plan.n_tickets;
-    pd.n_segs = (int)plan.segs.size();
-    pd.n_sketches = (int)n;
-    pd.segs = (const SegDev*)(ws + w.segs);
-    pd.sketches = (const SketchDev* const*)(ws + w.sketches);
-    pd.acc = (AccDev*)(ws + w.acc);
-    pd.ticket = (u64*)(ws + w.ticket);
+    XP_CUDA_R(cudaMemcpyAsync(ws, stage.data(), w.head, cudaMemcpyHostToDevice, stream));
     XP_CUDA_R(cudaEventRecord(e0, stream));
-    if (plan.n_tickets > 0) {
-        int dev = 0, sms = 1;
-        XP_CUDA_R(cudaGetDevice(&dev));
-        XP_CUDA_R(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        u64 ctas = (u64)sms * (u64)eval_ctas_per_sm();
-        if (ctas > plan.n_tickets) ctas = plan.n_tickets;
-        XP_CUDA_R(launch_eval(pd, (int)ctas, stream));
-        ++launches;
-    }
-    XP_CUDA_R(launch_finish(pd.acc, (int)plan.acc.size(), stream));
-    ++launches;
+    XP_CUDA_R(launch_search(ws, w, plan.n_tickets, (int)plan.segs.size(), (int)n, (int)plan.acc.size(),
+                            max_chunks_of(sketches, n), stream, &launches));
     XP_CUDA_R(cudaEventRecord(e1, stream));
-    XP_CUDA_R(cudaMemcpyAsync(acc.data(), pd.acc, sizeof(AccDev) * acc.size(), cudaMemcpyDeviceToHost, stream));
+    XP_CUDA_R(cudaMemcpyAsync(acc.data(), ws + w.acc, sizeof(AccDev) * acc.size(), cudaMemcpyDeviceToHost, stream));
     XP_CUDA_R(cudaStreamSynchronize(stream));
     XP_CUDA_R(cudaEventElapsedTime(&ms, e0, e1));
 #undef XP_CUDA_R
@@ -721,7 +714,7 @@ extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_o
     Plan plan;
     xp_status st = build_plan(&sketch, 1, o, &plan);
     if (st != XP_OK) return st;
-    const WsLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size());
+    const SearchLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size(), kSurvCapStatic);
     if (plan.acc.size() > 64)
         return fail(XP_ERR_TOO_LARGE, "xp_repair_static: the sketch has more than 64 holes; use xp_repair with a workspace");
     if (w.total > kStaticScratchBytes)
@@ -729,19 +722,14 @@ extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_o
                     " bytes of scratch, the fixed array holds " + std::to_string(kStaticScratchBytes) +
                     "; use xp_repair with a workspace");
     static thread_local char stage[kStaticScratchBytes];          // no heap use that grows with the call
-    memset(stage, 0, w.total);
+    memset(stage, 0, w.head);
     if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
     ((const SketchDev**)&stage[w.sketches])[0] = sketch->d_s;
     memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
     AccDev acc[64];
     cudaStream_t stream = (cudaStream_t)o->stream;
-    int dev = 0, sms = 1;
-    XP_CUDA(cudaGetDevice(&dev));
-    XP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    u64 ctas = (u64)sms * (u64)eval_ctas_per_sm();
-    if (ctas > plan.n_tickets) ctas = plan.n_tickets;
-    XP_CUDA(launch_search_static(stage, w.total, w.segs, w.sketches, w.acc, plan.n_tickets, (int)plan.segs.size(),
-                                 (int)plan.acc.size(), (int)ctas, acc, stream));
+    XP_CUDA(launch_search_static(stage, w, plan.n_tickets, (int)plan.segs.size(), (int)plan.acc.size(),
+                                 max_chunks_of(&sketch, 1), acc, stream));
     XP_CUDA(cudaStreamSynchronize(stream));
     for (int h = 0; h < sketch->n_holes; ++h) {
         xp_hole_summary& r = out[h];

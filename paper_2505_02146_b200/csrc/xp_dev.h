@@ -112,6 +112,13 @@ struct SegDev {
     i32 pad;
 };
 
+// A candidate that passed every probe point and waits for the whole-domain check.  The check
+// is cut into chunks of kVerifyChunk points that any CTA may take; state counts the chunks
+// that passed, its top bit says that some point failed.
+constexpr int kVerifyChunk = 4096;
+constexpr u32 kSurvFailed = 0x80000000u;
+struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, pad; };
+
 struct PlanDev {
     u64 n_tickets;
     i32 n_segs, n_sketches;
@@ -119,6 +126,11 @@ struct PlanDev {
     const SketchDev* const* sketches;  // device table of device pointers
     AccDev* acc;                     // device
     u64* ticket;                     // device counter, zero at launch
+    SurvDev* surv;                   // device queue of survivors
+    u32* surv_n;                     // device counter of pushes (may run past surv_cap), zero at launch
+    u64* verify_ticket;              // device counter, zero at launch
+    u32 surv_cap;
+    u32 max_chunks;                  // chunks of the largest domain among the sketches
 };
 
 }  // namespace xp

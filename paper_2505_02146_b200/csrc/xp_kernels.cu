@@ -6,7 +6,11 @@
 //                      from an atomic counter; no CTA ever waits for another.
 //                        stage 1 (tile segments): probe-point filter over a product of operand tiles;
 //                        stage 2: exact int64 check of a candidate on the probe points (lane = candidate);
-//                        stage 3: check on the whole domain (lane = point, block-wide early exit).
+//                      Survivors of stage 2 go to a global queue.
+//   verify_kernel   -- stage 3: check on the whole domain (lane = point, block-wide early exit),
+//                      cut into (survivor, chunk of points) items that any CTA takes.
+//   count_kernel    -- survivors that passed every chunk become matches: per-size counts (sum)
+//                      and least rank (min) by atomics.
 //   finish_kernel   -- reduction of the per-size results to the least solution per hole.
 //   int32_peak_*    -- integer-ALU peak microbenchmarks.
 #include <cuda_runtime.h>
@@ -142,16 +146,20 @@ struct __align__(16) BcRing { u32 t_add, t_sub, mul_mask, mul_tm; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
+// The candidate under whole-domain check, unranked once and shared by the CTA, leaves resolved.
+struct CandShared {
+    i32 len;
+    i32 var[kMaxSize];           // >= 0: variable; -1: constant; -2 - op: operator
+    i64 val[kMaxSize];
+};
+
 struct EvalShared {
     u64 ticket;
     SegDev seg;
     // survivors of the probe stage, waiting for the whole-domain check
-    u32 n_surv;
+    u32 n_surv, n_pass;          // entries of surv_rank; candidates that passed the probes since the last tally
     u64 surv_rank[kMaxSurvivors];
-    // the candidate under whole-domain check, leaves resolved
-    i32 cand_len;
-    i32 cand_var[kMaxSize];      // >= 0: variable; -1: constant; -2 - op: operator
-    i64 cand_val[kMaxSize];
+    CandShared cand;
     // results of the (sketch, hole) the CTA is working on
     i32 cur_acc;
     u64 match_count[kMaxSize + 1];
@@ -213,53 +221,78 @@ __device__ __noinline__ bool probe_check(const GrammarDev* g, const HoleDev* hol
     return true;
 }
 
-// Stage 3: the whole CTA checks one candidate on every domain point, kThreads points at a
-// time; a failing point anywhere ends the scan at the next block-wide vote.
+__device__ __forceinline__ void stage_candidate(CandShared& c, const GrammarDev* g, int nt, int size, u64 rank) {
+    u32 code[kMaxSize];
+    const int n = unrank(g, nt, size, rank, code);
+    c.len = n;
+    for (int k = 0; k < n; ++k) {
+        if (code[k] & kOpBit) { c.var[k] = -2 - (i32)(code[k] & 0xff); c.val[k] = 0; }
+        else { const LeafDev lf = g->leaves[code[k]]; c.var[k] = lf.var >= 0 ? lf.var : -1; c.val[k] = lf.value; }
+    }
+}
+
+// Stage 3 core: the whole CTA checks the staged candidate on the points [first, last),
+// kThreads points at a time; a failing point anywhere ends the scan at the next block-wide
+// vote.  Returns true if every point passed; adds the points tried by this thread to evals.
+__device__ __forceinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
+                                             i64 last, u64& evals) {
+    const int n = c.len;
+    for (i64 base = first; base < last; base += kThreads) {
+        const i64 pid = base + threadIdx.x;
+        bool bad = false;
+        if (pid < last) {
+            ++evals;
+            i64 pt[kMaxVars];
+            point_coords(sk, pid, pt);
+            i64 want = 0;
+            bool ok = true;
+            if (hole->spec_len == 0) want = hole->spec_table[pid];
+            else ok = eval_code(hole->spec, hole->spec_len, pt, 0, want);
+            i64 st[kCandStack];
+            int sp = 0;
+            for (int k = 0; k < n && ok; ++k) {
+                const i32 cv = c.var[k];
+                if (cv >= -1) st[sp++] = cv >= 0 ? pt[cv] : c.val[k];
+                else {
+                    const i64 b = st[--sp];
+                    i64 r;
+                    ok = apply_op(-2 - cv, st[sp - 1], b, r);
+                    st[sp - 1] = r;
+                }
+            }
+            bad = !ok || !ctx_matches(hole, pt, st[0], want);
+        }
+        if (__syncthreads_or(bad)) return false;
+    }
+    return true;
+}
+
+// A candidate that passed the probes: into the global queue for the verification kernel, or,
+// if that is full, into the CTA's own list (checked by the CTA itself, below).
+__device__ __forceinline__ void push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank) {
+    const u32 at = atomicAdd(plan.surv_n, 1u);
+    if (at < plan.surv_cap) {
+        SurvDev r;
+        r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
+        r.state = 0; r.pad = 0;
+        plan.surv[at] = r;
+    } else {
+        const u32 slot = atomicAdd(&sh.n_surv, 1u);
+        sh.surv_rank[slot] = rank;
+    }
+}
+
+// Whole-domain check of the CTA's own survivor list (only used when the global queue is full).
 __device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64& my_evals) {
     const GrammarDev* g = sk->g;
+    __syncthreads();
     const u32 ns = sh.n_surv;
     for (u32 i = 0; i < ns; ++i) {
         const u64 rank = sh.surv_rank[i];
-        if (threadIdx.x == 0) {
-            u32 code[kMaxSize];
-            const int n = unrank(g, hole->start_nt, size, rank, code);
-            sh.cand_len = n;
-            for (int k = 0; k < n; ++k) {
-                if (code[k] & kOpBit) { sh.cand_var[k] = -2 - (i32)(code[k] & 0xff); sh.cand_val[k] = 0; }
-                else { const LeafDev lf = g->leaves[code[k]]; sh.cand_var[k] = lf.var >= 0 ? lf.var : -1; sh.cand_val[k] = lf.value; }
-            }
-        }
+        if (threadIdx.x == 0) stage_candidate(sh.cand, g, hole->start_nt, size, rank);
         __syncthreads();
-        const int n = sh.cand_len;
-        bool failed = false;
-        for (i64 base = 0; base < sk->n_points; base += kThreads) {
-            const i64 pid = base + threadIdx.x;
-            bool bad = false;
-            if (pid < sk->n_points) {
-                ++my_evals;
-                i64 pt[kMaxVars];
-                point_coords(sk, pid, pt);
-                i64 want = 0;
-                bool ok = true;
-                if (hole->spec_len == 0) want = hole->spec_table[pid];
-                else ok = eval_code(hole->spec, hole->spec_len, pt, 0, want);
-                i64 st[kCandStack];
-                int sp = 0;
-                for (int k = 0; k < n && ok; ++k) {
-                    const i32 cv = sh.cand_var[k];
-                    if (cv >= -1) st[sp++] = cv >= 0 ? pt[cv] : sh.cand_val[k];
-                    else {
-                        const i64 b = st[--sp];
-                        i64 r;
-                        ok = apply_op(-2 - cv, st[sp - 1], b, r);
-                        st[sp - 1] = r;
-                    }
-                }
-                bad = !ok || !ctx_matches(hole, pt, st[0], want);
-            }
-            if (__syncthreads_or(bad)) { failed = true; break; }
-        }
-        if (!failed && threadIdx.x == 0) {
+        const bool ok = check_points(sh.cand, sk, hole, 0, sk->n_points, my_evals);
+        if (ok && threadIdx.x == 0) {
             sh.match_count[size] += 1;
             if (rank < sh.min_rank[size]) sh.min_rank[size] = rank;
         }
@@ -271,7 +304,8 @@ __device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* s
 }
 
 // A linear ticket: kLinearChunk consecutive ranks, each unranked and checked on its own.
-__device__ __noinline__ void linear_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
+__device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
+                                          u64 local, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     const u64 first = seg.rank_begin + local * (u64)kLinearChunk;
@@ -281,13 +315,13 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const SketchDev* sk, 
             u32 code[kMaxSize];
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
             if (probe_check(g, hole, code, n, my_evals)) {
-                const u32 slot = atomicAdd(&sh.n_surv, 1u);
-                sh.surv_rank[slot] = rank;
+                atomicAdd(&sh.n_pass, 1u);
+                push_survivor(sh, plan, rank);
             }
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) { sh.filter_survivors += sh.n_surv; sh.probe_survivors += sh.n_surv; }
+    if (threadIdx.x == 0) { sh.filter_survivors += sh.n_pass; sh.probe_survivors += sh.n_pass; sh.n_pass = 0; }
     verify_survivors(sh, sk, hole, seg.size, my_evals);
 }
 
@@ -622,8 +656,8 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive,
 
 // Stage 2 over the queue: every filter hit is rebuilt as a full candidate, checked exactly on
 // the probe points (lane = candidate), and the survivors go through the whole-domain check.
-__device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
-                                         u64 bc_first, u64& my_evals) {
+__device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
+                                         u64 reg_first, u64 bc_first, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     __syncthreads();
@@ -639,12 +673,12 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, co
             u32 code[kMaxSize];
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
             if (probe_check(g, hole, code, n, my_evals)) {
-                const u32 slot = atomicAdd(&sh.n_surv, 1u);
-                sh.surv_rank[slot] = rank;
+                atomicAdd(&sh.n_pass, 1u);
+                push_survivor(sh, plan, rank);
             }
         }
         __syncthreads();
-        if (threadIdx.x == 0) sh.probe_survivors += sh.n_surv;
+        if (threadIdx.x == 0) { sh.probe_survivors += sh.n_pass; sh.n_pass = 0; }
         verify_survivors(sh, sk, hole, seg.size, my_evals);
     }
     if (threadIdx.x == 0) { sh.filter_survivors += nq; sh.q_n = 0; }
@@ -652,7 +686,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const SketchDev* sk, co
 }
 
 template <bool SWAP>
-__device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
+__device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
                                           u64 bc_first, int n_reg, i64* a64, u32 alive, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const int nb = (int)sh.bc_n;
@@ -729,26 +763,27 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const SketchDev* sk, c
                 // Forget this chunk's hits, empty the queue, and redo the chunk one broadcast slot
                 // and one register operand at a time: at most kThreads * 5 hits per step.
                 if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
-                drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 for (int s = s0; s < s1; ++s)
                     for (int j = 0; j < kNA; ++j) {
                         run(s, s + 1, alive & (1u << j), part == 1);
-                        drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                        drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                     }
                 q_start = 0;
             } else if (qn > (u32)(kQueueCap / 2)) {
-                drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+                drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 q_start = 0;
             } else {
                 q_start = qn;
             }
         }
     }
-    drain_queue(sh, sk, hole, reg_first, bc_first, my_evals);
+    drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
     (void)n_reg;
 }
 
-__device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, u64 local, u64& my_evals) {
+__device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
+                                            u64 local, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
@@ -814,8 +849,8 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const SketchDev* sk,
     if (wide) sh.tile_wide = 1;
     __syncthreads();
     if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
-    if (swap) tile_body<true>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
-    else tile_body<false>(sh, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+    if (swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+    else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
 }
 
 #ifndef XP_MIN_CTAS
@@ -825,7 +860,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.n_surv = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.n_surv = 0; sh.n_pass = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) {
@@ -851,11 +886,64 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
         const SketchDev* sk = plan.sketches[sh.seg.sketch];
         const HoleDev* hole = &sk->holes[sh.seg.hole];
         const u64 local = t - sh.seg.first_ticket;
-        if (sh.seg.kind == kSegTile) tile_ticket(sh, sk, hole, local, my_evals);
-        else linear_ticket(sh, sk, hole, local, my_evals);
+        if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
+        else linear_ticket(sh, plan, sk, hole, local, my_evals);
         __syncthreads();
     }
     flush_acc(sh, plan, my_evals);
+}
+
+// ------------------------------------------------------------------------------------------
+// verify: whole-domain check of the queued survivors
+// ------------------------------------------------------------------------------------------
+
+// Items are (chunk of points, survivor), chunk-major: the first chunk of every survivor is
+// taken before any second chunk, so candidates that fail early cost one chunk.  An item whose
+// survivor has already failed is skipped.  No CTA waits for another.
+__global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
+    __shared__ CandShared cand;
+    __shared__ u64 s_ticket;
+    const u32 pushed = *plan.surv_n;
+    const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
+    const u64 total = n * plan.max_chunks;
+    for (;;) {
+        __syncthreads();
+        if (threadIdx.x == 0) s_ticket = atomicAdd(plan.verify_ticket, 1ull);
+        __syncthreads();
+        const u64 t = s_ticket;
+        if (t >= total) break;
+        const u64 c = t / n, i = t % n;
+        SurvDev* sv = &plan.surv[i];
+        const SketchDev* sk = plan.sketches[sv->sketch];
+        const i64 first = (i64)c * kVerifyChunk;
+        if (first >= sk->n_points) continue;
+        if (*(volatile u32*)&sv->state & kSurvFailed) continue;
+        const HoleDev* hole = &sk->holes[sv->hole];
+        if (threadIdx.x == 0) stage_candidate(cand, sk->g, hole->start_nt, sv->size, sv->rank);
+        __syncthreads();
+        const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
+        u64 evals = 0;
+        const bool ok = check_points(cand, sk, hole, first, last, evals);
+        if (threadIdx.x == 0) {
+            if (ok) atomicAdd(&sv->state, 1u); else atomicOr(&sv->state, kSurvFailed);
+            atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
+        }
+    }
+}
+
+// One thread per queued survivor: it is a match if no chunk failed and every chunk passed.
+__global__ void count_kernel(const PlanDev plan) {
+    const u32 pushed = *plan.surv_n;
+    const u32 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
+    const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const SurvDev sv = plan.surv[i];
+    const i64 np = plan.sketches[sv.sketch]->n_points;
+    const u32 chunks = (u32)((np + kVerifyChunk - 1) / kVerifyChunk);
+    if ((sv.state & kSurvFailed) || sv.state != chunks) return;
+    AccDev* a = &plan.acc[sv.acc];
+    atomicAdd(&a->match_count[sv.size], 1ull);
+    atomicMin(&a->min_rank[sv.size], sv.rank);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -924,43 +1012,65 @@ cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, u64 n
     return cudaGetLastError();
 }
 
-cudaError_t launch_eval(const PlanDev& plan, int n_ctas, cudaStream_t stream) {
-    eval_kernel<<<n_ctas, kThreads, 0, stream>>>(plan);
-    return cudaGetLastError();
+static int resident_ctas(const void* kernel) {
+    int dev = 0, sms = 1, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    return sms * per_sm;
 }
 
-cudaError_t launch_finish(AccDev* acc, int n_acc, cudaStream_t stream) {
+cudaError_t launch_search(char* base, const SearchLayout& L, u64 n_tickets, int n_segs, int n_sketches, int n_acc,
+                          u32 max_chunks, cudaStream_t stream, int* n_launches) {
+    PlanDev pd;
+    pd.n_tickets = n_tickets;
+    pd.n_segs = n_segs;
+    pd.n_sketches = n_sketches;
+    pd.ticket = (u64*)base;
+    pd.verify_ticket = (u64*)(base + 8);
+    pd.surv_n = (u32*)(base + 16);
+    pd.segs = (const SegDev*)(base + L.segs);
+    pd.sketches = (const SketchDev* const*)(base + L.sketches);
+    pd.acc = (AccDev*)(base + L.acc);
+    pd.surv = (SurvDev*)(base + L.surv);
+    pd.surv_cap = L.surv_cap;
+    pd.max_chunks = max_chunks;
+    cudaError_t e;
+    if (n_tickets > 0) {
+        u64 ctas = (u64)resident_ctas((const void*)eval_kernel);      // persistent CTAs: one wave
+        if (ctas > n_tickets) ctas = n_tickets;
+        eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        verify_kernel<<<resident_ctas((const void*)verify_kernel), kThreads, 0, stream>>>(pd);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        count_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        *n_launches += 3;
+    }
     const int warps_per_block = 8;
-    const int blocks = (n_acc + warps_per_block - 1) / warps_per_block;
-    finish_kernel<<<blocks, warps_per_block * 32, 0, stream>>>(acc, n_acc);
+    finish_kernel<<<(n_acc + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, stream>>>(pd.acc, n_acc);
+    *n_launches += 1;
     return cudaGetLastError();
-}
-
-int eval_ctas_per_sm() {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, eval_kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
-    return n;
 }
 
 // ------------------------------------------------------------------------------------------
 // search with the scratch in a fixed device array (no allocation at call time)
 // ------------------------------------------------------------------------------------------
 
-// Scratch of the allocation-free entry point: ticket counter, segment table, sketch pointer
-// and accumulators of ONE call.  Every GPU that loads the library holds these bytes until the
-// process exits.  In host code the name below is only a stand-in for the symbol; the device
-// address comes from cudaGetSymbolAddress.
+// Scratch of the allocation-free entry point: counters, segment table, sketch pointer,
+// accumulators and survivor queue of ONE call.  Every GPU that loads the library holds these
+// bytes until the process exits.  In host code the name below is only a stand-in for the
+// symbol; the device address comes from cudaGetSymbolAddress.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 static void* g_static_scratch_addr[64];      // per device, filled on the first call made on it
 
-// Copies the staged plan (host bytes laid out as ticket | segments | sketch table | accumulators;
-// the ticket and the accumulators staged in their start state, which also wipes what the last
-// call left) into the fixed array, runs the search and the reduction on it, and queues the copy
-// of the accumulators back to `acc_out`.  Allocates nothing.
-cudaError_t launch_search_static(const void* stage, size_t total, size_t off_segs, size_t off_sketches, size_t off_acc,
-                                 u64 n_tickets, int n_segs, int n_acc, int n_ctas, AccDev* acc_out, cudaStream_t stream) {
-    if (total > kStaticScratchBytes) return cudaErrorInvalidValue;
+// Copies the staged head of the plan (counters and accumulators in their start state, which
+// also wipes what the last call left) into the fixed array, runs the search on it, and queues
+// the copy of the accumulators back to `acc_out`.  Allocates nothing.
+cudaError_t launch_search_static(const void* stage, const SearchLayout& L, u64 n_tickets, int n_segs, int n_acc,
+                                 u32 max_chunks, AccDev* acc_out, cudaStream_t stream) {
+    if (L.total > kStaticScratchBytes) return cudaErrorInvalidValue;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -972,24 +1082,12 @@ cudaError_t launch_search_static(const void* stage, size_t total, size_t off_seg
         g_static_scratch_addr[dev] = p;
     }
     char* base = (char*)g_static_scratch_addr[dev];
-    e = cudaMemcpyAsync(base, stage, total, cudaMemcpyHostToDevice, stream);
+    e = cudaMemcpyAsync(base, stage, L.head, cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return e;
-    PlanDev pd;
-    pd.n_tickets = n_tickets;
-    pd.n_segs = n_segs;
-    pd.n_sketches = 1;
-    pd.ticket = (u64*)base;
-    pd.segs = (const SegDev*)(base + off_segs);
-    pd.sketches = (const SketchDev* const*)(base + off_sketches);
-    pd.acc = (AccDev*)(base + off_acc);
-    if (n_tickets > 0) {
-        eval_kernel<<<n_ctas, kThreads, 0, stream>>>(pd);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
-    e = launch_finish(pd.acc, n_acc, stream);
+    int launches = 0;
+    e = launch_search(base, L, n_tickets, n_segs, 1, n_acc, max_chunks, stream, &launches);
     if (e != cudaSuccess) return e;
-    return cudaMemcpyAsync(acc_out, pd.acc, sizeof(AccDev) * (size_t)n_acc, cudaMemcpyDeviceToHost, stream);
+    return cudaMemcpyAsync(acc_out, base + L.acc, sizeof(AccDev) * (size_t)n_acc, cudaMemcpyDeviceToHost, stream);
 }
 
 cudaError_t launch_int32_peak(int which, u32* out, int blocks, int iters, cudaStream_t stream) {

@@ -9,12 +9,18 @@ namespace xp {
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream);
 cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, u64 n_entries, cudaStream_t stream);
-cudaError_t launch_eval(const PlanDev& plan, int n_ctas, cudaStream_t stream);
-cudaError_t launch_finish(AccDev* acc, int n_acc, cudaStream_t stream);
-int eval_ctas_per_sm();
+// Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
+//   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32)   -- zero at launch
+//   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
+//   surv: the survivor queue (surv_cap entries), written by the kernels only
+struct SearchLayout { size_t segs, sketches, acc, head, surv, total; u32 surv_cap; };
+
+// The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel.
+cudaError_t launch_search(char* base, const SearchLayout& L, u64 n_tickets, int n_segs, int n_sketches, int n_acc,
+                          u32 max_chunks, cudaStream_t stream, int* n_launches);
 constexpr size_t kStaticScratchBytes = 1u << 20;     // fixed scratch of the allocation-free entry point
-cudaError_t launch_search_static(const void* stage, size_t total, size_t off_segs, size_t off_sketches, size_t off_acc,
-                                 u64 n_tickets, int n_segs, int n_acc, int n_ctas, AccDev* acc_out, cudaStream_t stream);
+cudaError_t launch_search_static(const void* stage, const SearchLayout& L, u64 n_tickets, int n_segs, int n_acc,
+                                 u32 max_chunks, AccDev* acc_out, cudaStream_t stream);
 cudaError_t launch_int32_peak(int which, u32* out, int blocks, int iters, cudaStream_t stream);
 
 }  // namespace xp
