@@ -903,24 +903,36 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
     __shared__ CandShared cand;
     __shared__ u64 s_ticket;
+    __shared__ i32 s_skip;
     const u32 pushed = *plan.surv_n;
     const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
     const u64 total = n * plan.max_chunks;
     for (;;) {
         __syncthreads();
-        if (threadIdx.x == 0) s_ticket = atomicAdd(plan.verify_ticket, 1ull);
+        // Thread 0 takes the item and decides for the whole CTA whether it is skipped (the
+        // survivor's state may change under other CTAs, so it is read once, by one thread).
+        if (threadIdx.x == 0) {
+            const u64 t = atomicAdd(plan.verify_ticket, 1ull);
+            s_ticket = t;
+            s_skip = 1;
+            if (t < total) {
+                const SurvDev* sv = &plan.surv[t % n];
+                const SketchDev* sk = plan.sketches[sv->sketch];
+                const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
+                if ((i64)(t / n) * kVerifyChunk < sk->n_points && !failed) {
+                    s_skip = 0;
+                    stage_candidate(cand, sk->g, sk->holes[sv->hole].start_nt, sv->size, sv->rank);
+                }
+            }
+        }
         __syncthreads();
         const u64 t = s_ticket;
         if (t >= total) break;
-        const u64 c = t / n, i = t % n;
-        SurvDev* sv = &plan.surv[i];
+        if (s_skip) continue;
+        SurvDev* sv = &plan.surv[t % n];
         const SketchDev* sk = plan.sketches[sv->sketch];
-        const i64 first = (i64)c * kVerifyChunk;
-        if (first >= sk->n_points) continue;
-        if (*(volatile u32*)&sv->state & kSurvFailed) continue;
         const HoleDev* hole = &sk->holes[sv->hole];
-        if (threadIdx.x == 0) stage_candidate(cand, sk->g, hole->start_nt, sv->size, sv->rank);
-        __syncthreads();
+        const i64 first = (i64)(t / n) * kVerifyChunk;
         const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
         u64 evals = 0;
         const bool ok = check_points(cand, sk, hole, first, last, evals);

@@ -1,0 +1,69 @@
+"""The five configurations at full size against results written by the CPU oracle alone
+(tests/golden/make_full_goldens.py, sharded over rank windows).  Everything the search
+outputs is compared bit for bit: candidate counts, match counts, the least solution."""
+import json
+import os
+
+import pytest
+
+from xp_instances import config2, config3, config4, config5
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _check_large(xp, name, make):
+    path = os.path.join(GOLDEN, f"{name}_seed0_full.json")
+    if not os.path.exists(path):
+        pytest.skip(f"{path} has not been generated")
+    want = json.load(open(path))["holes"]
+    sk = make(0)
+    gr = xp.xp_grammar_create(sk.grammar)
+    ls = xp.xp_sketch_load(gr, sk)
+    got = xp.xp_repair(ls)
+    assert len(got) == len(want)
+    for h, (g, w) in enumerate(zip(got, want)):
+        assert g.cand_count == w["cand_count"], (name, h)
+        assert g.match_count == w["match_count"], (name, h)
+        assert g.solved == w["solved"], (name, h)
+        if w["solved"]:
+            assert (g.least_size, g.least_rank, g.least_text) == (w["least_size"], w["least_rank"], w["least_text"]), (name, h)
+    return got
+
+
+def test_config2_full(xp):
+    got = _check_large(xp, "config2", config2)
+    assert sum(got[0].cand_count) == 213939625416
+
+
+def test_config3_full(xp):
+    got = _check_large(xp, "config3", config3)
+    assert [sum(g.cand_count) for g in got] == [134377694] * 3 and all(g.solved for g in got)
+
+
+def test_config4_full(xp):
+    got = _check_large(xp, "config4", config4)
+    assert sum(got[0].cand_count) == 322884631700
+
+
+def test_config5_full_batch(xp):
+    rows = [[int(x) for x in line.split()] for line in open(os.path.join(GOLDEN, "config5_seed0_full.txt"))
+            if not line.startswith("#")]
+    assert len(rows) == 4096
+    sks = config5(0, 4096)
+    grs, loaded = {}, []
+    for sk in sks:
+        key = tuple(v.hi for v in sk.grammar.variables)
+        if key not in grs:
+            grs[key] = xp.xp_grammar_create(sk.grammar)
+        loaded.append(xp.xp_sketch_load(grs[key], sk))
+    res = xp.xp_repair_batch(loaded)
+    unsolved = 0
+    for i, (r, row) in enumerate(zip(res, rows)):
+        g = r[0]
+        assert [g.match_count[1], g.match_count[3], g.match_count[5]] == row[:3], i
+        assert g.solved == (row[3] != 0), i
+        if g.solved:
+            assert (g.least_size, g.least_rank) == (row[3], row[4]), i
+        unsolved += not g.solved
+    assert 0 < unsolved < 4096 // 4          # the generator plants targets beyond the bound in about a tenth
