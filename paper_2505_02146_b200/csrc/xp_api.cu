@@ -2,6 +2,7 @@
 // decoding and the C ABI declared in include/xp.h.
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <chrono>
 #include <cstdio>
 #include <cstring>
@@ -236,6 +237,7 @@ static xp_status grammar_to_device(xp_grammar* g) {
 struct HoleHost {
     int start_nt = 0, max_size = 0;
     bool filter_ok = false;          // the probe filter applies (probe 0 exists, context affine there)
+    bool never = false;              // the spec is undefined at some point: no candidate can match
 };
 
 struct xp_sketch {
@@ -433,6 +435,38 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             XP_CUDA_S(launch_subvalues(s->d_s, h, k, at_size, nullptr));
         }
     }
+    // Points of a box and values of spec expressions, staged once so that the whole-domain
+    // check reads them instead of recomputing them for every surviving candidate.
+    if (n_points > 0 && (u64)n_points <= kStageMaxPoints) {
+        bool i32_ok = true;
+        for (int v = 0; v < nv; ++v) i32_ok = i32_ok && g->lo[v] >= INT32_MIN && g->hi[v] <= (i64)INT32_MAX + 1;
+        if (d->domain_kind == XP_DOMAIN_BOX && i32_ok && nv > 0) {
+            void* p = nullptr;
+            XP_CUDA_S(cudaMalloc(&p, sizeof(i32) * (size_t)n_points * (size_t)nv));
+            s->owned.push_back(p);
+            XP_CUDA_S(launch_stage_points(s->d_s, n_points, (i32*)p, nullptr));
+            XP_CUDA_S(cudaStreamSynchronize(nullptr));       // the kernel reads the sketch before its coords field changes
+            hs.coords = (const i32*)p;
+            XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
+        }
+        u32* d_bad = nullptr;
+        std::vector<u32> bad(d->n_holes, 0);
+        XP_CUDA_S(cudaMalloc((void**)&d_bad, sizeof(u32) * d->n_holes));
+        s->owned.push_back(d_bad);
+        XP_CUDA_S(cudaMemset(d_bad, 0, sizeof(u32) * d->n_holes));
+        for (int h = 0; h < d->n_holes; ++h) {
+            if (hh[h].spec_len == 0) continue;
+            void* p = nullptr;
+            XP_CUDA_S(cudaMalloc(&p, sizeof(i64) * (size_t)n_points));
+            s->owned.push_back(p);
+            XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)p, d_bad + h, nullptr));
+            XP_CUDA_S(cudaStreamSynchronize(nullptr));
+            hh[h].spec_table = (const i64*)p;
+            XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &hh[h], sizeof(HoleDev), cudaMemcpyHostToDevice));
+        }
+        XP_CUDA_S(cudaMemcpy(bad.data(), d_bad, sizeof(u32) * d->n_holes, cudaMemcpyDeviceToHost));
+        for (int h = 0; h < d->n_holes; ++h) s->holes[h].never = bad[h] != 0;
+    }
     XP_CUDA_S(cudaStreamSynchronize(nullptr));
 #undef XP_CUDA_S
     *out = s;
@@ -564,7 +598,7 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
             int kmin = 1, kmax = ho.max_size;
             if (o->size_min > 0) kmin = o->size_min;
             if (o->size_max > 0 && o->size_max < kmax) kmax = o->size_max;
-            for (int k = kmin; k <= kmax; ++k) {
+            for (int k = kmin; k <= kmax && !ho.never; ++k) {
                 u64 lo = 0, hi = s->g->cnt[ho.start_nt][k];
                 for (int r = 0; r < o->n_rank_ranges; ++r) {
                     const xp_rank_range& rr = o->rank_ranges[r];

@@ -26,6 +26,8 @@ constexpr int kLinearChunk = kThreads * 4;   // ranks per linear ticket
 constexpr int kNA = 8;                // tile tickets: register-side operands per thread
 constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
 constexpr int kBcTile = 512;          // broadcast-side operands per tile
+constexpr u64 kStageMaxPoints = 1ull << 26;  // largest box whose points and spec values are staged in HBM at load
+constexpr int kProgMax = 96;          // candidate substituted into its context: longest staged program
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 
@@ -47,7 +49,8 @@ struct GrammarDev {
 
 struct HoleDev {
     i32 start_nt, max_size, ctx_len, spec_len;   // spec_len == 0: the spec is a table
-    const i64* spec_table;                        // device, n_points values
+    const i64* spec_table;                        // device, n_points values: the caller's table, or the spec
+                                                  // expression evaluated once per point at load (null: evaluate)
     xp_instr ctx[kMaxCode];
     xp_instr spec[kMaxCode];
     // Probe points of this hole, most discriminating first (written by the prepare kernel).
@@ -75,7 +78,8 @@ struct SketchDev {
     const GrammarDev* g;                          // device
     i32 n_vars, n_holes, domain_kind, n_samples;
     i64 n_points;
-    const i32* coords;                            // device, table domains
+    const i32* coords;                            // device: the points of a table domain, or the staged
+                                                  // points of a box (null: derive them from the point id)
     i64 lo[kMaxVars], ext[kMaxVars];              // box: range start and extent per variable
     HoleDev* holes;                               // device
     i64 sample_id[kProbeSamples];                 // point ids the probes are chosen from (host-chosen)

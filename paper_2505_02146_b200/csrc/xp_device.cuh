@@ -143,7 +143,7 @@ __device__ __forceinline__ bool eval_code(const xp_instr* code, int n, const i64
 // the box (first variable slowest).
 __device__ __forceinline__ void point_coords(const SketchDev* __restrict__ s, i64 pid, i64* pt) {
     const int nv = s->n_vars;
-    if (s->domain_kind == XP_DOMAIN_TABLE) {
+    if (s->coords != nullptr) {
         const i32* row = s->coords + pid * nv;
         for (int d = 0; d < nv; ++d) pt[d] = row[d];
     } else {

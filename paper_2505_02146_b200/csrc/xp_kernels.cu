@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
         if (t < ns) {
             i64 v = 0;
             bool ok = true;
-            if (hole->spec_len == 0) v = hole->spec_table[s->sample_id[t]];
+            if (hole->spec_table != nullptr) v = hole->spec_table[s->sample_id[t]];
             else ok = eval_code(hole->spec, hole->spec_len, pt, 0, v);
             s_spec[t] = v;
             s_ok[t] = ok;
@@ -146,11 +146,17 @@ struct __align__(16) BcRing { u32 t_add, t_sub, mul_mask, mul_tm; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
-// The candidate under whole-domain check, unranked once and shared by the CTA, leaves resolved.
+// The candidate under whole-domain check as one postfix program shared by the CTA: the
+// hole's context with the candidate's code substituted for every HOLE leaf, leaves resolved.
+// depth = deepest operand stack; depth == 0 marks a program too long to stage (the slow
+// interpreters are used instead).
 struct CandShared {
-    i32 len;
-    i32 var[kMaxSize];           // >= 0: variable; -1: constant; -2 - op: operator
-    i64 val[kMaxSize];
+    i32 len, depth;
+    i32 cand_len;
+    i32 var[kProgMax];           // >= 0: variable; -1: constant; -2 - op: operator
+    i64 val[kProgMax];
+    i32 cvar[kMaxSize];          // the candidate alone (for the slow path)
+    i64 cval[kMaxSize];
 };
 
 struct EvalShared {
@@ -221,22 +227,94 @@ __device__ __noinline__ bool probe_check(const GrammarDev* g, const HoleDev* hol
     return true;
 }
 
-__device__ __forceinline__ void stage_candidate(CandShared& c, const GrammarDev* g, int nt, int size, u64 rank) {
+__device__ __noinline__ void stage_candidate(CandShared& c, const GrammarDev* g, const HoleDev* hole, int size, u64 rank) {
     u32 code[kMaxSize];
-    const int n = unrank(g, nt, size, rank, code);
-    c.len = n;
+    const int n = unrank(g, hole->start_nt, size, rank, code);
+    c.cand_len = n;
     for (int k = 0; k < n; ++k) {
-        if (code[k] & kOpBit) { c.var[k] = -2 - (i32)(code[k] & 0xff); c.val[k] = 0; }
-        else { const LeafDev lf = g->leaves[code[k]]; c.var[k] = lf.var >= 0 ? lf.var : -1; c.val[k] = lf.value; }
+        if (code[k] & kOpBit) { c.cvar[k] = -2 - (i32)(code[k] & 0xff); c.cval[k] = 0; }
+        else { const LeafDev lf = g->leaves[code[k]]; c.cvar[k] = lf.var >= 0 ? lf.var : -1; c.cval[k] = lf.value; }
     }
+    // the context with the candidate in place of each HOLE
+    int len = 0, sp = 0, depth = 0;
+    bool fits = true;
+    auto emit = [&](i32 var, i64 val) {
+        if (len >= kProgMax) { fits = false; return; }
+        c.var[len] = var; c.val[len] = val; ++len;
+        if (var >= -1) { if (++sp > depth) depth = sp; } else --sp;
+    };
+    if (hole->ctx_len == 0) {
+        for (int k = 0; k < n; ++k) emit(c.cvar[k], c.cval[k]);
+    } else {
+        for (int i = 0; i < hole->ctx_len && fits; ++i) {
+            const xp_instr in = hole->ctx[i];
+            if (in.kind == XP_I_HOLE) for (int k = 0; k < n; ++k) emit(c.cvar[k], c.cval[k]);
+            else if (in.kind == XP_I_OP) emit(-2 - in.arg, 0);
+            else emit(in.kind == XP_I_VAR ? in.arg : -1, in.value);
+        }
+    }
+    c.len = len;
+    c.depth = fits ? depth : 0;
+}
+
+// The staged program at one point with an operand stack of D registers (D >= its depth): a
+// push shifts the registers up, an operator combines the two lowest and shifts down.  The
+// program is the same for every thread, so all branches are uniform.
+template <int D>
+__device__ __forceinline__ bool run_program(const CandShared& c, const i32* __restrict__ row, i64& out) {
+    i64 st[D];
+#pragma unroll
+    for (int i = 0; i < D; ++i) st[i] = 0;
+    const int n = c.len;
+    for (int k = 0; k < n; ++k) {
+        const i32 cv = c.var[k];
+        if (cv >= -1) {
+            const i64 v = cv >= 0 ? (i64)row[cv] : c.val[k];
+#pragma unroll
+            for (int i = D - 1; i > 0; --i) st[i] = st[i - 1];
+            st[0] = v;
+        } else {
+            i64 r;
+            if (!apply_op(-2 - cv, st[1], st[0], r)) return false;
+            st[0] = r;
+#pragma unroll
+            for (int i = 1; i < D - 1; ++i) st[i] = st[i + 1];
+        }
+    }
+    out = st[0];
+    return true;
 }
 
 // Stage 3 core: the whole CTA checks the staged candidate on the points [first, last),
 // kThreads points at a time; a failing point anywhere ends the scan at the next block-wide
 // vote.  Returns true if every point passed; adds the points tried by this thread to evals.
-__device__ __forceinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
-                                             i64 last, u64& evals) {
-    const int n = c.len;
+// Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
+// and the program runs on a register stack.  Otherwise coordinates are derived from the point
+// id and the interpreters with a stack in local memory are used.
+template <int D>
+__device__ __forceinline__ bool check_points_fast(const CandShared& c, const SketchDev* sk, const HoleDev* hole,
+                                                  i64 first, i64 last, u64& evals) {
+    const int nv = sk->n_vars;
+    for (i64 base = first; base < last; base += kThreads) {
+        const i64 pid = base + threadIdx.x;
+        bool bad = false;
+        if (pid < last) {
+            ++evals;
+            i64 v;
+            bad = !run_program<D>(c, sk->coords + pid * nv, v) || v != hole->spec_table[pid];
+        }
+        if (__syncthreads_or(bad)) return false;
+    }
+    return true;
+}
+
+__device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
+                                          i64 last, u64& evals) {
+    if (sk->coords != nullptr && hole->spec_table != nullptr && c.depth >= 1) {
+        if (c.depth <= 4) return check_points_fast<4>(c, sk, hole, first, last, evals);
+        if (c.depth <= 8) return check_points_fast<8>(c, sk, hole, first, last, evals);
+    }
+    const int n = c.cand_len;
     for (i64 base = first; base < last; base += kThreads) {
         const i64 pid = base + threadIdx.x;
         bool bad = false;
@@ -246,13 +324,13 @@ __device__ __forceinline__ bool check_points(const CandShared& c, const SketchDe
             point_coords(sk, pid, pt);
             i64 want = 0;
             bool ok = true;
-            if (hole->spec_len == 0) want = hole->spec_table[pid];
+            if (hole->spec_table != nullptr) want = hole->spec_table[pid];
             else ok = eval_code(hole->spec, hole->spec_len, pt, 0, want);
             i64 st[kCandStack];
             int sp = 0;
             for (int k = 0; k < n && ok; ++k) {
-                const i32 cv = c.var[k];
-                if (cv >= -1) st[sp++] = cv >= 0 ? pt[cv] : c.val[k];
+                const i32 cv = c.cvar[k];
+                if (cv >= -1) st[sp++] = cv >= 0 ? pt[cv] : c.cval[k];
                 else {
                     const i64 b = st[--sp];
                     i64 r;
@@ -289,7 +367,7 @@ __device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* s
     const u32 ns = sh.n_surv;
     for (u32 i = 0; i < ns; ++i) {
         const u64 rank = sh.surv_rank[i];
-        if (threadIdx.x == 0) stage_candidate(sh.cand, g, hole->start_nt, size, rank);
+        if (threadIdx.x == 0) stage_candidate(sh.cand, g, hole, size, rank);
         __syncthreads();
         const bool ok = check_points(sh.cand, sk, hole, 0, sk->n_points, my_evals);
         if (ok && threadIdx.x == 0) {
@@ -439,6 +517,33 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
         }
     }
     return alive;
+}
+
+// Staging of a box domain at load: the coordinates of every point (int32 rows, like a table
+// domain) and, per hole with a spec expression, the spec's value at every point.  *bad is set
+// if the spec is undefined somewhere (then no candidate can match).
+__global__ void __launch_bounds__(256) stage_points_kernel(const SketchDev* sk, i32* coords) {
+    const i64 pid = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pid >= sk->n_points) return;
+    const int nv = sk->n_vars;
+    u64 rem = (u64)pid;
+    for (int d = nv - 1; d >= 0; --d) {
+        u64 q, r;
+        divmod_u64(rem, (u64)sk->ext[d], q, r);
+        coords[pid * nv + d] = (i32)(sk->lo[d] + (i64)r);
+        rem = q;
+    }
+}
+
+__global__ void __launch_bounds__(256) stage_spec_kernel(const SketchDev* sk, int hole_index, i64* spec, u32* bad) {
+    const i64 pid = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pid >= sk->n_points) return;
+    const HoleDev* hole = &sk->holes[hole_index];
+    i64 pt[kMaxVars];
+    point_coords(sk, pid, pt);
+    i64 v = 0;
+    if (!eval_code(hole->spec, hole->spec_len, pt, 0, v)) atomicOr(bad, 1u);
+    spec[pid] = v;
 }
 
 // Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
@@ -921,7 +1026,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
                 const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
                 if ((i64)(t / n) * kVerifyChunk < sk->n_points && !failed) {
                     s_skip = 0;
-                    stage_candidate(cand, sk->g, sk->holes[sv->hole].start_nt, sv->size, sv->rank);
+                    stage_candidate(cand, sk->g, &sk->holes[sv->hole], sv->size, sv->rank);
                 }
             }
         }
@@ -1015,6 +1120,16 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream) {
     prepare_kernel<<<1, kProbeSamples, 0, stream>>>(s);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_stage_points(const SketchDev* s, i64 n_points, i32* coords, cudaStream_t stream) {
+    stage_points_kernel<<<(unsigned)((n_points + 255) / 256), 256, 0, stream>>>(s, coords);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, i64* spec, u32* bad, cudaStream_t stream) {
+    stage_spec_kernel<<<(unsigned)((n_points + 255) / 256), 256, 0, stream>>>(s, hole_index, spec, bad);
     return cudaGetLastError();
 }
 
