@@ -359,7 +359,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
                 if (!dup) hs.sample_id[ns++] = id;
             }
         } else {
-            for (i64 id = 0; id < n_points && ns < 16; ++id) hs.sample_id[ns++] = id;
+            for (i64 id = 0; id < n_points && ns < 4; ++id) hs.sample_id[ns++] = id;
         }
         for (u64 k = 0; ns < kProbeSamples && k < 4 * kProbeSamples; ++k) {
             const i64 id = (i64)(mix64(k) % (u64)n_points);

@@ -62,18 +62,27 @@ __device__ bool ctx_affine(const HoleDev* hole, const i64* pt, u64& A, u64& B) {
     return true;
 }
 
-// One CTA of kProbeSamples threads per sketch.  Thread t evaluates sample point t; thread 0
-// then orders each hole's probes: the sample with the largest |spec| + sum |coordinate|
-// first (large, distinct operand values make coincidental matches rare), the rest in sample
-// order (box corners come first there).
-__global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
+// Choice of each hole's probe points, once per sketch (one CTA).  Threads evaluate the sample
+// points; then a sample of small candidates (sizes 1, 3, 5, ranks spread evenly) is run on
+// every sample point, giving each a bit set of the samples where it satisfies the constraint.
+// The probes are picked greedily: each next probe is the sample that the fewest of the
+// sampled candidates still alive (satisfying all probes picked so far) also satisfy; ties go
+// to the larger |spec| + sum |coordinate| (large, distinct operand values make coincidences
+// rare).  Only the amount of work downstream depends on this choice, never a result.
+constexpr int kPrepThreads = 256;
+constexpr int kPrepCands = 1024;
+__global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
     __shared__ i64 s_pt[kProbeSamples][kMaxVars];
     __shared__ i64 s_spec[kProbeSamples];
     __shared__ int s_ok[kProbeSamples];
     __shared__ u64 s_score[kProbeSamples];
+    __shared__ u64 s_sig[kPrepCands];
+    __shared__ u32 s_count[kProbeSamples];
+    __shared__ u64 s_chosen;
     const int t = threadIdx.x;
     const int ns = s->n_samples;
     const int nv = s->n_vars;
+    const GrammarDev* g = s->g;
     i64 pt[kMaxVars];
     u64 coord_mag = 0;
     if (t < ns) {
@@ -97,23 +106,62 @@ __global__ void __launch_bounds__(kProbeSamples) prepare_kernel(SketchDev* s) {
             s_score[t] = ok ? (mag > (1ull << 62) ? (1ull << 62) : mag) + coord_mag : 0;
         }
         __syncthreads();
-        if (t == 0) {
-            int best = 0;
-            for (int i = 1; i < ns; ++i) if (s_score[i] > s_score[best]) best = i;
-            int n = 0;
-            u32 okmask = 0;
-            for (int j = -1; j < ns && n < kMaxProbe; ++j) {
-                const int i = j < 0 ? best : j;
-                if (j >= 0 && i == best) continue;
-                if (ns == 0) break;
-                hole->probe_id[n] = s->sample_id[i];
-                for (int d = 0; d < nv; ++d) hole->probe_pt[n][d] = s_pt[i][d];
-                hole->probe_spec[n] = s_spec[i];
-                if (s_ok[i]) okmask |= 1u << n;
-                ++n;
+        // behaviour of sampled small candidates on the sample points
+        int sizes[3], nsz = 0;
+        for (int k = 1; k <= 5 && k <= hole->max_size; k += 2)
+            if (g->cnt[hole->start_nt][k] > 0) sizes[nsz++] = k;
+        const int ncand = nsz > 0 ? kPrepCands : 0;
+        for (int c = t; c < ncand; c += kPrepThreads) {
+            const int size = sizes[c % nsz];
+            const u64 cnt = g->cnt[hole->start_nt][size];
+            const u64 per = (u64)(kPrepCands / nsz) + 1;
+            const u64 slot = (u64)(c / nsz);
+            u64 sig = 0;
+            if (slot < cnt || cnt >= per) {                       // small sizes: every rank once, the rest unused
+                const u64 rank = cnt >= per ? slot * (cnt / per) : slot;
+                u32 code[kMaxSize];
+                const int n = unrank(g, hole->start_nt, size, rank, code);
+                for (int j = 0; j < ns; ++j) {
+                    i64 v;
+                    if (s_ok[j] && eval_cand(code, n, g->leaves, s_pt[j], v) && ctx_matches(hole, s_pt[j], v, s_spec[j]))
+                        sig |= 1ull << j;
+                }
             }
+            s_sig[c] = sig;
+        }
+        if (t == 0) s_chosen = 0;
+        __syncthreads();
+        int n = 0;
+        for (; n < kMaxProbe && n < ns; ++n) {
+            const u64 chosen = s_chosen;
+            if (t < ns) {
+                u32 count = 0xffffffffu;
+                if (!((chosen >> t) & 1ull)) {
+                    count = 0;
+                    const u64 need = chosen | (1ull << t);
+                    for (int c = 0; c < ncand; ++c) count += (s_sig[c] & need) == need;
+                }
+                s_count[t] = count;
+            }
+            __syncthreads();
+            if (t == 0) {
+                int best = -1;
+                for (int i = 0; i < ns; ++i) {
+                    if ((chosen >> i) & 1ull) continue;
+                    if (best < 0 || s_count[i] < s_count[best] || (s_count[i] == s_count[best] && s_score[i] > s_score[best])) best = i;
+                }
+                hole->probe_id[n] = s->sample_id[best];
+                for (int d = 0; d < nv; ++d) hole->probe_pt[n][d] = s_pt[best][d];
+                hole->probe_spec[n] = s_spec[best];
+                if (n == 0) hole->probe_spec_ok = 0;
+                if (s_ok[best]) hole->probe_spec_ok |= 1u << n;
+                s_chosen = chosen | (1ull << best);
+            }
+            __syncthreads();
+        }
+        if (t == 0) {
             hole->n_probe = n;
-            hole->probe_spec_ok = okmask;
+            if (n == 0) hole->probe_spec_ok = 0;
             u64 A = 0, B = 0;
             hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
             hole->aff_A = A;
@@ -253,8 +301,10 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const GrammarDev* g,
             else emit(in.kind == XP_I_VAR ? in.arg : -1, in.value);
         }
     }
+    bool has_hole = hole->ctx_len == 0;
+    for (int i = 0; i < hole->ctx_len; ++i) has_hole = has_hole || hole->ctx[i].kind == XP_I_HOLE;
     c.len = len;
-    c.depth = fits ? depth : 0;
+    c.depth = (fits && has_hole) ? depth : 0;     // a context that ignores the hole still needs the candidate to be defined
 }
 
 // The staged program at one point with an operand stack of D registers (D >= its depth): a
@@ -1119,7 +1169,7 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 // ------------------------------------------------------------------------------------------
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream) {
-    prepare_kernel<<<1, kProbeSamples, 0, stream>>>(s);
+    prepare_kernel<<<1, kPrepThreads, 0, stream>>>(s);
     return cudaGetLastError();
 }
 
