@@ -184,13 +184,14 @@ static_assert(kThreads * 5 <= kQueueCap / 2, "one replay step must fit the free 
 // A broadcast-side operand of a tile, as three 16-byte records so that each loop fetches what
 // it needs with one shared-memory load.  All per-operand arithmetic that does not depend on
 // the register operand is done once, when the tile is filled:
-//   BcRing: the values a register operand (times A) must equal for + and -, and the mask and
-//           value for *:  (A*a) * b == tp (mod 2^32)  <=>  ((A*a) & mask) == tm, where
+//   BcRing: t_add = the value a register operand (times A) must have for +; t_pm = the
+//           sign-free form that covers + and - in one comparison (see ring_pass); and the mask
+//           and value for *:  (A*a) * b == tp (mod 2^32)  <=>  ((A*a) & mask) == tm, where
 //           b = 2^k * o (o odd), mask = 2^(32-k) - 1, tm = (tp >> k) * o^-1 & mask, provided the
 //           low k bits of tp are zero (else tm lies outside the mask and nothing matches);
 //   BcDiv:  magnitudes for / and %, see div_pass;
 //   BcMeta: the value itself, and meta = index inside the tile | ctz(|value|) << 16.
-struct __align__(16) BcRing { u32 t_add, t_sub, mul_mask, mul_tm; };
+struct __align__(16) BcRing { u32 t_add, t_pm, mul_mask, mul_tm; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
@@ -636,6 +637,7 @@ __device__ __forceinline__ u32 rotr32(u32 x, u32 k) { return __funnelshift_r(x, 
 // The register-side operands of a tile as the 32-bit loops use them.
 struct RegOps {
     u32 aA[kNA];     // A * value (the affine context's factor folded in)
+    u32 ca[kNA];     // sign-free form of A * value (SWAP) or of A * value - tp, for the joint +/- test
     u32 ua[kNA];     // |value|
     u32 neg;         // bit j: value j is negative
     // register operand as DIVISOR (SWAP), magnitudes only:
@@ -651,32 +653,43 @@ struct RegOps {
 // set, instead of sharing one large frame with the rest of the kernel.
 // `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
 
+// x and -x have the same sign-free form: the smaller of the two as unsigned numbers.
+__device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x < y ? x : y; }
+
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
 // MASK: bit0 +, bit1 -, bit2 *.  The comparisons were brought to the register operand's side
 // when the tile was filled (tp = low 32 bits of target - B):
-//   A*(a + b) == tp  <=>  A*a == tp - A*b;    A*(a - b) == tp  <=>  A*a == tp + A*b;
-//   A*(b - a) == tp  <=>  A*a == A*b - tp;    A*(a * b) == tp  <=>  ((A*a) & mask) == tm.
-template <u32 MASK>
-__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, int s0, int s1, u32 opip) {
-    u32 aA[kNA];
+//   A*(a + b) == tp  <=>  A*a == tp - A*b  (= t_add);   A*(a * b) == tp  <=>  ((A*a) & mask) == tm;
+//   A*(a - b) == tp  <=>  A*a == tp + A*b;              A*(b - a) == tp  <=>  A*a == A*b - tp.
+// When + and - are both present they share one comparison: without SWAP the two wanted values
+// are tp -+ A*b, i.e. A*a - tp == -+ A*b; with SWAP they are +-(tp - A*b).  Either way the pair
+// hits iff the sign-free forms agree: ca == t_pm.  Which of the two hit is settled in the rare
+// path, from t_add.
+template <u32 MASK, bool SWAP>
+__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tp, int s0, int s1, u32 opip) {
+    constexpr bool kPair = (MASK & 3u) == 3u;
+    u32 aA[kNA], ca[kNA];
 #pragma unroll
-    for (int j = 0; j < kNA; ++j) aA[j] = Rm->aA[j];
+    for (int j = 0; j < kNA; ++j) { aA[j] = Rm->aA[j]; ca[j] = Rm->ca[j]; }
+    auto t_sub_of = [&](u32 t_add) { return SWAP ? 0u - t_add : 2u * tp - t_add; };
     auto scan = [&](const BcRing& e, bool& h0, bool& h1, bool& h2, bool& h3) {
+        const u32 t_one = (MASK & 1u) ? e.t_add : t_sub_of(e.t_add);       // used when only one of + - is present
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
-            if (MASK & 1u) { h0 |= aA[j] == e.t_add; h1 |= aA[j + 1] == e.t_add; }
-            if (MASK & 2u) { h2 |= aA[j] == e.t_sub; h3 |= aA[j + 1] == e.t_sub; }
+            if (kPair) { h0 |= ca[j] == e.t_pm; h3 |= ca[j + 1] == e.t_pm; }
+            else if (MASK & 3u) { h0 |= aA[j] == t_one; h3 |= aA[j + 1] == t_one; }
             if (MASK & 4u) { h1 |= (aA[j] & e.mul_mask) == e.mul_tm; h2 |= (aA[j + 1] & e.mul_mask) == e.mul_tm; }
         }
     };
     auto resolve = [&](int s) {                          // the rare path: which candidates hit
         const BcRing e = sh.bc_ring[s];
+        const u32 t_sub = t_sub_of(e.t_add);
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
             const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
             if ((MASK & 1u) && aA[j] == e.t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
-            if ((MASK & 2u) && aA[j] == e.t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
+            if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
             if ((MASK & 4u) && (aA[j] & e.mul_mask) == e.mul_tm) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
         }
     };
@@ -863,6 +876,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         const i32 v = (i32)a64[j];
         const u32 ua = abs_u32(v);
         R.aA[j] = (u32)v * A;
+        R.ca[j] = signfree(SWAP ? R.aA[j] : R.aA[j] - tp);
         R.ua[j] = ua;
         if (v < 0) R.neg |= 1u << j;
         R.low[j] = 0x80000000u; R.inv[j] = 1u; R.kk[j] = 0u; R.cc[j] = 0u;
@@ -883,7 +897,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_pass<M>(sh, &R, alv, s0, s1, opip); break;
+#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
@@ -977,7 +991,7 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan,
         BcRing r;
         const u32 bA = b * fA;
         r.t_add = ftp - bA;
-        r.t_sub = swap ? bA - ftp : ftp + bA;
+        r.t_pm = signfree(swap ? r.t_add : bA);
         if (ub == 0u) { r.mul_mask = 0u; r.mul_tm = ftp == 0u ? 0u : 1u; }
         else {
             r.mul_mask = 0xffffffffu >> k;
