@@ -421,18 +421,21 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         if (tmax == 0 || total == 0) continue;
         void* pv = nullptr;
         void* pk = nullptr;
-        XP_CUDA_S(cudaMalloc(&pv, sizeof(i64) * total));
+        const int probes = o.n_probe >= 2 ? 2 : 1;
+        XP_CUDA_S(cudaMalloc(&pv, sizeof(i64) * total * probes));
         s->owned.push_back(pv);
-        XP_CUDA_S(cudaMalloc(&pk, total));
+        XP_CUDA_S(cudaMalloc(&pk, total * probes));
         s->owned.push_back(pk);
         o.tab_val = (i64*)pv;
         o.tab_ok = (unsigned char*)pk;
         o.tab_max_size = tmax;
+        o.tab_probes = probes;
+        o.tab_total = total;
         XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &o, sizeof(HoleDev), cudaMemcpyHostToDevice));
         for (int k = 1; k <= tmax; ++k) {
             u64 at_size = 0;
             for (int nt = 0; nt < g->n_nt; ++nt) at_size += g->cnt[nt][k];
-            XP_CUDA_S(launch_subvalues(s->d_s, h, k, at_size, nullptr));
+            for (int pr = 0; pr < probes; ++pr) XP_CUDA_S(launch_subvalues(s->d_s, h, k, pr, at_size, nullptr));
         }
     }
     // Points of a box and values of spec expressions, staged once so that the whole-domain

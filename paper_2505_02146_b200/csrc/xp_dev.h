@@ -62,13 +62,16 @@ struct HoleDev {
     // Context at probe 0 as an affine map of the hole value, ctx(h) = aff_A * h + aff_B in
     // wrap-around arithmetic (possible when the hole only passes through + - * with
     // hole-free operands); aff_ok == 0: not of that form, the probe filter is not used.
-    i32 aff_ok, pad1;
-    u64 aff_A, aff_B;
+    i32 aff_ok, aff_ok1;                          // aff_ok1: the same holds at probe 1, with aff_A1, aff_B1
+    u64 aff_A, aff_B, aff_A1, aff_B1;
     // Values at probe 0 of every subtree of the small sizes 1..tab_max_size, by (nonterminal,
     // size, rank): tab_val[tab_off[nt][size] + rank], with tab_ok telling whether the subtree
     // is defined there (no zero divisor).  Built bottom-up once per sketch; operands of the
     // filter stage are looked up here instead of being unranked again in every tile.
-    i32 tab_max_size, pad2;
+    // tab_probes == 2: a second copy of the tables for probe 1 follows at offset tab_total; hits of the
+    // filter are screened there (two lookups and one operation) before they are unranked in full.
+    i32 tab_max_size, tab_probes;
+    u64 tab_total;
     u64 tab_off[kMaxNt][kMaxSize + 1];
     i64* tab_val;                                 // device
     unsigned char* tab_ok;                        // device

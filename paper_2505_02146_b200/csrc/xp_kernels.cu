@@ -166,6 +166,10 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
             hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
             hole->aff_A = A;
             hole->aff_B = B;
+            u64 A1 = 0, B1 = 0;
+            hole->aff_ok1 = (n > 1 && ctx_affine(hole, hole->probe_pt[1], A1, B1)) ? 1 : 0;
+            hole->aff_A1 = A1;
+            hole->aff_B1 = B1;
         }
     }
 }
@@ -482,19 +486,21 @@ __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, 
     else sh.q_overflow = 1u;
 }
 
-// Value of the subtree (nt, size, rank) at the hole's probe 0; false when a divisor is zero.
-// Small sizes come from the hole's subtree-value tables; a larger subtree whose operands are
-// both in the tables costs one level of unranking; anything else is unranked in full.
-__device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank, i64& v) {
+// Value of the subtree (nt, size, rank) at the hole's probe `pr` (0, or 1 when the hole has
+// tables for it); false when a divisor is zero.  Small sizes come from the hole's subtree-value
+// tables; a larger subtree whose operands are both in the tables costs one level of unranking;
+// anything else is unranked in full.
+__device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int pr, int nt, int size, u64 rank, i64& v) {
     const int tmax = hole->tab_max_size;
+    const u64 pbase = pr ? hole->tab_total : 0ull;
     if (size <= tmax) {
-        const u64 at = hole->tab_off[nt][size] + rank;
+        const u64 at = pbase + hole->tab_off[nt][size] + rank;
         v = hole->tab_val[at];
         return hole->tab_ok[at] != 0;
     }
     if (size == 1) {
         const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)rank];
-        v = lf.var >= 0 ? hole->probe_pt[0][lf.var] : lf.value;
+        v = lf.var >= 0 ? hole->probe_pt[pr][lf.var] : lf.value;
         return true;
     }
     if (tmax >= 1) {
@@ -502,14 +508,14 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
         u64 l, r;
         unrank_root(g, nt, size, rank, op, lnt, rnt, a, l, r);
         if (a <= tmax && size - 1 - a <= tmax) {
-            const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;
+            const u64 la = pbase + hole->tab_off[lnt][a] + l, ra = pbase + hole->tab_off[rnt][size - 1 - a] + r;
             if (!hole->tab_ok[la] || !hole->tab_ok[ra]) return false;
             return apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
         }
     }
     u32 code[kMaxSize];
     const int n = unrank(g, nt, size, rank, code);
-    return eval_cand(code, n, g->leaves, hole->probe_pt[0], v);
+    return eval_cand(code, n, g->leaves, hole->probe_pt[pr], v);
 }
 
 // Values at probe 0 of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
@@ -553,7 +559,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
         if (j == n) return alive;
         for (; j < n; ++j) {
             i64 v;
-            if (operand_value(g, hole, nt, size, rank + j, v)) {
+            if (operand_value(g, hole, 0, nt, size, rank + j, v)) {
                 out[j] = v; alive |= 1u << j;
                 wide |= !(v > -(1ll << 31) && v < (1ll << 31));
             }
@@ -562,7 +568,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
     }
     for (int j = 0; j < n; ++j) {
         i64 v;
-        if (operand_value(g, hole, nt, size, rank + j, v)) {
+        if (operand_value(g, hole, 0, nt, size, rank + j, v)) {
             out[j] = v; alive |= 1u << j;
             wide |= !(v > -(1ll << 31) && v < (1ll << 31));
         }
@@ -599,9 +605,10 @@ __global__ void __launch_bounds__(256) stage_spec_kernel(const SketchDev* sk, in
 
 // Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
 // rank); the operands' values come from the smaller sizes built by earlier launches.
-__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size) {
+__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size, int pr) {
     const GrammarDev* g = sk->g;
     HoleDev* hole = &sk->holes[hole_index];
+    const u64 pbase = pr ? hole->tab_total : 0ull;
     u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
     for (int nt = 0; nt < g->n_nt; ++nt) {
         const u64 c = g->cnt[nt][size];
@@ -610,15 +617,15 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int 
         bool ok = true;
         if (size == 1) {
             const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)idx];
-            v = lf.var >= 0 ? hole->probe_pt[0][lf.var] : lf.value;
+            v = lf.var >= 0 ? hole->probe_pt[pr][lf.var] : lf.value;
         } else {
             int op, lnt, rnt, a;
             u64 l, r;
             unrank_root(g, nt, size, idx, op, lnt, rnt, a, l, r);
-            const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;
+            const u64 la = pbase + hole->tab_off[lnt][a] + l, ra = pbase + hole->tab_off[rnt][size - 1 - a] + r;
             ok = hole->tab_ok[la] && hole->tab_ok[ra] && apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
         }
-        const u64 at = hole->tab_off[nt][size] + idx;
+        const u64 at = pbase + hole->tab_off[nt][size] + idx;
         hole->tab_val[at] = v;
         hole->tab_ok[at] = ok ? 1 : 0;
         return;
@@ -830,6 +837,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
     const GrammarDev* g = sk->g;
     __syncthreads();
     const u32 nq = sh.q_n < (u32)kQueueCap ? sh.q_n : (u32)kQueueCap;
+    const bool screen1 = hole->tab_probes == 2 && hole->aff_ok1 && ((hole->probe_spec_ok >> 1) & 1u);
     for (u32 base = 0; base < nq; base += kMaxSurvivors) {
         for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
             const u32 e = sh.queue[i];
@@ -838,6 +846,14 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
             const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
             if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
+            if (screen1) {                               // exact value at probe 1 from the operand tables
+                ++my_evals;
+                i64 rv, bv, v;
+                if (!operand_value(g, hole, 1, seg.reg_nt, seg.reg_size, rr, rv)) continue;
+                if (!operand_value(g, hole, 1, seg.bc_nt, seg.bc_size, br, bv)) continue;
+                if (!apply_op(seg.op[e >> 21], seg.swap ? bv : rv, seg.swap ? rv : bv, v)) continue;
+                if ((u64)v * hole->aff_A1 + hole->aff_B1 != (u64)hole->probe_spec[1]) continue;
+            }
             u32 code[kMaxSize];
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
             if (probe_check(g, hole, code, n, my_evals)) {
@@ -976,7 +992,7 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan,
     bool wide = false;
     for (int i = threadIdx.x; i < n_bc; i += kThreads) {
         i64 v;
-        if (!operand_value(g, hole, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
+        if (!operand_value(g, hole, 0, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
         const bool special = v >= -1 && v <= 1;
         const u32 slot = special ? (u32)kBcTile - 1u - atomicAdd(&sh.bc_nspecial, 1u) : atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
@@ -1197,9 +1213,9 @@ cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, u64 n_entries, cudaStream_t stream) {
+cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int probe, u64 n_entries, cudaStream_t stream) {
     if (n_entries == 0) return cudaSuccess;
-    subvalue_kernel<<<(unsigned)((n_entries + 255) / 256), 256, 0, stream>>>(s, hole_index, size);
+    subvalue_kernel<<<(unsigned)((n_entries + 255) / 256), 256, 0, stream>>>(s, hole_index, size, probe);
     return cudaGetLastError();
 }
 
