@@ -567,10 +567,35 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
             if (bd.op == XP_OP_DIV || bd.op == XP_OP_MOD) sg->has_div = 1;
         }
     }
+    // Families: segments with the same register-side operands and a single broadcast tile are
+    // put next to each other; the first takes the tickets (one per register tile) and visits
+    // the others, so the register operands are fetched once for all of them.
+    std::vector<SegDev> ordered;
+    std::vector<char> placed(plan->segs.size() - first_seg, 0);
+    for (size_t i = first_seg; i < plan->segs.size(); ++i) {
+        if (placed[i - first_seg]) continue;
+        const SegDev head = plan->segs[i];
+        placed[i - first_seg] = 1;
+        const size_t at = ordered.size();
+        ordered.push_back(head);
+        int members = 1;
+        if (head.bc_tiles == 1)
+            for (size_t j = i + 1; j < plan->segs.size(); ++j) {
+                const SegDev& c = plan->segs[j];
+                if (placed[j - first_seg] || c.bc_tiles != 1 || c.reg_nt != head.reg_nt || c.reg_size != head.reg_size ||
+                    c.reg_begin != head.reg_begin || c.reg_count != head.reg_count) continue;
+                placed[j - first_seg] = 1;
+                ordered.push_back(c);
+                ordered.back().family = 0;
+                ++members;
+            }
+        ordered[at].family = members;
+    }
+    for (size_t i = 0; i < ordered.size(); ++i) plan->segs[first_seg + i] = ordered[i];
     for (size_t i = first_seg; i < plan->segs.size(); ++i) {
         SegDev& c = plan->segs[i];
-        c.first_ticket = plan->n_tickets;
-        plan->n_tickets += (u64)c.reg_tiles * c.bc_tiles;
+        c.first_ticket = plan->n_tickets;                          // members: where the next head starts
+        if (c.family >= 1) plan->n_tickets += (u64)c.reg_tiles * c.bc_tiles;
         // cost model: operation + comparison per evaluation; / and % share one reciprocal division
         u64 per_pair = 0;
         bool div = false, mod = false;

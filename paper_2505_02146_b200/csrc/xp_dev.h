@@ -116,7 +116,9 @@ struct SegDev {
     u64 right_count;                 // trees of the right operand (rank = base + l * right_count + r)
     u32 reg_tiles, bc_tiles;         // tickets = reg_tiles * bc_tiles
     i32 has_div;                     // some production of the group is / or %
-    i32 pad;
+    i32 family;                      // tile segments that share the register-side operands sit next to each
+                                     // other: the first holds the tickets and the count of them (>= 1), the
+                                     // others (family == 0) are visited by its tickets, one fill for all
 };
 
 // A candidate that passed every probe point and waits for the whole-domain check.  The check

@@ -214,6 +214,7 @@ struct CandShared {
 
 struct EvalShared {
     u64 ticket;
+    i32 seg_index;
     SegDev seg;
     // survivors of the probe stage, waiting for the whole-domain check
     u32 n_surv, n_pass;          // entries of surv_rank; candidates that passed the probes since the last tally
@@ -967,24 +968,11 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     (void)n_reg;
 }
 
-__device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
-                                            u64 local, u64& my_evals) {
+// Fills the broadcast side of a tile: operand values at probe 0, with everything the loops
+// need that depends on them alone.  Returns (per thread) whether a value did not fit int32.
+__device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, u64 bc_first, int n_bc) {
     const SegDev& seg = sh.seg;
-    const GrammarDev* g = sk->g;
-    if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
-    const u64 reg_tile = local / seg.bc_tiles, bc_tile = local % seg.bc_tiles;
-    const u64 reg_first = seg.reg_begin + reg_tile * (u64)kRegTile;
-    const u64 bc_first = seg.bc_begin + bc_tile * (u64)kBcTile;
-    const u64 reg_left = seg.reg_begin + seg.reg_count - reg_first;
-    const u64 bc_left = seg.bc_begin + seg.bc_count - bc_first;
-    const int n_reg = reg_left < (u64)kRegTile ? (int)reg_left : kRegTile;
-    const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
     const bool swap = seg.swap != 0;
-
-    if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
-    __syncthreads();
-
-    // operand values at probe 0, with everything the loops need that depends on them alone
     const u32 fA = (u32)hole->aff_A;
     const u64 ftq = (u64)hole->probe_spec[0] - hole->aff_B;
     const u32 ftp = (u32)ftq;
@@ -1027,15 +1015,50 @@ __device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan,
         }
         sh.bc_div[slot] = d;
     }
+    return wide;
+}
+
+// Copies segment `index` of the plan into shared memory with the first warp.
+__device__ __forceinline__ void load_segment(EvalShared& sh, const PlanDev& plan, int index) {
+    if (threadIdx.x < 32) {
+        const u32* src = (const u32*)&plan.segs[index];
+        u32* dst = (u32*)&sh.seg;
+        for (int w = threadIdx.x; w < (int)(sizeof(SegDev) / 4); w += 32) dst[w] = src[w];
+    }
+}
+
+__device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
+                                            u64 local, u64& my_evals) {
+    const GrammarDev* g = sk->g;
+    if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
+    // the register side: the same for every member of the segment's family
+    const int family = sh.seg.family > 1 ? sh.seg.family : 1;
+    const int seg_index = sh.seg_index;
+    const u64 reg_tile = local / sh.seg.bc_tiles, bc_tile0 = local % sh.seg.bc_tiles;
+    const u64 reg_first = sh.seg.reg_begin + reg_tile * (u64)kRegTile;
+    const u64 reg_left = sh.seg.reg_begin + sh.seg.reg_count - reg_first;
+    const int n_reg = reg_left < (u64)kRegTile ? (int)reg_left : kRegTile;
     i64 a64[kNA];
+    bool wide_reg = false;
     const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
-    const u32 alive = fill_reg_operands(g, hole, seg.reg_nt, seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
-                                        mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide);
-    if (wide) sh.tile_wide = 1;
-    __syncthreads();
-    if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
-    if (swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
-    else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+    const u32 alive = fill_reg_operands(g, hole, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+                                        mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
+    for (int m = 0; m < family; ++m) {
+        __syncthreads();
+        if (m > 0) load_segment(sh, plan, seg_index + m);
+        if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
+        __syncthreads();
+        const SegDev& seg = sh.seg;
+        const u64 bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
+        const u64 bc_left = seg.bc_begin + seg.bc_count - bc_first;
+        const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
+        const bool wide_bc = fill_bc_operands(sh, g, hole, bc_first, n_bc);
+        if (wide_reg || wide_bc) sh.tile_wide = 1;
+        __syncthreads();
+        if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+    }
 }
 
 #ifndef XP_MIN_CTAS
@@ -1048,21 +1071,27 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     if (threadIdx.x == 0) { sh.cur_acc = -1; sh.n_surv = 0; sh.n_pass = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
     __syncthreads();
     for (;;) {
-        if (threadIdx.x == 0) {
-            const u64 t = atomicAdd(plan.ticket, 1ull);
-            sh.ticket = t;
-            if (t < plan.n_tickets) {
-                int lo = 0, hi = plan.n_segs - 1;             // last segment with first_ticket <= t
-                while (lo < hi) {
-                    const int mid = (lo + hi + 1) >> 1;
-                    if (plan.segs[mid].first_ticket <= t) lo = mid; else hi = mid - 1;
-                }
-                sh.seg = plan.segs[lo];
-            }
-        }
+        if (threadIdx.x == 0) sh.ticket = atomicAdd(plan.ticket, 1ull);
         __syncthreads();
         const u64 t = sh.ticket;
         if (t >= plan.n_tickets) break;
+        if (threadIdx.x < 32) {
+            // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
+            int lo = 0, n = plan.n_segs;
+            while (n > 1) {
+                const int step = (n + 31) / 32;
+                const int pos = lo + (int)threadIdx.x * step;
+                const bool le = pos < lo + n && plan.segs[pos].first_ticket <= t;
+                const u32 mask = __ballot_sync(0xffffffffu, le);          // lane 0 always holds
+                const int k = 31 - __clz((int)(mask | 1u));
+                const int nlo = lo + k * step;
+                n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
+                lo = nlo;
+            }
+            if (threadIdx.x == 0) sh.seg_index = lo;
+            load_segment(sh, plan, lo);
+        }
+        __syncthreads();
         if (sh.seg.acc != sh.cur_acc) {
             flush_acc(sh, plan, my_evals);
             if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
