@@ -5,6 +5,7 @@
 #include <climits>
 #include <chrono>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -517,6 +518,8 @@ static void add_linear(Plan* plan, int sketch, int hole, int acc, int k, u64 lo,
     plan->n_tickets += (hi - lo + (u64)kLinearChunk - 1) / (u64)kLinearChunk;
 }
 
+constexpr u64 kFamilyMaxWork = 512;          // candidates per register operand below which segments share a fill
+
 // Tile segments of (start nonterminal, size k) restricted to ranks [lo, hi): one per
 // (left size, group of productions with the same operand nonterminals and the same rows).
 static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int hole, int acc, int k, u64 lo, u64 hi) {
@@ -579,10 +582,11 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
         const size_t at = ordered.size();
         ordered.push_back(head);
         int members = 1;
-        if (head.bc_tiles == 1)
+        // (worth it only for segments with little work per register operand: the fill is then a large share)
+        if (head.bc_tiles == 1 && head.bc_count * (u64)head.n_ops < kFamilyMaxWork)
             for (size_t j = i + 1; j < plan->segs.size(); ++j) {
                 const SegDev& c = plan->segs[j];
-                if (placed[j - first_seg] || c.bc_tiles != 1 || c.reg_nt != head.reg_nt || c.reg_size != head.reg_size ||
+                if (placed[j - first_seg] || c.bc_tiles != 1 || c.bc_count * (u64)c.n_ops >= kFamilyMaxWork || c.reg_nt != head.reg_nt || c.reg_size != head.reg_size ||
                     c.reg_begin != head.reg_begin || c.reg_count != head.reg_count) continue;
                 placed[j - first_seg] = 1;
                 ordered.push_back(c);

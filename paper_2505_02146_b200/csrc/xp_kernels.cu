@@ -1027,7 +1027,7 @@ __device__ __forceinline__ void load_segment(EvalShared& sh, const PlanDev& plan
     }
 }
 
-__device__ __forceinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
+__device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
                                             u64 local, u64& my_evals) {
     const GrammarDev* g = sk->g;
     if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
