@@ -422,7 +422,8 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         if (tmax == 0 || total == 0) continue;
         void* pv = nullptr;
         void* pk = nullptr;
-        const int probes = o.n_probe >= 2 ? 2 : 1;
+        int probes = o.n_probe;                      // as many probes as the table budget allows
+        while (probes > 1 && total * 9 * (u64)probes > kTabBudgetBytes) --probes;
         XP_CUDA_S(cudaMalloc(&pv, sizeof(i64) * total * probes));
         s->owned.push_back(pv);
         XP_CUDA_S(cudaMalloc(&pk, total * probes));
@@ -436,7 +437,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         for (int k = 1; k <= tmax; ++k) {
             u64 at_size = 0;
             for (int nt = 0; nt < g->n_nt; ++nt) at_size += g->cnt[nt][k];
-            for (int pr = 0; pr < probes; ++pr) XP_CUDA_S(launch_subvalues(s->d_s, h, k, pr, at_size, nullptr));
+            XP_CUDA_S(launch_subvalues(s->d_s, h, k, probes, at_size, nullptr));
         }
     }
     // Points of a box and values of spec expressions, staged once so that the whole-domain
@@ -651,7 +652,13 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
     return XP_OK;
 }
 
-constexpr u32 kSurvCap = 65536;              // survivor queue entries of a call with its own workspace
+constexpr u32 kSurvCap = 65536;              // survivor queue entries of a call with its own workspace (at least)
+
+// Batches get 256 entries per sketch, up to 2^20.
+static u32 surv_cap_for(size_t n_sketches) {
+    const size_t want = n_sketches * 256;
+    return (u32)(want < kSurvCap ? kSurvCap : (want > (1u << 20) ? (1u << 20) : want));
+}
 constexpr u32 kSurvCapStatic = 8192;         // ... of a call on the library's fixed scratch
 
 static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap) {
@@ -677,7 +684,7 @@ extern "C" size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n,
     if (!sketches || n == 0) return 0;
     Plan plan;
     if (build_plan(sketches, n, opts ? opts : &kDefaultOpts, &plan) != XP_OK) return 0;
-    return ws_layout(plan.segs.size(), n, plan.acc.size(), kSurvCap).total;
+    return ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n)).total;
 }
 
 extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
@@ -693,7 +700,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
-    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), kSurvCap);
+    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
     char* ws = (char*)o->workspace;
     bool own_ws = false;
     if (ws) {

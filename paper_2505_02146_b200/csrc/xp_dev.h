@@ -28,6 +28,7 @@ constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
 constexpr int kBcTile = 512;          // broadcast-side operands per tile
 constexpr u64 kStageMaxPoints = 1ull << 26;  // largest box whose points and spec values are staged in HBM at load
 constexpr int kProgMax = 96;          // candidate substituted into its context: longest staged program
+constexpr u64 kTabBudgetBytes = 64ull << 20;   // subtree-value tables of one hole, all probes together
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 
@@ -62,14 +63,17 @@ struct HoleDev {
     // Context at probe 0 as an affine map of the hole value, ctx(h) = aff_A * h + aff_B in
     // wrap-around arithmetic (possible when the hole only passes through + - * with
     // hole-free operands); aff_ok == 0: not of that form, the probe filter is not used.
-    i32 aff_ok, aff_ok1;                          // aff_ok1: the same holds at probe 1, with aff_A1, aff_B1
-    u64 aff_A, aff_B, aff_A1, aff_B1;
+    i32 aff_ok;
+    u32 aff_okmask;                               // bit j: the context is affine in the hole at probe j too,
+    u64 aff_A, aff_B;                             //        ctx(h) = aff_Aj[j] * h + aff_Bj[j]
+    u64 aff_Aj[kMaxProbe], aff_Bj[kMaxProbe];
     // Values at probe 0 of every subtree of the small sizes 1..tab_max_size, by (nonterminal,
     // size, rank): tab_val[tab_off[nt][size] + rank], with tab_ok telling whether the subtree
     // is defined there (no zero divisor).  Built bottom-up once per sketch; operands of the
     // filter stage are looked up here instead of being unranked again in every tile.
-    // tab_probes == 2: a second copy of the tables for probe 1 follows at offset tab_total; hits of the
-    // filter are screened there (two lookups and one operation) before they are unranked in full.
+    // The tables exist for the probes 0 .. tab_probes-1, one copy after the other (stride tab_total).
+    // Hits of the filter are checked exactly there (two lookups and one operation per probe); only
+    // probes without tables need the candidate unranked in full.
     i32 tab_max_size, tab_probes;
     u64 tab_total;
     u64 tab_off[kMaxNt][kMaxSize + 1];

@@ -166,10 +166,14 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
             hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
             hole->aff_A = A;
             hole->aff_B = B;
-            u64 A1 = 0, B1 = 0;
-            hole->aff_ok1 = (n > 1 && ctx_affine(hole, hole->probe_pt[1], A1, B1)) ? 1 : 0;
-            hole->aff_A1 = A1;
-            hole->aff_B1 = B1;
+            u32 okmask = 0;
+            for (int j = 0; j < n; ++j) {
+                u64 Aj = 0, Bj = 0;
+                if (ctx_affine(hole, hole->probe_pt[j], Aj, Bj)) okmask |= 1u << j;
+                hole->aff_Aj[j] = Aj;
+                hole->aff_Bj[j] = Bj;
+            }
+            hole->aff_okmask = okmask;
         }
     }
 }
@@ -487,13 +491,13 @@ __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, 
     else sh.q_overflow = 1u;
 }
 
-// Value of the subtree (nt, size, rank) at the hole's probe `pr` (0, or 1 when the hole has
-// tables for it); false when a divisor is zero.  Small sizes come from the hole's subtree-value
+// Value of the subtree (nt, size, rank) at the hole's probe `pr` (one the hole has tables
+// for); false when a divisor is zero.  Small sizes come from the hole's subtree-value
 // tables; a larger subtree whose operands are both in the tables costs one level of unranking;
 // anything else is unranked in full.
 __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int pr, int nt, int size, u64 rank, i64& v) {
     const int tmax = hole->tab_max_size;
-    const u64 pbase = pr ? hole->tab_total : 0ull;
+    const u64 pbase = (u64)pr * hole->tab_total;
     if (size <= tmax) {
         const u64 at = pbase + hole->tab_off[nt][size] + rank;
         v = hole->tab_val[at];
@@ -606,10 +610,11 @@ __global__ void __launch_bounds__(256) stage_spec_kernel(const SketchDev* sk, in
 
 // Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
 // rank); the operands' values come from the smaller sizes built by earlier launches.
-__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size, int pr) {
+__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size) {
+    const int pr = blockIdx.y;                          // one grid row per probe
     const GrammarDev* g = sk->g;
     HoleDev* hole = &sk->holes[hole_index];
-    const u64 pbase = pr ? hole->tab_total : 0ull;
+    const u64 pbase = (u64)pr * hole->tab_total;
     u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
     for (int nt = 0; nt < g->n_nt; ++nt) {
         const u64 c = g->cnt[nt][size];
@@ -838,7 +843,9 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
     const GrammarDev* g = sk->g;
     __syncthreads();
     const u32 nq = sh.q_n < (u32)kQueueCap ? sh.q_n : (u32)kQueueCap;
-    const bool screen1 = hole->tab_probes == 2 && hole->aff_ok1 && ((hole->probe_spec_ok >> 1) & 1u);
+    // probes 0 .. n_tab-1 can be checked from the tables: the spec is defined and the context affine there
+    int n_tab = 0;
+    while (n_tab < hole->tab_probes && n_tab < hole->n_probe && ((hole->probe_spec_ok & hole->aff_okmask) >> n_tab & 1u)) ++n_tab;
     for (u32 base = 0; base < nq; base += kMaxSurvivors) {
         for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
             const u32 e = sh.queue[i];
@@ -847,13 +854,22 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
             const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
             if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
-            if (screen1) {                               // exact value at probe 1 from the operand tables
+            // exact values at the probes that have operand tables: two lookups (or one level of
+            // unranking over the tables) and one operation each
+            bool dead = false;
+            for (int j = 0; j < n_tab && !dead; ++j) {
                 ++my_evals;
                 i64 rv, bv, v;
-                if (!operand_value(g, hole, 1, seg.reg_nt, seg.reg_size, rr, rv)) continue;
-                if (!operand_value(g, hole, 1, seg.bc_nt, seg.bc_size, br, bv)) continue;
-                if (!apply_op(seg.op[e >> 21], seg.swap ? bv : rv, seg.swap ? rv : bv, v)) continue;
-                if ((u64)v * hole->aff_A1 + hole->aff_B1 != (u64)hole->probe_spec[1]) continue;
+                dead = !operand_value(g, hole, j, seg.reg_nt, seg.reg_size, rr, rv) ||
+                       !operand_value(g, hole, j, seg.bc_nt, seg.bc_size, br, bv) ||
+                       !apply_op(seg.op[e >> 21], seg.swap ? bv : rv, seg.swap ? rv : bv, v) ||
+                       (u64)v * hole->aff_Aj[j] + hole->aff_Bj[j] != (u64)hole->probe_spec[j];
+            }
+            if (dead) continue;
+            if (n_tab == hole->n_probe) {                // every probe checked: no need to rebuild the candidate
+                atomicAdd(&sh.n_pass, 1u);
+                push_survivor(sh, plan, rank);
+                continue;
             }
             u32 code[kMaxSize];
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
@@ -1242,9 +1258,9 @@ cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int probe, u64 n_entries, cudaStream_t stream) {
+cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int n_probes, u64 n_entries, cudaStream_t stream) {
     if (n_entries == 0) return cudaSuccess;
-    subvalue_kernel<<<(unsigned)((n_entries + 255) / 256), 256, 0, stream>>>(s, hole_index, size, probe);
+    subvalue_kernel<<<dim3((unsigned)((n_entries + 255) / 256), (unsigned)n_probes), 256, 0, stream>>>(s, hole_index, size);
     return cudaGetLastError();
 }
 

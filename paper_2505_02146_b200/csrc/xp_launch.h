@@ -10,7 +10,7 @@ namespace xp {
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream);
 cudaError_t launch_stage_points(const SketchDev* s, i64 n_points, i32* coords, cudaStream_t stream);
 cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, i64* spec, u32* bad, cudaStream_t stream);
-cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int probe, u64 n_entries, cudaStream_t stream);
+cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int n_probes, u64 n_entries, cudaStream_t stream);
 // Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
 //   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32)   -- zero at launch
 //   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
