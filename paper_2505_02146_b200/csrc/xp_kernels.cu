@@ -232,6 +232,7 @@ struct EvalShared {
     u64 warp_evals[kThreads / 32];
     // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
     // dropped), the reciprocal of each as a divisor, and the queue of filter hits
+    i32 chunk_hint;              // broadcast slots per look at the hit queue (adapts to the hit rate)
     u32 bc_n, bc_nspecial;       // general operands fill slots from 0 up, those of magnitude <= 1 from the top down
     u32 q_n, q_overflow;
     i32 tile_wide;               // some operand of the tile does not fit int32
@@ -948,38 +949,46 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     };
 
     // The broadcast operands sit in two runs of slots: the general ones from slot 0 up, the
-    // ones of magnitude <= 1 (special as divisors) from the last slot down.
+    // ones of magnitude <= 1 (special as divisors) from the last slot down.  The runs are walked
+    // in chunks of `chunk` slots with a block-wide look at the hit queue after each.  A chunk
+    // that overflows the queue (a spec that many candidates satisfy at probe 0) is forgotten and
+    // redone with a quarter of the chunk size, down to one slot and one register operand at a
+    // time (at most kThreads * 5 hits, which always fit).  The chunk size is kept per CTA from
+    // tile to tile and grows back slowly.
     const int n_special = (int)sh.bc_nspecial;
+    int chunk = sh.chunk_hint;
+    bool shrunk = false;
     u32 q_start = 0;                                    // queue length when the current chunk began
     for (int part = 0; part < 2; ++part) {
         const int lo = part == 0 ? 0 : kBcTile - n_special, hi = part == 0 ? nb : kBcTile;
-        for (int s0 = lo; s0 < hi; s0 += kChunkB) {
-            const int s1 = s0 + kChunkB < hi ? s0 + kChunkB : hi;
+        int s0 = lo;
+        while (s0 < hi) {
+            const int s1 = s0 + chunk < hi ? s0 + chunk : hi;
             run(s0, s1, alive, part == 1);
             __syncthreads();
             const u32 qn = sh.q_n;
             const bool overflow = sh.q_overflow != 0;
             __syncthreads();
             if (overflow) {
-                // More hits than the queue holds (a spec that most candidates satisfy at probe 0).
-                // Forget this chunk's hits, empty the queue, and redo the chunk one broadcast slot
-                // and one register operand at a time: at most kThreads * 5 hits per step.
                 if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
                 drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
-                for (int s = s0; s < s1; ++s)
-                    for (int j = 0; j < kNA; ++j) {
-                        run(s, s + 1, alive & (1u << j), part == 1);
-                        drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
-                    }
                 q_start = 0;
+                shrunk = true;
+                if (chunk > 1) { chunk = chunk / 4 > 1 ? chunk / 4 : 1; continue; }
+                for (int j = 0; j < kNA; ++j) {
+                    run(s0, s0 + 1, alive & (1u << j), part == 1);
+                    drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
+                }
             } else if (qn > (u32)(kQueueCap / 2)) {
                 drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 q_start = 0;
             } else {
                 q_start = qn;
             }
+            s0 = s1;
         }
     }
+    if (threadIdx.x == 0) sh.chunk_hint = shrunk ? chunk : (chunk * 2 < kChunkB ? chunk * 2 : kChunkB);
     drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
     (void)n_reg;
 }
@@ -1084,7 +1093,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.n_surv = 0; sh.n_pass = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.chunk_hint = kChunkB; sh.n_surv = 0; sh.n_pass = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) sh.ticket = atomicAdd(plan.ticket, 1ull);
