@@ -352,32 +352,42 @@ __device__ __forceinline__ bool run_program(const CandShared& c, const i32* __re
 // Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
 // and the program runs on a register stack.  Otherwise coordinates are derived from the point
 // id and the interpreters with a stack in local memory are used.
-template <int D>
+// WIDE = true: the whole CTA works on the range (kThreads points per step, block-wide vote);
+// WIDE = false: one warp does (32 points per step, warp vote), other warps are not involved.
+template <bool WIDE>
+__device__ __forceinline__ bool any_bad(bool bad) {
+    return WIDE ? (__syncthreads_or(bad) != 0) : (__any_sync(0xffffffffu, bad) != 0);
+}
+
+template <int D, bool WIDE>
 __device__ __forceinline__ bool check_points_fast(const CandShared& c, const SketchDev* sk, const HoleDev* hole,
                                                   i64 first, i64 last, u64& evals) {
     const int nv = sk->n_vars;
-    for (i64 base = first; base < last; base += kThreads) {
-        const i64 pid = base + threadIdx.x;
+    const int step = WIDE ? kThreads : 32, me = WIDE ? (int)threadIdx.x : (int)(threadIdx.x & 31);
+    for (i64 base = first; base < last; base += step) {
+        const i64 pid = base + me;
         bool bad = false;
         if (pid < last) {
             ++evals;
             i64 v;
             bad = !run_program<D>(c, sk->coords + pid * nv, v) || v != hole->spec_table[pid];
         }
-        if (__syncthreads_or(bad)) return false;
+        if (any_bad<WIDE>(bad)) return false;
     }
     return true;
 }
 
+template <bool WIDE>
 __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
                                           i64 last, u64& evals) {
     if (sk->coords != nullptr && hole->spec_table != nullptr && c.depth >= 1) {
-        if (c.depth <= 4) return check_points_fast<4>(c, sk, hole, first, last, evals);
-        if (c.depth <= 8) return check_points_fast<8>(c, sk, hole, first, last, evals);
+        if (c.depth <= 4) return check_points_fast<4, WIDE>(c, sk, hole, first, last, evals);
+        if (c.depth <= 8) return check_points_fast<8, WIDE>(c, sk, hole, first, last, evals);
     }
     const int n = c.cand_len;
-    for (i64 base = first; base < last; base += kThreads) {
-        const i64 pid = base + threadIdx.x;
+    const int step = WIDE ? kThreads : 32, me = WIDE ? (int)threadIdx.x : (int)(threadIdx.x & 31);
+    for (i64 base = first; base < last; base += step) {
+        const i64 pid = base + me;
         bool bad = false;
         if (pid < last) {
             ++evals;
@@ -401,7 +411,7 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
             }
             bad = !ok || !ctx_matches(hole, pt, st[0], want);
         }
-        if (__syncthreads_or(bad)) return false;
+        if (any_bad<WIDE>(bad)) return false;
     }
     return true;
 }
@@ -430,7 +440,7 @@ __device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* s
         const u64 rank = sh.surv_rank[i];
         if (threadIdx.x == 0) stage_candidate(sh.cand, g, hole, size, rank);
         __syncthreads();
-        const bool ok = check_points(sh.cand, sk, hole, 0, sk->n_points, my_evals);
+        const bool ok = check_points<true>(sh.cand, sk, hole, 0, sk->n_points, my_evals);
         if (ok && threadIdx.x == 0) {
             sh.match_count[size] += 1;
             if (rank < sh.min_rank[size]) sh.min_rank[size] = rank;
@@ -1137,48 +1147,49 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 // ------------------------------------------------------------------------------------------
 
 // Items are (chunk of points, survivor), chunk-major: the first chunk of every survivor is
-// taken before any second chunk, so candidates that fail early cost one chunk.  An item whose
-// survivor has already failed is skipped.  No CTA waits for another.
+// taken before any second chunk, so candidates that fail early cost one chunk.  Each WARP
+// takes items on its own (lane = point, 32 points per step, warp vote): nothing in this
+// kernel synchronises a CTA, and no warp waits for another.  An item whose survivor has
+// already failed is skipped; lane 0 reads that flag once and shares the decision.
 __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
-    __shared__ CandShared cand;
-    __shared__ u64 s_ticket;
-    __shared__ i32 s_skip;
+    __shared__ CandShared cands[kThreads / 32];
+    CandShared& cand = cands[threadIdx.x >> 5];
+    const int lane = threadIdx.x & 31;
     const u32 pushed = *plan.surv_n;
     const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
     const u64 total = n * plan.max_chunks;
     for (;;) {
-        __syncthreads();
-        // Thread 0 takes the item and decides for the whole CTA whether it is skipped (the
-        // survivor's state may change under other CTAs, so it is read once, by one thread).
-        if (threadIdx.x == 0) {
-            const u64 t = atomicAdd(plan.verify_ticket, 1ull);
-            s_ticket = t;
-            s_skip = 1;
+        u64 t = 0;
+        int skip = 1;
+        if (lane == 0) {
+            t = atomicAdd(plan.verify_ticket, 1ull);
             if (t < total) {
                 const SurvDev* sv = &plan.surv[t % n];
                 const SketchDev* sk = plan.sketches[sv->sketch];
                 const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
                 if ((i64)(t / n) * kVerifyChunk < sk->n_points && !failed) {
-                    s_skip = 0;
+                    skip = 0;
                     stage_candidate(cand, sk->g, &sk->holes[sv->hole], sv->size, sv->rank);
                 }
             }
         }
-        __syncthreads();
-        const u64 t = s_ticket;
+        __syncwarp();
+        t = __shfl_sync(0xffffffffu, t, 0);
+        skip = __shfl_sync(0xffffffffu, skip, 0);
         if (t >= total) break;
-        if (s_skip) continue;
+        if (skip) continue;
         SurvDev* sv = &plan.surv[t % n];
         const SketchDev* sk = plan.sketches[sv->sketch];
         const HoleDev* hole = &sk->holes[sv->hole];
         const i64 first = (i64)(t / n) * kVerifyChunk;
         const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
         u64 evals = 0;
-        const bool ok = check_points(cand, sk, hole, first, last, evals);
-        if (threadIdx.x == 0) {
+        const bool ok = check_points<false>(cand, sk, hole, first, last, evals);
+        if (lane == 0) {
             if (ok) atomicAdd(&sv->state, 1u); else atomicOr(&sv->state, kSurvFailed);
             atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
         }
+        __syncwarp();                                   // the staged candidate is free for the next item
     }
 }
 
