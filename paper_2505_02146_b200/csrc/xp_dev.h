@@ -27,7 +27,7 @@ constexpr int kNA = 8;                // tile tickets: register-side operands pe
 constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
 constexpr int kBcTile = 512;          // broadcast-side operands per tile
 constexpr u64 kStageMaxPoints = 1ull << 26;  // largest box whose points and spec values are staged in HBM at load
-constexpr int kProgMax = 96;          // candidate substituted into its context: longest staged program
+constexpr int kProgMax = 64;          // candidate substituted into its context: longest staged program
 constexpr u64 kTabBudgetBytes = 64ull << 20;   // subtree-value tables of one hole, all probes together
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index

@@ -183,11 +183,12 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
 // ------------------------------------------------------------------------------------------
 
 constexpr int kLinearPerThread = kLinearChunk / kThreads; // ranks per thread per linear ticket
-constexpr int kMaxSurvivors = kLinearChunk;
-constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check
+constexpr int kWarps = kThreads / 32;
+constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check (all warps)
+constexpr int kWarpQueue = kQueueCap / kWarps;            // ... per warp: every warp keeps and empties its own queue
 constexpr int kChunkB = 128;                              // broadcast operands between block-wide queue checks
 static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
-static_assert(kThreads * 5 <= kQueueCap / 2, "one replay step must fit the free half of the queue");
+static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the free half of its queue");
 
 // A broadcast-side operand of a tile, as three 16-byte records so that each loop fetches what
 // it needs with one shared-memory load.  All per-operand arithmetic that does not depend on
@@ -220,10 +221,7 @@ struct EvalShared {
     u64 ticket;
     i32 seg_index;
     SegDev seg;
-    // survivors of the probe stage, waiting for the whole-domain check
-    u32 n_surv, n_pass;          // entries of surv_rank; candidates that passed the probes since the last tally
-    u64 surv_rank[kMaxSurvivors];
-    CandShared cand;
+    CandShared wcand[kWarps];    // per warp: the candidate of a whole-domain check the warp does itself
     // results of the (sketch, hole) the CTA is working on
     i32 cur_acc;
     u64 match_count[kMaxSize + 1];
@@ -232,14 +230,14 @@ struct EvalShared {
     u64 warp_evals[kThreads / 32];
     // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
     // dropped), the reciprocal of each as a divisor, and the queue of filter hits
-    i32 chunk_hint;              // broadcast slots per look at the hit queue (adapts to the hit rate)
+    i32 chunk_hint[kWarps];      // broadcast slots per look at the hit queue (adapts to the hit rate)
     u32 bc_n, bc_nspecial;       // general operands fill slots from 0 up, those of magnitude <= 1 from the top down
-    u32 q_n, q_overflow;
+    u32 wq_n[kWarps], wq_over[kWarps];
     i32 tile_wide;               // some operand of the tile does not fit int32
     BcRing bc_ring[kBcTile];
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
-    u32 queue[kQueueCap];        // reg index | broadcast slot << 11 | op index << 21
+    u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
@@ -352,42 +350,40 @@ __device__ __forceinline__ bool run_program(const CandShared& c, const i32* __re
 // Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
 // and the program runs on a register stack.  Otherwise coordinates are derived from the point
 // id and the interpreters with a stack in local memory are used.
-// WIDE = true: the whole CTA works on the range (kThreads points per step, block-wide vote);
-// WIDE = false: one warp does (32 points per step, warp vote), other warps are not involved.
-template <bool WIDE>
-__device__ __forceinline__ bool any_bad(bool bad) {
-    return WIDE ? (__syncthreads_or(bad) != 0) : (__any_sync(0xffffffffu, bad) != 0);
-}
-
-template <int D, bool WIDE>
+// Stage 3 core: one WARP checks the staged candidate on the points [first, last), 32 points
+// per step; a failing point anywhere ends the scan at the next warp vote.  Returns true if
+// every point passed; adds the points tried by this lane to evals.
+// Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
+// and the program runs on a register stack.  Otherwise coordinates are derived from the point
+// id and the interpreters with a stack in local memory are used.
+template <int D>
 __device__ __forceinline__ bool check_points_fast(const CandShared& c, const SketchDev* sk, const HoleDev* hole,
                                                   i64 first, i64 last, u64& evals) {
     const int nv = sk->n_vars;
-    const int step = WIDE ? kThreads : 32, me = WIDE ? (int)threadIdx.x : (int)(threadIdx.x & 31);
-    for (i64 base = first; base < last; base += step) {
-        const i64 pid = base + me;
+    const int lane = threadIdx.x & 31;
+    for (i64 base = first; base < last; base += 32) {
+        const i64 pid = base + lane;
         bool bad = false;
         if (pid < last) {
             ++evals;
             i64 v;
             bad = !run_program<D>(c, sk->coords + pid * nv, v) || v != hole->spec_table[pid];
         }
-        if (any_bad<WIDE>(bad)) return false;
+        if (__any_sync(0xffffffffu, bad)) return false;
     }
     return true;
 }
 
-template <bool WIDE>
 __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
                                           i64 last, u64& evals) {
     if (sk->coords != nullptr && hole->spec_table != nullptr && c.depth >= 1) {
-        if (c.depth <= 4) return check_points_fast<4, WIDE>(c, sk, hole, first, last, evals);
-        if (c.depth <= 8) return check_points_fast<8, WIDE>(c, sk, hole, first, last, evals);
+        if (c.depth <= 4) return check_points_fast<4>(c, sk, hole, first, last, evals);
+        if (c.depth <= 8) return check_points_fast<8>(c, sk, hole, first, last, evals);
     }
     const int n = c.cand_len;
-    const int step = WIDE ? kThreads : 32, me = WIDE ? (int)threadIdx.x : (int)(threadIdx.x & 31);
-    for (i64 base = first; base < last; base += step) {
-        const i64 pid = base + me;
+    const int lane = threadIdx.x & 31;
+    for (i64 base = first; base < last; base += 32) {
+        const i64 pid = base + lane;
         bool bad = false;
         if (pid < last) {
             ++evals;
@@ -411,45 +407,55 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
             }
             bad = !ok || !ctx_matches(hole, pt, st[0], want);
         }
-        if (any_bad<WIDE>(bad)) return false;
+        if (__any_sync(0xffffffffu, bad)) return false;
     }
     return true;
 }
 
-// A candidate that passed the probes: into the global queue for the verification kernel, or,
-// if that is full, into the CTA's own list (checked by the CTA itself, below).
-__device__ __forceinline__ void push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank) {
+// A candidate that passed the probes goes into the global queue for the verification kernel.
+// Returns false if the queue is full: the caller's warp then checks the candidate itself.
+__device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank) {
     const u32 at = atomicAdd(plan.surv_n, 1u);
-    if (at < plan.surv_cap) {
-        SurvDev r;
-        r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
-        r.state = 0; r.pad = 0;
-        plan.surv[at] = r;
-    } else {
-        const u32 slot = atomicAdd(&sh.n_surv, 1u);
-        sh.surv_rank[slot] = rank;
+    if (at >= plan.surv_cap) return false;
+    SurvDev r;
+    r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
+    r.state = 0; r.pad = 0;
+    plan.surv[at] = r;
+    return true;
+}
+
+// The warp checks one candidate on the whole domain itself and records a match in the CTA's
+// private results.  Called by all 32 lanes together.
+__device__ __noinline__ void warp_verify(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64 rank,
+                                         u64& my_evals) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) stage_candidate(sh.wcand[warp], sk->g, hole, size, rank);
+    __syncwarp();
+    const bool ok = check_points(sh.wcand[warp], sk, hole, 0, sk->n_points, my_evals);
+    if (ok && lane == 0) {
+        atomicAdd(&sh.match_count[size], 1ull);
+        atomicMin(&sh.min_rank[size], rank);
+    }
+    __syncwarp();
+}
+
+// Lanes holding a survivor that the global queue did not take hand it to their warp, one
+// after the other.  Called by all 32 lanes together.
+__device__ __forceinline__ void warp_verify_pending(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size,
+                                                    bool pending, u64 rank, u64& my_evals) {
+    u32 m = __ballot_sync(0xffffffffu, pending);
+    while (m) {
+        const int src = __ffs((int)m) - 1;
+        m &= m - 1;
+        const u64 r = __shfl_sync(0xffffffffu, rank, src);
+        warp_verify(sh, sk, hole, size, r, my_evals);
     }
 }
 
-// Whole-domain check of the CTA's own survivor list (only used when the global queue is full).
-__device__ __noinline__ void verify_survivors(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64& my_evals) {
-    const GrammarDev* g = sk->g;
-    __syncthreads();
-    const u32 ns = sh.n_surv;
-    for (u32 i = 0; i < ns; ++i) {
-        const u64 rank = sh.surv_rank[i];
-        if (threadIdx.x == 0) stage_candidate(sh.cand, g, hole, size, rank);
-        __syncthreads();
-        const bool ok = check_points<true>(sh.cand, sk, hole, 0, sk->n_points, my_evals);
-        if (ok && threadIdx.x == 0) {
-            sh.match_count[size] += 1;
-            if (rank < sh.min_rank[size]) sh.min_rank[size] = rank;
-        }
-        __syncthreads();
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) sh.n_surv = 0;
-    __syncthreads();
+// Adds a per-lane count over the warp into a counter of the CTA's private results.
+__device__ __forceinline__ void warp_tally(u64* counter, u32 mine) {
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, o);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(counter, (u64)mine);
 }
 
 // A linear ticket: kLinearChunk consecutive ranks, each unranked and checked on its own.
@@ -458,20 +464,22 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, 
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
     const u64 first = seg.rank_begin + local * (u64)kLinearChunk;
+    u32 passes = 0;
     for (int i = 0; i < kLinearPerThread; ++i) {
         const u64 rank = first + (u64)i * kThreads + threadIdx.x;
+        bool pending = false;
         if (rank < seg.rank_end) {
             u32 code[kMaxSize];
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
             if (probe_check(g, hole, code, n, my_evals)) {
-                atomicAdd(&sh.n_pass, 1u);
-                push_survivor(sh, plan, rank);
+                ++passes;
+                pending = !push_survivor(sh, plan, rank);
             }
         }
+        warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
     }
-    __syncthreads();
-    if (threadIdx.x == 0) { sh.filter_survivors += sh.n_pass; sh.probe_survivors += sh.n_pass; sh.n_pass = 0; }
-    verify_survivors(sh, sk, hole, seg.size, my_evals);
+    warp_tally(&sh.filter_survivors, passes);
+    warp_tally(&sh.probe_survivors, passes);
 }
 
 
@@ -497,9 +505,10 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, 
 __device__ __forceinline__ u32 abs_u32(i32 x) { return x < 0 ? 0u - (u32)x : (u32)x; }
 
 __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, u32 opi) {
-    const u32 at = atomicAdd(&sh.q_n, 1u);
-    if (at < (u32)kQueueCap) sh.queue[at] = reg_idx | (slot << 11) | (opi << 21);
-    else sh.q_overflow = 1u;
+    const int warp = threadIdx.x >> 5;
+    const u32 at = atomicAdd(&sh.wq_n[warp], 1u);
+    if (at < (u32)kWarpQueue) sh.queue[warp][at] = reg_idx | (slot << 11) | (opi << 21);
+    else sh.wq_over[warp] = 1u;
 }
 
 // Value of the subtree (nt, size, rank) at the hole's probe `pr` (one the hole has tables
@@ -846,28 +855,32 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive,
     }
 }
 
-// Stage 2 over the queue: every filter hit is rebuilt as a full candidate, checked exactly on
-// the probe points (lane = candidate), and the survivors go through the whole-domain check.
+// Stage 2 over the warp's queue (lane = hit): exact values at the probes that have operand
+// tables (two lookups, or one level of unranking over the tables, and one operation each);
+// for the remaining probes the candidate is rebuilt by full unranking.  Survivors go to the
+// global queue, or are checked by the warp itself when that is full.  Called by all 32 lanes.
 __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
                                          u64 reg_first, u64 bc_first, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const GrammarDev* g = sk->g;
-    __syncthreads();
-    const u32 nq = sh.q_n < (u32)kQueueCap ? sh.q_n : (u32)kQueueCap;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncwarp();
+    const u32 nq = sh.wq_n[warp] < (u32)kWarpQueue ? sh.wq_n[warp] : (u32)kWarpQueue;
     // probes 0 .. n_tab-1 can be checked from the tables: the spec is defined and the context affine there
     int n_tab = 0;
     while (n_tab < hole->tab_probes && n_tab < hole->n_probe && ((hole->probe_spec_ok & hole->aff_okmask) >> n_tab & 1u)) ++n_tab;
-    for (u32 base = 0; base < nq; base += kMaxSurvivors) {
-        for (u32 i = base + threadIdx.x; i < nq && i < base + kMaxSurvivors; i += kThreads) {
-            const u32 e = sh.queue[i];
+    u32 passes = 0;
+    for (u32 base = 0; base < nq; base += 32) {
+        const u32 i = base + lane;
+        bool pending = false;
+        u64 rank = 0;
+        if (i < nq) {
+            const u32 e = sh.queue[warp][i];
             const u64 rr = reg_first + (e & 2047u);
             const u64 br = bc_first + (sh.bc_meta[(e >> 11) & 1023u].meta & 0xffffu);
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
-            const u64 rank = seg.op_base[e >> 21] + l * seg.right_count + r;
-            if (rank < seg.rank_begin || rank >= seg.rank_end) continue;
-            // exact values at the probes that have operand tables: two lookups (or one level of
-            // unranking over the tables) and one operation each
-            bool dead = false;
+            rank = seg.op_base[e >> 21] + l * seg.right_count + r;
+            bool dead = rank < seg.rank_begin || rank >= seg.rank_end;
             for (int j = 0; j < n_tab && !dead; ++j) {
                 ++my_evals;
                 i64 rv, bv, v;
@@ -876,25 +889,21 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
                        !apply_op(seg.op[e >> 21], seg.swap ? bv : rv, seg.swap ? rv : bv, v) ||
                        (u64)v * hole->aff_Aj[j] + hole->aff_Bj[j] != (u64)hole->probe_spec[j];
             }
-            if (dead) continue;
-            if (n_tab == hole->n_probe) {                // every probe checked: no need to rebuild the candidate
-                atomicAdd(&sh.n_pass, 1u);
-                push_survivor(sh, plan, rank);
-                continue;
+            if (!dead && n_tab < hole->n_probe) {        // some probes have no tables: rebuild the candidate
+                u32 code[kMaxSize];
+                const int n = unrank(g, hole->start_nt, seg.size, rank, code);
+                dead = !probe_check(g, hole, code, n, my_evals);
             }
-            u32 code[kMaxSize];
-            const int n = unrank(g, hole->start_nt, seg.size, rank, code);
-            if (probe_check(g, hole, code, n, my_evals)) {
-                atomicAdd(&sh.n_pass, 1u);
-                push_survivor(sh, plan, rank);
+            if (!dead) {
+                ++passes;
+                pending = !push_survivor(sh, plan, rank);
             }
         }
-        __syncthreads();
-        if (threadIdx.x == 0) { sh.probe_survivors += sh.n_pass; sh.n_pass = 0; }
-        verify_survivors(sh, sk, hole, seg.size, my_evals);
+        warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
     }
-    if (threadIdx.x == 0) { sh.filter_survivors += nq; sh.q_n = 0; }
-    __syncthreads();
+    warp_tally(&sh.probe_survivors, passes);
+    if (lane == 0) { if (nq) atomicAdd(&sh.filter_survivors, (u64)nq); sh.wq_n[warp] = 0; }
+    __syncwarp();
 }
 
 template <bool SWAP>
@@ -959,14 +968,16 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     };
 
     // The broadcast operands sit in two runs of slots: the general ones from slot 0 up, the
-    // ones of magnitude <= 1 (special as divisors) from the last slot down.  The runs are walked
-    // in chunks of `chunk` slots with a block-wide look at the hit queue after each.  A chunk
-    // that overflows the queue (a spec that many candidates satisfy at probe 0) is forgotten and
-    // redone with a quarter of the chunk size, down to one slot and one register operand at a
-    // time (at most kThreads * 5 hits, which always fit).  The chunk size is kept per CTA from
-    // tile to tile and grows back slowly.
+    // ones of magnitude <= 1 (special as divisors) from the last slot down.  Every warp walks
+    // the runs on its own, in chunks of `chunk` slots, and looks at its hit queue after each:
+    // no CTA-wide synchronisation happens inside a tile.  A chunk that overflows the queue (a
+    // spec that many candidates satisfy at probe 0) is forgotten and redone with a quarter of
+    // the chunk size, down to one slot and one register operand per lane at a time (at most
+    // 32 * 5 hits, which always fit).  The chunk size is kept per warp from tile to tile and
+    // grows back slowly.
+    const int warp = threadIdx.x >> 5;
     const int n_special = (int)sh.bc_nspecial;
-    int chunk = sh.chunk_hint;
+    int chunk = sh.chunk_hint[warp];
     bool shrunk = false;
     u32 q_start = 0;                                    // queue length when the current chunk began
     for (int part = 0; part < 2; ++part) {
@@ -975,12 +986,12 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         while (s0 < hi) {
             const int s1 = s0 + chunk < hi ? s0 + chunk : hi;
             run(s0, s1, alive, part == 1);
-            __syncthreads();
-            const u32 qn = sh.q_n;
-            const bool overflow = sh.q_overflow != 0;
-            __syncthreads();
+            __syncwarp();
+            const u32 qn = sh.wq_n[warp];
+            const bool overflow = sh.wq_over[warp] != 0;
+            __syncwarp();
             if (overflow) {
-                if (threadIdx.x == 0) { sh.q_n = q_start; sh.q_overflow = 0; }
+                if ((threadIdx.x & 31) == 0) { sh.wq_n[warp] = q_start; sh.wq_over[warp] = 0; }
                 drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 q_start = 0;
                 shrunk = true;
@@ -989,7 +1000,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
                     run(s0, s0 + 1, alive & (1u << j), part == 1);
                     drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 }
-            } else if (qn > (u32)(kQueueCap / 2)) {
+            } else if (qn > (u32)(kWarpQueue / 2)) {
                 drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 q_start = 0;
             } else {
@@ -998,7 +1009,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
             s0 = s1;
         }
     }
-    if (threadIdx.x == 0) sh.chunk_hint = shrunk ? chunk : (chunk * 2 < kChunkB ? chunk * 2 : kChunkB);
+    if ((threadIdx.x & 31) == 0) sh.chunk_hint[warp] = shrunk ? chunk : (chunk * 2 < kChunkB ? chunk * 2 : kChunkB);
     drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
     (void)n_reg;
 }
@@ -1081,7 +1092,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     for (int m = 0; m < family; ++m) {
         __syncthreads();
         if (m > 0) load_segment(sh, plan, seg_index + m);
-        if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.q_n = 0; sh.q_overflow = 0; sh.tile_wide = 0; }
+        if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.tile_wide = 0; }
         __syncthreads();
         const SegDev& seg = sh.seg;
         const u64 bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
@@ -1103,7 +1114,8 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.chunk_hint = kChunkB; sh.n_surv = 0; sh.n_pass = 0; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) sh.ticket = atomicAdd(plan.ticket, 1ull);
@@ -1152,7 +1164,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 // kernel synchronises a CTA, and no warp waits for another.  An item whose survivor has
 // already failed is skipped; lane 0 reads that flag once and shares the decision.
 __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
-    __shared__ CandShared cands[kThreads / 32];
+    __shared__ CandShared cands[kWarps];
     CandShared& cand = cands[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const u32 pushed = *plan.surv_n;
@@ -1184,7 +1196,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
         const i64 first = (i64)(t / n) * kVerifyChunk;
         const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
         u64 evals = 0;
-        const bool ok = check_points<false>(cand, sk, hole, first, last, evals);
+        const bool ok = check_points(cand, sk, hole, first, last, evals);
         if (lane == 0) {
             if (ok) atomicAdd(&sv->state, 1u); else atomicOr(&sv->state, kSurvFailed);
             atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
