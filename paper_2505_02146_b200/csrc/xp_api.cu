@@ -595,6 +595,15 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
                 ++members;
             }
         ordered[at].family = members;
+        // broadcast slots side by side when the whole family fits the tile and has one tile each
+        u64 slots = 0;
+        bool one_tile = true;
+        for (int m = 0; m < members; ++m) { slots += ordered[at + m].bc_count; one_tile = one_tile && ordered[at + m].bc_tiles == 1; }
+        if (one_tile && slots <= (u64)kBcTile && members <= 8) {
+            u64 base = 0;
+            for (int m = 0; m < members; ++m) { ordered[at + m].bc_base = (i32)base; base += ordered[at + m].bc_count; }
+            ordered[at].bc_keep = 1;
+        }
     }
     for (size_t i = 0; i < ordered.size(); ++i) plan->segs[first_seg + i] = ordered[i];
     for (size_t i = first_seg; i < plan->segs.size(); ++i) {

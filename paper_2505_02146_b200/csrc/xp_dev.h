@@ -120,6 +120,9 @@ struct SegDev {
     u64 right_count;                 // trees of the right operand (rank = base + l * right_count + r)
     u32 reg_tiles, bc_tiles;         // tickets = reg_tiles * bc_tiles
     i32 has_div;                     // some production of the group is / or %
+    i32 bc_base, bc_keep;            // slots [bc_base, bc_base + bc_count) of the CTA's broadcast tile belong to this
+                                     // segment; bc_keep (first of a family): all members' broadcast operands fit the
+                                     // tile side by side and do not depend on the ticket, so a CTA fills them once
     i32 family;                      // tile segments that share the register-side operands sit next to each
                                      // other: the first holds the tickets and the count of them (>= 1), the
                                      // others (family == 0) are visited by its tickets, one fill for all

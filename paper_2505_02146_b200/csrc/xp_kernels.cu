@@ -231,7 +231,16 @@ struct EvalShared {
     // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
     // dropped), the reciprocal of each as a divisor, and the queue of filter hits
     i32 chunk_hint[kWarps];      // broadcast slots per look at the hit queue (adapts to the hit rate)
-    u32 bc_n, bc_nspecial;       // general operands fill slots from 0 up, those of magnitude <= 1 from the top down
+    // Broadcast slots of the segment at hand: [bc_lo, bc_hi); general operands fill it from bc_lo up
+    // (bc_n of them), those of magnitude <= 1 from bc_hi down (bc_nspecial).  For a family whose
+    // members' slots lie side by side (bc_keep) the per-member counts are kept in kept_*, and
+    // kept_head names the family resident in the tile (-1: none), so the next ticket of the same
+    // family does not fill again.
+    i32 bc_lo, bc_hi;
+    u32 bc_n, bc_nspecial;
+    i32 kept_head;
+    u32 kept_n[8], kept_nspecial[8];
+    i32 kept_wide[8];
     u32 wq_n[kWarps], wq_over[kWarps];
     i32 tile_wide;               // some operand of the tile does not fit int32
     BcRing bc_ring[kBcTile];
@@ -910,7 +919,7 @@ template <bool SWAP>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
                                           u64 bc_first, int n_reg, i64* a64, u32 alive, u64& my_evals) {
     const SegDev& seg = sh.seg;
-    const int nb = (int)sh.bc_n;
+    const int nb = (int)sh.bc_n, bc_lo = sh.bc_lo, bc_hi = sh.bc_hi;
     const bool tile_wide = sh.tile_wide != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
     u32 opip = 0, mask = 0;
@@ -981,7 +990,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     bool shrunk = false;
     u32 q_start = 0;                                    // queue length when the current chunk began
     for (int part = 0; part < 2; ++part) {
-        const int lo = part == 0 ? 0 : kBcTile - n_special, hi = part == 0 ? nb : kBcTile;
+        const int lo = part == 0 ? bc_lo : bc_hi - n_special, hi = part == 0 ? bc_lo + nb : bc_hi;
         int s0 = lo;
         while (s0 < hi) {
             const int s1 = s0 + chunk < hi ? s0 + chunk : hi;
@@ -1028,7 +1037,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         i64 v;
         if (!operand_value(g, hole, 0, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
         const bool special = v >= -1 && v <= 1;
-        const u32 slot = special ? (u32)kBcTile - 1u - atomicAdd(&sh.bc_nspecial, 1u) : atomicAdd(&sh.bc_n, 1u);
+        const u32 slot = special ? (u32)sh.bc_hi - 1u - atomicAdd(&sh.bc_nspecial, 1u) : (u32)sh.bc_lo + atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
         const u32 b = (u32)(u64)v, ub = abs_u32((i32)v);
@@ -1089,17 +1098,36 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
     const u32 alive = fill_reg_operands(g, hole, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
                                         mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
+    const bool keep = sh.seg.bc_keep != 0;
+    const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
     for (int m = 0; m < family; ++m) {
         __syncthreads();
         if (m > 0) load_segment(sh, plan, seg_index + m);
-        if (threadIdx.x == 0) { sh.bc_n = 0; sh.bc_nspecial = 0; sh.tile_wide = 0; }
         __syncthreads();
         const SegDev& seg = sh.seg;
         const u64 bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
         const u64 bc_left = seg.bc_begin + seg.bc_count - bc_first;
         const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
-        const bool wide_bc = fill_bc_operands(sh, g, hole, bc_first, n_bc);
-        if (wide_reg || wide_bc) sh.tile_wide = 1;
+        if (threadIdx.x == 0) {
+            sh.bc_lo = keep ? seg.bc_base : 0;
+            sh.bc_hi = keep ? seg.bc_base + n_bc : kBcTile;
+            sh.bc_n = resident ? sh.kept_n[m] : 0;
+            sh.bc_nspecial = resident ? sh.kept_nspecial[m] : 0;
+            sh.tile_wide = resident ? sh.kept_wide[m] : 0;
+            if (!resident) sh.kept_head = -1;
+        }
+        __syncthreads();
+        if (!resident) {
+            const bool wide_bc = fill_bc_operands(sh, g, hole, bc_first, n_bc);
+            if (wide_bc) sh.tile_wide = 1;
+            __syncthreads();
+            if (threadIdx.x == 0 && keep) {
+                sh.kept_n[m] = sh.bc_n; sh.kept_nspecial[m] = sh.bc_nspecial; sh.kept_wide[m] = sh.tile_wide;
+                if (m == family - 1) sh.kept_head = seg_index;
+            }
+            __syncthreads();
+        }
+        if (wide_reg) sh.tile_wide = 1;                 // the kept flag is the broadcast side's alone
         __syncthreads();
         if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
         if (seg.swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
@@ -1114,7 +1142,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
