@@ -65,6 +65,10 @@ class ClockSampler:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
         sm = sorted(int(r[0]) for r in self.rows if r and r[0].isdigit())
         mx = [int(r[1]) for r in self.rows if len(r) > 1 and r[1].isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -176,6 +180,8 @@ def main():
         l2 = xp.xp_sketch_load(g2, sk)
         r2 = xp.xp_repair(l2, rank_ranges=rr)[0]
         e2e_evals += r2.evals_executed
+        if os.environ.get("XP_BENCH_DEBUG"):
+            print("e2e step: kernel_ms %.2f total_ms %.2f since start %.1f ms" % (r2.kernel_ms, r2.total_ms, 1e3 * (time.perf_counter() - t0)), file=sys.stderr)
         del l2, g2
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
