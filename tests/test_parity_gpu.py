@@ -92,6 +92,23 @@ def test_larger_sizes_small_grammar(xp):
         check_sketch(xp, Sketch(gq, [Hole(0, 9, spec_expr=parse_expr("((x/2)*3)+(y%4)", vs))], name="typed K9"), flags=flags)
 
 
+def test_repeated_productions_and_the_largest_size(xp):
+    """Two productions with the same operator are distinct candidates (they cannot share a
+    filter segment); size 15 is the library's limit (8 leaves, operand stack of 8)."""
+    from xp_instances.model import OP_CODE, P_BIN, Production
+    g2 = free_grammar([Variable("x", 0, 4)], [1, 2], ops=["+", "*"])
+    g2.productions.append(Production(lhs=0, kind=P_BIN, op=OP_CODE["+"], left=0, right=0))
+    sk = Sketch(g2, [Hole(0, 7, spec_expr=parse_expr("(x*2)+1", g2.variables))], name="two plus productions")
+    for flags in PATHS:
+        res = check_sketch(xp, sk, flags=flags)
+        assert res[0].cand_count == [0, 3, 0, 27, 0, 486, 0, 10935]
+    g3 = free_grammar([Variable("x", 0, 3)], [1], ops=["+"])
+    sk3 = Sketch(g3, [Hole(0, 15, spec_expr=parse_expr("((x+x)+(x+1))+((1+1)+(x+1))", g3.variables))], name="size 15")
+    for flags in PATHS:
+        res = check_sketch(xp, sk3, flags=flags)
+        assert res[0].cand_count[15] == 109824 and res[0].match_count[15] == 30030
+
+
 def test_zero_divisors_and_wraparound(xp):
     vs = [Variable("x", 0, 3)]
     for flags in PATHS:

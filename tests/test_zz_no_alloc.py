@@ -49,6 +49,19 @@ def test_static_entry_point_matches_xp_repair_on_two_calls_in_a_row(xp):
         _same(xp.xp_repair_static(lb)[0], rb[0])
 
 
+def test_static_entry_point_when_its_survivor_queue_is_full(xp):
+    """The fixed array holds a survivor queue of 8192 entries; a spec with 60 878 matches of size 5
+    overflows it, and the warps then check their survivors themselves: same counts."""
+    vs = [Variable("i", 0, 16), Variable("j", 0, 16)]
+    g = free_grammar(vs, list(range(-8, 9)))
+    ls = xp.xp_sketch_load(xp.xp_grammar_create(g), Sketch(g, [Hole(0, 5, spec_expr=parse_expr("0", vs))]))
+    ref = xp.xp_repair(ls)
+    assert ref[0].match_count == [0, 1, 0, 301, 0, 60878]
+    for _ in range(2):
+        _same(xp.xp_repair_static(ls)[0], ref[0])
+        _same(xp.xp_repair_static(ls, flags=xp.XP_FLAG_NO_FILTER)[0], ref[0])
+
+
 def test_static_entry_point_rejects_what_does_not_fit(xp):
     vs = [Variable("x", 0, 4)]
     g = free_grammar(vs, [0, 1, 2])
