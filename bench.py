@@ -126,7 +126,7 @@ def main():
     assert torch.cuda.is_available(), "bench.py needs a CUDA device: there is no CPU fallback"
     torch.cuda.set_device(local)
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torchrun: one rank per GPU over NCCL
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     xp.load()
