@@ -231,16 +231,15 @@ struct EvalShared {
     // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
     // dropped), the reciprocal of each as a divisor, and the queue of filter hits
     i32 chunk_hint[kWarps];      // broadcast slots per look at the hit queue (adapts to the hit rate)
-    // Broadcast slots of the segment at hand: [bc_lo, bc_hi); odd operand values fill it from bc_lo up
-    // (bc_n of them), even ones from bc_hi down (bc_neven): the loops over odd values need no mask
-    // for * and no rotation for %.  For a family whose
+    // Broadcast slots of the segment at hand: [bc_lo, bc_hi); general operands fill it from bc_lo up
+    // (bc_n of them), those of magnitude <= 1 from bc_hi down (bc_nspecial).  For a family whose
     // members' slots lie side by side (bc_keep) the per-member counts are kept in kept_*, and
     // kept_head names the family resident in the tile (-1: none), so the next ticket of the same
     // family does not fill again.
     i32 bc_lo, bc_hi;
-    u32 bc_n, bc_neven;
+    u32 bc_n, bc_nspecial;
     i32 kept_head;
-    u32 kept_n[8], kept_neven[8];
+    u32 kept_n[8], kept_nspecial[8];
     i32 kept_wide[8];
     u32 wq_n[kWarps], wq_over[kWarps];
     i32 tile_wide;               // some operand of the tile does not fit int32
@@ -708,8 +707,7 @@ __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x 
 // are tp -+ A*b, i.e. A*a - tp == -+ A*b; with SWAP they are +-(tp - A*b).  Either way the pair
 // hits iff the sign-free forms agree: ca == t_pm.  Which of the two hit is settled in the rare
 // path, from t_add.
-// ODD: every broadcast value in [s0, s1) is odd, so the mask of * is all ones and is left out.
-template <u32 MASK, bool SWAP, bool ODD>
+template <u32 MASK, bool SWAP>
 __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tp, int s0, int s1, u32 opip) {
     constexpr bool kPair = (MASK & 3u) == 3u;
     u32 aA[kNA], ca[kNA];
@@ -722,10 +720,7 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
         for (int j = 0; j < kNA; j += 2) {
             if (kPair) { h0 |= ca[j] == e.t_pm; h3 |= ca[j + 1] == e.t_pm; }
             else if (MASK & 3u) { h0 |= aA[j] == t_one; h3 |= aA[j + 1] == t_one; }
-            if (MASK & 4u) {
-                if (ODD) { h1 |= aA[j] == e.mul_tm; h2 |= aA[j + 1] == e.mul_tm; }
-                else { h1 |= (aA[j] & e.mul_mask) == e.mul_tm; h2 |= (aA[j + 1] & e.mul_mask) == e.mul_tm; }
-            }
+            if (MASK & 4u) { h1 |= (aA[j] & e.mul_mask) == e.mul_tm; h2 |= (aA[j + 1] & e.mul_mask) == e.mul_tm; }
         }
     };
     auto resolve = [&](int s) {                          // the rare path: which candidates hit
@@ -766,11 +761,9 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
 //   n mod d == tabs       <=>  d divides n - tabs (and tabs < d, n >= tabs); for d = 2^k * o,
 //                              d | x  <=>  rotr(x * o^-1, k) <= floor((2^32-1) / d).
 // SWAP = false: register operand / broadcast operand; SWAP = true: broadcast / register.
-// ODD (without SWAP): every divisor in [s0, s1) is odd, so k = 0 and the rotation is left out.
-// The divisors 0 and +-1 need no special case: for d = 1 the tests read n == tabs and
-// (tabs == 0); for d = 0 the quotient test never holds and the remainder test only for
-// n == tabs, which the exact check then rejects as a division by zero.
-template <u32 MASK, bool SWAP, bool ODD>
+// SPECIAL (without SWAP only): the slots hold the divisors 0 and +-1: 0 is skipped (invalid),
+// +-1 gives |quotient| = |dividend| and remainder 0.
+template <u32 MASK, bool SWAP, bool SPECIAL>
 __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tabs, int s0, int s1, u32 opip) {
     u32 ua[kNA], xa[kNA], low[kNA], inv[kNA], kk[kNA], cc[kNA];
 #pragma unroll
@@ -784,9 +777,12 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
         if (SWAP) {                 // e.ub: dividend magnitude; e.low: dividend - tabs (or 1)
             hq = (e.ub - low[j]) < ua[j];
             hr = rotr32(e.low * inv[j], kk[j]) <= cc[j];
+        } else if (SPECIAL) {
+            hq = e.ub == 1u && ua[j] == tabs;
+            hr = e.ub == 1u && tabs == 0u;
         } else {                    // e.low: tabs * divisor (or never); e.ub: divisor magnitude
             hq = (ua[j] - e.low) < e.ub;
-            hr = (ODD ? xa[j] * e.inv : rotr32(xa[j] * e.inv, ek)) <= e.cmax;
+            hr = rotr32(xa[j] * e.inv, ek) <= e.cmax;
         }
     };
     auto scan = [&](const BcDiv& e, u32 ek, bool& h0, bool& h1, bool& h2, bool& h3) {
@@ -811,7 +807,7 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
             if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
         }
     };
-    const bool need_k = !SWAP && !ODD && (MASK & 2u);
+    const bool need_k = !SWAP && !SPECIAL && (MASK & 2u);
     int s = s0;
     for (; s + 2 <= s1; s += 2) {                       // one warp vote per two broadcast operands
         const BcDiv e0 = sh.bc_div[s], e1 = sh.bc_div[s + 1];
@@ -957,14 +953,13 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
-    auto run = [&](int s0, int s1, u32 alv, bool odd) {
+    auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide) {
             wide_chunk(sh, a64, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: if (odd) ring_pass<M, SWAP, true>(sh, &R, alv, tp, s0, s1, opip); \
-                           else ring_pass<M, SWAP, false>(sh, &R, alv, tp, s0, s1, opip); break;
+#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
@@ -973,7 +968,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         if (A != 1u) { div_pass_signed<SWAP>(sh, &R, alv, mask, A, tp, s0, s1, opip); return; }
         if (!t_small) return;                            // no int32 quotient or remainder can be the target
         switch ((mask >> 3) & 3u) {
-#define XP_DIV(M) case M: if (odd && !SWAP) div_pass<M, SWAP, true>(sh, &R, alv, tabs, s0, s1, opip); \
+#define XP_DIV(M) case M: if (special && !SWAP) div_pass<M, SWAP, true>(sh, &R, alv, tabs, s0, s1, opip); \
                           else div_pass<M, SWAP, false>(sh, &R, alv, tabs, s0, s1, opip); break;
             XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
 #undef XP_DIV
@@ -981,8 +976,8 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         }
     };
 
-    // The broadcast operands sit in two runs of slots: the odd values from the first slot up, the
-    // even ones from the last slot down.  Every warp walks
+    // The broadcast operands sit in two runs of slots: the general ones from slot 0 up, the
+    // ones of magnitude <= 1 (special as divisors) from the last slot down.  Every warp walks
     // the runs on its own, in chunks of `chunk` slots, and looks at its hit queue after each:
     // no CTA-wide synchronisation happens inside a tile.  A chunk that overflows the queue (a
     // spec that many candidates satisfy at probe 0) is forgotten and redone with a quarter of
@@ -990,16 +985,16 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     // 32 * 5 hits, which always fit).  The chunk size is kept per warp from tile to tile and
     // grows back slowly.
     const int warp = threadIdx.x >> 5;
-    const int n_even = (int)sh.bc_neven;
+    const int n_special = (int)sh.bc_nspecial;
     int chunk = sh.chunk_hint[warp];
     bool shrunk = false;
     u32 q_start = 0;                                    // queue length when the current chunk began
     for (int part = 0; part < 2; ++part) {
-        const int lo = part == 0 ? bc_lo : bc_hi - n_even, hi = part == 0 ? bc_lo + nb : bc_hi;
+        const int lo = part == 0 ? bc_lo : bc_hi - n_special, hi = part == 0 ? bc_lo + nb : bc_hi;
         int s0 = lo;
         while (s0 < hi) {
             const int s1 = s0 + chunk < hi ? s0 + chunk : hi;
-            run(s0, s1, alive, part == 0);
+            run(s0, s1, alive, part == 1);
             __syncwarp();
             const u32 qn = sh.wq_n[warp];
             const bool overflow = sh.wq_over[warp] != 0;
@@ -1011,7 +1006,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
                 shrunk = true;
                 if (chunk > 1) { chunk = chunk / 4 > 1 ? chunk / 4 : 1; continue; }
                 for (int j = 0; j < kNA; ++j) {
-                    run(s0, s0 + 1, alive & (1u << j), part == 0);
+                    run(s0, s0 + 1, alive & (1u << j), part == 1);
                     drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
                 }
             } else if (qn > (u32)(kWarpQueue / 2)) {
@@ -1041,8 +1036,8 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
     for (int i = threadIdx.x; i < n_bc; i += kThreads) {
         i64 v;
         if (!operand_value(g, hole, 0, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
-        const bool odd = ((u32)(u64)v & 1u) != 0u;
-        const u32 slot = odd ? (u32)sh.bc_lo + atomicAdd(&sh.bc_n, 1u) : (u32)sh.bc_hi - 1u - atomicAdd(&sh.bc_neven, 1u);
+        const bool special = v >= -1 && v <= 1;
+        const u32 slot = special ? (u32)sh.bc_hi - 1u - atomicAdd(&sh.bc_nspecial, 1u) : (u32)sh.bc_lo + atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
         const u32 b = (u32)(u64)v, ub = abs_u32((i32)v);
@@ -1117,7 +1112,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             sh.bc_lo = keep ? seg.bc_base : 0;
             sh.bc_hi = keep ? seg.bc_base + n_bc : kBcTile;
             sh.bc_n = resident ? sh.kept_n[m] : 0;
-            sh.bc_neven = resident ? sh.kept_neven[m] : 0;
+            sh.bc_nspecial = resident ? sh.kept_nspecial[m] : 0;
             sh.tile_wide = resident ? sh.kept_wide[m] : 0;
             if (!resident) sh.kept_head = -1;
         }
@@ -1127,7 +1122,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (wide_bc) sh.tile_wide = 1;
             __syncthreads();
             if (threadIdx.x == 0 && keep) {
-                sh.kept_n[m] = sh.bc_n; sh.kept_neven[m] = sh.bc_neven; sh.kept_wide[m] = sh.tile_wide;
+                sh.kept_n[m] = sh.bc_n; sh.kept_nspecial[m] = sh.bc_nspecial; sh.kept_wide[m] = sh.tile_wide;
                 if (m == family - 1) sh.kept_head = seg_index;
             }
             __syncthreads();
