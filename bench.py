@@ -222,7 +222,7 @@ def main():
         "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G int32-op/s", "frac": achieved / peak,
                      "traffic": None, "kernel": "eval_kernel",
                      "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
-                     "model": "operation + comparison per candidate-point evaluation (see DESIGN.md)"},
+                     "model": "32-bit operations of one operation + one comparison per candidate-point evaluation of the filter stage"},
     }
     if not args.no_cpu_baseline and args.workload == "config2":
         e, dt, sample = oracle_sample(0, ORACLE_SAMPLE_RANKS)

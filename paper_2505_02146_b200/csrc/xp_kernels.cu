@@ -2,13 +2,15 @@
 //
 //   prepare_kernel  -- per sketch, once at load: coordinates and spec values of the sample
 //                      points, choice and order of each hole's probe points.
+//   subvalue_kernel, stage_points_kernel, stage_spec_kernel -- per sketch, once at load: values
+//                      of all small subtrees at the probes; points and spec values of a box.
 //   eval_kernel     -- the search.  Persistent CTAs take tickets (pieces of the rank space)
 //                      from an atomic counter; no CTA ever waits for another.
 //                        stage 1 (tile segments): probe-point filter over a product of operand tiles;
-//                        stage 2: exact int64 check of a candidate on the probe points (lane = candidate);
+//                        stage 2: exact int64 check of a hit on the probe points (lane = candidate).
 //                      Survivors of stage 2 go to a global queue.
-//   verify_kernel   -- stage 3: check on the whole domain (lane = point, block-wide early exit),
-//                      cut into (survivor, chunk of points) items that any CTA takes.
+//   verify_kernel   -- stage 3: check on the whole domain (lane = point, warp-wide early exit),
+//                      cut into (survivor, chunk of points) items that any warp takes.
 //   count_kernel    -- survivors that passed every chunk become matches: per-size counts (sum)
 //                      and least rank (min) by atomics.
 //   finish_kernel   -- reduction of the per-size results to the least solution per hole.
@@ -228,8 +230,8 @@ struct EvalShared {
     u64 min_rank[kMaxSize + 1];
     u64 filter_survivors, probe_survivors;
     u64 warp_evals[kThreads / 32];
-    // tile tickets: the broadcast-side operand values at probe 0 (entries invalid there are
-    // dropped), the reciprocal of each as a divisor, and the queue of filter hits
+    // tile tickets: the broadcast-side operands at probe 0 (entries invalid there are dropped) with
+    // what the loops need of each, and the warps' queues of filter hits
     i32 chunk_hint[kWarps];      // broadcast slots per look at the hit queue (adapts to the hit rate)
     // Broadcast slots of the segment at hand: [bc_lo, bc_hi); general operands fill it from bc_lo up
     // (bc_n of them), those of magnitude <= 1 from bc_hi down (bc_nspecial).  For a family whose
