@@ -67,7 +67,8 @@ enum {
     XP_MAX_CODE = 64          /* instructions in one context or spec expression */
 };
 
-/* Operators.  The first five may appear in grammar productions; all of them in context and
+/* Operators.  The first five and MIN, MAX may appear in grammar productions (min and max let a
+ * hole express the bound of a remainder tile, e.g. min(T, N - io*T)); all of them in context and
  * spec expressions. */
 enum {
     XP_OP_ADD = 0, XP_OP_SUB = 1, XP_OP_MUL = 2, XP_OP_DIV = 3, XP_OP_MOD = 4,
@@ -84,7 +85,7 @@ typedef struct {
     int32_t lhs;        /* nonterminal index, 0 <= lhs < n_nonterminals */
     int32_t kind;       /* XP_PROD_* */
     int32_t var;        /* XP_PROD_VAR: variable index */
-    int32_t op;         /* XP_PROD_BIN: XP_OP_ADD .. XP_OP_MOD */
+    int32_t op;         /* XP_PROD_BIN: XP_OP_ADD .. XP_OP_MOD, XP_OP_MIN, XP_OP_MAX */
     int32_t left;       /* XP_PROD_BIN: nonterminal of the left operand */
     int32_t right;      /* XP_PROD_BIN: nonterminal of the right operand */
     int64_t value;      /* XP_PROD_CONST: the constant */
@@ -173,13 +174,13 @@ typedef struct {
     uint64_t least_rank;
     const xp_instr* least_code;     /* postfix of the least solution */
     int32_t least_len;
-    const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))" */
+    const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))"; min and max as calls, "min(a,b)" */
     uint64_t evals_executed;        /* candidate-point evaluations the GPU carried out for this hole */
     uint64_t filter_survivors;      /* candidates that passed the first probe point */
     uint64_t probe_survivors;       /* candidates that passed every probe point */
     uint64_t nominal_ops;           /* 32-bit integer operations the filter stage's candidate-point evaluations
                                        amount to under the library's cost model: one operation and one
-                                       comparison per evaluation, with + - * = 1, a reciprocal division = 7
+                                       comparison per evaluation, with + - * min max = 1, a reciprocal division = 7
                                        (/ and % of one operand pair share it), a remainder's multiply-subtract = 1 */
     double kernel_ms;               /* device time of the whole call's kernels (CUDA events) */
     double total_ms;                /* host wall time of the whole call */
@@ -188,7 +189,7 @@ typedef struct {
 
 /* Grammar (Section 4.4: the expressions the synthesis step may put into a hole).  Builds the
  * per-(nonterminal, size) candidate counts and rank offsets on the host; no GPU is touched.
- * Errors: XP_ERR_GRAMMAR (bad indices, operator outside + - * / %), XP_ERR_TOO_LARGE. */
+ * Errors: XP_ERR_GRAMMAR (bad indices, operator outside + - * / % min max), XP_ERR_TOO_LARGE. */
 xp_status xp_grammar_create(const xp_grammar_desc* desc, xp_grammar** out);
 void xp_grammar_destroy(xp_grammar* g);
 

@@ -29,7 +29,9 @@
 //   * a zero divisor anywhere in a tree (or in the context, or in the spec) at a
 //     point makes the candidate fail at that point, with no short-circuiting;
 //   * comparison and logic operators (context / spec only) yield 0 or 1 and
-//     evaluate both operands.
+//     evaluate both operands;
+//   * a grammar may also use min and max as binary operators (printed min(a,b)):
+//     the remainder-tile bounds of a split loop need them.
 //
 // Parity against the paper itself is unpinned: it prints no instance, query or
 // solution for this step (its constraint figure is not available).  The functions
@@ -221,6 +223,10 @@ bool eval_tree(const Node* n, const i64* pt, i64& out) {
 void tree_text(const xo_grammar* g, const Node* n, std::string& s) {
     if (n->p->kind == P_VAR) { s += g->var_names ? g->var_names[n->p->var] : ("v" + std::to_string(n->p->var)); return; }
     if (n->p->kind == P_CONST) { s += std::to_string((long long)n->p->value); return; }
+    if (n->p->op == OP_MIN || n->p->op == OP_MAX) {
+        s += OP_TEXT[n->p->op]; s += "("; tree_text(g, n->l, s); s += ","; tree_text(g, n->r, s); s += ")";
+        return;
+    }
     s += "("; tree_text(g, n->l, s); s += OP_TEXT[n->p->op]; tree_text(g, n->r, s); s += ")";
 }
 

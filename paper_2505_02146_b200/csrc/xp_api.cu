@@ -107,7 +107,7 @@ extern "C" xp_status xp_grammar_create(const xp_grammar_desc* d, xp_grammar** ou
         const xp_production& p = d->productions[i];
         bool ok = p.lhs >= 0 && p.lhs < g->n_nt;
         if (p.kind == XP_PROD_VAR) ok = ok && p.var >= 0 && p.var < g->n_vars;
-        else if (p.kind == XP_PROD_BIN) ok = ok && p.op >= XP_OP_ADD && p.op <= XP_OP_MOD && p.left >= 0 && p.left < g->n_nt && p.right >= 0 && p.right < g->n_nt;
+        else if (p.kind == XP_PROD_BIN) ok = ok && ((p.op >= XP_OP_ADD && p.op <= XP_OP_MOD) || p.op == XP_OP_MIN || p.op == XP_OP_MAX) && p.left >= 0 && p.left < g->n_nt && p.right >= 0 && p.right < g->n_nt;
         else if (p.kind != XP_PROD_CONST) ok = false;
         if (!ok) { delete g; return fail(XP_ERR_GRAMMAR, "production " + std::to_string(i) + " is malformed"); }
         g->prods.push_back(p);
@@ -177,9 +177,10 @@ static bool host_unrank(const xp_grammar* g, int nt, int size, u64 rank, std::ve
         const u64 cr = g->cnt[b.rnt][size - 1 - a];
         const u64 block = g->cnt[b.lnt][a] * cr;
         if (rem >= block) { rem -= block; continue; }
-        *text += "(";
+        const bool call = b.op == XP_OP_MIN || b.op == XP_OP_MAX;      // printed min(l,r) / max(l,r)
+        *text += call ? std::string(kOpText[b.op]) + "(" : std::string("(");
         if (!host_unrank(g, b.lnt, a, rem / cr, code, text)) return false;
-        *text += kOpText[b.op];
+        *text += call ? "," : kOpText[b.op];
         if (!host_unrank(g, b.rnt, size - 1 - a, rem % cr, code, text)) return false;
         *text += ")";
         xp_instr in;

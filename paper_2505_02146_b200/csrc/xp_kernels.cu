@@ -683,6 +683,7 @@ struct RegOps {
     u32 aA[kNA];     // A * value (the affine context's factor folded in)
     u32 ca[kNA];     // sign-free form of A * value (SWAP) or of A * value - tp, for the joint +/- test
     u32 ua[kNA];     // |value|
+    i32 av[kNA];     // the value itself (min and max compare signed numbers)
     u32 neg;         // bit j: value j is negative
     // register operand as DIVISOR (SWAP), magnitudes only:
     u32 low[kNA];    // tabs * |value| (0x80000000 when that is 2^31 or more: never matches)
@@ -696,6 +697,10 @@ struct RegOps {
 // operand arrays it needs from the tile's RegOps into registers and runs with a small live
 // set, instead of sharing one large frame with the rest of the kernel.
 // `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
+
+// Position of a grammar operator among the seven a segment may hold: + - * / % min max.
+__device__ __forceinline__ int op_slot(int op) { return op <= XP_OP_MOD ? op : op - XP_OP_MIN + 5; }
+constexpr int kSlotMin = 5, kSlotMax = 6;
 
 // x and -x have the same sign-free form: the smaller of the two as unsigned numbers.
 __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x < y ? x : y; }
@@ -828,6 +833,44 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
     }
 }
 
+// min and max of int32-exact operands (exact signed comparison), times the context factor A,
+// against tp.  MASK: bit0 min, bit1 max.  Both are symmetric, so SWAP plays no role.
+template <u32 MASK, bool HAS_A>
+__device__ __noinline__ void minmax_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, int s0, int s1, u32 opip) {
+    i32 av[kNA];
+#pragma unroll
+    for (int j = 0; j < kNA; ++j) av[j] = Rm->av[j];
+    auto test = [&](i32 b, int j, bool& hmin, bool& hmax) {
+        u32 lo = (u32)(av[j] < b ? av[j] : b), hi = (u32)(av[j] < b ? b : av[j]);
+        if (HAS_A) { lo *= A; hi *= A; }
+        hmin = lo == tp;
+        hmax = hi == tp;
+    };
+    for (int s = s0; s < s1; ++s) {
+        const i32 b = (i32)sh.bc_meta[s].lo;
+        bool h0 = false, h1 = false, h2 = false, h3 = false;
+#pragma unroll
+        for (int j = 0; j < kNA; j += 2) {
+            bool m0, x0, m1, x1;
+            test(b, j, m0, x0);
+            test(b, j + 1, m1, x1);
+            if (MASK & 1u) { h0 |= m0; h1 |= m1; }
+            if (MASK & 2u) { h2 |= x0; h3 |= x1; }
+        }
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
+#pragma unroll
+            for (int j = 0; j < kNA; ++j) {
+                if (!((alive >> j) & 1u)) continue;
+                bool hmin, hmax;
+                test(b, j, hmin, hmax);
+                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
+                if ((MASK & 1u) && hmin) push_hit(sh, idx, (u32)s, (opip >> (3 * kSlotMin)) & 7u);
+                if ((MASK & 2u) && hmax) push_hit(sh, idx, (u32)s, (opip >> (3 * kSlotMax)) & 7u);
+            }
+        }
+    }
+}
+
 // / and % on int32-exact operands under a context factor A != 1: signed results times A are
 // compared with tp.  Plain 32-bit division; this form only serves sketches whose hole sits
 // under a multiplication (small searches).
@@ -925,7 +968,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     const bool tile_wide = sh.tile_wide != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
     u32 opip = 0, mask = 0;
-    for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * seg.op[o]); mask |= 1u << seg.op[o]; }
+    for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * op_slot(seg.op[o])); mask |= 1u << op_slot(seg.op[o]); }
 
     const u32 A = (u32)A64, tp = (u32)tq;
     // With A == 1 a quotient or remainder of int32 operands can only equal a target of
@@ -940,6 +983,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         const i32 v = (i32)a64[j];
         const u32 ua = abs_u32(v);
         R.aA[j] = (u32)v * A;
+        R.av[j] = v;
         R.ca[j] = signfree(SWAP ? R.aA[j] : R.aA[j] - tp);
         R.ua[j] = ua;
         if (v < 0) R.neg |= 1u << j;
@@ -964,6 +1008,13 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
 #define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
+            default: break;
+        }
+        switch ((mask >> kSlotMin) & 3u) {
+#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, &R, alv, A, tp, s0, s1, opip); \
+                         else minmax_pass<M, false>(sh, &R, alv, A, tp, s0, s1, opip); break;
+            XP_MM(1u) XP_MM(2u) XP_MM(3u)
+#undef XP_MM
             default: break;
         }
         if (!(mask & 24u)) return;

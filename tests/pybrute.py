@@ -76,6 +76,8 @@ def tree_value(t: tuple, pt: Sequence[int]) -> Optional[int]:
 def tree_text(t: tuple, g: Grammar) -> str:
     if t[0] == "v": return g.variables[t[1]].name
     if t[0] == "c": return str(t[1])
+    if t[0] in ("min", "max"):
+        return f"{t[0]}({tree_text(t[1], g)},{tree_text(t[2], g)})"
     return f"({tree_text(t[1], g)}{t[0]}{tree_text(t[2], g)})"
 
 
@@ -143,6 +145,15 @@ def text_value(text: str, g: Grammar, pt: Sequence[int]) -> Optional[int]:
 
     def node() -> Optional[int]:
         nonlocal pos
+        if text.startswith(("min(", "max("), pos):
+            op = text[pos:pos + 3]; pos += 4
+            a = node()
+            assert text[pos] == ","; pos += 1
+            b = node()
+            assert text[pos] == ")"; pos += 1
+            if a is None or b is None:
+                return None
+            return c_op(op, a, b)
         if text[pos] == "(":
             pos += 1
             a = node()

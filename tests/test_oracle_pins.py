@@ -343,6 +343,35 @@ def test_context_operators():
         assert oracle.eval_code(parse_expr(text, vs), pt, hole=10) == want, text
 
 
+def test_min_max_as_grammar_operators():
+    """min and max in the grammar: counts follow the closed form with 7 operators, listing and
+    search agree with the materialised brute force, and the trip count of a remainder tile
+    (8, 8, 8, 6 for io = 0..3 of a 30-long loop split by 8) is found as min(8,(30-(io*8)))."""
+    vs = [Variable("io", 0, 4)]
+    g = free_grammar(vs, [8, 30], ops=["-", "*", "min"])
+    assert oracle.counts(g, 0, 7) == [0, 3, 0, 27, 0, 486, 0, 10935]
+    T = pybrute.all_trees(g, 5)
+    for size in (1, 3, 5):
+        assert oracle.listing(g, 0, size) == [pybrute.tree_text(t, g) for t in T[(0, size)]]
+    coords = np.array([[0], [1], [2], [3]], dtype=np.int32)
+    sk = Sketch(g, [Hole(0, 7, spec_table=np.array([8, 8, 8, 6], dtype=np.int64))], coords)
+    r = oracle.repair_hole(sk)
+    cand, match, least, _ = pybrute.repair(sk)
+    assert r.cand_count == cand and r.match_count == match == [0, 0, 0, 0, 0, 0, 0, 4]
+    assert (r.least_size, r.least_rank, r.least_text) == least == (7, 7840, "min(8,(30-(io*8)))")
+    for io in range(4):
+        assert pybrute.text_value(r.least_text, g, (io,)) == min(8, 30 - io * 8)
+    full = free_grammar([Variable("a", -3, 4), Variable("b", 0, 3)], [0, 2], ops=["+", "-", "*", "/", "%", "min", "max"])
+    assert oracle.counts(full, 0, 5) == [0, 4, 0, 7 * 16, 0, 2 * 49 * 64]
+    for spec in ["max(a,0)", "min(a,b)*2", "max(a,b)-min(a,b)"]:
+        sk = Sketch(full, [Hole(0, 5, spec_expr=parse_expr(spec, full.variables))])
+        cand, match, least, _ = pybrute.repair(sk)
+        r = oracle.repair_hole(sk)
+        assert r.match_count == match and r.solved == (least is not None)
+        if least is not None:
+            assert (r.least_size, r.least_rank, r.least_text) == least
+
+
 def test_loop_bound_hole_reading():
     """Loop-bound holes are checked through the guard predicate on the enclosing box:
     ``kh < HOLE`` against ``(oh+kh-1) < 6`` is solved by ``7-oh`` (small version of the 56-wide case)."""

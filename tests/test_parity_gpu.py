@@ -109,6 +109,26 @@ def test_repeated_productions_and_the_largest_size(xp):
         assert res[0].cand_count[15] == 109824 and res[0].match_count[15] == 30030
 
 
+def test_min_max_as_grammar_operators(xp):
+    coords = np.array([[0], [1], [2], [3]], dtype=np.int32)
+    g = free_grammar([Variable("io", 0, 4)], [8, 30], ops=["-", "*", "min"])
+    sk = Sketch(g, [Hole(0, 7, spec_table=np.array([8, 8, 8, 6], dtype=np.int64))], coords, name="remainder tile")
+    for flags in PATHS:
+        res = check_sketch(xp, sk, flags=flags)
+        assert res[0].least_text == "min(8,(30-(io*8)))"
+    vs = [Variable("a", -3, 4), Variable("b", 0, 3)]
+    full = free_grammar(vs, [0, 2, -5, 7], ops=["+", "-", "*", "/", "%", "min", "max"])
+    for spec, ctx in [("max(a,0)", ""), ("min(a,b)*2", ""), ("max(a,b)-min(a,b)", ""), ("(max(a,2)*3)+b", "(HOLE*3)+b"),
+                      ("min(a,b)<1", "HOLE<1")]:
+        sk = Sketch(full, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))], name=f"minmax:{spec}")
+        for flags in PATHS:
+            check_sketch(xp, sk, flags=flags)
+    # a larger space so that whole tiles of every operator group run (7 operators: two segments per split)
+    big = free_grammar([Variable("i", 0, 16), Variable("j", 0, 16)], constant_set(-8, 8), ops=["+", "-", "*", "/", "%", "min", "max"])
+    for spec in ["min(i,j)+3", "max((i*2),j)"]:
+        check_sketch(xp, Sketch(big, [Hole(0, 5, spec_expr=parse_expr(spec, big.variables))], name=f"minmax big:{spec}"))
+
+
 def test_zero_divisors_and_wraparound(xp):
     vs = [Variable("x", 0, 3)]
     for flags in PATHS:
