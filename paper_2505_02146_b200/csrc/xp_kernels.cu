@@ -1010,7 +1010,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
 #undef XP_RING
             default: break;
         }
-        switch ((mask >> kSlotMin) & 3u) {
+        if (mask >> kSlotMin) switch ((mask >> kSlotMin) & 3u) {
 #define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, &R, alv, A, tp, s0, s1, opip); \
                          else minmax_pass<M, false>(sh, &R, alv, A, tp, s0, s1, opip); break;
             XP_MM(1u) XP_MM(2u) XP_MM(3u)
