@@ -188,7 +188,7 @@ constexpr int kLinearPerThread = kLinearChunk / kThreads; // ranks per thread pe
 constexpr int kWarps = kThreads / 32;
 constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check (all warps)
 constexpr int kWarpQueue = kQueueCap / kWarps;            // ... per warp: every warp keeps and empties its own queue
-constexpr int kChunkB = 128;                              // broadcast operands between block-wide queue checks
+constexpr int kChunkB = 512;                              // broadcast operands between block-wide queue checks
 static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
 static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the free half of its queue");
 
@@ -979,22 +979,31 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     RegOps R;
     R.alive = alive;
     R.neg = 0;
+    // Only the arrays that this segment's loops read are written (the struct lives in the
+    // thread's local memory, and every store there is traffic).
+    const bool want_ring = (mask & 7u) != 0, want_div = (mask & 24u) != 0, want_mm = (mask >> kSlotMin) != 0;
     for (int j = 0; j < kNA; ++j) {
         const i32 v = (i32)a64[j];
         const u32 ua = abs_u32(v);
-        R.aA[j] = (u32)v * A;
-        R.av[j] = v;
-        R.ca[j] = signfree(SWAP ? R.aA[j] : R.aA[j] - tp);
-        R.ua[j] = ua;
-        if (v < 0) R.neg |= 1u << j;
-        R.low[j] = 0x80000000u; R.inv[j] = 1u; R.kk[j] = 0u; R.cc[j] = 0u;
-        if (SWAP && !tile_wide && (mask & 24u) && A == 1u && ua != 0u) {
-            const u64 lw = (u64)tabs * ua;
-            if (lw < (1ull << 31)) R.low[j] = (u32)lw;
-            const u32 k = (u32)__ffs((int)ua) - 1u;
-            R.kk[j] = k;
-            R.inv[j] = inv_odd(ua >> k);
-            R.cc[j] = tabs < ua ? 0xffffffffu / ua : 0u;
+        if (want_ring) {
+            R.aA[j] = (u32)v * A;
+            R.ca[j] = signfree(SWAP ? R.aA[j] : R.aA[j] - tp);
+        }
+        if (want_mm) R.av[j] = v;
+        if (want_div) {
+            R.ua[j] = ua;
+            if (v < 0) R.neg |= 1u << j;
+        }
+        if (SWAP && want_div && !tile_wide && A == 1u) {
+            u32 low = 0x80000000u, inv = 1u, k = 0u, cc = 0u;
+            if (ua != 0u) {
+                const u64 lw = (u64)tabs * ua;
+                if (lw < (1ull << 31)) low = (u32)lw;
+                k = (u32)__ffs((int)ua) - 1u;
+                inv = inv_odd(ua >> k);
+                cc = tabs < ua ? 0xffffffffu / ua : 0u;
+            }
+            R.low[j] = low; R.inv[j] = inv; R.kk[j] = k; R.cc[j] = cc;
         }
     }
 
