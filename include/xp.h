@@ -148,7 +148,8 @@ typedef struct {
     const xp_rank_range* rank_ranges;
     void* stream;                       /* cudaStream_t to launch on; NULL: the default stream */
     void* workspace;                    /* DEVICE memory for the call's scratch (256-byte aligned), */
-    size_t workspace_bytes;             /*   at least xp_workspace_bytes(); NULL: the library allocates */
+    size_t workspace_bytes;             /*   at least xp_workspace_bytes(); NULL: the library uses a block of its
+                                             own that it keeps from call to call (cudaMalloc when it must grow) */
     uint32_t flags;                     /* XP_FLAG_* */
     const volatile int32_t* cancel;     /* optional host word polled between launches */
 } xp_repair_opts;

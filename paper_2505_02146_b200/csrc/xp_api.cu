@@ -55,9 +55,7 @@ struct xp_grammar {
     int ok_size = kMaxSize;          // counts are exact (< 2^63) up to this size
     // device copy, made on first use
     std::mutex mu;
-    GrammarDev* d_g = nullptr;
-    LeafDev* d_leaves = nullptr;
-    BinDev* d_bins = nullptr;
+    GrammarDev* d_g = nullptr;       // one block: header, leaves, binary productions
 };
 
 // cnt[nt][s] by the recurrence over productions and left sizes; off[s] of a binary production
@@ -141,8 +139,6 @@ extern "C" xp_status xp_grammar_create(const xp_grammar_desc* d, xp_grammar** ou
 extern "C" void xp_grammar_destroy(xp_grammar* g) {
     if (!g) return;
     if (g->d_g) cudaFree(g->d_g);
-    if (g->d_leaves) cudaFree(g->d_leaves);
-    if (g->d_bins) cudaFree(g->d_bins);
     delete g;
 }
 
@@ -219,16 +215,21 @@ static xp_status grammar_to_device(xp_grammar* g) {
     memcpy(h.leaf_begin, g->leaf_begin, sizeof(h.leaf_begin));
     memcpy(h.bin_begin, g->bin_begin, sizeof(h.bin_begin));
     memcpy(h.cnt, g->cnt, sizeof(h.cnt));
-    XP_CUDA(cudaMalloc(&g->d_leaves, sizeof(LeafDev) * (g->leaves.size() + 1)));
-    XP_CUDA(cudaMalloc(&g->d_bins, sizeof(BinDev) * (g->bins.size() + 1)));
-    XP_CUDA(cudaMemcpy(g->d_leaves, g->leaves.data(), sizeof(LeafDev) * g->leaves.size(), cudaMemcpyHostToDevice));
-    XP_CUDA(cudaMemcpy(g->d_bins, g->bins.data(), sizeof(BinDev) * g->bins.size(), cudaMemcpyHostToDevice));
-    h.leaves = g->d_leaves;
-    h.bins = g->d_bins;
-    GrammarDev* d = nullptr;
-    XP_CUDA(cudaMalloc(&d, sizeof(GrammarDev)));
-    XP_CUDA(cudaMemcpy(d, &h, sizeof(h), cudaMemcpyHostToDevice));
-    g->d_g = d;
+    // one device block and one copy: header | leaves | binary productions
+    const size_t off_leaves = (sizeof(GrammarDev) + 255) & ~(size_t)255;
+    const size_t off_bins = off_leaves + ((sizeof(LeafDev) * (g->leaves.size() + 1) + 255) & ~(size_t)255);
+    const size_t total = off_bins + sizeof(BinDev) * (g->bins.size() + 1);
+    char* block = nullptr;
+    XP_CUDA(cudaMalloc((void**)&block, total));
+    h.leaves = (const LeafDev*)(block + off_leaves);
+    h.bins = (const BinDev*)(block + off_bins);
+    std::vector<char> stage(total, 0);
+    memcpy(&stage[0], &h, sizeof(h));
+    if (!g->leaves.empty()) memcpy(&stage[off_leaves], g->leaves.data(), sizeof(LeafDev) * g->leaves.size());
+    if (!g->bins.empty()) memcpy(&stage[off_bins], g->bins.data(), sizeof(BinDev) * g->bins.size());
+    cudaError_t e = cudaMemcpy(block, stage.data(), total, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(block); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
+    g->d_g = (GrammarDev*)block;
     return XP_OK;
 }
 
@@ -249,7 +250,12 @@ struct xp_sketch {
     std::vector<HoleHost> holes;
     SketchDev* d_s = nullptr;
     HoleDev* d_holes = nullptr;
-    std::vector<void*> owned;        // device copies of host tables
+    // Device memory of the sketch: one block sized at load for everything the load may need
+    // (copies of host tables, staged points and specs, subtree-value tables), handed out in
+    // 256-byte aligned pieces; anything beyond the estimate gets a block of its own.
+    char* arena = nullptr;
+    size_t arena_bytes = 0, arena_used = 0;
+    std::vector<void*> owned;
 };
 
 // Checks a postfix expression; returns false when malformed or too deep.
@@ -281,9 +287,37 @@ static u64 mix64(u64 x) {            // SplitMix64 finaliser: spreads sample ids
 extern "C" void xp_sketch_destroy(xp_sketch* s) {
     if (!s) return;
     for (void* p : s->owned) cudaFree(p);
-    if (s->d_holes) cudaFree(s->d_holes);
-    if (s->d_s) cudaFree(s->d_s);
+    if (s->arena) cudaFree(s->arena);
     delete s;
+}
+
+static cudaError_t sketch_alloc(xp_sketch* s, void** out, size_t bytes) {
+    const size_t need = (bytes + 255) & ~(size_t)255;
+    if (s->arena && s->arena_used + need <= s->arena_bytes) {
+        *out = s->arena + s->arena_used;
+        s->arena_used += need;
+        return cudaSuccess;
+    }
+    cudaError_t e = cudaMalloc(out, bytes ? bytes : 256);
+    if (e == cudaSuccess) s->owned.push_back(*out);
+    return e;
+}
+
+// Entries of the subtree-value tables of a hole with size bound max_size: sizes 1, 2, ... while
+// every nonterminal has at most kTabMaxEntries trees of that size, and never the sizes that only
+// occur as whole candidates (operands have at most max_size - 2 nodes).
+static u64 table_entries(const xp_grammar* g, int max_size, u64 (*off)[kMaxSize + 1], int* tmax_out) {
+    u64 total = 0;
+    int tmax = 0;
+    for (int k = 1; k <= max_size - 2; ++k) {
+        bool fits = true;
+        for (int nt = 0; nt < g->n_nt; ++nt) fits = fits && g->cnt[nt][k] <= kTabMaxEntries;
+        if (!fits) break;
+        for (int nt = 0; nt < g->n_nt; ++nt) { if (off) off[nt][k] = total; total += g->cnt[nt][k]; }
+        tmax = k;
+    }
+    if (tmax_out) *tmax_out = tmax;
+    return total;
 }
 
 extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* d, xp_sketch** out) {
@@ -328,6 +362,25 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
 #define XP_CUDA_S(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { xp_sketch_destroy(s); \
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
 
+    {   // one device block for the whole load
+        auto al = [](size_t b) { return (b + 255) & ~(size_t)255; };
+        size_t need = al(sizeof(SketchDev)) + al(sizeof(HoleDev) * d->n_holes) + al(sizeof(u32) * d->n_holes);
+        const size_t np = (size_t)n_points, row = (size_t)(nv ? nv : 1);
+        const bool stage = n_points > 0 && (u64)n_points <= kStageMaxPoints;
+        if (np > 0 && ((d->domain_kind == XP_DOMAIN_TABLE && !d->coords_on_device) || (d->domain_kind == XP_DOMAIN_BOX && stage)))
+            need += al(sizeof(i32) * np * row);
+        for (int h = 0; h < d->n_holes; ++h) {
+            const xp_hole_desc& hd = d->holes[h];
+            if (np > 0 && ((hd.spec_kind == XP_SPEC_TABLE && !hd.spec_table_on_device) || (hd.spec_kind == XP_SPEC_EXPR && stage)))
+                need += al(sizeof(i64) * np);
+            const u64 entries = table_entries(g, hd.max_size, nullptr, nullptr);
+            u64 probes = kMaxProbe;
+            while (probes > 1 && entries * 9 * probes > kTabBudgetBytes) --probes;
+            need += al(sizeof(i64) * entries * probes) + al(entries * probes);
+        }
+        if (cudaMalloc((void**)&s->arena, need) == cudaSuccess) s->arena_bytes = need;
+        else { s->arena = nullptr; (void)cudaGetLastError(); }          // fall back to piecewise allocation
+    }
     SketchDev hs;
     memset(&hs, 0, sizeof(hs));
     hs.g = g->d_g; hs.n_vars = nv; hs.n_holes = d->n_holes; hs.domain_kind = d->domain_kind; hs.n_points = n_points;
@@ -337,8 +390,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         else {
             void* p = nullptr;
             const size_t bytes = sizeof(i32) * (size_t)n_points * (size_t)(nv ? nv : 1);
-            XP_CUDA_S(cudaMalloc(&p, bytes));
-            s->owned.push_back(p);
+            XP_CUDA_S(sketch_alloc(s, &p, bytes));
             XP_CUDA_S(cudaMemcpy(p, d->coords, bytes, cudaMemcpyHostToDevice));
             hs.coords = (const i32*)p;
         }
@@ -386,8 +438,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             if (hd.spec_table_on_device) o.spec_table = (const i64*)hd.spec_table;
             else {
                 void* p = nullptr;
-                XP_CUDA_S(cudaMalloc(&p, sizeof(i64) * (size_t)n_points));
-                s->owned.push_back(p);
+                XP_CUDA_S(sketch_alloc(s, &p, sizeof(i64) * (size_t)n_points));
                 XP_CUDA_S(cudaMemcpy(p, hd.spec_table, sizeof(i64) * (size_t)n_points, cudaMemcpyHostToDevice));
                 o.spec_table = (const i64*)p;
             }
@@ -396,10 +447,10 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
         s->holes.push_back(ho);
     }
-    XP_CUDA_S(cudaMalloc(&s->d_holes, sizeof(HoleDev) * d->n_holes));
+    XP_CUDA_S(sketch_alloc(s, (void**)&s->d_holes, sizeof(HoleDev) * d->n_holes));
     XP_CUDA_S(cudaMemcpy(s->d_holes, hh.data(), sizeof(HoleDev) * d->n_holes, cudaMemcpyHostToDevice));
     hs.holes = s->d_holes;
-    XP_CUDA_S(cudaMalloc(&s->d_s, sizeof(SketchDev)));
+    XP_CUDA_S(sketch_alloc(s, (void**)&s->d_s, sizeof(SketchDev)));
     XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
     XP_CUDA_S(launch_prepare(s->d_s, nullptr));
     XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
@@ -410,25 +461,15 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     for (int h = 0; h < d->n_holes; ++h) {
         if (!s->holes[h].filter_ok) continue;
         HoleDev& o = hh[h];
-        u64 total = 0;
         int tmax = 0;
-        for (int k = 1; k <= o.max_size - 2; ++k) {
-            u64 at_size = 0;
-            bool fits = true;
-            for (int nt = 0; nt < g->n_nt; ++nt) { fits = fits && g->cnt[nt][k] <= kTabMaxEntries; at_size += g->cnt[nt][k]; }
-            if (!fits) break;
-            for (int nt = 0; nt < g->n_nt; ++nt) { o.tab_off[nt][k] = total; total += g->cnt[nt][k]; }
-            tmax = k;
-        }
+        const u64 total = table_entries(g, o.max_size, o.tab_off, &tmax);
         if (tmax == 0 || total == 0) continue;
         void* pv = nullptr;
         void* pk = nullptr;
         int probes = o.n_probe;                      // as many probes as the table budget allows
         while (probes > 1 && total * 9 * (u64)probes > kTabBudgetBytes) --probes;
-        XP_CUDA_S(cudaMalloc(&pv, sizeof(i64) * total * probes));
-        s->owned.push_back(pv);
-        XP_CUDA_S(cudaMalloc(&pk, total * probes));
-        s->owned.push_back(pk);
+        XP_CUDA_S(sketch_alloc(s, &pv, sizeof(i64) * total * probes));
+        XP_CUDA_S(sketch_alloc(s, &pk, total * probes));
         o.tab_val = (i64*)pv;
         o.tab_ok = (unsigned char*)pk;
         o.tab_max_size = tmax;
@@ -448,8 +489,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         for (int v = 0; v < nv; ++v) i32_ok = i32_ok && g->lo[v] >= INT32_MIN && g->hi[v] <= (i64)INT32_MAX + 1;
         if (d->domain_kind == XP_DOMAIN_BOX && i32_ok && nv > 0) {
             void* p = nullptr;
-            XP_CUDA_S(cudaMalloc(&p, sizeof(i32) * (size_t)n_points * (size_t)nv));
-            s->owned.push_back(p);
+            XP_CUDA_S(sketch_alloc(s, &p, sizeof(i32) * (size_t)n_points * (size_t)nv));
             XP_CUDA_S(launch_stage_points(s->d_s, n_points, (i32*)p, nullptr));
             XP_CUDA_S(cudaStreamSynchronize(nullptr));       // the kernel reads the sketch before its coords field changes
             hs.coords = (const i32*)p;
@@ -457,14 +497,12 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         }
         u32* d_bad = nullptr;
         std::vector<u32> bad(d->n_holes, 0);
-        XP_CUDA_S(cudaMalloc((void**)&d_bad, sizeof(u32) * d->n_holes));
-        s->owned.push_back(d_bad);
+        XP_CUDA_S(sketch_alloc(s, (void**)&d_bad, sizeof(u32) * d->n_holes));
         XP_CUDA_S(cudaMemset(d_bad, 0, sizeof(u32) * d->n_holes));
         for (int h = 0; h < d->n_holes; ++h) {
             if (hh[h].spec_len == 0) continue;
             void* p = nullptr;
-            XP_CUDA_S(cudaMalloc(&p, sizeof(i64) * (size_t)n_points));
-            s->owned.push_back(p);
+            XP_CUDA_S(sketch_alloc(s, &p, sizeof(i64) * (size_t)n_points));
             XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)p, d_bad + h, nullptr));
             XP_CUDA_S(cudaStreamSynchronize(nullptr));
             hh[h].spec_table = (const i64*)p;
@@ -505,6 +543,13 @@ struct Plan {
     std::vector<u64> nominal_ops;    // per accumulator: cost-model operations of the filter stage
     u64 n_tickets = 0;
 };
+
+// Scratch of calls that bring no workspace: one block per process, reused while no other call
+// is using it (a concurrent call allocates its own).
+static std::mutex g_ws_mu;
+static char* g_ws = nullptr;
+static size_t g_ws_bytes = 0;
+static int g_ws_device = -1;
 
 static const xp_repair_opts kDefaultOpts = {0, 0, 0, nullptr, nullptr, nullptr, 0, 0u, nullptr};
 
@@ -712,10 +757,24 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
 
     const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
     char* ws = (char*)o->workspace;
-    bool own_ws = false;
+    bool own_ws = false, cached_ws = false;
     if (ws) {
         if (o->workspace_bytes < w.total || ((uintptr_t)ws & 255)) return fail(XP_ERR_NOMEM, "workspace too small or misaligned");
-    } else {
+    } else if (g_ws_mu.try_lock()) {
+        // the library's own scratch, kept from call to call (grown when a call needs more)
+        cached_ws = true;
+        int dev = -1;
+        cudaGetDevice(&dev);
+        if (g_ws_bytes < w.total || g_ws_device != dev) {
+            if (g_ws) cudaFree(g_ws);                // (a block of another device is freed from here as well)
+            g_ws_device = dev;
+            g_ws = nullptr; g_ws_bytes = 0;
+            cudaError_t e = cudaMalloc((void**)&g_ws, w.total);
+            if (e != cudaSuccess) { g_ws_mu.unlock(); return fail(XP_ERR_NOMEM, std::string("cudaMalloc: ") + cudaGetErrorString(e)); }
+            g_ws_bytes = w.total;
+        }
+        ws = g_ws;
+    } else {                                       // another call holds the kept scratch
         XP_CUDA(cudaMalloc((void**)&ws, w.total));
         own_ws = true;
     }
@@ -728,7 +787,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     float ms = 0.f;
     int launches = 0;
     std::vector<AccDev> acc(plan.acc.size());
-#define XP_CUDA_R(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { if (own_ws) cudaFree(ws); \
+#define XP_CUDA_R(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { if (own_ws) cudaFree(ws); if (cached_ws) g_ws_mu.unlock(); \
         if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1); \
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
     XP_CUDA_R(cudaEventCreate(&e0));
@@ -745,6 +804,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (own_ws) cudaFree(ws);
+    if (cached_ws) g_ws_mu.unlock();
 
     size_t ai = 0;
     for (size_t i = 0; i < n; ++i) {
