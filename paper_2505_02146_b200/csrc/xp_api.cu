@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
@@ -36,6 +37,58 @@ static xp_status fail(xp_status st, const std::string& msg) {
                         std::string(#call) + ": " + cudaGetErrorString(e_));                   \
     } while (0)
 
+// ------------------------------------------------------------------------------------------
+// device memory of grammars and sketches
+// ------------------------------------------------------------------------------------------
+//
+// Blocks up to kPoolBigBytes are carved from 64 MiB slabs and, when released, kept in a
+// free list by size for the next load (a loop that loads and destroys the same sketch never
+// reaches cudaMalloc or cudaFree, whose cost and device-wide synchronisation would otherwise
+// dominate small searches).  Larger blocks go to cudaMalloc / cudaFree directly.  Slabs are
+// returned to the driver when the process ends.  One pool per device.
+namespace {
+constexpr size_t kPoolSlabBytes = 64ull << 20, kPoolBigBytes = 16ull << 20;
+struct DevPool {
+    std::multimap<size_t, char*> free_blocks;
+    char* slab = nullptr;
+    size_t slab_left = 0;
+};
+std::mutex g_pool_mu;
+std::map<int, DevPool> g_pools;
+
+cudaError_t pool_alloc(void** out, size_t bytes, int* device_out) {
+    const size_t need = ((bytes ? bytes : 1) + 255) & ~(size_t)255;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    *device_out = dev;
+    if (need > kPoolBigBytes) return cudaMalloc(out, need);
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    DevPool& p = g_pools[dev];
+    auto it = p.free_blocks.find(need);
+    if (it != p.free_blocks.end()) { *out = it->second; p.free_blocks.erase(it); return cudaSuccess; }
+    if (p.slab_left < need) {
+        char* slab = nullptr;
+        e = cudaMalloc((void**)&slab, kPoolSlabBytes);
+        if (e != cudaSuccess) return e;
+        p.slab = slab;                     // what was left of the previous slab stays unused
+        p.slab_left = kPoolSlabBytes;
+    }
+    *out = p.slab;
+    p.slab += need;
+    p.slab_left -= need;
+    return cudaSuccess;
+}
+
+void pool_release(void* ptr, size_t bytes, int device) {
+    if (!ptr) return;
+    const size_t need = ((bytes ? bytes : 1) + 255) & ~(size_t)255;
+    if (need > kPoolBigBytes) { cudaFree(ptr); return; }
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    g_pools[device].free_blocks.insert({need, (char*)ptr});
+}
+}  // namespace
+
 static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
 
 // ------------------------------------------------------------------------------------------
@@ -56,6 +109,8 @@ struct xp_grammar {
     // device copy, made on first use
     std::mutex mu;
     GrammarDev* d_g = nullptr;       // one block: header, leaves, binary productions
+    size_t d_bytes = 0;
+    int d_device = 0;
 };
 
 // cnt[nt][s] by the recurrence over productions and left sizes; off[s] of a binary production
@@ -138,7 +193,7 @@ extern "C" xp_status xp_grammar_create(const xp_grammar_desc* d, xp_grammar** ou
 
 extern "C" void xp_grammar_destroy(xp_grammar* g) {
     if (!g) return;
-    if (g->d_g) cudaFree(g->d_g);
+    pool_release(g->d_g, g->d_bytes, g->d_device);
     delete g;
 }
 
@@ -220,7 +275,8 @@ static xp_status grammar_to_device(xp_grammar* g) {
     const size_t off_bins = off_leaves + ((sizeof(LeafDev) * (g->leaves.size() + 1) + 255) & ~(size_t)255);
     const size_t total = off_bins + sizeof(BinDev) * (g->bins.size() + 1);
     char* block = nullptr;
-    XP_CUDA(cudaMalloc((void**)&block, total));
+    XP_CUDA(pool_alloc((void**)&block, total, &g->d_device));
+    g->d_bytes = total;
     h.leaves = (const LeafDev*)(block + off_leaves);
     h.bins = (const BinDev*)(block + off_bins);
     std::vector<char> stage(total, 0);
@@ -228,7 +284,7 @@ static xp_status grammar_to_device(xp_grammar* g) {
     if (!g->leaves.empty()) memcpy(&stage[off_leaves], g->leaves.data(), sizeof(LeafDev) * g->leaves.size());
     if (!g->bins.empty()) memcpy(&stage[off_bins], g->bins.data(), sizeof(BinDev) * g->bins.size());
     cudaError_t e = cudaMemcpy(block, stage.data(), total, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) { cudaFree(block); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
+    if (e != cudaSuccess) { pool_release(block, total, g->d_device); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
     g->d_g = (GrammarDev*)block;
     return XP_OK;
 }
@@ -255,6 +311,7 @@ struct xp_sketch {
     // 256-byte aligned pieces; anything beyond the estimate gets a block of its own.
     char* arena = nullptr;
     size_t arena_bytes = 0, arena_used = 0;
+    int arena_device = 0;
     std::vector<void*> owned;
 };
 
@@ -287,7 +344,7 @@ static u64 mix64(u64 x) {            // SplitMix64 finaliser: spreads sample ids
 extern "C" void xp_sketch_destroy(xp_sketch* s) {
     if (!s) return;
     for (void* p : s->owned) cudaFree(p);
-    if (s->arena) cudaFree(s->arena);
+    pool_release(s->arena, s->arena_bytes, s->arena_device);
     delete s;
 }
 
@@ -378,7 +435,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             while (probes > 1 && entries * 9 * probes > kTabBudgetBytes) --probes;
             need += al(sizeof(i64) * entries * probes) + al(entries * probes);
         }
-        if (cudaMalloc((void**)&s->arena, need) == cudaSuccess) s->arena_bytes = need;
+        if (pool_alloc((void**)&s->arena, need, &s->arena_device) == cudaSuccess) s->arena_bytes = need;
         else { s->arena = nullptr; (void)cudaGetLastError(); }          // fall back to piecewise allocation
     }
     SketchDev hs;
@@ -423,6 +480,15 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         }
     }
     hs.n_samples = ns;
+    {   // small searches get a cheaper probe choice: the load should not outweigh the search
+        u64 most = 0;
+        for (int h = 0; h < d->n_holes; ++h) {
+            u64 c = 0;
+            for (int k = 1; k <= d->holes[h].max_size; ++k) c += g->cnt[d->holes[h].start_nt][k];
+            most = c > most ? c : most;
+        }
+        hs.prep_cands = most <= 100000000ull ? 256 : 1024;
+    }
 
     std::vector<HoleDev> hh(d->n_holes);
     for (int h = 0; h < d->n_holes; ++h) {

@@ -84,6 +84,7 @@ struct HoleDev {
 struct SketchDev {
     const GrammarDev* g;                          // device
     i32 n_vars, n_holes, domain_kind, n_samples;
+    i32 prep_cands, pad0;                         // sampled candidates the probe choice is based on (<= 1024)
     i64 n_points;
     const i32* coords;                            // device: the points of a table domain, or the staged
                                                   // points of a box (null: derive them from the point id)

@@ -112,11 +112,11 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
         int sizes[3], nsz = 0;
         for (int k = 1; k <= 5 && k <= hole->max_size; k += 2)
             if (g->cnt[hole->start_nt][k] > 0) sizes[nsz++] = k;
-        const int ncand = nsz > 0 ? kPrepCands : 0;
+        const int ncand = nsz > 0 ? (s->prep_cands < kPrepCands ? s->prep_cands : kPrepCands) : 0;
         for (int c = t; c < ncand; c += kPrepThreads) {
             const int size = sizes[c % nsz];
             const u64 cnt = g->cnt[hole->start_nt][size];
-            const u64 per = (u64)(kPrepCands / nsz) + 1;
+            const u64 per = (u64)(ncand / nsz) + 1;
             const u64 slot = (u64)(c / nsz);
             u64 sig = 0;
             if (slot < cnt || cnt >= per) {                       // small sizes: every rank once, the rest unused
