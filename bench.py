@@ -100,6 +100,41 @@ def run_reference(args):
     }))
 
 
+def run_batch(args, xp, torch, sketches, stream):
+    """Profiling aid (single GPU): the batched workload, 4096 small instances in one
+    ``xp_repair_batch`` call per step; prints a short JSON line of its own."""
+    grammars, loaded = {}, []
+    for sk in sketches:
+        key = tuple(v.hi for v in sk.grammar.variables)
+        if key not in grammars:
+            grammars[key] = xp.xp_grammar_create(sk.grammar)
+        loaded.append(xp.xp_sketch_load(grammars[key], sk))
+    ws = torch.empty(xp.xp_workspace_bytes(loaded), dtype=torch.uint8, device="cuda")
+    peak_add, _ = xp.xp_int32_peak()
+    for _ in range(max(3, args.warmup)):
+        xp.xp_repair_batch(loaded, workspace=ws, stream=stream.cuda_stream)
+    torch.cuda.synchronize()
+    dev_ms = kern_ms = 0.0
+    evals = ops = cand = 0
+    for _ in range(args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        res = xp.xp_repair_batch(loaded, workspace=ws, stream=stream.cuda_stream)
+        e1.record(stream)
+        e1.synchronize()
+        dev_ms += e0.elapsed_time(e1)
+        kern_ms += res[0][0].kernel_ms
+        evals += sum(r[0].evals_executed for r in res)
+        ops += sum(r[0].nominal_ops for r in res)
+        cand += sum(sum(r[0].cand_count) for r in res)
+    print(json.dumps({"metric": METRIC, "value": evals / (dev_ms * 1e-3) / 1e9, "unit": UNIT, "steps": args.steps,
+                      "ms_per_step": dev_ms / args.steps, "kernel_ms_per_step": kern_ms / args.steps,
+                      "config": {"workload": "config5_batch_%d_instances" % len(loaded), "candidates_per_step": cand // args.steps},
+                      "candidates_per_s": cand / (dev_ms * 1e-3),
+                      "roofline": {"bound": "alu", "achieved": ops / (kern_ms * 1e-3) / 1e9, "peak": peak_add / 1e9,
+                                   "unit": "G int32-op/s", "frac": ops / (kern_ms * 1e-3) / peak_add}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -107,8 +142,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4"],
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5"],
                     help="profiling aid: time another config's instance instead (the bench line is config2's)")
+    ap.add_argument("--instances", type=int, default=4096,
+                    help="profiling aid: number of instances of the config5 batch (a small case of the same kernels)")
     ap.add_argument("--window", type=int, default=0,
                     help="profiling aid: search only the first WINDOW ranks of size 7 (a small case of the same kernel)")
     args = ap.parse_args()
@@ -118,7 +155,7 @@ def main():
 
     import torch
     import paper_2505_02146_b200 as xp
-    from xp_instances import config2, config3, config4
+    from xp_instances import config2, config3, config4, config5
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -132,10 +169,13 @@ def main():
     xp.load()
 
     # Independent problems shard with no data-path exchange: rank r searches the instance of seed r.
+    stream = torch.cuda.current_stream()
+    if args.workload == "config5":
+        run_batch(args, xp, torch, config5(rank, args.instances), stream)
+        return
     sk = {"config2": config2, "config3": config3, "config4": config4}[args.workload](rank)
     gr = xp.xp_grammar_create(sk.grammar)
     ls = xp.xp_sketch_load(gr, sk)
-    stream = torch.cuda.current_stream()
     ws = torch.empty(xp.xp_workspace_bytes([ls]), dtype=torch.uint8, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > L2 (126 MB), written between steps
 

@@ -441,7 +441,12 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     SketchDev hs;
     memset(&hs, 0, sizeof(hs));
     hs.g = g->d_g; hs.n_vars = nv; hs.n_holes = d->n_holes; hs.domain_kind = d->domain_kind; hs.n_points = n_points;
-    for (int v = 0; v < nv; ++v) { hs.lo[v] = g->lo[v]; hs.ext[v] = g->hi[v] - g->lo[v]; }
+    for (int v = 0; v < nv; ++v) {
+        hs.lo[v] = g->lo[v]; hs.ext[v] = g->hi[v] - g->lo[v];
+        const bool table = d->domain_kind == XP_DOMAIN_TABLE;      // a table's bounds are reduced over its rows below
+        hs.vmin[v] = table ? LLONG_MAX : g->lo[v];
+        hs.vmax[v] = table ? LLONG_MIN : g->hi[v] - 1;
+    }
     if (d->domain_kind == XP_DOMAIN_TABLE && n_points > 0) {
         if (d->coords_on_device) hs.coords = d->coords;
         else {
@@ -518,6 +523,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     hs.holes = s->d_holes;
     XP_CUDA_S(sketch_alloc(s, (void**)&s->d_s, sizeof(SketchDev)));
     XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
+    if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
     XP_CUDA_S(launch_prepare(s->d_s, nullptr));
     XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
     for (int h = 0; h < d->n_holes; ++h) s->holes[h].filter_ok = hh[h].n_probe > 0 && hh[h].aff_ok != 0;

@@ -89,6 +89,8 @@ struct SketchDev {
     const i32* coords;                            // device: the points of a table domain, or the staged
                                                   // points of a box (null: derive them from the point id)
     i64 lo[kMaxVars], ext[kMaxVars];              // box: range start and extent per variable
+    i64 vmin[kMaxVars], vmax[kMaxVars];           // smallest and largest coordinate of each variable over the domain
+                                                  // (box: from the ranges; table: reduced over the rows at load)
     HoleDev* holes;                               // device
     i64 sample_id[kProbeSamples];                 // point ids the probes are chosen from (host-chosen)
 };

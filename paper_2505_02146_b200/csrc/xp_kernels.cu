@@ -17,6 +17,8 @@
 //   int32_peak_*    -- integer-ALU peak microbenchmarks.
 #include <cuda_runtime.h>
 
+#include <climits>
+
 #include "xp_device.cuh"
 #include "xp_launch.h"
 
@@ -213,6 +215,8 @@ struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 struct CandShared {
     i32 len, depth;
     i32 cand_len;
+    i32 narrow;                  // every value the program can produce over the domain fits int32 (proved from
+                                 // the variables' coordinate bounds): the check may run in 32-bit arithmetic
     i32 var[kProgMax];           // >= 0: variable; -1: constant; -2 - op: operator
     i64 val[kProgMax];
     i32 cvar[kMaxSize];          // the candidate alone (for the slow path)
@@ -295,7 +299,8 @@ __device__ __noinline__ bool probe_check(const GrammarDev* g, const HoleDev* hol
     return true;
 }
 
-__device__ __noinline__ void stage_candidate(CandShared& c, const GrammarDev* g, const HoleDev* hole, int size, u64 rank) {
+__device__ __noinline__ void stage_candidate(CandShared& c, const SketchDev* sk, const HoleDev* hole, int size, u64 rank) {
+    const GrammarDev* g = sk->g;
     u32 code[kMaxSize];
     const int n = unrank(g, hole->start_nt, size, rank, code);
     c.cand_len = n;
@@ -303,13 +308,37 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const GrammarDev* g,
         if (code[k] & kOpBit) { c.cvar[k] = -2 - (i32)(code[k] & 0xff); c.cval[k] = 0; }
         else { const LeafDev lf = g->leaves[code[k]]; c.cvar[k] = lf.var >= 0 ? lf.var : -1; c.cval[k] = lf.value; }
     }
-    // the context with the candidate in place of each HOLE
+    // the context with the candidate in place of each HOLE; alongside, an upper bound of the
+    // magnitude of every value on the operand stack (saturating at 2^62), from the coordinate
+    // bounds of the variables: if no bound reaches 2^31 the program is exact in int32
     int len = 0, sp = 0, depth = 0;
-    bool fits = true;
+    bool fits = true, narrow = true;
+    constexpr u64 kSat = 1ull << 62;
+    u64 mag[kMaxStack + kCandStack + 1];
+    auto mag_of = [](i64 v) { return v < 0 ? 0ull - (u64)v : (u64)v; };
     auto emit = [&](i32 var, i64 val) {
-        if (len >= kProgMax) { fits = false; return; }
+        if (len >= kProgMax || sp > kMaxStack + kCandStack - 1) { fits = false; return; }
         c.var[len] = var; c.val[len] = val; ++len;
-        if (var >= -1) { if (++sp > depth) depth = sp; } else --sp;
+        u64 m;
+        if (var >= -1) {
+            if (var >= 0) { const u64 a = mag_of(sk->vmin[var]), b = mag_of(sk->vmax[var]); m = a > b ? a : b; }
+            else m = mag_of(val);
+            mag[sp] = m < kSat ? m : kSat;
+            if (++sp > depth) depth = sp;
+        } else {
+            --sp;
+            const u64 a = mag[sp - 1], b = mag[sp];
+            switch (-2 - var) {
+                case XP_OP_ADD: case XP_OP_SUB: m = a + b; break;
+                case XP_OP_MUL: m = (a >> 31 || b >> 31) ? kSat : a * b; break;
+                case XP_OP_DIV: m = a; break;
+                case XP_OP_MOD: m = a < b ? a : b; break;
+                case XP_OP_MIN: case XP_OP_MAX: m = a > b ? a : b; break;
+                default: m = 1; break;
+            }
+            mag[sp - 1] = m < kSat ? m : kSat;
+        }
+        narrow = narrow && (m >> 31) == 0;
     };
     if (hole->ctx_len == 0) {
         for (int k = 0; k < n; ++k) emit(c.cvar[k], c.cval[k]);
@@ -325,6 +354,7 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const GrammarDev* g,
     for (int i = 0; i < hole->ctx_len; ++i) has_hole = has_hole || hole->ctx[i].kind == XP_I_HOLE;
     c.len = len;
     c.depth = (fits && has_hole) ? depth : 0;     // a context that ignores the hole still needs the candidate to be defined
+    c.narrow = narrow ? 1 : 0;
 }
 
 // The staged program at one point with an operand stack of D registers (D >= its depth): a
@@ -385,6 +415,106 @@ __device__ __forceinline__ bool check_points_fast(const CandShared& c, const Ske
     return true;
 }
 
+// Stage 3, the form the verification kernel uses: every lane runs the staged program on P
+// points at once (points base + i*32 + lane, so that the table reads of a step are coalesced),
+// 32*P points per step and warp vote.  The top of the operand stack is kept in registers; the
+// entries below it live in shared memory, one 16-byte slot per lane and level (read and
+// written as one vector access).  T = i32 with P = 4 when the program is proved exact in
+// int32 (CandShared::narrow), else T = i64 with P = 2.  The program is the same for all
+// lanes, so the dispatch branches are uniform.  Points and spec values come from the tables.
+constexpr int kVecDepth = 8;                              // deepest operand stack this form takes
+template <typename T, int P>
+__device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __restrict__ stack, const SketchDev* sk,
+                                                 const HoleDev* hole, i64 first, i64 last) {
+    static_assert(sizeof(T) * P == sizeof(uint4), "one stack level of a lane is one 16-byte slot");
+    const int nv = sk->n_vars;
+    const int lane = threadIdx.x & 31;
+    const int n = c.len;
+    const i32* __restrict__ coords = sk->coords;
+    const i64* __restrict__ spec = hole->spec_table;
+    union Slot { uint4 q; T v[P]; };
+    for (i64 base = first; base < last; base += 32 * P) {
+        const i32* row[P];
+        i64 want[P];
+        bool in[P];
+#pragma unroll
+        for (int i = 0; i < P; ++i) {
+            const i64 pid = base + i * 32 + lane;
+            in[i] = pid < last;
+            const i64 at = in[i] ? pid : first;           // lanes past the end repeat a valid point
+            row[i] = coords + at * nv;
+            want[i] = spec[at];
+        }
+        Slot t;
+#pragma unroll
+        for (int i = 0; i < P; ++i) t.v[i] = 0;
+        bool bad = false;
+        int below = 0;                                    // entries under the top of the stack
+        for (int k = 0; k < n; ++k) {
+            const i32 cv = c.var[k];
+            if (cv >= -1) {
+                stack[below * 32 + lane] = t.q;           // (the very first push stores an unused slot)
+                ++below;
+                if (cv >= 0) {
+#pragma unroll
+                    for (int i = 0; i < P; ++i) t.v[i] = (T)row[i][cv];
+                } else {
+                    const T v = (T)c.val[k];
+#pragma unroll
+                    for (int i = 0; i < P; ++i) t.v[i] = v;
+                }
+                continue;
+            }
+            --below;
+            Slot a;
+            a.q = stack[below * 32 + lane];
+            const int op = -2 - cv;
+            if (sizeof(T) == 8) {
+#pragma unroll
+                for (int i = 0; i < P; ++i) {
+                    i64 r = 0;
+                    bad |= !apply_op(op, (i64)a.v[i], (i64)t.v[i], r);
+                    t.v[i] = (T)r;
+                }
+                continue;
+            }
+            switch (op) {                                 // int32: no result can overflow (proved at staging)
+#define XP_EACH(expr) _Pragma("unroll") for (int i = 0; i < P; ++i) { const i32 x = (i32)a.v[i], y = (i32)t.v[i]; t.v[i] = (T)(expr); } break;
+                case XP_OP_ADD: XP_EACH(x + y)
+                case XP_OP_SUB: XP_EACH(x - y)
+                case XP_OP_MUL: XP_EACH(x * y)
+                case XP_OP_DIV:
+                case XP_OP_MOD:
+#pragma unroll
+                    for (int i = 0; i < P; ++i) {
+                        const i32 x = (i32)a.v[i], y = (i32)t.v[i];
+                        bad |= y == 0;
+                        const i32 d = y == 0 ? 1 : y;     // |x| < 2^31, so x / -1 does not overflow
+                        const i32 q = x / d;
+                        t.v[i] = (T)(op == XP_OP_DIV ? q : x - q * d);
+                    }
+                    break;
+                case XP_OP_LT: XP_EACH(x < y)
+                case XP_OP_LE: XP_EACH(x <= y)
+                case XP_OP_EQ: XP_EACH(x == y)
+                case XP_OP_NE: XP_EACH(x != y)
+                case XP_OP_MIN: XP_EACH(x < y ? x : y)
+                case XP_OP_MAX: XP_EACH(x > y ? x : y)
+                case XP_OP_AND: XP_EACH((x != 0) & (y != 0))
+                case XP_OP_OR: XP_EACH((x != 0) | (y != 0))
+#undef XP_EACH
+                default: bad = true; break;
+            }
+        }
+        // a zero divisor at a repeated point is a zero divisor at a real point of this candidate
+        // too (the repeated point is `first`, which lane 0 holds in range), so `bad` needs no mask
+#pragma unroll
+        for (int i = 0; i < P; ++i) bad |= in[i] && (i64)t.v[i] != want[i];
+        if (__any_sync(0xffffffffu, bad)) return false;
+    }
+    return true;
+}
+
 __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
                                           i64 last, u64& evals) {
     if (sk->coords != nullptr && hole->spec_table != nullptr && c.depth >= 1) {
@@ -440,7 +570,7 @@ __device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& pla
 __device__ __noinline__ void warp_verify(EvalShared& sh, const SketchDev* sk, const HoleDev* hole, int size, u64 rank,
                                          u64& my_evals) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) stage_candidate(sh.wcand[warp], sk->g, hole, size, rank);
+    if (lane == 0) stage_candidate(sh.wcand[warp], sk, hole, size, rank);
     __syncwarp();
     const bool ok = check_points(sh.wcand[warp], sk, hole, 0, sk->n_points, my_evals);
     if (ok && lane == 0) {
@@ -625,6 +755,28 @@ __global__ void __launch_bounds__(256) stage_points_kernel(const SketchDev* sk, 
         divmod_u64(rem, (u64)sk->ext[d], q, r);
         coords[pid * nv + d] = (i32)(sk->lo[d] + (i64)r);
         rem = q;
+    }
+}
+
+// Smallest and largest coordinate of every variable over the rows of a table domain, into the
+// sketch (whose vmin / vmax start at the extreme values).  Warp shuffles, then one atomic pair
+// per warp and variable.
+__global__ void __launch_bounds__(256) coord_bounds_kernel(SketchDev* sk) {
+    const int nv = sk->n_vars;
+    const i64 n = sk->n_points;
+    for (int v = 0; v < nv; ++v) {
+        i64 lo = LLONG_MAX, hi = LLONG_MIN;
+        for (i64 pid = (i64)blockIdx.x * blockDim.x + threadIdx.x; pid < n; pid += (i64)gridDim.x * blockDim.x) {
+            const i64 x = sk->coords[pid * nv + v];
+            lo = x < lo ? x : lo;
+            hi = x > hi ? x : hi;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const i64 l2 = __shfl_down_sync(0xffffffffu, lo, o), h2 = __shfl_down_sync(0xffffffffu, hi, o);
+            lo = l2 < lo ? l2 : lo;
+            hi = h2 > hi ? h2 : hi;
+        }
+        if ((threadIdx.x & 31) == 0 && lo <= hi) { atomicMin(&sk->vmin[v], lo); atomicMax(&sk->vmax[v], hi); }
     }
 }
 
@@ -1255,6 +1407,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 // already failed is skipped; lane 0 reads that flag once and shares the decision.
 __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
     __shared__ CandShared cands[kWarps];
+    __shared__ uint4 stacks[kWarps][kVecDepth * 32];    // operand stacks below the top, per warp, level and lane
     CandShared& cand = cands[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const u32 pushed = *plan.surv_n;
@@ -1271,7 +1424,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
                 const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
                 if ((i64)(t / n) * kVerifyChunk < sk->n_points && !failed) {
                     skip = 0;
-                    stage_candidate(cand, sk->g, &sk->holes[sv->hole], sv->size, sv->rank);
+                    stage_candidate(cand, sk, &sk->holes[sv->hole], sv->size, sv->rank);
                 }
             }
         }
@@ -1286,7 +1439,14 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
         const i64 first = (i64)(t / n) * kVerifyChunk;
         const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
         u64 evals = 0;
-        const bool ok = check_points(cand, sk, hole, first, last, evals);
+        bool ok;
+        if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
+            uint4* stack = stacks[threadIdx.x >> 5];
+            ok = cand.narrow ? check_points_vec<i32, 4>(cand, stack, sk, hole, first, last)
+                             : check_points_vec<i64, 2>(cand, stack, sk, hole, first, last);
+        } else {
+            ok = check_points(cand, sk, hole, first, last, evals);
+        }
         if (lane == 0) {
             if (ok) atomicAdd(&sv->state, 1u); else atomicOr(&sv->state, kSurvFailed);
             atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
@@ -1367,6 +1527,13 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 
 cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream) {
     prepare_kernel<<<1, kPrepThreads, 0, stream>>>(s);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_coord_bounds(SketchDev* s, i64 n_points, cudaStream_t stream) {
+    if (n_points <= 0) return cudaSuccess;
+    const i64 blocks = (n_points + 255) / 256;
+    coord_bounds_kernel<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, stream>>>(s);
     return cudaGetLastError();
 }
 
