@@ -547,6 +547,15 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         o.tab_max_size = tmax;
         o.tab_probes = probes;
         o.tab_total = total;
+        {   // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
+            // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
+            // probe 0 alone lets many through.
+            u64 cands = 0;
+            for (int k = 1; k <= o.max_size; ++k) cands += g->cnt[o.start_nt][k];
+            const bool possible = o.n_probe >= 2 && probes >= 2 && ((o.probe_spec_ok & o.aff_okmask) >> 1 & 1u);
+            const bool frequent = o.sample_n > 0 && (u64)o.sample_pass0 * 256 >= (u64)o.sample_n;
+            o.second = possible && (cands <= 100000000ull || frequent) ? 1 : 0;
+        }
         XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &o, sizeof(HoleDev), cudaMemcpyHostToDevice));
         for (int k = 1; k <= tmax; ++k) {
             u64 at_size = 0;

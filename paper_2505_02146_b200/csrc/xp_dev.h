@@ -74,6 +74,10 @@ struct HoleDev {
     // The tables exist for the probes 0 .. tab_probes-1, one copy after the other (stride tab_total).
     // Hits of the filter are checked exactly there (two lookups and one operation per probe); only
     // probes without tables need the candidate unranked in full.
+    // second: filter hits are also checked exactly at probe 1 before they are queued (needs tables, a
+    // defined spec and an affine context at probe 1); sample_pass0: how many of the candidates
+    // sampled at load satisfied probe 0 (a high rate makes the second look worth its cost).
+    i32 second, sample_pass0, sample_n, pad1;
     i32 tab_max_size, tab_probes;
     u64 tab_total;
     u64 tab_off[kMaxNt][kMaxSize + 1];

@@ -166,6 +166,12 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
         if (t == 0) {
             hole->n_probe = n;
             if (n == 0) hole->probe_spec_ok = 0;
+            int pass0 = 0;                                  // sampled candidates that satisfy the first probe chosen
+            for (int i = 0; i < ns; ++i)
+                if (n > 0 && s->sample_id[i] == hole->probe_id[0])
+                    for (int c = 0; c < ncand; ++c) pass0 += (int)((s_sig[c] >> i) & 1ull);
+            hole->sample_pass0 = pass0;
+            hole->sample_n = ncand;
             u64 A = 0, B = 0;
             hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
             hole->aff_A = A;
@@ -203,7 +209,8 @@ static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the 
 //           b = 2^k * o (o odd), mask = 2^(32-k) - 1, tm = (tp >> k) * o^-1 & mask, provided the
 //           low k bits of tp are zero (else tm lies outside the mask and nothing matches);
 //   BcDiv:  magnitudes for / and %, see div_pass;
-//   BcMeta: the value itself, and meta = index inside the tile | ctz(|value|) << 16.
+//   BcMeta: the value itself, meta = index inside the tile | ctz(|value|) << 16 | bit 31: pad holds
+//           the operand's exact value at probe 1 (second look).
 struct __align__(16) BcRing { u32 t_add, t_pm, mul_mask, mul_tm; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
@@ -249,6 +256,9 @@ struct EvalShared {
     i32 kept_wide[8];
     u32 wq_n[kWarps], wq_over[kWarps];
     i32 tile_wide;               // some operand of the tile does not fit int32
+    // second look (HoleDev::second): context factor, offset and spec value at probe 1 of the hole at hand
+    i32 p1_on;
+    u64 p1_A, p1_B, p1_spec;
     BcRing bc_ring[kBcTile];
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
@@ -684,15 +694,16 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
     return eval_cand(code, n, g->leaves, hole->probe_pt[pr], v);
 }
 
-// Values at probe 0 of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
+// Values at probe `pr` of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
 // returns the mask of those that are defined there and sets `wide` if one does not fit int32.
 // A subtree above the table sizes whose operands are in the tables is unranked one level for
 // the first rank only; the following ranks advance the operand ranks like an odometer (right
 // operand fastest), so the left operand's value is fetched once per run.
-__device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank,
+__device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev* hole, int pr, int nt, int size, u64 rank,
                                               int n, i64* out, bool& wide) {
     u32 alive = 0;
     const int tmax = hole->tab_max_size;
+    const u64 pbase = (u64)pr * hole->tab_total;
     for (int j = 0; j < kNA; ++j) out[j] = 0;
     if (n <= 0) return 0;
     if (size > tmax && tmax >= 1 && size >= 3) {
@@ -703,7 +714,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
         int j = 0;
         while (tables && j < n) {
             const u64 cl = g->cnt[lnt][a], cr = g->cnt[rnt][size - 1 - a];
-            const u64 lbase = hole->tab_off[lnt][a], rbase = hole->tab_off[rnt][size - 1 - a];
+            const u64 lbase = pbase + hole->tab_off[lnt][a], rbase = pbase + hole->tab_off[rnt][size - 1 - a];
             for (; j < n && l < cl; ++l, r = 0) {
                 const bool lok = hole->tab_ok[lbase + l] != 0;
                 const i64 lv = hole->tab_val[lbase + l];
@@ -725,7 +736,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
         if (j == n) return alive;
         for (; j < n; ++j) {
             i64 v;
-            if (operand_value(g, hole, 0, nt, size, rank + j, v)) {
+            if (operand_value(g, hole, pr, nt, size, rank + j, v)) {
                 out[j] = v; alive |= 1u << j;
                 wide |= !(v > -(1ll << 31) && v < (1ll << 31));
             }
@@ -734,7 +745,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
     }
     for (int j = 0; j < n; ++j) {
         i64 v;
-        if (operand_value(g, hole, 0, nt, size, rank + j, v)) {
+        if (operand_value(g, hole, pr, nt, size, rank + j, v)) {
             out[j] = v; alive |= 1u << j;
             wide |= !(v > -(1ll << 31) && v < (1ll << 31));
         }
@@ -842,8 +853,23 @@ struct RegOps {
     u32 inv[kNA];    // inverse mod 2^32 of the odd part of |value|
     u32 kk[kNA];     // number of trailing zero bits of |value|
     u32 cc[kNA];     // floor((2^32-1) / |value|), or 0 when the remainder tabs is impossible
-    u32 alive;       // bit j: operand j exists and is valid at probe 0
+    u32 alive;       // bit j: operand j exists and is valid at probe 0 (and at probe 1, when that is looked at)
+    i32 a1[kNA];     // value at probe 1
+    u32 a1ok;        // bit j: a1[j] is the exact value (it fits int32)
 };
+
+// The second look: the candidate's exact value at probe 1 from its operands' values there,
+// through the affine context, against the spec.  Operand values that are not known exactly in
+// int32 pass (the exact stages decide).  Runs for filter hits only.
+__device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok, i32 a1, u32 bc_meta, u32 b1, bool swap) {
+    if (!sh.p1_on) return true;
+    if (!a_ok || !(bc_meta >> 31)) return true;
+    const i64 x = swap ? (i64)(i32)b1 : (i64)a1, y = swap ? (i64)a1 : (i64)(i32)b1;
+    i64 v;
+    if (!apply_op(op, x, y, v)) return false;
+    return (u64)v * sh.p1_A + sh.p1_B == sh.p1_spec;
+}
+#define XP_P1(op, j, s) probe1_pass(sh, op, (Rm->a1ok >> (j)) & 1u, Rm->a1[j], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
 
 // The loops below are separate (not inlined) functions on purpose: each copies just the
 // operand arrays it needs from the tile's RegOps into registers and runs with a small live
@@ -856,6 +882,42 @@ constexpr int kSlotMin = 5, kSlotMax = 6;
 
 // x and -x have the same sign-free form: the smaller of the two as unsigned numbers.
 __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x < y ? x : y; }
+
+// The rare paths of the loops below: a warp vote said that some lane has a hit among the
+// candidates of broadcast slot s.  Each lane repeats its tests from registers and collects bit
+// sets of the register operands that hit; a lane with a non-empty set calls one of these
+// compact functions, which walks the set bits, looks at each hit once more at probe 1 (when
+// the hole has that second look) and queues what is left.  Keeping this part out of line and
+// rolled keeps the loops' instruction footprint small, which matters where the filter is not
+// selective (small value ranges) and the rare path is not rare.
+__device__ __noinline__ void emit_ring(EvalShared& sh, const RegOps* Rm, int s, u32 m_as, u32 m_mul, u32 tp, u32 opip,
+                                       u32 mask, bool SWAP) {
+    const BcRing e = sh.bc_ring[s];
+    const u32 t_sub = SWAP ? 0u - e.t_add : 2u * tp - e.t_add;
+    for (u32 m = m_as; m; m &= m - 1) {                 // + and -: which of the two (or both) it was
+        const int j = __ffs((int)m) - 1;
+        const u32 a = Rm->aA[j];
+        const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
+        if ((mask & 1u) && a == e.t_add && XP_P1(XP_OP_ADD, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
+        if ((mask & 2u) && a == t_sub && XP_P1(XP_OP_SUB, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
+    }
+    for (u32 m = m_mul; m; m &= m - 1) {
+        const int j = __ffs((int)m) - 1;
+        if (XP_P1(XP_OP_MUL, j, s)) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
+    }
+}
+
+__device__ __noinline__ void emit_pairs(EvalShared& sh, const RegOps* Rm, int s, u32 m0, int op0, u32 m1, int op1, u32 opip,
+                                        bool SWAP) {
+    for (u32 m = m0; m; m &= m - 1) {
+        const int j = __ffs((int)m) - 1;
+        if (XP_P1(op0, j, s)) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (opip >> (3 * op_slot(op0))) & 7u);
+    }
+    for (u32 m = m1; m; m &= m - 1) {
+        const int j = __ffs((int)m) - 1;
+        if (XP_P1(op1, j, s)) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (opip >> (3 * op_slot(op1))) & 7u);
+    }
+}
 
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
 // MASK: bit0 +, bit1 -, bit2 *.  The comparisons were brought to the register operand's side
@@ -884,15 +946,16 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     };
     auto resolve = [&](int s) {                          // the rare path: which candidates hit
         const BcRing e = sh.bc_ring[s];
-        const u32 t_sub = t_sub_of(e.t_add);
+        const u32 t_one = (MASK & 1u) ? e.t_add : t_sub_of(e.t_add);
+        u32 m_as = 0, m_mul = 0;
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
-            if (!((alive >> j) & 1u)) continue;
-            const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-            if ((MASK & 1u) && aA[j] == e.t_add) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
-            if ((MASK & 2u) && aA[j] == t_sub) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
-            if ((MASK & 4u) && (aA[j] & e.mul_mask) == e.mul_tm) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MUL)) & 7u);
+            if (kPair) m_as |= (u32)(ca[j] == e.t_pm) << j;
+            else if (MASK & 3u) m_as |= (u32)(aA[j] == t_one) << j;
+            if (MASK & 4u) m_mul |= (u32)((aA[j] & e.mul_mask) == e.mul_tm) << j;
         }
+        m_as &= alive; m_mul &= alive;
+        if (m_as | m_mul) emit_ring(sh, Rm, s, m_as, m_mul, tp, opip, MASK, SWAP);
     };
     int s = s0;
     for (; s + 4 <= s1; s += 4) {                       // one warp vote per four broadcast operands
@@ -955,22 +1018,25 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
         }
     };
     auto resolve = [&](const BcDiv& e, u32 ek, int s) {
+        u32 mq = 0, mr = 0, nz = 0;
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
-            // register operands that are invalid, or (SWAP) zero divisors, are dropped here
-            if (!((alive >> j) & 1u) || (SWAP && ua[j] == 0u)) continue;
             bool hq, hr;
             test(e, ek, j, hq, hr);
-            const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-            if ((MASK & 1u) && hq) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
-            if ((MASK & 2u) && hr) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
+            if (MASK & 1u) mq |= (u32)hq << j;
+            if (MASK & 2u) mr |= (u32)hr << j;
+            nz |= (u32)(ua[j] != 0u) << j;
         }
+        // register operands that are invalid, or (SWAP) zero divisors, are dropped here
+        const u32 keep = SWAP ? alive & nz : alive;
+        mq &= keep; mr &= keep;
+        if (mq | mr) emit_pairs(sh, Rm, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     };
     const bool need_k = !SWAP && !SPECIAL && (MASK & 2u);
     int s = s0;
     for (; s + 2 <= s1; s += 2) {                       // one warp vote per two broadcast operands
         const BcDiv e0 = sh.bc_div[s], e1 = sh.bc_div[s + 1];
-        const u32 k0 = need_k ? sh.bc_meta[s].meta >> 16 : 0u, k1 = need_k ? sh.bc_meta[s + 1].meta >> 16 : 0u;
+        const u32 k0 = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u, k1 = need_k ? (sh.bc_meta[s + 1].meta >> 16) & 63u : 0u;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
         scan(e0, k0, h0, h1, h2, h3);
         scan(e1, k1, h0, h1, h2, h3);
@@ -978,7 +1044,7 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
     }
     for (; s < s1; ++s) {
         const BcDiv e0 = sh.bc_div[s];
-        const u32 k0 = need_k ? sh.bc_meta[s].meta >> 16 : 0u;
+        const u32 k0 = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
         scan(e0, k0, h0, h1, h2, h3);
         if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(e0, k0, s);
@@ -1010,15 +1076,16 @@ __device__ __noinline__ void minmax_pass(EvalShared& sh, const RegOps* Rm, u32 a
             if (MASK & 2u) { h2 |= x0; h3 |= x1; }
         }
         if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
+            u32 mmin = 0, mmax = 0;
 #pragma unroll
             for (int j = 0; j < kNA; ++j) {
-                if (!((alive >> j) & 1u)) continue;
                 bool hmin, hmax;
                 test(b, j, hmin, hmax);
-                const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-                if ((MASK & 1u) && hmin) push_hit(sh, idx, (u32)s, (opip >> (3 * kSlotMin)) & 7u);
-                if ((MASK & 2u) && hmax) push_hit(sh, idx, (u32)s, (opip >> (3 * kSlotMax)) & 7u);
+                if (MASK & 1u) mmin |= (u32)hmin << j;
+                if (MASK & 2u) mmax |= (u32)hmax << j;
             }
+            mmin &= alive; mmax &= alive;
+            if (mmin | mmax) emit_pairs(sh, Rm, s, mmin, XP_OP_MIN, mmax, XP_OP_MAX, opip, false);
         }
     }
 }
@@ -1039,15 +1106,16 @@ __device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegOps* Rm, u
             const i32 q = n / d;                         // magnitudes are below 2^31: no overflow case
             const u32 r = (u32)n - (u32)q * (u32)d;
             const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
-            if ((mask & 8u) && (u32)q * A == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
-            if ((mask & 16u) && r * A == tp) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
+            if ((mask & 8u) && (u32)q * A == tp && XP_P1(XP_OP_DIV, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_DIV)) & 7u);
+            if ((mask & 16u) && r * A == tp && XP_P1(XP_OP_MOD, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_MOD)) & 7u);
         }
     }
 }
 
 // Any operator on int64 operands (tiles with an operand outside int32): exact, slow, rare.
-__device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive, bool swap, u64 A, u64 tq,
+__device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, const RegOps* Rm, u32 alive, bool swap, u64 A, u64 tq,
                                         int s0, int s1, int n_ops, const i32* ops) {
+    const bool SWAP = swap;
     for (int s = s0; s < s1; ++s) {
         const i64 b = (i64)(((u64)sh.bc_meta[s].hi << 32) | sh.bc_meta[s].lo);
         for (int j = 0; j < kNA; ++j) {
@@ -1055,7 +1123,7 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, u32 alive,
             for (int o = 0; o < n_ops; ++o) {
                 i64 v;
                 if (!apply_op(ops[o], swap ? b : a[j], swap ? a[j] : b, v)) continue;
-                if ((u64)v * A == tq) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
+                if ((u64)v * A == tq && XP_P1(ops[o], j, s)) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
             }
         }
     }
@@ -1114,7 +1182,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
 
 template <bool SWAP>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
-                                          u64 bc_first, int n_reg, i64* a64, u32 alive, u64& my_evals) {
+                                          u64 bc_first, int n_reg, i64* a64, const i32* a1, u32 a1ok, u32 alive, u64& my_evals) {
     const SegDev& seg = sh.seg;
     const int nb = (int)sh.bc_n, bc_lo = sh.bc_lo, bc_hi = sh.bc_hi;
     const bool tile_wide = sh.tile_wide != 0;
@@ -1131,6 +1199,8 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     RegOps R;
     R.alive = alive;
     R.neg = 0;
+    R.a1ok = a1ok;
+    if (sh.p1_on) for (int j = 0; j < kNA; ++j) R.a1[j] = a1[j];
     // Only the arrays that this segment's loops read are written (the struct lives in the
     // thread's local memory, and every store there is traffic).
     const bool want_ring = (mask & 7u) != 0, want_div = (mask & 24u) != 0, want_mm = (mask >> kSlotMin) != 0;
@@ -1162,7 +1232,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
     auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide) {
-            wide_chunk(sh, a64, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
+            wide_chunk(sh, a64, &R, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
             return;
         }
         switch (mask & 7u) {
@@ -1242,6 +1312,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
 __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, u64 bc_first, int n_bc) {
     const SegDev& seg = sh.seg;
     const bool swap = seg.swap != 0;
+    const bool second = hole->second != 0;
     const u32 fA = (u32)hole->aff_A;
     const u64 ftq = (u64)hole->probe_spec[0] - hole->aff_B;
     const u32 ftp = (u32)ftq;
@@ -1250,6 +1321,9 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
     for (int i = threadIdx.x; i < n_bc; i += kThreads) {
         i64 v;
         if (!operand_value(g, hole, 0, seg.bc_nt, seg.bc_size, bc_first + i, v)) continue;
+        i64 v1 = 0;                                         // second look: value at probe 1 (undefined there: no match)
+        if (second && !operand_value(g, hole, 1, seg.bc_nt, seg.bc_size, bc_first + i, v1)) continue;
+        const bool v1_exact = second && v1 > -(1ll << 31) && v1 < (1ll << 31);
         const bool special = v >= -1 && v <= 1;
         const u32 slot = special ? (u32)sh.bc_hi - 1u - atomicAdd(&sh.bc_nspecial, 1u) : (u32)sh.bc_lo + atomicAdd(&sh.bc_n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
@@ -1258,7 +1332,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         const u32 k = ub ? (u32)__ffs((int)ub) - 1u : 0u;
         const u32 io = ub ? inv_odd(ub >> k) : 1u;          // inverse of the odd part of |v|
         BcMeta m;
-        m.lo = b; m.hi = (u32)((u64)v >> 32); m.meta = (u32)i | (k << 16); m.pad = 0;
+        m.lo = b; m.hi = (u32)((u64)v >> 32); m.meta = (u32)i | (k << 16) | (v1_exact ? 0x80000000u : 0u); m.pad = (u32)(u64)v1;
         sh.bc_meta[slot] = m;
         // + and -: the value A*a must have; *: mask and value of A*a's low bits
         BcRing r;
@@ -1310,8 +1384,28 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     i64 a64[kNA];
     bool wide_reg = false;
     const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
-    const u32 alive = fill_reg_operands(g, hole, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
-                                        mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
+    u32 alive = fill_reg_operands(g, hole, 0, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+                                  mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
+    // second look: the same operands at probe 1; one that is undefined there can be in no match
+    i32 a1[kNA];
+    u32 a1ok = 0;
+    const bool second = hole->second != 0;
+    if (second) {
+        i64 b64[kNA];
+        bool wide1 = false;
+        alive &= fill_reg_operands(g, hole, 1, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+                                   mine < 0 ? 0 : (mine > kNA ? kNA : mine), b64, wide1);
+        for (int j = 0; j < kNA; ++j) {
+            a1[j] = (i32)b64[j];
+            if (b64[j] > -(1ll << 31) && b64[j] < (1ll << 31)) a1ok |= 1u << j;
+        }
+    } else {
+        for (int j = 0; j < kNA; ++j) a1[j] = 0;
+    }
+    if (threadIdx.x == 0) {
+        sh.p1_on = second ? 1 : 0;
+        sh.p1_A = hole->aff_Aj[1]; sh.p1_B = hole->aff_Bj[1]; sh.p1_spec = (u64)hole->probe_spec[1];
+    }
     const bool keep = sh.seg.bc_keep != 0;
     const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
     for (int m = 0; m < family; ++m) {
@@ -1344,8 +1438,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         if (wide_reg) sh.tile_wide = 1;                 // the kept flag is the broadcast side's alone
         __syncthreads();
         if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, alive, my_evals);
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, a1, a1ok, alive, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, a1, a1ok, alive, my_evals);
     }
 }
 
