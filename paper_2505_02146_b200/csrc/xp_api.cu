@@ -433,7 +433,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             const u64 entries = table_entries(g, hd.max_size, nullptr, nullptr);
             u64 probes = kMaxProbe;
             while (probes > 1 && entries * 9 * probes > kTabBudgetBytes) --probes;
-            need += al(sizeof(i64) * entries * probes) + al(entries * probes);
+            need += al(sizeof(i64) * entries * probes) + al(entries * probes) + al(entries);
         }
         if (pool_alloc((void**)&s->arena, need, &s->arena_device) == cudaSuccess) s->arena_bytes = need;
         else { s->arena = nullptr; (void)cudaGetLastError(); }          // fall back to piecewise allocation
@@ -514,6 +514,13 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
                 o.spec_table = (const i64*)p;
             }
         }
+        {   // variables the context and the spec mention (a caller's spec table may depend on all)
+            u32 fv = hd.spec_kind == XP_SPEC_EXPR ? 0u : 0xffffffffu;
+            for (int i = 0; i < hd.ctx_len; ++i) if (hd.ctx[i].kind == XP_I_VAR) fv |= 1u << hd.ctx[i].arg;
+            if (hd.spec_kind == XP_SPEC_EXPR)
+                for (int i = 0; i < hd.spec_len; ++i) if (hd.spec_expr[i].kind == XP_I_VAR) fv |= 1u << hd.spec_expr[i].arg;
+            o.fixed_vars = fv;
+        }
         HoleHost ho;
         ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
         s->holes.push_back(ho);
@@ -542,8 +549,11 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         while (probes > 1 && total * 9 * (u64)probes > kTabBudgetBytes) --probes;
         XP_CUDA_S(sketch_alloc(s, &pv, sizeof(i64) * total * probes));
         XP_CUDA_S(sketch_alloc(s, &pk, total * probes));
+        void* pm = nullptr;
+        XP_CUDA_S(sketch_alloc(s, &pm, total));
         o.tab_val = (i64*)pv;
         o.tab_ok = (unsigned char*)pk;
+        o.tab_vars = (unsigned char*)pm;
         o.tab_max_size = tmax;
         o.tab_probes = probes;
         o.tab_total = total;
@@ -574,6 +584,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             XP_CUDA_S(launch_stage_points(s->d_s, n_points, (i32*)p, nullptr));
             XP_CUDA_S(cudaStreamSynchronize(nullptr));       // the kernel reads the sketch before its coords field changes
             hs.coords = (const i32*)p;
+            hs.project = 1;
             XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
         }
         u32* d_bad = nullptr;

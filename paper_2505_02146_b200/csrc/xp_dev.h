@@ -83,12 +83,17 @@ struct HoleDev {
     u64 tab_off[kMaxNt][kMaxSize + 1];
     i64* tab_val;                                 // device
     unsigned char* tab_ok;                        // device
+    unsigned char* tab_vars;                      // device, one copy: bit v set if variable v occurs in the subtree
+    // Variables that the context or the spec expression mention (all of them when the spec is the
+    // caller's table).  On a box domain a candidate is checked on the sub-box of these and its
+    // own variables only: no other variable can change either side of the constraint.
+    u32 fixed_vars, pad2;
 };
 
 struct SketchDev {
     const GrammarDev* g;                          // device
     i32 n_vars, n_holes, domain_kind, n_samples;
-    i32 prep_cands, pad0;                         // sampled candidates the probe choice is based on (<= 1024)
+    i32 prep_cands, project;                      // project: box domain with staged points (see HoleDev::fixed_vars)                         // sampled candidates the probe choice is based on (<= 1024)
     i64 n_points;
     const i32* coords;                            // device: the points of a table domain, or the staged
                                                   // points of a box (null: derive them from the point id)
@@ -140,7 +145,7 @@ struct SegDev {
 // that passed, its top bit says that some point failed.
 constexpr int kVerifyChunk = 4096;
 constexpr u32 kSurvFailed = 0x80000000u;
-struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, pad; };
+struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, vars; };   // vars: variables the candidate mentions
 
 struct PlanDev {
     u64 n_tickets;

@@ -222,6 +222,10 @@ struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 struct CandShared {
     i32 len, depth;
     i32 cand_len;
+    // Sub-box the check runs on (see proj_points): its variables from the fastest down, with the
+    // extent of each and its stride in point ids of the full box; n_proj_vars == 0: every point.
+    i32 n_proj_vars;
+    u32 proj_ext[kMaxVars], proj_stride[kMaxVars];
     i32 narrow;                  // every value the program can produce over the domain fits int32 (proved from
                                  // the variables' coordinate bounds): the check may run in 32-bit arithmetic
     i32 var[kProgMax];           // >= 0: variable; -1: constant; -2 - op: operator
@@ -363,6 +367,7 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const SketchDev* sk,
     bool has_hole = hole->ctx_len == 0;
     for (int i = 0; i < hole->ctx_len; ++i) has_hole = has_hole || hole->ctx[i].kind == XP_I_HOLE;
     c.len = len;
+    c.n_proj_vars = 0;                            // every point, unless the caller sets a sub-box (proj_points)
     c.depth = (fits && has_hole) ? depth : 0;     // a context that ignores the hole still needs the candidate to be defined
     c.narrow = narrow ? 1 : 0;
 }
@@ -395,6 +400,46 @@ __device__ __forceinline__ bool run_program(const CandShared& c, const i32* __re
     return true;
 }
 
+// Points that the whole-domain check of a survivor has to visit.  On a box whose points are
+// staged, variables that neither the candidate nor the context nor the spec mention cannot
+// change either side of the constraint, so the sub-box of the mentioned variables (the others
+// at their first value) decides for the whole box.  Returns the number of points of that
+// sub-box (the whole domain when nothing can be left out, or when the sub-box does not fit 31
+// bits) and, if `c` is given, writes its digits there.
+__device__ __forceinline__ i64 proj_points(const SketchDev* sk, const HoleDev* hole, u32 cand_vars, CandShared* c) {
+    if (c) c->n_proj_vars = 0;
+    const int nv = sk->n_vars;
+    const u32 all = nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
+    const u32 used = (cand_vars | hole->fixed_vars) & all;
+    if (!sk->project || used == all) return sk->n_points;
+    u64 n = 1, stride = 1;
+    int k = 0;
+    for (int v = nv - 1; v >= 0; --v) {                 // last variable fastest
+        const u64 ext = (u64)sk->ext[v];
+        if ((used >> v) & 1u) {
+            if (stride >> 31 || ext >> 31) return sk->n_points;
+            if (c) { c->proj_ext[k] = (u32)ext; c->proj_stride[k] = (u32)stride; }
+            ++k;
+            n *= ext;
+            if (n >> 31) return sk->n_points;
+        }
+        stride *= ext;
+    }
+    if (c) c->n_proj_vars = k;
+    return (i64)n;
+}
+
+// Point id in the full box of point q of the sub-box.
+__device__ __forceinline__ i64 proj_pid(const CandShared& c, i64 q) {
+    u32 rem = (u32)q, pid = 0;
+    for (int k = 0; k < c.n_proj_vars; ++k) {
+        const u32 e = c.proj_ext[k], d = rem / e;
+        pid += (rem - d * e) * c.proj_stride[k];
+        rem = d;
+    }
+    return (i64)pid;
+}
+
 // Stage 3 core: the whole CTA checks the staged candidate on the points [first, last),
 // kThreads points at a time; a failing point anywhere ends the scan at the next block-wide
 // vote.  Returns true if every point passed; adds the points tried by this thread to evals.
@@ -413,9 +458,9 @@ __device__ __forceinline__ bool check_points_fast(const CandShared& c, const Ske
     const int nv = sk->n_vars;
     const int lane = threadIdx.x & 31;
     for (i64 base = first; base < last; base += 32) {
-        const i64 pid = base + lane;
         bool bad = false;
-        if (pid < last) {
+        if (base + lane < last) {
+            const i64 pid = c.n_proj_vars ? proj_pid(c, base + lane) : base + lane;
             ++evals;
             i64 v;
             bad = !run_program<D>(c, sk->coords + pid * nv, v) || v != hole->spec_table[pid];
@@ -451,7 +496,8 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
         for (int i = 0; i < P; ++i) {
             const i64 pid = base + i * 32 + lane;
             in[i] = pid < last;
-            const i64 at = in[i] ? pid : first;           // lanes past the end repeat a valid point
+            i64 at = in[i] ? pid : first;                 // lanes past the end repeat a valid point
+            if (c.n_proj_vars) at = proj_pid(c, at);      // (uniform branch)
             row[i] = coords + at * nv;
             want[i] = spec[at];
         }
@@ -534,9 +580,9 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
     const int n = c.cand_len;
     const int lane = threadIdx.x & 31;
     for (i64 base = first; base < last; base += 32) {
-        const i64 pid = base + lane;
         bool bad = false;
-        if (pid < last) {
+        if (base + lane < last) {
+            const i64 pid = c.n_proj_vars ? proj_pid(c, base + lane) : base + lane;
             ++evals;
             i64 pt[kMaxVars];
             point_coords(sk, pid, pt);
@@ -565,12 +611,12 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
 
 // A candidate that passed the probes goes into the global queue for the verification kernel.
 // Returns false if the queue is full: the caller's warp then checks the candidate itself.
-__device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank) {
+__device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank, u32 vars) {
     const u32 at = atomicAdd(plan.surv_n, 1u);
     if (at >= plan.surv_cap) return false;
     SurvDev r;
     r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
-    r.state = 0; r.pad = 0;
+    r.state = 0; r.vars = vars;
     plan.surv[at] = r;
     return true;
 }
@@ -624,7 +670,10 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, 
             const int n = unrank(g, hole->start_nt, seg.size, rank, code);
             if (probe_check(g, hole, code, n, my_evals)) {
                 ++passes;
-                pending = !push_survivor(sh, plan, rank);
+                u32 vars = 0;
+                for (int k = 0; k < n; ++k)
+                    if (!(code[k] & kOpBit)) { const i32 var = g->leaves[code[k]].var; if (var >= 0) vars |= 1u << var; }
+                pending = !push_survivor(sh, plan, rank, vars);
             }
         }
         warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
@@ -692,6 +741,21 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
     u32 code[kMaxSize];
     const int n = unrank(g, nt, size, rank, code);
     return eval_cand(code, n, g->leaves, hole->probe_pt[pr], v);
+}
+
+// Variables that the subtree (nt, size, rank) mentions, from the tables where they reach (one
+// level of unranking above them); all variables otherwise, which is always a safe answer.
+__device__ __noinline__ u32 operand_vars(const GrammarDev* g, const HoleDev* hole, int nt, int size, u64 rank) {
+    const int tmax = hole->tab_max_size;
+    if (size <= tmax) return hole->tab_vars[hole->tab_off[nt][size] + rank];
+    if (tmax >= 1 && size >= 3) {
+        int op, lnt, rnt, a;
+        u64 l, r;
+        unrank_root(g, nt, size, rank, op, lnt, rnt, a, l, r);
+        if (a <= tmax && size - 1 - a <= tmax)
+            return (u32)hole->tab_vars[hole->tab_off[lnt][a] + l] | (u32)hole->tab_vars[hole->tab_off[rnt][size - 1 - a] + r];
+    }
+    return 0xffu;
 }
 
 // Values at probe `pr` of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
@@ -815,19 +879,23 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int 
         if (idx >= c) { idx -= c; continue; }
         i64 v = 0;
         bool ok = true;
+        u32 vars = 0;
         if (size == 1) {
             const LeafDev lf = g->leaves[g->leaf_begin[nt] + (i32)idx];
             v = lf.var >= 0 ? hole->probe_pt[pr][lf.var] : lf.value;
+            vars = lf.var >= 0 ? 1u << lf.var : 0u;
         } else {
             int op, lnt, rnt, a;
             u64 l, r;
             unrank_root(g, nt, size, idx, op, lnt, rnt, a, l, r);
             const u64 la = pbase + hole->tab_off[lnt][a] + l, ra = pbase + hole->tab_off[rnt][size - 1 - a] + r;
             ok = hole->tab_ok[la] && hole->tab_ok[ra] && apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
+            vars = (u32)hole->tab_vars[hole->tab_off[lnt][a] + l] | (u32)hole->tab_vars[hole->tab_off[rnt][size - 1 - a] + r];
         }
         const u64 at = pbase + hole->tab_off[nt][size] + idx;
         hole->tab_val[at] = v;
         hole->tab_ok[at] = ok ? 1 : 0;
+        if (pr == 0) hole->tab_vars[hole->tab_off[nt][size] + idx] = (unsigned char)vars;
         return;
     }
 }
@@ -878,7 +946,7 @@ __device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok
 
 // Position of a grammar operator among the seven a segment may hold: + - * / % min max.
 __device__ __forceinline__ int op_slot(int op) { return op <= XP_OP_MOD ? op : op - XP_OP_MIN + 5; }
-constexpr int kSlotMin = 5, kSlotMax = 6;
+constexpr int kSlotMin = 5;                         // (max follows at 6)
 
 // x and -x have the same sign-free form: the smaller of the two as unsigned numbers.
 __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x < y ? x : y; }
@@ -1170,7 +1238,9 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
             }
             if (!dead) {
                 ++passes;
-                pending = !push_survivor(sh, plan, rank);
+                const u32 vars = sk->project ? operand_vars(g, hole, seg.reg_nt, seg.reg_size, rr) |
+                                               operand_vars(g, hole, seg.bc_nt, seg.bc_size, br) : 0xffu;
+                pending = !push_survivor(sh, plan, rank, vars);
             }
         }
         warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
@@ -1499,7 +1569,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 // takes items on its own (lane = point, 32 points per step, warp vote): nothing in this
 // kernel synchronises a CTA, and no warp waits for another.  An item whose survivor has
 // already failed is skipped; lane 0 reads that flag once and shares the decision.
-__global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
+__global__ void __launch_bounds__(kThreads, 3) verify_kernel(const PlanDev plan) {
     __shared__ CandShared cands[kWarps];
     __shared__ uint4 stacks[kWarps][kVecDepth * 32];    // operand stacks below the top, per warp, level and lane
     CandShared& cand = cands[threadIdx.x >> 5];
@@ -1507,31 +1577,39 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const PlanDev plan) {
     const u32 pushed = *plan.surv_n;
     const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
     const u64 total = n * plan.max_chunks;
+    constexpr u64 kBatch = 8;                           // tickets a warp takes per atomic
+    u64 next = 0, batch_end = 0;
     for (;;) {
-        u64 t = 0;
+        if (next == batch_end) {
+            if (lane == 0) next = atomicAdd(plan.verify_ticket, kBatch);
+            next = __shfl_sync(0xffffffffu, next, 0);
+            batch_end = next + kBatch;
+        }
+        const u64 t = next++;
+        if (t >= total) break;
         int skip = 1;
+        i64 np = 0;
         if (lane == 0) {
-            t = atomicAdd(plan.verify_ticket, 1ull);
-            if (t < total) {
-                const SurvDev* sv = &plan.surv[t % n];
-                const SketchDev* sk = plan.sketches[sv->sketch];
-                const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
-                if ((i64)(t / n) * kVerifyChunk < sk->n_points && !failed) {
-                    skip = 0;
-                    stage_candidate(cand, sk, &sk->holes[sv->hole], sv->size, sv->rank);
-                }
+            const SurvDev* sv = &plan.surv[t % n];
+            const SketchDev* sk = plan.sketches[sv->sketch];
+            const HoleDev* hole = &sk->holes[sv->hole];
+            const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
+            np = proj_points(sk, hole, sv->vars, nullptr);
+            if ((i64)(t / n) * kVerifyChunk < np && !failed) {
+                skip = 0;
+                stage_candidate(cand, sk, hole, sv->size, sv->rank);
+                proj_points(sk, hole, sv->vars, &cand);
             }
         }
         __syncwarp();
-        t = __shfl_sync(0xffffffffu, t, 0);
         skip = __shfl_sync(0xffffffffu, skip, 0);
-        if (t >= total) break;
         if (skip) continue;
+        np = __shfl_sync(0xffffffffu, np, 0);
         SurvDev* sv = &plan.surv[t % n];
         const SketchDev* sk = plan.sketches[sv->sketch];
         const HoleDev* hole = &sk->holes[sv->hole];
         const i64 first = (i64)(t / n) * kVerifyChunk;
-        const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
+        const i64 last = first + kVerifyChunk < np ? first + kVerifyChunk : np;
         u64 evals = 0;
         bool ok;
         if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
@@ -1556,7 +1634,8 @@ __global__ void count_kernel(const PlanDev plan) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const SurvDev sv = plan.surv[i];
-    const i64 np = plan.sketches[sv.sketch]->n_points;
+    const SketchDev* sk = plan.sketches[sv.sketch];
+    const i64 np = proj_points(sk, &sk->holes[sv.hole], sv.vars, nullptr);
     const u32 chunks = (u32)((np + kVerifyChunk - 1) / kVerifyChunk);
     if ((sv.state & kSurvFailed) || sv.state != chunks) return;
     AccDev* a = &plan.acc[sv.acc];
