@@ -204,14 +204,13 @@ static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the 
 // it needs with one shared-memory load.  All per-operand arithmetic that does not depend on
 // the register operand is done once, when the tile is filled:
 //   BcRing: t_add = the value a register operand (times A) must have for +; t_pm = the
-//           sign-free form that covers + and - in one comparison (see ring_pass); and the mask
-//           and value for *:  (A*a) * b == tp (mod 2^32)  <=>  ((A*a) & mask) == tm, where
-//           b = 2^k * o (o odd), mask = 2^(32-k) - 1, tm = (tp >> k) * o^-1 & mask, provided the
-//           low k bits of tp are zero (else tm lies outside the mask and nothing matches);
+//           sign-free form that covers + and - in one comparison (see ring_pass); and for *
+//           the operand itself and the target:  (A*a) * b == tp (mod 2^32)  (the multiplication
+//           issues on the multiply-add pipe, which the comparisons do not use);
 //   BcDiv:  magnitudes for / and %, see div_pass;
 //   BcMeta: the value itself, meta = index inside the tile | ctz(|value|) << 16 | bit 31: pad holds
 //           the operand's exact value at probe 1 (second look).
-struct __align__(16) BcRing { u32 t_add, t_pm, mul_mask, mul_tm; };
+struct __align__(16) BcRing { u32 t_add, t_pm, mul_b, mul_t; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
@@ -234,6 +233,9 @@ struct CandShared {
     i64 cval[kMaxSize];
 };
 
+constexpr int kMaxFamily = 8;
+struct MemberState { u64 bc_first; i32 lo, hi; u32 n, nspecial; i32 wide, pad; };
+
 struct EvalShared {
     u64 ticket;
     i32 seg_index;
@@ -248,25 +250,24 @@ struct EvalShared {
     // tile tickets: the broadcast-side operands at probe 0 (entries invalid there are dropped) with
     // what the loops need of each, and the warps' queues of filter hits
     i32 chunk_hint[kWarps];      // broadcast slots per look at the hit queue (adapts to the hit rate)
-    // Broadcast slots of the segment at hand: [bc_lo, bc_hi); general operands fill it from bc_lo up
-    // (bc_n of them), those of magnitude <= 1 from bc_hi down (bc_nspecial).  For a family whose
-    // members' slots lie side by side (bc_keep) the per-member counts are kept in kept_*, and
-    // kept_head names the family resident in the tile (-1: none), so the next ticket of the same
-    // family does not fill again.
-    i32 bc_lo, bc_hi;
-    u32 bc_n, bc_nspecial;
+    // The members of the family at hand (a single segment is a family of one): their segments and,
+    // per member, the broadcast slots [lo, hi) it owns in the tile; general operands fill them from lo
+    // up (n of them), those of magnitude <= 1 from hi down (nspecial).  When all members' slots lie
+    // side by side (bc_keep) they stay valid from ticket to ticket: kept_head names the family
+    // resident in the tile (-1: none), and the next ticket of that family does not fill again.
+    SegDev mseg[kMaxFamily];
+    MemberState mb[kMaxFamily];
     i32 kept_head;
-    u32 kept_n[8], kept_nspecial[8];
-    i32 kept_wide[8];
+    i32 reg_wide;                // some register-side operand of the ticket does not fit int32
+    u32 wmember[kWarps];         // member the warp is working on (tags its queue entries)
     u32 wq_n[kWarps], wq_over[kWarps];
-    i32 tile_wide;               // some operand of the tile does not fit int32
     // second look (HoleDev::second): context factor, offset and spec value at probe 1 of the hole at hand
     i32 p1_on;
     u64 p1_A, p1_B, p1_spec;
     BcRing bc_ring[kBcTile];
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
-    u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21
+    u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21 | member << 24
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
@@ -707,7 +708,7 @@ __device__ __forceinline__ u32 abs_u32(i32 x) { return x < 0 ? 0u - (u32)x : (u3
 __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, u32 opi) {
     const int warp = threadIdx.x >> 5;
     const u32 at = atomicAdd(&sh.wq_n[warp], 1u);
-    if (at < (u32)kWarpQueue) sh.queue[warp][at] = reg_idx | (slot << 11) | (opi << 21);
+    if (at < (u32)kWarpQueue) sh.queue[warp][at] = reg_idx | (slot << 11) | (opi << 21) | (sh.wmember[warp] << 24);
     else sh.wq_over[warp] = 1u;
 }
 
@@ -990,7 +991,7 @@ __device__ __noinline__ void emit_pairs(EvalShared& sh, const RegOps* Rm, int s,
 // Ring operators on int32-exact operands, mod 2^32, for the broadcast slots [s0, s1).
 // MASK: bit0 +, bit1 -, bit2 *.  The comparisons were brought to the register operand's side
 // when the tile was filled (tp = low 32 bits of target - B):
-//   A*(a + b) == tp  <=>  A*a == tp - A*b  (= t_add);   A*(a * b) == tp  <=>  ((A*a) & mask) == tm;
+//   A*(a + b) == tp  <=>  A*a == tp - A*b  (= t_add);   A*(a * b) == tp  <=>  (A*a) * b == tp;
 //   A*(a - b) == tp  <=>  A*a == tp + A*b;              A*(b - a) == tp  <=>  A*a == A*b - tp.
 // When + and - are both present they share one comparison: without SWAP the two wanted values
 // are tp -+ A*b, i.e. A*a - tp == -+ A*b; with SWAP they are +-(tp - A*b).  Either way the pair
@@ -1009,7 +1010,7 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
         for (int j = 0; j < kNA; j += 2) {
             if (kPair) { h0 |= ca[j] == e.t_pm; h3 |= ca[j + 1] == e.t_pm; }
             else if (MASK & 3u) { h0 |= aA[j] == t_one; h3 |= aA[j + 1] == t_one; }
-            if (MASK & 4u) { h1 |= (aA[j] & e.mul_mask) == e.mul_tm; h2 |= (aA[j + 1] & e.mul_mask) == e.mul_tm; }
+            if (MASK & 4u) { h1 |= aA[j] * e.mul_b == e.mul_t; h2 |= aA[j + 1] * e.mul_b == e.mul_t; }
         }
     };
     auto resolve = [&](int s) {                          // the rare path: which candidates hit
@@ -1020,7 +1021,7 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
         for (int j = 0; j < kNA; ++j) {
             if (kPair) m_as |= (u32)(ca[j] == e.t_pm) << j;
             else if (MASK & 3u) m_as |= (u32)(aA[j] == t_one) << j;
-            if (MASK & 4u) m_mul |= (u32)((aA[j] & e.mul_mask) == e.mul_tm) << j;
+            if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b == e.mul_t) << j;
         }
         m_as &= alive; m_mul &= alive;
         if (m_as | m_mul) emit_ring(sh, Rm, s, m_as, m_mul, tp, opip, MASK, SWAP);
@@ -1202,12 +1203,12 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, const RegO
 // for the remaining probes the candidate is rebuilt by full unranking.  Survivors go to the
 // global queue, or are checked by the warp itself when that is full.  Called by all 32 lanes.
 __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
-                                         u64 reg_first, u64 bc_first, u64& my_evals) {
-    const SegDev& seg = sh.seg;
+                                         u64 reg_first, u64& my_evals) {
     const GrammarDev* g = sk->g;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncwarp();
     const u32 nq = sh.wq_n[warp] < (u32)kWarpQueue ? sh.wq_n[warp] : (u32)kWarpQueue;
+    if (nq == 0) return;
     // probes 0 .. n_tab-1 can be checked from the tables: the spec is defined and the context affine there
     int n_tab = 0;
     while (n_tab < hole->tab_probes && n_tab < hole->n_probe && ((hole->probe_spec_ok & hole->aff_okmask) >> n_tab & 1u)) ++n_tab;
@@ -1218,17 +1219,19 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
         u64 rank = 0;
         if (i < nq) {
             const u32 e = sh.queue[warp][i];
+            const SegDev& seg = sh.mseg[(e >> 24) & 7u];
+            const u32 opi = (e >> 21) & 7u;
             const u64 rr = reg_first + (e & 2047u);
-            const u64 br = bc_first + (sh.bc_meta[(e >> 11) & 1023u].meta & 0xffffu);
+            const u64 br = sh.mb[(e >> 24) & 7u].bc_first + (sh.bc_meta[(e >> 11) & 1023u].meta & 0xffffu);
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
-            rank = seg.op_base[e >> 21] + l * seg.right_count + r;
+            rank = seg.op_base[opi] + l * seg.right_count + r;
             bool dead = rank < seg.rank_begin || rank >= seg.rank_end;
             for (int j = 0; j < n_tab && !dead; ++j) {
                 ++my_evals;
                 i64 rv, bv, v;
                 dead = !operand_value(g, hole, j, seg.reg_nt, seg.reg_size, rr, rv) ||
                        !operand_value(g, hole, j, seg.bc_nt, seg.bc_size, br, bv) ||
-                       !apply_op(seg.op[e >> 21], seg.swap ? bv : rv, seg.swap ? rv : bv, v) ||
+                       !apply_op(seg.op[opi], seg.swap ? bv : rv, seg.swap ? rv : bv, v) ||
                        (u64)v * hole->aff_Aj[j] + hole->aff_Bj[j] != (u64)hole->probe_spec[j];
             }
             if (!dead && n_tab < hole->n_probe) {        // some probes have no tables: rebuild the candidate
@@ -1243,19 +1246,21 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
                 pending = !push_survivor(sh, plan, rank, vars);
             }
         }
-        warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
+        warp_verify_pending(sh, sk, hole, sh.seg.size, pending, rank, my_evals);
     }
     warp_tally(&sh.probe_survivors, passes);
-    if (lane == 0) { if (nq) atomicAdd(&sh.filter_survivors, (u64)nq); sh.wq_n[warp] = 0; }
+    if (lane == 0) { atomicAdd(&sh.filter_survivors, (u64)nq); sh.wq_n[warp] = 0; }
     __syncwarp();
 }
 
 template <bool SWAP>
-__device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, u64 reg_first,
-                                          u64 bc_first, int n_reg, i64* a64, const i32* a1, u32 a1ok, u32 alive, u64& my_evals) {
-    const SegDev& seg = sh.seg;
-    const int nb = (int)sh.bc_n, bc_lo = sh.bc_lo, bc_hi = sh.bc_hi;
-    const bool tile_wide = sh.tile_wide != 0;
+__device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
+                                          u64 reg_first, i64* a64, const i32* a1, u32 a1ok, u32 alive, bool drain_at_end,
+                                          u64& my_evals) {
+    const SegDev& seg = sh.mseg[m];
+    const MemberState& mbs = sh.mb[m];
+    const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
+    const bool tile_wide = (sh.reg_wide | mbs.wide) != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
     u32 opip = 0, mask = 0;
     for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * op_slot(seg.op[o])); mask |= 1u << op_slot(seg.op[o]); }
@@ -1339,10 +1344,13 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     // 32 * 5 hits, which always fit).  The chunk size is kept per warp from tile to tile and
     // grows back slowly.
     const int warp = threadIdx.x >> 5;
-    const int n_special = (int)sh.bc_nspecial;
+    const int n_special = (int)mbs.nspecial;
     int chunk = sh.chunk_hint[warp];
     bool shrunk = false;
-    u32 q_start = 0;                                    // queue length when the current chunk began
+    if ((threadIdx.x & 31) == 0) sh.wmember[warp] = (u32)m;
+    __syncwarp();
+    u32 q_start = sh.wq_n[warp];                        // queue length when the current chunk began (hits of
+                                                        // earlier members of the family may still wait there)
     for (int part = 0; part < 2; ++part) {
         const int lo = part == 0 ? bc_lo : bc_hi - n_special, hi = part == 0 ? bc_lo + nb : bc_hi;
         int s0 = lo;
@@ -1355,16 +1363,16 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
             __syncwarp();
             if (overflow) {
                 if ((threadIdx.x & 31) == 0) { sh.wq_n[warp] = q_start; sh.wq_over[warp] = 0; }
-                drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
+                drain_queue(sh, plan, sk, hole, reg_first, my_evals);
                 q_start = 0;
                 shrunk = true;
                 if (chunk > 1) { chunk = chunk / 4 > 1 ? chunk / 4 : 1; continue; }
                 for (int j = 0; j < kNA; ++j) {
                     run(s0, s0 + 1, alive & (1u << j), part == 1);
-                    drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
+                    drain_queue(sh, plan, sk, hole, reg_first, my_evals);
                 }
             } else if (qn > (u32)(kWarpQueue / 2)) {
-                drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
+                drain_queue(sh, plan, sk, hole, reg_first, my_evals);
                 q_start = 0;
             } else {
                 q_start = qn;
@@ -1373,14 +1381,15 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         }
     }
     if ((threadIdx.x & 31) == 0) sh.chunk_hint[warp] = shrunk ? chunk : (chunk * 2 < kChunkB ? chunk * 2 : kChunkB);
-    drain_queue(sh, plan, sk, hole, reg_first, bc_first, my_evals);
-    (void)n_reg;
+    if (drain_at_end) drain_queue(sh, plan, sk, hole, reg_first, my_evals);
 }
 
 // Fills the broadcast side of a tile: operand values at probe 0, with everything the loops
 // need that depends on them alone.  Returns (per thread) whether a value did not fit int32.
-__device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, u64 bc_first, int n_bc) {
-    const SegDev& seg = sh.seg;
+__device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, int m, int n_bc) {
+    const SegDev& seg = sh.mseg[m];
+    MemberState& mbs = sh.mb[m];
+    const u64 bc_first = mbs.bc_first;
     const bool swap = seg.swap != 0;
     const bool second = hole->second != 0;
     const u32 fA = (u32)hole->aff_A;
@@ -1395,7 +1404,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         if (second && !operand_value(g, hole, 1, seg.bc_nt, seg.bc_size, bc_first + i, v1)) continue;
         const bool v1_exact = second && v1 > -(1ll << 31) && v1 < (1ll << 31);
         const bool special = v >= -1 && v <= 1;
-        const u32 slot = special ? (u32)sh.bc_hi - 1u - atomicAdd(&sh.bc_nspecial, 1u) : (u32)sh.bc_lo + atomicAdd(&sh.bc_n, 1u);
+        const u32 slot = special ? (u32)mbs.hi - 1u - atomicAdd(&mbs.nspecial, 1u) : (u32)mbs.lo + atomicAdd(&mbs.n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
         const u32 b = (u32)(u64)v, ub = abs_u32((i32)v);
@@ -1404,18 +1413,13 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         BcMeta m;
         m.lo = b; m.hi = (u32)((u64)v >> 32); m.meta = (u32)i | (k << 16) | (v1_exact ? 0x80000000u : 0u); m.pad = (u32)(u64)v1;
         sh.bc_meta[slot] = m;
-        // + and -: the value A*a must have; *: mask and value of A*a's low bits
+        // + and -: the value A*a must have; *: the operand and the target
         BcRing r;
         const u32 bA = b * fA;
         r.t_add = ftp - bA;
         r.t_pm = signfree(swap ? r.t_add : bA);
-        if (ub == 0u) { r.mul_mask = 0u; r.mul_tm = ftp == 0u ? 0u : 1u; }
-        else {
-            r.mul_mask = 0xffffffffu >> k;
-            const bool feasible = k == 0u || (ftp << (32u - k)) == 0u;
-            const u32 io_signed = (i32)b < 0 ? 0u - io : io;  // b = 2^k * (+-o)
-            r.mul_tm = feasible ? ((ftp >> k) * io_signed) & r.mul_mask : 0xffffffffu;
-        }
+        r.mul_b = b;
+        r.mul_t = ftp;
         sh.bc_ring[slot] = r;
         // / and %: this operand as divisor (not swap) or as dividend (swap)
         BcDiv d;
@@ -1440,30 +1444,50 @@ __device__ __forceinline__ void load_segment(EvalShared& sh, const PlanDev& plan
     }
 }
 
+// Copies the segments of a family (head at `index`) into shared memory, one warp per member.
+__device__ __forceinline__ void load_family(EvalShared& sh, const PlanDev& plan, int index, int family) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int m = warp; m < family; m += kWarps) {
+        const u32* src = (const u32*)&plan.segs[index + m];
+        u32* dst = (u32*)&sh.mseg[m];
+        for (int w = lane; w < (int)(sizeof(SegDev) / 4); w += 32) dst[w] = src[w];
+    }
+}
+
 __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
                                             u64 local, u64& my_evals) {
     const GrammarDev* g = sk->g;
     if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
     // the register side: the same for every member of the segment's family
-    const int family = sh.seg.family > 1 ? sh.seg.family : 1;
+    int family = sh.seg.family > 1 ? sh.seg.family : 1;
+    if (family > kMaxFamily) family = kMaxFamily;        // (the host builds none larger)
     const int seg_index = sh.seg_index;
     const u64 reg_tile = local / sh.seg.bc_tiles, bc_tile0 = local % sh.seg.bc_tiles;
     const u64 reg_first = sh.seg.reg_begin + reg_tile * (u64)kRegTile;
     const u64 reg_left = sh.seg.reg_begin + sh.seg.reg_count - reg_first;
     const int n_reg = reg_left < (u64)kRegTile ? (int)reg_left : kRegTile;
+    const bool keep = sh.seg.bc_keep != 0;
+    const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
+    const int reg_nt = sh.seg.reg_nt, reg_size = sh.seg.reg_size;
+    const bool second = hole->second != 0;
+    load_family(sh, plan, seg_index, family);
+    if (threadIdx.x == 0) {
+        sh.reg_wide = 0;
+        sh.p1_on = second ? 1 : 0;
+        sh.p1_A = hole->aff_Aj[1]; sh.p1_B = hole->aff_Bj[1]; sh.p1_spec = (u64)hole->probe_spec[1];
+    }
     i64 a64[kNA];
     bool wide_reg = false;
     const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
-    u32 alive = fill_reg_operands(g, hole, 0, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+    u32 alive = fill_reg_operands(g, hole, 0, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA,
                                   mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
     // second look: the same operands at probe 1; one that is undefined there can be in no match
     i32 a1[kNA];
     u32 a1ok = 0;
-    const bool second = hole->second != 0;
     if (second) {
         i64 b64[kNA];
         bool wide1 = false;
-        alive &= fill_reg_operands(g, hole, 1, sh.seg.reg_nt, sh.seg.reg_size, reg_first + threadIdx.x * (u64)kNA,
+        alive &= fill_reg_operands(g, hole, 1, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA,
                                    mine < 0 ? 0 : (mine > kNA ? kNA : mine), b64, wide1);
         for (int j = 0; j < kNA; ++j) {
             a1[j] = (i32)b64[j];
@@ -1472,44 +1496,55 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     } else {
         for (int j = 0; j < kNA; ++j) a1[j] = 0;
     }
-    if (threadIdx.x == 0) {
-        sh.p1_on = second ? 1 : 0;
-        sh.p1_A = hole->aff_Aj[1]; sh.p1_B = hole->aff_Bj[1]; sh.p1_spec = (u64)hole->probe_spec[1];
-    }
-    const bool keep = sh.seg.bc_keep != 0;
-    const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
-    for (int m = 0; m < family; ++m) {
-        __syncthreads();
-        if (m > 0) load_segment(sh, plan, seg_index + m);
-        __syncthreads();
-        const SegDev& seg = sh.seg;
-        const u64 bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
-        const u64 bc_left = seg.bc_begin + seg.bc_count - bc_first;
-        const int n_bc = bc_left < (u64)kBcTile ? (int)bc_left : kBcTile;
-        if (threadIdx.x == 0) {
-            sh.bc_lo = keep ? seg.bc_base : 0;
-            sh.bc_hi = keep ? seg.bc_base + n_bc : kBcTile;
-            sh.bc_n = resident ? sh.kept_n[m] : 0;
-            sh.bc_nspecial = resident ? sh.kept_nspecial[m] : 0;
-            sh.tile_wide = resident ? sh.kept_wide[m] : 0;
-            if (!resident) sh.kept_head = -1;
-        }
-        __syncthreads();
+    __syncthreads();                                    // the members' segments are in place, reg_wide is clear
+    if (wide_reg) sh.reg_wide = 1;
+    // broadcast operands of member m: tile bc_tile0 of the head (a family's other members have one tile)
+    auto n_bc_of = [&](int m) {
+        const SegDev& seg = sh.mseg[m];
+        const u64 first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
+        const u64 left = seg.bc_begin + seg.bc_count - first;
+        return left < (u64)kBcTile ? (int)left : kBcTile;
+    };
+    auto start_member = [&](int m) {                    // (one thread) empty slots for member m
+        const SegDev& seg = sh.mseg[m];
+        MemberState& mbs = sh.mb[m];
+        mbs.bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
+        mbs.lo = keep ? seg.bc_base : 0;
+        mbs.hi = keep ? seg.bc_base + n_bc_of(m) : kBcTile;
+        mbs.n = 0; mbs.nspecial = 0; mbs.wide = 0;
+    };
+    if (keep) {
+        // Every member's operands fit the tile side by side.  They are filled once (by the first
+        // ticket of the family that this CTA takes); after that the warps go through the members on
+        // their own, with no CTA-wide synchronisation, and look at their hit queues when those fill
+        // up and once at the end.
         if (!resident) {
-            const bool wide_bc = fill_bc_operands(sh, g, hole, bc_first, n_bc);
-            if (wide_bc) sh.tile_wide = 1;
+            if ((int)threadIdx.x < family) start_member((int)threadIdx.x);
             __syncthreads();
-            if (threadIdx.x == 0 && keep) {
-                sh.kept_n[m] = sh.bc_n; sh.kept_nspecial[m] = sh.bc_nspecial; sh.kept_wide[m] = sh.tile_wide;
-                if (m == family - 1) sh.kept_head = seg_index;
-            }
-            __syncthreads();
+            for (int m = 0; m < family; ++m)
+                if (fill_bc_operands(sh, g, hole, m, n_bc_of(m))) sh.mb[m].wide = 1;
+            if (threadIdx.x == 0) sh.kept_head = seg_index;
         }
-        if (wide_reg) sh.tile_wide = 1;                 // the kept flag is the broadcast side's alone
         __syncthreads();
-        if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, a1, a1ok, alive, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, reg_first, bc_first, n_reg, a64, a1, a1ok, alive, my_evals);
+        for (int m = 0; m < family; ++m) {
+            const SegDev& seg = sh.mseg[m];
+            if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc_of(m) * (u64)seg.n_ops;
+            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
+            else tile_body<false>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
+        }
+        drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+        return;
+    }
+    for (int m = 0; m < family; ++m) {                  // members take turns in the tile
+        if (m > 0) __syncthreads();                     // every warp is done with the previous member's operands
+        if (threadIdx.x == 0) { start_member(m); sh.kept_head = -1; }      // (whatever was resident is overwritten)
+        __syncthreads();
+        if (fill_bc_operands(sh, g, hole, m, n_bc_of(m))) sh.mb[m].wide = 1;
+        __syncthreads();
+        const SegDev& seg = sh.mseg[m];
+        if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc_of(m) * (u64)seg.n_ops;
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, true, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, true, my_evals);
     }
 }
 
@@ -1521,7 +1556,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
     if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; }
-    if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; }
+    if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) sh.ticket = atomicAdd(plan.ticket, 1ull);

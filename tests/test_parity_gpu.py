@@ -168,6 +168,45 @@ def test_table_domain_host_and_device_tensors(xp):
     assert dev[0].match_count == res[0].match_count and dev[0].least_text == res[0].least_text
 
 
+def test_box_check_on_the_mentioned_variables_only(xp):
+    """On a box the whole-domain check leaves out variables that neither the candidate nor the
+    context nor the spec mention.  17 920 points (five chunks of the check); the sub-boxes have
+    between 1 and 17 920 points depending on the candidate."""
+    vs = [Variable("i", 0, 64), Variable("j", 0, 40), Variable("k", 0, 7)]
+    g = free_grammar(vs, [0, 1, 2, 7])
+    cases = [("i*2", ""), ("k", ""), ("(i*2)+k", ""), ("7", ""), ("i<3", "HOLE<3"), ("(j*5)+i", "(HOLE*5)+i"),
+             ("k<2", "k<HOLE"), ("(i+j)+k", ""), ("(j/7)*0", "")]
+    for spec, ctx in cases:
+        sk = Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))], name=f"subbox:{spec}")
+        for flags in PATHS:
+            check_sketch(xp, sk, flags=flags)
+    # a spec TABLE on the same kind of points may depend on any variable: nothing is left out
+    pts = np.stack(np.meshgrid(np.arange(12), np.arange(9), np.arange(50), indexing="ij"), axis=-1).reshape(-1, 3).astype(np.int32)
+    vt = [Variable("i", 0, 12), Variable("j", 0, 9), Variable("k", 0, 50)]
+    table = pts[:, 0].astype(np.int64) * 2
+    table[-1] += 1                                  # only the last point tells i*2 from the spec
+    r = check_sketch(xp, Sketch(free_grammar(vt, [0, 1, 2]), [Hole(0, 3, spec_table=table)], pts, name="table: last point differs"))
+    assert not r[0].solved
+
+
+def test_whole_domain_check_in_64_bit(xp):
+    """Coordinates of a table domain, not the declared ranges, bound the values: rows far outside
+    the ranges make products that need 64 bits; small rows let the check run in 32 bits."""
+    vs = [Variable("x", 0, 4), Variable("y", 0, 4)]
+    g = free_grammar(vs, [1, 3, 70000])
+    rnd = np.random.default_rng(5)
+    for xmax, ymax in [(200000, 100000), (300, 200), (2 ** 31 - 1, 3)]:
+        coords = np.stack([rnd.integers(0, xmax, 6000), rnd.integers(0, ymax, 6000)], axis=1).astype(np.int32)
+        coords[0] = (xmax - 1, ymax - 1)
+        spec = coords[:, 0].astype(np.int64) * coords[:, 1] + 3
+        sk = Sketch(g, [Hole(0, 5, spec_table=spec)], coords, name=f"bounds:{xmax}x{ymax}")
+        res = check_sketch(xp, sk)
+        assert res[0].solved and res[0].least_text in ("((x*y)+3)", "(3+(x*y))")
+    coords = np.stack([rnd.integers(-2 ** 31, -2 ** 31 + 5, 5000), rnd.integers(0, 3, 5000)], axis=1).astype(np.int32)
+    spec = coords[:, 0].astype(np.int64) - coords[:, 1]            # INT32_MIN itself among the coordinates
+    check_sketch(xp, Sketch(g, [Hole(0, 3, spec_table=spec)], coords, name="bounds:int32 min"))
+
+
 def test_edge_domains(xp):
     vs = [Variable("u", 0, 4)]
     g = free_grammar(vs, [0, 1])
