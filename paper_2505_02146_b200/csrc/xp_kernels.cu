@@ -205,12 +205,12 @@ static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the 
 // the register operand is done once, when the tile is filled:
 //   BcRing: t_add = the value a register operand (times A) must have for +; t_pm = the
 //           sign-free form that covers + and - in one comparison (see ring_pass); and for *
-//           the operand itself and the target:  (A*a) * b == tp (mod 2^32)  (the multiplication
-//           issues on the multiply-add pipe, which the comparisons do not use);
+//           the operand itself and the negated target:  (A*a) * b - tp == 0 (mod 2^32)  (one
+//           multiply-add, which issues on a pipe that the comparisons do not use);
 //   BcDiv:  magnitudes for / and %, see div_pass;
 //   BcMeta: the value itself, meta = index inside the tile | ctz(|value|) << 16 | bit 31: pad holds
 //           the operand's exact value at probe 1 (second look).
-struct __align__(16) BcRing { u32 t_add, t_pm, mul_b, mul_t; };
+struct __align__(16) BcRing { u32 t_add, t_pm, mul_b, mul_nt; };
 struct __align__(16) BcDiv { u32 low, ub, inv, cmax; };
 struct __align__(16) BcMeta { u32 lo, hi, meta, pad; };
 
@@ -1004,13 +1004,20 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
 #pragma unroll
     for (int j = 0; j < kNA; ++j) { aA[j] = Rm->aA[j]; ca[j] = Rm->ca[j]; }
     auto t_sub_of = [&](u32 t_add) { return SWAP ? 0u - t_add : 2u * tp - t_add; };
-    auto scan = [&](const BcRing& e, bool& h0, bool& h1, bool& h2, bool& h3) {
+    // The products' distances from the target (one multiply-add each, mul_nt = -tp) are folded
+    // into running minima: a candidate hits iff its distance is zero, so one comparison per vote
+    // group replaces one per candidate.
+    auto scan = [&](const BcRing& e, bool& h0, bool& h3, u32& m1, u32& m2) {
         const u32 t_one = (MASK & 1u) ? e.t_add : t_sub_of(e.t_add);       // used when only one of + - is present
 #pragma unroll
         for (int j = 0; j < kNA; j += 2) {
             if (kPair) { h0 |= ca[j] == e.t_pm; h3 |= ca[j + 1] == e.t_pm; }
             else if (MASK & 3u) { h0 |= aA[j] == t_one; h3 |= aA[j + 1] == t_one; }
-            if (MASK & 4u) { h1 |= aA[j] * e.mul_b == e.mul_t; h2 |= aA[j + 1] * e.mul_b == e.mul_t; }
+            if (MASK & 4u) {
+                const u32 d0 = aA[j] * e.mul_b + e.mul_nt, d1 = aA[j + 1] * e.mul_b + e.mul_nt;
+                m1 = d0 < m1 ? d0 : m1;
+                m2 = d1 < m2 ? d1 : m2;
+            }
         }
     };
     auto resolve = [&](int s) {                          // the rare path: which candidates hit
@@ -1021,7 +1028,7 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
         for (int j = 0; j < kNA; ++j) {
             if (kPair) m_as |= (u32)(ca[j] == e.t_pm) << j;
             else if (MASK & 3u) m_as |= (u32)(aA[j] == t_one) << j;
-            if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b == e.mul_t) << j;
+            if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b + e.mul_nt == 0u) << j;
         }
         m_as &= alive; m_mul &= alive;
         if (m_as | m_mul) emit_ring(sh, Rm, s, m_as, m_mul, tp, opip, MASK, SWAP);
@@ -1029,18 +1036,20 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     int s = s0;
     for (; s + 4 <= s1; s += 4) {                       // one warp vote per four broadcast operands
         const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
-        bool h0 = false, h1 = false, h2 = false, h3 = false;      // independent chains of comparisons
-        scan(e0, h0, h1, h2, h3);
-        scan(e1, h0, h1, h2, h3);
-        scan(e2, h0, h1, h2, h3);
-        scan(e3, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(s); resolve(s + 1); resolve(s + 2); resolve(s + 3); }
+        bool h0 = false, h3 = false;                    // independent chains of comparisons
+        u32 m1 = 0xffffffffu, m2 = 0xffffffffu;         // ... and of minima
+        scan(e0, h0, h3, m1, m2);
+        scan(e1, h0, h3, m1, m2);
+        scan(e2, h0, h3, m1, m2);
+        scan(e3, h0, h3, m1, m2);
+        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) { resolve(s); resolve(s + 1); resolve(s + 2); resolve(s + 3); }
     }
     for (; s < s1; ++s) {
         const BcRing e0 = sh.bc_ring[s];
-        bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(e0, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(s);
+        bool h0 = false, h3 = false;
+        u32 m1 = 0xffffffffu, m2 = 0xffffffffu;
+        scan(e0, h0, h3, m1, m2);
+        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) resolve(s);
     }
 }
 
@@ -1419,7 +1428,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         r.t_add = ftp - bA;
         r.t_pm = signfree(swap ? r.t_add : bA);
         r.mul_b = b;
-        r.mul_t = ftp;
+        r.mul_nt = 0u - ftp;
         sh.bc_ring[slot] = r;
         // / and %: this operand as divisor (not swap) or as dividend (swap)
         BcDiv d;
