@@ -23,6 +23,10 @@ if ROOT not in sys.path:
 METRIC = "candidate_point_evals_per_s"
 UNIT = "GInt-evals/s"
 WORKLOAD = "config2_thread_binding_matmul256_size7"
+# dram__bytes_read.sum + dram__bytes_write.sum of one eval_kernel launch on this workload, from the ncu capture
+# summarised in profiles/eval_kernel_config2.md (local-memory frames; the path is bound by the integer ALUs).
+# Set to None whenever eval_kernel changes, until the capture has been taken again.
+EVAL_KERNEL_DRAM_BYTES = 4.85e9
 ORACLE_SAMPLE_RANKS = 500_000_000          # ranks of size 7 the oracle is timed on (about 15-25 s of one core)
 
 
@@ -264,7 +268,8 @@ def main():
         "e2e": {"value": e2e_evals / e2e_s / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G int32-op/s", "frac": achieved / peak,
-                     "traffic": None, "kernel": "eval_kernel",
+                     "traffic": EVAL_KERNEL_DRAM_BYTES if args.workload == "config2" and not args.window else None,
+                     "kernel": "eval_kernel",
                      "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
                      "model": "32-bit operations of one operation + one comparison per candidate-point evaluation of the filter stage"},
     }

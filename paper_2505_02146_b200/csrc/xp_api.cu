@@ -297,6 +297,7 @@ struct HoleHost {
     int start_nt = 0, max_size = 0;
     bool filter_ok = false;          // the probe filter applies (probe 0 exists, context affine there)
     bool never = false;              // the spec is undefined at some point: no candidate can match
+    bool compares = false;           // the filter works on an interval of hole values (the context compares)
 };
 
 struct xp_sketch {
@@ -533,7 +534,12 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
     XP_CUDA_S(launch_prepare(s->d_s, nullptr));
     XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
-    for (int h = 0; h < d->n_holes; ++h) s->holes[h].filter_ok = hh[h].n_probe > 0 && hh[h].aff_ok != 0;
+    // the filter applies where the context at probe 0 is affine in the hole, or a comparison
+    for (int h = 0; h < d->n_holes; ++h)
+    {
+        s->holes[h].filter_ok = hh[h].n_probe > 0 && (hh[h].aff_ok != 0 || (hh[h].rng_okmask & hh[h].probe_spec_ok & 1u));
+        s->holes[h].compares = s->holes[h].filter_ok && hh[h].aff_ok == 0;
+    }
     // Subtree-value tables at probe 0 for the holes that use the filter: sizes 1, 2, ... while
     // every nonterminal has at most kTabMaxEntries trees of that size, and never the sizes that
     // only occur as whole candidates (operands have at most max_size - 2 nodes).
@@ -562,7 +568,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
             // probe 0 alone lets many through.
             u64 cands = 0;
             for (int k = 1; k <= o.max_size; ++k) cands += g->cnt[o.start_nt][k];
-            const bool possible = o.n_probe >= 2 && probes >= 2 && ((o.probe_spec_ok & o.aff_okmask) >> 1 & 1u);
+            const bool possible = o.n_probe >= 2 && probes >= 2 && ((o.probe_spec_ok & (o.aff_okmask | o.rng_okmask)) >> 1 & 1u);
             const bool frequent = o.sample_n > 0 && (u64)o.sample_pass0 * 256 >= (u64)o.sample_n;
             o.second = possible && (cands <= 100000000ull || frequent) ? 1 : 0;
         }
@@ -661,7 +667,7 @@ constexpr u64 kFamilyMaxWork = 512;          // candidates per register operand 
 
 // Tile segments of (start nonterminal, size k) restricted to ranks [lo, hi): one per
 // (left size, group of productions with the same operand nonterminals and the same rows).
-static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int hole, int acc, int k, u64 lo, u64 hi) {
+static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int hole, int acc, int k, u64 lo, u64 hi, int bc_tile) {
     const size_t first_seg = plan->segs.size();
     for (int b = g->bin_begin[nt]; b < g->bin_begin[nt + 1]; ++b) {
         const BinDev& bd = g->bins[b];
@@ -699,7 +705,8 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
                 n.bc_begin = reg_left ? 0 : l0;         n.bc_count = reg_left ? cr : l1 - l0;
                 n.right_count = cr;
                 n.reg_tiles = (u32)((n.reg_count + kRegTile - 1) / kRegTile);
-                n.bc_tiles = (u32)((n.bc_count + kBcTile - 1) / kBcTile);
+                n.bc_tile = bc_tile;
+                n.bc_tiles = (u32)((n.bc_count + bc_tile - 1) / bc_tile);
                 plan->segs.push_back(n);
                 sg = &plan->segs.back();
             }
@@ -791,7 +798,7 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
                 const bool forced = (o->flags & XP_FLAG_ALWAYS_FILTER) != 0;
                 const bool tiles = k >= 3 && ho.filter_ok && !(o->flags & XP_FLAG_NO_FILTER) &&
                                    (forced || hi - lo >= kTileMinRanks);
-                if (tiles) add_tiles(plan, s->g, ho.start_nt, (int)i, h, acc, k, lo, hi);
+                if (tiles) add_tiles(plan, s->g, ho.start_nt, (int)i, h, acc, k, lo, hi, ho.compares ? kBcTileSlow : kBcTile);
                 else add_linear(plan, (int)i, h, acc, k, lo, hi);
             }
         }

@@ -26,6 +26,7 @@ constexpr int kLinearChunk = kThreads * 4;   // ranks per linear ticket
 constexpr int kNA = 8;                // tile tickets: register-side operands per thread
 constexpr int kRegTile = kThreads * kNA;     // register-side operands per tile
 constexpr int kBcTile = 512;          // broadcast-side operands per tile
+constexpr int kBcTileSlow = 8;        // ... of a hole whose context compares (interval test in 64 bits per candidate)
 constexpr u64 kStageMaxPoints = 1ull << 26;  // largest box whose points and spec values are staged in HBM at load
 constexpr int kProgMax = 64;          // candidate substituted into its context: longest staged program
 constexpr u64 kTabBudgetBytes = 64ull << 20;   // subtree-value tables of one hole, all probes together
@@ -67,6 +68,13 @@ struct HoleDev {
     u32 aff_okmask;                               // bit j: the context is affine in the hole at probe j too,
     u64 aff_A, aff_B;                             //        ctx(h) = aff_Aj[j] * h + aff_Bj[j]
     u64 aff_Aj[kMaxProbe], aff_Bj[kMaxProbe];
+    // Contexts that compare: when the context is  X < c,  X <= c,  c < X  or  c <= X  with X = +-h + B
+    // (h the hole value, B and c hole-free), the hole values that satisfy the constraint at probe j
+    // form the interval [rng_lo[j], rng_hi[j]] (LLONG_MIN / LLONG_MAX for an open end; lo > hi: none).
+    // Such a hole (a loop bound stated through its guard predicate) is filtered on that interval
+    // where an affine context is filtered on equality.  Bit j of rng_okmask: probe j has the form.
+    u32 rng_okmask, pad3;
+    i64 rng_lo[kMaxProbe], rng_hi[kMaxProbe];
     // Values at probe 0 of every subtree of the small sizes 1..tab_max_size, by (nonterminal,
     // size, rank): tab_val[tab_off[nt][size] + rank], with tab_ok telling whether the subtree
     // is defined there (no zero divisor).  Built bottom-up once per sketch; operands of the
@@ -135,6 +143,8 @@ struct SegDev {
     i32 bc_base, bc_keep;            // slots [bc_base, bc_base + bc_count) of the CTA's broadcast tile belong to this
                                      // segment; bc_keep (first of a family): all members' broadcast operands fit the
                                      // tile side by side and do not depend on the ticket, so a CTA fills them once
+    i32 bc_tile;                     // broadcast operands per ticket (<= kBcTile; smaller where a candidate costs
+                                     // more than a comparison, so that the search still spreads over all SMs)
     i32 family;                      // tile segments that share the register-side operands sit next to each
                                      // other: the first holds the tickets and the count of them (>= 1), the
                                      // others (family == 0) are visited by its tickets, one fill for all

@@ -2,15 +2,18 @@
 //
 //   prepare_kernel  -- per sketch, once at load: coordinates and spec values of the sample
 //                      points, choice and order of each hole's probe points.
-//   subvalue_kernel, stage_points_kernel, stage_spec_kernel -- per sketch, once at load: values
-//                      of all small subtrees at the probes; points and spec values of a box.
+//   subvalue_kernel, stage_points_kernel, stage_spec_kernel, coord_bounds_kernel -- per sketch,
+//                      once at load: values (and variable sets) of all small subtrees at the probes;
+//                      points and spec values of a box; coordinate bounds of a table.
 //   eval_kernel     -- the search.  Persistent CTAs take tickets (pieces of the rank space)
 //                      from an atomic counter; no CTA ever waits for another.
-//                        stage 1 (tile segments): probe-point filter over a product of operand tiles;
+//                        stage 1 (tile segments): probe-point filter over a product of operand tiles,
+//                                 with a second, exact look at probe 1 for what the filter lets through;
 //                        stage 2: exact int64 check of a hit on the probe points (lane = candidate).
 //                      Survivors of stage 2 go to a global queue.
-//   verify_kernel   -- stage 3: check on the whole domain (lane = point, warp-wide early exit),
-//                      cut into (survivor, chunk of points) items that any warp takes.
+//   verify_kernel   -- stage 3: check on the whole domain (lane = 2 or 4 points, warp-wide early
+//                      exit), cut into (survivor, chunk of points) items that any warp takes; on a
+//                      box only the sub-box of the variables that occur is visited.
 //   count_kernel    -- survivors that passed every chunk become matches: per-size counts (sum)
 //                      and least rank (min) by atomics.
 //   finish_kernel   -- reduction of the per-size results to the least solution per hole.
@@ -64,6 +67,56 @@ __device__ bool ctx_affine(const HoleDev* hole, const i64* pt, u64& A, u64& B) {
     }
     A = sa[0]; B = sb[0];
     return true;
+}
+
+// Context of a hole at one point as a comparison of +-h + B with a hole-free value (see
+// HoleDev::rng_lo): walks the postfix code with entries that are a constant, the form a*h + b
+// with a = +-1, or (last instruction only) the predicate.  On success gives the interval of
+// hole values h for which the context's value equals `spec`.  All magnitudes are kept below
+// 2^61, so that the interval is exact for every h below 2^62 in magnitude.
+__device__ bool ctx_interval(const HoleDev* hole, const i64* pt, i64 spec, i64& lo, i64& hi) {
+    constexpr i64 kBig = 1ll << 61;
+    i64 sa[kMaxStack], sb[kMaxStack];                   // entry = sa * h + sb; sa == 0: a constant
+    int sp = 0;
+    const int n = hole->ctx_len;
+    if (n < 3) return false;
+    for (int i = 0; i < n; ++i) {
+        const xp_instr c = hole->ctx[i];
+        if (c.kind != XP_I_OP) {
+            sa[sp] = c.kind == XP_I_HOLE ? 1 : 0;
+            sb[sp] = c.kind == XP_I_VAR ? pt[c.arg] : (c.kind == XP_I_CONST ? c.value : 0);
+            ++sp;
+            continue;
+        }
+        --sp;
+        const i64 xa = sa[sp - 1], xb = sb[sp - 1], ya = sa[sp], yb = sb[sp];
+        if (xb <= -kBig || xb >= kBig || yb <= -kBig || yb >= kBig) return false;
+        if (xa == 0 && ya == 0) {
+            i64 r;
+            if (!apply_op(c.arg, xb, yb, r)) return false;
+            sb[sp - 1] = r;
+            continue;
+        }
+        if (i == n - 1 && (c.arg == XP_OP_LT || c.arg == XP_OP_LE) && (xa == 0) != (ya == 0)) {
+            // value = [ a*h + b < T ] xor neg
+            i64 a, b, T;
+            bool neg;
+            if (ya == 0) { a = xa; b = xb; T = c.arg == XP_OP_LT ? yb : yb + 1; neg = false; }      // X < c, X <= c
+            else { a = ya; b = yb; T = c.arg == XP_OP_LT ? xb + 1 : xb; neg = true; }              // c < X, c <= X
+            if (spec != 0 && spec != 1) { lo = 1; hi = 0; return true; }
+            const bool want = (spec == 1) != neg;                  // a*h + b < T must be `want`
+            if (a == 1) {                                          // h < T - b
+                if (want) { lo = LLONG_MIN; hi = T - b - 1; } else { lo = T - b; hi = LLONG_MAX; }
+            } else {                                               // -h + b < T  <=>  h > b - T
+                if (want) { lo = b - T + 1; hi = LLONG_MAX; } else { lo = LLONG_MIN; hi = b - T; }
+            }
+            return true;
+        }
+        if (c.arg == XP_OP_ADD && (xa == 0 || ya == 0)) { sa[sp - 1] = xa + ya; sb[sp - 1] = xb + yb; }
+        else if (c.arg == XP_OP_SUB && (xa == 0 || ya == 0)) { sa[sp - 1] = xa - ya; sb[sp - 1] = xb - yb; }
+        else return false;
+    }
+    return false;
 }
 
 // Choice of each hole's probe points, once per sketch (one CTA).  Threads evaluate the sample
@@ -184,6 +237,15 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
                 hole->aff_Bj[j] = Bj;
             }
             hole->aff_okmask = okmask;
+            u32 rmask = 0;
+            for (int j = 0; j < n; ++j) {
+                i64 lo = 1, hi = 0;
+                if (!((okmask >> j) & 1u) && ((hole->probe_spec_ok >> j) & 1u) &&
+                    ctx_interval(hole, hole->probe_pt[j], hole->probe_spec[j], lo, hi)) rmask |= 1u << j;
+                hole->rng_lo[j] = lo;
+                hole->rng_hi[j] = hi;
+            }
+            hole->rng_okmask = rmask;
         }
     }
 }
@@ -262,8 +324,9 @@ struct EvalShared {
     u32 wmember[kWarps];         // member the warp is working on (tags its queue entries)
     u32 wq_n[kWarps], wq_over[kWarps];
     // second look (HoleDev::second): context factor, offset and spec value at probe 1 of the hole at hand
-    i32 p1_on;
+    i32 p1_on, p1_rng;           // p1_rng: the context compares at probe 1; the value must lie in [p1_lo, p1_hi]
     u64 p1_A, p1_B, p1_spec;
+    i64 p1_lo, p1_hi;
     BcRing bc_ring[kBcTile];
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
@@ -441,12 +504,6 @@ __device__ __forceinline__ i64 proj_pid(const CandShared& c, i64 q) {
     return (i64)pid;
 }
 
-// Stage 3 core: the whole CTA checks the staged candidate on the points [first, last),
-// kThreads points at a time; a failing point anywhere ends the scan at the next block-wide
-// vote.  Returns true if every point passed; adds the points tried by this thread to evals.
-// Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
-// and the program runs on a register stack.  Otherwise coordinates are derived from the point
-// id and the interpreters with a stack in local memory are used.
 // Stage 3 core: one WARP checks the staged candidate on the points [first, last), 32 points
 // per step; a failing point anywhere ends the scan at the next warp vote.  Returns true if
 // every point passed; adds the points tried by this lane to evals.
@@ -700,7 +757,7 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, 
 //   * an affine context  A*h + B  is folded into the operands (ring operators) or applied to
 //     the quotient / remainder;
 //   * everything that depends on one operand only is computed when the tile is filled, so a
-//     candidate costs one comparison for + and -, a mask and a comparison for *, and for / and %
+//     candidate costs one comparison for + and -, a multiply-add and a minimum for *, and for / and %
 //     a range test and a divisibility test on magnitudes (see ring_pass and div_pass).
 
 __device__ __forceinline__ u32 abs_u32(i32 x) { return x < 0 ? 0u - (u32)x : (u32)x; }
@@ -936,6 +993,7 @@ __device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok
     const i64 x = swap ? (i64)(i32)b1 : (i64)a1, y = swap ? (i64)a1 : (i64)(i32)b1;
     i64 v;
     if (!apply_op(op, x, y, v)) return false;
+    if (sh.p1_rng) return v >= sh.p1_lo && v <= sh.p1_hi;
     return (u64)v * sh.p1_A + sh.p1_B == sh.p1_spec;
 }
 #define XP_P1(op, j, s) probe1_pass(sh, op, (Rm->a1ok >> (j)) & 1u, Rm->a1[j], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
@@ -1191,8 +1249,10 @@ __device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegOps* Rm, u
 }
 
 // Any operator on int64 operands (tiles with an operand outside int32): exact, slow, rare.
+// rng 1: the context compares (HoleDev::rng_lo) and the value must lie in [lo, hi] instead;
+// rng 2: every defined value passes.
 __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, const RegOps* Rm, u32 alive, bool swap, u64 A, u64 tq,
-                                        int s0, int s1, int n_ops, const i32* ops) {
+                                        int rng, i64 lo, i64 hi, int s0, int s1, int n_ops, const i32* ops) {
     const bool SWAP = swap;
     for (int s = s0; s < s1; ++s) {
         const i64 b = (i64)(((u64)sh.bc_meta[s].hi << 32) | sh.bc_meta[s].lo);
@@ -1201,7 +1261,8 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, const RegO
             for (int o = 0; o < n_ops; ++o) {
                 i64 v;
                 if (!apply_op(ops[o], swap ? b : a[j], swap ? a[j] : b, v)) continue;
-                if ((u64)v * A == tq && XP_P1(ops[o], j, s)) push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
+                if ((rng == 0 ? (u64)v * A == tq : (rng == 2 || (v >= lo && v <= hi))) && XP_P1(ops[o], j, s))
+                    push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
             }
         }
     }
@@ -1218,9 +1279,11 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
     __syncwarp();
     const u32 nq = sh.wq_n[warp] < (u32)kWarpQueue ? sh.wq_n[warp] : (u32)kWarpQueue;
     if (nq == 0) return;
-    // probes 0 .. n_tab-1 can be checked from the tables: the spec is defined and the context affine there
+    // probes 0 .. n_tab-1 can be checked from the tables: the spec is defined and the context affine
+    // (or a comparison) there
     int n_tab = 0;
-    while (n_tab < hole->tab_probes && n_tab < hole->n_probe && ((hole->probe_spec_ok & hole->aff_okmask) >> n_tab & 1u)) ++n_tab;
+    while (n_tab < hole->tab_probes && n_tab < hole->n_probe &&
+           ((hole->probe_spec_ok & (hole->aff_okmask | hole->rng_okmask)) >> n_tab & 1u)) ++n_tab;
     u32 passes = 0;
     for (u32 base = 0; base < nq; base += 32) {
         const u32 i = base + lane;
@@ -1240,8 +1303,11 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
                 i64 rv, bv, v;
                 dead = !operand_value(g, hole, j, seg.reg_nt, seg.reg_size, rr, rv) ||
                        !operand_value(g, hole, j, seg.bc_nt, seg.bc_size, br, bv) ||
-                       !apply_op(seg.op[opi], seg.swap ? bv : rv, seg.swap ? rv : bv, v) ||
-                       (u64)v * hole->aff_Aj[j] + hole->aff_Bj[j] != (u64)hole->probe_spec[j];
+                       !apply_op(seg.op[opi], seg.swap ? bv : rv, seg.swap ? rv : bv, v);
+                if (dead) break;
+                if ((hole->aff_okmask >> j) & 1u) dead = (u64)v * hole->aff_Aj[j] + hole->aff_Bj[j] != (u64)hole->probe_spec[j];
+                else if (v > -(1ll << 62) && v < (1ll << 62)) dead = v < hole->rng_lo[j] || v > hole->rng_hi[j];
+                // (a value of 2^62 or more in magnitude is left to the whole-domain check)
             }
             if (!dead && n_tab < hole->n_probe) {        // some probes have no tables: rebuild the candidate
                 u32 code[kMaxSize];
@@ -1271,6 +1337,10 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
     const bool tile_wide = (sh.reg_wide | mbs.wide) != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
+    // a context that compares: interval test on int32-exact operands (results stay below 2^62 in
+    // magnitude, where the interval is exact); wider operands are all passed on to the exact stages
+    const int rng = hole->aff_ok ? 0 : (tile_wide ? 2 : 1);
+    const i64 rng_lo = hole->rng_lo[0], rng_hi = hole->rng_hi[0];
     u32 opip = 0, mask = 0;
     for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * op_slot(seg.op[o])); mask |= 1u << op_slot(seg.op[o]); }
 
@@ -1315,8 +1385,8 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
     auto run = [&](int s0, int s1, u32 alv, bool special) {
-        if (tile_wide) {
-            wide_chunk(sh, a64, &R, alv, SWAP, A64, tq, s0, s1, seg.n_ops, seg.op);
+        if (tile_wide || rng) {
+            wide_chunk(sh, a64, &R, alv, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
             return;
         }
         switch (mask & 7u) {
@@ -1484,6 +1554,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         sh.reg_wide = 0;
         sh.p1_on = second ? 1 : 0;
         sh.p1_A = hole->aff_Aj[1]; sh.p1_B = hole->aff_Bj[1]; sh.p1_spec = (u64)hole->probe_spec[1];
+        sh.p1_rng = (hole->rng_okmask >> 1) & 1u;
+        sh.p1_lo = hole->rng_lo[1]; sh.p1_hi = hole->rng_hi[1];
     }
     i64 a64[kNA];
     bool wide_reg = false;
@@ -1510,14 +1582,14 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     // broadcast operands of member m: tile bc_tile0 of the head (a family's other members have one tile)
     auto n_bc_of = [&](int m) {
         const SegDev& seg = sh.mseg[m];
-        const u64 first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
+        const u64 first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)seg.bc_tile;
         const u64 left = seg.bc_begin + seg.bc_count - first;
-        return left < (u64)kBcTile ? (int)left : kBcTile;
+        return left < (u64)seg.bc_tile ? (int)left : seg.bc_tile;
     };
     auto start_member = [&](int m) {                    // (one thread) empty slots for member m
         const SegDev& seg = sh.mseg[m];
         MemberState& mbs = sh.mb[m];
-        mbs.bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)kBcTile;
+        mbs.bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)seg.bc_tile;
         mbs.lo = keep ? seg.bc_base : 0;
         mbs.hi = keep ? seg.bc_base + n_bc_of(m) : kBcTile;
         mbs.n = 0; mbs.nspecial = 0; mbs.wide = 0;

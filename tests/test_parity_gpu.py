@@ -42,6 +42,25 @@ def test_contexts(xp, ctx, flags):
     check_sketch(xp, _c1("(i+j)<9" if "<" in ctx or "==" in ctx else "i+j", ctx), flags=flags)
 
 
+@pytest.mark.parametrize("ctx,spec", [("HOLE<=i", "(j*2)<=i"), ("(i+3)<HOLE", "(i+3)<(j+5)"), ("(7-HOLE)<=j", "(7-(i/2))<=j"),
+                                       ("i<(HOLE-2)", "i<((i*j)-2)"), ("j<=(3-HOLE)", "j<=(3-(i%3))"), ("i<HOLE", "i+j"),
+                                       ("(HOLE+HOLE)<i", "(j+j)<i"), ("(HOLE<i)+1", "(j<i)+1")])
+def test_comparison_contexts_through_the_filter(xp, ctx, spec):
+    """Guard predicates (loop bounds): the filter works on the interval of hole values that
+    satisfies the comparison at a probe; other shapes fall back to rank-by-rank search."""
+    for flags in PATHS:
+        check_sketch(xp, _c1(spec, ctx), flags=flags)
+
+
+def test_comparison_context_with_wide_values(xp):
+    vs = [Variable("x", 2 ** 40, 2 ** 40 + 3), Variable("y", -2, 2)]
+    g = free_grammar(vs, [1, 2 ** 31, -2 ** 62], ops=["+", "-", "*"])
+    for ctx, spec in [("y<HOLE", "y<(x*y)"), ("HOLE<=(x*2)", "((x+x)+y)<=(x*2)")]:
+        sk = Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs), spec_expr=parse_expr(spec, vs))], name=f"wide cmp:{ctx}")
+        for flags in PATHS:
+            check_sketch(xp, sk, flags=flags)
+
+
 @pytest.mark.parametrize("ctx,spec", [("(HOLE*3)+(i*16)", "((i+j)*3)+(i*16)"), ("j-(HOLE*-5)", "j+(i*40)"),
                                        ("(2*HOLE)-(HOLE*3)", "0-(i%5)"), ("HOLE*0", "0"), ("(i*j)+7", "(i*j)+7")])
 def test_affine_contexts_through_the_filter(xp, ctx, spec):
