@@ -1091,23 +1091,27 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
         m_as &= alive; m_mul &= alive;
         if (m_as | m_mul) emit_ring(sh, Rm, s, m_as, m_mul, tp, opip, MASK, SWAP);
     };
-    int s = s0;
-    for (; s + 4 <= s1; s += 4) {                       // one warp vote per four broadcast operands
-        const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
+    // One warp vote per four broadcast operands (fewer at the end of the run).  The rare path has
+    // a single, rolled call site: its code is large, and every copy of it competes with the loops
+    // for the instruction cache.
+    for (int s = s0; s < s1; s += 4) {
+        const int n = s1 - s < 4 ? s1 - s : 4;
         bool h0 = false, h3 = false;                    // independent chains of comparisons
         u32 m1 = 0xffffffffu, m2 = 0xffffffffu;         // ... and of minima
-        scan(e0, h0, h3, m1, m2);
-        scan(e1, h0, h3, m1, m2);
-        scan(e2, h0, h3, m1, m2);
-        scan(e3, h0, h3, m1, m2);
-        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) { resolve(s); resolve(s + 1); resolve(s + 2); resolve(s + 3); }
-    }
-    for (; s < s1; ++s) {
-        const BcRing e0 = sh.bc_ring[s];
-        bool h0 = false, h3 = false;
-        u32 m1 = 0xffffffffu, m2 = 0xffffffffu;
-        scan(e0, h0, h3, m1, m2);
-        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) resolve(s);
+        if (n == 4) {
+            const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
+            scan(e0, h0, h3, m1, m2);
+            scan(e1, h0, h3, m1, m2);
+            scan(e2, h0, h3, m1, m2);
+            scan(e3, h0, h3, m1, m2);
+        } else {
+#pragma unroll 1
+            for (int q = 0; q < n; ++q) { const BcRing e0 = sh.bc_ring[s + q]; scan(e0, h0, h3, m1, m2); }
+        }
+        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) {
+#pragma unroll 1
+            for (int q = 0; q < n; ++q) resolve(s + q);
+        }
     }
 }
 
@@ -1153,7 +1157,10 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
             if (MASK & 2u) { h2 |= r0; h3 |= r1; }
         }
     };
-    auto resolve = [&](const BcDiv& e, u32 ek, int s) {
+    const bool need_k = !SWAP && !SPECIAL && (MASK & 2u);
+    auto resolve = [&](int s) {
+        const BcDiv e = sh.bc_div[s];
+        const u32 ek = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u;
         u32 mq = 0, mr = 0, nz = 0;
 #pragma unroll
         for (int j = 0; j < kNA; ++j) {
@@ -1168,22 +1175,21 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
         mq &= keep; mr &= keep;
         if (mq | mr) emit_pairs(sh, Rm, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     };
-    const bool need_k = !SWAP && !SPECIAL && (MASK & 2u);
-    int s = s0;
-    for (; s + 2 <= s1; s += 2) {                       // one warp vote per two broadcast operands
-        const BcDiv e0 = sh.bc_div[s], e1 = sh.bc_div[s + 1];
-        const u32 k0 = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u, k1 = need_k ? (sh.bc_meta[s + 1].meta >> 16) & 63u : 0u;
-        bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(e0, k0, h0, h1, h2, h3);
-        scan(e1, k1, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) { resolve(e0, k0, s); resolve(e1, k1, s + 1); }
-    }
-    for (; s < s1; ++s) {
+    for (int s = s0; s < s1; s += 2) {                  // one warp vote per two broadcast operands; one rare-path site
+        const int n = s1 - s < 2 ? 1 : 2;
         const BcDiv e0 = sh.bc_div[s];
         const u32 k0 = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
         scan(e0, k0, h0, h1, h2, h3);
-        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) resolve(e0, k0, s);
+        if (n == 2) {
+            const BcDiv e1 = sh.bc_div[s + 1];
+            const u32 k1 = need_k ? (sh.bc_meta[s + 1].meta >> 16) & 63u : 0u;
+            scan(e1, k1, h0, h1, h2, h3);
+        }
+        if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
+#pragma unroll 1
+            for (int q = 0; q < n; ++q) resolve(s + q);
+        }
     }
 }
 
