@@ -532,7 +532,7 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
     XP_CUDA_S(sketch_alloc(s, (void**)&s->d_s, sizeof(SketchDev)));
     XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
     if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
-    XP_CUDA_S(launch_prepare(s->d_s, nullptr));
+    XP_CUDA_S(launch_prepare(s->d_s, d->n_holes, nullptr));
     XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
     // the filter applies where the context at probe 0 is affine in the hole, or a comparison
     for (int h = 0; h < d->n_holes; ++h)

@@ -119,132 +119,141 @@ __device__ bool ctx_interval(const HoleDev* hole, const i64* pt, i64 spec, i64& 
     return false;
 }
 
-// Choice of each hole's probe points, once per sketch (one CTA).  Threads evaluate the sample
+// Choice of each hole's probe points, once per sketch (one CTA per hole).  Threads evaluate the sample
 // points; then a sample of small candidates (sizes 1, 3, 5, ranks spread evenly) is run on
 // every sample point, giving each a bit set of the samples where it satisfies the constraint.
 // The probes are picked greedily: each next probe is the sample that the fewest of the
 // sampled candidates still alive (satisfying all probes picked so far) also satisfy; ties go
 // to the larger |spec| + sum |coordinate| (large, distinct operand values make coincidences
 // rare).  Only the amount of work downstream depends on this choice, never a result.
-constexpr int kPrepThreads = 256;
+constexpr int kPrepThreads = 1024;
 constexpr int kPrepCands = 1024;
+constexpr int kPrepParts = 4;                           // a sampled candidate's sample points are split over this many threads
 __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
     __shared__ i64 s_pt[kProbeSamples][kMaxVars];
     __shared__ i64 s_spec[kProbeSamples];
     __shared__ int s_ok[kProbeSamples];
     __shared__ u64 s_score[kProbeSamples];
-    __shared__ u64 s_sig[kPrepCands];
+    __shared__ u64 s_sig[kPrepCands];                   // per sampled candidate: bit j = it satisfies sample j
+    __shared__ u32 s_mask[kProbeSamples][kPrepCands / 32];    // the same bits, per sample over the candidates
+    __shared__ u32 s_alive[kPrepCands / 32];            // candidates that satisfy every probe chosen so far
     __shared__ u32 s_count[kProbeSamples];
     __shared__ u64 s_chosen;
+    __shared__ int s_best;
     const int t = threadIdx.x;
     const int ns = s->n_samples;
     const int nv = s->n_vars;
     const GrammarDev* g = s->g;
-    i64 pt[kMaxVars];
-    u64 coord_mag = 0;
+    HoleDev* hole = &s->holes[blockIdx.x];              // one CTA per hole
     if (t < ns) {
+        i64 pt[kMaxVars];
+        u64 coord_mag = 0;
         point_coords(s, s->sample_id[t], pt);
         for (int d = 0; d < nv; ++d) {
             s_pt[t][d] = pt[d];
             coord_mag += (u64)(pt[d] < 0 ? -pt[d] : pt[d]);
         }
+        i64 v = 0;
+        bool ok = true;
+        if (hole->spec_table != nullptr) v = hole->spec_table[s->sample_id[t]];
+        else ok = eval_code(hole->spec, hole->spec_len, pt, 0, v);
+        s_spec[t] = v;
+        s_ok[t] = ok;
+        const u64 mag = (u64)(v < 0 ? -v : v);
+        s_score[t] = ok ? (mag > (1ull << 62) ? (1ull << 62) : mag) + coord_mag : 0;
     }
-    for (int h = 0; h < s->n_holes; ++h) {
-        HoleDev* hole = &s->holes[h];
-        __syncthreads();
-        if (t < ns) {
-            i64 v = 0;
-            bool ok = true;
-            if (hole->spec_table != nullptr) v = hole->spec_table[s->sample_id[t]];
-            else ok = eval_code(hole->spec, hole->spec_len, pt, 0, v);
-            s_spec[t] = v;
-            s_ok[t] = ok;
-            const u64 mag = (u64)(v < 0 ? -v : v);
-            s_score[t] = ok ? (mag > (1ull << 62) ? (1ull << 62) : mag) + coord_mag : 0;
-        }
-        __syncthreads();
-        // behaviour of sampled small candidates on the sample points
-        int sizes[3], nsz = 0;
-        for (int k = 1; k <= 5 && k <= hole->max_size; k += 2)
-            if (g->cnt[hole->start_nt][k] > 0) sizes[nsz++] = k;
-        const int ncand = nsz > 0 ? (s->prep_cands < kPrepCands ? s->prep_cands : kPrepCands) : 0;
-        for (int c = t; c < ncand; c += kPrepThreads) {
-            const int size = sizes[c % nsz];
-            const u64 cnt = g->cnt[hole->start_nt][size];
-            const u64 per = (u64)(ncand / nsz) + 1;
-            const u64 slot = (u64)(c / nsz);
+    // behaviour of sampled small candidates on the sample points
+    int sizes[3], nsz = 0;
+    for (int k = 1; k <= 5 && k <= hole->max_size; k += 2)
+        if (g->cnt[hole->start_nt][k] > 0) sizes[nsz++] = k;
+    const int ncand = nsz > 0 ? (s->prep_cands < kPrepCands ? s->prep_cands : kPrepCands) : 0;
+    for (int c = t; c < kPrepCands; c += kPrepThreads) s_sig[c] = 0;
+    if (t == 0) s_chosen = 0;
+    __syncthreads();
+    for (int item = t; item < ncand * kPrepParts; item += kPrepThreads) {
+        const int c = item / kPrepParts, part = item % kPrepParts;
+        const int size = sizes[c % nsz];
+        const u64 cnt = g->cnt[hole->start_nt][size];
+        const u64 per = (u64)(ncand / nsz) + 1;
+        const u64 slot = (u64)(c / nsz);
+        if (slot < cnt || cnt >= per) {                       // small sizes: every rank once, the rest unused
+            const u64 rank = cnt >= per ? slot * (cnt / per) : slot;
+            u32 code[kMaxSize];
+            const int n = unrank(g, hole->start_nt, size, rank, code);
             u64 sig = 0;
-            if (slot < cnt || cnt >= per) {                       // small sizes: every rank once, the rest unused
-                const u64 rank = cnt >= per ? slot * (cnt / per) : slot;
-                u32 code[kMaxSize];
-                const int n = unrank(g, hole->start_nt, size, rank, code);
-                for (int j = 0; j < ns; ++j) {
-                    i64 v;
-                    if (s_ok[j] && eval_cand(code, n, g->leaves, s_pt[j], v) && ctx_matches(hole, s_pt[j], v, s_spec[j]))
-                        sig |= 1ull << j;
-                }
+            for (int j = part; j < ns; j += kPrepParts) {
+                i64 v;
+                if (s_ok[j] && eval_cand(code, n, g->leaves, s_pt[j], v) && ctx_matches(hole, s_pt[j], v, s_spec[j]))
+                    sig |= 1ull << j;
             }
-            s_sig[c] = sig;
+            if (sig) atomicOr(&s_sig[c], sig);
         }
-        if (t == 0) s_chosen = 0;
+    }
+    __syncthreads();
+    const int nw = (ncand + 31) / 32;
+    for (int i = t; i < ns * nw; i += kPrepThreads) {         // transpose the bits: per sample, a set of candidates
+        const int j = i / nw, w = i % nw;
+        u32 word = 0;
+        for (int b = 0; b < 32 && w * 32 + b < ncand; ++b) word |= (u32)((s_sig[w * 32 + b] >> j) & 1ull) << b;
+        s_mask[j][w] = word;
+    }
+    if (t < nw) s_alive[t] = (t + 1) * 32 <= ncand ? 0xffffffffu : (1u << (ncand - t * 32)) - 1u;
+    __syncthreads();
+    int n = 0;
+    int pass0 = 0;
+    for (; n < kMaxProbe && n < ns; ++n) {
+        const u64 chosen = s_chosen;
+        if (t < ns) {
+            u32 count = 0xffffffffu;
+            if (!((chosen >> t) & 1ull)) {
+                count = 0;
+                for (int w = 0; w < nw; ++w) count += (u32)__popc(s_alive[w] & s_mask[t][w]);
+            }
+            s_count[t] = count;
+        }
         __syncthreads();
-        int n = 0;
-        for (; n < kMaxProbe && n < ns; ++n) {
-            const u64 chosen = s_chosen;
-            if (t < ns) {
-                u32 count = 0xffffffffu;
-                if (!((chosen >> t) & 1ull)) {
-                    count = 0;
-                    const u64 need = chosen | (1ull << t);
-                    for (int c = 0; c < ncand; ++c) count += (s_sig[c] & need) == need;
-                }
-                s_count[t] = count;
-            }
-            __syncthreads();
-            if (t == 0) {
-                int best = -1;
-                for (int i = 0; i < ns; ++i) {
-                    if ((chosen >> i) & 1ull) continue;
-                    if (best < 0 || s_count[i] < s_count[best] || (s_count[i] == s_count[best] && s_score[i] > s_score[best])) best = i;
-                }
-                hole->probe_id[n] = s->sample_id[best];
-                for (int d = 0; d < nv; ++d) hole->probe_pt[n][d] = s_pt[best][d];
-                hole->probe_spec[n] = s_spec[best];
-                if (n == 0) hole->probe_spec_ok = 0;
-                if (s_ok[best]) hole->probe_spec_ok |= 1u << n;
-                s_chosen = chosen | (1ull << best);
-            }
-            __syncthreads();
-        }
         if (t == 0) {
-            hole->n_probe = n;
-            if (n == 0) hole->probe_spec_ok = 0;
-            int pass0 = 0;                                  // sampled candidates that satisfy the first probe chosen
-            for (int i = 0; i < ns; ++i)
-                if (n > 0 && s->sample_id[i] == hole->probe_id[0])
-                    for (int c = 0; c < ncand; ++c) pass0 += (int)((s_sig[c] >> i) & 1ull);
-            hole->sample_pass0 = pass0;
-            hole->sample_n = ncand;
-            u64 A = 0, B = 0;
-            hole->aff_ok = (n > 0 && ctx_affine(hole, hole->probe_pt[0], A, B)) ? 1 : 0;
-            hole->aff_A = A;
-            hole->aff_B = B;
-            u32 okmask = 0;
-            for (int j = 0; j < n; ++j) {
-                u64 Aj = 0, Bj = 0;
-                if (ctx_affine(hole, hole->probe_pt[j], Aj, Bj)) okmask |= 1u << j;
-                hole->aff_Aj[j] = Aj;
-                hole->aff_Bj[j] = Bj;
+            int best = -1;
+            for (int i = 0; i < ns; ++i) {
+                if ((chosen >> i) & 1ull) continue;
+                if (best < 0 || s_count[i] < s_count[best] || (s_count[i] == s_count[best] && s_score[i] > s_score[best])) best = i;
             }
-            hole->aff_okmask = okmask;
-            u32 rmask = 0;
-            for (int j = 0; j < n; ++j) {
-                i64 lo = 1, hi = 0;
-                if (!((okmask >> j) & 1u) && ((hole->probe_spec_ok >> j) & 1u) &&
-                    ctx_interval(hole, hole->probe_pt[j], hole->probe_spec[j], lo, hi)) rmask |= 1u << j;
-                hole->rng_lo[j] = lo;
-                hole->rng_hi[j] = hi;
-            }
+            hole->probe_id[n] = s->sample_id[best];
+            for (int d = 0; d < nv; ++d) hole->probe_pt[n][d] = s_pt[best][d];
+            hole->probe_spec[n] = s_spec[best];
+            if (n == 0) { hole->probe_spec_ok = 0; pass0 = (int)s_count[best]; }
+            if (s_ok[best]) hole->probe_spec_ok |= 1u << n;
+            s_chosen = chosen | (1ull << best);
+            s_best = best;
+        }
+        __syncthreads();
+        if (t < nw) s_alive[t] &= s_mask[s_best][t];
+        __syncthreads();
+    }
+    if (t == 0) {
+        hole->n_probe = n;
+        if (n == 0) hole->probe_spec_ok = 0;
+        hole->sample_pass0 = pass0;                       // sampled candidates that satisfy the first probe chosen
+        hole->sample_n = ncand;
+    }
+    __syncthreads();
+    // the context at every probe: affine in the hole, or a comparison (one thread per probe)
+    if (t < kMaxProbe) {
+        u64 A = 0, B = 0;
+        const bool aff = t < n && ctx_affine(hole, hole->probe_pt[t], A, B);
+        i64 lo = 1, hi = 0;
+        const bool rng = t < n && !aff && ((hole->probe_spec_ok >> t) & 1u) &&
+                         ctx_interval(hole, hole->probe_pt[t], hole->probe_spec[t], lo, hi);
+        hole->aff_Aj[t] = aff ? A : 0;
+        hole->aff_Bj[t] = aff ? B : 0;
+        hole->rng_lo[t] = lo;
+        hole->rng_hi[t] = hi;
+        const u32 amask = __ballot_sync(0x0000ffffu, aff), rmask = __ballot_sync(0x0000ffffu, rng);
+        if (t == 0) {
+            hole->aff_ok = aff ? 1 : 0;
+            hole->aff_A = aff ? A : 0;
+            hole->aff_B = aff ? B : 0;
+            hole->aff_okmask = amask;
             hole->rng_okmask = rmask;
         }
     }
@@ -1820,8 +1829,8 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 // launchers
 // ------------------------------------------------------------------------------------------
 
-cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream) {
-    prepare_kernel<<<1, kPrepThreads, 0, stream>>>(s);
+cudaError_t launch_prepare(SketchDev* s, int n_holes, cudaStream_t stream) {
+    prepare_kernel<<<n_holes, kPrepThreads, 0, stream>>>(s);
     return cudaGetLastError();
 }
 

@@ -7,7 +7,7 @@
 
 namespace xp {
 
-cudaError_t launch_prepare(SketchDev* s, cudaStream_t stream);
+cudaError_t launch_prepare(SketchDev* s, int n_holes, cudaStream_t stream);
 cudaError_t launch_coord_bounds(SketchDev* s, i64 n_points, cudaStream_t stream);
 cudaError_t launch_stage_points(const SketchDev* s, i64 n_points, i32* coords, cudaStream_t stream);
 cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, i64* spec, u32* bad, cudaStream_t stream);
