@@ -307,13 +307,11 @@ struct xp_sketch {
     std::vector<HoleHost> holes;
     SketchDev* d_s = nullptr;
     HoleDev* d_holes = nullptr;
-    // Device memory of the sketch: one block sized at load for everything the load may need
-    // (copies of host tables, staged points and specs, subtree-value tables), handed out in
-    // 256-byte aligned pieces; anything beyond the estimate gets a block of its own.
+    // Device memory of the sketch: one block laid out at load for everything (sketch and hole
+    // records, copies of host tables, staged points and specs, subtree-value tables).
     char* arena = nullptr;
     size_t arena_bytes = 0, arena_used = 0;
     int arena_device = 0;
-    std::vector<void*> owned;
 };
 
 // Checks a postfix expression; returns false when malformed or too deep.
@@ -344,21 +342,8 @@ static u64 mix64(u64 x) {            // SplitMix64 finaliser: spreads sample ids
 
 extern "C" void xp_sketch_destroy(xp_sketch* s) {
     if (!s) return;
-    for (void* p : s->owned) cudaFree(p);
     pool_release(s->arena, s->arena_bytes, s->arena_device);
     delete s;
-}
-
-static cudaError_t sketch_alloc(xp_sketch* s, void** out, size_t bytes) {
-    const size_t need = (bytes + 255) & ~(size_t)255;
-    if (s->arena && s->arena_used + need <= s->arena_bytes) {
-        *out = s->arena + s->arena_used;
-        s->arena_used += need;
-        return cudaSuccess;
-    }
-    cudaError_t e = cudaMalloc(out, bytes ? bytes : 256);
-    if (e == cudaSuccess) s->owned.push_back(*out);
-    return e;
 }
 
 // Entries of the subtree-value tables of a hole with size bound max_size: sizes 1, 2, ... while
@@ -420,44 +405,76 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
 #define XP_CUDA_S(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { xp_sketch_destroy(s); \
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
 
-    {   // one device block for the whole load
-        auto al = [](size_t b) { return (b + 255) & ~(size_t)255; };
-        size_t need = al(sizeof(SketchDev)) + al(sizeof(HoleDev) * d->n_holes) + al(sizeof(u32) * d->n_holes);
-        const size_t np = (size_t)n_points, row = (size_t)(nv ? nv : 1);
-        const bool stage = n_points > 0 && (u64)n_points <= kStageMaxPoints;
-        if (np > 0 && ((d->domain_kind == XP_DOMAIN_TABLE && !d->coords_on_device) || (d->domain_kind == XP_DOMAIN_BOX && stage)))
-            need += al(sizeof(i32) * np * row);
-        for (int h = 0; h < d->n_holes; ++h) {
-            const xp_hole_desc& hd = d->holes[h];
-            if (np > 0 && ((hd.spec_kind == XP_SPEC_TABLE && !hd.spec_table_on_device) || (hd.spec_kind == XP_SPEC_EXPR && stage)))
-                need += al(sizeof(i64) * np);
-            const u64 entries = table_entries(g, hd.max_size, nullptr, nullptr);
-            u64 probes = kMaxProbe;
-            while (probes > 1 && entries * 9 * probes > kTabBudgetBytes) --probes;
-            need += al(sizeof(i64) * entries * probes) + al(entries * probes) + al(entries);
+    // One device block for the whole sketch, laid out here before anything runs: first what the
+    // host provides (sketch, holes, flags, small tables: one staged copy), then what the load's
+    // kernels produce (staged points and specs, subtree tables).  The host then looks at the
+    // device once more, at the end, to read back what the kernels decided.
+    const int nh = d->n_holes;
+    const size_t np = (size_t)n_points, row = (size_t)(nv ? nv : 1);
+    auto al = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    constexpr size_t kPackMax = 256u << 10;              // host tables up to this size travel in the staged copy
+    bool i32_ok = true;
+    for (int v = 0; v < nv; ++v) i32_ok = i32_ok && g->lo[v] >= INT32_MIN && g->hi[v] <= (i64)INT32_MAX + 1;
+    const bool stage = n_points > 0 && (u64)n_points <= kStageMaxPoints;
+    const bool stage_box = d->domain_kind == XP_DOMAIN_BOX && stage && i32_ok && nv > 0;
+    const bool copy_coords = d->domain_kind == XP_DOMAIN_TABLE && np > 0 && !d->coords_on_device;
+    const size_t coords_bytes = sizeof(i32) * np * row, spec_bytes = sizeof(i64) * np;
+    size_t off = 0;
+    const size_t off_sketch = off;  off += al(sizeof(SketchDev));
+    const size_t off_holes = off;   off += al(sizeof(HoleDev) * nh + sizeof(u32) * nh);       // holes, then one flag each
+    const size_t off_bad = off_holes + sizeof(HoleDev) * nh;
+    size_t off_coords = 0;
+    std::vector<size_t> off_spec(nh, 0), off_tabv(nh, 0), off_tabk(nh, 0), off_tabm(nh, 0);
+    if (copy_coords && coords_bytes <= kPackMax) { off_coords = off; off += al(coords_bytes); }
+    for (int h = 0; h < nh; ++h)
+        if (d->holes[h].spec_kind == XP_SPEC_TABLE && np > 0 && !d->holes[h].spec_table_on_device && spec_bytes <= kPackMax) {
+            off_spec[h] = off; off += al(spec_bytes);
         }
-        if (pool_alloc((void**)&s->arena, need, &s->arena_device) == cudaSuccess) s->arena_bytes = need;
-        else { s->arena = nullptr; (void)cudaGetLastError(); }          // fall back to piecewise allocation
+    const size_t head = off;                              // [0, head): staged on the host and copied in one piece
+    if ((copy_coords && coords_bytes > kPackMax) || stage_box) { off_coords = off; off += al(coords_bytes); }
+    std::vector<HoleDev> hh(nh);
+    for (int h = 0; h < nh; ++h) {
+        const xp_hole_desc& hd = d->holes[h];
+        HoleDev& o = hh[h];
+        memset(&o, 0, sizeof(o));
+        if (np > 0 && off_spec[h] == 0 &&
+            ((hd.spec_kind == XP_SPEC_TABLE && !hd.spec_table_on_device) || (hd.spec_kind == XP_SPEC_EXPR && stage))) {
+            off_spec[h] = off; off += al(spec_bytes);
+        }
+        const u64 entries = table_entries(g, hd.max_size, o.tab_off, &o.tab_size_cap);
+        u64 probes = kMaxProbe;
+        while (probes > 1 && entries * 9 * probes > kTabBudgetBytes) --probes;
+        o.tab_total = entries;
+        o.tab_probes_cap = entries > 0 ? (i32)probes : 0;
+        if (entries > 0) {
+            off_tabv[h] = off; off += al(sizeof(i64) * entries * probes);
+            off_tabk[h] = off; off += al(entries * probes);
+            off_tabm[h] = off; off += al(entries);
+        }
     }
+    if (pool_alloc((void**)&s->arena, off, &s->arena_device) != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete s;
+        return fail(XP_ERR_NOMEM, "device memory for the sketch (" + std::to_string(off) + " bytes)");
+    }
+    s->arena_bytes = off;
+    s->arena_used = off;
+    char* base = s->arena;
+    s->d_s = (SketchDev*)(base + off_sketch);
+    s->d_holes = (HoleDev*)(base + off_holes);
+
     SketchDev hs;
     memset(&hs, 0, sizeof(hs));
-    hs.g = g->d_g; hs.n_vars = nv; hs.n_holes = d->n_holes; hs.domain_kind = d->domain_kind; hs.n_points = n_points;
+    hs.g = g->d_g; hs.n_vars = nv; hs.n_holes = nh; hs.domain_kind = d->domain_kind; hs.n_points = n_points;
+    hs.holes = s->d_holes;
     for (int v = 0; v < nv; ++v) {
         hs.lo[v] = g->lo[v]; hs.ext[v] = g->hi[v] - g->lo[v];
         const bool table = d->domain_kind == XP_DOMAIN_TABLE;      // a table's bounds are reduced over its rows below
         hs.vmin[v] = table ? LLONG_MAX : g->lo[v];
         hs.vmax[v] = table ? LLONG_MIN : g->hi[v] - 1;
     }
-    if (d->domain_kind == XP_DOMAIN_TABLE && n_points > 0) {
-        if (d->coords_on_device) hs.coords = d->coords;
-        else {
-            void* p = nullptr;
-            const size_t bytes = sizeof(i32) * (size_t)n_points * (size_t)(nv ? nv : 1);
-            XP_CUDA_S(sketch_alloc(s, &p, bytes));
-            XP_CUDA_S(cudaMemcpy(p, d->coords, bytes, cudaMemcpyHostToDevice));
-            hs.coords = (const i32*)p;
-        }
-    }
+    if (d->domain_kind == XP_DOMAIN_TABLE && np > 0) hs.coords = d->coords_on_device ? d->coords : (const i32*)(base + off_coords);
+    if (stage_box) { hs.coords = (const i32*)(base + off_coords); hs.project = 1; }
     // Sample points the probes are chosen from: box corners first (they expose bound and
     // padding mistakes), then ids spread over the domain by a fixed hash.
     int ns = 0;
@@ -486,130 +503,91 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         }
     }
     hs.n_samples = ns;
-    {   // small searches get a cheaper probe choice: the load should not outweigh the search
-        u64 most = 0;
-        for (int h = 0; h < d->n_holes; ++h) {
-            u64 c = 0;
-            for (int k = 1; k <= d->holes[h].max_size; ++k) c += g->cnt[d->holes[h].start_nt][k];
-            most = c > most ? c : most;
-        }
-        hs.prep_cands = most <= 100000000ull ? 256 : 1024;
+    u64 most = 0;                                         // small searches get a cheaper probe choice: the load
+    for (int h = 0; h < nh; ++h) {                        // should not outweigh the search
+        u64 c = 0;
+        for (int k = 1; k <= d->holes[h].max_size; ++k) c += g->cnt[d->holes[h].start_nt][k];
+        most = c > most ? c : most;
+        hh[h].small_search = c <= 100000000ull ? 1 : 0;
     }
+    hs.prep_cands = most <= 100000000ull ? 256 : 1024;
 
-    std::vector<HoleDev> hh(d->n_holes);
-    for (int h = 0; h < d->n_holes; ++h) {
+    for (int h = 0; h < nh; ++h) {
         const xp_hole_desc& hd = d->holes[h];
         HoleDev& o = hh[h];
-        memset(&o, 0, sizeof(o));
         o.start_nt = hd.start_nt; o.max_size = hd.max_size; o.ctx_len = hd.ctx_len;
         if (hd.ctx_len) memcpy(o.ctx, hd.ctx, sizeof(xp_instr) * hd.ctx_len);
         if (hd.spec_kind == XP_SPEC_EXPR) {
             o.spec_len = hd.spec_len;
             memcpy(o.spec, hd.spec_expr, sizeof(xp_instr) * hd.spec_len);
-        } else if (n_points > 0) {
-            if (hd.spec_table_on_device) o.spec_table = (const i64*)hd.spec_table;
-            else {
-                void* p = nullptr;
-                XP_CUDA_S(sketch_alloc(s, &p, sizeof(i64) * (size_t)n_points));
-                XP_CUDA_S(cudaMemcpy(p, hd.spec_table, sizeof(i64) * (size_t)n_points, cudaMemcpyHostToDevice));
-                o.spec_table = (const i64*)p;
-            }
+            if (off_spec[h]) o.spec_table = (const i64*)(base + off_spec[h]);       // staged below, before anything reads it
+        } else if (np > 0) {
+            o.spec_table = hd.spec_table_on_device ? (const i64*)hd.spec_table : (const i64*)(base + off_spec[h]);
         }
-        {   // variables the context and the spec mention (a caller's spec table may depend on all)
-            u32 fv = hd.spec_kind == XP_SPEC_EXPR ? 0u : 0xffffffffu;
-            for (int i = 0; i < hd.ctx_len; ++i) if (hd.ctx[i].kind == XP_I_VAR) fv |= 1u << hd.ctx[i].arg;
-            if (hd.spec_kind == XP_SPEC_EXPR)
-                for (int i = 0; i < hd.spec_len; ++i) if (hd.spec_expr[i].kind == XP_I_VAR) fv |= 1u << hd.spec_expr[i].arg;
-            o.fixed_vars = fv;
+        if (o.tab_total > 0) {
+            o.tab_val = (i64*)(base + off_tabv[h]);
+            o.tab_ok = (unsigned char*)(base + off_tabk[h]);
+            o.tab_vars = (unsigned char*)(base + off_tabm[h]);
         }
+        // variables the context and the spec mention (a caller's spec table may depend on all)
+        u32 fv = hd.spec_kind == XP_SPEC_EXPR ? 0u : 0xffffffffu;
+        for (int i = 0; i < hd.ctx_len; ++i) if (hd.ctx[i].kind == XP_I_VAR) fv |= 1u << hd.ctx[i].arg;
+        if (hd.spec_kind == XP_SPEC_EXPR)
+            for (int i = 0; i < hd.spec_len; ++i) if (hd.spec_expr[i].kind == XP_I_VAR) fv |= 1u << hd.spec_expr[i].arg;
+        o.fixed_vars = fv;
         HoleHost ho;
         ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
         s->holes.push_back(ho);
     }
-    XP_CUDA_S(sketch_alloc(s, (void**)&s->d_holes, sizeof(HoleDev) * d->n_holes));
-    XP_CUDA_S(cudaMemcpy(s->d_holes, hh.data(), sizeof(HoleDev) * d->n_holes, cudaMemcpyHostToDevice));
-    hs.holes = s->d_holes;
-    XP_CUDA_S(sketch_alloc(s, (void**)&s->d_s, sizeof(SketchDev)));
-    XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
-    if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
-    XP_CUDA_S(launch_prepare(s->d_s, d->n_holes, nullptr));
-    XP_CUDA_S(cudaMemcpy(hh.data(), s->d_holes, sizeof(HoleDev) * d->n_holes, cudaMemcpyDeviceToHost));
-    // the filter applies where the context at probe 0 is affine in the hole, or a comparison
-    for (int h = 0; h < d->n_holes; ++h)
-    {
-        s->holes[h].filter_ok = hh[h].n_probe > 0 && (hh[h].aff_ok != 0 || (hh[h].rng_okmask & hh[h].probe_spec_ok & 1u));
-        s->holes[h].compares = s->holes[h].filter_ok && hh[h].aff_ok == 0;
+
+    // the staged copy, then the tables too large for it
+    std::vector<char> stg(head, 0);
+    memcpy(&stg[off_sketch], &hs, sizeof(hs));
+    memcpy(&stg[off_holes], hh.data(), sizeof(HoleDev) * nh);
+    if (copy_coords && coords_bytes <= kPackMax) memcpy(&stg[off_coords], d->coords, coords_bytes);
+    for (int h = 0; h < nh; ++h) {
+        const xp_hole_desc& hd = d->holes[h];
+        if (hd.spec_kind == XP_SPEC_TABLE && np > 0 && !hd.spec_table_on_device && spec_bytes <= kPackMax)
+            memcpy(&stg[off_spec[h]], hd.spec_table, spec_bytes);
     }
-    // Subtree-value tables at probe 0 for the holes that use the filter: sizes 1, 2, ... while
-    // every nonterminal has at most kTabMaxEntries trees of that size, and never the sizes that
-    // only occur as whole candidates (operands have at most max_size - 2 nodes).
-    for (int h = 0; h < d->n_holes; ++h) {
-        if (!s->holes[h].filter_ok) continue;
-        HoleDev& o = hh[h];
-        int tmax = 0;
-        const u64 total = table_entries(g, o.max_size, o.tab_off, &tmax);
-        if (tmax == 0 || total == 0) continue;
-        void* pv = nullptr;
-        void* pk = nullptr;
-        int probes = o.n_probe;                      // as many probes as the table budget allows
-        while (probes > 1 && total * 9 * (u64)probes > kTabBudgetBytes) --probes;
-        XP_CUDA_S(sketch_alloc(s, &pv, sizeof(i64) * total * probes));
-        XP_CUDA_S(sketch_alloc(s, &pk, total * probes));
-        void* pm = nullptr;
-        XP_CUDA_S(sketch_alloc(s, &pm, total));
-        o.tab_val = (i64*)pv;
-        o.tab_ok = (unsigned char*)pk;
-        o.tab_vars = (unsigned char*)pm;
-        o.tab_max_size = tmax;
-        o.tab_probes = probes;
-        o.tab_total = total;
-        {   // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
-            // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
-            // probe 0 alone lets many through.
-            u64 cands = 0;
-            for (int k = 1; k <= o.max_size; ++k) cands += g->cnt[o.start_nt][k];
-            const bool possible = o.n_probe >= 2 && probes >= 2 && ((o.probe_spec_ok & (o.aff_okmask | o.rng_okmask)) >> 1 & 1u);
-            const bool frequent = o.sample_n > 0 && (u64)o.sample_pass0 * 256 >= (u64)o.sample_n;
-            o.second = possible && (cands <= 100000000ull || frequent) ? 1 : 0;
-        }
-        XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &o, sizeof(HoleDev), cudaMemcpyHostToDevice));
-        for (int k = 1; k <= tmax; ++k) {
+    XP_CUDA_S(cudaMemcpyAsync(base, stg.data(), head, cudaMemcpyHostToDevice, nullptr));
+    if (copy_coords && coords_bytes > kPackMax) XP_CUDA_S(cudaMemcpyAsync(base + off_coords, d->coords, coords_bytes, cudaMemcpyHostToDevice, nullptr));
+    for (int h = 0; h < nh; ++h) {
+        const xp_hole_desc& hd = d->holes[h];
+        if (hd.spec_kind == XP_SPEC_TABLE && np > 0 && !hd.spec_table_on_device && spec_bytes > kPackMax)
+            XP_CUDA_S(cudaMemcpyAsync(base + off_spec[h], hd.spec_table, spec_bytes, cudaMemcpyHostToDevice, nullptr));
+    }
+    // The load's kernels, in stream order: points of a box and values of spec expressions (so that
+    // the whole-domain check, and the probe choice, read tables for every kind of domain); bounds of a
+    // table's coordinates; the probe choice; the subtree tables, bottom-up, for as many sizes and
+    // probes as there can be (launches beyond what the probe choice settled on return at once).
+    if (stage_box) XP_CUDA_S(launch_stage_points(s->d_s, n_points, (i32*)(base + off_coords), nullptr));
+    if (stage)
+        for (int h = 0; h < nh; ++h)
+            if (hh[h].spec_len != 0)
+                XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)(base + off_spec[h]), (u32*)(base + off_bad) + h, nullptr));
+    if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
+    XP_CUDA_S(launch_prepare(s->d_s, nh, nullptr));
+    for (int h = 0; h < nh; ++h)
+        for (int k = 1; k <= hh[h].tab_size_cap; ++k) {
             u64 at_size = 0;
             for (int nt = 0; nt < g->n_nt; ++nt) at_size += g->cnt[nt][k];
-            XP_CUDA_S(launch_subvalues(s->d_s, h, k, probes, at_size, nullptr));
+            XP_CUDA_S(launch_subvalues(s->d_s, h, k, hh[h].tab_probes_cap, at_size, nullptr));
         }
-    }
-    // Points of a box and values of spec expressions, staged once so that the whole-domain
-    // check reads them instead of recomputing them for every surviving candidate.
-    if (n_points > 0 && (u64)n_points <= kStageMaxPoints) {
-        bool i32_ok = true;
-        for (int v = 0; v < nv; ++v) i32_ok = i32_ok && g->lo[v] >= INT32_MIN && g->hi[v] <= (i64)INT32_MAX + 1;
-        if (d->domain_kind == XP_DOMAIN_BOX && i32_ok && nv > 0) {
-            void* p = nullptr;
-            XP_CUDA_S(sketch_alloc(s, &p, sizeof(i32) * (size_t)n_points * (size_t)nv));
-            XP_CUDA_S(launch_stage_points(s->d_s, n_points, (i32*)p, nullptr));
-            XP_CUDA_S(cudaStreamSynchronize(nullptr));       // the kernel reads the sketch before its coords field changes
-            hs.coords = (const i32*)p;
-            hs.project = 1;
-            XP_CUDA_S(cudaMemcpy(s->d_s, &hs, sizeof(hs), cudaMemcpyHostToDevice));
-        }
-        u32* d_bad = nullptr;
-        std::vector<u32> bad(d->n_holes, 0);
-        XP_CUDA_S(sketch_alloc(s, (void**)&d_bad, sizeof(u32) * d->n_holes));
-        XP_CUDA_S(cudaMemset(d_bad, 0, sizeof(u32) * d->n_holes));
-        for (int h = 0; h < d->n_holes; ++h) {
-            if (hh[h].spec_len == 0) continue;
-            void* p = nullptr;
-            XP_CUDA_S(sketch_alloc(s, &p, sizeof(i64) * (size_t)n_points));
-            XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)p, d_bad + h, nullptr));
-            XP_CUDA_S(cudaStreamSynchronize(nullptr));
-            hh[h].spec_table = (const i64*)p;
-            XP_CUDA_S(cudaMemcpy(&s->d_holes[h], &hh[h], sizeof(HoleDev), cudaMemcpyHostToDevice));
-        }
-        XP_CUDA_S(cudaMemcpy(bad.data(), d_bad, sizeof(u32) * d->n_holes, cudaMemcpyDeviceToHost));
-        for (int h = 0; h < d->n_holes; ++h) s->holes[h].never = bad[h] != 0;
-    }
+    // what the kernels decided, per hole
+    std::vector<char> back(sizeof(HoleDev) * nh + sizeof(u32) * nh);
+    XP_CUDA_S(cudaMemcpyAsync(back.data(), base + off_holes, back.size(), cudaMemcpyDeviceToHost, nullptr));
     XP_CUDA_S(cudaStreamSynchronize(nullptr));
+    for (int h = 0; h < nh; ++h) {
+        HoleDev o;
+        memcpy(&o, &back[sizeof(HoleDev) * h], sizeof(o));
+        u32 bad = 0;
+        memcpy(&bad, &back[sizeof(HoleDev) * nh + sizeof(u32) * h], sizeof(bad));
+        // the filter applies where the context at probe 0 is affine in the hole, or a comparison
+        s->holes[h].filter_ok = o.filter_ok != 0;
+        s->holes[h].compares = o.filter_ok != 0 && o.aff_ok == 0;
+        s->holes[h].never = bad != 0;                     // the spec is undefined at some point
+    }
 #undef XP_CUDA_S
     *out = s;
     return XP_OK;

@@ -86,6 +86,12 @@ struct HoleDev {
     // defined spec and an affine context at probe 1); sample_pass0: how many of the candidates
     // sampled at load satisfied probe 0 (a high rate makes the second look worth its cost).
     i32 second, sample_pass0, sample_n, pad1;
+    // Set by the host before the load's kernels run: the largest subtree size and the number of
+    // probes that the tables may cover (their memory is laid out for that many), and whether the
+    // search is small (then the second look is always taken).  prepare_kernel derives
+    // tab_max_size, tab_probes, second and filter_ok from them and from the probes it chose.
+    i32 tab_size_cap, tab_probes_cap, small_search;
+    i32 filter_ok;                                // the probe filter applies: probe 0 exists, its context is affine or compares
     i32 tab_max_size, tab_probes;
     u64 tab_total;
     u64 tab_off[kMaxNt][kMaxSize + 1];

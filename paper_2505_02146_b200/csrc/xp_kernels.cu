@@ -255,6 +255,20 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
             hole->aff_B = aff ? B : 0;
             hole->aff_okmask = amask;
             hole->rng_okmask = rmask;
+            // what the rest of the load and the searches go by
+            const u32 spec_ok = hole->probe_spec_ok;
+            const bool filter_ok = n > 0 && (aff || (rmask & spec_ok & 1u));
+            hole->filter_ok = filter_ok ? 1 : 0;
+            int probes = 0;
+            if (filter_ok && hole->tab_size_cap > 0 && hole->tab_total > 0) probes = n < hole->tab_probes_cap ? n : hole->tab_probes_cap;
+            hole->tab_probes = probes;
+            hole->tab_max_size = probes > 0 ? hole->tab_size_cap : 0;
+            // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
+            // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
+            // probe 0 alone lets many through.
+            const bool possible = n >= 2 && probes >= 2 && ((spec_ok & (amask | rmask)) >> 1 & 1u);
+            const bool frequent = ncand > 0 && (u64)pass0 * 256 >= (u64)ncand;
+            hole->second = possible && (hole->small_search || frequent) ? 1 : 0;
         }
     }
 }
@@ -939,6 +953,7 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int 
     const int pr = blockIdx.y;                          // one grid row per probe
     const GrammarDev* g = sk->g;
     HoleDev* hole = &sk->holes[hole_index];
+    if (pr >= hole->tab_probes || size > hole->tab_max_size) return;      // (the grid is sized for the most there can be)
     const u64 pbase = (u64)pr * hole->tab_total;
     u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
     for (int nt = 0; nt < g->n_nt; ++nt) {
