@@ -209,6 +209,17 @@ xp_status xp_grammar_unrank(const xp_grammar* g, int32_t nt, int32_t size, uint6
 xp_status xp_sketch_load(const xp_grammar* g, const xp_sketch_desc* desc, xp_sketch** out);
 void xp_sketch_destroy(xp_sketch* s);
 
+/* The same for n sketches at once (Algorithm 3 runs once per failing snippet, and a pass can leave
+ * many of them): descs[i] is loaded against grammars[i] (the same grammar may appear many times)
+ * and outs[i] receives its handle.  The sketches come out exactly as n calls of xp_sketch_load
+ * would leave them; the difference is cost: the copies and the load's kernels of the whole batch
+ * are queued together (one launch covers every sketch) and the host waits for the device once,
+ * where n single loads wait n times.  On error nothing is loaded and every outs[i] is NULL; the
+ * message names the first offending sketch.
+ * Errors: as xp_sketch_load. */
+xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, const xp_sketch_desc* descs, size_t n,
+                               xp_sketch** outs);
+
 /* Device scratch a call over these sketches needs (0 on invalid arguments). */
 size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts);
 

@@ -23,7 +23,7 @@ _STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_
            5: "XP_ERR_NOMEM", 6: "XP_ERR_CUDA", 7: "XP_ERR_TIMEOUT", 8: "XP_ERR_CANCELLED"}
 
 EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_grammar_unrank",
-           "xp_sketch_load", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
+           "xp_sketch_load", "xp_sketch_load_batch", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
            "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static"]
 
 
@@ -104,6 +104,7 @@ def load(path: Optional[str] = None):
     lib.xp_grammar_unrank.argtypes = [vp, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(xp_instr), C.c_int32,
                                       C.c_char_p, C.c_size_t]
     lib.xp_sketch_load.argtypes = [vp, C.POINTER(xp_sketch_desc), C.POINTER(vp)]
+    lib.xp_sketch_load_batch.argtypes = [C.POINTER(vp), C.POINTER(xp_sketch_desc), C.c_size_t, C.POINTER(vp)]
     lib.xp_sketch_destroy.argtypes = [vp]
     lib.xp_sketch_destroy.restype = None
     lib.xp_workspace_bytes.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_repair_opts)]
@@ -200,14 +201,11 @@ def _ptr_of(x) -> Tuple[int, int, object]:
     return int(x.data_ptr()), int(x.is_cuda), x      # torch tensor: device memory only, no torch compute
 
 
-def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int, object]] = None) -> LoadedSketch:
-    """``sk``: an ``xp_instances.Sketch``.  ``coords`` / ``spec_tables[hole]`` may override the
-    sketch's host tables with contiguous torch CUDA tensors (int32 [n, n_vars] / int64 [n]),
-    which the library then uses in place."""
-    lib = load()
-    keep = []
+def _fill_sketch_desc(desc, sk, coords, spec_tables, keep) -> int:
+    """Marshals one ``xp_instances.Sketch`` into ``desc``; everything that must outlive the call goes to ``keep``."""
     nh = len(sk.holes)
     holes = (xp_hole_desc * nh)()
+    keep.append(holes)
     for i, h in enumerate(sk.holes):
         d = holes[i]
         d.start_nt, d.max_size = h.start_nt, h.max_size
@@ -223,7 +221,6 @@ def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int,
         else:
             se = _code(h.spec_expr); keep.append(se)
             d.spec_kind, d.spec_len, d.spec_expr = 0, len(h.spec_expr), se
-    desc = xp_sketch_desc()
     co = coords if coords is not None else sk.coords
     if co is not None:
         if isinstance(co, np.ndarray):
@@ -233,9 +230,37 @@ def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int,
         desc.coords, desc.coords_on_device, k = _ptr_of(co)
         keep.append(k)
     desc.n_holes, desc.holes = nh, holes
+    return nh
+
+
+def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int, object]] = None) -> LoadedSketch:
+    """``sk``: an ``xp_instances.Sketch``.  ``coords`` / ``spec_tables[hole]`` may override the
+    sketch's host tables with contiguous torch CUDA tensors (int32 [n, n_vars] / int64 [n]),
+    which the library then uses in place."""
+    lib = load()
+    keep = []
+    desc = xp_sketch_desc()
+    nh = _fill_sketch_desc(desc, sk, coords, spec_tables, keep)
     out = C.c_void_p()
     _check(lib.xp_sketch_load(gr.handle, C.byref(desc), C.byref(out)))
     return LoadedSketch(out.value, gr, nh, [k for k in keep if not isinstance(k, C.Array)])
+
+
+def xp_sketch_load_batch(grs: Sequence[Grammar], sks: Sequence) -> List[LoadedSketch]:
+    """Loads ``sks[i]`` against ``grs[i]`` in one call (one wait for the device for the whole batch)."""
+    lib = load()
+    n = len(sks)
+    assert len(grs) == n and n > 0
+    descs = (xp_sketch_desc * n)()
+    keeps, nhs = [], []
+    for i, sk in enumerate(sks):
+        keep = []
+        nhs.append(_fill_sketch_desc(descs[i], sk, None, None, keep))
+        keeps.append(keep)
+    handles = (C.c_void_p * n)(*[g.handle for g in grs])
+    outs = (C.c_void_p * n)()
+    _check(lib.xp_sketch_load_batch(handles, descs, n, outs))
+    return [LoadedSketch(outs[i], grs[i], nhs[i], [k for k in keeps[i] if not isinstance(k, C.Array)]) for i in range(n)]
 
 
 @dataclass

@@ -363,9 +363,23 @@ static u64 table_entries(const xp_grammar* g, int max_size, u64 (*off)[kMaxSize 
     return total;
 }
 
-extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* d, xp_sketch** out) {
-    if (!gc || !d || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load: null argument");
-    *out = nullptr;
+// One sketch on its way through a load: everything between its description and the moment the
+// load's kernels have run.
+struct LoadState {
+    xp_sketch* s = nullptr;
+    std::vector<HoleDev> hh;
+    std::vector<char> back;          // holes and flags as the kernels left them
+    size_t off_holes = 0;
+    i64 table_points = 0;            // rows of a table domain (0 for a box)
+    u64 entries_at[kMaxSize + 1] = {0};      // subtree-table entries per size (all nonterminals)
+    int size_cap = 0, probes_cap = 0;        // over the holes
+};
+
+// First half of a load: checks the description, lays out and allocates the sketch's device
+// block, queues the copies of what the host provides and, for a box, the kernels that stage its
+// points and spec values.  Nothing here waits for the device.
+static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadState* L) {
+    if (!gc || !d) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load: null argument");
     xp_grammar* g = const_cast<xp_grammar*>(gc);
     if (d->n_holes < 1 || !d->holes) return fail(XP_ERR_SKETCH, "a sketch needs at least one hole");
     if (d->domain_kind != XP_DOMAIN_BOX && d->domain_kind != XP_DOMAIN_TABLE) return fail(XP_ERR_SKETCH, "bad domain_kind");
@@ -432,7 +446,8 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         }
     const size_t head = off;                              // [0, head): staged on the host and copied in one piece
     if ((copy_coords && coords_bytes > kPackMax) || stage_box) { off_coords = off; off += al(coords_bytes); }
-    std::vector<HoleDev> hh(nh);
+    std::vector<HoleDev>& hh = L->hh;
+    hh.resize(nh);
     for (int h = 0; h < nh; ++h) {
         const xp_hole_desc& hd = d->holes[h];
         HoleDev& o = hh[h];
@@ -566,31 +581,110 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* gc, const xp_sketch_desc* 
         for (int h = 0; h < nh; ++h)
             if (hh[h].spec_len != 0)
                 XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)(base + off_spec[h]), (u32*)(base + off_bad) + h, nullptr));
-    if (d->domain_kind == XP_DOMAIN_TABLE) XP_CUDA_S(launch_coord_bounds(s->d_s, n_points, nullptr));
-    XP_CUDA_S(launch_prepare(s->d_s, nh, nullptr));
-    for (int h = 0; h < nh; ++h)
-        for (int k = 1; k <= hh[h].tab_size_cap; ++k) {
-            u64 at_size = 0;
-            for (int nt = 0; nt < g->n_nt; ++nt) at_size += g->cnt[nt][k];
-            XP_CUDA_S(launch_subvalues(s->d_s, h, k, hh[h].tab_probes_cap, at_size, nullptr));
-        }
-    // what the kernels decided, per hole
-    std::vector<char> back(sizeof(HoleDev) * nh + sizeof(u32) * nh);
-    XP_CUDA_S(cudaMemcpyAsync(back.data(), base + off_holes, back.size(), cudaMemcpyDeviceToHost, nullptr));
-    XP_CUDA_S(cudaStreamSynchronize(nullptr));
+    L->s = s;
+    L->off_holes = off_holes;
+    L->table_points = d->domain_kind == XP_DOMAIN_TABLE ? n_points : 0;
     for (int h = 0; h < nh; ++h) {
-        HoleDev o;
-        memcpy(&o, &back[sizeof(HoleDev) * h], sizeof(o));
-        u32 bad = 0;
-        memcpy(&bad, &back[sizeof(HoleDev) * nh + sizeof(u32) * h], sizeof(bad));
-        // the filter applies where the context at probe 0 is affine in the hole, or a comparison
-        s->holes[h].filter_ok = o.filter_ok != 0;
-        s->holes[h].compares = o.filter_ok != 0 && o.aff_ok == 0;
-        s->holes[h].never = bad != 0;                     // the spec is undefined at some point
+        if (hh[h].tab_size_cap > L->size_cap) L->size_cap = hh[h].tab_size_cap;
+        if (hh[h].tab_probes_cap > L->probes_cap) L->probes_cap = hh[h].tab_probes_cap;
     }
+    for (int k = 1; k <= kMaxSize; ++k)
+        for (int nt = 0; nt < g->n_nt; ++nt) L->entries_at[k] += g->cnt[nt][k];
 #undef XP_CUDA_S
-    *out = s;
     return XP_OK;
+}
+
+extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, const xp_sketch_desc* descs, size_t n,
+                                          xp_sketch** outs) {
+    if (!grammars || !descs || !outs || n == 0) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load_batch: null argument");
+    for (size_t i = 0; i < n; ++i) outs[i] = nullptr;
+    std::vector<LoadState> st(n);
+    char* jobs_dev = nullptr;
+    size_t jobs_bytes = 0;
+    int jobs_device = 0;
+    auto undo = [&]() {
+        cudaStreamSynchronize(nullptr);                   // nothing may still be writing into the blocks
+        for (size_t i = 0; i < n; ++i) if (st[i].s) xp_sketch_destroy(st[i].s);
+        pool_release(jobs_dev, jobs_bytes, jobs_device);
+    };
+    size_t n_jobs = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const xp_status r = load_begin(grammars[i], &descs[i], &st[i]);
+        if (r != XP_OK) { const std::string msg = g_last_error; undo(); return fail(r, "sketch " + std::to_string(i) + ": " + msg); }
+        n_jobs += (size_t)st[i].s->n_holes;
+    }
+#define XP_CUDA_B(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { undo(); \
+        return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
+    // the batch's kernels: one list of sketches, one list of (sketch, hole) jobs
+    const size_t list_bytes = (sizeof(SketchDev*) * n + 255) & ~(size_t)255;
+    std::vector<char> stage(list_bytes + sizeof(LoadJob) * n_jobs, 0);
+    {
+        size_t j = 0;
+        for (size_t i = 0; i < n; ++i) {
+            ((SketchDev**)stage.data())[i] = st[i].s->d_s;
+            for (int h = 0; h < st[i].s->n_holes; ++h, ++j) {
+                LoadJob job;
+                job.s = st[i].s->d_s; job.hole = h; job.pad = 0;
+                memcpy(&stage[list_bytes + sizeof(LoadJob) * j], &job, sizeof(job));
+            }
+        }
+    }
+    jobs_bytes = stage.size();
+    XP_CUDA_B(pool_alloc((void**)&jobs_dev, jobs_bytes, &jobs_device));
+    XP_CUDA_B(cudaMemcpyAsync(jobs_dev, stage.data(), jobs_bytes, cudaMemcpyHostToDevice, nullptr));
+    SketchDev* const* d_list = (SketchDev* const*)jobs_dev;
+    const LoadJob* d_jobs = (const LoadJob*)(jobs_dev + list_bytes);
+    // In stream order after the copies and the boxes' staging: bounds of the tables' coordinates;
+    // the probe choice; the subtree tables, bottom-up, for as many sizes and probes as there can be
+    // (blocks beyond what the probe choice settled on for their hole return at once).  Grids are
+    // cut into pieces of at most kPiece jobs (a grid dimension holds 65 535).
+    constexpr size_t kPiece = 32768;
+    i64 most_points = 0;
+    int size_cap = 0, probes_cap = 0;
+    u64 most_entries[kMaxSize + 1] = {0};
+    for (size_t i = 0; i < n; ++i) {
+        most_points = st[i].table_points > most_points ? st[i].table_points : most_points;
+        size_cap = st[i].size_cap > size_cap ? st[i].size_cap : size_cap;
+        probes_cap = st[i].probes_cap > probes_cap ? st[i].probes_cap : probes_cap;
+        for (int k = 1; k <= st[i].size_cap; ++k) most_entries[k] = st[i].entries_at[k] > most_entries[k] ? st[i].entries_at[k] : most_entries[k];
+    }
+    for (size_t at = 0; at < n; at += kPiece)
+        XP_CUDA_B(launch_coord_bounds(d_list + at, (int)(n - at < kPiece ? n - at : kPiece), most_points, nullptr));
+    for (size_t at = 0; at < n_jobs; at += kPiece)
+        XP_CUDA_B(launch_prepare(d_jobs + at, (int)(n_jobs - at < kPiece ? n_jobs - at : kPiece), nullptr));
+    for (int k = 1; k <= size_cap; ++k)
+        for (size_t at = 0; at < n_jobs; at += kPiece)
+            XP_CUDA_B(launch_subvalues(d_jobs + at, (int)(n_jobs - at < kPiece ? n_jobs - at : kPiece), k, probes_cap, most_entries[k], nullptr));
+    // what the kernels decided, per hole
+    for (size_t i = 0; i < n; ++i) {
+        const int nh = st[i].s->n_holes;
+        st[i].back.resize(sizeof(HoleDev) * nh + sizeof(u32) * nh);
+        XP_CUDA_B(cudaMemcpyAsync(st[i].back.data(), st[i].s->arena + st[i].off_holes, st[i].back.size(), cudaMemcpyDeviceToHost, nullptr));
+    }
+    XP_CUDA_B(cudaStreamSynchronize(nullptr));
+#undef XP_CUDA_B
+    pool_release(jobs_dev, jobs_bytes, jobs_device);
+    for (size_t i = 0; i < n; ++i) {
+        xp_sketch* s = st[i].s;
+        const int nh = s->n_holes;
+        for (int h = 0; h < nh; ++h) {
+            HoleDev o;
+            memcpy(&o, &st[i].back[sizeof(HoleDev) * h], sizeof(o));
+            u32 bad = 0;
+            memcpy(&bad, &st[i].back[sizeof(HoleDev) * nh + sizeof(u32) * h], sizeof(bad));
+            // the filter applies where the context at probe 0 is affine in the hole, or a comparison
+            s->holes[h].filter_ok = o.filter_ok != 0;
+            s->holes[h].compares = o.filter_ok != 0 && o.aff_ok == 0;
+            s->holes[h].never = bad != 0;                 // the spec is undefined at some point
+        }
+        outs[i] = s;
+    }
+    return XP_OK;
+}
+
+extern "C" xp_status xp_sketch_load(const xp_grammar* g, const xp_sketch_desc* d, xp_sketch** out) {
+    if (!g || !d || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load: null argument");
+    return xp_sketch_load_batch(&g, d, 1, out);
 }
 
 // ------------------------------------------------------------------------------------------

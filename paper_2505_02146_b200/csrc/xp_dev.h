@@ -118,6 +118,9 @@ struct SketchDev {
     i64 sample_id[kProbeSamples];                 // point ids the probes are chosen from (host-chosen)
 };
 
+// One hole of one sketch, for the kernels that run at load over a whole batch of sketches.
+struct LoadJob { SketchDev* s; i32 hole, pad; };
+
 // Per (sketch, hole) accumulators, zeroed (min_rank to all-ones) by the host before the launch.
 struct AccDev {
     u64 match_count[kMaxSize + 1];

@@ -129,7 +129,8 @@ __device__ bool ctx_interval(const HoleDev* hole, const i64* pt, i64 spec, i64& 
 constexpr int kPrepThreads = 1024;
 constexpr int kPrepCands = 1024;
 constexpr int kPrepParts = 4;                           // a sampled candidate's sample points are split over this many threads
-__global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
+__global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jobs) {
+    SketchDev* s = jobs[blockIdx.x].s;
     __shared__ i64 s_pt[kProbeSamples][kMaxVars];
     __shared__ i64 s_spec[kProbeSamples];
     __shared__ int s_ok[kProbeSamples];
@@ -144,7 +145,7 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(SketchDev* s) {
     const int ns = s->n_samples;
     const int nv = s->n_vars;
     const GrammarDev* g = s->g;
-    HoleDev* hole = &s->holes[blockIdx.x];              // one CTA per hole
+    HoleDev* hole = &s->holes[jobs[blockIdx.x].hole];    // one CTA per hole
     if (t < ns) {
         i64 pt[kMaxVars];
         u64 coord_mag = 0;
@@ -917,7 +918,9 @@ __global__ void __launch_bounds__(256) stage_points_kernel(const SketchDev* sk, 
 // Smallest and largest coordinate of every variable over the rows of a table domain, into the
 // sketch (whose vmin / vmax start at the extreme values).  Warp shuffles, then one atomic pair
 // per warp and variable.
-__global__ void __launch_bounds__(256) coord_bounds_kernel(SketchDev* sk) {
+__global__ void __launch_bounds__(256) coord_bounds_kernel(SketchDev* const* list) {
+    SketchDev* sk = list[blockIdx.y];                   // one grid row per sketch of the batch
+    if (sk->domain_kind != XP_DOMAIN_TABLE) return;
     const int nv = sk->n_vars;
     const i64 n = sk->n_points;
     for (int v = 0; v < nv; ++v) {
@@ -949,7 +952,9 @@ __global__ void __launch_bounds__(256) stage_spec_kernel(const SketchDev* sk, in
 
 // Bottom-up construction of one size of a hole's subtree-value tables: thread = (nonterminal,
 // rank); the operands' values come from the smaller sizes built by earlier launches.
-__global__ void __launch_bounds__(256) subvalue_kernel(const SketchDev* sk, int hole_index, int size) {
+__global__ void __launch_bounds__(256) subvalue_kernel(const LoadJob* jobs, int size) {
+    const SketchDev* sk = jobs[blockIdx.z].s;           // one grid layer per hole of the batch
+    const int hole_index = jobs[blockIdx.z].hole;
     const int pr = blockIdx.y;                          // one grid row per probe
     const GrammarDev* g = sk->g;
     HoleDev* hole = &sk->holes[hole_index];
@@ -1844,15 +1849,16 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
 // launchers
 // ------------------------------------------------------------------------------------------
 
-cudaError_t launch_prepare(SketchDev* s, int n_holes, cudaStream_t stream) {
-    prepare_kernel<<<n_holes, kPrepThreads, 0, stream>>>(s);
+cudaError_t launch_prepare(const LoadJob* jobs, int n_jobs, cudaStream_t stream) {
+    if (n_jobs <= 0) return cudaSuccess;
+    prepare_kernel<<<n_jobs, kPrepThreads, 0, stream>>>(jobs);
     return cudaGetLastError();
 }
 
-cudaError_t launch_coord_bounds(SketchDev* s, i64 n_points, cudaStream_t stream) {
-    if (n_points <= 0) return cudaSuccess;
-    const i64 blocks = (n_points + 255) / 256;
-    coord_bounds_kernel<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, stream>>>(s);
+cudaError_t launch_coord_bounds(SketchDev* const* list, int n_sketches, i64 most_points, cudaStream_t stream) {
+    if (most_points <= 0 || n_sketches <= 0) return cudaSuccess;
+    const i64 blocks = (most_points + 255) / 256;
+    coord_bounds_kernel<<<dim3((unsigned)(blocks < 64 ? blocks : 64), (unsigned)n_sketches), 256, 0, stream>>>(list);
     return cudaGetLastError();
 }
 
@@ -1866,9 +1872,9 @@ cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_subvalues(const SketchDev* s, int hole_index, int size, int n_probes, u64 n_entries, cudaStream_t stream) {
-    if (n_entries == 0) return cudaSuccess;
-    subvalue_kernel<<<dim3((unsigned)((n_entries + 255) / 256), (unsigned)n_probes), 256, 0, stream>>>(s, hole_index, size);
+cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most_probes, u64 most_entries, cudaStream_t stream) {
+    if (most_entries == 0 || most_probes <= 0 || n_jobs <= 0) return cudaSuccess;
+    subvalue_kernel<<<dim3((unsigned)((most_entries + 255) / 256), (unsigned)most_probes, (unsigned)n_jobs), 256, 0, stream>>>(jobs, size);
     return cudaGetLastError();
 }
 

@@ -51,12 +51,12 @@ def test_config5_full_batch(xp):
             if not line.startswith("#")]
     assert len(rows) == 4096
     sks = config5(0, 4096)
-    grs, loaded = {}, []
+    grs = {}
     for sk in sks:
         key = tuple(v.hi for v in sk.grammar.variables)
         if key not in grs:
             grs[key] = xp.xp_grammar_create(sk.grammar)
-        loaded.append(xp.xp_sketch_load(grs[key], sk))
+    loaded = xp.xp_sketch_load_batch([grs[tuple(v.hi for v in sk.grammar.variables)] for sk in sks], sks)
     res = xp.xp_repair_batch(loaded)
     unsolved = 0
     for i, (r, row) in enumerate(zip(res, rows)):

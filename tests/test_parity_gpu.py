@@ -269,6 +269,32 @@ def test_config5_batch_slice(xp):
     assert single[0].match_count == res[3][0].match_count and single[0].least_rank == res[3][0].least_rank
 
 
+def test_batch_load_equals_single_loads(xp):
+    """xp_sketch_load_batch leaves every sketch as xp_sketch_load would: table and box domains,
+    several holes, different grammars in one batch; a bad description fails the whole batch."""
+    sks = config5(1, 12) + [config1(2), _c1("i<3", "HOLE<3"), _c1("(i*8)+j")]
+    vs = [Variable("i", 0, 64), Variable("j", 0, 40), Variable("k", 0, 7)]
+    g3 = free_grammar(vs, [0, 1, 2, 7])
+    sks.append(Sketch(g3, [Hole(0, 5, spec_expr=parse_expr("(i*2)+k", vs)), Hole(0, 3, ctx=parse_expr("k<HOLE", vs), spec_expr=parse_expr("k<2", vs)),
+                           Hole(0, 3, spec_expr=parse_expr("j/0", vs))], name="three holes"))
+    grs = [xp.xp_grammar_create(sk.grammar) for sk in sks]
+    batch = xp.xp_sketch_load_batch(grs, sks)
+    together = xp.xp_repair_batch(batch)
+    for sk, gr, ls, res in zip(sks, grs, batch, together):
+        alone = xp.xp_repair(xp.xp_sketch_load(gr, sk))
+        one_by_one = xp.xp_repair(ls)
+        for h in range(len(sk.holes)):
+            want = oracle.repair_hole(sk, h)
+            assert_same(res[h], want, f"{sk.name} hole {h} (batch load, batch search)")
+            assert_same(one_by_one[h], want, f"{sk.name} hole {h} (batch load)")
+            assert_same(alone[h], want, f"{sk.name} hole {h} (single load)")
+            assert (res[h].filter_survivors, res[h].probe_survivors) == (alone[h].filter_survivors, alone[h].probe_survivors)
+    bad = Sketch(g3, [Hole(7, 5, spec_expr=parse_expr("i", vs))], name="bad start symbol")
+    with pytest.raises(xp.XpError, match="sketch 1"):
+        xp.xp_sketch_load_batch([grs[0], xp.xp_grammar_create(g3)], [sks[0], bad])
+    assert xp.xp_repair(xp.xp_sketch_load(grs[0], sks[0]))[0].match_count == together[0][0].match_count      # still usable
+
+
 def test_config2_rank_slices(xp):
     sk = config2(0)
     n7 = 213813760000
