@@ -44,12 +44,15 @@ static xp_status fail(xp_status st, const std::string& msg) {
 // Blocks up to kPoolBigBytes are carved from 64 MiB slabs and, when released, kept in a
 // free list by size for the next load (a loop that loads and destroys the same sketch never
 // reaches cudaMalloc or cudaFree, whose cost and device-wide synchronisation would otherwise
-// dominate small searches).  Larger blocks go to cudaMalloc / cudaFree directly.  Slabs are
-// returned to the driver when the process ends.  One pool per device.
+// dominate small searches).  Larger blocks come from cudaMalloc; released ones are kept too,
+// up to kPoolBigKeep bytes in all, and handed out again to a request of the same size.  Slabs
+// and kept blocks are returned to the driver when the process ends.  One pool per device.
 namespace {
-constexpr size_t kPoolSlabBytes = 64ull << 20, kPoolBigBytes = 16ull << 20;
+constexpr size_t kPoolSlabBytes = 64ull << 20, kPoolBigBytes = 16ull << 20, kPoolBigKeep = 1ull << 30;
 struct DevPool {
     std::multimap<size_t, char*> free_blocks;
+    std::multimap<size_t, char*> big_blocks;
+    size_t big_kept = 0;
     char* slab = nullptr;
     size_t slab_left = 0;
 };
@@ -62,9 +65,16 @@ cudaError_t pool_alloc(void** out, size_t bytes, int* device_out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     *device_out = dev;
-    if (need > kPoolBigBytes) return cudaMalloc(out, need);
     std::lock_guard<std::mutex> lock(g_pool_mu);
     DevPool& p = g_pools[dev];
+    if (need > kPoolBigBytes) {
+        auto big = p.big_blocks.find(need);
+        if (big == p.big_blocks.end()) return cudaMalloc(out, need);
+        *out = big->second;
+        p.big_blocks.erase(big);
+        p.big_kept -= need;
+        return cudaSuccess;
+    }
     auto it = p.free_blocks.find(need);
     if (it != p.free_blocks.end()) { *out = it->second; p.free_blocks.erase(it); return cudaSuccess; }
     if (p.slab_left < need) {
@@ -83,9 +93,15 @@ cudaError_t pool_alloc(void** out, size_t bytes, int* device_out) {
 void pool_release(void* ptr, size_t bytes, int device) {
     if (!ptr) return;
     const size_t need = ((bytes ? bytes : 1) + 255) & ~(size_t)255;
-    if (need > kPoolBigBytes) { cudaFree(ptr); return; }
     std::lock_guard<std::mutex> lock(g_pool_mu);
-    g_pools[device].free_blocks.insert({need, (char*)ptr});
+    DevPool& p = g_pools[device];
+    if (need > kPoolBigBytes) {
+        if (p.big_kept + need > kPoolBigKeep) { cudaFree(ptr); return; }
+        p.big_blocks.insert({need, (char*)ptr});
+        p.big_kept += need;
+        return;
+    }
+    p.free_blocks.insert({need, (char*)ptr});
 }
 }  // namespace
 
