@@ -1144,6 +1144,25 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     }
 }
 
+// The divisors 0 and +-1 among the broadcast operands (register operand / broadcast operand) sit
+// in a run of their own: 0 is skipped (invalid), +-1 gives |quotient| = |dividend| and remainder
+// 0.  There are at most a few such slots per tile, so this is a small rolled routine rather than
+// another instance of the loop below.
+__device__ __noinline__ void div_special(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tabs, int s0, int s1, u32 opip, u32 mask) {
+    constexpr bool SWAP = false;
+    for (int s = s0; s < s1; ++s) {
+        if (sh.bc_div[s].ub != 1u) continue;
+        u32 mq = 0, mr = 0;
+        for (int j = 0; j < kNA; ++j) {
+            if ((mask & 1u) && Rm->ua[j] == tabs) mq |= 1u << j;
+            if ((mask & 2u) && tabs == 0u) mr |= 1u << j;
+        }
+        mq &= alive; mr &= alive;
+        const bool any = (mq | mr) != 0;
+        if (__any_sync(0xffffffffu, any) && any) emit_pairs(sh, Rm, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
+    }
+}
+
 // / and % on int32-exact operands with the context factor A == 1.  MASK: bit0 /, bit1 %.
 // Only magnitudes are compared (|quotient| or |remainder| against tabs = |target|): still a
 // necessary condition, the signs are settled by the exact check.  With n the dividend's and d
@@ -1441,7 +1460,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         if (A != 1u) { div_pass_signed<SWAP>(sh, &R, alv, mask, A, tp, s0, s1, opip); return; }
         if (!t_small) return;                            // no int32 quotient or remainder can be the target
         switch ((mask >> 3) & 3u) {
-#define XP_DIV(M) case M: if (special && !SWAP) div_pass<M, SWAP, true>(sh, &R, alv, tabs, s0, s1, opip); \
+#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, &R, alv, tabs, s0, s1, opip, M); \
                           else div_pass<M, SWAP, false>(sh, &R, alv, tabs, s0, s1, opip); break;
             XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
 #undef XP_DIV
@@ -1644,6 +1663,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         __syncthreads();
         for (int m = 0; m < family; ++m) {
             const SegDev& seg = sh.mseg[m];
+            if (m > 0) __syncthreads();
             if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc_of(m) * (u64)seg.n_ops;
             if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
             else tile_body<false>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
