@@ -237,15 +237,15 @@ def main():
     # Bytes that cross the bus per end-to-end step (structure sizes of the library, 256-byte aligned pieces):
     # grammar block (header 1128, leaves 16 each, binary productions 152 each); sketch head (sketch record 824,
     # hole record 5008 and a flag word per hole); job list of the load; plan head of the search (counters,
-    # segments 200 each, sketch pointer, accumulators 288 per hole).  Back: hole records and flags after the load,
+    # segments 200 each, sketch pointer, accumulators 296 per hole).  Back: hole records and flags after the load,
     # accumulators after the search.  Host tables of a table domain would add their own size (config 2 is a box).
     al = lambda b: (b + 255) // 256 * 256
     n_bin = sum(1 for p in sk.grammar.productions if p.kind == 2)
     n_leaf = len(sk.grammar.productions) - n_bin
     nh, n_segs = len(sk.holes), 16
     h2d = (al(1128) + al(16 * (n_leaf + 1)) + 152 * (n_bin + 1)) + (al(824) + al(5012 * nh)) + (al(8) + 16 * nh) + \
-          (256 + al(200 * (n_segs + 1)) + al(8 * 2) + al(288 * (nh + 1)))
-    d2h = 5012 * nh + 288 * nh
+          (256 + al(200 * (n_segs + 1)) + al(8 * 2) + al(296 * (nh + 1)))
+    d2h = 5012 * nh + 296 * nh
 
     tot = torch.tensor([dev_ms, float(evals), e2e_s, float(e2e_evals), kern_ms, float(ops)], dtype=torch.float64, device="cuda")
     if dist is not None:

@@ -180,7 +180,7 @@ typedef struct {
     uint64_t filter_survivors;      /* candidates that passed the first probe point */
     uint64_t probe_survivors;       /* candidates that passed every probe point */
     uint64_t nominal_ops;           /* 32-bit integer operations the filter stage's candidate-point evaluations
-                                       amount to under the library's cost model: one operation and one
+                                       that were carried out amount to under the library's cost model: one operation and one
                                        comparison per evaluation, with + - * min max = 1, a reciprocal division = 7
                                        (/ and % of one operand pair share it), a remainder's multiply-subtract = 1 */
     double kernel_ms;               /* device time of the whole call's kernels (CUDA events) */

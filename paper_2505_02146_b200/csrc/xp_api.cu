@@ -1011,7 +1011,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
                 hr.match_count[k] = a.match_count[k];
             }
             hr.evals = a.evals; hr.filter_survivors = a.filter_survivors; hr.probe_survivors = a.probe_survivors;
-            hr.nominal_ops = plan.nominal_ops[ai];
+            hr.nominal_ops = plan.nominal_ops[ai] - (a.ops_skipped < plan.nominal_ops[ai] ? a.ops_skipped : plan.nominal_ops[ai]);
             const int ls = (int)a.pad;
             if (ls >= 1 && ls <= hr.max_size && a.match_count[ls] > 0) {
                 hr.solved = 1; hr.least_size = ls; hr.least_rank = a.min_rank[ls];

@@ -126,6 +126,8 @@ struct AccDev {
     u64 match_count[kMaxSize + 1];
     u64 min_rank[kMaxSize + 1];
     u64 evals, filter_survivors, probe_survivors, pad;
+    u64 ops_skipped;                 // cost-model operations that the filter did not have to carry out (remainders
+                                     // of a tile none of whose divisors exceeds the target's magnitude)
 };
 
 // One contiguous piece of work.  kind 0 (linear): ranks [rank_begin, rank_end) of `size`,

@@ -320,7 +320,11 @@ struct CandShared {
 };
 
 constexpr int kMaxFamily = 8;
-struct MemberState { u64 bc_first; i32 lo, hi; u32 n, nspecial; i32 wide, pad; };
+struct MemberState {
+    u64 bc_first; i32 lo, hi; u32 n, nspecial; i32 wide;
+    i32 mod_possible;            // some operand of the member, as a divisor, exceeds the target's magnitude: only
+                                 // then can a remainder equal the target (|n % d| < |d|)
+};
 
 struct EvalShared {
     u64 ticket;
@@ -331,7 +335,7 @@ struct EvalShared {
     i32 cur_acc;
     u64 match_count[kMaxSize + 1];
     u64 min_rank[kMaxSize + 1];
-    u64 filter_survivors, probe_survivors;
+    u64 filter_survivors, probe_survivors, ops_skipped;
     u64 warp_evals[kThreads / 32];
     // tile tickets: the broadcast-side operands at probe 0 (entries invalid there are dropped) with
     // what the loops need of each, and the warps' queues of filter hits
@@ -378,11 +382,12 @@ __device__ __noinline__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64&
             if (tot) atomicAdd(&acc->evals, tot);
             if (sh.filter_survivors) atomicAdd(&acc->filter_survivors, sh.filter_survivors);
             if (sh.probe_survivors) atomicAdd(&acc->probe_survivors, sh.probe_survivors);
+            if (sh.ops_skipped) atomicAdd(&acc->ops_skipped, sh.ops_skipped);
         }
     }
     __syncthreads();
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; }
     my_evals = 0;
     __syncthreads();
 }
@@ -1384,8 +1389,8 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
 
 template <bool SWAP>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
-                                          u64 reg_first, i64* a64, const i32* a1, u32 a1ok, u32 alive, bool drain_at_end,
-                                          u64& my_evals) {
+                                          u64 reg_first, u64 pairs, i64* a64, const i32* a1, u32 a1ok, u32 alive,
+                                          bool drain_at_end, u64& my_evals) {
     const SegDev& seg = sh.mseg[m];
     const MemberState& mbs = sh.mb[m];
     const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
@@ -1437,6 +1442,11 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         }
     }
 
+    // A remainder is smaller in magnitude than its divisor: when no divisor of the tile exceeds the
+    // target's magnitude no candidate  a % b  can match, and the loops leave the remainders out.
+    const bool skip_mod = !SWAP && (mask & 16u) && !mbs.mod_possible && !tile_wide && !rng && A == 1u && t_small;
+    if (skip_mod && threadIdx.x == 0) sh.ops_skipped += pairs * ((mask & 8u) ? 2ull : 9ull);     // (cost model of the host plan)
+
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
     auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide || rng) {
@@ -1459,7 +1469,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         if (!(mask & 24u)) return;
         if (A != 1u) { div_pass_signed<SWAP>(sh, &R, alv, mask, A, tp, s0, s1, opip); return; }
         if (!t_small) return;                            // no int32 quotient or remainder can be the target
-        switch ((mask >> 3) & 3u) {
+        switch (skip_mod ? (mask >> 3) & 1u : (mask >> 3) & 3u) {
 #define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, &R, alv, tabs, s0, s1, opip, M); \
                           else div_pass<M, SWAP, false>(sh, &R, alv, tabs, s0, s1, opip); break;
             XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
@@ -1562,6 +1572,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
             const u64 lw = (u64)ftabs * ub;
             d.low = lw < (1ull << 31) ? (u32)lw : 0x80000000u;
             d.cmax = (ub != 0u && ftabs < ub) ? 0xffffffffu / ub : 0u;
+            if (d.cmax != 0u || !fits) mbs.mod_possible = 1;         // (benign race: every writer stores 1)
         }
         sh.bc_div[slot] = d;
     }
@@ -1646,7 +1657,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         mbs.bc_first = seg.bc_begin + (m == 0 ? bc_tile0 : 0) * (u64)seg.bc_tile;
         mbs.lo = keep ? seg.bc_base : 0;
         mbs.hi = keep ? seg.bc_base + n_bc_of(m) : kBcTile;
-        mbs.n = 0; mbs.nspecial = 0; mbs.wide = 0;
+        mbs.n = 0; mbs.nspecial = 0; mbs.wide = 0; mbs.mod_possible = 0;
     };
     if (keep) {
         // Every member's operands fit the tile side by side.  They are filled once (by the first
@@ -1664,9 +1675,10 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         for (int m = 0; m < family; ++m) {
             const SegDev& seg = sh.mseg[m];
             if (m > 0) __syncthreads();
-            if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc_of(m) * (u64)seg.n_ops;
-            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
-            else tile_body<false>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, false, my_evals);
+            const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
+            if (threadIdx.x == 0) my_evals += pairs * (u64)seg.n_ops;
+            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
+            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
         }
         drain_queue(sh, plan, sk, hole, reg_first, my_evals);
         return;
@@ -1678,9 +1690,10 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         if (fill_bc_operands(sh, g, hole, m, n_bc_of(m))) sh.mb[m].wide = 1;
         __syncthreads();
         const SegDev& seg = sh.mseg[m];
-        if (threadIdx.x == 0) my_evals += (u64)n_reg * (u64)n_bc_of(m) * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, true, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, m, reg_first, a64, a1, a1ok, alive, true, my_evals);
+        const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
+        if (threadIdx.x == 0) my_evals += pairs * (u64)seg.n_ops;
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
     }
 }
 
@@ -1691,7 +1704,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
