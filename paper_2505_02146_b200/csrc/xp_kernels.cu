@@ -1099,16 +1099,15 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     // The products' distances from the target (one multiply-add each, mul_nt = -tp) are folded
     // into running minima: a candidate hits iff its distance is zero, so one comparison per vote
     // group replaces one per candidate.
-    auto scan = [&](const BcRing& e, bool& h0, bool& h3, u32& m1, u32& m2) {
+    auto scan = [&](const BcRing& e, bool (&h)[4], u32 (&m)[4]) {
         const u32 t_one = (MASK & 1u) ? e.t_add : t_sub_of(e.t_add);       // used when only one of + - is present
 #pragma unroll
-        for (int j = 0; j < kNA; j += 2) {
-            if (kPair) { h0 |= ca[j] == e.t_pm; h3 |= ca[j + 1] == e.t_pm; }
-            else if (MASK & 3u) { h0 |= aA[j] == t_one; h3 |= aA[j + 1] == t_one; }
+        for (int j = 0; j < kNA; ++j) {
+            if (kPair) h[j & 3] |= ca[j] == e.t_pm;
+            else if (MASK & 3u) h[j & 3] |= aA[j] == t_one;
             if (MASK & 4u) {
-                const u32 d0 = aA[j] * e.mul_b + e.mul_nt, d1 = aA[j + 1] * e.mul_b + e.mul_nt;
-                m1 = d0 < m1 ? d0 : m1;
-                m2 = d1 < m2 ? d1 : m2;
+                const u32 d = aA[j] * e.mul_b + e.mul_nt;
+                m[j & 3] = d < m[j & 3] ? d : m[j & 3];
             }
         }
     };
@@ -1130,19 +1129,20 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
     // for the instruction cache.
     for (int s = s0; s < s1; s += 4) {
         const int n = s1 - s < 4 ? s1 - s : 4;
-        bool h0 = false, h3 = false;                    // independent chains of comparisons
-        u32 m1 = 0xffffffffu, m2 = 0xffffffffu;         // ... and of minima
+        bool h[4] = {false, false, false, false};       // independent chains of comparisons
+        u32 m[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};       // ... and of minima
         if (n == 4) {
             const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
-            scan(e0, h0, h3, m1, m2);
-            scan(e1, h0, h3, m1, m2);
-            scan(e2, h0, h3, m1, m2);
-            scan(e3, h0, h3, m1, m2);
+            scan(e0, h, m);
+            scan(e1, h, m);
+            scan(e2, h, m);
+            scan(e3, h, m);
         } else {
 #pragma unroll 1
-            for (int q = 0; q < n; ++q) { const BcRing e0 = sh.bc_ring[s + q]; scan(e0, h0, h3, m1, m2); }
+            for (int q = 0; q < n; ++q) { const BcRing e0 = sh.bc_ring[s + q]; scan(e0, h, m); }
         }
-        if (__any_sync(0xffffffffu, h0 | h3 | (m1 == 0u) | (m2 == 0u))) {
+        const u32 mm = (m[0] < m[1] ? m[0] : m[1]) < (m[2] < m[3] ? m[2] : m[3]) ? (m[0] < m[1] ? m[0] : m[1]) : (m[2] < m[3] ? m[2] : m[3]);
+        if (__any_sync(0xffffffffu, h[0] | h[1] | h[2] | h[3] | (mm == 0u))) {
 #pragma unroll 1
             for (int q = 0; q < n; ++q) resolve(s + q);
         }
