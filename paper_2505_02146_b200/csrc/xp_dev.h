@@ -85,7 +85,9 @@ struct HoleDev {
     // second: filter hits are also checked exactly at probe 1 before they are queued (needs tables, a
     // defined spec and an affine context at probe 1); sample_pass0: how many of the candidates
     // sampled at load satisfied probe 0 (a high rate makes the second look worth its cost).
-    i32 second, sample_pass0, sample_n, pad1;
+    i32 second, sample_pass0, sample_n;
+    i32 second_ok;                                // the second look is possible (tables, spec and context at probe 1): a
+                                                  // CTA that sees many filter hits for this hole turns it on for itself
     // Set by the host before the load's kernels run: the largest subtree size and the number of
     // probes that the tables may cover (their memory is laid out for that many), and whether the
     // search is small (then the second look is always taken).  prepare_kernel derives

@@ -270,6 +270,7 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
             const bool possible = n >= 2 && probes >= 2 && ((spec_ok & (amask | rmask)) >> 1 & 1u);
             const bool frequent = ncand > 0 && (u64)pass0 * 256 >= (u64)ncand;
             hole->second = possible && (hole->small_search || frequent) ? 1 : 0;
+            hole->second_ok = possible ? 1 : 0;
         }
     }
 }
@@ -279,6 +280,7 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
 // ------------------------------------------------------------------------------------------
 
 constexpr int kLinearPerThread = kLinearChunk / kThreads; // ranks per thread per linear ticket
+constexpr u64 kAdaptRate = 4096;                          // filter hits per evaluation above 1 / kAdaptRate are "many"
 constexpr int kWarps = kThreads / 32;
 constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check (all warps)
 constexpr int kWarpQueue = kQueueCap / kWarps;            // ... per warp: every warp keeps and empties its own queue
@@ -352,6 +354,8 @@ struct EvalShared {
     u32 wmember[kWarps];         // member the warp is working on (tags its queue entries)
     u32 wq_n[kWarps], wq_over[kWarps];
     // second look (HoleDev::second): context factor, offset and spec value at probe 1 of the hole at hand
+    i32 adapt_second;            // this CTA has seen more than one filter hit per kAdaptRate evaluations for the
+                                 // hole it works on: it takes the second look from now on (until it changes hole)
     i32 p1_on, p1_rng;           // p1_rng: the context compares at probe 1; the value must lie in [p1_lo, p1_hi]
     u64 p1_A, p1_B, p1_spec;
     i64 p1_lo, p1_hi;
@@ -387,7 +391,7 @@ __device__ __noinline__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64&
     }
     __syncthreads();
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; }
+    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; }
     my_evals = 0;
     __syncthreads();
 }
@@ -1534,7 +1538,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
     MemberState& mbs = sh.mb[m];
     const u64 bc_first = mbs.bc_first;
     const bool swap = seg.swap != 0;
-    const bool second = hole->second != 0;
+    const bool second = hole->second_ok != 0;           // (kept even while the second look is off: the CTA may turn it on)
     const u32 fA = (u32)hole->aff_A;
     const u64 ftq = (u64)hole->probe_spec[0] - hole->aff_B;
     const u32 ftp = (u32)ftq;
@@ -1613,7 +1617,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     const bool keep = sh.seg.bc_keep != 0;
     const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
     const int reg_nt = sh.seg.reg_nt, reg_size = sh.seg.reg_size;
-    const bool second = hole->second != 0;
+    const bool second = hole->second != 0 || (hole->second_ok != 0 && sh.adapt_second != 0);
     load_family(sh, plan, seg_index, family);
     if (threadIdx.x == 0) {
         sh.reg_wide = 0;
@@ -1704,11 +1708,15 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
-        if (threadIdx.x == 0) sh.ticket = atomicAdd(plan.ticket, 1ull);
+        if (threadIdx.x == 0) {
+            sh.ticket = atomicAdd(plan.ticket, 1ull);
+            // many filter hits so far for the hole at hand (this CTA's own counts): second look from now on
+            if (!sh.adapt_second && sh.filter_survivors * kAdaptRate > my_evals) sh.adapt_second = 1;
+        }
         __syncthreads();
         const u64 t = sh.ticket;
         if (t >= plan.n_tickets) break;
