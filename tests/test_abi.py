@@ -96,3 +96,19 @@ def test_no_cpu_fallback_without_a_device():
     with pytest.raises(xp.XpError) as e:
         xp.xp_sketch_load(gr, config1(0))
     assert e.value.status == 6
+    with pytest.raises(xp.XpError) as e:
+        xp.xp_sketch_load_batch([gr, gr], [config1(0), config1(1)])
+    assert e.value.status == 6 and "sketch 0" in str(e.value)
+
+
+def test_batch_load_checks_its_arguments_before_touching_a_device():
+    lib = xp.load()
+    outs = (C.c_void_p * 2)()
+    assert lib.xp_sketch_load_batch(None, None, 2, outs) == 1
+    assert b"null" in lib.xp_last_error()
+    gr = xp.xp_grammar_create(config1(0).grammar)
+    sk = config1(0)
+    sk.holes[0].max_size = 99                       # beyond XP_MAX_SIZE: refused by the host-side checks
+    with pytest.raises(xp.XpError) as e:
+        xp.xp_sketch_load_batch([gr], [sk])
+    assert e.value.status == 3 and "sketch 0" in str(e.value)
