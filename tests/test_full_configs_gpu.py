@@ -12,12 +12,21 @@ pytestmark = pytest.mark.gpu
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
-def _check_large(xp, name, make):
-    path = os.path.join(GOLDEN, f"{name}_seed0_full.json")
+def _seeds_with_goldens(name):
+    """Seeds for which tests/golden/ holds a full-size result of this configuration."""
+    seeds = []
+    for f in sorted(os.listdir(GOLDEN)):
+        if f.startswith(f"{name}_seed") and f.endswith("_full.json"):
+            seeds.append(int(f[len(name) + 5:-len("_full.json")]))
+    return seeds
+
+
+def _check_large(xp, name, make, seed=0):
+    path = os.path.join(GOLDEN, f"{name}_seed{seed}_full.json")
     if not os.path.exists(path):
         pytest.skip(f"{path} has not been generated")
     want = json.load(open(path))["holes"]
-    sk = make(0)
+    sk = make(seed)
     gr = xp.xp_grammar_create(sk.grammar)
     ls = xp.xp_sketch_load(gr, sk)
     got = xp.xp_repair(ls)
@@ -44,6 +53,14 @@ def test_config3_full(xp):
 def test_config4_full(xp):
     got = _check_large(xp, "config4", config4)
     assert sum(got[0].cand_count) == 322884631700
+
+
+@pytest.mark.parametrize("name,make,seed", [(n, m, sd) for n, m in (("config2", config2), ("config3", config3), ("config4", config4))
+                                            for sd in _seeds_with_goldens(n) if sd != 0])
+def test_other_seeds_full(xp, name, make, seed):
+    """Every further seed that has a golden: among them instances whose target is small at the probes, where a
+    large share of the candidates passes the filter (queue overflows, the second look turned on by the CTAs)."""
+    _check_large(xp, name, make, seed)
 
 
 def test_config5_full_batch(xp):
