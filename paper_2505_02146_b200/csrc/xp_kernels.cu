@@ -469,6 +469,32 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const SketchDev* sk,
     c.narrow = narrow ? 1 : 0;
 }
 
+// Operators that exist only inside a staged int32 program: division and remainder by a constant
+// that is not zero.  "push c; x / y" becomes one instruction on the top of the stack whose val
+// holds the constant (low half) and floor(2^32 / |c|) (high half), so that a point costs a
+// multiply-high and a correction instead of a 32-bit division.
+constexpr int kOpDivC = 32, kOpModC = 33;
+
+// Rewrites the constant divisions of a staged program that runs in int32 (only the vectorised
+// whole-domain check understands the result).  One lane.
+__device__ void fold_constant_divisors(CandShared& c) {
+    int w = 0;
+    for (int k = 0; k < c.len; ++k) {
+        const i32 cv = c.var[k];
+        const bool divmod = cv == -2 - XP_OP_DIV || cv == -2 - XP_OP_MOD;
+        if (divmod && w > 0 && c.var[w - 1] == -1 && c.val[w - 1] != 0 && c.val[w - 1] > -(1ll << 31) && c.val[w - 1] < (1ll << 31)) {
+            const i32 d = (i32)c.val[w - 1];
+            const u32 ad = d < 0 ? 0u - (u32)d : (u32)d;
+            const u32 M = ad == 1u ? 0xffffffffu : (u32)((1ull << 32) / ad);
+            c.var[w - 1] = -2 - (cv == -2 - XP_OP_DIV ? kOpDivC : kOpModC);
+            c.val[w - 1] = (i64)(((u64)M << 32) | (u32)d);
+            continue;                                     // (the operator took the place of the push)
+        }
+        c.var[w] = cv; c.val[w] = c.val[k]; ++w;
+    }
+    c.len = w;
+}
+
 // The staged program at one point with an operand stack of D registers (D >= its depth): a
 // push shifts the registers up, an operator combines the two lowest and shifts down.  The
 // program is the same for every thread, so all branches are uniform.
@@ -612,10 +638,23 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
                 }
                 continue;
             }
+            const int op = -2 - cv;
+            if (sizeof(T) == 4 && op >= kOpDivC) {          // x / c or x % c on the top of the stack, c != 0 a constant
+                const i32 d = (i32)(u32)(u64)c.val[k];
+                const u32 M = (u32)((u64)c.val[k] >> 32), ad = d < 0 ? 0u - (u32)d : (u32)d;
+#pragma unroll
+                for (int i = 0; i < P; ++i) {
+                    const i32 x = (i32)t.v[i];
+                    const u32 ux = x < 0 ? 0u - (u32)x : (u32)x;      // |x| < 2^31: the estimate is the quotient or one less
+                    u32 q = __umulhi(ux, M), r = ux - q * ad;
+                    if (r >= ad) { ++q; r -= ad; }
+                    t.v[i] = (T)(op == kOpDivC ? (((x < 0) != (d < 0)) ? (i32)(0u - q) : (i32)q) : (x < 0 ? (i32)(0u - r) : (i32)r));
+                }
+                continue;
+            }
             --below;
             Slot a;
             a.q = stack[below * 32 + lane];
-            const int op = -2 - cv;
             if (sizeof(T) == 8) {
 #pragma unroll
                 for (int i = 0; i < P; ++i) {
@@ -1791,6 +1830,8 @@ __global__ void __launch_bounds__(kThreads, 3) verify_kernel(const PlanDev plan)
                 skip = 0;
                 stage_candidate(cand, sk, hole, sv->size, sv->rank);
                 proj_points(sk, hole, sv->vars, &cand);
+                if (cand.narrow && sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth)
+                    fold_constant_divisors(cand);         // (exactly the case that takes the int32 vectorised check below)
             }
         }
         __syncwarp();
