@@ -382,3 +382,14 @@ def _structural_rank(g, text):
         raise KeyError(t)
 
     return rank(parse(text), 0)
+
+
+def test_integer_peak_microbenchmark_is_plausible(xp):
+    """The roofline denominator: independent 32-bit add chains reach about SMs x 128 lanes x clock,
+    multiply-add chains about half of that (they issue on one pipe of 64 lanes per SM)."""
+    import torch
+    add, mad = xp.xp_int32_peak()
+    props = torch.cuda.get_device_properties(0)
+    lanes = props.multi_processor_count * 128
+    assert 0.3e9 * lanes < add < 2.3e9 * lanes          # between 0.3 and 2.3 GHz worth of one add per lane and clock
+    assert 0.35 * add < mad < 0.75 * add
