@@ -26,7 +26,7 @@ WORKLOAD = "config2_thread_binding_matmul256_size7"
 # dram__bytes_read.sum + dram__bytes_write.sum of one eval_kernel launch on this workload, from the ncu capture
 # summarised in profiles/eval_kernel_config2.md (local-memory frames; the path is bound by the integer ALUs).
 # Set to None whenever eval_kernel changes, until the capture has been taken again.
-EVAL_KERNEL_DRAM_BYTES = 4.91e9
+EVAL_KERNEL_DRAM_BYTES = 5.02e9
 ORACLE_SAMPLE_RANKS = 500_000_000          # ranks of size 7 the oracle is timed on (about 15-25 s of one core)
 
 
