@@ -328,6 +328,15 @@ struct xp_sketch {
     char* arena = nullptr;
     size_t arena_bytes = 0, arena_used = 0;
     int arena_device = 0;
+    // The sketch's part of a launch plan under default options (every size, no rank window, no flag), as
+    // if it were the only sketch of the call: built on the first such call and copied, with ticket, sketch
+    // and accumulator numbers shifted, into the plan of every later one (a batch of thousands of small
+    // sketches would otherwise spend longer planning than some of its searches take).
+    mutable std::mutex plan_mu;
+    mutable bool plan_cached = false;
+    mutable std::vector<SegDev> plan_segs;
+    mutable std::vector<u64> plan_ops;
+    mutable u64 plan_tickets = 0;
 };
 
 // Checks a postfix expression; returns false when malformed or too deep.
@@ -858,10 +867,47 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
 
 constexpr u64 kTileMinRanks = 4096;          // smaller windows are searched rank by rank
 
+static void plan_sketch(const xp_sketch* s, size_t i, const xp_repair_opts* o, Plan* plan);
+
 static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
+    const bool plain = o->size_min <= 0 && o->size_max <= 0 && o->n_rank_ranges == 0 && o->flags == 0;
+    if (n > 16) { plan->segs.reserve(n * 8); plan->acc.reserve(n * 2); plan->nominal_ops.reserve(n * 2); }
     for (size_t i = 0; i < n; ++i) {
         const xp_sketch* s = sk[i];
         if (!s) return fail(XP_ERR_INVALID_ARG, "null sketch in batch");
+        if (!plain) { plan_sketch(s, i, o, plan); continue; }
+        {
+            std::lock_guard<std::mutex> lock(s->plan_mu);
+            if (!s->plan_cached) {
+                Plan own;
+                plan_sketch(s, 0, o, &own);
+                s->plan_segs = std::move(own.segs);
+                s->plan_ops = std::move(own.nominal_ops);
+                s->plan_tickets = own.n_tickets;
+                s->plan_cached = true;
+            }
+        }
+        const int acc_base = (int)plan->acc.size();
+        AccDev a;
+        memset(&a, 0, sizeof(a));
+        for (int k = 0; k <= kMaxSize; ++k) a.min_rank[k] = ~0ull;
+        for (int h = 0; h < s->n_holes; ++h) { plan->acc.push_back(a); plan->nominal_ops.push_back(s->plan_ops[h]); }
+        const size_t at = plan->segs.size();
+        plan->segs.insert(plan->segs.end(), s->plan_segs.begin(), s->plan_segs.end());
+        for (size_t j = at; j < plan->segs.size(); ++j) {
+            SegDev& c = plan->segs[j];
+            c.first_ticket += plan->n_tickets;
+            c.sketch = (i32)i;
+            c.acc += acc_base;
+        }
+        plan->n_tickets += s->plan_tickets;
+    }
+    return XP_OK;
+}
+
+// One sketch's segments, accumulators and tickets, appended to the plan as sketch number i.
+static void plan_sketch(const xp_sketch* s, size_t i, const xp_repair_opts* o, Plan* plan) {
+    {
         for (int h = 0; h < s->n_holes; ++h) {
             const HoleHost& ho = s->holes[h];
             AccDev a;
@@ -891,7 +937,6 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
             }
         }
     }
-    return XP_OK;
 }
 
 constexpr u32 kSurvCap = 65536;              // survivor queue entries of a call with its own workspace (at least)
