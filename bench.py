@@ -1,14 +1,20 @@
 #!/usr/bin/env python
-"""Benchmark of the repair search on the thread-binding workload (256x256 matmul tile nest:
-bx in [0,64), tx in [0,256), k in [0,8); 136 leaves; expression size <= 7; 213 939 625 416
-candidates x 131 072 domain points).
+"""Benchmark of the repair search.
 
-A step is one complete search (every size, counts and least solution) of one seeded instance.
-Prints one JSON line.  ``--impl reference`` times the CPU oracle on a bounded sample instead.
+Headline workload: the large search (4 variables, typed quasi-affine grammar, expression size <= 9,
+322 884 631 700 candidates, 2^20 explicit domain points with a caller-supplied spec table).  A step is
+one complete search (every size, counts and least solution) of the seed-0 instance.  The same JSON line
+carries, under ``per_config``, the same measurements for the thread-binding search (config 2), the
+three-hole convolution sketch (config 3, holes summed) and the batch of 4096 small instances (config 5).
+
+``--impl reference`` times the CPU oracle on a bounded sample of the headline workload instead.
+``--gpus N`` (under torchrun) runs one search per rank; ``--shard`` cuts ONE search into rank windows,
+one per rank, and merges the results over the process group.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -22,26 +28,68 @@ if ROOT not in sys.path:
 
 METRIC = "candidate_point_evals_per_s"
 UNIT = "GInt-evals/s"
-WORKLOAD = "config2_thread_binding_matmul256_size7"
-# dram__bytes_read.sum + dram__bytes_write.sum of one eval_kernel launch on this workload, from the ncu capture
-# summarised in profiles/eval_kernel_config2.md (local-memory frames; the path is bound by the integer ALUs).
-# Set to None whenever eval_kernel changes, until the capture has been taken again.
-EVAL_KERNEL_DRAM_BYTES = 5.02e9
-ORACLE_SAMPLE_RANKS = 500_000_000          # ranks of size 7 the oracle is timed on (about 15-25 s of one core)
+WORKLOADS = {
+    "config2": "config2_thread_binding_matmul256_size7",
+    "config3": "config3_conv2d_im2col_three_holes_size6",
+    "config4": "config4_large_quasi_affine_size9_table_2p20_points",
+    "config5": "config5_batch_4096_instances_size6",
+}
+HEADLINE = "config4"
+
+# Counters of one eval_kernel launch per workload, from the ncu captures summarised under profiles/
+# (dram = dram__bytes_read.sum + dram__bytes_write.sum, thread_inst = smsp__thread_inst_executed.sum).
+# They describe the kernel sources whose hash is given; bench.py reports them (roofline.traffic,
+# roofline.frac_executed) only while the sources still have that hash.
+NCU_CAPTURE = {
+    "kernel_hash": None,
+    "date": None,
+    "config2": {"dram_bytes": None, "thread_inst": None},
+    "config4": {"dram_bytes": None, "thread_inst": None},
+    "config5": {"dram_bytes": None, "thread_inst": None},
+}
 
 
-def oracle_sample(seed: int, n_ranks: int):
-    """Times the CPU oracle, as it stands, on a rank window of the benchmark instance."""
+def kernel_hash() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2505_02146_b200", "csrc")
+    for name in ("xp_dev.h", "xp_device.cuh", "xp_kernels.cu"):
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+# ------------------------------------------------------------------------------------------
+# the CPU oracle on a bounded sample of a workload (reported baseline; single thread)
+# ------------------------------------------------------------------------------------------
+
+def oracle_sample(name: str, scale: float = 1.0):
+    """Times the oracle, as it stands, on a fixed part of workload ``name``; returns
+    (candidate-point evaluations, seconds, description)."""
     import oracle
-    from xp_instances import config2
-    sk = config2(seed)
+    from xp_instances import config2, config3, config4, config5_instance
     oracle.build()
-    n7 = oracle.counts(sk.grammar, 0, 7)[7]
-    lo = n7 // 3                            # a window inside the size-7 space, away from its first block
+    if name == "config5":
+        n = max(1, int(48 * scale))
+        t0 = time.perf_counter()
+        ev = sum(oracle.repair_hole(config5_instance(0, i)).evals for i in range(n))
+        return ev, time.perf_counter() - t0, f"instances 0..{n - 1} of seed 0 in full, single thread"
+    sk = {"config2": config2, "config3": config3, "config4": config4}[name](0)
+    K = sk.holes[0].max_size - (1 - sk.holes[0].max_size % 2)       # the largest non-empty size
+    total = oracle.counts(sk.grammar, sk.holes[0].start_nt, K)[K]
+    n_ranks = int({"config2": 3.0e8, "config3": 1.0e8, "config4": 2.5e8}[name] * scale)
+    n_ranks = max(1, min(n_ranks, total))
+    lo = min(total // 3, total - n_ranks)                            # a window away from the first block
+    rr = {s: (0, 0) for s in range(1, sk.holes[0].max_size + 1)}
+    rr[K] = (lo, lo + n_ranks)
+    first = list(range(min(64, sk.n_points))) if sk.coords is not None else None
     t0 = time.perf_counter()
-    r = oracle.repair_hole(sk, rank_ranges={1: (0, 0), 3: (0, 0), 5: (0, 0), 7: (lo, lo + n_ranks)})
-    dt = time.perf_counter() - t0
-    return r.evals, dt, f"size-7 ranks [{lo}, {lo + n_ranks}) of seed {seed}, single thread"
+    r = oracle.repair_hole(sk, 0, rank_ranges=rr, first_points=first)
+    return r.evals, time.perf_counter() - t0, f"hole 0, size-{K} ranks [{lo}, {lo + n_ranks}) of seed 0, single thread"
+
+
+def cpu_baseline(name: str, scale: float = 1.0):
+    ev, dt, sample = oracle_sample(name, scale)
+    return {"value": ev / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+            "seconds": dt, "host_cores_present": os.cpu_count()}
 
 
 class ClockSampler:
@@ -85,12 +133,13 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    per_step = max(1_000_000, ORACLE_SAMPLE_RANKS // max(1, args.steps + args.warmup))
+    name = args.workload or HEADLINE
+    scale = 1.0 / max(1, args.steps + args.warmup) * 3.0           # the whole run stays within about a minute
     for _ in range(args.warmup):
-        oracle_sample(0, per_step // 8)
+        oracle_sample(name, scale / 8)
     evals, secs, sample = 0, 0.0, ""
     for _ in range(args.steps):
-        e, dt, sample = oracle_sample(0, per_step)
+        e, dt, sample = oracle_sample(name, scale)
         evals += e
         secs += dt
     value = evals / secs / 1e9
@@ -98,61 +147,196 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "note": "CPU oracle on a bounded rank window per step"},
+        "config": {"workload": WORKLOADS[name], "note": "CPU oracle on a bounded rank window per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample + " per step"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def run_batch(args, xp, torch, sketches, stream):
-    """Profiling aid (single GPU): the batched workload, 4096 small instances in one
-    ``xp_repair_batch`` call per step; prints a short JSON line of its own."""
-    grammars, loaded = {}, []
-    for sk in sketches:
-        key = tuple(v.hi for v in sk.grammar.variables)
-        if key not in grammars:
-            grammars[key] = xp.xp_grammar_create(sk.grammar)
-        loaded.append(xp.xp_sketch_load(grammars[key], sk))
-    ws = torch.empty(xp.xp_workspace_bytes(loaded), dtype=torch.uint8, device="cuda")
-    peak_add, _ = xp.xp_int32_peak()
+# ------------------------------------------------------------------------------------------
+# one workload on the GPU
+# ------------------------------------------------------------------------------------------
+
+class Workload:
+    """One config loaded on the device: ``step()`` is one complete search with everything resident;
+    ``e2e_step()`` encodes grammar and sketch from host descriptors, copies the host tables, searches
+    and reads the result back."""
+
+    def __init__(self, xp, torch, name, stream, instances=4096, window=0):
+        from xp_instances import config2, config3, config4, config5
+        self.xp, self.torch, self.name, self.stream = xp, torch, name, stream
+        self.batch = name == "config5"
+        self.rr = None
+        if self.batch:
+            self.sks = config5(0, instances)
+            self.keys = [tuple(v.hi for v in sk.grammar.variables) for sk in self.sks]
+            self.grs = {}
+            for sk, key in zip(self.sks, self.keys):
+                if key not in self.grs:
+                    self.grs[key] = xp.xp_grammar_create(sk.grammar)
+            self.marshalled = xp.marshal_sketches(self.sks)      # the C descriptors, in host memory, built once
+            self.loaded = xp.xp_sketch_load_batch([self.grs[k] for k in self.keys], self.sks, self.marshalled)
+            self.n_points = self.sks[0].n_points
+        else:
+            self.sk = {"config2": config2, "config3": config3, "config4": config4}[name](0)
+            self.gr = xp.xp_grammar_create(self.sk.grammar)
+            self.loaded = [xp.xp_sketch_load(self.gr, self.sk)]
+            self.n_points = self.sk.n_points
+            if window:
+                K = self.sk.holes[0].max_size - (1 - self.sk.holes[0].max_size % 2)
+                self.rr = [(-1, K, 0, window)]
+        self.ws = torch.empty(xp.xp_workspace_bytes(self.loaded, rank_ranges=self.rr), dtype=torch.uint8, device="cuda")
+
+    def step(self):
+        """Returns the flat list of hole results (batch: a packed array and the first hole's view)."""
+        xp = self.xp
+        if self.batch:
+            return xp.xp_repair_batch(self.loaded, packed=True, workspace=self.ws, stream=self.stream.cuda_stream)
+        return xp.xp_repair(self.loaded[0], workspace=self.ws, stream=self.stream.cuda_stream, rank_ranges=self.rr)
+
+    @staticmethod
+    def tally(res, batch):
+        """(evals, candidates, kernel_ms, launches, view of the first hole) of one step's results."""
+        if batch:
+            import paper_2505_02146_b200 as xp
+            packed, view = res
+            a = xp.summaries_as_numpy(packed)
+            return int(a["evals_executed"].sum()), int(a["cand_count"].sum()), view.kernel_ms, view.n_launches, view
+        ev = sum(r.evals_executed for r in res)
+        cand = sum(sum(r.cand_count) for r in res)
+        return ev, cand, res[0].kernel_ms, res[0].n_launches, res[0]
+
+    def e2e_step(self):
+        """Host descriptors and host tables in, results out; returns (evals, h2d bytes, d2h bytes, load s, search s).
+        The timed part is the library calls: grammar create, sketch load (host tables are copied to the device
+        here), search, result read-back."""
+        xp = self.xp
+        t0 = time.perf_counter()
+        if self.batch:
+            grs = {k: xp.xp_grammar_create(g.model) for k, g in self.grs.items()}
+            loaded = xp.xp_sketch_load_batch([grs[k] for k in self.keys], self.sks, self.marshalled)
+            t1 = time.perf_counter()
+            res = xp.xp_repair_batch(loaded, packed=True)
+        else:
+            gr = xp.xp_grammar_create(self.sk.grammar)
+            loaded = [xp.xp_sketch_load(gr, self.sk)]
+            t1 = time.perf_counter()
+            res = xp.xp_repair(loaded[0], rank_ranges=self.rr)
+        t2 = time.perf_counter()
+        ev, _, _, _, view = self.tally(res, self.batch)
+        infos = [xp.xp_sketch_info_get(l) for l in loaded]
+        h2d = sum(int(i.load_h2d_bytes) for i in infos) + view.h2d_bytes
+        d2h = sum(int(i.load_d2h_bytes) for i in infos) + view.d2h_bytes
+        del loaded
+        return ev, h2d, d2h, t1 - t0, t2 - t1
+
+
+def measure(xp, torch, name, args, stream, flush, peak_add, barrier, sampler=None, with_cpu=True, with_e2e=True):
+    """Times ``args.steps`` device-resident steps and as many end-to-end steps of one workload."""
+    w = Workload(xp, torch, name, stream, instances=args.instances, window=args.window)
     for _ in range(max(3, args.warmup)):
-        xp.xp_repair_batch(loaded, workspace=ws, stream=stream.cuda_stream)
+        res = w.step()
     torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.start()
+    barrier()
     dev_ms = kern_ms = 0.0
-    evals = ops = cand = 0
+    evals = launches = 0
     for _ in range(args.steps):
+        flush.fill_(1)                                    # L2 flush (256 MiB write), outside the events
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        res = xp.xp_repair_batch(loaded, workspace=ws, stream=stream.cuda_stream)
+        res = w.step()
         e1.record(stream)
         e1.synchronize()
         dev_ms += e0.elapsed_time(e1)
-        kern_ms += res[0][0].kernel_ms
-        evals += sum(r[0].evals_executed for r in res)
-        ops += sum(r[0].nominal_ops for r in res)
-        cand += sum(sum(r[0].cand_count) for r in res)
-    print(json.dumps({"metric": METRIC, "value": evals / (dev_ms * 1e-3) / 1e9, "unit": UNIT, "steps": args.steps,
-                      "ms_per_step": dev_ms / args.steps, "kernel_ms_per_step": kern_ms / args.steps,
-                      "time_to_solution_ms": res[0][0].total_ms,
-                      "config": {"workload": "config5_batch_%d_instances" % len(loaded), "candidates_per_step": cand // args.steps},
-                      "candidates_per_s": cand / (dev_ms * 1e-3),
-                      "roofline": {"bound": "alu", "achieved": ops / (kern_ms * 1e-3) / 1e9, "peak": peak_add / 1e9,
-                                   "unit": "G int32-op/s", "frac": ops / (kern_ms * 1e-3) / peak_add}}))
+        ev, cand, k_ms, n_l, view = w.tally(res, w.batch)
+        evals += ev
+        kern_ms += k_ms
+        launches += n_l
+    barrier()
+    clocks = sampler.stop() if sampler is not None else None
+    out = {"workload": WORKLOADS[name], "dev_ms": dev_ms, "kern_ms": kern_ms, "evals": evals, "launches": launches,
+           "cand": cand, "n_points": w.n_points, "view": view, "clocks": clocks, "res": res, "batch": w.batch}
+    if with_e2e:
+        for _ in range(2):                                # untimed: the first loads after other work are erratic
+            w.e2e_step()
+        torch.cuda.synchronize()
+        barrier()
+        e_ev = h2d = d2h = 0
+        load_s = search_s = 0.0
+        for _ in range(args.steps):
+            flush.fill_(1)
+            torch.cuda.synchronize()
+            ev, a, b, ls, ss = w.e2e_step()                # (both parts end with the device idle: every call waits for it)
+            e_ev += ev; h2d += a; d2h += b; load_s += ls; search_s += ss
+        out["e2e_s"] = load_s + search_s
+        out["e2e_evals"] = e_ev
+        out["e2e"] = {"h2d": h2d // args.steps, "d2h": d2h // args.steps, "load_ms": 1e3 * load_s / args.steps,
+                      "search_ms": 1e3 * search_s / args.steps}
+    if with_cpu:
+        out["cpu_baseline"] = cpu_baseline(name, 0.5 if name != HEADLINE else 1.0)
+    return out
+
+
+def roofline(m, steps, world, peak_add, peak_mad, name):
+    """Both accountings of the integer-ALU roofline for one workload's measurement."""
+    kern_s = m["kern_ms"] * 1e-3
+    floor_ops = 2.0 * m["evals"] / world                   # one operation + one comparison per evaluation that ran
+    achieved = floor_ops / kern_s / 1e9
+    peak = peak_add / 1e9
+    cap = NCU_CAPTURE.get(name) or {}
+    fresh = NCU_CAPTURE.get("kernel_hash") == kernel_hash()
+    thread_inst = cap.get("thread_inst") if fresh else None
+    out = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G int32-op/s", "frac": achieved / peak,
+           "frac_executed": (thread_inst * steps / kern_s / peak_add) if thread_inst else None,
+           "frac_cost_model": (m["model_ops"] / world) / kern_s / peak_add if m.get("model_ops") else None,
+           "traffic": cap.get("dram_bytes") if fresh else None,
+           "kernel": "eval_kernel",
+           "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
+           "model": "frac: 2 x candidate-point evaluations that ran (one 32-bit operation + one comparison each) / kernel time / peak; "
+                    "frac_executed: thread instructions of eval_kernel per launch (ncu capture %s, kernel sources %s) / live kernel time / peak; "
+                    "frac_cost_model: the library's nominal_ops (a straightforward 32-bit evaluator with a 7-operation reciprocal division)"
+                    % (NCU_CAPTURE.get("date"), NCU_CAPTURE.get("kernel_hash"))}
+    return out
+
+
+def summarise(m, steps, world, peak_add, peak_mad, name):
+    value = m["evals"] / (m["dev_ms"] * 1e-3) / 1e9
+    view = m["view"]
+    rec = {"workload": m["workload"], "value": value, "unit": UNIT, "ms_per_step": m["dev_ms"] / steps,
+           "kernel_ms_per_step": m["kern_ms"] / steps, "time_to_solution_ms": view.total_ms,
+           "candidates_per_step": m["cand"], "domain_points": m["n_points"],
+           "nominal_evals_per_step": m["cand"] * m["n_points"],
+           "evals_executed_per_step": m["evals"] // steps,
+           "candidates_per_s": m["cand"] * steps * world / (m["dev_ms"] * 1e-3),
+           "gpu_launches_per_step": m["launches"] // steps,
+           "roofline": roofline(m, steps, world, peak_add, peak_mad, name)}
+    if "e2e" in m:
+        rec["e2e"] = {"value": m["e2e_evals"] / m["e2e_s"] / 1e9, "unit": UNIT, "ms_per_step": 1e3 * m["e2e_s"] / steps,
+                      "h2d_bytes_per_step": m["e2e"]["h2d"], "d2h_bytes_per_step": m["e2e"]["d2h"],
+                      "load_ms": m["e2e"]["load_ms"], "search_ms": m["e2e"]["search_ms"], "l2": "flushed between steps"}
+    if "cpu_baseline" in m:
+        rec["cpu_baseline"] = m["cpu_baseline"]
+    return rec
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5"],
-                    help="profiling aid: time another config's instance instead (the bench line is config2's)")
+    ap.add_argument("--no-per-config", action="store_true", help="time the headline workload only")
+    ap.add_argument("--shard", action="store_true",
+                    help="with --gpus N: cut ONE headline search into N rank windows (one per rank) and merge the results")
+    ap.add_argument("--workload", default=None, choices=sorted(WORKLOADS),
+                    help="profiling aid: time this config alone (the default line's headline is config4)")
     ap.add_argument("--instances", type=int, default=4096,
                     help="profiling aid: number of instances of the config5 batch (a small case of the same kernels)")
     ap.add_argument("--window", type=int, default=0,
-                    help="profiling aid: search only the first WINDOW ranks of size 7 (a small case of the same kernel)")
+                    help="profiling aid: search only the first WINDOW ranks of the largest size (a small case of the same kernel)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -160,7 +344,6 @@ def main():
 
     import torch
     import paper_2505_02146_b200 as xp
-    from xp_instances import config2, config3, config4, config5
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -172,18 +355,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     xp.load()
-
-    # Independent problems shard with no data-path exchange.  Every rank searches its own copy of the seed-0
-    # instance: the work per GPU is then the same at every N (instances of other seeds differ in cost by up to
-    # 2.5x, which would measure the instances rather than the machine).
     stream = torch.cuda.current_stream()
-    if args.workload == "config5":
-        run_batch(args, xp, torch, config5(0, args.instances), stream)
-        return
-    sk = {"config2": config2, "config3": config3, "config4": config4}[args.workload](0)
-    gr = xp.xp_grammar_create(sk.grammar)
-    ls = xp.xp_sketch_load(gr, sk)
-    ws = torch.empty(xp.xp_workspace_bytes([ls]), dtype=torch.uint8, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > L2 (126 MB), written between steps
 
     def barrier():
@@ -192,104 +364,115 @@ def main():
         torch.cuda.synchronize()
 
     peak_add, peak_mad = xp.xp_int32_peak()
-    rr = [(0, 7, 0, args.window)] if args.window else None
-    for _ in range(max(3, args.warmup)):
-        res = xp.xp_repair(ls, workspace=ws, stream=stream.cuda_stream, rank_ranges=rr)[0]
+    head = args.workload or HEADLINE
+    if args.shard:
+        run_shard(args, xp, torch, dist, rank, world, stream, flush, barrier)
+        return
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    barrier()
-    dev_ms = kern_ms = 0.0
-    evals = ops = launches = 0
-    for _ in range(args.steps):
-        flush.fill_(1)                                    # L2 flush, outside the events
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        res = xp.xp_repair(ls, workspace=ws, stream=stream.cuda_stream, rank_ranges=rr)[0]
-        e1.record(stream)
-        e1.synchronize()
-        dev_ms += e0.elapsed_time(e1)
-        kern_ms += res.kernel_ms
-        evals += res.evals_executed
-        ops += res.nominal_ops
-        launches += res.n_launches
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-
-    # End to end through the public API with host buffers: grammar and sketch are encoded and
-    # copied to the device, searched, and the result read back, every step.
-    for _ in range(2):                                   # untimed: the first loads after the sampler exits are erratic
-        l2 = xp.xp_sketch_load(xp.xp_grammar_create(sk.grammar), sk)
-        xp.xp_repair(l2, rank_ranges=rr)
-        del l2
-    barrier()
-    t0 = time.perf_counter()
-    e2e_evals = 0
-    for _ in range(args.steps):
-        g2 = xp.xp_grammar_create(sk.grammar)
-        l2 = xp.xp_sketch_load(g2, sk)
-        r2 = xp.xp_repair(l2, rank_ranges=rr)[0]
-        e2e_evals += r2.evals_executed
-        if os.environ.get("XP_BENCH_DEBUG"):
-            print("e2e step: kernel_ms %.2f total_ms %.2f since start %.1f ms" % (r2.kernel_ms, r2.total_ms, 1e3 * (time.perf_counter() - t0)), file=sys.stderr)
-        del l2, g2
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    # Bytes that cross the bus per end-to-end step (structure sizes of the library, 256-byte aligned pieces):
-    # grammar block (header 1128, leaves 16 each, binary productions 152 each); sketch head (sketch record 824,
-    # hole record 5008 and a flag word per hole); job list of the load; plan head of the search (counters,
-    # segments 200 each, sketch pointer, accumulators 296 per hole).  Back: hole records and flags after the load,
-    # accumulators after the search.  Host tables of a table domain would add their own size (config 2 is a box).
-    al = lambda b: (b + 255) // 256 * 256
-    n_bin = sum(1 for p in sk.grammar.productions if p.kind == 2)
-    n_leaf = len(sk.grammar.productions) - n_bin
-    nh, n_segs = len(sk.holes), 16
-    h2d = (al(1128) + al(16 * (n_leaf + 1)) + 152 * (n_bin + 1)) + (al(824) + al(5012 * nh)) + (al(8) + 16 * nh) + \
-          (256 + al(200 * (n_segs + 1)) + al(8 * 2) + al(296 * (nh + 1)))
-    d2h = 5012 * nh + 296 * nh
-
-    tot = torch.tensor([dev_ms, float(evals), e2e_s, float(e2e_evals), kern_ms, float(ops)], dtype=torch.float64, device="cuda")
+    # Independent problems shard with no data-path exchange: every rank searches its own copy of the seed-0
+    # instance, so the work per GPU is the same at every N (instances of other seeds differ in cost).
+    sampler = ClockSampler(local) if rank == 0 else None
+    solo = world == 1
+    m = measure(xp, torch, head, args, stream, flush, peak_add, barrier, sampler,
+                with_cpu=solo and not args.no_cpu_baseline, with_e2e=True)
+    tot = torch.tensor([m["dev_ms"], float(m["evals"]), m["e2e_s"], float(m["e2e_evals"]), m["kern_ms"]], dtype=torch.float64, device="cuda")
     if dist is not None:
         mx = tot.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
         sm = tot.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        dev_ms, e2e_s, kern_ms = float(mx[0]), float(mx[2]), float(mx[4])
-        evals, e2e_evals, ops = float(sm[1]), float(sm[3]), float(sm[5])
+        m["dev_ms"], m["e2e_s"], m["kern_ms"] = float(mx[0]), float(mx[2]), float(mx[4])
+        m["evals"], m["e2e_evals"] = float(sm[1]), float(sm[3])
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
-
-    value = evals / (dev_ms * 1e-3) / 1e9
-    cand = sum(res.cand_count)
-    achieved = (ops / world) / (kern_ms * 1e-3) / 1e9                  # per GPU, G int32-op/s
-    peak = peak_add / 1e9
+    m["model_ops"] = sum(r.nominal_ops for r in m["res"]) * args.steps * world if not m["batch"] else None
+    rec = summarise(m, args.steps, world, peak_add, peak_mad, head)
+    view = m["view"]
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
-        "ms_per_step": dev_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int64", "data": "synthetic",
-        "config": {"workload": (WORKLOAD if args.workload == "config2" else args.workload) +
-                               (f"_first_{args.window}_ranks_of_size7" if args.window else ""),
-                   "candidates_per_step": cand, "domain_points": sk.n_points,
-                   "nominal_evals_per_step": cand * sk.n_points, "l2": "flushed between steps (256 MiB write)",
-                   "time_to_solution_ms": res.total_ms, "kernel_ms_per_step": kern_ms / args.steps,
-                   "candidates_per_s": cand * args.steps * world / (dev_ms * 1e-3),
-                   "filter_survivors": res.filter_survivors, "probe_survivors": res.probe_survivors,
-                   "least": res.least_text, "match_count": res.match_count},
-        "clocks": clocks,
-        "e2e": {"value": e2e_evals / e2e_s / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches,
-        "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G int32-op/s", "frac": achieved / peak,
-                     "traffic": EVAL_KERNEL_DRAM_BYTES if args.workload == "config2" and not args.window else None,
-                     "kernel": "eval_kernel",
-                     "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
-                     "model": "32-bit operations of one operation + one comparison per candidate-point evaluation of the filter stage"},
+        "config": {"workload": rec["workload"] + (f"_first_{args.window}_ranks_of_largest_size" if args.window else ""),
+                   "candidates_per_step": rec["candidates_per_step"], "domain_points": rec["domain_points"],
+                   "nominal_evals_per_step": rec["nominal_evals_per_step"],
+                   "evals_executed_per_step": rec["evals_executed_per_step"],
+                   "l2": "flushed between steps (256 MiB write)",
+                   "time_to_solution_ms": rec["time_to_solution_ms"], "kernel_ms_per_step": rec["kernel_ms_per_step"],
+                   "candidates_per_s": rec["candidates_per_s"],
+                   "value_counts": "candidate-point evaluations that ran (filter tests at the first probe, exact probe checks, "
+                                   "whole-domain points); candidates decided without a test are left out",
+                   "parallelism": "one search per GPU, no data-path collective" if world > 1 else "one GPU"},
+        "clocks": m["clocks"],
+        "e2e": {k: rec["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step", "load_ms", "search_ms", "l2")},
+        "gpu_launches": m["launches"],
+        "roofline": rec["roofline"],
     }
-    if not args.no_cpu_baseline and args.workload == "config2":
-        e, dt, sample = oracle_sample(0, ORACLE_SAMPLE_RANKS)
-        out["cpu_baseline"] = {"value": e / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-                               "seconds": dt, "host_cores_present": os.cpu_count()}
+    if not m["batch"]:
+        out["config"].update({"filter_tests": view.filter_tests, "candidates_skipped": view.candidates_skipped,
+                              "filter_survivors": view.filter_survivors, "probe_survivors": view.probe_survivors,
+                              "least": view.least_text, "match_count": view.match_count})
+    if "cpu_baseline" in rec:
+        out["cpu_baseline"] = rec["cpu_baseline"]
+    if solo and not args.no_per_config and args.workload is None:
+        out["per_config"] = {}
+        for name in ("config2", "config3", "config5"):
+            mm = measure(xp, torch, name, args, stream, flush, peak_add, barrier, None,
+                         with_cpu=not args.no_cpu_baseline, with_e2e=True)
+            mm["model_ops"] = sum(r.nominal_ops for r in mm["res"]) * args.steps if not mm["batch"] else None
+            out["per_config"][name] = summarise(mm, args.steps, 1, peak_add, peak_mad, name)
     print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_shard(args, xp, torch, dist, rank, world, stream, flush, barrier):
+    """ONE headline search cut into ``world`` contiguous rank windows per size; every rank searches its
+    window, the per-hole results are merged over the process group (counts add, least rank is the
+    minimum), and rank 0 compares the merged result with the stored full-size expected values."""
+    from paper_2505_02146_b200.sharding import merge_results, shard_rank_windows
+    from xp_instances import config4
+    sk = config4(0)
+    gr = xp.xp_grammar_create(sk.grammar)
+    ls = xp.xp_sketch_load(gr, sk)
+    counts = xp.xp_grammar_count(gr, sk.holes[0].start_nt, sk.holes[0].max_size)
+    rr = shard_rank_windows(counts, world, rank, hole=0)
+    ws = torch.empty(xp.xp_workspace_bytes([ls], rank_ranges=rr), dtype=torch.uint8, device="cuda")
+    for _ in range(max(3, args.warmup)):
+        res = xp.xp_repair(ls, workspace=ws, stream=stream.cuda_stream, rank_ranges=rr)[0]
+    barrier()
+    dev_ms, evals = 0.0, 0
+    for _ in range(args.steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        res = xp.xp_repair(ls, workspace=ws, stream=stream.cuda_stream, rank_ranges=rr)[0]
+        if dist is not None:
+            merged = merge_results(res.match_count, res.solved, res.least_size, res.least_rank)
+        else:
+            merged = (res.match_count, res.solved, res.least_size, res.least_rank)
+        e1.record(stream)
+        e1.synchronize()
+        dev_ms += e0.elapsed_time(e1)
+        evals += res.evals_executed
+    barrier()
+    tot = torch.tensor([dev_ms, float(evals)], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        mx = tot.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = tot.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        dev_ms, evals = float(mx[0]), float(sm[1])
+    if rank == 0:
+        gold_path = os.path.join(ROOT, "tests", "golden", "config4_seed0_full.json")
+        gold = json.load(open(gold_path))["holes"][0]
+        ok = (list(merged[0]) == gold["match_count"] and bool(merged[1]) == gold["solved"] and
+              (not gold["solved"] or (merged[2], merged[3]) == (gold["least_size"], gold["least_rank"])))
+        assert ok, "the merged result of the sharded search differs from the stored expected values"
+        print(json.dumps({"metric": METRIC, "value": evals / (dev_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": dev_ms / args.steps,
+                          "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "int64",
+                          "data": "synthetic",
+                          "config": {"workload": WORKLOADS["config4"], "parallelism": f"one search in {world} rank windows per size, "
+                                     "merged by all-reduce (sum of counts) and all-gather (least rank)",
+                                     "merged_equals_expected": True}}))
     if dist is not None:
         dist.destroy_process_group()
 

@@ -55,8 +55,8 @@ enum {
     XP_ERR_TOO_LARGE = 4,     /* a candidate count reaches 2^63, or a size limit of the library is exceeded */
     XP_ERR_NOMEM = 5,         /* host or device allocation failed, or the caller's workspace is too small */
     XP_ERR_CUDA = 6,          /* a CUDA call failed (message in xp_last_error) */
-    XP_ERR_TIMEOUT = 7,
-    XP_ERR_CANCELLED = 8      /* the caller's cancel word became non-zero between launches */
+    XP_ERR_TIMEOUT = 7,       /* the call's time limit (xp_repair_opts.timeout_ms) ran out between launches */
+    XP_ERR_CANCELLED = 8      /* the caller's cancel word became non-zero before or between launches */
 };
 
 /* Library limits. */
@@ -151,8 +151,15 @@ typedef struct {
     size_t workspace_bytes;             /*   at least xp_workspace_bytes(); NULL: the library uses a block of its
                                              own that it keeps from call to call (cudaMalloc when it must grow) */
     uint32_t flags;                     /* XP_FLAG_* */
-    const volatile int32_t* cancel;     /* optional host word polled between launches */
+    const volatile int32_t* cancel;     /* optional host word.  When it is given (or timeout_ms is), the search runs
+                                           as a series of bounded launches (at most XP_CANCEL_TICKETS work tickets,
+                                           a few milliseconds, each); the host waits for each, then reads the word:
+                                           non-zero ends the call with XP_ERR_CANCELLED and no result.  Nothing on
+                                           the device waits for the word, and no kernel is in flight on return. */
+    int64_t timeout_ms;                 /* > 0: the same series of launches, and the call ends with XP_ERR_TIMEOUT
+                                           once this much wall time has passed when a launch has finished */
 } xp_repair_opts;
+enum { XP_CANCEL_TICKETS = 8192 };
 
 enum {
     XP_FLAG_NO_FILTER = 1u,             /* skip the probe-point filter stage (every candidate is unranked
@@ -176,7 +183,9 @@ typedef struct {
     const xp_instr* least_code;     /* postfix of the least solution */
     int32_t least_len;
     const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))"; min and max as calls, "min(a,b)" */
-    uint64_t evals_executed;        /* candidate-point evaluations the GPU carried out for this hole */
+    uint64_t evals_executed;        /* candidate-point evaluations that ran for this hole: filter_tests plus the exact
+                                       evaluations of stage 2 (a hit at a probe point) and stage 3 (a survivor at a
+                                       domain point).  Candidates decided without a test are not in here. */
     uint64_t filter_survivors;      /* candidates that passed the first probe point */
     uint64_t probe_survivors;       /* candidates that passed every probe point */
     uint64_t nominal_ops;           /* 32-bit integer operations the filter stage's candidate-point evaluations
@@ -186,6 +195,14 @@ typedef struct {
     double kernel_ms;               /* device time of the whole call's kernels (CUDA events) */
     double total_ms;                /* host wall time of the whole call */
     int32_t n_launches;             /* kernels the call launched */
+    uint64_t filter_tests;          /* filter-stage tests at the first probe point that ran: pairs of operand subtrees
+                                       both defined there, times the operators whose test loop was entered */
+    uint64_t candidates_skipped;    /* candidates of the operand tiles visited that were decided without a test: an
+                                       operand undefined at the probe (a zero divisor inside it), a remainder whose
+                                       divisor cannot exceed the target's magnitude, a quotient or remainder of 32-bit
+                                       operands against a target outside 32 bits.  With a rank window the tiles also
+                                       cover some ranks outside it; those count here or in filter_tests as well. */
+    uint64_t h2d_bytes, d2h_bytes;  /* bytes the call copied to and from the device (the whole call, every hole) */
 } xp_result_view;
 
 /* Grammar (Section 4.4: the expressions the synthesis step may put into a hole).  Builds the
@@ -220,6 +237,32 @@ void xp_sketch_destroy(xp_sketch* s);
 xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, const xp_sketch_desc* descs, size_t n,
                                xp_sketch** outs);
 
+/* What a loaded sketch holds and what its load moved (no GPU is touched). */
+typedef struct {
+    int32_t n_holes, device;        /* device: the CUDA device the sketch was loaded on; calls on it must be made
+                                       with that device current (XP_ERR_INVALID_ARG otherwise) */
+    int64_t n_points;
+    uint64_t device_bytes;          /* device memory of the sketch (tables included, the caller's own tables not) */
+    uint64_t load_h2d_bytes, load_d2h_bytes;   /* bytes the load copied to and from the device (grammar tables
+                                                  included when this load was the grammar's first) */
+    int32_t n_probes[8];            /* probe points of the first 8 holes */
+    int32_t n_refined;              /* points promoted to probes by xp_sketch_refine so far */
+} xp_sketch_info;
+xp_status xp_sketch_info_get(const xp_sketch* s, xp_sketch_info* out);
+
+/* Counterexample-guided refinement of the probe points (the enumerative counterpart of the solver
+ * loop inside Algorithm 3's SynthesisCode: a candidate that satisfies every constraint looked at so
+ * far and then fails one gives that constraint to the next round).  Every search notes, per hole,
+ * the domain points at which candidates that had passed all probe points failed their whole-domain
+ * check.  This call promotes the most frequent of them (at most max_promote per hole, 0: the
+ * default of 4) to probe points, directly behind the first one, rebuilds the probe tables and
+ * clears the notes; n_promoted (may be NULL) receives how many points were promoted over all holes.
+ * Results of later searches are unchanged (a probe point is a domain point, and a match must hold
+ * at every domain point); only the work changes: candidates that used to reach the whole-domain
+ * check now end at a probe.  The sketch must not be in use by a search during the call.
+ * Errors: XP_ERR_INVALID_ARG, XP_ERR_CUDA. */
+xp_status xp_sketch_refine(xp_sketch* s, int32_t max_promote, int32_t* n_promoted);
+
 /* Device scratch a call over these sketches needs (0 on invalid arguments). */
 size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts);
 
@@ -249,12 +292,15 @@ void xp_result_free(xp_result* r);
  *
  *  - Inputs and outputs stay the caller's: the sketch (loaded earlier with xp_sketch_load,
  *    which does allocate) and `out`, an array of at least n_holes summaries, filled in place.
- *  - opts->workspace is ignored; size / rank windows, flags, stream and cancel work as in
- *    xp_repair.  The call returns after the stream has been synchronised.
+ *  - opts->workspace is ignored; size / rank windows, flags and stream work as in xp_repair;
+ *    cancel is read once, before the launch; timeout_ms is ignored.  The call copies from
+ *    pageable host memory and returns after the stream has been synchronised.
  *  - A call whose plan needs more than the fixed array, or a sketch with more than 64 holes,
  *    fails with XP_ERR_TOO_LARGE and a message giving the limit; nothing is launched.
  *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
- *    keeps it; make that first call before any stream capture begins.
+ *    keeps it per device; make that first call before any stream capture begins elsewhere in
+ *    the process.  Two threads making their first calls on one device at the same moment both
+ *    look the address up and store the same value: harmless, and not locked.
  *  - All calls share the one array per device.  Each call overwrites the whole part it uses
  *    (counter and accumulators are staged in their start state), so earlier contents never
  *    leak into a result; but two calls that overlap in time on the same device race on it.
@@ -273,6 +319,12 @@ typedef struct {
 } xp_hole_summary;
 xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_opts* opts, xp_hole_summary* out,
                            int32_t out_cap);
+
+/* The answers of n results (as xp_repair_batch returns them) in one array: the summaries of result 0's
+ * holes, then result 1's, and so on (Algorithm 3's hand-back step for a batch of snippets).  out_cap is
+ * the number of entries `out` holds; *n_out (may be NULL) receives the number written.
+ * Errors: XP_ERR_INVALID_ARG (null result, out too short). */
+xp_status xp_result_pack(const xp_result* const* results, size_t n, xp_hole_summary* out, size_t out_cap, size_t* n_out);
 
 /* Message of the calling thread's last failed call ("" if none). */
 const char* xp_last_error(void);

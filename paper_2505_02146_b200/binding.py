@@ -24,7 +24,8 @@ _STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_
 
 EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_grammar_unrank",
            "xp_sketch_load", "xp_sketch_load_batch", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
-           "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static"]
+           "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static",
+           "xp_sketch_info_get", "xp_sketch_refine", "xp_result_pack"]
 
 
 class XpError(RuntimeError):
@@ -69,7 +70,8 @@ class xp_rank_range(C.Structure):
 class xp_repair_opts(C.Structure):
     _fields_ = [("size_min", C.c_int32), ("size_max", C.c_int32), ("n_rank_ranges", C.c_int32),
                 ("rank_ranges", C.POINTER(xp_rank_range)), ("stream", C.c_void_p), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32), ("cancel", C.POINTER(C.c_int32))]
+                ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32), ("cancel", C.POINTER(C.c_int32)),
+                ("timeout_ms", C.c_int64)]
 
 
 class xp_result_view(C.Structure):
@@ -77,7 +79,15 @@ class xp_result_view(C.Structure):
                 ("match_count", C.POINTER(C.c_uint64)), ("least_size", C.c_int32), ("least_rank", C.c_uint64),
                 ("least_code", C.POINTER(xp_instr)), ("least_len", C.c_int32), ("least_text", C.c_char_p),
                 ("evals_executed", C.c_uint64), ("filter_survivors", C.c_uint64), ("probe_survivors", C.c_uint64),
-                ("nominal_ops", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
+                ("nominal_ops", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32),
+                ("filter_tests", C.c_uint64), ("candidates_skipped", C.c_uint64), ("h2d_bytes", C.c_uint64),
+                ("d2h_bytes", C.c_uint64)]
+
+
+class xp_sketch_info(C.Structure):
+    _fields_ = [("n_holes", C.c_int32), ("device", C.c_int32), ("n_points", C.c_int64), ("device_bytes", C.c_uint64),
+                ("load_h2d_bytes", C.c_uint64), ("load_d2h_bytes", C.c_uint64), ("n_probes", C.c_int32 * 8),
+                ("n_refined", C.c_int32)]
 
 
 class xp_hole_summary(C.Structure):
@@ -95,7 +105,8 @@ def load(path: Optional[str] = None):
     global _lib
     if _lib is not None:
         return _lib
-    lib = C.CDLL(path or _build.build())
+    # XP_CHECKED_BUILD=1 in the environment selects the variant with index checks compiled in
+    lib = C.CDLL(path or _build.build(checked=os.environ.get("XP_CHECKED_BUILD", "") == "1"))
     vp = C.c_void_p
     lib.xp_grammar_create.argtypes = [C.POINTER(xp_grammar_desc), C.POINTER(vp)]
     lib.xp_grammar_destroy.argtypes = [vp]
@@ -117,6 +128,9 @@ def load(path: Optional[str] = None):
     lib.xp_last_error.restype = C.c_char_p
     lib.xp_int32_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.xp_repair_static.argtypes = [vp, C.POINTER(xp_repair_opts), C.POINTER(xp_hole_summary), C.c_int32]
+    lib.xp_sketch_info_get.argtypes = [vp, C.POINTER(xp_sketch_info)]
+    lib.xp_sketch_refine.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32)]
+    lib.xp_result_pack.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_hole_summary), C.c_size_t, C.POINTER(C.c_size_t)]
     for name in EXPORTS:
         getattr(lib, name)
     _lib = lib
@@ -246,17 +260,26 @@ def xp_sketch_load(gr: Grammar, sk, coords=None, spec_tables: Optional[Dict[int,
     return LoadedSketch(out.value, gr, nh, [k for k in keep if not isinstance(k, C.Array)])
 
 
-def xp_sketch_load_batch(grs: Sequence[Grammar], sks: Sequence) -> List[LoadedSketch]:
-    """Loads ``sks[i]`` against ``grs[i]`` in one call (one wait for the device for the whole batch)."""
-    lib = load()
+def marshal_sketches(sks: Sequence):
+    """The C descriptors (``xp_sketch_desc`` array and what it points to, all in host memory) of a
+    list of sketches, for callers that load the same descriptions more than once."""
     n = len(sks)
-    assert len(grs) == n and n > 0
     descs = (xp_sketch_desc * n)()
     keeps, nhs = [], []
     for i, sk in enumerate(sks):
         keep = []
         nhs.append(_fill_sketch_desc(descs[i], sk, None, None, keep))
         keeps.append(keep)
+    return descs, nhs, keeps
+
+
+def xp_sketch_load_batch(grs: Sequence[Grammar], sks: Sequence, marshalled=None) -> List[LoadedSketch]:
+    """Loads ``sks[i]`` against ``grs[i]`` in one call (one wait for the device for the whole batch).
+    ``marshalled``: the result of ``marshal_sketches(sks)``, to skip building the descriptors again."""
+    lib = load()
+    n = len(sks)
+    assert len(grs) == n and n > 0
+    descs, nhs, keeps = marshalled if marshalled is not None else marshal_sketches(sks)
     handles = (C.c_void_p * n)(*[g.handle for g in grs])
     outs = (C.c_void_p * n)()
     _check(lib.xp_sketch_load_batch(handles, descs, n, outs))
@@ -279,6 +302,10 @@ class HoleResult:
     kernel_ms: float
     total_ms: float
     n_launches: int
+    filter_tests: int = 0
+    candidates_skipped: int = 0
+    h2d_bytes: int = 0
+    d2h_bytes: int = 0
 
 
 def xp_result_get(result_handle: int, hole: int) -> HoleResult:
@@ -290,13 +317,17 @@ def xp_result_get(result_handle: int, hole: int) -> HoleResult:
                       v.least_text.decode() if v.solved else "",
                       [(v.least_code[i].kind, v.least_code[i].arg, v.least_code[i].value) for i in range(v.least_len)],
                       int(v.evals_executed), int(v.filter_survivors), int(v.probe_survivors),
-                      int(v.nominal_ops), float(v.kernel_ms), float(v.total_ms), int(v.n_launches))
+                      int(v.nominal_ops), float(v.kernel_ms), float(v.total_ms), int(v.n_launches),
+                      int(v.filter_tests), int(v.candidates_skipped), int(v.h2d_bytes), int(v.d2h_bytes))
 
 
-def _opts(size_min=0, size_max=0, rank_ranges=None, stream=None, workspace=None, flags=0):
+def _opts(size_min=0, size_max=0, rank_ranges=None, stream=None, workspace=None, flags=0, cancel=None, timeout_ms=0):
     o = xp_repair_opts()
-    o.size_min, o.size_max, o.flags = size_min, size_max, flags
+    o.size_min, o.size_max, o.flags, o.timeout_ms = size_min, size_max, flags, int(timeout_ms)
     keep = []
+    if cancel is not None:             # a ctypes.c_int32 that another thread may set
+        o.cancel = C.pointer(cancel)
+        keep.append(cancel)
     if rank_ranges:
         rr = (xp_rank_range * len(rank_ranges))()
         for i, (hole, size, b, e) in enumerate(rank_ranges):
@@ -319,7 +350,8 @@ def xp_workspace_bytes(sketches: Sequence[LoadedSketch], **kw) -> int:
 
 def xp_repair(sketch: LoadedSketch, **kw) -> List[HoleResult]:
     """Keyword options: size_min, size_max, rank_ranges=[(hole, size, begin, end)], stream (raw
-    cudaStream_t), workspace (torch CUDA uint8 tensor), flags.  Returns one result per hole."""
+    cudaStream_t), workspace (torch CUDA uint8 tensor), flags, cancel (a ``ctypes.c_int32`` polled
+    between launches), timeout_ms.  Returns one result per hole."""
     o, _keep = _opts(**kw)
     out = C.c_void_p()
     _check(load().xp_repair(sketch.handle, C.byref(o), C.byref(out)))
@@ -329,17 +361,42 @@ def xp_repair(sketch: LoadedSketch, **kw) -> List[HoleResult]:
         load().xp_result_free(out.value)
 
 
-def xp_repair_batch(sketches: Sequence[LoadedSketch], **kw) -> List[List[HoleResult]]:
+def xp_repair_batch(sketches: Sequence[LoadedSketch], packed: bool = False, **kw):
+    """``packed=False``: one list of ``HoleResult`` per sketch.  ``packed=True``: ``(summaries, view)``
+    where ``summaries`` is ONE ctypes array of ``xp_hole_summary`` (the holes of sketch 0, then of sketch 1,
+    ...) filled by a single ``xp_result_pack`` call, and ``view`` is the full ``HoleResult`` of the first
+    hole (timings, counters and byte counts of the whole call)."""
     o, _keep = _opts(**kw)
+    lib = load()
     n = len(sketches)
     arr = (C.c_void_p * n)(*[s.handle for s in sketches])
     outs = (C.c_void_p * n)()
-    _check(load().xp_repair_batch(arr, n, C.byref(o), outs))
+    _check(lib.xp_repair_batch(arr, n, C.byref(o), outs))
     try:
+        if packed:
+            total = sum(s.n_holes for s in sketches)
+            out = (xp_hole_summary * total)()
+            got = C.c_size_t()
+            _check(lib.xp_result_pack(outs, n, out, total, C.byref(got)))
+            return out, xp_result_get(outs[0], 0)
         return [[xp_result_get(outs[i], h) for h in range(sketches[i].n_holes)] for i in range(n)]
     finally:
         for i in range(n):
-            load().xp_result_free(outs[i])
+            lib.xp_result_free(outs[i])
+
+
+def xp_sketch_info_get(sketch: LoadedSketch) -> xp_sketch_info:
+    out = xp_sketch_info()
+    _check(load().xp_sketch_info_get(sketch.handle, C.byref(out)))
+    return out
+
+
+def xp_sketch_refine(sketch: LoadedSketch, max_promote: int = 0) -> int:
+    """Promotes the domain points that ended whole-domain checks in earlier searches to probe
+    points; returns how many were promoted."""
+    n = C.c_int32()
+    _check(load().xp_sketch_refine(sketch.handle, max_promote, C.byref(n)))
+    return int(n.value)
 
 
 def xp_repair_static(sketch: LoadedSketch, **kw) -> List[xp_hole_summary]:
@@ -351,6 +408,17 @@ def xp_repair_static(sketch: LoadedSketch, **kw) -> List[xp_hole_summary]:
     out = (xp_hole_summary * sketch.n_holes)()
     _check(load().xp_repair_static(sketch.handle, C.byref(o), out, sketch.n_holes))
     return list(out)
+
+
+SUMMARY_DTYPE = np.dtype([("solved", "<i4"), ("max_size", "<i4"), ("least_size", "<i4"), ("pad", "<i4"),
+                          ("least_rank", "<u8"), ("cand_count", "<u8", (XP_MAX_SIZE + 1,)),
+                          ("match_count", "<u8", (XP_MAX_SIZE + 1,)), ("evals_executed", "<u8"), ("least_text", "S256")])
+
+
+def summaries_as_numpy(packed) -> np.ndarray:
+    """A structured numpy view (no copy) of an array of ``xp_hole_summary``."""
+    assert C.sizeof(xp_hole_summary) == SUMMARY_DTYPE.itemsize
+    return np.frombuffer(packed, dtype=SUMMARY_DTYPE)
 
 
 def xp_int32_peak() -> Tuple[float, float]:

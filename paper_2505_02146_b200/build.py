@@ -9,28 +9,31 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libxpiler_repair.so")
+LIB_CHECKED = os.path.join(HERE, "libxpiler_repair_checked.so")       # the same sources with -DXP_CHECKS (index checks)
 SOURCES = ["xp_api.cu", "xp_kernels.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "xp.h"), __file__]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compiles the CUDA sources into the shared library next to this file; returns its path."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compiles the CUDA sources into the shared library next to this file; returns its path.
+    ``checked``: the variant with index checks compiled in (a library of its own beside the normal one)."""
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
+    if not force and not _stale(LIB):
         return LIB
     objs = []
     procs = []
     for src in SOURCES:
-        obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = ["nvcc", *FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        obj = os.path.join(CSRC, src.replace(".cu", ".checked.o" if checked else ".o"))
+        cmd = ["nvcc", *FLAGS, *(["-DXP_CHECKS"] if checked else []), "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas"); cmd.insert(2, "-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -48,4 +51,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

@@ -2,6 +2,7 @@
 // decoding and the C ABI declared in include/xp.h.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <climits>
 #include <chrono>
 #include <cstdio>
@@ -59,29 +60,39 @@ struct DevPool {
 std::mutex g_pool_mu;
 std::map<int, DevPool> g_pools;
 
-cudaError_t pool_alloc(void** out, size_t bytes, int* device_out) {
+// *granted receives the size of the block handed out (>= bytes): it is what pool_release must be given.
+cudaError_t pool_alloc(void** out, size_t bytes, int* device_out, size_t* granted) {
     const size_t need = ((bytes ? bytes : 1) + 255) & ~(size_t)255;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     *device_out = dev;
+    *granted = need;
     std::lock_guard<std::mutex> lock(g_pool_mu);
     DevPool& p = g_pools[dev];
+    // a kept block fits a request when it wastes at most an eighth of itself (sketches of varying
+    // sizes then reuse each other's blocks instead of growing the pool without bound)
+    auto fits = [&](std::multimap<size_t, char*>& m) {
+        auto it = m.lower_bound(need);
+        return (it != m.end() && it->first - need <= it->first / 8) ? it : m.end();
+    };
     if (need > kPoolBigBytes) {
-        auto big = p.big_blocks.find(need);
+        auto big = fits(p.big_blocks);
         if (big == p.big_blocks.end()) return cudaMalloc(out, need);
         *out = big->second;
+        *granted = big->first;
+        p.big_kept -= big->first;
         p.big_blocks.erase(big);
-        p.big_kept -= need;
         return cudaSuccess;
     }
-    auto it = p.free_blocks.find(need);
-    if (it != p.free_blocks.end()) { *out = it->second; p.free_blocks.erase(it); return cudaSuccess; }
+    auto it = fits(p.free_blocks);
+    if (it != p.free_blocks.end()) { *out = it->second; *granted = it->first; p.free_blocks.erase(it); return cudaSuccess; }
     if (p.slab_left < need) {
+        if (p.slab_left >= 256) p.free_blocks.insert({p.slab_left, p.slab});      // the old slab's tail stays usable
         char* slab = nullptr;
         e = cudaMalloc((void**)&slab, kPoolSlabBytes);
-        if (e != cudaSuccess) return e;
-        p.slab = slab;                     // what was left of the previous slab stays unused
+        if (e != cudaSuccess) { p.slab = nullptr; p.slab_left = 0; return e; }
+        p.slab = slab;
         p.slab_left = kPoolSlabBytes;
     }
     *out = p.slab;
@@ -104,6 +115,9 @@ void pool_release(void* ptr, size_t bytes, int device) {
     p.free_blocks.insert({need, (char*)ptr});
 }
 }  // namespace
+
+struct xp_sketch;
+static xp_status check_device(const xp_sketch* const* sk, size_t n);
 
 static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
 
@@ -276,9 +290,17 @@ extern "C" xp_status xp_grammar_unrank(const xp_grammar* g, int32_t nt, int32_t 
     return XP_OK;
 }
 
-static xp_status grammar_to_device(xp_grammar* g) {
+static xp_status grammar_to_device(xp_grammar* g, size_t* copied) {
+    *copied = 0;
     std::lock_guard<std::mutex> lock(g->mu);
-    if (g->d_g) return XP_OK;
+    if (g->d_g) {
+        // the device copy was made on the device that was current at the first load and serves that device only
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev != g->d_device)
+            return fail(XP_ERR_INVALID_ARG, "the grammar's tables live on device " + std::to_string(g->d_device) +
+                        ", the current device is " + std::to_string(dev) + ": use one grammar handle per device");
+        return XP_OK;
+    }
     GrammarDev h;
     memset(&h, 0, sizeof(h));
     h.n_vars = g->n_vars; h.n_nt = g->n_nt;
@@ -291,8 +313,9 @@ static xp_status grammar_to_device(xp_grammar* g) {
     const size_t off_bins = off_leaves + ((sizeof(LeafDev) * (g->leaves.size() + 1) + 255) & ~(size_t)255);
     const size_t total = off_bins + sizeof(BinDev) * (g->bins.size() + 1);
     char* block = nullptr;
-    XP_CUDA(pool_alloc((void**)&block, total, &g->d_device));
-    g->d_bytes = total;
+    size_t granted = 0;
+    XP_CUDA(pool_alloc((void**)&block, total, &g->d_device, &granted));
+    g->d_bytes = granted;
     h.leaves = (const LeafDev*)(block + off_leaves);
     h.bins = (const BinDev*)(block + off_bins);
     std::vector<char> stage(total, 0);
@@ -300,8 +323,9 @@ static xp_status grammar_to_device(xp_grammar* g) {
     if (!g->leaves.empty()) memcpy(&stage[off_leaves], g->leaves.data(), sizeof(LeafDev) * g->leaves.size());
     if (!g->bins.empty()) memcpy(&stage[off_bins], g->bins.data(), sizeof(BinDev) * g->bins.size());
     cudaError_t e = cudaMemcpy(block, stage.data(), total, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) { pool_release(block, total, g->d_device); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
+    if (e != cudaSuccess) { pool_release(block, g->d_bytes, g->d_device); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
     g->d_g = (GrammarDev*)block;
+    *copied = total;
     return XP_OK;
 }
 
@@ -328,6 +352,13 @@ struct xp_sketch {
     char* arena = nullptr;
     size_t arena_bytes = 0, arena_used = 0;
     int arena_device = 0;
+    size_t load_h2d = 0, load_d2h = 0;               // bytes the load moved
+    std::vector<int> n_probes;                       // per hole, as the load (or the last refinement) left them
+    int n_refined = 0;                               // points promoted to probes by xp_sketch_refine
+    std::vector<size_t> off_kill;                    // per hole: offset of its table of whole-domain failures in the arena
+    size_t off_holes = 0;
+    int tab_size_cap = 0, tab_probes_cap = 0;        // most sizes / probes that the subtree tables of a hole cover
+    u64 entries_at[kMaxSize + 1] = {0};              // subtree-table entries per size (all nonterminals)
     // The sketch's part of a launch plan under default options (every size, no rank window, no flag), as
     // if it were the only sketch of the call: built on the first such call and copied, with ticket, sketch
     // and accumulator numbers shifted, into the plan of every later one (a batch of thousands of small
@@ -435,7 +466,8 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(XP_ERR_CUDA, "no CUDA device is usable");
-    xp_status st = grammar_to_device(g);
+    size_t grammar_bytes = 0;
+    xp_status st = grammar_to_device(g, &grammar_bytes);
     if (st != XP_OK) return st;
 
     xp_sketch* s = new (std::nothrow) xp_sketch;
@@ -469,6 +501,8 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
         if (d->holes[h].spec_kind == XP_SPEC_TABLE && np > 0 && !d->holes[h].spec_table_on_device && spec_bytes <= kPackMax) {
             off_spec[h] = off; off += al(spec_bytes);
         }
+    s->off_kill.assign(nh, 0);
+    for (int h = 0; h < nh; ++h) { s->off_kill[h] = off; off += al((sizeof(i64) + sizeof(u32)) * kKillSlots); }
     const size_t head = off;                              // [0, head): staged on the host and copied in one piece
     if ((copy_coords && coords_bytes > kPackMax) || stage_box) { off_coords = off; off += al(coords_bytes); }
     std::vector<HoleDev>& hh = L->hh;
@@ -492,12 +526,13 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
             off_tabm[h] = off; off += al(entries);
         }
     }
-    if (pool_alloc((void**)&s->arena, off, &s->arena_device) != cudaSuccess) {
+    size_t arena_granted = 0;
+    if (pool_alloc((void**)&s->arena, off, &s->arena_device, &arena_granted) != cudaSuccess) {
         (void)cudaGetLastError();
         delete s;
         return fail(XP_ERR_NOMEM, "device memory for the sketch (" + std::to_string(off) + " bytes)");
     }
-    s->arena_bytes = off;
+    s->arena_bytes = arena_granted;
     s->arena_used = off;
     char* base = s->arena;
     s->d_s = (SketchDev*)(base + off_sketch);
@@ -575,6 +610,8 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
         if (hd.spec_kind == XP_SPEC_EXPR)
             for (int i = 0; i < hd.spec_len; ++i) if (hd.spec_expr[i].kind == XP_I_VAR) fv |= 1u << hd.spec_expr[i].arg;
         o.fixed_vars = fv;
+        o.kill_pid = (i64*)(base + s->off_kill[h]);
+        o.kill_cnt = (u32*)(base + s->off_kill[h] + sizeof(i64) * kKillSlots);
         HoleHost ho;
         ho.start_nt = hd.start_nt; ho.max_size = hd.max_size;
         s->holes.push_back(ho);
@@ -589,13 +626,20 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
         const xp_hole_desc& hd = d->holes[h];
         if (hd.spec_kind == XP_SPEC_TABLE && np > 0 && !hd.spec_table_on_device && spec_bytes <= kPackMax)
             memcpy(&stg[off_spec[h]], hd.spec_table, spec_bytes);
+        memset(&stg[s->off_kill[h]], 0xff, sizeof(i64) * kKillSlots);           // no point noted yet (ids -1, counts 0)
     }
+    s->load_h2d = grammar_bytes + head;
     XP_CUDA_S(cudaMemcpyAsync(base, stg.data(), head, cudaMemcpyHostToDevice, nullptr));
-    if (copy_coords && coords_bytes > kPackMax) XP_CUDA_S(cudaMemcpyAsync(base + off_coords, d->coords, coords_bytes, cudaMemcpyHostToDevice, nullptr));
+    if (copy_coords && coords_bytes > kPackMax) {
+        XP_CUDA_S(cudaMemcpyAsync(base + off_coords, d->coords, coords_bytes, cudaMemcpyHostToDevice, nullptr));
+        s->load_h2d += coords_bytes;
+    }
     for (int h = 0; h < nh; ++h) {
         const xp_hole_desc& hd = d->holes[h];
-        if (hd.spec_kind == XP_SPEC_TABLE && np > 0 && !hd.spec_table_on_device && spec_bytes > kPackMax)
+        if (hd.spec_kind == XP_SPEC_TABLE && np > 0 && !hd.spec_table_on_device && spec_bytes > kPackMax) {
             XP_CUDA_S(cudaMemcpyAsync(base + off_spec[h], hd.spec_table, spec_bytes, cudaMemcpyHostToDevice, nullptr));
+            s->load_h2d += spec_bytes;
+        }
     }
     // The load's kernels, in stream order: points of a box and values of spec expressions (so that
     // the whole-domain check, and the probe choice, read tables for every kind of domain); bounds of a
@@ -608,6 +652,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
                 XP_CUDA_S(launch_stage_spec(s->d_s, h, n_points, (i64*)(base + off_spec[h]), (u32*)(base + off_bad) + h, nullptr));
     L->s = s;
     L->off_holes = off_holes;
+    s->off_holes = off_holes;
     L->table_points = d->domain_kind == XP_DOMAIN_TABLE ? n_points : 0;
     for (int h = 0; h < nh; ++h) {
         if (hh[h].tab_size_cap > L->size_cap) L->size_cap = hh[h].tab_size_cap;
@@ -615,6 +660,8 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     }
     for (int k = 1; k <= kMaxSize; ++k)
         for (int nt = 0; nt < g->n_nt; ++nt) L->entries_at[k] += g->cnt[nt][k];
+    s->tab_size_cap = L->size_cap; s->tab_probes_cap = L->probes_cap;
+    memcpy(s->entries_at, L->entries_at, sizeof(s->entries_at));
 #undef XP_CUDA_S
     return XP_OK;
 }
@@ -654,9 +701,8 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
             }
         }
     }
-    jobs_bytes = stage.size();
-    XP_CUDA_B(pool_alloc((void**)&jobs_dev, jobs_bytes, &jobs_device));
-    XP_CUDA_B(cudaMemcpyAsync(jobs_dev, stage.data(), jobs_bytes, cudaMemcpyHostToDevice, nullptr));
+    XP_CUDA_B(pool_alloc((void**)&jobs_dev, stage.size(), &jobs_device, &jobs_bytes));
+    XP_CUDA_B(cudaMemcpyAsync(jobs_dev, stage.data(), stage.size(), cudaMemcpyHostToDevice, nullptr));
     SketchDev* const* d_list = (SketchDev* const*)jobs_dev;
     const LoadJob* d_jobs = (const LoadJob*)(jobs_dev + list_bytes);
     // In stream order after the copies and the boxes' staging: bounds of the tables' coordinates;
@@ -685,6 +731,8 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
         const int nh = st[i].s->n_holes;
         st[i].back.resize(sizeof(HoleDev) * nh + sizeof(u32) * nh);
         XP_CUDA_B(cudaMemcpyAsync(st[i].back.data(), st[i].s->arena + st[i].off_holes, st[i].back.size(), cudaMemcpyDeviceToHost, nullptr));
+        st[i].s->load_d2h = st[i].back.size();
+        st[i].s->load_h2d += sizeof(SketchDev*) + sizeof(LoadJob) * (size_t)nh;       // its lines of the batch's job lists
     }
     XP_CUDA_B(cudaStreamSynchronize(nullptr));
 #undef XP_CUDA_B
@@ -701,6 +749,7 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
             s->holes[h].filter_ok = o.filter_ok != 0;
             s->holes[h].compares = o.filter_ok != 0 && o.aff_ok == 0;
             s->holes[h].never = bad != 0;                 // the spec is undefined at some point
+            s->n_probes.push_back(o.n_probe);
         }
         outs[i] = s;
     }
@@ -710,6 +759,99 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
 extern "C" xp_status xp_sketch_load(const xp_grammar* g, const xp_sketch_desc* d, xp_sketch** out) {
     if (!g || !d || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load: null argument");
     return xp_sketch_load_batch(&g, d, 1, out);
+}
+
+extern "C" xp_status xp_sketch_info_get(const xp_sketch* s, xp_sketch_info* out) {
+    if (!s || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_info_get: null argument");
+    memset(out, 0, sizeof(*out));
+    out->n_holes = s->n_holes; out->device = s->arena_device; out->n_points = s->n_points;
+    out->device_bytes = s->arena_bytes; out->load_h2d_bytes = s->load_h2d; out->load_d2h_bytes = s->load_d2h;
+    for (int h = 0; h < s->n_holes && h < 8; ++h) out->n_probes[h] = s->n_probes[h];
+    out->n_refined = s->n_refined;
+    return XP_OK;
+}
+
+// Promotes the points that ended whole-domain checks to probes (see include/xp.h).  The hole
+// records and the tables of noted points are read back; per hole the new probe list is
+// [probe 0, promoted points by how many survivors each ended, the other old probes]; the records
+// go back with the new ids, one small kernel derives coordinates, spec values and context forms
+// of the probes again, and the subtree tables are rebuilt for them.
+extern "C" xp_status xp_sketch_refine(xp_sketch* s, int32_t max_promote, int32_t* n_promoted) {
+    if (n_promoted) *n_promoted = 0;
+    if (!s || max_promote < 0) return fail(XP_ERR_INVALID_ARG, "xp_sketch_refine: bad argument");
+    const xp_sketch* cs = s;
+    xp_status st = check_device(&cs, 1);
+    if (st != XP_OK) return st;
+    const int nh = s->n_holes;
+    const int most = max_promote == 0 ? 4 : max_promote;
+    const size_t kill_bytes = (sizeof(i64) + sizeof(u32)) * kKillSlots;
+    std::vector<HoleDev> hh(nh);
+    std::vector<char> kills(kill_bytes * nh);
+    XP_CUDA(cudaStreamSynchronize(nullptr));
+    XP_CUDA(cudaMemcpy(hh.data(), s->arena + s->off_holes, sizeof(HoleDev) * nh, cudaMemcpyDeviceToHost));
+    for (int h = 0; h < nh; ++h)
+        XP_CUDA(cudaMemcpy(&kills[kill_bytes * h], s->arena + s->off_kill[h], kill_bytes, cudaMemcpyDeviceToHost));
+    int promoted = 0;
+    std::vector<LoadJob> jobs;
+    for (int h = 0; h < nh; ++h) {
+        HoleDev& o = hh[h];
+        const i64* pid = (const i64*)&kills[kill_bytes * h];
+        const u32* cnt = (const u32*)(&kills[kill_bytes * h] + sizeof(i64) * kKillSlots);
+        std::vector<std::pair<u32, i64>> found;          // (survivors ended, point), most frequent first
+        for (int k = 0; k < kKillSlots; ++k)
+            if (pid[k] >= 0 && pid[k] < s->n_points && cnt[k] > 0) found.push_back({cnt[k], pid[k]});
+        std::sort(found.begin(), found.end(), [](const std::pair<u32, i64>& a, const std::pair<u32, i64>& b) {
+            return a.first != b.first ? a.first > b.first : a.second < b.second; });
+        if (found.empty() || o.n_probe < 1) continue;
+        std::vector<i64> ids;
+        ids.push_back(o.probe_id[0]);
+        int taken = 0;
+        for (size_t k = 0; k < found.size() && taken < most && (int)ids.size() < kMaxProbe; ++k) {
+            bool dup = false;
+            for (int j = 0; j < o.n_probe; ++j) dup = dup || o.probe_id[j] == found[k].second;
+            if (!dup) { ids.push_back(found[k].second); ++taken; }
+        }
+        if (taken == 0) continue;
+        for (int j = 1; j < o.n_probe && (int)ids.size() < kMaxProbe; ++j) ids.push_back(o.probe_id[j]);
+        o.n_probe = (i32)ids.size();
+        for (int j = 0; j < o.n_probe; ++j) o.probe_id[j] = ids[j];
+        promoted += taken;
+        LoadJob job;
+        job.s = s->d_s; job.hole = h; job.pad = 0;
+        jobs.push_back(job);
+    }
+    // the notes start afresh whether or not anything was promoted
+    std::vector<char> fresh(kill_bytes, 0);
+    memset(fresh.data(), 0xff, sizeof(i64) * kKillSlots);
+    for (int h = 0; h < nh; ++h) XP_CUDA(cudaMemcpyAsync(s->arena + s->off_kill[h], fresh.data(), kill_bytes, cudaMemcpyHostToDevice, nullptr));
+    if (!jobs.empty()) {
+        char* jobs_dev = nullptr;
+        size_t jobs_bytes = 0;
+        int jobs_device = 0;
+        XP_CUDA(pool_alloc((void**)&jobs_dev, sizeof(LoadJob) * jobs.size(), &jobs_device, &jobs_bytes));
+        cudaError_t e = cudaMemcpyAsync(s->arena + s->off_holes, hh.data(), sizeof(HoleDev) * nh, cudaMemcpyHostToDevice, nullptr);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(jobs_dev, jobs.data(), sizeof(LoadJob) * jobs.size(), cudaMemcpyHostToDevice, nullptr);
+        if (e == cudaSuccess) e = launch_reprobe((const LoadJob*)jobs_dev, (int)jobs.size(), nullptr);
+        for (int k = 1; k <= s->tab_size_cap && e == cudaSuccess; ++k)
+            e = launch_subvalues((const LoadJob*)jobs_dev, (int)jobs.size(), k, s->tab_probes_cap, s->entries_at[k], nullptr);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(hh.data(), s->arena + s->off_holes, sizeof(HoleDev) * nh, cudaMemcpyDeviceToHost, nullptr);
+        const cudaError_t e2 = cudaStreamSynchronize(nullptr);
+        pool_release(jobs_dev, jobs_bytes, jobs_device);
+        if (e != cudaSuccess || e2 != cudaSuccess)
+            return fail(XP_ERR_CUDA, std::string("xp_sketch_refine: ") + cudaGetErrorString(e != cudaSuccess ? e : e2));
+        for (int h = 0; h < nh; ++h) {
+            s->holes[h].filter_ok = hh[h].filter_ok != 0;
+            s->holes[h].compares = hh[h].filter_ok != 0 && hh[h].aff_ok == 0;
+            s->n_probes[h] = hh[h].n_probe;
+        }
+        std::lock_guard<std::mutex> lock(s->plan_mu);
+        s->plan_cached = false;                           // (the plan depends on which holes the filter serves)
+    } else {
+        XP_CUDA(cudaStreamSynchronize(nullptr));
+    }
+    s->n_refined += promoted;
+    if (n_promoted) *n_promoted = promoted;
+    return XP_OK;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -724,12 +866,14 @@ struct HoleResult {
     std::vector<xp_instr> code;
     std::string text;
     u64 evals = 0, filter_survivors = 0, probe_survivors = 0, nominal_ops = 0;
+    u64 filter_tests = 0, skipped = 0;
 };
 
 struct xp_result {
     std::vector<HoleResult> holes;
     double kernel_ms = 0, total_ms = 0;
     int n_launches = 0;
+    u64 h2d_bytes = 0, d2h_bytes = 0;
 };
 
 struct Plan {
@@ -746,7 +890,7 @@ static char* g_ws = nullptr;
 static size_t g_ws_bytes = 0;
 static int g_ws_device = -1;
 
-static const xp_repair_opts kDefaultOpts = {0, 0, 0, nullptr, nullptr, nullptr, 0, 0u, nullptr};
+static const xp_repair_opts kDefaultOpts = {0, 0, 0, nullptr, nullptr, nullptr, 0, 0u, nullptr, 0};
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -829,6 +973,7 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
         if (head.bc_tiles == 1 && head.bc_count * (u64)head.n_ops < kFamilyMaxWork)
             for (size_t j = i + 1; j < plan->segs.size(); ++j) {
                 const SegDev& c = plan->segs[j];
+                if (members == kMaxFamily) break;               // the rest head families of their own
                 if (placed[j - first_seg] || c.bc_tiles != 1 || c.bc_count * (u64)c.n_ops >= kFamilyMaxWork || c.reg_nt != head.reg_nt || c.reg_size != head.reg_size ||
                     c.reg_begin != head.reg_begin || c.reg_count != head.reg_count) continue;
                 placed[j - first_seg] = 1;
@@ -841,7 +986,7 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
         u64 slots = 0;
         bool one_tile = true;
         for (int m = 0; m < members; ++m) { slots += ordered[at + m].bc_count; one_tile = one_tile && ordered[at + m].bc_tiles == 1; }
-        if (one_tile && slots <= (u64)kBcTile && members <= 8) {
+        if (one_tile && slots <= (u64)kBcTile) {
             u64 base = 0;
             for (int m = 0; m < members; ++m) { ordered[at + m].bc_base = (i32)base; base += ordered[at + m].bc_count; }
             ordered[at].bc_keep = 1;
@@ -868,6 +1013,18 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
 constexpr u64 kTileMinRanks = 4096;          // smaller windows are searched rank by rank
 
 static void plan_sketch(const xp_sketch* s, size_t i, const xp_repair_opts* o, Plan* plan);
+
+// A sketch's tables, and the library's scratch, live on the device that was current when the sketch was
+// loaded: a call made with another device current would hand the kernels pointers of the wrong GPU.
+static xp_status check_device(const xp_sketch* const* sk, size_t n) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return fail(XP_ERR_CUDA, "no CUDA device is usable");
+    for (size_t i = 0; i < n; ++i)
+        if (sk[i] && sk[i]->arena_device != dev)
+            return fail(XP_ERR_INVALID_ARG, "sketch " + std::to_string(i) + " was loaded on device " + std::to_string(sk[i]->arena_device) +
+                        ", the current device is " + std::to_string(dev));
+    return XP_OK;
+}
 
 static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
     const bool plain = o->size_min <= 0 && o->size_max <= 0 && o->n_rank_ranges == 0 && o->flags == 0;
@@ -984,6 +1141,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     const auto t0 = std::chrono::steady_clock::now();
     Plan plan;
     xp_status st = build_plan(sketches, n, o, &plan);
+    if (st == XP_OK) st = check_device(sketches, n);
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
@@ -1019,6 +1177,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     float ms = 0.f;
     int launches = 0;
     std::vector<AccDev> acc(plan.acc.size());
+    u32 check_word = 0;
 #define XP_CUDA_R(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { if (own_ws) cudaFree(ws); if (cached_ws) g_ws_mu.unlock(); \
         if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1); \
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)
@@ -1026,17 +1185,40 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     XP_CUDA_R(cudaEventCreate(&e1));
     XP_CUDA_R(cudaMemcpyAsync(ws, stage.data(), w.head, cudaMemcpyHostToDevice, stream));
     XP_CUDA_R(cudaEventRecord(e0, stream));
-    XP_CUDA_R(launch_search(ws, w, plan.n_tickets, (int)plan.segs.size(), (int)n, (int)plan.acc.size(),
-                            max_chunks_of(sketches, n), stream, &launches));
-    XP_CUDA_R(cudaEventRecord(e1, stream));
-    XP_CUDA_R(cudaMemcpyAsync(acc.data(), ws + w.acc, sizeof(AccDev) * acc.size(), cudaMemcpyDeviceToHost, stream));
-    XP_CUDA_R(cudaStreamSynchronize(stream));
-    XP_CUDA_R(cudaEventElapsedTime(&ms, e0, e1));
+    const int n_segs = (int)plan.segs.size(), n_acc = (int)plan.acc.size();
+    const u32 max_chunks = max_chunks_of(sketches, n);
+    xp_status stopped = XP_OK;
+    if (!o->cancel && o->timeout_ms <= 0) {
+        XP_CUDA_R(launch_search_part(ws, w, 0, plan.n_tickets, false, n_segs, (int)n, max_chunks, stream, &launches));
+    } else {
+        // Bounded launches: the host waits for each and then looks at the cancel word and the clock.
+        // Nothing on the device waits for either, and when the call gives up no kernel is in flight.
+        for (u64 t = 0; t < plan.n_tickets && stopped == XP_OK; t += (u64)XP_CANCEL_TICKETS) {
+            const u64 t_end = t + (u64)XP_CANCEL_TICKETS < plan.n_tickets ? t + (u64)XP_CANCEL_TICKETS : plan.n_tickets;
+            XP_CUDA_R(launch_search_part(ws, w, t, t_end, t > 0, n_segs, (int)n, max_chunks, stream, &launches));
+            XP_CUDA_R(cudaStreamSynchronize(stream));
+            if (o->cancel && *o->cancel) stopped = XP_ERR_CANCELLED;
+            else if (o->timeout_ms > 0 && t_end < plan.n_tickets &&
+                     std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count() >= (double)o->timeout_ms)
+                stopped = XP_ERR_TIMEOUT;
+        }
+    }
+    if (stopped == XP_OK) {
+        XP_CUDA_R(launch_search_end(ws, w, plan.n_tickets > 0, n_segs, (int)n, n_acc, max_chunks, stream, &launches));
+        XP_CUDA_R(cudaEventRecord(e1, stream));
+        XP_CUDA_R(cudaMemcpyAsync(acc.data(), ws + w.acc, sizeof(AccDev) * acc.size(), cudaMemcpyDeviceToHost, stream));
+        XP_CUDA_R(cudaMemcpyAsync(&check_word, ws + 20, sizeof(check_word), cudaMemcpyDeviceToHost, stream));
+        XP_CUDA_R(cudaStreamSynchronize(stream));
+        XP_CUDA_R(cudaEventElapsedTime(&ms, e0, e1));
+    }
 #undef XP_CUDA_R
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (own_ws) cudaFree(ws);
     if (cached_ws) g_ws_mu.unlock();
+    if (stopped == XP_ERR_CANCELLED) return fail(stopped, "cancelled between launches (" + std::to_string(launches) + " done)");
+    if (stopped == XP_ERR_TIMEOUT) return fail(stopped, "time limit of " + std::to_string((long long)o->timeout_ms) + " ms reached between launches (" + std::to_string(launches) + " done)");
+    if (check_word != 0) return fail(XP_ERR_CUDA, "an index check of the checked build failed (code " + std::to_string(check_word) + ")");
 
     size_t ai = 0;
     for (size_t i = 0; i < n; ++i) {
@@ -1055,7 +1237,9 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
                 hr.cand_count[k] = s->g->cnt[s->holes[h].start_nt][k];
                 hr.match_count[k] = a.match_count[k];
             }
-            hr.evals = a.evals; hr.filter_survivors = a.filter_survivors; hr.probe_survivors = a.probe_survivors;
+            hr.evals = a.evals + a.filter_tests; hr.filter_survivors = a.filter_survivors; hr.probe_survivors = a.probe_survivors;
+            hr.filter_tests = a.filter_tests;
+            hr.skipped = a.tile_cands > a.filter_tests ? a.tile_cands - a.filter_tests : 0;
             hr.nominal_ops = plan.nominal_ops[ai] - (a.ops_skipped < plan.nominal_ops[ai] ? a.ops_skipped : plan.nominal_ops[ai]);
             const int ls = (int)a.pad;
             if (ls >= 1 && ls <= hr.max_size && a.match_count[ls] > 0) {
@@ -1065,6 +1249,8 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
         }
         r->kernel_ms = ms;
         r->n_launches = launches;
+        r->h2d_bytes = w.head;
+        r->d2h_bytes = sizeof(AccDev) * acc.size() + sizeof(check_word);
         outs[i] = r;
     }
     const double total = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
@@ -1088,6 +1274,7 @@ extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_o
     if (o->cancel && *o->cancel) return fail(XP_ERR_CANCELLED, "cancelled before launch");
     Plan plan;
     xp_status st = build_plan(&sketch, 1, o, &plan);
+    if (st == XP_OK) st = check_device(&sketch, 1);
     if (st != XP_OK) return st;
     const SearchLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size(), kSurvCapStatic);
     if (plan.acc.size() > 64)
@@ -1115,7 +1302,7 @@ extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_o
             r.cand_count[k] = sketch->g->cnt[sketch->holes[h].start_nt][k];
             r.match_count[k] = a.match_count[k];
         }
-        r.evals_executed = a.evals;
+        r.evals_executed = a.evals + a.filter_tests;
         const int ls = (int)a.pad;
         if (ls >= 1 && ls <= r.max_size && a.match_count[ls] > 0) {
             r.solved = 1; r.least_size = ls; r.least_rank = a.min_rank[ls];
@@ -1147,6 +1334,31 @@ extern "C" xp_status xp_result_get(const xp_result* r, int32_t hole, xp_result_v
     v->kernel_ms = r->kernel_ms;
     v->total_ms = r->total_ms;
     v->n_launches = r->n_launches;
+    v->filter_tests = h.filter_tests;
+    v->candidates_skipped = h.skipped;
+    v->h2d_bytes = r->h2d_bytes;
+    v->d2h_bytes = r->d2h_bytes;
+    return XP_OK;
+}
+
+extern "C" xp_status xp_result_pack(const xp_result* const* results, size_t n, xp_hole_summary* out, size_t out_cap, size_t* n_out) {
+    if (n_out) *n_out = 0;
+    if (!results || !out) return fail(XP_ERR_INVALID_ARG, "xp_result_pack: null argument");
+    size_t at = 0;
+    for (size_t i = 0; i < n; ++i) {
+        if (!results[i]) return fail(XP_ERR_INVALID_ARG, "xp_result_pack: result " + std::to_string(i) + " is null");
+        for (const HoleResult& h : results[i]->holes) {
+            if (at >= out_cap) return fail(XP_ERR_INVALID_ARG, "xp_result_pack: out holds fewer entries than the results have holes");
+            xp_hole_summary& r = out[at++];
+            memset(&r, 0, sizeof(r));
+            r.solved = h.solved; r.max_size = h.max_size; r.least_size = h.least_size; r.least_rank = h.least_rank;
+            memcpy(r.cand_count, h.cand_count, sizeof(r.cand_count));
+            memcpy(r.match_count, h.match_count, sizeof(r.match_count));
+            r.evals_executed = h.evals;
+            snprintf(r.least_text, sizeof(r.least_text), "%s", h.text.c_str());
+        }
+    }
+    if (n_out) *n_out = at;
     return XP_OK;
 }
 

@@ -32,6 +32,8 @@ constexpr int kProgMax = 64;          // candidate substituted into its context:
 constexpr u64 kTabBudgetBytes = 64ull << 20;   // subtree-value tables of one hole, all probes together
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
+constexpr int kMaxFamily = 8;         // tile segments that may share one fill of the register-side operands (a hit's
+                                      // queue entry names its member in 3 bits)
 
 // A leaf production: a variable (var >= 0) or a constant.
 struct LeafDev { i32 var; i32 pad; i64 value; };
@@ -104,7 +106,14 @@ struct HoleDev {
     // caller's table).  On a box domain a candidate is checked on the sub-box of these and its
     // own variables only: no other variable can change either side of the constraint.
     u32 fixed_vars, pad2;
+    // Points that ended a survivor's whole-domain check (a candidate that passed every probe and then
+    // failed somewhere): a small open-addressed table of point ids (-1: free) with the number of
+    // survivors each has ended.  Written by verify_kernel, read and cleared by xp_sketch_refine, which
+    // promotes the most frequent ones to probes.  (Counters only: nothing in a search reads them.)
+    i64* kill_pid;                                // device, kKillSlots entries
+    u32* kill_cnt;                                // device, kKillSlots entries
 };
+constexpr int kKillSlots = 64;
 
 struct SketchDev {
     const GrammarDev* g;                          // device
@@ -127,9 +136,13 @@ struct LoadJob { SketchDev* s; i32 hole, pad; };
 struct AccDev {
     u64 match_count[kMaxSize + 1];
     u64 min_rank[kMaxSize + 1];
-    u64 evals, filter_survivors, probe_survivors, pad;
+    u64 evals;                       // exact candidate-point evaluations that ran: stage 2 (probes) and stage 3 (domain points)
+    u64 filter_survivors, probe_survivors, pad;
     u64 ops_skipped;                 // cost-model operations that the filter did not have to carry out (remainders
                                      // of a tile none of whose divisors exceeds the target's magnitude)
+    u64 filter_tests;                // filter-stage tests at probe 0 that ran: (register operand defined there) x
+                                     // (broadcast operand defined there) x (operators whose loop was entered)
+    u64 tile_cands;                  // candidates of the tiles visited, tested or not
 };
 
 // One contiguous piece of work.  kind 0 (linear): ranks [rank_begin, rank_end) of `size`,
@@ -171,6 +184,8 @@ constexpr u32 kSurvFailed = 0x80000000u;
 struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, vars; };   // vars: variables the candidate mentions
 
 struct PlanDev {
+    u64 ticket_base;                 // tickets [ticket_base, n_tickets) belong to this launch (a search that polls a
+                                     // cancel word is cut into several launches); the counter starts at zero each time
     u64 n_tickets;
     i32 n_segs, n_sketches;
     const SegDev* segs;              // device
@@ -182,6 +197,7 @@ struct PlanDev {
     u64* verify_ticket;              // device counter, zero at launch
     u32 surv_cap;
     u32 max_chunks;                  // chunks of the largest domain among the sketches
+    u32* err;                        // device word for the checked build's index checks (0: none failed)
 };
 
 }  // namespace xp

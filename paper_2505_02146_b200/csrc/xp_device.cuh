@@ -6,6 +6,23 @@
 
 namespace xp {
 
+// Index checks of the checked build (-DXP_CHECKS; the stand-in for a memory checker on tiny
+// cases): XP_CHECKED(cond, code) is `true` and costs nothing in the normal build; in the checked
+// build a false condition is recorded (the first code wins) and the caller takes a safe value
+// instead of the bad index.  Nothing traps, spins or faults: the search finishes, and the host
+// turns a recorded code into an error status.
+#ifdef XP_CHECKS
+__device__ unsigned int g_check_word;
+__device__ __forceinline__ bool xp_checked(bool cond, unsigned int code) {
+    if (!cond) atomicCAS(&g_check_word, 0u, code);
+    return cond;
+}
+#define XP_CHECKED(cond, code) xp_checked((cond), (code))
+#else
+#define XP_CHECKED(cond, code) true
+#endif
+enum { kChkRank = 1, kChkTable = 2, kChkQueue = 3, kChkStack = 4, kChkPoint = 5, kChkSlot = 6, kChkSegment = 7 };
+
 // One binary operation in int64 C semantics with wrap-around.  Returns false when the
 // divisor is zero (the candidate is then invalid at this point).  INT64_MIN / -1 wraps to
 // INT64_MIN and INT64_MIN % -1 is 0; the trapping machine division is never issued.
@@ -49,6 +66,7 @@ __device__ __noinline__ int unrank(const GrammarDev* __restrict__ g, int nt, int
     struct Frame { u64 rank; i32 nt; i32 size; };
     Frame st[kMaxSize + 1];
     int sp = 0, n = 0;
+    if (!XP_CHECKED(size >= 1 && size <= kMaxSize && rank < g->cnt[nt][size], kChkRank)) { rank = 0; size = 1; }
     st[sp++] = Frame{rank, nt, size};
     while (sp > 0) {
         const Frame f = st[--sp];
@@ -81,6 +99,7 @@ __device__ __noinline__ int unrank(const GrammarDev* __restrict__ g, int nt, int
 // the tree of (nt, size >= 3) with the given rank.
 __device__ __forceinline__ void unrank_root(const GrammarDev* __restrict__ g, int nt, int size, u64 rank,
                                             int& op, int& lnt, int& rnt, int& a, u64& l, u64& r) {
+    if (!XP_CHECKED(size >= 3 && rank < g->cnt[nt][size], kChkRank)) rank = 0;
     int p = g->bin_begin[nt];
     const int pe = g->bin_begin[nt + 1];
     while (p + 1 < pe && g->bins[p + 1].off[size] <= rank) ++p;
@@ -112,6 +131,7 @@ __device__ __forceinline__ bool eval_cand(const u32* code, int n, const LeafDev*
             st[sp - 1] = r;
         } else {
             const LeafDev lf = leaves[w];
+            if (!XP_CHECKED(sp < kCandStack, kChkStack)) return false;
             st[sp++] = lf.var >= 0 ? pt[lf.var] : lf.value;
         }
     }
@@ -132,6 +152,7 @@ __device__ __forceinline__ bool eval_code(const xp_instr* code, int n, const i64
             if (!apply_op(c.arg, a, b, r)) return false;
             st[sp - 1] = r;
         } else {
+            if (!XP_CHECKED(sp < kMaxStack, kChkStack)) return false;
             st[sp++] = c.kind == XP_I_VAR ? pt[c.arg] : (c.kind == XP_I_CONST ? c.value : hole);
         }
     }
@@ -143,6 +164,7 @@ __device__ __forceinline__ bool eval_code(const xp_instr* code, int n, const i64
 // the box (first variable slowest).
 __device__ __forceinline__ void point_coords(const SketchDev* __restrict__ s, i64 pid, i64* pt) {
     const int nv = s->n_vars;
+    if (!XP_CHECKED(pid >= 0 && pid < s->n_points, kChkPoint)) pid = 0;
     if (s->coords != nullptr) {
         const i32* row = s->coords + pid * nv;
         for (int d = 0; d < nv; ++d) pt[d] = row[d];

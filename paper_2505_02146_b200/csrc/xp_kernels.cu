@@ -119,6 +119,48 @@ __device__ bool ctx_interval(const HoleDev* hole, const i64* pt, i64 spec, i64& 
     return false;
 }
 
+// The context at every probe (affine in the hole, or a comparison; one thread per probe), and what
+// the rest of the load and the searches go by.  Called by every thread of the CTA once the n
+// probes (ids, coordinates, spec values) are in place; ncand / pass0: how many sampled candidates
+// the probe choice looked at and how many of them satisfied the first probe.
+__device__ __forceinline__ void probe_contexts(HoleDev* hole, int n, int ncand, int pass0) {
+    const int t = threadIdx.x;
+    if (t < kMaxProbe) {
+        u64 A = 0, B = 0;
+        const bool aff = t < n && ctx_affine(hole, hole->probe_pt[t], A, B);
+        i64 lo = 1, hi = 0;
+        const bool rng = t < n && !aff && ((hole->probe_spec_ok >> t) & 1u) &&
+                         ctx_interval(hole, hole->probe_pt[t], hole->probe_spec[t], lo, hi);
+        hole->aff_Aj[t] = aff ? A : 0;
+        hole->aff_Bj[t] = aff ? B : 0;
+        hole->rng_lo[t] = lo;
+        hole->rng_hi[t] = hi;
+        const u32 amask = __ballot_sync(0x0000ffffu, aff), rmask = __ballot_sync(0x0000ffffu, rng);
+        if (t == 0) {
+            hole->aff_ok = aff ? 1 : 0;
+            hole->aff_A = aff ? A : 0;
+            hole->aff_B = aff ? B : 0;
+            hole->aff_okmask = amask;
+            hole->rng_okmask = rmask;
+            // what the rest of the load and the searches go by
+            const u32 spec_ok = hole->probe_spec_ok;
+            const bool filter_ok = n > 0 && (aff || (rmask & spec_ok & 1u));
+            hole->filter_ok = filter_ok ? 1 : 0;
+            int probes = 0;
+            if (filter_ok && hole->tab_size_cap > 0 && hole->tab_total > 0) probes = n < hole->tab_probes_cap ? n : hole->tab_probes_cap;
+            hole->tab_probes = probes;
+            hole->tab_max_size = probes > 0 ? hole->tab_size_cap : 0;
+            // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
+            // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
+            // probe 0 alone lets many through.
+            const bool possible = n >= 2 && probes >= 2 && ((spec_ok & (amask | rmask)) >> 1 & 1u);
+            const bool frequent = ncand > 0 && (u64)pass0 * 256 >= (u64)ncand;
+            hole->second = possible && (hole->small_search || frequent) ? 1 : 0;
+            hole->second_ok = possible ? 1 : 0;
+        }
+    }
+}
+
 // Choice of each hole's probe points, once per sketch (one CTA per hole).  Threads evaluate the sample
 // points; then a sample of small candidates (sizes 1, 3, 5, ranks spread evenly) is run on
 // every sample point, giving each a bit set of the samples where it satisfies the constraint.
@@ -238,41 +280,31 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
         hole->sample_n = ncand;
     }
     __syncthreads();
-    // the context at every probe: affine in the hole, or a comparison (one thread per probe)
-    if (t < kMaxProbe) {
-        u64 A = 0, B = 0;
-        const bool aff = t < n && ctx_affine(hole, hole->probe_pt[t], A, B);
-        i64 lo = 1, hi = 0;
-        const bool rng = t < n && !aff && ((hole->probe_spec_ok >> t) & 1u) &&
-                         ctx_interval(hole, hole->probe_pt[t], hole->probe_spec[t], lo, hi);
-        hole->aff_Aj[t] = aff ? A : 0;
-        hole->aff_Bj[t] = aff ? B : 0;
-        hole->rng_lo[t] = lo;
-        hole->rng_hi[t] = hi;
-        const u32 amask = __ballot_sync(0x0000ffffu, aff), rmask = __ballot_sync(0x0000ffffu, rng);
-        if (t == 0) {
-            hole->aff_ok = aff ? 1 : 0;
-            hole->aff_A = aff ? A : 0;
-            hole->aff_B = aff ? B : 0;
-            hole->aff_okmask = amask;
-            hole->rng_okmask = rmask;
-            // what the rest of the load and the searches go by
-            const u32 spec_ok = hole->probe_spec_ok;
-            const bool filter_ok = n > 0 && (aff || (rmask & spec_ok & 1u));
-            hole->filter_ok = filter_ok ? 1 : 0;
-            int probes = 0;
-            if (filter_ok && hole->tab_size_cap > 0 && hole->tab_total > 0) probes = n < hole->tab_probes_cap ? n : hole->tab_probes_cap;
-            hole->tab_probes = probes;
-            hole->tab_max_size = probes > 0 ? hole->tab_size_cap : 0;
-            // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
-            // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
-            // probe 0 alone lets many through.
-            const bool possible = n >= 2 && probes >= 2 && ((spec_ok & (amask | rmask)) >> 1 & 1u);
-            const bool frequent = ncand > 0 && (u64)pass0 * 256 >= (u64)ncand;
-            hole->second = possible && (hole->small_search || frequent) ? 1 : 0;
-            hole->second_ok = possible ? 1 : 0;
-        }
+    probe_contexts(hole, n, ncand, pass0);
+}
+
+// The probes of a hole replaced by the host (xp_sketch_refine: points that ended whole-domain
+// checks are promoted): hole->probe_id[0 .. n_probe) is given; coordinates, spec values and the
+// context forms are derived again, as prepare_kernel does for the probes it picks.  One warp per hole.
+__global__ void __launch_bounds__(32) reprobe_kernel(const LoadJob* jobs) {
+    SketchDev* s = jobs[blockIdx.x].s;
+    HoleDev* hole = &s->holes[jobs[blockIdx.x].hole];
+    const int t = threadIdx.x, n = hole->n_probe;
+    bool ok = false;
+    if (t < n) {
+        i64 pt[kMaxVars];
+        point_coords(s, hole->probe_id[t], pt);
+        for (int d = 0; d < s->n_vars; ++d) hole->probe_pt[t][d] = pt[d];
+        i64 v = 0;
+        ok = true;
+        if (hole->spec_table != nullptr) v = hole->spec_table[hole->probe_id[t]];
+        else ok = eval_code(hole->spec, hole->spec_len, pt, 0, v);
+        hole->probe_spec[t] = v;
     }
+    const u32 okmask = __ballot_sync(0xffffffffu, ok);
+    if (t == 0) hole->probe_spec_ok = okmask;
+    __syncthreads();
+    probe_contexts(hole, n, hole->sample_n, hole->sample_pass0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -321,7 +353,6 @@ struct CandShared {
     i64 cval[kMaxSize];
 };
 
-constexpr int kMaxFamily = 8;
 struct MemberState {
     u64 bc_first; i32 lo, hi; u32 n, nspecial; i32 wide;
     i32 mod_possible;            // some operand of the member, as a divisor, exceeds the target's magnitude: only
@@ -338,6 +369,7 @@ struct EvalShared {
     u64 match_count[kMaxSize + 1];
     u64 min_rank[kMaxSize + 1];
     u64 filter_survivors, probe_survivors, ops_skipped;
+    u64 filter_tests, tile_cands;
     u64 warp_evals[kThreads / 32];
     // tile tickets: the broadcast-side operands at probe 0 (entries invalid there are dropped) with
     // what the loops need of each, and the warps' queues of filter hits
@@ -387,11 +419,13 @@ __device__ __noinline__ void flush_acc(EvalShared& sh, const PlanDev& plan, u64&
             if (sh.filter_survivors) atomicAdd(&acc->filter_survivors, sh.filter_survivors);
             if (sh.probe_survivors) atomicAdd(&acc->probe_survivors, sh.probe_survivors);
             if (sh.ops_skipped) atomicAdd(&acc->ops_skipped, sh.ops_skipped);
+            if (sh.filter_tests) atomicAdd(&acc->filter_tests, sh.filter_tests);
+            if (sh.tile_cands) atomicAdd(&acc->tile_cands, sh.tile_cands);
         }
     }
     __syncthreads();
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; }
+    if (threadIdx.x == 0) { sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; sh.filter_tests = 0; sh.tile_cands = 0; }
     my_evals = 0;
     __syncthreads();
 }
@@ -569,20 +603,27 @@ __device__ __forceinline__ i64 proj_pid(const CandShared& c, i64 q) {
 // Fast form: points and spec values come from tables in HBM (the caller's, or staged at load)
 // and the program runs on a register stack.  Otherwise coordinates are derived from the point
 // id and the interpreters with a stack in local memory are used.
+// On failure *fail_pid is the domain point id of one point that failed (the same for all lanes).
 template <int D>
 __device__ __forceinline__ bool check_points_fast(const CandShared& c, const SketchDev* sk, const HoleDev* hole,
-                                                  i64 first, i64 last, u64& evals) {
+                                                  i64 first, i64 last, u64& evals, i64* fail_pid) {
     const int nv = sk->n_vars;
     const int lane = threadIdx.x & 31;
     for (i64 base = first; base < last; base += 32) {
         bool bad = false;
         if (base + lane < last) {
-            const i64 pid = c.n_proj_vars ? proj_pid(c, base + lane) : base + lane;
+            i64 pid = c.n_proj_vars ? proj_pid(c, base + lane) : base + lane;
+            if (!XP_CHECKED(pid >= 0 && pid < sk->n_points, kChkPoint)) pid = 0;
             ++evals;
             i64 v;
             bad = !run_program<D>(c, sk->coords + pid * nv, v) || v != hole->spec_table[pid];
         }
-        if (__any_sync(0xffffffffu, bad)) return false;
+        const u32 bm = __ballot_sync(0xffffffffu, bad);
+        if (bm) {
+            const i64 q = base + (__ffs((int)bm) - 1);
+            *fail_pid = c.n_proj_vars ? proj_pid(c, q) : q;
+            return false;
+        }
     }
     return true;
 }
@@ -597,7 +638,7 @@ __device__ __forceinline__ bool check_points_fast(const CandShared& c, const Ske
 constexpr int kVecDepth = 8;                              // deepest operand stack this form takes
 template <typename T, int P>
 __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __restrict__ stack, const SketchDev* sk,
-                                                 const HoleDev* hole, i64 first, i64 last) {
+                                                 const HoleDev* hole, i64 first, i64 last, i64* fail_pid) {
     static_assert(sizeof(T) * P == sizeof(uint4), "one stack level of a lane is one 16-byte slot");
     const int nv = sk->n_vars;
     const int lane = threadIdx.x & 31;
@@ -615,6 +656,7 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
             in[i] = pid < last;
             i64 at = in[i] ? pid : first;                 // lanes past the end repeat a valid point
             if (c.n_proj_vars) at = proj_pid(c, at);      // (uniform branch)
+            if (!XP_CHECKED(at >= 0 && at < sk->n_points, kChkPoint)) at = 0;
             row[i] = coords + at * nv;
             want[i] = spec[at];
         }
@@ -694,18 +736,27 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
         }
         // a zero divisor at a repeated point is a zero divisor at a real point of this candidate
         // too (the repeated point is `first`, which lane 0 holds in range), so `bad` needs no mask
+        u32 which = bad ? 1u : 0u;                        // bit i: this lane's point i failed (a zero divisor: point 0)
 #pragma unroll
-        for (int i = 0; i < P; ++i) bad |= in[i] && (i64)t.v[i] != want[i];
-        if (__any_sync(0xffffffffu, bad)) return false;
+        for (int i = 0; i < P; ++i) which |= (u32)(in[i] && (i64)t.v[i] != want[i]) << i;
+        const u32 bm = __ballot_sync(0xffffffffu, which != 0u);
+        if (bm) {
+            const int src = __ffs((int)bm) - 1;
+            const u32 w = __shfl_sync(0xffffffffu, which, src);
+            const i64 q = base + (i64)(__ffs((int)w) - 1) * 32 + src;
+            const i64 qq = q < last ? q : first;
+            *fail_pid = c.n_proj_vars ? proj_pid(c, qq) : qq;
+            return false;
+        }
     }
     return true;
 }
 
 __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* sk, const HoleDev* hole, i64 first,
-                                          i64 last, u64& evals) {
+                                          i64 last, u64& evals, i64* fail_pid) {
     if (sk->coords != nullptr && hole->spec_table != nullptr && c.depth >= 1) {
-        if (c.depth <= 4) return check_points_fast<4>(c, sk, hole, first, last, evals);
-        if (c.depth <= 8) return check_points_fast<8>(c, sk, hole, first, last, evals);
+        if (c.depth <= 4) return check_points_fast<4>(c, sk, hole, first, last, evals, fail_pid);
+        if (c.depth <= 8) return check_points_fast<8>(c, sk, hole, first, last, evals, fail_pid);
     }
     const int n = c.cand_len;
     const int lane = threadIdx.x & 31;
@@ -734,7 +785,12 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
             }
             bad = !ok || !ctx_matches(hole, pt, st[0], want);
         }
-        if (__any_sync(0xffffffffu, bad)) return false;
+        const u32 bm = __ballot_sync(0xffffffffu, bad);
+        if (bm) {
+            const i64 q = base + (__ffs((int)bm) - 1);
+            *fail_pid = c.n_proj_vars ? proj_pid(c, q) : q;
+            return false;
+        }
     }
     return true;
 }
@@ -742,6 +798,9 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
 // A candidate that passed the probes goes into the global queue for the verification kernel.
 // Returns false if the queue is full: the caller's warp then checks the candidate itself.
 __device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank, u32 vars) {
+    // (the counter saturates: once the queue is full nothing is added, so it cannot wrap around
+    // and hand out a slot twice however many survivors a search has)
+    if (*(volatile const u32*)plan.surv_n >= plan.surv_cap) return false;
     const u32 at = atomicAdd(plan.surv_n, 1u);
     if (at >= plan.surv_cap) return false;
     SurvDev r;
@@ -758,7 +817,8 @@ __device__ __noinline__ void warp_verify(EvalShared& sh, const SketchDev* sk, co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (lane == 0) stage_candidate(sh.wcand[warp], sk, hole, size, rank);
     __syncwarp();
-    const bool ok = check_points(sh.wcand[warp], sk, hole, 0, sk->n_points, my_evals);
+    i64 fail_pid = 0;
+    const bool ok = check_points(sh.wcand[warp], sk, hole, 0, sk->n_points, my_evals, &fail_pid);
     if (ok && lane == 0) {
         atomicAdd(&sh.match_count[size], 1ull);
         atomicMin(&sh.min_rank[size], rank);
@@ -849,7 +909,8 @@ __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* h
     const int tmax = hole->tab_max_size;
     const u64 pbase = (u64)pr * hole->tab_total;
     if (size <= tmax) {
-        const u64 at = pbase + hole->tab_off[nt][size] + rank;
+        u64 at = pbase + hole->tab_off[nt][size] + rank;
+        if (!XP_CHECKED(pr < hole->tab_probes && hole->tab_off[nt][size] + rank < hole->tab_total && rank < g->cnt[nt][size], kChkTable)) at = 0;
         v = hole->tab_val[at];
         return hole->tab_ok[at] != 0;
     }
@@ -1396,10 +1457,13 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
             const SegDev& seg = sh.mseg[(e >> 24) & 7u];
             const u32 opi = (e >> 21) & 7u;
             const u64 rr = reg_first + (e & 2047u);
-            const u64 br = sh.mb[(e >> 24) & 7u].bc_first + (sh.bc_meta[(e >> 11) & 1023u].meta & 0xffffu);
+            const u32 q_slot = XP_CHECKED(((e >> 11) & 1023u) < (u32)kBcTile && opi < (u32)seg.n_ops, kChkQueue) ? (e >> 11) & 1023u : 0u;
+            const u64 br = sh.mb[(e >> 24) & 7u].bc_first + (sh.bc_meta[q_slot].meta & 0xffffu);
             const u64 l = seg.swap ? br : rr, r = seg.swap ? rr : br;
             rank = seg.op_base[opi] + l * seg.right_count + r;
             bool dead = rank < seg.rank_begin || rank >= seg.rank_end;
+            if (!XP_CHECKED(rr < g->cnt[seg.reg_nt][seg.reg_size] && br < g->cnt[seg.bc_nt][seg.bc_size] &&
+                            rank < g->cnt[hole->start_nt][seg.size], kChkQueue)) dead = true;
             for (int j = 0; j < n_tab && !dead; ++j) {
                 ++my_evals;
                 i64 rv, bv, v;
@@ -1489,6 +1553,18 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     // target's magnitude no candidate  a % b  can match, and the loops leave the remainders out.
     const bool skip_mod = !SWAP && (mask & 16u) && !mbs.mod_possible && !tile_wide && !rng && A == 1u && t_small;
     if (skip_mod && threadIdx.x == 0) sh.ops_skipped += pairs * ((mask & 8u) ? 2ull : 9ull);     // (cost model of the host plan)
+    // Tests of this member that run: this thread's operands that are defined at the probe, times the
+    // member's broadcast operands that are, times the operators whose loop is entered (the 32-bit
+    // loops leave / and % out when the target cannot be a quotient or remainder of int32 operands, and
+    // the remainders alone when no divisor exceeds the target).
+    {
+        int tested_ops = seg.n_ops;
+        if (!tile_wide && !rng && (mask & 24u) && A == 1u) {
+            if (!t_small) tested_ops -= __popc(mask & 24u);
+            else if (skip_mod) tested_ops -= 1;
+        }
+        warp_tally(&sh.filter_tests, (u32)__popc(alive) * (u32)(nb + (int)mbs.nspecial) * (u32)tested_ops);
+    }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
     auto run = [&](int s0, int s1, u32 alv, bool special) {
@@ -1593,6 +1669,7 @@ __device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDe
         const u32 slot = special ? (u32)mbs.hi - 1u - atomicAdd(&mbs.nspecial, 1u) : (u32)mbs.lo + atomicAdd(&mbs.n, 1u);
         const bool fits = v > -(1ll << 31) && v < (1ll << 31);
         wide |= !fits;
+        if (!XP_CHECKED(slot < (u32)kBcTile && (i32)slot >= mbs.lo && (i32)slot < mbs.hi, kChkSlot)) continue;
         const u32 b = (u32)(u64)v, ub = abs_u32((i32)v);
         const u32 k = ub ? (u32)__ffs((int)ub) - 1u : 0u;
         const u32 io = ub ? inv_odd(ub >> k) : 1u;          // inverse of the odd part of |v|
@@ -1647,7 +1724,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     if (!(hole->probe_spec_ok & 1u)) return;            // spec undefined at probe 0: nothing can match
     // the register side: the same for every member of the segment's family
     int family = sh.seg.family > 1 ? sh.seg.family : 1;
-    if (family > kMaxFamily) family = kMaxFamily;        // (the host builds none larger)
+    if (family > kMaxFamily) family = kMaxFamily;        // (the host's plan builder stops at kMaxFamily members)
     const int seg_index = sh.seg_index;
     const u64 reg_tile = local / sh.seg.bc_tiles, bc_tile0 = local % sh.seg.bc_tiles;
     const u64 reg_first = sh.seg.reg_begin + reg_tile * (u64)kRegTile;
@@ -1719,7 +1796,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             const SegDev& seg = sh.mseg[m];
             if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
-            if (threadIdx.x == 0) my_evals += pairs * (u64)seg.n_ops;
+            if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
             if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
             else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
         }
@@ -1734,7 +1811,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         __syncthreads();
         const SegDev& seg = sh.mseg[m];
         const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
-        if (threadIdx.x == 0) my_evals += pairs * (u64)seg.n_ops;
+        if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
         if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
         else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
     }
@@ -1747,14 +1824,14 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
-    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; }
+    if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; sh.filter_tests = 0; sh.tile_cands = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) {
-            sh.ticket = atomicAdd(plan.ticket, 1ull);
+            sh.ticket = plan.ticket_base + atomicAdd(plan.ticket, 1ull);
             // many filter hits so far for the hole at hand (this CTA's own counts): second look from now on
-            if (!sh.adapt_second && sh.filter_survivors * kAdaptRate > my_evals) sh.adapt_second = 1;
+            if (!sh.adapt_second && sh.filter_survivors * kAdaptRate > sh.tile_cands) sh.adapt_second = 1;
         }
         __syncthreads();
         const u64 t = sh.ticket;
@@ -1772,6 +1849,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
                 n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
                 lo = nlo;
             }
+            if (!XP_CHECKED(lo >= 0 && lo < plan.n_segs && plan.segs[lo].first_ticket <= t, kChkSegment)) lo = 0;
             if (threadIdx.x == 0) sh.seg_index = lo;
             load_segment(sh, plan, lo);
         }
@@ -1794,6 +1872,17 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
 // ------------------------------------------------------------------------------------------
 // verify: whole-domain check of the queued survivors
 // ------------------------------------------------------------------------------------------
+
+// Notes, for xp_sketch_refine, that domain point `pid` ended a survivor's whole-domain check.
+__device__ __noinline__ void record_killer(const HoleDev* hole, i64 pid) {
+    if (hole->kill_pid == nullptr) return;
+    u64 x = (u64)pid * 0x9E3779B97F4A7C15ull;
+    u32 slot = (u32)(x >> 40) % (u32)kKillSlots;
+    for (int k = 0; k < 8; ++k, slot = (slot + 1u) % (u32)kKillSlots) {
+        const u64 old = atomicCAS((u64*)&hole->kill_pid[slot], ~0ull, (u64)pid);
+        if (old == ~0ull || old == (u64)pid) { atomicAdd(&hole->kill_cnt[slot], 1u); return; }
+    }                                                   // (table crowded around this slot: the point goes unrecorded)
+}
 
 // Items are (chunk of points, survivor), chunk-major: the first chunk of every survivor is
 // taken before any second chunk, so candidates that fail early cost one chunk.  Each WARP
@@ -1844,16 +1933,18 @@ __global__ void __launch_bounds__(kThreads, 3) verify_kernel(const PlanDev plan)
         const i64 first = (i64)(t / n) * kVerifyChunk;
         const i64 last = first + kVerifyChunk < np ? first + kVerifyChunk : np;
         u64 evals = 0;
+        i64 fail_pid = 0;
         bool ok;
         if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
             uint4* stack = stacks[threadIdx.x >> 5];
-            ok = cand.narrow ? check_points_vec<i32, 4>(cand, stack, sk, hole, first, last)
-                             : check_points_vec<i64, 2>(cand, stack, sk, hole, first, last);
+            ok = cand.narrow ? check_points_vec<i32, 4>(cand, stack, sk, hole, first, last, &fail_pid)
+                             : check_points_vec<i64, 2>(cand, stack, sk, hole, first, last, &fail_pid);
         } else {
-            ok = check_points(cand, sk, hole, first, last, evals);
+            ok = check_points(cand, sk, hole, first, last, evals, &fail_pid);
         }
         if (lane == 0) {
-            if (ok) atomicAdd(&sv->state, 1u); else atomicOr(&sv->state, kSurvFailed);
+            if (ok) atomicAdd(&sv->state, 1u);
+            else if (!(atomicOr(&sv->state, kSurvFailed) & kSurvFailed)) record_killer(hole, fail_pid);   // (once per survivor)
             atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
         }
         __syncwarp();                                   // the staged candidate is free for the next item
@@ -1881,9 +1972,14 @@ __global__ void count_kernel(const PlanDev plan) {
 // ------------------------------------------------------------------------------------------
 
 // One warp per accumulator: lane = size; ballot finds the smallest size with a match.
-__global__ void finish_kernel(AccDev* acc, int n_acc) {
+__global__ void finish_kernel(AccDev* acc, int n_acc, u32* err) {
     const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
+#ifdef XP_CHECKS
+    if (blockIdx.x == 0 && threadIdx.x == 0) *err = atomicExch(&g_check_word, 0u);     // what the checks recorded, if anything
+#else
+    (void)err;
+#endif
     if (w >= n_acc) return;
     AccDev* a = &acc[w];
     const bool has = lane <= kMaxSize && a->match_count[lane] > 0;
@@ -1937,6 +2033,12 @@ cudaError_t launch_prepare(const LoadJob* jobs, int n_jobs, cudaStream_t stream)
     return cudaGetLastError();
 }
 
+cudaError_t launch_reprobe(const LoadJob* jobs, int n_jobs, cudaStream_t stream) {
+    if (n_jobs <= 0) return cudaSuccess;
+    reprobe_kernel<<<n_jobs, 32, 0, stream>>>(jobs);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_coord_bounds(SketchDev* const* list, int n_sketches, i64 most_points, cudaStream_t stream) {
     if (most_points <= 0 || n_sketches <= 0) return cudaSuccess;
     const i64 blocks = (most_points + 255) / 256;
@@ -1968,37 +2070,67 @@ static int resident_ctas(const void* kernel) {
     return sms * per_sm;
 }
 
-cudaError_t launch_search(char* base, const SearchLayout& L, u64 n_tickets, int n_segs, int n_sketches, int n_acc,
-                          u32 max_chunks, cudaStream_t stream, int* n_launches) {
+static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sketches, u32 max_chunks) {
     PlanDev pd;
-    pd.n_tickets = n_tickets;
+    pd.ticket_base = 0;
+    pd.n_tickets = 0;
     pd.n_segs = n_segs;
     pd.n_sketches = n_sketches;
     pd.ticket = (u64*)base;
     pd.verify_ticket = (u64*)(base + 8);
     pd.surv_n = (u32*)(base + 16);
+    pd.err = (u32*)(base + 20);
     pd.segs = (const SegDev*)(base + L.segs);
     pd.sketches = (const SketchDev* const*)(base + L.sketches);
     pd.acc = (AccDev*)(base + L.acc);
     pd.surv = (SurvDev*)(base + L.surv);
     pd.surv_cap = L.surv_cap;
     pd.max_chunks = max_chunks;
+    return pd;
+}
+
+// Stages 1 and 2 for the tickets [t_begin, t_end) of the plan staged at `base`.  A search is one
+// such launch, or several in a row when the host wants to look at a cancel word or a clock in
+// between; `restart` says that the ticket counter has to be set back to zero first (every launch
+// but the first, whose counter the staged copy has just zeroed).
+cudaError_t launch_search_part(char* base, const SearchLayout& L, u64 t_begin, u64 t_end, bool restart, int n_segs,
+                               int n_sketches, u32 max_chunks, cudaStream_t stream, int* n_launches) {
+    if (t_end <= t_begin) return cudaSuccess;
     cudaError_t e;
-    if (n_tickets > 0) {
-        u64 ctas = (u64)resident_ctas((const void*)eval_kernel);      // persistent CTAs: one wave
-        if (ctas > n_tickets) ctas = n_tickets;
-        eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (restart && (e = cudaMemsetAsync(base, 0, 8, stream)) != cudaSuccess) return e;
+    PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
+    pd.ticket_base = t_begin;
+    pd.n_tickets = t_end;
+    u64 ctas = (u64)resident_ctas((const void*)eval_kernel);      // persistent CTAs: one wave
+    if (ctas > t_end - t_begin) ctas = t_end - t_begin;
+    eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
+    *n_launches += 1;
+    return cudaGetLastError();
+}
+
+// Stage 3 and the reductions, after every part of the search has been queued.
+cudaError_t launch_search_end(char* base, const SearchLayout& L, bool any_tickets, int n_segs, int n_sketches, int n_acc,
+                              u32 max_chunks, cudaStream_t stream, int* n_launches) {
+    PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
+    cudaError_t e;
+    if (any_tickets) {
         verify_kernel<<<resident_ctas((const void*)verify_kernel), kThreads, 0, stream>>>(pd);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         count_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        *n_launches += 3;
+        *n_launches += 2;
     }
     const int warps_per_block = 8;
-    finish_kernel<<<(n_acc + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, stream>>>(pd.acc, n_acc);
+    finish_kernel<<<(n_acc + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, stream>>>(pd.acc, n_acc, pd.err);
     *n_launches += 1;
     return cudaGetLastError();
+}
+
+cudaError_t launch_search(char* base, const SearchLayout& L, u64 n_tickets, int n_segs, int n_sketches, int n_acc,
+                          u32 max_chunks, cudaStream_t stream, int* n_launches) {
+    cudaError_t e = launch_search_part(base, L, 0, n_tickets, false, n_segs, n_sketches, max_chunks, stream, n_launches);
+    if (e != cudaSuccess) return e;
+    return launch_search_end(base, L, n_tickets > 0, n_segs, n_sketches, n_acc, max_chunks, stream, n_launches);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -8,17 +8,24 @@
 namespace xp {
 
 cudaError_t launch_prepare(const LoadJob* jobs, int n_jobs, cudaStream_t stream);
+cudaError_t launch_reprobe(const LoadJob* jobs, int n_jobs, cudaStream_t stream);
 cudaError_t launch_coord_bounds(SketchDev* const* list, int n_sketches, i64 most_points, cudaStream_t stream);
 cudaError_t launch_stage_points(const SketchDev* s, i64 n_points, i32* coords, cudaStream_t stream);
 cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, i64* spec, u32* bad, cudaStream_t stream);
 cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most_probes, u64 most_entries, cudaStream_t stream);
 // Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
-//   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32)   -- zero at launch
+//   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32), 20: failed-check word (u32; checked
+//      build only)   -- zero at launch
 //   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
 //   surv: the survivor queue (surv_cap entries), written by the kernels only
 struct SearchLayout { size_t segs, sketches, acc, head, surv, total; u32 surv_cap; };
 
-// The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel.
+// The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel;
+// or the same in pieces: eval_kernel over one range of tickets at a time, then the rest.
+cudaError_t launch_search_part(char* base, const SearchLayout& L, u64 t_begin, u64 t_end, bool restart, int n_segs,
+                               int n_sketches, u32 max_chunks, cudaStream_t stream, int* n_launches);
+cudaError_t launch_search_end(char* base, const SearchLayout& L, bool any_tickets, int n_segs, int n_sketches, int n_acc,
+                              u32 max_chunks, cudaStream_t stream, int* n_launches);
 cudaError_t launch_search(char* base, const SearchLayout& L, u64 n_tickets, int n_segs, int n_sketches, int n_acc,
                           u32 max_chunks, cudaStream_t stream, int* n_launches);
 constexpr size_t kStaticScratchBytes = 1u << 20;     // fixed scratch of the allocation-free entry point

@@ -63,11 +63,17 @@ def test_other_seeds_full(xp, name, make, seed):
     _check_large(xp, name, make, seed)
 
 
-def test_config5_full_batch(xp):
-    rows = [[int(x) for x in line.split()] for line in open(os.path.join(GOLDEN, "config5_seed0_full.txt"))
+def _config5_seeds():
+    return [int(f[len("config5_seed"):-len("_full.txt")]) for f in sorted(os.listdir(GOLDEN))
+            if f.startswith("config5_seed") and f.endswith("_full.txt")]
+
+
+@pytest.mark.parametrize("seed", _config5_seeds())
+def test_config5_full_batch(xp, seed):
+    rows = [[int(x) for x in line.split()] for line in open(os.path.join(GOLDEN, f"config5_seed{seed}_full.txt"))
             if not line.startswith("#")]
     assert len(rows) == 4096
-    sks = config5(0, 4096)
+    sks = config5(seed, 4096)
     grs = {}
     for sk in sks:
         key = tuple(v.hi for v in sk.grammar.variables)

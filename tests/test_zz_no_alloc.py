@@ -49,6 +49,26 @@ def test_static_entry_point_matches_xp_repair_on_two_calls_in_a_row(xp):
         _same(xp.xp_repair_static(lb)[0], rb[0])
 
 
+def test_static_entry_point_leaves_device_memory_as_it_found_it(xp):
+    """The property the entry point is named for: once a first call on the device has been made,
+    further calls, on different sketches and with different options, neither take nor give back
+    device memory (free memory as the driver reports it stays the same to the byte)."""
+    import torch
+    sketches = []
+    for sk in (config1(0), config1(4), config5_instance(0, 2), config3(0)):
+        sketches.append(xp.xp_sketch_load(xp.xp_grammar_create(sk.grammar), sk))      # (loading does allocate)
+    xp.xp_repair_static(sketches[0])                                                   # first call: address look-up
+    torch.cuda.synchronize()
+    free0, total0 = torch.cuda.mem_get_info()
+    for ls in sketches:
+        xp.xp_repair_static(ls)
+        xp.xp_repair_static(ls, flags=xp.XP_FLAG_NO_FILTER, size_max=3)
+        xp.xp_repair_static(ls, rank_ranges=[(-1, 5, 0, 100_000)])
+        assert torch.cuda.mem_get_info() == (free0, total0)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info() == (free0, total0)
+
+
 def test_static_entry_point_when_its_survivor_queue_is_full(xp):
     """The fixed array holds a survivor queue of 8192 entries; a spec with 60 878 matches of size 5
     overflows it, and the warps then check their survivors themselves: same counts."""
