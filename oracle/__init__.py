@@ -63,6 +63,21 @@ class _Result(C.Structure):
                 ("evals", C.c_uint64), ("least_text", C.c_char * 1024)]
 
 
+class _JointProblem(C.Structure):
+    _fields_ = [("g", _Grammar), ("n_points", C.c_int64), ("coords", C.POINTER(C.c_int32)),
+                ("start_nt", C.c_int32 * 2), ("max_size", C.c_int32 * 2),
+                ("ctx_len", C.c_int32), ("ctx", C.POINTER(_Instr)),
+                ("spec_len", C.c_int32), ("spec_expr", C.POINTER(_Instr)),
+                ("spec_table", C.POINTER(C.c_int64))]
+
+
+class _JointResult(C.Structure):
+    _fields_ = [("cand_count", C.c_uint64 * (2 * XO_MAX_SIZE + 1)), ("match_count", C.c_uint64 * (2 * XO_MAX_SIZE + 1)),
+                ("solved", C.c_int32), ("least_total", C.c_int32), ("least_size0", C.c_int32), ("pad", C.c_int32),
+                ("least_rank0", C.c_uint64), ("least_rank1", C.c_uint64), ("evals", C.c_uint64),
+                ("least_text0", C.c_char * 512), ("least_text1", C.c_char * 512)]
+
+
 _lib = None
 
 
@@ -78,6 +93,8 @@ def _load():
         lib.xo_eval_code.argtypes = [C.POINTER(_Instr), C.c_int, C.POINTER(C.c_int64), C.c_int64, C.POINTER(C.c_int64)]
         lib.xo_repair.restype = C.c_int
         lib.xo_repair.argtypes = [C.POINTER(_Problem), C.POINTER(_Result)]
+        lib.xo_repair_joint.restype = C.c_int
+        lib.xo_repair_joint.argtypes = [C.POINTER(_JointProblem), C.POINTER(_JointResult)]
         _lib = lib
     return _lib
 
@@ -193,3 +210,51 @@ def repair_hole(sk: Sketch, hole_index: int = 0, rank_ranges: Optional[dict] = N
     K = h.max_size
     return OracleResult([int(x) for x in R.cand_count[:K + 1]], [int(x) for x in R.match_count[:K + 1]],
                         bool(R.solved), int(R.least_size), int(R.least_rank), R.least_text.decode(), int(R.evals))
+
+
+@dataclass
+class JointResult:
+    cand_count: List[int]          # index = total size of the pair
+    match_count: List[int]
+    solved: bool
+    least_total: int
+    least_size0: int
+    least_rank0: int
+    least_rank1: int
+    least_text0: str
+    least_text1: str
+    evals: int
+
+
+def repair_joint(sk: Sketch, joint) -> JointResult:
+    """The repair search for two holes inside one constraint (``joint``: a ``JointHole``) over the
+    domain and grammar of ``sk``: every pair of trees, by total size, then size of part 0, then
+    rank of part 0, then rank of part 1."""
+    gc = _GrammarC(sk.grammar)
+    P = _JointProblem()
+    P.g = gc.c
+    P.n_points = sk.n_points
+    keep = []
+    if sk.coords is not None:
+        co = np.ascontiguousarray(sk.coords, dtype=np.int32)
+        keep.append(co)
+        P.coords = co.ctypes.data_as(C.POINTER(C.c_int32))
+    P.start_nt[0], P.start_nt[1] = joint.start_nt
+    P.max_size[0], P.max_size[1] = joint.max_size
+    ctx = _code(joint.ctx); keep.append(ctx)
+    P.ctx_len, P.ctx = len(joint.ctx), ctx
+    if joint.spec_table is not None:
+        st = np.ascontiguousarray(joint.spec_table, dtype=np.int64)
+        assert st.shape[0] == sk.n_points
+        keep.append(st)
+        P.spec_table = st.ctypes.data_as(C.POINTER(C.c_int64))
+    else:
+        se = _code(joint.spec_expr); keep.append(se)
+        P.spec_len, P.spec_expr = len(joint.spec_expr), se
+    R = _JointResult()
+    if _load().xo_repair_joint(C.byref(P), C.byref(R)):
+        raise ValueError("oracle rejected the joint problem")
+    K = joint.max_size[0] + joint.max_size[1]
+    return JointResult([int(x) for x in R.cand_count[:K + 1]], [int(x) for x in R.match_count[:K + 1]], bool(R.solved),
+                       int(R.least_total), int(R.least_size0), int(R.least_rank0), int(R.least_rank1),
+                       R.least_text0.decode(), R.least_text1.decode(), int(R.evals))

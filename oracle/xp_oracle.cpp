@@ -31,7 +31,13 @@
 //   * comparison and logic operators (context / spec only) yield 0 or 1 and
 //     evaluate both operands;
 //   * a grammar may also use min and max as binary operators (printed min(a,b)):
-//     the remainder-tile bounds of a split loop need them.
+//     the remainder-tile bounds of a split loop need them;
+//   * and the shifts << and >> (strength-reduced index arithmetic): the count must lie in
+//     0..63, anything else makes the candidate fail at that point like a zero divisor;
+//     << wraps, >> keeps the sign;
+//   * a joint sketch has two holes inside ONE constraint (xo_repair_joint): the candidates
+//     are the pairs of trees, ordered by total size, then the size of the first tree, then
+//     its rank, then the second tree's rank; counts are per total size.
 //
 // Parity against the paper itself is unpinned: it prints no instance, query or
 // solution for this step (its constraint figure is not available).  The functions
@@ -49,7 +55,7 @@ typedef uint64_t u64;
 typedef int64_t i64;
 
 enum { XO_MAX_SIZE = 15 };
-enum { OP_ADD = 0, OP_SUB, OP_MUL, OP_DIV, OP_MOD, OP_LT, OP_LE, OP_EQ, OP_NE, OP_MIN, OP_MAX, OP_AND, OP_OR, OP_COUNT };
+enum { OP_ADD = 0, OP_SUB, OP_MUL, OP_DIV, OP_MOD, OP_LT, OP_LE, OP_EQ, OP_NE, OP_MIN, OP_MAX, OP_AND, OP_OR, OP_SHL, OP_SHR, OP_COUNT };
 enum { K_VAR = 0, K_CONST = 1, K_HOLE = 2, K_OP = 3 };
 enum { P_VAR = 0, P_CONST = 1, P_BIN = 2 };
 
@@ -91,6 +97,26 @@ struct xo_result {
     char least_text[1024];
 };
 
+// Two holes in one constraint.  HOLE instructions of ctx carry the part (0 or 1) in arg.
+struct xo_joint_problem {
+    xo_grammar g;
+    i64 n_points;
+    const int32_t* coords;
+    int32_t start_nt[2], max_size[2];
+    int32_t ctx_len;  const xo_instr* ctx;         // must mention both parts
+    int32_t spec_len; const xo_instr* spec_expr;
+    const i64* spec_table;
+};
+
+struct xo_joint_result {
+    u64 cand_count[2 * XO_MAX_SIZE + 1];           // index = total size
+    u64 match_count[2 * XO_MAX_SIZE + 1];
+    int32_t solved, least_total, least_size0, pad;
+    u64 least_rank0, least_rank1;
+    u64 evals;
+    char least_text0[512], least_text1[512];
+};
+
 }  // extern "C"
 
 namespace {
@@ -118,21 +144,30 @@ bool apply_op(int op, i64 a, i64 b, i64& out) {
         case OP_MAX: out = a > b ? a : b; return true;
         case OP_AND: out = (a != 0) && (b != 0); return true;
         case OP_OR: out = (a != 0) || (b != 0); return true;
+        case OP_SHL:
+            if (b < 0 || b > 63) return false;
+            out = (i64)((u64)a << b);
+            return true;
+        case OP_SHR:
+            if (b < 0 || b > 63) return false;
+            out = a < 0 ? ~(~a >> b) : a >> b;           // sign-propagating, written without relying on the compiler's choice
+            return true;
     }
     return false;
 }
 
-const char* const OP_TEXT[OP_COUNT] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
+const char* const OP_TEXT[OP_COUNT] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||", "<<", ">>"};
 
-// Postfix evaluation of a context or spec expression at one point.
-bool eval_code(const xo_instr* code, int n, const i64* pt, i64 hole, i64& out) {
+// Postfix evaluation of a context or spec expression at one point.  `holes`: the value of the
+// hole (a joint sketch: of its parts; a HOLE instruction's arg says which).
+bool eval_code(const xo_instr* code, int n, const i64* pt, const i64* holes, i64& out) {
     i64 st[64];
     int sp = 0;
     for (int i = 0; i < n; ++i) {
         const xo_instr& c = code[i];
         if (c.kind == K_VAR) st[sp++] = pt[c.arg];
         else if (c.kind == K_CONST) st[sp++] = c.value;
-        else if (c.kind == K_HOLE) st[sp++] = hole;
+        else if (c.kind == K_HOLE) st[sp++] = holes[c.arg];
         else {
             i64 b = st[--sp], a = st[--sp], r;
             if (!apply_op(c.arg, a, b, r)) return false;
@@ -255,7 +290,7 @@ i64 xo_list(const xo_grammar* g, int nt, int size, u64 begin, u64 end, char* buf
 
 // Value of a postfix expression at one point (returns 0 when a divisor is zero).
 int xo_eval_code(const xo_instr* code, int n, const i64* pt, i64 hole, i64* out) {
-    return eval_code(code, n, pt, hole, *out) ? 1 : 0;
+    return eval_code(code, n, pt, &hole, *out) ? 1 : 0;
 }
 
 // The repair search for one hole.  Returns 0, or 1 on a malformed problem.
@@ -286,7 +321,7 @@ int xo_repair(const xo_problem* P, xo_result* R) {
     std::vector<char> spec_ok(np, 1);
     for (i64 p = 0; p < np; ++p) {
         if (P->spec_table) spec[p] = P->spec_table[p];
-        else spec_ok[p] = eval_code(P->spec_expr, P->spec_len, &pts[p * nv], 0, spec[p]);
+        else { const i64 none = 0; spec_ok[p] = eval_code(P->spec_expr, P->spec_len, &pts[p * nv], &none, spec[p]); }
     }
     // Order in which points are tried: the caller's "first" points, then all of them.
     std::vector<i64> order;
@@ -312,7 +347,7 @@ int xo_repair(const xo_problem* P, xo_result* R) {
                 ok = spec_ok[p] && eval_tree(root, pt, h);
                 if (ok) {
                     if (P->ctx_len == 0) v = h;
-                    else ok = eval_code(P->ctx, P->ctx_len, pt, h, v);
+                    else ok = eval_code(P->ctx, P->ctx_len, pt, &h, v);
                 }
                 ok = ok && v == spec[p];
                 if (!ok) break;
@@ -327,6 +362,78 @@ int xo_repair(const xo_problem* P, xo_result* R) {
             }
             ++rank;
         });
+    }
+    return 0;
+}
+
+// The repair search for a joint sketch: every pair (tree of part 0, tree of part 1), by total
+// size, then size of part 0, then rank of part 0, then rank of part 1.  Returns 0, or 1 on a
+// malformed problem.
+int xo_repair_joint(const xo_joint_problem* P, xo_joint_result* R) {
+    memset(R, 0, sizeof(*R));
+    const xo_grammar* g = &P->g;
+    const int K0 = P->max_size[0], K1 = P->max_size[1];
+    if (K0 < 1 || K0 > XO_MAX_SIZE || K1 < 1 || K1 > XO_MAX_SIZE || g->n_vars > 16 || P->ctx_len < 1) return 1;
+    Gram G(g, K0 > K1 ? K0 : K1);
+    if (G.overflow) return 1;
+    const int nv = g->n_vars;
+    const i64 np = P->n_points;
+    std::vector<i64> pts((size_t)np * (nv ? nv : 1));
+    for (i64 p = 0; p < np; ++p) {
+        if (P->coords) for (int d = 0; d < nv; ++d) pts[p * nv + d] = P->coords[p * nv + d];
+        else {
+            i64 rem = p;
+            for (int d = nv - 1; d >= 0; --d) {
+                const i64 ext = g->hi[d] - g->lo[d];
+                pts[p * nv + d] = g->lo[d] + rem % ext;
+                rem /= ext;
+            }
+        }
+    }
+    std::vector<i64> spec(np);
+    std::vector<char> spec_ok(np, 1);
+    const i64 none[2] = {0, 0};
+    for (i64 p = 0; p < np; ++p) {
+        if (P->spec_table) spec[p] = P->spec_table[p];
+        else spec_ok[p] = eval_code(P->spec_expr, P->spec_len, &pts[p * nv], none, spec[p]);
+    }
+    for (int s = 2; s <= K0 + K1; ++s) {
+        for (int s0 = 1; s0 < s; ++s0) {
+            const int s1 = s - s0;
+            if (s0 > K0 || s1 > K1) continue;
+            const u64 c0 = G.cnt[P->start_nt[0]][s0], c1 = G.cnt[P->start_nt[1]][s1];
+            const unsigned __int128 prod = (unsigned __int128)c0 * c1;
+            if ((prod >> 63) || R->cand_count[s] + (u64)prod < R->cand_count[s]) return 1;
+            R->cand_count[s] += (u64)prod;
+            Node* t0 = nullptr;
+            u64 r0 = 0;
+            gen(G, P->start_nt[0], s0, 0, c0, t0, [&]() {
+                Node* t1 = nullptr;
+                u64 r1 = 0;
+                gen(G, P->start_nt[1], s1, 0, c1, t1, [&]() {
+                    bool ok = true;
+                    for (i64 p = 0; p < np && ok; ++p) {
+                        ++R->evals;
+                        const i64* pt = &pts[p * nv];
+                        i64 h[2], v;
+                        const bool d0 = eval_tree(t0, pt, h[0]);
+                        const bool d1 = eval_tree(t1, pt, h[1]);
+                        ok = spec_ok[p] && d0 && d1 && eval_code(P->ctx, P->ctx_len, pt, h, v) && v == spec[p];
+                    }
+                    if (ok) {
+                        ++R->match_count[s];
+                        if (!R->solved) {
+                            R->solved = 1; R->least_total = s; R->least_size0 = s0; R->least_rank0 = r0; R->least_rank1 = r1;
+                            std::string a, b; tree_text(g, t0, a); tree_text(g, t1, b);
+                            snprintf(R->least_text0, sizeof(R->least_text0), "%s", a.c_str());
+                            snprintf(R->least_text1, sizeof(R->least_text1), "%s", b.c_str());
+                        }
+                    }
+                    ++r1;
+                });
+                ++r0;
+            });
+        }
     }
     return 0;
 }

@@ -881,6 +881,8 @@ struct Plan {
     std::vector<AccDev> acc;
     std::vector<u64> nominal_ops;    // per accumulator: cost-model operations of the filter stage
     u64 n_tickets = 0;
+    std::vector<u64> groups;         // first ticket of every group of tickets, and the end (empty: no grouping)
+    u64 n_items() const { return groups.empty() ? n_tickets : (u64)groups.size() - 1; }
 };
 
 // Scratch of calls that bring no workspace: one block per process, reused while no other call
@@ -1026,6 +1028,35 @@ static xp_status check_device(const xp_sketch* const* sk, size_t n) {
     return XP_OK;
 }
 
+// Plans over many holes (batches of small sketches) hand the CTAs runs of consecutive tickets of one
+// hole instead of single tickets: a CTA that stays with a hole flushes its private results once and
+// fills the hole's broadcast operands once.  A run never crosses into another hole and is at most
+// as long as leaves about eight runs per resident CTA (load balance).  Plans over few holes (large
+// searches) keep single tickets: their tickets are long, and a run of them would unbalance the end.
+constexpr size_t kGroupMinAccs = 256;
+constexpr u64 kGroupCtas = 148 * 3;
+static void group_tickets(Plan* plan) {
+    plan->groups.clear();
+#ifdef XP_NO_GROUPS
+    return;
+#endif
+    if (plan->acc.size() < kGroupMinAccs || plan->n_tickets == 0) return;
+    u64 most = plan->n_tickets / (kGroupCtas * 8);
+    most = most < 1 ? 1 : (most > 64 ? 64 : most);
+    if (most == 1) return;
+    int cur_acc = -1;
+    u64 cur_len = 0;
+    for (size_t i = 0; i < plan->segs.size(); ++i) {
+        const SegDev& c = plan->segs[i];
+        const u64 end = i + 1 < plan->segs.size() ? plan->segs[i + 1].first_ticket : plan->n_tickets;
+        for (u64 t = c.first_ticket; t < end; ++t) {
+            if (c.acc != cur_acc || cur_len == most) { plan->groups.push_back(t); cur_acc = c.acc; cur_len = 0; }
+            ++cur_len;
+        }
+    }
+    plan->groups.push_back(plan->n_tickets);
+}
+
 static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
     const bool plain = o->size_min <= 0 && o->size_max <= 0 && o->n_rank_ranges == 0 && o->flags == 0;
     if (n > 16) { plan->segs.reserve(n * 8); plan->acc.reserve(n * 2); plan->nominal_ops.reserve(n * 2); }
@@ -1059,6 +1090,7 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
         }
         plan->n_tickets += s->plan_tickets;
     }
+    group_tickets(plan);
     return XP_OK;
 }
 
@@ -1105,14 +1137,20 @@ static u32 surv_cap_for(size_t n_sketches) {
 }
 constexpr u32 kSurvCapStatic = 8192;         // ... of a call on the library's fixed scratch
 
-static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap) {
+static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap, size_t n_group_entries = 0) {
     SearchLayout w;
     w.segs = 256;
     w.sketches = w.segs + align256(sizeof(SegDev) * (n_segs + 1));
     w.acc = w.sketches + align256(sizeof(SketchDev*) * (n_sketches + 1));
-    w.head = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
+    w.groups = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
+    w.n_groups = n_group_entries ? n_group_entries - 1 : 0;
+    w.hist = w.groups + align256(sizeof(u64) * n_group_entries);
+    w.head = w.hist + align256(sizeof(u32) * (n_acc + 1));
     w.surv = w.head;
-    w.total = w.surv + align256(sizeof(SurvDev) * (size_t)surv_cap);
+    w.sort_off = w.surv + align256(sizeof(SurvDev) * (size_t)surv_cap);
+    w.sorted = w.sort_off + align256(sizeof(u32) * (n_acc + 2));
+    w.total = w.sorted + align256(sizeof(u32) * (size_t)surv_cap);
+    w.n_acc = (int)n_acc;
     w.surv_cap = surv_cap;
     return w;
 }
@@ -1128,7 +1166,7 @@ extern "C" size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n,
     if (!sketches || n == 0) return 0;
     Plan plan;
     if (build_plan(sketches, n, opts ? opts : &kDefaultOpts, &plan) != XP_OK) return 0;
-    return ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n)).total;
+    return ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n), plan.groups.size()).total;
 }
 
 extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
@@ -1145,7 +1183,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
-    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
+    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n), plan.groups.size());
     char* ws = (char*)o->workspace;
     bool own_ws = false, cached_ws = false;
     if (ws) {
@@ -1172,6 +1210,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
     for (size_t i = 0; i < n; ++i) ((const SketchDev**)&stage[w.sketches])[i] = sketches[i]->d_s;
     memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
+    if (!plan.groups.empty()) memcpy(&stage[w.groups], plan.groups.data(), sizeof(u64) * plan.groups.size());
 
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     float ms = 0.f;
@@ -1189,16 +1228,17 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     const u32 max_chunks = max_chunks_of(sketches, n);
     xp_status stopped = XP_OK;
     if (!o->cancel && o->timeout_ms <= 0) {
-        XP_CUDA_R(launch_search_part(ws, w, 0, plan.n_tickets, false, n_segs, (int)n, max_chunks, stream, &launches));
+        XP_CUDA_R(launch_search_part(ws, w, 0, plan.n_items(), false, n_segs, (int)n, max_chunks, stream, &launches));
     } else {
         // Bounded launches: the host waits for each and then looks at the cancel word and the clock.
         // Nothing on the device waits for either, and when the call gives up no kernel is in flight.
-        for (u64 t = 0; t < plan.n_tickets && stopped == XP_OK; t += (u64)XP_CANCEL_TICKETS) {
-            const u64 t_end = t + (u64)XP_CANCEL_TICKETS < plan.n_tickets ? t + (u64)XP_CANCEL_TICKETS : plan.n_tickets;
+        const u64 n_items = plan.n_items();               // (an item is a ticket, or a short run of them)
+        for (u64 t = 0; t < n_items && stopped == XP_OK; t += (u64)XP_CANCEL_TICKETS) {
+            const u64 t_end = t + (u64)XP_CANCEL_TICKETS < n_items ? t + (u64)XP_CANCEL_TICKETS : n_items;
             XP_CUDA_R(launch_search_part(ws, w, t, t_end, t > 0, n_segs, (int)n, max_chunks, stream, &launches));
             XP_CUDA_R(cudaStreamSynchronize(stream));
             if (o->cancel && *o->cancel) stopped = XP_ERR_CANCELLED;
-            else if (o->timeout_ms > 0 && t_end < plan.n_tickets &&
+            else if (o->timeout_ms > 0 && t_end < n_items &&
                      std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count() >= (double)o->timeout_ms)
                 stopped = XP_ERR_TIMEOUT;
         }

@@ -184,9 +184,14 @@ constexpr u32 kSurvFailed = 0x80000000u;
 struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, vars; };   // vars: variables the candidate mentions
 
 struct PlanDev {
-    u64 ticket_base;                 // tickets [ticket_base, n_tickets) belong to this launch (a search that polls a
-                                     // cancel word is cut into several launches); the counter starts at zero each time
-    u64 n_tickets;
+    // What a CTA takes from the counter is a WORK ITEM: one ticket, or (group_first != null) the run of
+    // consecutive tickets [group_first[i], group_first[i+1]) of one hole.  Plans of many small sketches
+    // are grouped, so that a CTA stays with a hole for several tickets (one flush of its private
+    // results, operands filled once) instead of meeting a new hole at every ticket.
+    u64 item_base;                   // items [item_base, n_items) belong to this launch (a search that polls a cancel
+                                     // word is cut into several launches); the counter starts at zero each time
+    u64 n_items;
+    const u64* group_first;          // device, n_items + 1 entries, or null: item i is ticket i
     i32 n_segs, n_sketches;
     const SegDev* segs;              // device
     const SketchDev* const* sketches;  // device table of device pointers
@@ -198,6 +203,13 @@ struct PlanDev {
     u32 surv_cap;
     u32 max_chunks;                  // chunks of the largest domain among the sketches
     u32* err;                        // device word for the checked build's index checks (0: none failed)
+    // Survivors in hole order (null when the call has one hole): queued survivors per accumulator slot
+    // (counted by eval_kernel), the slots' offsets (a scan of the counts) and, per slot side by side, the
+    // queue indices of its survivors (a scatter).  The verification kernel walks surv_sorted.
+    i32 n_acc;
+    u32* surv_hist;                  // device, n_acc, zero at launch
+    u32* surv_off;                   // device, n_acc + 1
+    u32* surv_sorted;                // device, surv_cap
 };
 
 }  // namespace xp

@@ -360,7 +360,7 @@ struct MemberState {
 };
 
 struct EvalShared {
-    u64 ticket;
+    u64 item;
     i32 seg_index;
     SegDev seg;
     CandShared wcand[kWarps];    // per warp: the candidate of a whole-domain check the warp does itself
@@ -395,6 +395,12 @@ struct EvalShared {
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
     u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21 | member << 24
+    // The register-side operands of the ticket at hand, one column per thread ([j][thread]; a thread
+    // reads and writes only its own column, so nothing synchronises on them): low and high words of
+    // the values at probe 0, and the values at probe 1 (second look).  The loops copy their column
+    // into registers when they start; keeping the columns here rather than in per-thread local
+    // memory keeps them out of the L1 cache, which the frames of all resident threads overflow.
+    u32 rv[kNA][kThreads], rh[kNA][kThreads], r1[kNA][kThreads];
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
@@ -636,6 +642,64 @@ __device__ __forceinline__ bool check_points_fast(const CandShared& c, const Ske
 // int32 (CandShared::narrow), else T = i64 with P = 2.  The program is the same for all
 // lanes, so the dispatch branches are uniform.  Points and spec values come from the tables.
 constexpr int kVecDepth = 8;                              // deepest operand stack this form takes
+template <typename T, int P> union VecSlot { uint4 q; T v[P]; };
+
+// One operator of a staged program on P points at once.  Binary: t = a op t.  The folded constant
+// divisions (int32 programs only; kval = the constant and floor(2^32 / |constant|)) work on t alone.
+// `bad` collects zero divisors.
+template <typename T, int P>
+__device__ __forceinline__ void vec_op(int op, i64 kval, const VecSlot<T, P>& a, VecSlot<T, P>& t, bool& bad) {
+    if (sizeof(T) == 4 && op >= kOpDivC) {                // x / c or x % c, c != 0 a constant
+        const i32 d = (i32)(u32)(u64)kval;
+        const u32 M = (u32)((u64)kval >> 32), ad = d < 0 ? 0u - (u32)d : (u32)d;
+#pragma unroll
+        for (int i = 0; i < P; ++i) {
+            const i32 x = (i32)t.v[i];
+            const u32 ux = x < 0 ? 0u - (u32)x : (u32)x;      // |x| < 2^31: the estimate is the quotient or one less
+            u32 q = __umulhi(ux, M), r = ux - q * ad;
+            if (r >= ad) { ++q; r -= ad; }
+            t.v[i] = (T)(op == kOpDivC ? (((x < 0) != (d < 0)) ? (i32)(0u - q) : (i32)q) : (x < 0 ? (i32)(0u - r) : (i32)r));
+        }
+        return;
+    }
+    if (sizeof(T) == 8) {
+#pragma unroll
+        for (int i = 0; i < P; ++i) {
+            i64 r = 0;
+            bad |= !apply_op(op, (i64)a.v[i], (i64)t.v[i], r);
+            t.v[i] = (T)r;
+        }
+        return;
+    }
+    switch (op) {                                         // int32: no result can overflow (proved at staging)
+#define XP_EACH(expr) _Pragma("unroll") for (int i = 0; i < P; ++i) { const i32 x = (i32)a.v[i], y = (i32)t.v[i]; t.v[i] = (T)(expr); } break;
+        case XP_OP_ADD: XP_EACH(x + y)
+        case XP_OP_SUB: XP_EACH(x - y)
+        case XP_OP_MUL: XP_EACH(x * y)
+        case XP_OP_DIV:
+        case XP_OP_MOD:
+#pragma unroll
+            for (int i = 0; i < P; ++i) {
+                const i32 x = (i32)a.v[i], y = (i32)t.v[i];
+                bad |= y == 0;
+                const i32 d = y == 0 ? 1 : y;             // |x| < 2^31, so x / -1 does not overflow
+                const i32 q = x / d;
+                t.v[i] = (T)(op == XP_OP_DIV ? q : x - q * d);
+            }
+            break;
+        case XP_OP_LT: XP_EACH(x < y)
+        case XP_OP_LE: XP_EACH(x <= y)
+        case XP_OP_EQ: XP_EACH(x == y)
+        case XP_OP_NE: XP_EACH(x != y)
+        case XP_OP_MIN: XP_EACH(x < y ? x : y)
+        case XP_OP_MAX: XP_EACH(x > y ? x : y)
+        case XP_OP_AND: XP_EACH((x != 0) & (y != 0))
+        case XP_OP_OR: XP_EACH((x != 0) | (y != 0))
+#undef XP_EACH
+        default: bad = true; break;
+    }
+}
+
 template <typename T, int P>
 __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __restrict__ stack, const SketchDev* sk,
                                                  const HoleDev* hole, i64 first, i64 last, i64* fail_pid) {
@@ -645,7 +709,7 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
     const int n = c.len;
     const i32* __restrict__ coords = sk->coords;
     const i64* __restrict__ spec = hole->spec_table;
-    union Slot { uint4 q; T v[P]; };
+    typedef VecSlot<T, P> Slot;
     for (i64 base = first; base < last; base += 32 * P) {
         const i32* row[P];
         i64 want[P];
@@ -681,58 +745,10 @@ __device__ __forceinline__ bool check_points_vec(const CandShared& c, uint4* __r
                 continue;
             }
             const int op = -2 - cv;
-            if (sizeof(T) == 4 && op >= kOpDivC) {          // x / c or x % c on the top of the stack, c != 0 a constant
-                const i32 d = (i32)(u32)(u64)c.val[k];
-                const u32 M = (u32)((u64)c.val[k] >> 32), ad = d < 0 ? 0u - (u32)d : (u32)d;
-#pragma unroll
-                for (int i = 0; i < P; ++i) {
-                    const i32 x = (i32)t.v[i];
-                    const u32 ux = x < 0 ? 0u - (u32)x : (u32)x;      // |x| < 2^31: the estimate is the quotient or one less
-                    u32 q = __umulhi(ux, M), r = ux - q * ad;
-                    if (r >= ad) { ++q; r -= ad; }
-                    t.v[i] = (T)(op == kOpDivC ? (((x < 0) != (d < 0)) ? (i32)(0u - q) : (i32)q) : (x < 0 ? (i32)(0u - r) : (i32)r));
-                }
-                continue;
-            }
-            --below;
             Slot a;
-            a.q = stack[below * 32 + lane];
-            if (sizeof(T) == 8) {
-#pragma unroll
-                for (int i = 0; i < P; ++i) {
-                    i64 r = 0;
-                    bad |= !apply_op(op, (i64)a.v[i], (i64)t.v[i], r);
-                    t.v[i] = (T)r;
-                }
-                continue;
-            }
-            switch (op) {                                 // int32: no result can overflow (proved at staging)
-#define XP_EACH(expr) _Pragma("unroll") for (int i = 0; i < P; ++i) { const i32 x = (i32)a.v[i], y = (i32)t.v[i]; t.v[i] = (T)(expr); } break;
-                case XP_OP_ADD: XP_EACH(x + y)
-                case XP_OP_SUB: XP_EACH(x - y)
-                case XP_OP_MUL: XP_EACH(x * y)
-                case XP_OP_DIV:
-                case XP_OP_MOD:
-#pragma unroll
-                    for (int i = 0; i < P; ++i) {
-                        const i32 x = (i32)a.v[i], y = (i32)t.v[i];
-                        bad |= y == 0;
-                        const i32 d = y == 0 ? 1 : y;     // |x| < 2^31, so x / -1 does not overflow
-                        const i32 q = x / d;
-                        t.v[i] = (T)(op == XP_OP_DIV ? q : x - q * d);
-                    }
-                    break;
-                case XP_OP_LT: XP_EACH(x < y)
-                case XP_OP_LE: XP_EACH(x <= y)
-                case XP_OP_EQ: XP_EACH(x == y)
-                case XP_OP_NE: XP_EACH(x != y)
-                case XP_OP_MIN: XP_EACH(x < y ? x : y)
-                case XP_OP_MAX: XP_EACH(x > y ? x : y)
-                case XP_OP_AND: XP_EACH((x != 0) & (y != 0))
-                case XP_OP_OR: XP_EACH((x != 0) | (y != 0))
-#undef XP_EACH
-                default: bad = true; break;
-            }
+            a.q = t.q;
+            if (!(sizeof(T) == 4 && op >= kOpDivC)) { --below; a.q = stack[below * 32 + lane]; }
+            vec_op<T, P>(op, c.val[k], a, t, bad);
         }
         // a zero divisor at a repeated point is a zero divisor at a real point of this candidate
         // too (the repeated point is `first`, which lane 0 holds in range), so `bad` needs no mask
@@ -807,6 +823,7 @@ __device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& pla
     r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
     r.state = 0; r.vars = vars;
     plan.surv[at] = r;
+    if (plan.surv_hist) atomicAdd(&plan.surv_hist[r.acc], 1u);       // (for the hole order the verification walks)
     return true;
 }
 
@@ -949,24 +966,32 @@ __device__ __noinline__ u32 operand_vars(const GrammarDev* g, const HoleDev* hol
     return 0xffu;
 }
 
-// Values at probe `pr` of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`;
-// returns the mask of those that are defined there and sets `wide` if one does not fit int32.
+// Values at probe `pr` of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`, written
+// to the calling thread's column (lo[j * kThreads], and hi[...] for the high words unless hi is
+// null); returns the mask of those that are defined there and, in `fits`, of those that fit int32.
 // A subtree above the table sizes whose operands are in the tables is unranked one level for
 // the first rank only; the following ranks advance the operand ranks like an odometer (right
 // operand fastest), so the left operand's value is fetched once per run.
 __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev* hole, int pr, int nt, int size, u64 rank,
-                                              int n, i64* out, bool& wide) {
+                                              int n, u32* lo, u32* hi, u32& fits) {
     u32 alive = 0;
+    fits = 0;
     const int tmax = hole->tab_max_size;
     const u64 pbase = (u64)pr * hole->tab_total;
-    for (int j = 0; j < kNA; ++j) out[j] = 0;
+    for (int j = 0; j < kNA; ++j) { lo[j * kThreads] = 0; if (hi) hi[j * kThreads] = 0; }
     if (n <= 0) return 0;
+    auto put = [&](int j, i64 v) {
+        lo[j * kThreads] = (u32)(u64)v;
+        if (hi) hi[j * kThreads] = (u32)((u64)v >> 32);
+        alive |= 1u << j;
+        if (v > -(1ll << 31) && v < (1ll << 31)) fits |= 1u << j;
+    };
+    int j = 0;
     if (size > tmax && tmax >= 1 && size >= 3) {
         int op, lnt, rnt, a;
         u64 l, r;
         unrank_root(g, nt, size, rank, op, lnt, rnt, a, l, r);
         bool tables = a <= tmax && size - 1 - a <= tmax;
-        int j = 0;
         while (tables && j < n) {
             const u64 cl = g->cnt[lnt][a], cr = g->cnt[rnt][size - 1 - a];
             const u64 lbase = pbase + hole->tab_off[lnt][a], rbase = pbase + hole->tab_off[rnt][size - 1 - a];
@@ -975,11 +1000,7 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
                 const i64 lv = hole->tab_val[lbase + l];
                 for (; j < n && r < cr; ++r, ++j) {
                     i64 v;
-                    if (lok && hole->tab_ok[rbase + r] && apply_op(op, lv, hole->tab_val[rbase + r], v)) {
-                        out[j] = v;
-                        alive |= 1u << j;
-                        wide |= !(v > -(1ll << 31) && v < (1ll << 31));
-                    }
+                    if (lok && hole->tab_ok[rbase + r] && apply_op(op, lv, hole->tab_val[rbase + r], v)) put(j, v);
                 }
                 if (j == n) break;
             }
@@ -988,22 +1009,10 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
                 tables = a <= tmax && size - 1 - a <= tmax;
             }
         }
-        if (j == n) return alive;
-        for (; j < n; ++j) {
-            i64 v;
-            if (operand_value(g, hole, pr, nt, size, rank + j, v)) {
-                out[j] = v; alive |= 1u << j;
-                wide |= !(v > -(1ll << 31) && v < (1ll << 31));
-            }
-        }
-        return alive;
     }
-    for (int j = 0; j < n; ++j) {
+    for (; j < n; ++j) {
         i64 v;
-        if (operand_value(g, hole, pr, nt, size, rank + j, v)) {
-            out[j] = v; alive |= 1u << j;
-            wide |= !(v > -(1ll << 31) && v < (1ll << 31));
-        }
+        if (operand_value(g, hole, pr, nt, size, rank + j, v)) put(j, v);
     }
     return alive;
 }
@@ -1105,23 +1114,6 @@ __device__ __forceinline__ u32 inv_odd(u32 o) {
 
 __device__ __forceinline__ u32 rotr32(u32 x, u32 k) { return __funnelshift_r(x, x, k); }
 
-// The register-side operands of a tile as the 32-bit loops use them.
-struct RegOps {
-    u32 aA[kNA];     // A * value (the affine context's factor folded in)
-    u32 ca[kNA];     // sign-free form of A * value (SWAP) or of A * value - tp, for the joint +/- test
-    u32 ua[kNA];     // |value|
-    i32 av[kNA];     // the value itself (min and max compare signed numbers)
-    u32 neg;         // bit j: value j is negative
-    // register operand as DIVISOR (SWAP), magnitudes only:
-    u32 low[kNA];    // tabs * |value| (0x80000000 when that is 2^31 or more: never matches)
-    u32 inv[kNA];    // inverse mod 2^32 of the odd part of |value|
-    u32 kk[kNA];     // number of trailing zero bits of |value|
-    u32 cc[kNA];     // floor((2^32-1) / |value|), or 0 when the remainder tabs is impossible
-    u32 alive;       // bit j: operand j exists and is valid at probe 0 (and at probe 1, when that is looked at)
-    i32 a1[kNA];     // value at probe 1
-    u32 a1ok;        // bit j: a1[j] is the exact value (it fits int32)
-};
-
 // The second look: the candidate's exact value at probe 1 from its operands' values there,
 // through the affine context, against the spec.  Operand values that are not known exactly in
 // int32 pass (the exact stages decide).  Runs for filter hits only.
@@ -1134,11 +1126,13 @@ __device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok
     if (sh.p1_rng) return v >= sh.p1_lo && v <= sh.p1_hi;
     return (u64)v * sh.p1_A + sh.p1_B == sh.p1_spec;
 }
-#define XP_P1(op, j, s) probe1_pass(sh, op, (Rm->a1ok >> (j)) & 1u, Rm->a1[j], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
+// (a1ok: bit j says that this thread's operand j is known exactly at probe 1)
+#define XP_P1(op, j, s) probe1_pass(sh, op, (a1ok >> (j)) & 1u, (i32)sh.r1[j][threadIdx.x], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
 
-// The loops below are separate (not inlined) functions on purpose: each copies just the
-// operand arrays it needs from the tile's RegOps into registers and runs with a small live
-// set, instead of sharing one large frame with the rest of the kernel.
+// The loops below are separate (not inlined) functions on purpose: each copies the thread's
+// column of register-side operands from shared memory into registers, derives what it needs of
+// them (a handful of instructions per operand, once per call) and runs with a small live set,
+// instead of sharing one large frame with the rest of the kernel.
 // `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
 
 // Position of a grammar operator among the seven a segment may hold: + - * / % min max.
@@ -1155,13 +1149,13 @@ __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x 
 // the hole has that second look) and queues what is left.  Keeping this part out of line and
 // rolled keeps the loops' instruction footprint small, which matters where the filter is not
 // selective (small value ranges) and the rare path is not rare.
-__device__ __noinline__ void emit_ring(EvalShared& sh, const RegOps* Rm, int s, u32 m_as, u32 m_mul, u32 tp, u32 opip,
+__device__ __noinline__ void emit_ring(EvalShared& sh, u32 a1ok, int s, u32 m_as, u32 m_mul, u32 A, u32 tp, u32 opip,
                                        u32 mask, bool SWAP) {
     const BcRing e = sh.bc_ring[s];
     const u32 t_sub = SWAP ? 0u - e.t_add : 2u * tp - e.t_add;
     for (u32 m = m_as; m; m &= m - 1) {                 // + and -: which of the two (or both) it was
         const int j = __ffs((int)m) - 1;
-        const u32 a = Rm->aA[j];
+        const u32 a = sh.rv[j][threadIdx.x] * A;
         const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
         if ((mask & 1u) && a == e.t_add && XP_P1(XP_OP_ADD, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
         if ((mask & 2u) && a == t_sub && XP_P1(XP_OP_SUB, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
@@ -1172,7 +1166,7 @@ __device__ __noinline__ void emit_ring(EvalShared& sh, const RegOps* Rm, int s, 
     }
 }
 
-__device__ __noinline__ void emit_pairs(EvalShared& sh, const RegOps* Rm, int s, u32 m0, int op0, u32 m1, int op1, u32 opip,
+__device__ __noinline__ void emit_pairs(EvalShared& sh, u32 a1ok, int s, u32 m0, int op0, u32 m1, int op1, u32 opip,
                                         bool SWAP) {
     for (u32 m = m0; m; m &= m - 1) {
         const int j = __ffs((int)m) - 1;
@@ -1194,11 +1188,14 @@ __device__ __noinline__ void emit_pairs(EvalShared& sh, const RegOps* Rm, int s,
 // hits iff the sign-free forms agree: ca == t_pm.  Which of the two hit is settled in the rare
 // path, from t_add.
 template <u32 MASK, bool SWAP>
-__device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tp, int s0, int s1, u32 opip) {
+__device__ __noinline__ void ring_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
     constexpr bool kPair = (MASK & 3u) == 3u;
-    u32 aA[kNA], ca[kNA];
+    u32 aA[kNA], ca[kNA];                               // A * value, and the sign-free form for the joint +/- test
 #pragma unroll
-    for (int j = 0; j < kNA; ++j) { aA[j] = Rm->aA[j]; ca[j] = Rm->ca[j]; }
+    for (int j = 0; j < kNA; ++j) {
+        aA[j] = sh.rv[j][threadIdx.x] * A;
+        ca[j] = signfree(SWAP ? aA[j] : aA[j] - tp);
+    }
     auto t_sub_of = [&](u32 t_add) { return SWAP ? 0u - t_add : 2u * tp - t_add; };
     // The products' distances from the target (one multiply-add each, mul_nt = -tp) are folded
     // into running minima: a candidate hits iff its distance is zero, so one comparison per vote
@@ -1226,7 +1223,7 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
             if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b + e.mul_nt == 0u) << j;
         }
         m_as &= alive; m_mul &= alive;
-        if (m_as | m_mul) emit_ring(sh, Rm, s, m_as, m_mul, tp, opip, MASK, SWAP);
+        if (m_as | m_mul) emit_ring(sh, a1ok, s, m_as, m_mul, A, tp, opip, MASK, SWAP);
     };
     // One warp vote per four broadcast operands (fewer at the end of the run).  The rare path has
     // a single, rolled call site: its code is large, and every copy of it competes with the loops
@@ -1257,18 +1254,18 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegOps* Rm, u32 ali
 // in a run of their own: 0 is skipped (invalid), +-1 gives |quotient| = |dividend| and remainder
 // 0.  There are at most a few such slots per tile, so this is a small rolled routine rather than
 // another instance of the loop below.
-__device__ __noinline__ void div_special(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tabs, int s0, int s1, u32 opip, u32 mask) {
+__device__ __noinline__ void div_special(EvalShared& sh, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip, u32 mask) {
     constexpr bool SWAP = false;
     for (int s = s0; s < s1; ++s) {
         if (sh.bc_div[s].ub != 1u) continue;
         u32 mq = 0, mr = 0;
         for (int j = 0; j < kNA; ++j) {
-            if ((mask & 1u) && Rm->ua[j] == tabs) mq |= 1u << j;
+            if ((mask & 1u) && abs_u32((i32)sh.rv[j][threadIdx.x]) == tabs) mq |= 1u << j;
             if ((mask & 2u) && tabs == 0u) mr |= 1u << j;
         }
         mq &= alive; mr &= alive;
         const bool any = (mq | mr) != 0;
-        if (__any_sync(0xffffffffu, any) && any) emit_pairs(sh, Rm, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
+        if (__any_sync(0xffffffffu, any) && any) emit_pairs(sh, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     }
 }
 
@@ -1283,13 +1280,26 @@ __device__ __noinline__ void div_special(EvalShared& sh, const RegOps* Rm, u32 a
 // SPECIAL (without SWAP only): the slots hold the divisors 0 and +-1: 0 is skipped (invalid),
 // +-1 gives |quotient| = |dividend| and remainder 0.
 template <u32 MASK, bool SWAP, bool SPECIAL>
-__device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 tabs, int s0, int s1, u32 opip) {
+__device__ __noinline__ void div_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip) {
+    // ua: |value|.  xa: |value| - tabs as a dividend (register operand / broadcast operand).  With SWAP the
+    // register operand is the DIVISOR: low = tabs * |value| (0x80000000 when that is 2^31 or more: never
+    // matches), inv = inverse mod 2^32 of the odd part of |value|, kk = its trailing zero bits, cc =
+    // floor((2^32-1) / |value|), or 0 when the remainder tabs is impossible.
     u32 ua[kNA], xa[kNA], low[kNA], inv[kNA], kk[kNA], cc[kNA];
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
-        ua[j] = Rm->ua[j];
+        ua[j] = abs_u32((i32)sh.rv[j][threadIdx.x]);
         xa[j] = ua[j] >= tabs ? ua[j] - tabs : 1u;      // 1 is a multiple of no divisor >= 2
-        if (SWAP) { low[j] = Rm->low[j]; inv[j] = Rm->inv[j]; kk[j] = Rm->kk[j]; cc[j] = Rm->cc[j]; }
+        if (SWAP) {
+            low[j] = 0x80000000u; inv[j] = 1u; kk[j] = 0u; cc[j] = 0u;
+            if (ua[j] != 0u) {
+                const u64 lw = (u64)tabs * ua[j];
+                if (lw < (1ull << 31)) low[j] = (u32)lw;
+                kk[j] = (u32)__ffs((int)ua[j]) - 1u;
+                inv[j] = inv_odd(ua[j] >> kk[j]);
+                cc[j] = tabs < ua[j] ? 0xffffffffu / ua[j] : 0u;
+            }
+        }
     }
     // hits of register operand j against broadcast entry e (quotient, remainder)
     auto test = [&](const BcDiv& e, u32 ek, int j, bool& hq, bool& hr) {
@@ -1330,7 +1340,7 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
         // register operands that are invalid, or (SWAP) zero divisors, are dropped here
         const u32 keep = SWAP ? alive & nz : alive;
         mq &= keep; mr &= keep;
-        if (mq | mr) emit_pairs(sh, Rm, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
+        if (mq | mr) emit_pairs(sh, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     };
     for (int s = s0; s < s1; s += 2) {                  // one warp vote per two broadcast operands; one rare-path site
         const int n = s1 - s < 2 ? 1 : 2;
@@ -1353,10 +1363,10 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegOps* Rm, u32 aliv
 // min and max of int32-exact operands (exact signed comparison), times the context factor A,
 // against tp.  MASK: bit0 min, bit1 max.  Both are symmetric, so SWAP plays no role.
 template <u32 MASK, bool HAS_A>
-__device__ __noinline__ void minmax_pass(EvalShared& sh, const RegOps* Rm, u32 alive, u32 A, u32 tp, int s0, int s1, u32 opip) {
+__device__ __noinline__ void minmax_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
     i32 av[kNA];
 #pragma unroll
-    for (int j = 0; j < kNA; ++j) av[j] = Rm->av[j];
+    for (int j = 0; j < kNA; ++j) av[j] = (i32)sh.rv[j][threadIdx.x];
     auto test = [&](i32 b, int j, bool& hmin, bool& hmax) {
         u32 lo = (u32)(av[j] < b ? av[j] : b), hi = (u32)(av[j] < b ? b : av[j]);
         if (HAS_A) { lo *= A; hi *= A; }
@@ -1384,7 +1394,7 @@ __device__ __noinline__ void minmax_pass(EvalShared& sh, const RegOps* Rm, u32 a
                 if (MASK & 2u) mmax |= (u32)hmax << j;
             }
             mmin &= alive; mmax &= alive;
-            if (mmin | mmax) emit_pairs(sh, Rm, s, mmin, XP_OP_MIN, mmax, XP_OP_MAX, opip, false);
+            if (mmin | mmax) { constexpr bool SWAP = false; emit_pairs(sh, a1ok, s, mmin, XP_OP_MIN, mmax, XP_OP_MAX, opip, SWAP); }
         }
     }
 }
@@ -1393,13 +1403,13 @@ __device__ __noinline__ void minmax_pass(EvalShared& sh, const RegOps* Rm, u32 a
 // compared with tp.  Plain 32-bit division; this form only serves sketches whose hole sits
 // under a multiplication (small searches).
 template <bool SWAP>
-__device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegOps* Rm, u32 alive, u32 mask, u32 A, u32 tp,
+__device__ __noinline__ void div_pass_signed(EvalShared& sh, u32 alive, u32 a1ok, u32 mask, u32 A, u32 tp,
                                              int s0, int s1, u32 opip) {
     for (int s = s0; s < s1; ++s) {
         const i32 b = (i32)sh.bc_meta[s].lo;
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
-            const i32 a = ((Rm->neg >> j) & 1u) ? (i32)(0u - Rm->ua[j]) : (i32)Rm->ua[j];
+            const i32 a = (i32)sh.rv[j][threadIdx.x];
             const i32 n = SWAP ? b : a, d = SWAP ? a : b;
             if (d == 0) continue;
             const i32 q = n / d;                         // magnitudes are below 2^31: no overflow case
@@ -1414,16 +1424,17 @@ __device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegOps* Rm, u
 // Any operator on int64 operands (tiles with an operand outside int32): exact, slow, rare.
 // rng 1: the context compares (HoleDev::rng_lo) and the value must lie in [lo, hi] instead;
 // rng 2: every defined value passes.
-__device__ __noinline__ void wide_chunk(EvalShared& sh, const i64* a, const RegOps* Rm, u32 alive, bool swap, u64 A, u64 tq,
+__device__ __noinline__ void wide_chunk(EvalShared& sh, u32 alive, u32 a1ok, bool swap, u64 A, u64 tq,
                                         int rng, i64 lo, i64 hi, int s0, int s1, int n_ops, const i32* ops) {
     const bool SWAP = swap;
     for (int s = s0; s < s1; ++s) {
         const i64 b = (i64)(((u64)sh.bc_meta[s].hi << 32) | sh.bc_meta[s].lo);
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
+            const i64 aj = (i64)(((u64)sh.rh[j][threadIdx.x] << 32) | sh.rv[j][threadIdx.x]);
             for (int o = 0; o < n_ops; ++o) {
                 i64 v;
-                if (!apply_op(ops[o], swap ? b : a[j], swap ? a[j] : b, v)) continue;
+                if (!apply_op(ops[o], swap ? b : aj, swap ? aj : b, v)) continue;
                 if ((rng == 0 ? (u64)v * A == tq : (rng == 2 || (v >= lo && v <= hi))) && XP_P1(ops[o], j, s))
                     push_hit(sh, threadIdx.x * (u32)kNA + (u32)j, (u32)s, (u32)o);
             }
@@ -1496,8 +1507,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
 
 template <bool SWAP>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
-                                          u64 reg_first, u64 pairs, i64* a64, const i32* a1, u32 a1ok, u32 alive,
-                                          bool drain_at_end, u64& my_evals) {
+                                          u64 reg_first, u64 pairs, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
     const SegDev& seg = sh.mseg[m];
     const MemberState& mbs = sh.mb[m];
     const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
@@ -1516,39 +1526,6 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     const i64 T = (i64)tq;
     const bool t_small = T > -(1ll << 31) && T < (1ll << 31);
     const u32 tabs = (u32)(T < 0 ? -T : T);
-    RegOps R;
-    R.alive = alive;
-    R.neg = 0;
-    R.a1ok = a1ok;
-    if (sh.p1_on) for (int j = 0; j < kNA; ++j) R.a1[j] = a1[j];
-    // Only the arrays that this segment's loops read are written (the struct lives in the
-    // thread's local memory, and every store there is traffic).
-    const bool want_ring = (mask & 7u) != 0, want_div = (mask & 24u) != 0, want_mm = (mask >> kSlotMin) != 0;
-    for (int j = 0; j < kNA; ++j) {
-        const i32 v = (i32)a64[j];
-        const u32 ua = abs_u32(v);
-        if (want_ring) {
-            R.aA[j] = (u32)v * A;
-            R.ca[j] = signfree(SWAP ? R.aA[j] : R.aA[j] - tp);
-        }
-        if (want_mm) R.av[j] = v;
-        if (want_div) {
-            R.ua[j] = ua;
-            if (v < 0) R.neg |= 1u << j;
-        }
-        if (SWAP && want_div && !tile_wide && A == 1u) {
-            u32 low = 0x80000000u, inv = 1u, k = 0u, cc = 0u;
-            if (ua != 0u) {
-                const u64 lw = (u64)tabs * ua;
-                if (lw < (1ull << 31)) low = (u32)lw;
-                k = (u32)__ffs((int)ua) - 1u;
-                inv = inv_odd(ua >> k);
-                cc = tabs < ua ? 0xffffffffu / ua : 0u;
-            }
-            R.low[j] = low; R.inv[j] = inv; R.kk[j] = k; R.cc[j] = cc;
-        }
-    }
-
     // A remainder is smaller in magnitude than its divisor: when no divisor of the tile exceeds the
     // target's magnitude no candidate  a % b  can match, and the loops leave the remainders out.
     const bool skip_mod = !SWAP && (mask & 16u) && !mbs.mod_possible && !tile_wide && !rng && A == 1u && t_small;
@@ -1569,28 +1546,28 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
     auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide || rng) {
-            wide_chunk(sh, a64, &R, alv, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
+            wide_chunk(sh, alv, a1ok, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, &R, alv, tp, s0, s1, opip); break;
+#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, alv, a1ok, A, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
         }
         if (mask >> kSlotMin) switch ((mask >> kSlotMin) & 3u) {
-#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, &R, alv, A, tp, s0, s1, opip); \
-                         else minmax_pass<M, false>(sh, &R, alv, A, tp, s0, s1, opip); break;
+#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, alv, a1ok, A, tp, s0, s1, opip); \
+                         else minmax_pass<M, false>(sh, alv, a1ok, A, tp, s0, s1, opip); break;
             XP_MM(1u) XP_MM(2u) XP_MM(3u)
 #undef XP_MM
             default: break;
         }
         if (!(mask & 24u)) return;
-        if (A != 1u) { div_pass_signed<SWAP>(sh, &R, alv, mask, A, tp, s0, s1, opip); return; }
+        if (A != 1u) { div_pass_signed<SWAP>(sh, alv, a1ok, mask, A, tp, s0, s1, opip); return; }
         if (!t_small) return;                            // no int32 quotient or remainder can be the target
         switch (skip_mod ? (mask >> 3) & 1u : (mask >> 3) & 3u) {
-#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, &R, alv, tabs, s0, s1, opip, M); \
-                          else div_pass<M, SWAP, false>(sh, &R, alv, tabs, s0, s1, opip); break;
+#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, alv, a1ok, tabs, s0, s1, opip, M); \
+                          else div_pass<M, SWAP, false>(sh, alv, a1ok, tabs, s0, s1, opip); break;
             XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
 #undef XP_DIV
             default: break;
@@ -1742,26 +1719,18 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         sh.p1_rng = (hole->rng_okmask >> 1) & 1u;
         sh.p1_lo = hole->rng_lo[1]; sh.p1_hi = hole->rng_hi[1];
     }
-    i64 a64[kNA];
-    bool wide_reg = false;
-    const int mine = n_reg - (int)threadIdx.x * kNA;      // this thread's operands: kNA consecutive ranks
-    u32 alive = fill_reg_operands(g, hole, 0, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA,
-                                  mine < 0 ? 0 : (mine > kNA ? kNA : mine), a64, wide_reg);
+    // this thread's operands: kNA consecutive ranks, into its column of the tile
+    const int mine = n_reg - (int)threadIdx.x * kNA;
+    const int n_mine = mine < 0 ? 0 : (mine > kNA ? kNA : mine);
+    u32 fits0 = 0;
+    u32 alive = fill_reg_operands(g, hole, 0, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA, n_mine,
+                                  &sh.rv[0][threadIdx.x], &sh.rh[0][threadIdx.x], fits0);
+    const bool wide_reg = fits0 != alive;
     // second look: the same operands at probe 1; one that is undefined there can be in no match
-    i32 a1[kNA];
     u32 a1ok = 0;
-    if (second) {
-        i64 b64[kNA];
-        bool wide1 = false;
-        alive &= fill_reg_operands(g, hole, 1, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA,
-                                   mine < 0 ? 0 : (mine > kNA ? kNA : mine), b64, wide1);
-        for (int j = 0; j < kNA; ++j) {
-            a1[j] = (i32)b64[j];
-            if (b64[j] > -(1ll << 31) && b64[j] < (1ll << 31)) a1ok |= 1u << j;
-        }
-    } else {
-        for (int j = 0; j < kNA; ++j) a1[j] = 0;
-    }
+    if (second)
+        alive &= fill_reg_operands(g, hole, 1, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA, n_mine,
+                                   &sh.r1[0][threadIdx.x], nullptr, a1ok);
     __syncthreads();                                    // the members' segments are in place, reg_wide is clear
     if (wide_reg) sh.reg_wide = 1;
     // broadcast operands of member m: tile bc_tile0 of the head (a family's other members have one tile)
@@ -1797,8 +1766,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
             if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
-            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, false, my_evals);
+            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, false, my_evals);
+            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, false, my_evals);
         }
         drain_queue(sh, plan, sk, hole, reg_first, my_evals);
         return;
@@ -1812,8 +1781,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         const SegDev& seg = sh.mseg[m];
         const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
         if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a64, a1, a1ok, alive, true, my_evals);
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, true, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, true, my_evals);
     }
 }
 
@@ -1821,50 +1790,53 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
 #define XP_MIN_CTAS 3
 #endif
 __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanDev plan) {
-    __shared__ EvalShared sh;
+    extern __shared__ __align__(16) unsigned char eval_smem[];      // (more than the 48 KB a static array may have)
+    EvalShared& sh = *reinterpret_cast<EvalShared*>(eval_smem);
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
     if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; sh.filter_tests = 0; sh.tile_cands = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
-        if (threadIdx.x == 0) {
-            sh.ticket = plan.ticket_base + atomicAdd(plan.ticket, 1ull);
+        if (threadIdx.x == 0) sh.item = plan.item_base + atomicAdd(plan.ticket, 1ull);
+        __syncthreads();
+        const u64 item = sh.item;
+        if (item >= plan.n_items) break;
+        const u64 t_first = plan.group_first ? plan.group_first[item] : item;
+        const u64 t_last = plan.group_first ? plan.group_first[item + 1] : item + 1;
+        for (u64 t = t_first; t < t_last; ++t) {
             // many filter hits so far for the hole at hand (this CTA's own counts): second look from now on
-            if (!sh.adapt_second && sh.filter_survivors * kAdaptRate > sh.tile_cands) sh.adapt_second = 1;
-        }
-        __syncthreads();
-        const u64 t = sh.ticket;
-        if (t >= plan.n_tickets) break;
-        if (threadIdx.x < 32) {
-            // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
-            int lo = 0, n = plan.n_segs;
-            while (n > 1) {
-                const int step = (n + 31) / 32;
-                const int pos = lo + (int)threadIdx.x * step;
-                const bool le = pos < lo + n && plan.segs[pos].first_ticket <= t;
-                const u32 mask = __ballot_sync(0xffffffffu, le);          // lane 0 always holds
-                const int k = 31 - __clz((int)(mask | 1u));
-                const int nlo = lo + k * step;
-                n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
-                lo = nlo;
+            if (threadIdx.x == 0 && !sh.adapt_second && sh.filter_survivors * kAdaptRate > sh.tile_cands) sh.adapt_second = 1;
+            if (threadIdx.x < 32) {
+                // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
+                int lo = 0, n = plan.n_segs;
+                while (n > 1) {
+                    const int step = (n + 31) / 32;
+                    const int pos = lo + (int)threadIdx.x * step;
+                    const bool le = pos < lo + n && plan.segs[pos].first_ticket <= t;
+                    const u32 mask = __ballot_sync(0xffffffffu, le);          // lane 0 always holds
+                    const int k = 31 - __clz((int)(mask | 1u));
+                    const int nlo = lo + k * step;
+                    n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
+                    lo = nlo;
+                }
+                if (!XP_CHECKED(lo >= 0 && lo < plan.n_segs && plan.segs[lo].first_ticket <= t, kChkSegment)) lo = 0;
+                if (threadIdx.x == 0) sh.seg_index = lo;
+                load_segment(sh, plan, lo);
             }
-            if (!XP_CHECKED(lo >= 0 && lo < plan.n_segs && plan.segs[lo].first_ticket <= t, kChkSegment)) lo = 0;
-            if (threadIdx.x == 0) sh.seg_index = lo;
-            load_segment(sh, plan, lo);
-        }
-        __syncthreads();
-        if (sh.seg.acc != sh.cur_acc) {
-            flush_acc(sh, plan, my_evals);
-            if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
+            __syncthreads();
+            if (sh.seg.acc != sh.cur_acc) {
+                flush_acc(sh, plan, my_evals);
+                if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
+                __syncthreads();
+            }
+            const SketchDev* sk = plan.sketches[sh.seg.sketch];
+            const HoleDev* hole = &sk->holes[sh.seg.hole];
+            const u64 local = t - sh.seg.first_ticket;
+            if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
+            else linear_ticket(sh, plan, sk, hole, local, my_evals);
             __syncthreads();
         }
-        const SketchDev* sk = plan.sketches[sh.seg.sketch];
-        const HoleDev* hole = &sk->holes[sh.seg.hole];
-        const u64 local = t - sh.seg.first_ticket;
-        if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
-        else linear_ticket(sh, plan, sk, hole, local, my_evals);
-        __syncthreads();
     }
     flush_acc(sh, plan, my_evals);
 }
@@ -1884,20 +1856,297 @@ __device__ __noinline__ void record_killer(const HoleDev* hole, i64 pid) {
     }                                                   // (table crowded around this slot: the point goes unrecorded)
 }
 
-// Items are (chunk of points, survivor), chunk-major: the first chunk of every survivor is
-// taken before any second chunk, so candidates that fail early cost one chunk.  Each WARP
-// takes items on its own (lane = point, 32 points per step, warp vote): nothing in this
-// kernel synchronises a CTA, and no warp waits for another.  An item whose survivor has
-// already failed is skipped; lane 0 reads that flag once and shares the decision.
-__global__ void __launch_bounds__(kThreads, 3) verify_kernel(const PlanDev plan) {
-    __shared__ CandShared cands[kWarps];
-    __shared__ uint4 stacks[kWarps][kVecDepth * 32];    // operand stacks below the top, per warp, level and lane
-    CandShared& cand = cands[threadIdx.x >> 5];
+// ---- survivors in hole order ----
+//
+// eval_kernel counts the queued survivors per accumulator slot (= per hole of the call); a scan turns
+// the counts into offsets and a scatter writes, per slot, the queue indices of its survivors side by
+// side.  The verification kernel walks that order, so the survivors a warp takes together mostly
+// belong to one hole: same points, same spec values.
+
+// One CTA: exclusive scan of hist[0 .. n_acc) into off[0 .. n_acc]; hist is cleared for the scatter.
+__global__ void __launch_bounds__(1024) surv_scan_kernel(u32* hist, u32* off, int n_acc) {
+    __shared__ u32 part[1024];
+    const int t = threadIdx.x;
+    const int per = (n_acc + 1023) / 1024;
+    const int lo = t * per < n_acc ? t * per : n_acc, hi = lo + per < n_acc ? lo + per : n_acc;
+    u32 sum = 0;
+    for (int i = lo; i < hi; ++i) sum += hist[i];
+    part[t] = sum;
+    __syncthreads();
+    for (int d = 1; d < 1024; d <<= 1) {
+        const u32 v = t >= d ? part[t - d] : 0u;
+        __syncthreads();
+        part[t] += v;
+        __syncthreads();
+    }
+    u32 run = part[t] - sum;
+    for (int i = lo; i < hi; ++i) { const u32 h = hist[i]; off[i] = run; run += h; hist[i] = 0; }
+    if (t == 1023) off[n_acc] = part[1023];
+}
+
+__global__ void __launch_bounds__(256) surv_scatter_kernel(const PlanDev plan) {
+    const u32 pushed = *plan.surv_n;
+    const u32 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
+    const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int acc = plan.surv[i].acc;
+    plan.surv_sorted[plan.surv_off[acc] + atomicAdd(&plan.surv_hist[acc], 1u)] = i;
+}
+
+// ---- whole-domain check of several survivors of one hole together ----
+//
+// For table domains.  The warp's lanes each stage one survivor (unranking, substitution into the
+// context, magnitude bounds, constant-divisor folding: all 32 at once, where one lane used to do it
+// for one survivor while 31 waited) as a compact program in the warp's arena.  Then the chunk is
+// walked in steps of 128 points (4 per lane): the step's coordinates go to shared memory and its
+// spec values to registers ONCE, and every staged survivor still alive is run on them; a survivor
+// that fails at some point of the step leaves the set.
+constexpr int kVArena = 256;                              // program entries a warp stages at once
+constexpr int kVStep = 128;                               // points per step
+struct __align__(16) VerifyWarp {
+    i32 pvar[kVArena];                                    // >= 0: variable; -1: constant; -2 - op: operator
+    i64 pval[kVArena];
+    i32 coords[kMaxVars][kVStep];                         // the step's points, [variable][point]
+    uint4 stack[kVecDepth * 32];                          // operand stacks below the top, per level and lane
+    CandShared cand;                                      // the one-survivor form (boxes, long programs)
+};
+
+// Length of the program that candidate code of `n` nodes gives in the hole's context; -1 if the
+// context never mentions the hole (the one-survivor form handles that).
+__device__ __forceinline__ int staged_length(const HoleDev* hole, int n) {
+    if (hole->ctx_len == 0) return n;
+    int holes = 0;
+    for (int i = 0; i < hole->ctx_len; ++i) holes += hole->ctx[i].kind == XP_I_HOLE;
+    return holes ? hole->ctx_len + holes * (n - 1) : -1;
+}
+
+// One lane: stages survivor (size, rank) at w.pvar / w.pval [off ...).  Returns the final length
+// (constant divisors folded when the program is exact in int32), or -1 when the operand stack gets
+// deeper than the vectorised check takes.
+__device__ __noinline__ int stage_compact(VerifyWarp& w, int off, const SketchDev* sk, const HoleDev* hole, int size, u64 rank,
+                                         bool& narrow_out) {
+    const GrammarDev* g = sk->g;
+    u32 code[kMaxSize];
+    const int n = unrank(g, hole->start_nt, size, rank, code);
+    int len = 0, sp = 0, depth = 0;
+    bool narrow = true;
+    constexpr u64 kSat = 1ull << 62;
+    u64 mag[kMaxStack + kCandStack + 1];
+    auto mag_of = [](i64 v) { return v < 0 ? 0ull - (u64)v : (u64)v; };
+    auto emit = [&](i32 var, i64 val) {
+        if (sp > kMaxStack + kCandStack - 1) { depth = kVecDepth + 1; return; }
+        w.pvar[off + len] = var; w.pval[off + len] = val; ++len;
+        u64 m;
+        if (var >= -1) {
+            if (var >= 0) { const u64 a = mag_of(sk->vmin[var]), b = mag_of(sk->vmax[var]); m = a > b ? a : b; }
+            else m = mag_of(val);
+            mag[sp] = m < kSat ? m : kSat;
+            if (++sp > depth) depth = sp;
+        } else {
+            --sp;
+            const u64 a = mag[sp - 1], b = mag[sp];
+            switch (-2 - var) {
+                case XP_OP_ADD: case XP_OP_SUB: m = a + b; break;
+                case XP_OP_MUL: m = (a >> 31 || b >> 31) ? kSat : a * b; break;
+                case XP_OP_DIV: m = a; break;
+                case XP_OP_MOD: m = a < b ? a : b; break;
+                case XP_OP_MIN: case XP_OP_MAX: m = a > b ? a : b; break;
+                default: m = 1; break;
+            }
+            mag[sp - 1] = m < kSat ? m : kSat;
+        }
+        narrow = narrow && (m >> 31) == 0;
+    };
+    auto emit_cand = [&]() {
+        for (int k = 0; k < n; ++k) {
+            if (code[k] & kOpBit) emit(-2 - (i32)(code[k] & 0xff), 0);
+            else { const LeafDev lf = g->leaves[code[k]]; emit(lf.var >= 0 ? lf.var : -1, lf.value); }
+        }
+    };
+    if (hole->ctx_len == 0) emit_cand();
+    else
+        for (int i = 0; i < hole->ctx_len; ++i) {
+            const xp_instr in = hole->ctx[i];
+            if (in.kind == XP_I_HOLE) emit_cand();
+            else if (in.kind == XP_I_OP) emit(-2 - in.arg, 0);
+            else emit(in.kind == XP_I_VAR ? in.arg : -1, in.value);
+        }
+    narrow_out = narrow;
+    if (depth > kVecDepth) return -1;
+    if (narrow) {                                         // "push c; x / y" -> one instruction on the top of the stack
+        int wr = 0;
+        for (int k = 0; k < len; ++k) {
+            const i32 cv = w.pvar[off + k];
+            const bool divmod = cv == -2 - XP_OP_DIV || cv == -2 - XP_OP_MOD;
+            if (divmod && wr > 0 && w.pvar[off + wr - 1] == -1 && w.pval[off + wr - 1] != 0 &&
+                w.pval[off + wr - 1] > -(1ll << 31) && w.pval[off + wr - 1] < (1ll << 31)) {
+                const i32 d = (i32)w.pval[off + wr - 1];
+                const u32 ad = d < 0 ? 0u - (u32)d : (u32)d;
+                const u32 M = ad == 1u ? 0xffffffffu : (u32)((1ull << 32) / ad);
+                w.pvar[off + wr - 1] = -2 - (cv == -2 - XP_OP_DIV ? kOpDivC : kOpModC);
+                w.pval[off + wr - 1] = (i64)(((u64)M << 32) | (u32)d);
+                continue;
+            }
+            w.pvar[off + wr] = cv; w.pval[off + wr] = w.pval[off + k]; ++wr;
+        }
+        len = wr;
+    }
+    return len;
+}
+
+// The staged program [off, off + len) on the lane's points of the step (P at a time: points
+// lane*4 + half*P + i).  Returns the bit set of the lane's points that fail (a zero divisor: bit 0).
+template <typename T, int P>
+__device__ __forceinline__ u32 run_staged(VerifyWarp& w, int off, int len, int half, const i64* want, u32 in_mask) {
+    typedef VecSlot<T, P> Slot;
+    const int lane = threadIdx.x & 31;
+    Slot t;
+#pragma unroll
+    for (int i = 0; i < P; ++i) t.v[i] = 0;
+    bool bad = false;
+    int below = 0;
+    for (int k = 0; k < len; ++k) {
+        const i32 cv = w.pvar[off + k];
+        if (cv >= -1) {
+            w.stack[below * 32 + lane] = t.q;
+            ++below;
+            if (cv >= 0) {
+                if (sizeof(T) == 4) t.q = *reinterpret_cast<const uint4*>(&w.coords[cv][lane * 4]);
+                else {
+#pragma unroll
+                    for (int i = 0; i < P; ++i) t.v[i] = (T)w.coords[cv][lane * 4 + half * P + i];
+                }
+            } else {
+                const T v = (T)w.pval[off + k];
+#pragma unroll
+                for (int i = 0; i < P; ++i) t.v[i] = v;
+            }
+            continue;
+        }
+        const int op = -2 - cv;
+        Slot a;
+        a.q = t.q;
+        if (!(sizeof(T) == 4 && op >= kOpDivC)) { --below; a.q = w.stack[below * 32 + lane]; }
+        vec_op<T, P>(op, w.pval[off + k], a, t, bad);
+    }
+    u32 which = 0;
+#pragma unroll
+    for (int i = 0; i < P; ++i) which |= (u32)(((in_mask >> (half * P + i)) & 1u) && (i64)t.v[i] != want[half * P + i]) << (half * P + i);
+    // (points past the end of the chunk repeat its first point, so a zero divisor there is one at a real point too)
+    return which | (bad ? 1u : 0u);
+}
+
+// The survivors of `now` (bit b = lane b holds one, all of one hole) on chunk `chunk` of the hole's
+// table domain.  Each lane ends up with `failed` set if its survivor failed at some point
+// (fail_pid), and the warp with the number of candidate-point evaluations it made.
+__device__ __noinline__ void verify_batch(VerifyWarp& w, const SketchDev* sk, const HoleDev* hole, u32 now, int my_off, int my_len,
+                                          bool my_narrow, i64 first, i64 last, bool& failed, i64& fail_pid, u64& evals) {
+    const int lane = threadIdx.x & 31;
+    const int nv = sk->n_vars;
+    const i32* __restrict__ coords = sk->coords;
+    const i64* __restrict__ spec = hole->spec_table;
+    u32 alive = now;
+    for (i64 base = first; base < last && alive; base += kVStep) {
+        const int npts = last - base < kVStep ? (int)(last - base) : kVStep;
+        __syncwarp();                                     // everyone is done with the previous step's points
+        for (int idx = lane; idx < kVStep * nv; idx += 32) {      // rows are contiguous: coalesced reads
+            const int p = idx / nv, v = idx - p * nv;
+            const int src = p < npts ? idx : v;           // points past the end repeat the step's first point
+            w.coords[v][p] = coords[base * nv + src];
+        }
+        i64 want[4];
+        u32 in_mask = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = lane * 4 + i;
+            if (p < npts) in_mask |= 1u << i;
+            want[i] = spec[base + (p < npts ? p : 0)];
+        }
+        __syncwarp();
+        evals += (u64)npts * (u64)__popc(alive);
+        for (u32 m = alive; m; m &= m - 1) {
+            const int b = __ffs((int)m) - 1;
+            const int off = __shfl_sync(0xffffffffu, my_off, b), len = __shfl_sync(0xffffffffu, my_len, b);
+            const bool narrow = __shfl_sync(0xffffffffu, (int)my_narrow, b) != 0;
+            u32 which;
+            if (narrow) which = run_staged<i32, 4>(w, off, len, 0, want, in_mask);
+            else which = run_staged<i64, 2>(w, off, len, 0, want, in_mask) | run_staged<i64, 2>(w, off, len, 1, want, in_mask);
+            const u32 bm = __ballot_sync(0xffffffffu, which != 0u);
+            if (bm) {
+                const int src = __ffs((int)bm) - 1;
+                const u32 wsrc = __shfl_sync(0xffffffffu, which, src);
+                alive &= ~(1u << b);
+                if (lane == b) {
+                    const int p = src * 4 + (__ffs((int)wsrc) - 1);
+                    failed = true;
+                    fail_pid = base + (p < npts ? p : 0);
+                }
+            }
+        }
+    }
+}
+
+// One survivor on one chunk, staged by the warp's first lane (boxes with their sub-box projection,
+// programs that do not fit the arena, contexts that never mention the hole).
+__device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 si, u64 chunk) {
+    const int lane = threadIdx.x & 31;
+    CandShared& cand = w.cand;
+    int skip = 1;
+    i64 np = 0;
+    SurvDev* sv = &plan.surv[si];
+    const SketchDev* sk = plan.sketches[sv->sketch];
+    const HoleDev* hole = &sk->holes[sv->hole];
+    if (lane == 0) {
+        const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
+        np = proj_points(sk, hole, sv->vars, nullptr);
+        if ((i64)chunk * kVerifyChunk < np && !failed) {
+            skip = 0;
+            stage_candidate(cand, sk, hole, sv->size, sv->rank);
+            proj_points(sk, hole, sv->vars, &cand);
+            if (cand.narrow && sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth)
+                fold_constant_divisors(cand);             // (exactly the case that takes the int32 vectorised check below)
+        }
+    }
+    __syncwarp();
+    skip = __shfl_sync(0xffffffffu, skip, 0);
+    if (skip) return;
+    np = __shfl_sync(0xffffffffu, np, 0);
+    const i64 first = (i64)chunk * kVerifyChunk;
+    const i64 last = first + kVerifyChunk < np ? first + kVerifyChunk : np;
+    u64 evals = 0;
+    i64 fail_pid = 0;
+    bool ok;
+    if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
+        ok = cand.narrow ? check_points_vec<i32, 4>(cand, w.stack, sk, hole, first, last, &fail_pid)
+                         : check_points_vec<i64, 2>(cand, w.stack, sk, hole, first, last, &fail_pid);
+    } else {
+        ok = check_points(cand, sk, hole, first, last, evals, &fail_pid);
+    }
+    if (lane == 0) {
+        if (ok) atomicAdd(&sv->state, 1u);
+        else if (!(atomicOr(&sv->state, kSurvFailed) & kSurvFailed)) record_killer(hole, fail_pid);   // (once per survivor)
+        atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
+    }
+    __syncwarp();                                       // the staged candidate is free for the next item
+}
+
+// Items are (chunk of points, block of 32 survivors in hole order), chunk-major: the first chunk
+// of every survivor is taken before any second chunk, so candidates that fail early cost one
+// chunk.  Each WARP takes items on its own: nothing in this kernel synchronises a CTA, and no
+// warp waits for another.  Within a block the survivors of one hole are handled together when the
+// hole's domain is a table (verify_batch), one after the other otherwise (verify_one).  A survivor
+// that has already failed is skipped.
+constexpr int kVerifyThreads = 256;
+constexpr int kVerifyWarps = kVerifyThreads / 32;
+__global__ void __launch_bounds__(kVerifyThreads, 2) verify_kernel(const PlanDev plan) {
+    extern __shared__ __align__(16) unsigned char verify_smem[];
+    VerifyWarp& w = reinterpret_cast<VerifyWarp*>(verify_smem)[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const u32 pushed = *plan.surv_n;
     const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
-    const u64 total = n * plan.max_chunks;
-    constexpr u64 kBatch = 8;                           // tickets a warp takes per atomic
+    const u64 n_blocks = (n + 31) / 32;
+    const u64 total = n_blocks * plan.max_chunks;
+    constexpr u64 kBatch = 2;                           // items a warp takes per atomic
     u64 next = 0, batch_end = 0;
     for (;;) {
         if (next == batch_end) {
@@ -1907,47 +2156,70 @@ __global__ void __launch_bounds__(kThreads, 3) verify_kernel(const PlanDev plan)
         }
         const u64 t = next++;
         if (t >= total) break;
-        int skip = 1;
-        i64 np = 0;
-        if (lane == 0) {
-            const SurvDev* sv = &plan.surv[t % n];
-            const SketchDev* sk = plan.sketches[sv->sketch];
-            const HoleDev* hole = &sk->holes[sv->hole];
-            const bool failed = (*(volatile const u32*)&sv->state & kSurvFailed) != 0;
-            np = proj_points(sk, hole, sv->vars, nullptr);
-            if ((i64)(t / n) * kVerifyChunk < np && !failed) {
-                skip = 0;
-                stage_candidate(cand, sk, hole, sv->size, sv->rank);
-                proj_points(sk, hole, sv->vars, &cand);
-                if (cand.narrow && sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth)
-                    fold_constant_divisors(cand);         // (exactly the case that takes the int32 vectorised check below)
+        const u64 chunk = t / n_blocks, block = t % n_blocks;
+        const u64 pos = block * 32 + lane;
+        const bool have = pos < n;
+        const u32 si = have ? (plan.surv_sorted ? plan.surv_sorted[pos] : (u32)pos) : 0u;
+        const int my_acc = have ? plan.surv[si].acc : -1;
+        u32 remaining = __ballot_sync(0xffffffffu, have);
+        while (remaining) {
+            const int leader = __ffs((int)remaining) - 1;
+            const int acc = __shfl_sync(0xffffffffu, my_acc, leader);
+            const u32 run = __ballot_sync(0xffffffffu, have && my_acc == acc) & remaining;
+            remaining &= ~run;
+            const u32 lsi = __shfl_sync(0xffffffffu, si, leader);
+            const SketchDev* sk = plan.sketches[plan.surv[lsi].sketch];
+            const HoleDev* hole = &sk->holes[plan.surv[lsi].hole];
+            const bool table = sk->domain_kind == XP_DOMAIN_TABLE && sk->coords != nullptr && hole->spec_table != nullptr;
+            const i64 first = (i64)chunk * kVerifyChunk;
+            const bool mine = (run >> lane) & 1u;
+            u32 single = 0;                               // survivors of the run that go one by one
+            if (!table) single = run;
+            else if (first < sk->n_points) {
+                const i64 last = first + kVerifyChunk < sk->n_points ? first + kVerifyChunk : sk->n_points;
+                SurvDev* sv = &plan.surv[si];
+                const bool live = mine && !(*(volatile const u32*)&sv->state & kSurvFailed);
+                const int want_len = live ? staged_length(hole, sv->size) : 0;
+                single = __ballot_sync(0xffffffffu, live && (want_len < 0 || want_len > kVArena));
+                u32 todo = __ballot_sync(0xffffffffu, live) & ~single;
+                while (todo) {                            // as many as the arena holds at a time
+                    int off = 0, my_off = 0;
+                    u32 now = 0;
+                    for (u32 m = todo; m; m &= m - 1) {   // (uniform: every lane walks the same set)
+                        const int b = __ffs((int)m) - 1;
+                        const int len_b = __shfl_sync(0xffffffffu, want_len, b);
+                        if (off + len_b > kVArena) break;
+                        if (lane == b) my_off = off;
+                        now |= 1u << b;
+                        off += len_b;
+                    }
+                    todo &= ~now;
+                    __syncwarp();                         // the arena is free (the previous round's programs are done)
+                    bool narrow = false, failed = false;
+                    int len = 0;
+                    if ((now >> lane) & 1u) {
+                        len = stage_compact(w, my_off, sk, hole, sv->size, sv->rank, narrow);
+                        if (len < 0) { len = 0; }
+                    }
+                    const u32 deep = __ballot_sync(0xffffffffu, ((now >> lane) & 1u) && len == 0);      // stack too deep: one by one
+                    single |= deep;
+                    now &= ~deep;
+                    __syncwarp();
+                    i64 fail_pid = 0;
+                    u64 evals = 0;
+                    verify_batch(w, sk, hole, now, my_off, len, narrow, first, last, failed, fail_pid, evals);
+                    if ((now >> lane) & 1u) {
+                        if (!failed) atomicAdd(&sv->state, 1u);
+                        else if (!(atomicOr(&sv->state, kSurvFailed) & kSurvFailed)) record_killer(hole, fail_pid);
+                    }
+                    if (lane == 0 && evals) atomicAdd(&plan.acc[acc].evals, evals);
+                }
+            }
+            for (u32 m = single; m; m &= m - 1) {
+                const int b = __ffs((int)m) - 1;
+                verify_one(plan, w, __shfl_sync(0xffffffffu, si, b), chunk);
             }
         }
-        __syncwarp();
-        skip = __shfl_sync(0xffffffffu, skip, 0);
-        if (skip) continue;
-        np = __shfl_sync(0xffffffffu, np, 0);
-        SurvDev* sv = &plan.surv[t % n];
-        const SketchDev* sk = plan.sketches[sv->sketch];
-        const HoleDev* hole = &sk->holes[sv->hole];
-        const i64 first = (i64)(t / n) * kVerifyChunk;
-        const i64 last = first + kVerifyChunk < np ? first + kVerifyChunk : np;
-        u64 evals = 0;
-        i64 fail_pid = 0;
-        bool ok;
-        if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
-            uint4* stack = stacks[threadIdx.x >> 5];
-            ok = cand.narrow ? check_points_vec<i32, 4>(cand, stack, sk, hole, first, last, &fail_pid)
-                             : check_points_vec<i64, 2>(cand, stack, sk, hole, first, last, &fail_pid);
-        } else {
-            ok = check_points(cand, sk, hole, first, last, evals, &fail_pid);
-        }
-        if (lane == 0) {
-            if (ok) atomicAdd(&sv->state, 1u);
-            else if (!(atomicOr(&sv->state, kSurvFailed) & kSurvFailed)) record_killer(hole, fail_pid);   // (once per survivor)
-            atomicAdd(&plan.acc[sv->acc].evals, (u64)(last - first));     // points of the chunk (an early exit tries fewer)
-        }
-        __syncwarp();                                   // the staged candidate is free for the next item
     }
 }
 
@@ -2062,18 +2334,19 @@ cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most
     return cudaGetLastError();
 }
 
-static int resident_ctas(const void* kernel) {
+static int resident_ctas(const void* kernel, size_t dynamic_smem = 0) {
     int dev = 0, sms = 1, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 1;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, dynamic_smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     return sms * per_sm;
 }
 
 static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sketches, u32 max_chunks) {
     PlanDev pd;
-    pd.ticket_base = 0;
-    pd.n_tickets = 0;
+    pd.item_base = 0;
+    pd.n_items = 0;
+    pd.group_first = L.n_groups ? (const u64*)(base + L.groups) : nullptr;
     pd.n_segs = n_segs;
     pd.n_sketches = n_sketches;
     pd.ticket = (u64*)base;
@@ -2086,10 +2359,16 @@ static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sket
     pd.surv = (SurvDev*)(base + L.surv);
     pd.surv_cap = L.surv_cap;
     pd.max_chunks = max_chunks;
+    pd.n_acc = L.n_acc;
+    const bool order = L.n_acc > 1;                       // (one hole: the queue is in hole order as it is)
+    pd.surv_hist = order ? (u32*)(base + L.hist) : nullptr;
+    pd.surv_off = order ? (u32*)(base + L.sort_off) : nullptr;
+    pd.surv_sorted = order ? (u32*)(base + L.sorted) : nullptr;
     return pd;
 }
 
-// Stages 1 and 2 for the tickets [t_begin, t_end) of the plan staged at `base`.  A search is one
+// Stages 1 and 2 for the work items [t_begin, t_end) of the plan staged at `base` (an item is a
+// ticket, or a group of tickets when the layout carries groups).  A search is one
 // such launch, or several in a row when the host wants to look at a cancel word or a clock in
 // between; `restart` says that the ticket counter has to be set back to zero first (every launch
 // but the first, whose counter the staged copy has just zeroed).
@@ -2099,11 +2378,15 @@ cudaError_t launch_search_part(char* base, const SearchLayout& L, u64 t_begin, u
     cudaError_t e;
     if (restart && (e = cudaMemsetAsync(base, 0, 8, stream)) != cudaSuccess) return e;
     PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
-    pd.ticket_base = t_begin;
-    pd.n_tickets = t_end;
-    u64 ctas = (u64)resident_ctas((const void*)eval_kernel);      // persistent CTAs: one wave
+    pd.item_base = t_begin;
+    pd.n_items = t_end;
+    if ((e = cudaFuncSetAttribute((const void*)eval_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EvalShared))) != cudaSuccess) return e;
+#ifdef XP_CARVEOUT
+    if ((e = cudaFuncSetAttribute((const void*)eval_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, XP_CARVEOUT)) != cudaSuccess) return e;
+#endif
+    u64 ctas = (u64)resident_ctas((const void*)eval_kernel, sizeof(EvalShared));      // persistent CTAs: one wave
     if (ctas > t_end - t_begin) ctas = t_end - t_begin;
-    eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
+    eval_kernel<<<(unsigned)ctas, kThreads, sizeof(EvalShared), stream>>>(pd);
     *n_launches += 1;
     return cudaGetLastError();
 }
@@ -2114,7 +2397,16 @@ cudaError_t launch_search_end(char* base, const SearchLayout& L, bool any_ticket
     PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
     cudaError_t e;
     if (any_tickets) {
-        verify_kernel<<<resident_ctas((const void*)verify_kernel), kThreads, 0, stream>>>(pd);
+        if (pd.surv_sorted) {
+            surv_scan_kernel<<<1, 1024, 0, stream>>>(pd.surv_hist, pd.surv_off, pd.n_acc);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            surv_scatter_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            *n_launches += 2;
+        }
+        const size_t vsmem = sizeof(VerifyWarp) * kVerifyWarps;
+        if ((e = cudaFuncSetAttribute((const void*)verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vsmem)) != cudaSuccess) return e;
+        verify_kernel<<<resident_ctas((const void*)verify_kernel, vsmem), kVerifyThreads, vsmem, stream>>>(pd);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         count_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;

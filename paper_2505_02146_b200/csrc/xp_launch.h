@@ -16,9 +16,10 @@ cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most
 // Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
 //   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32), 20: failed-check word (u32; checked
 //      build only)   -- zero at launch
-//   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
-//   surv: the survivor queue (surv_cap entries), written by the kernels only
-struct SearchLayout { size_t segs, sketches, acc, head, surv, total; u32 surv_cap; };
+//   segs, sketches, acc, groups (first ticket of every group of tickets, when the plan is grouped): staged from the host;  [0, head) is what the host copies in
+//   hist: survivors per accumulator slot, zero at launch (staged);
+//   surv: the survivor queue (surv_cap entries); sort_off, sorted: its hole order -- written by the kernels only
+struct SearchLayout { size_t segs, sketches, acc, groups, hist, head, surv, sort_off, sorted, total; u32 surv_cap; u64 n_groups; int n_acc; };
 
 // The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel;
 // or the same in pieces: eval_kernel over one range of tickets at a time, then the rest.

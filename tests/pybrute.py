@@ -38,6 +38,10 @@ def c_op(op: str, a: int, b: int) -> Optional[int]:
     if op == "max": return max(a, b)
     if op == "&&": return int(a != 0 and b != 0)
     if op == "||": return int(a != 0 or b != 0)
+    if op in ("<<", ">>"):                    # a shift count outside 0..63 is undefined, like a zero divisor
+        if b < 0 or b > 63:
+            return None
+        return wrap(a * (1 << b)) if op == "<<" else a // (1 << b)      # >> keeps the sign (floor division)
     raise ValueError(op)
 
 
@@ -81,13 +85,14 @@ def tree_text(t: tuple, g: Grammar) -> str:
     return f"({tree_text(t[1], g)}{t[0]}{tree_text(t[2], g)})"
 
 
-def code_value(code, pt: Sequence[int], hole: int = 0) -> Optional[int]:
+def code_value(code, pt: Sequence[int], hole=0) -> Optional[int]:
+    """``hole``: the hole's value, or a sequence of values for the parts of a joint sketch."""
     st: List[Optional[int]] = []
     bad = False
     for kind, arg, value in code:
         if kind == K_VAR: st.append(pt[arg])
         elif kind == K_CONST: st.append(value)
-        elif kind == K_HOLE: st.append(hole)
+        elif kind == K_HOLE: st.append(hole[arg] if isinstance(hole, (list, tuple)) else hole)
         else:
             b = st.pop(); a = st.pop()
             r = c_op(OPS[arg], a, b)
@@ -138,6 +143,37 @@ def repair(sk: Sketch, hole_index: int = 0):
     return cand, match, least, matches
 
 
+def repair_joint(g: Grammar, starts, max_sizes, ctx, pts, spec):
+    """Two holes in one context, brute force: (cand_count, match_count, least) by TOTAL size, where
+    least = (total size, size of part 0, rank of part 0, rank of part 1, text 0, text 1) in the order
+    total size, size of part 0, rank of part 0, rank of part 1."""
+    T = all_trees(g, max(max_sizes))
+    K = max_sizes[0] + max_sizes[1]
+    cand = [0] * (K + 1)
+    match = [0] * (K + 1)
+    least = None
+    for s in range(2, K + 1):
+        for s0 in range(1, s):
+            s1 = s - s0
+            if s0 > max_sizes[0] or s1 > max_sizes[1]:
+                continue
+            A, B = T[(starts[0], s0)], T[(starts[1], s1)]
+            cand[s] += len(A) * len(B)
+            for r0, t0 in enumerate(A):
+                for r1, t1 in enumerate(B):
+                    good = True
+                    for p, want in zip(pts, spec):
+                        v0, v1 = tree_value(t0, p), tree_value(t1, p)
+                        v = None if v0 is None or v1 is None else code_value(ctx, p, (v0, v1))
+                        if v is None or want is None or v != want:
+                            good = False
+                    if good:
+                        match[s] += 1
+                        if least is None:
+                            least = (s, s0, r0, r1, tree_text(t0, g), tree_text(t1, g))
+    return cand, match, least
+
+
 def text_value(text: str, g: Grammar, pt: Sequence[int]) -> Optional[int]:
     """Re-evaluates a solution text ``(L op R)`` / leaf independently of any postfix code."""
     names = {v.name: i for i, v in enumerate(g.variables)}
@@ -157,7 +193,9 @@ def text_value(text: str, g: Grammar, pt: Sequence[int]) -> Optional[int]:
         if text[pos] == "(":
             pos += 1
             a = node()
-            op = text[pos]; pos += 1          # solutions use the five grammar operators only
+            op = text[pos]; pos += 1
+            if op in "<>" and text[pos] == op:  # a shift
+                op += op; pos += 1
             b = node()
             assert text[pos] == ")"; pos += 1
             if a is None or b is None:

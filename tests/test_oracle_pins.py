@@ -11,7 +11,7 @@ import pytest
 
 import oracle
 from tests import pybrute
-from xp_instances import (Hole, Sketch, Variable, config1, config2_grammar, config3, config4,
+from xp_instances import (Hole, JointHole, Sketch, Variable, config1, config2_grammar, config3, config4,
                           config5_instance, constant_set, free_grammar, parse_expr,
                           quasi_affine_grammar)
 
@@ -383,3 +383,107 @@ def test_loop_bound_hole_reading():
     assert r.match_count == match and (r.least_size, r.least_rank, r.least_text) == least
     texts = oracle.listing(g, 0, 3)
     assert (3, texts.index("(7-oh)")) in matches
+
+
+# ---------------------------------------------------------------------------------------------
+# shifts as operators; two holes inside one constraint
+# ---------------------------------------------------------------------------------------------
+
+def test_shift_semantics():
+    """<< is a multiplication by 2^b with wrap-around, >> the floor division by 2^b (sign kept);
+    a count outside 0..63 is undefined.  Checked against Python's unbounded integers."""
+    rnd = random.Random(7)
+    vs = [Variable("a", 0, 1), Variable("b", 0, 1)]
+    shl, shr = parse_expr("a<<b", vs), parse_expr("a>>b", vs)
+    cases = [(1, 0), (1, 63), (-1, 63), (-2 ** 63, 63), (-2 ** 63, 1), (2 ** 62, 1), (5, 64), (5, -1), (-7, 1), (7, 1)]
+    cases += [(rnd.randrange(-2 ** 63, 2 ** 63), rnd.randrange(-3, 67)) for _ in range(2000)]
+    for a, b in cases:
+        l, r = oracle.eval_code(shl, [a, b]), oracle.eval_code(shr, [a, b])
+        if b < 0 or b > 63:
+            assert l is None and r is None
+            continue
+        want = (a * 2 ** b) & (2 ** 64 - 1)
+        assert l == (want - 2 ** 64 if want >= 2 ** 63 else want)
+        assert r == a // 2 ** b
+    assert oracle.eval_code(parse_expr("(a<<1)<b+1", vs), [3, 6]) == 1        # precedence: + above << above <
+
+
+def test_shifts_as_grammar_operators_equal_brute_force():
+    vs = [Variable("i", 0, 5), Variable("j", -2, 3)]
+    g = free_grammar(vs, [1, 2, 64], ops=["+", "<<", ">>"])
+    for spec in ["(i<<2)+j", "i>>1", "(i+j)<<1", "j>>64"]:
+        sk = Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, vs))])
+        got = oracle.repair_hole(sk)
+        cand, match, least, _ = pybrute.repair(sk)
+        assert got.cand_count == cand and got.match_count == match
+        assert (got.solved, got.least_size, got.least_rank, got.least_text) == \
+            ((True,) + least if least else (False, 0, 0, ""))
+    sk = Sketch(g, [Hole(0, 5, spec_expr=parse_expr("(i<<2)+j", vs))])
+    assert oracle.repair_hole(sk).least_text == "(j+(i<<2))"
+
+
+def test_joint_counts_are_products_of_closed_forms():
+    vs = [Variable("i", 0, 3)]
+    g = free_grammar(vs, [0, 1, 2, 3], ops=["+", "-", "*"])                 # L = 5, B = 3
+    cnt = {1: 5, 3: 3 * 25, 5: 2 * 9 * 125}
+    J = JointHole((0, 0), (5, 3), parse_expr("HOLE0+HOLE1", vs), spec_expr=parse_expr("i", vs))
+    r = oracle.repair_joint(Sketch(g, [Hole(0, 1, spec_expr=parse_expr("i", vs))]), J)
+    want = [0] * 9
+    for s0 in (1, 3, 5):
+        for s1 in (1, 3):
+            want[s0 + s1] += cnt[s0] * cnt[s1]
+    assert r.cand_count == want
+
+
+def test_joint_hand_derived():
+    """ctx HOLE0*4 + HOLE1 against i*4 + j over i in [0,4), j in [0,4), leaves i j 0 1 4: part 1
+    must be j up to multiples of 4 moved into part 0; at total size 2 the only pair is (i, j); it is
+    the least.  At total size 4 the pairs are (size 1, size 3) and (size 3, size 1): with part 0 = i
+    the size-3 trees equal to j on the whole domain are j+0, 0+j, j-0, j*1, 1*j, j/1 and j%4 (j < 4):
+    seven; with part 1 = j the size-3 trees equal to i are the same seven forms of i: 14 in all."""
+    vs = [Variable("i", 0, 4), Variable("j", 0, 4)]
+    g = free_grammar(vs, [0, 1, 4])
+    base = Sketch(g, [Hole(0, 1, spec_expr=parse_expr("i", vs))])
+    J = JointHole((0, 0), (3, 3), parse_expr("(HOLE0*4)+HOLE1", vs), spec_expr=parse_expr("(i*4)+j", vs))
+    r = oracle.repair_joint(base, J)
+    assert r.cand_count[2] == 25 and r.match_count[2] == 1
+    assert (r.solved, r.least_total, r.least_size0, r.least_rank0, r.least_rank1, r.least_text0, r.least_text1) == \
+        (True, 2, 1, 0, 1, "i", "j")
+    assert r.match_count[4] == 14
+
+
+def test_joint_equals_brute_force():
+    rnd = random.Random(11)
+    vs = [Variable("p", 0, 3), Variable("q", -1, 2)]
+    cases = [(free_grammar(vs, [0, 2], ops=["+", "*"]), "(HOLE0*3)+HOLE1", "(p*3)+(q+2)", (3, 3)),
+             (free_grammar(vs, [1, -1], ops=["-", "/"]), "HOLE0-HOLE1", "p-(q/1)", (3, 3)),
+             (free_grammar(vs, [1, 2], ops=["+", "%"]), "HOLE1<HOLE0", "q<(p+1)", (3, 1)),
+             (quasi_affine_grammar(vs, [-1, 2], [1, 2]), "(HOLE0+HOLE1)*HOLE1", "(p+q)*q", (3, 3))]
+    for g, ctx, spec, K in cases:
+        sk = Sketch(g, [Hole(0, 1, spec_expr=parse_expr("p", vs))])
+        J = JointHole((0, 0), K, parse_expr(ctx, vs), spec_expr=parse_expr(spec, vs))
+        r = oracle.repair_joint(sk, J)
+        pts = pybrute.points_of(sk)
+        want = [pybrute.code_value(J.spec_expr, p) for p in pts]
+        cand, match, least = pybrute.repair_joint(g, J.start_nt, J.max_size, J.ctx, pts, want)
+        assert r.cand_count == cand and r.match_count == match
+        if least is None:
+            assert not r.solved
+        else:
+            assert (r.least_total, r.least_size0, r.least_rank0, r.least_rank1, r.least_text0, r.least_text1) == least
+    assert rnd is not None
+
+
+def test_joint_reduces_to_the_single_hole_search_when_one_part_is_cancelled():
+    """With a context that multiplies part 1 by zero and a grammar without division (every tree
+    defined everywhere), a pair matches iff part 0 matches on its own: the joint match count at
+    total size s is the sum over s0 + s1 = s of match_single[s0] * cnt[s1]."""
+    vs = [Variable("i", 0, 4), Variable("j", 0, 3)]
+    g = free_grammar(vs, [0, 1, 2], ops=["+", "-", "*"])
+    single = oracle.repair_hole(Sketch(g, [Hole(0, 5, spec_expr=parse_expr("(i*2)+j", vs))]))
+    cnt = oracle.counts(g, 0, 3)
+    J = JointHole((0, 0), (5, 3), parse_expr("HOLE0+(HOLE1*0)", vs), spec_expr=parse_expr("(i*2)+j", vs))
+    r = oracle.repair_joint(Sketch(g, [Hole(0, 1, spec_expr=parse_expr("i", vs))]), J)
+    for s in range(2, 9):
+        assert r.match_count[s] == sum(single.match_count[s0] * cnt[s - s0] for s0 in range(1, 6) if 1 <= s - s0 <= 3)
+    assert r.solved and r.least_size0 == single.least_size and r.least_rank0 == single.least_rank and r.least_rank1 == 0

@@ -17,9 +17,9 @@ from typing import List, Optional, Sequence, Tuple, Union
 
 import numpy as np
 
-# Operator codes.  The first five are the grammar operators; the rest may
-# only appear in context and spec expressions.
-OPS = ["+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"]
+# Operator codes.  The first five, min, max and the two shifts may appear in grammar
+# productions; all of them in context and spec expressions.
+OPS = ["+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||", "<<", ">>"]
 OP_CODE = {s: i for i, s in enumerate(OPS)}
 GRAMMAR_OPS = OPS[:5]
 
@@ -71,6 +71,19 @@ class Hole:
     spec_expr: Optional[List[Instr]] = None              # spec as expression ...
     spec_table: Optional[np.ndarray] = None              # ... or int64[n_points]
     note: str = ""                                       # e.g. text of the planted target
+
+
+@dataclass
+class JointHole:
+    """Two holes inside ONE constraint: ``ctx`` mentions ``HOLE0`` and ``HOLE1``; the candidates
+    are pairs of expressions (part 0 from ``start_nt[0]`` up to ``max_size[0]`` nodes, part 1
+    likewise) and the constraint is stated once for the pair."""
+    start_nt: Tuple[int, int]
+    max_size: Tuple[int, int]
+    ctx: List[Instr]
+    spec_expr: Optional[List[Instr]] = None
+    spec_table: Optional[np.ndarray] = None
+    note: str = ""
 
 
 @dataclass
@@ -144,7 +157,7 @@ def constant_set(lo: int, hi: int, extra: Sequence[int] = ()) -> List[int]:
 # Text <-> postfix for context / spec expressions (syntax only)
 # --------------------------------------------------------------------------
 
-_BINARY_LEVELS = [["||"], ["&&"], ["==", "!="], ["<", "<="], ["+", "-"], ["*", "/", "%"]]
+_BINARY_LEVELS = [["||"], ["&&"], ["==", "!="], ["<", "<="], ["<<", ">>"], ["+", "-"], ["*", "/", "%"]]
 
 
 def _tokenize(text: str) -> List[str]:
@@ -164,7 +177,7 @@ def _tokenize(text: str) -> List[str]:
             while j < n and text[j].isdigit():
                 j += 1
             toks.append(text[i:j]); i = j
-        elif text[i:i + 2] in ("<=", "==", "!=", "&&", "||"):
+        elif text[i:i + 2] in ("<<", ">>", "<=", "==", "!=", "&&", "||"):
             toks.append(text[i:i + 2]); i += 2
         elif ch in "+-*/%<(),":
             toks.append(ch); i += 1
@@ -174,7 +187,8 @@ def _tokenize(text: str) -> List[str]:
 
 
 def parse_expr(text: str, variables: Sequence[Variable]) -> List[Instr]:
-    """Infix text -> postfix instruction list.  ``HOLE`` names the hole; ``min(a,b)``
+    """Infix text -> postfix instruction list.  ``HOLE`` names the hole (``HOLE0``, ``HOLE1`` the
+    parts of a joint sketch); ``<<`` and ``>>`` bind tighter than comparisons and looser than ``+``; ``min(a,b)``
     and ``max(a,b)`` are calls; a minus sign directly before a number literal in
     operand position is part of the literal (there is no unary minus operator)."""
     names = {v.name: i for i, v in enumerate(variables)}
@@ -206,8 +220,8 @@ def parse_expr(text: str, variables: Sequence[Variable]) -> List[Instr]:
         elif t in ("min", "max"):
             take("("); level(0); take(","); level(0); take(")")
             out.append((K_OP, OP_CODE[t], 0))
-        elif t == "HOLE":
-            out.append((K_HOLE, 0, 0))
+        elif t == "HOLE" or (t.startswith("HOLE") and t[4:].isdigit()):
+            out.append((K_HOLE, int(t[4:] or 0), 0))      # HOLE = HOLE0; HOLE1, ... name the other parts of a joint sketch
         elif t in names:
             out.append((K_VAR, names[t], 0))
         else:
@@ -238,7 +252,7 @@ def postfix_to_text(code: Sequence[Instr], variables: Sequence[Variable]) -> str
         elif kind == K_CONST:
             st.append(str(int(value)))
         elif kind == K_HOLE:
-            st.append("HOLE")
+            st.append("HOLE" if arg == 0 else f"HOLE{arg}")
         else:
             r = st.pop(); l = st.pop()
             s = OPS[arg]
