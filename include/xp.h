@@ -67,13 +67,14 @@ enum {
     XP_MAX_CODE = 64          /* instructions in one context or spec expression */
 };
 
-/* Operators.  The first five and MIN, MAX may appear in grammar productions (min and max let a
- * hole express the bound of a remainder tile, e.g. min(T, N - io*T)); all of them in context and
- * spec expressions. */
+/* Operators.  The first five, MIN, MAX and the shifts may appear in grammar productions (min and max
+ * let a hole express the bound of a remainder tile, e.g. min(T, N - io*T); shifts are what strength-
+ * reduced index arithmetic uses); all of them in context and spec expressions.  A shift count outside
+ * 0..63 makes the candidate fail at the point, like a zero divisor; << wraps around, >> keeps the sign. */
 enum {
     XP_OP_ADD = 0, XP_OP_SUB = 1, XP_OP_MUL = 2, XP_OP_DIV = 3, XP_OP_MOD = 4,
     XP_OP_LT = 5, XP_OP_LE = 6, XP_OP_EQ = 7, XP_OP_NE = 8, XP_OP_MIN = 9, XP_OP_MAX = 10,
-    XP_OP_AND = 11, XP_OP_OR = 12
+    XP_OP_AND = 11, XP_OP_OR = 12, XP_OP_SHL = 13, XP_OP_SHR = 14
 };
 
 /* Variables of the snippet: name (copied) and range lo <= v < hi. */
@@ -85,7 +86,7 @@ typedef struct {
     int32_t lhs;        /* nonterminal index, 0 <= lhs < n_nonterminals */
     int32_t kind;       /* XP_PROD_* */
     int32_t var;        /* XP_PROD_VAR: variable index */
-    int32_t op;         /* XP_PROD_BIN: XP_OP_ADD .. XP_OP_MOD, XP_OP_MIN, XP_OP_MAX */
+    int32_t op;         /* XP_PROD_BIN: XP_OP_ADD .. XP_OP_MOD, XP_OP_MIN, XP_OP_MAX, XP_OP_SHL, XP_OP_SHR */
     int32_t left;       /* XP_PROD_BIN: nonterminal of the left operand */
     int32_t right;      /* XP_PROD_BIN: nonterminal of the right operand */
     int64_t value;      /* XP_PROD_CONST: the constant */
@@ -182,7 +183,7 @@ typedef struct {
     uint64_t least_rank;
     const xp_instr* least_code;     /* postfix of the least solution */
     int32_t least_len;
-    const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))"; min and max as calls, "min(a,b)" */
+    const char* least_text;         /* fully parenthesised infix, e.g. "(j+(i*8))", "(i<<2)"; min and max as calls, "min(a,b)" */
     uint64_t evals_executed;        /* candidate-point evaluations that ran for this hole: filter_tests plus the exact
                                        evaluations of stage 2 (a hit at a probe point) and stage 3 (a survivor at a
                                        domain point).  Candidates decided without a test are not in here. */
@@ -207,7 +208,7 @@ typedef struct {
 
 /* Grammar (Section 4.4: the expressions the synthesis step may put into a hole).  Builds the
  * per-(nonterminal, size) candidate counts and rank offsets on the host; no GPU is touched.
- * Errors: XP_ERR_GRAMMAR (bad indices, operator outside + - * / % min max), XP_ERR_TOO_LARGE. */
+ * Errors: XP_ERR_GRAMMAR (bad indices, operator outside + - * / % min max << >>), XP_ERR_TOO_LARGE. */
 xp_status xp_grammar_create(const xp_grammar_desc* desc, xp_grammar** out);
 void xp_grammar_destroy(xp_grammar* g);
 
@@ -325,6 +326,88 @@ xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_opts* opts, 
  * the number of entries `out` holds; *n_out (may be NULL) receives the number written.
  * Errors: XP_ERR_INVALID_ARG (null result, out too short). */
 xp_status xp_result_pack(const xp_result* const* results, size_t n, xp_hole_summary* out, size_t out_cap, size_t* n_out);
+
+/* Two holes inside ONE constraint (a product search, for small products): `ctx` mentions both parts
+ * (XP_I_HOLE with arg = 0 or 1) and the constraint "ctx(e0(p), e1(p), p) == spec(p) at every point p" is
+ * stated for the PAIR (e0, e1), e_k a tree of start_nt[k] with at most max_size[k] nodes.  Where a snippet's
+ * missing expressions cannot be given a spec of their own each (a wrong stride AND a wrong offset inside
+ * one index), this is the form SynthesisCode's query takes.  The pairs are ordered by total size s0 + s1,
+ * then s0, then the rank of e0, then the rank of e1; counts are per total size.  Domain, variables and
+ * grammar are those of `sketch` (its own holes play no role).  Every candidate of either part up to its
+ * bound is tabulated at up to 16 probe points (so each count per size must stay below 2^22), every pair
+ * is tested on the probes from the tables, and a pair that passes them is checked on the whole domain.
+ * Errors: XP_ERR_INVALID_ARG, XP_ERR_SKETCH (malformed ctx / spec, ctx without both parts),
+ * XP_ERR_TOO_LARGE (a count of 2^22 or more, or more than 2^40 pairs), XP_ERR_NOMEM, XP_ERR_CUDA. */
+typedef struct {
+    int32_t start_nt[2], max_size[2];
+    int32_t ctx_len; const xp_instr* ctx;
+    int32_t spec_kind;              /* XP_SPEC_EXPR or XP_SPEC_TABLE */
+    int32_t spec_len; const xp_instr* spec_expr;
+    const int64_t* spec_table;      /* n_points values, point order of the domain */
+    int32_t spec_table_on_device;
+} xp_joint_desc;
+typedef struct xp_joint_result xp_joint_result;
+typedef struct {
+    int32_t solved, max_total;      /* max_total = max_size[0] + max_size[1] */
+    const uint64_t* cand_count;     /* [max_total + 1], index = total size of the pair */
+    const uint64_t* match_count;
+    int32_t least_total, least_size[2];
+    uint64_t least_rank[2];
+    const char* least_text[2];
+    uint64_t evals_executed;        /* (pair, point) evaluations that ran: probe tests and whole-domain points */
+    uint64_t probe_survivors;       /* pairs that passed every probe point */
+    double kernel_ms, total_ms;
+    int32_t n_launches;
+} xp_joint_view;
+xp_status xp_repair_joint(const xp_sketch* sketch, const xp_joint_desc* joint, const xp_repair_opts* opts, xp_joint_result** out);
+xp_status xp_joint_result_get(const xp_joint_result* r, xp_joint_view* out);
+void xp_joint_result_free(xp_joint_result* r);
+
+/* Algorithm 3 from end to end for one expression: the source snippet's expression S_s and the
+ * erroneous expression S_e that the transformed program computes in its place go in, the repaired
+ * expression comes out.
+ *   GenerateCodeSketch: every subtree of S_e in turn is taken out and replaced by a hole, giving one
+ *     single-hole sketch per node of S_e (context = the rest of S_e);
+ *   CreateSMTQuery: the constraint per concrete index is "sketch == S_s at this point" over the box of
+ *     the grammar's variables; where the two snippets iterate over different variables (a loop that the
+ *     pass split, fused or bound to threads), var_map gives the value of each source variable as an
+ *     expression over the grammar's (= the transformed program's) variables, and S_s is rewritten with it;
+ *   SynthesisCode: all sketches are searched in one batch (xp_sketch_load_batch + xp_repair_batch);
+ *   StitchBack: among the sketches that have a solution the one with the smallest solution is taken
+ *     (ties: the smallest subtree taken out, then the leftmost) and its solution is put in place of
+ *     the subtree.
+ * S_s is postfix over source variables (XP_I_VAR arg < n_source_vars) and constants; S_e postfix over the
+ * grammar's variables and constants; both may use every operator.  var_map may be NULL when the snippets
+ * share their variables (n_source_vars must then equal the grammar's n_vars).
+ * Errors: XP_ERR_INVALID_ARG, XP_ERR_SKETCH (malformed expression, rewritten spec longer than XP_MAX_CODE),
+ * and those of the load and the search. */
+typedef struct {
+    const xp_instr* source;    int32_t source_len;       /* S_s */
+    const xp_instr* erroneous; int32_t erroneous_len;    /* S_e */
+    int32_t n_source_vars;
+    const xp_instr* const* var_map;                      /* [n_source_vars] postfix expressions, or NULL */
+    const int32_t* var_map_len;
+    int32_t start_nt, max_size;                          /* what a hole is filled from */
+} xp_pair_desc;
+typedef struct xp_pair_result xp_pair_result;
+typedef struct {
+    int32_t solved;                 /* some single-subtree replacement makes S_e agree with S_s everywhere */
+    int32_t n_sketches;             /* sketches generated (= nodes of S_e) and searched */
+    int32_t node_first, node_last;  /* the subtree taken out: instructions [node_first, node_last] of S_e */
+    int32_t least_size;             /* the solution that replaced it */
+    uint64_t least_rank;
+    const char* hole_text;          /* ... as text */
+    const char* sketch_text;        /* S_e with HOLE in place of the subtree */
+    const char* stitched_text;      /* the repaired expression */
+    const xp_instr* stitched_code;  /* ... and as postfix */
+    int32_t stitched_len;
+    uint64_t candidates;            /* candidates of all sketches together */
+    uint64_t evals_executed;
+    double load_ms, search_ms;
+} xp_pair_view;
+xp_status xp_repair_pair(const xp_grammar* g, const xp_pair_desc* desc, xp_pair_result** out);
+xp_status xp_pair_result_get(const xp_pair_result* r, xp_pair_view* out);
+void xp_pair_result_free(xp_pair_result* r);
 
 /* Message of the calling thread's last failed call ("" if none). */
 const char* xp_last_error(void);

@@ -25,7 +25,9 @@ _STATUS = {0: "XP_OK", 1: "XP_ERR_INVALID_ARG", 2: "XP_ERR_GRAMMAR", 3: "XP_ERR_
 EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_grammar_unrank",
            "xp_sketch_load", "xp_sketch_load_batch", "xp_sketch_destroy", "xp_workspace_bytes", "xp_repair", "xp_repair_batch",
            "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static",
-           "xp_sketch_info_get", "xp_sketch_refine", "xp_result_pack"]
+           "xp_sketch_info_get", "xp_sketch_refine", "xp_result_pack",
+           "xp_repair_pair", "xp_pair_result_get", "xp_pair_result_free",
+           "xp_repair_joint", "xp_joint_result_get", "xp_joint_result_free"]
 
 
 class XpError(RuntimeError):
@@ -97,6 +99,33 @@ class xp_hole_summary(C.Structure):
                 ("least_text", C.c_char * 256)]
 
 
+class xp_pair_desc(C.Structure):
+    _fields_ = [("source", C.POINTER(xp_instr)), ("source_len", C.c_int32), ("erroneous", C.POINTER(xp_instr)),
+                ("erroneous_len", C.c_int32), ("n_source_vars", C.c_int32), ("var_map", C.POINTER(C.POINTER(xp_instr))),
+                ("var_map_len", C.POINTER(C.c_int32)), ("start_nt", C.c_int32), ("max_size", C.c_int32)]
+
+
+class xp_pair_view(C.Structure):
+    _fields_ = [("solved", C.c_int32), ("n_sketches", C.c_int32), ("node_first", C.c_int32), ("node_last", C.c_int32),
+                ("least_size", C.c_int32), ("least_rank", C.c_uint64), ("hole_text", C.c_char_p),
+                ("sketch_text", C.c_char_p), ("stitched_text", C.c_char_p), ("stitched_code", C.POINTER(xp_instr)),
+                ("stitched_len", C.c_int32), ("candidates", C.c_uint64), ("evals_executed", C.c_uint64),
+                ("load_ms", C.c_double), ("search_ms", C.c_double)]
+
+
+class xp_joint_desc(C.Structure):
+    _fields_ = [("start_nt", C.c_int32 * 2), ("max_size", C.c_int32 * 2), ("ctx_len", C.c_int32), ("ctx", C.POINTER(xp_instr)),
+                ("spec_kind", C.c_int32), ("spec_len", C.c_int32), ("spec_expr", C.POINTER(xp_instr)),
+                ("spec_table", C.c_void_p), ("spec_table_on_device", C.c_int32)]
+
+
+class xp_joint_view(C.Structure):
+    _fields_ = [("solved", C.c_int32), ("max_total", C.c_int32), ("cand_count", C.POINTER(C.c_uint64)),
+                ("match_count", C.POINTER(C.c_uint64)), ("least_total", C.c_int32), ("least_size", C.c_int32 * 2),
+                ("least_rank", C.c_uint64 * 2), ("least_text", C.c_char_p * 2), ("evals_executed", C.c_uint64),
+                ("probe_survivors", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double), ("n_launches", C.c_int32)]
+
+
 _lib = None
 
 
@@ -131,6 +160,14 @@ def load(path: Optional[str] = None):
     lib.xp_sketch_info_get.argtypes = [vp, C.POINTER(xp_sketch_info)]
     lib.xp_sketch_refine.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32)]
     lib.xp_result_pack.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_hole_summary), C.c_size_t, C.POINTER(C.c_size_t)]
+    lib.xp_repair_joint.argtypes = [vp, C.POINTER(xp_joint_desc), C.POINTER(xp_repair_opts), C.POINTER(vp)]
+    lib.xp_joint_result_get.argtypes = [vp, C.POINTER(xp_joint_view)]
+    lib.xp_joint_result_free.argtypes = [vp]
+    lib.xp_joint_result_free.restype = None
+    lib.xp_repair_pair.argtypes = [vp, C.POINTER(xp_pair_desc), C.POINTER(vp)]
+    lib.xp_pair_result_get.argtypes = [vp, C.POINTER(xp_pair_view)]
+    lib.xp_pair_result_free.argtypes = [vp]
+    lib.xp_pair_result_free.restype = None
     for name in EXPORTS:
         getattr(lib, name)
     _lib = lib
@@ -419,6 +456,109 @@ def summaries_as_numpy(packed) -> np.ndarray:
     """A structured numpy view (no copy) of an array of ``xp_hole_summary``."""
     assert C.sizeof(xp_hole_summary) == SUMMARY_DTYPE.itemsize
     return np.frombuffer(packed, dtype=SUMMARY_DTYPE)
+
+
+@dataclass
+class JointResult:
+    solved: bool
+    cand_count: List[int]          # index = total size of the pair
+    match_count: List[int]
+    least_total: int
+    least_size0: int
+    least_rank0: int
+    least_rank1: int
+    least_text0: str
+    least_text1: str
+    evals_executed: int
+    probe_survivors: int
+    kernel_ms: float
+    total_ms: float
+    n_launches: int
+
+
+def xp_repair_joint(sketch: LoadedSketch, joint, stream=None) -> JointResult:
+    """``joint``: an ``xp_instances.JointHole`` (two parts inside one constraint) searched over the
+    domain and grammar of ``sketch``."""
+    lib = load()
+    d = xp_joint_desc()
+    d.start_nt[0], d.start_nt[1] = joint.start_nt
+    d.max_size[0], d.max_size[1] = joint.max_size
+    ctx = _code(joint.ctx)
+    d.ctx_len, d.ctx = len(joint.ctx), ctx
+    keep = [ctx]
+    if joint.spec_table is not None:
+        table = joint.spec_table
+        if isinstance(table, np.ndarray):
+            table = np.ascontiguousarray(table, dtype=np.int64)
+        d.spec_kind = 1
+        d.spec_table, d.spec_table_on_device, k = _ptr_of(table)
+        keep.append(k)
+    else:
+        se = _code(joint.spec_expr); keep.append(se)
+        d.spec_kind, d.spec_len, d.spec_expr = 0, len(joint.spec_expr), se
+    o, _keep = _opts(stream=stream)
+    out = C.c_void_p()
+    _check(lib.xp_repair_joint(sketch.handle, C.byref(d), C.byref(o), C.byref(out)))
+    try:
+        v = xp_joint_view()
+        _check(lib.xp_joint_result_get(out.value, C.byref(v)))
+        K = v.max_total
+        return JointResult(bool(v.solved), [int(v.cand_count[k]) for k in range(K + 1)], [int(v.match_count[k]) for k in range(K + 1)],
+                           int(v.least_total), int(v.least_size[0]), int(v.least_rank[0]), int(v.least_rank[1]),
+                           (v.least_text[0] or b"").decode(), (v.least_text[1] or b"").decode(), int(v.evals_executed),
+                           int(v.probe_survivors), float(v.kernel_ms), float(v.total_ms), int(v.n_launches))
+    finally:
+        lib.xp_joint_result_free(out.value)
+
+
+@dataclass
+class PairResult:
+    solved: bool
+    n_sketches: int
+    node_first: int
+    node_last: int
+    least_size: int
+    least_rank: int
+    hole_text: str
+    sketch_text: str
+    stitched_text: str
+    stitched_code: List[Tuple[int, int, int]]
+    candidates: int
+    evals_executed: int
+    load_ms: float
+    search_ms: float
+
+
+def xp_repair_pair(gr: Grammar, source, erroneous, start_nt: int, max_size: int, var_map=None, n_source_vars=None) -> PairResult:
+    """``source`` / ``erroneous``: postfix instruction lists; ``var_map``: per source variable its value
+    as a postfix list over the grammar's variables (None: the snippets share their variables)."""
+    lib = load()
+    d = xp_pair_desc()
+    src, err = _code(source), _code(erroneous)
+    d.source, d.source_len, d.erroneous, d.erroneous_len = src, len(source), err, len(erroneous)
+    d.start_nt, d.max_size = start_nt, max_size
+    keep = []
+    if var_map is not None:
+        arrs = [_code(m) for m in var_map]
+        keep.append(arrs)
+        ptrs = (C.POINTER(xp_instr) * len(var_map))(*[C.cast(a, C.POINTER(xp_instr)) for a in arrs])
+        lens = (C.c_int32 * len(var_map))(*[len(m) for m in var_map])
+        d.var_map, d.var_map_len, d.n_source_vars = ptrs, lens, len(var_map)
+        keep += [ptrs, lens]
+    else:
+        d.n_source_vars = n_source_vars if n_source_vars is not None else len(gr.model.variables)
+    out = C.c_void_p()
+    _check(lib.xp_repair_pair(gr.handle, C.byref(d), C.byref(out)))
+    try:
+        v = xp_pair_view()
+        _check(lib.xp_pair_result_get(out.value, C.byref(v)))
+        return PairResult(bool(v.solved), int(v.n_sketches), int(v.node_first), int(v.node_last), int(v.least_size),
+                          int(v.least_rank), (v.hole_text or b"").decode(), (v.sketch_text or b"").decode(),
+                          (v.stitched_text or b"").decode(),
+                          [(v.stitched_code[i].kind, v.stitched_code[i].arg, v.stitched_code[i].value) for i in range(v.stitched_len)],
+                          int(v.candidates), int(v.evals_executed), float(v.load_ms), float(v.search_ms))
+    finally:
+        lib.xp_pair_result_free(out.value)
 
 
 def xp_int32_peak() -> Tuple[float, float]:

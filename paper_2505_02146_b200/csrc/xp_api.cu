@@ -30,6 +30,10 @@ static xp_status fail(xp_status st, const std::string& msg) {
     return st;
 }
 
+namespace xp {
+xp_status set_error(xp_status st, const char* msg) { return fail(st, msg); }      // for the library's other source files
+}
+
 #define XP_CUDA(call)                                                                          \
     do {                                                                                       \
         cudaError_t e_ = (call);                                                               \
@@ -119,7 +123,7 @@ void pool_release(void* ptr, size_t bytes, int device) {
 struct xp_sketch;
 static xp_status check_device(const xp_sketch* const* sk, size_t n);
 
-static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||"};
+static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||", "<<", ">>"};
 
 // ------------------------------------------------------------------------------------------
 // grammar
@@ -190,7 +194,7 @@ extern "C" xp_status xp_grammar_create(const xp_grammar_desc* d, xp_grammar** ou
         const xp_production& p = d->productions[i];
         bool ok = p.lhs >= 0 && p.lhs < g->n_nt;
         if (p.kind == XP_PROD_VAR) ok = ok && p.var >= 0 && p.var < g->n_vars;
-        else if (p.kind == XP_PROD_BIN) ok = ok && ((p.op >= XP_OP_ADD && p.op <= XP_OP_MOD) || p.op == XP_OP_MIN || p.op == XP_OP_MAX) && p.left >= 0 && p.left < g->n_nt && p.right >= 0 && p.right < g->n_nt;
+        else if (p.kind == XP_PROD_BIN) ok = ok && ((p.op >= XP_OP_ADD && p.op <= XP_OP_MOD) || p.op == XP_OP_MIN || p.op == XP_OP_MAX || p.op == XP_OP_SHL || p.op == XP_OP_SHR) && p.left >= 0 && p.left < g->n_nt && p.right >= 0 && p.right < g->n_nt;
         else if (p.kind != XP_PROD_CONST) ok = false;
         if (!ok) { delete g; return fail(XP_ERR_GRAMMAR, "production " + std::to_string(i) + " is malformed"); }
         g->prods.push_back(p);
@@ -377,7 +381,7 @@ static bool check_code(const xp_instr* code, int n, int n_vars, bool hole_allowe
     for (int i = 0; i < n; ++i) {
         const xp_instr& c = code[i];
         if (c.kind == XP_I_OP) {
-            if (c.arg < XP_OP_ADD || c.arg > XP_OP_OR || sp < 2) return false;
+            if (c.arg < XP_OP_ADD || c.arg > XP_OP_SHR || sp < 2) return false;
             --sp;
         } else {
             if (c.kind == XP_I_VAR) { if (c.arg < 0 || c.arg >= n_vars) return false; }
@@ -761,6 +765,15 @@ extern "C" xp_status xp_sketch_load(const xp_grammar* g, const xp_sketch_desc* d
     return xp_sketch_load_batch(&g, d, 1, out);
 }
 
+namespace xp {
+SketchInternals sketch_internals(const xp_sketch* s) { return SketchInternals{s->d_s, s->g, s->n_points, s->arena_device, s->g->n_vars}; }
+u64 grammar_cnt(const xp_grammar* g, int nt, int size) { return g->cnt[nt][size]; }
+int grammar_nonterminals(const xp_grammar* g) { return g->n_nt; }
+int grammar_ok_size(const xp_grammar* g) { return g->ok_size; }
+cudaError_t device_alloc(void** out, size_t bytes, int* device, size_t* granted) { return pool_alloc(out, bytes, device, granted); }
+void device_release(void* ptr, size_t granted, int device) { pool_release(ptr, granted, device); }
+}  // namespace xp
+
 extern "C" xp_status xp_sketch_info_get(const xp_sketch* s, xp_sketch_info* out) {
     if (!s || !out) return fail(XP_ERR_INVALID_ARG, "xp_sketch_info_get: null argument");
     memset(out, 0, sizeof(*out));
@@ -881,8 +894,6 @@ struct Plan {
     std::vector<AccDev> acc;
     std::vector<u64> nominal_ops;    // per accumulator: cost-model operations of the filter stage
     u64 n_tickets = 0;
-    std::vector<u64> groups;         // first ticket of every group of tickets, and the end (empty: no grouping)
-    u64 n_items() const { return groups.empty() ? n_tickets : (u64)groups.size() - 1; }
 };
 
 // Scratch of calls that bring no workspace: one block per process, reused while no other call
@@ -957,6 +968,7 @@ static void add_tiles(Plan* plan, const xp_grammar* g, int nt, int sketch, int h
             sg->op_base[sg->n_ops] = this_base;
             sg->n_ops += 1;
             if (bd.op == XP_OP_DIV || bd.op == XP_OP_MOD) sg->has_div = 1;
+            if (bd.op == XP_OP_SHL || bd.op == XP_OP_SHR) sg->generic = 1;
         }
     }
     // Families: segments with the same register-side operands and a single broadcast tile are
@@ -1028,35 +1040,6 @@ static xp_status check_device(const xp_sketch* const* sk, size_t n) {
     return XP_OK;
 }
 
-// Plans over many holes (batches of small sketches) hand the CTAs runs of consecutive tickets of one
-// hole instead of single tickets: a CTA that stays with a hole flushes its private results once and
-// fills the hole's broadcast operands once.  A run never crosses into another hole and is at most
-// as long as leaves about eight runs per resident CTA (load balance).  Plans over few holes (large
-// searches) keep single tickets: their tickets are long, and a run of them would unbalance the end.
-constexpr size_t kGroupMinAccs = 256;
-constexpr u64 kGroupCtas = 148 * 3;
-static void group_tickets(Plan* plan) {
-    plan->groups.clear();
-#ifdef XP_NO_GROUPS
-    return;
-#endif
-    if (plan->acc.size() < kGroupMinAccs || plan->n_tickets == 0) return;
-    u64 most = plan->n_tickets / (kGroupCtas * 8);
-    most = most < 1 ? 1 : (most > 64 ? 64 : most);
-    if (most == 1) return;
-    int cur_acc = -1;
-    u64 cur_len = 0;
-    for (size_t i = 0; i < plan->segs.size(); ++i) {
-        const SegDev& c = plan->segs[i];
-        const u64 end = i + 1 < plan->segs.size() ? plan->segs[i + 1].first_ticket : plan->n_tickets;
-        for (u64 t = c.first_ticket; t < end; ++t) {
-            if (c.acc != cur_acc || cur_len == most) { plan->groups.push_back(t); cur_acc = c.acc; cur_len = 0; }
-            ++cur_len;
-        }
-    }
-    plan->groups.push_back(plan->n_tickets);
-}
-
 static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repair_opts* o, Plan* plan) {
     const bool plain = o->size_min <= 0 && o->size_max <= 0 && o->n_rank_ranges == 0 && o->flags == 0;
     if (n > 16) { plan->segs.reserve(n * 8); plan->acc.reserve(n * 2); plan->nominal_ops.reserve(n * 2); }
@@ -1090,7 +1073,6 @@ static xp_status build_plan(const xp_sketch* const* sk, size_t n, const xp_repai
         }
         plan->n_tickets += s->plan_tickets;
     }
-    group_tickets(plan);
     return XP_OK;
 }
 
@@ -1137,14 +1119,12 @@ static u32 surv_cap_for(size_t n_sketches) {
 }
 constexpr u32 kSurvCapStatic = 8192;         // ... of a call on the library's fixed scratch
 
-static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap, size_t n_group_entries = 0) {
+static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u32 surv_cap) {
     SearchLayout w;
     w.segs = 256;
     w.sketches = w.segs + align256(sizeof(SegDev) * (n_segs + 1));
     w.acc = w.sketches + align256(sizeof(SketchDev*) * (n_sketches + 1));
-    w.groups = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
-    w.n_groups = n_group_entries ? n_group_entries - 1 : 0;
-    w.hist = w.groups + align256(sizeof(u64) * n_group_entries);
+    w.hist = w.acc + align256(sizeof(AccDev) * (n_acc + 1));
     w.head = w.hist + align256(sizeof(u32) * (n_acc + 1));
     w.surv = w.head;
     w.sort_off = w.surv + align256(sizeof(SurvDev) * (size_t)surv_cap);
@@ -1166,7 +1146,7 @@ extern "C" size_t xp_workspace_bytes(const xp_sketch* const* sketches, size_t n,
     if (!sketches || n == 0) return 0;
     Plan plan;
     if (build_plan(sketches, n, opts ? opts : &kDefaultOpts, &plan) != XP_OK) return 0;
-    return ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n), plan.groups.size()).total;
+    return ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n)).total;
 }
 
 extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n, const xp_repair_opts* opts,
@@ -1183,7 +1163,7 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
-    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n), plan.groups.size());
+    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
     char* ws = (char*)o->workspace;
     bool own_ws = false, cached_ws = false;
     if (ws) {
@@ -1210,7 +1190,6 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (!plan.segs.empty()) memcpy(&stage[w.segs], plan.segs.data(), sizeof(SegDev) * plan.segs.size());
     for (size_t i = 0; i < n; ++i) ((const SketchDev**)&stage[w.sketches])[i] = sketches[i]->d_s;
     memcpy(&stage[w.acc], plan.acc.data(), sizeof(AccDev) * plan.acc.size());
-    if (!plan.groups.empty()) memcpy(&stage[w.groups], plan.groups.data(), sizeof(u64) * plan.groups.size());
 
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     float ms = 0.f;
@@ -1228,11 +1207,11 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     const u32 max_chunks = max_chunks_of(sketches, n);
     xp_status stopped = XP_OK;
     if (!o->cancel && o->timeout_ms <= 0) {
-        XP_CUDA_R(launch_search_part(ws, w, 0, plan.n_items(), false, n_segs, (int)n, max_chunks, stream, &launches));
+        XP_CUDA_R(launch_search_part(ws, w, 0, plan.n_tickets, false, n_segs, (int)n, max_chunks, stream, &launches));
     } else {
         // Bounded launches: the host waits for each and then looks at the cancel word and the clock.
         // Nothing on the device waits for either, and when the call gives up no kernel is in flight.
-        const u64 n_items = plan.n_items();               // (an item is a ticket, or a short run of them)
+        const u64 n_items = plan.n_tickets;
         for (u64 t = 0; t < n_items && stopped == XP_OK; t += (u64)XP_CANCEL_TICKETS) {
             const u64 t_end = t + (u64)XP_CANCEL_TICKETS < n_items ? t + (u64)XP_CANCEL_TICKETS : n_items;
             XP_CUDA_R(launch_search_part(ws, w, t, t_end, t > 0, n_segs, (int)n, max_chunks, stream, &launches));

@@ -166,6 +166,8 @@ struct SegDev {
     u64 right_count;                 // trees of the right operand (rank = base + l * right_count + r)
     u32 reg_tiles, bc_tiles;         // tickets = reg_tiles * bc_tiles
     i32 has_div;                     // some production of the group is / or %
+    i32 generic;                     // some production of the group has no 32-bit filter loop (the shifts): the group's
+                                     // candidates are evaluated exactly, in 64 bits, at the probe
     i32 bc_base, bc_keep;            // slots [bc_base, bc_base + bc_count) of the CTA's broadcast tile belong to this
                                      // segment; bc_keep (first of a family): all members' broadcast operands fit the
                                      // tile side by side and do not depend on the ticket, so a CTA fills them once
@@ -184,14 +186,9 @@ constexpr u32 kSurvFailed = 0x80000000u;
 struct SurvDev { u64 rank; i32 sketch, hole, size, acc; u32 state, vars; };   // vars: variables the candidate mentions
 
 struct PlanDev {
-    // What a CTA takes from the counter is a WORK ITEM: one ticket, or (group_first != null) the run of
-    // consecutive tickets [group_first[i], group_first[i+1]) of one hole.  Plans of many small sketches
-    // are grouped, so that a CTA stays with a hole for several tickets (one flush of its private
-    // results, operands filled once) instead of meeting a new hole at every ticket.
-    u64 item_base;                   // items [item_base, n_items) belong to this launch (a search that polls a cancel
-                                     // word is cut into several launches); the counter starts at zero each time
-    u64 n_items;
-    const u64* group_first;          // device, n_items + 1 entries, or null: item i is ticket i
+    u64 ticket_base;                 // tickets [ticket_base, n_tickets) belong to this launch (a search that polls a
+                                     // cancel word is cut into several launches); the counter starts at zero each time
+    u64 n_tickets;
     i32 n_segs, n_sketches;
     const SegDev* segs;              // device
     const SketchDev* const* sketches;  // device table of device pointers

@@ -12,7 +12,7 @@ namespace xp {
 // instead of the bad index.  Nothing traps, spins or faults: the search finishes, and the host
 // turns a recorded code into an error status.
 #ifdef XP_CHECKS
-__device__ unsigned int g_check_word;
+static __device__ unsigned int g_check_word;      // (one per source file; the search kernels' copy is the one the host reads)
 __device__ __forceinline__ bool xp_checked(bool cond, unsigned int code) {
     if (!cond) atomicCAS(&g_check_word, 0u, code);
     return cond;
@@ -49,6 +49,8 @@ __device__ __forceinline__ bool apply_op(int op, i64 a, i64 b, i64& r) {
         case XP_OP_MAX: r = a > b ? a : b; return true;
         case XP_OP_AND: r = (a != 0) & (b != 0); return true;
         case XP_OP_OR: r = (a != 0) | (b != 0); return true;
+        case XP_OP_SHL: r = (i64)((u64)a << (b & 63)); return b >= 0 && b <= 63;
+        case XP_OP_SHR: r = a >> (b & 63); return b >= 0 && b <= 63;      // (device >> on a signed value keeps the sign)
     }
     return false;
 }
@@ -62,7 +64,7 @@ __device__ __forceinline__ void divmod_u64(u64 n, u64 d, u64& q, u64& r) {
 // code[i] is a leaf index into GrammarDev::leaves, or kOpBit | operator.  Returns the length
 // (== size).  Walks the tree with an explicit stack: a frame is a subtree still to be
 // expanded, or (size 0) an operator to be emitted after its operands.
-__device__ __noinline__ int unrank(const GrammarDev* __restrict__ g, int nt, int size, u64 rank, u32* code) {
+static __device__ __noinline__ int unrank(const GrammarDev* __restrict__ g, int nt, int size, u64 rank, u32* code) {
     struct Frame { u64 rank; i32 nt; i32 size; };
     Frame st[kMaxSize + 1];
     int sp = 0, n = 0;

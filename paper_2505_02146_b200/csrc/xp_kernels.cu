@@ -360,7 +360,7 @@ struct MemberState {
 };
 
 struct EvalShared {
-    u64 item;
+    u64 ticket;
     i32 seg_index;
     SegDev seg;
     CandShared wcand[kWarps];    // per warp: the candidate of a whole-domain check the warp does itself
@@ -395,12 +395,6 @@ struct EvalShared {
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
     u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21 | member << 24
-    // The register-side operands of the ticket at hand, one column per thread ([j][thread]; a thread
-    // reads and writes only its own column, so nothing synchronises on them): low and high words of
-    // the values at probe 0, and the values at probe 1 (second look).  The loops copy their column
-    // into registers when they start; keeping the columns here rather than in per-thread local
-    // memory keeps them out of the L1 cache, which the frames of all resident threads overflow.
-    u32 rv[kNA][kThreads], rh[kNA][kThreads], r1[kNA][kThreads];
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
@@ -485,6 +479,8 @@ __device__ __noinline__ void stage_candidate(CandShared& c, const SketchDev* sk,
                 case XP_OP_DIV: m = a; break;
                 case XP_OP_MOD: m = a < b ? a : b; break;
                 case XP_OP_MIN: case XP_OP_MAX: m = a > b ? a : b; break;
+                case XP_OP_SHL: m = kSat; break;
+                case XP_OP_SHR: m = a; break;
                 default: m = 1; break;
             }
             mag[sp - 1] = m < kSat ? m : kSat;
@@ -695,6 +691,14 @@ __device__ __forceinline__ void vec_op(int op, i64 kval, const VecSlot<T, P>& a,
         case XP_OP_MAX: XP_EACH(x > y ? x : y)
         case XP_OP_AND: XP_EACH((x != 0) & (y != 0))
         case XP_OP_OR: XP_EACH((x != 0) | (y != 0))
+        case XP_OP_SHR:                                   // (a left shift never stays in an int32 program: its bound saturates)
+#pragma unroll
+            for (int i = 0; i < P; ++i) {
+                const i32 x = (i32)a.v[i], y = (i32)t.v[i];
+                bad |= y < 0 || y > 63;
+                t.v[i] = (T)(x >> (y > 31 ? 31 : (y < 0 ? 0 : y)));
+            }
+            break;
 #undef XP_EACH
         default: bad = true; break;
     }
@@ -967,8 +971,7 @@ __device__ __noinline__ u32 operand_vars(const GrammarDev* g, const HoleDev* hol
 }
 
 // Values at probe `pr` of `n` (<= kNA) consecutive subtrees of (nt, size) starting at `rank`, written
-// to the calling thread's column (lo[j * kThreads], and hi[...] for the high words unless hi is
-// null); returns the mask of those that are defined there and, in `fits`, of those that fit int32.
+// to lo[j] (and hi[j] for the high words unless hi is null); returns the mask of those that are defined there and, in `fits`, of those that fit int32.
 // A subtree above the table sizes whose operands are in the tables is unranked one level for
 // the first rank only; the following ranks advance the operand ranks like an odometer (right
 // operand fastest), so the left operand's value is fetched once per run.
@@ -978,11 +981,11 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
     fits = 0;
     const int tmax = hole->tab_max_size;
     const u64 pbase = (u64)pr * hole->tab_total;
-    for (int j = 0; j < kNA; ++j) { lo[j * kThreads] = 0; if (hi) hi[j * kThreads] = 0; }
+    for (int j = 0; j < kNA; ++j) { lo[j] = 0; if (hi) hi[j] = 0; }
     if (n <= 0) return 0;
     auto put = [&](int j, i64 v) {
-        lo[j * kThreads] = (u32)(u64)v;
-        if (hi) hi[j * kThreads] = (u32)((u64)v >> 32);
+        lo[j] = (u32)(u64)v;
+        if (hi) hi[j] = (u32)((u64)v >> 32);
         alive |= 1u << j;
         if (v > -(1ll << 31) && v < (1ll << 31)) fits |= 1u << j;
     };
@@ -1114,6 +1117,15 @@ __device__ __forceinline__ u32 inv_odd(u32 o) {
 
 __device__ __forceinline__ u32 rotr32(u32 x, u32 k) { return __funnelshift_r(x, x, k); }
 
+// The register-side operands of a thread for the ticket at hand: low and high words of the values
+// at probe 0 and the values at probe 1 (second look).  The loops below are not inlined and get a
+// pointer to this record; each copies the low words into registers when it starts and derives what
+// it needs of them there (a handful of instructions per operand, once per call).  The record is
+// kept this small on purpose: it lives in the thread's local memory, and the records of all
+// resident threads together (96 bytes x 768 threads per SM) stay in the L1 cache, where a record
+// with every derived array (ten times the size) did not and went through L2 to DRAM on every tile.
+struct RegVals { u32 lo[kNA], hi[kNA], p1[kNA]; };
+
 // The second look: the candidate's exact value at probe 1 from its operands' values there,
 // through the affine context, against the spec.  Operand values that are not known exactly in
 // int32 pass (the exact stages decide).  Runs for filter hits only.
@@ -1127,12 +1139,11 @@ __device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok
     return (u64)v * sh.p1_A + sh.p1_B == sh.p1_spec;
 }
 // (a1ok: bit j says that this thread's operand j is known exactly at probe 1)
-#define XP_P1(op, j, s) probe1_pass(sh, op, (a1ok >> (j)) & 1u, (i32)sh.r1[j][threadIdx.x], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
+#define XP_P1(op, j, s) probe1_pass(sh, op, (a1ok >> (j)) & 1u, (i32)R->p1[j], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
 
 // The loops below are separate (not inlined) functions on purpose: each copies the thread's
-// column of register-side operands from shared memory into registers, derives what it needs of
-// them (a handful of instructions per operand, once per call) and runs with a small live set,
-// instead of sharing one large frame with the rest of the kernel.
+// register-side operands into registers, derives what it needs of them and runs with a small
+// live set, instead of sharing one large frame with the rest of the kernel.
 // `opip` packs the index of each operator inside the segment's list, 3 bits per operator.
 
 // Position of a grammar operator among the seven a segment may hold: + - * / % min max.
@@ -1149,13 +1160,13 @@ __device__ __forceinline__ u32 signfree(u32 x) { const u32 y = 0u - x; return x 
 // the hole has that second look) and queues what is left.  Keeping this part out of line and
 // rolled keeps the loops' instruction footprint small, which matters where the filter is not
 // selective (small value ranges) and the rare path is not rare.
-__device__ __noinline__ void emit_ring(EvalShared& sh, u32 a1ok, int s, u32 m_as, u32 m_mul, u32 A, u32 tp, u32 opip,
+__device__ __noinline__ void emit_ring(EvalShared& sh, const RegVals* R, u32 a1ok, int s, u32 m_as, u32 m_mul, u32 A, u32 tp, u32 opip,
                                        u32 mask, bool SWAP) {
     const BcRing e = sh.bc_ring[s];
     const u32 t_sub = SWAP ? 0u - e.t_add : 2u * tp - e.t_add;
     for (u32 m = m_as; m; m &= m - 1) {                 // + and -: which of the two (or both) it was
         const int j = __ffs((int)m) - 1;
-        const u32 a = sh.rv[j][threadIdx.x] * A;
+        const u32 a = R->lo[j] * A;
         const u32 idx = threadIdx.x * (u32)kNA + (u32)j;
         if ((mask & 1u) && a == e.t_add && XP_P1(XP_OP_ADD, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_ADD)) & 7u);
         if ((mask & 2u) && a == t_sub && XP_P1(XP_OP_SUB, j, s)) push_hit(sh, idx, (u32)s, (opip >> (3 * XP_OP_SUB)) & 7u);
@@ -1166,7 +1177,7 @@ __device__ __noinline__ void emit_ring(EvalShared& sh, u32 a1ok, int s, u32 m_as
     }
 }
 
-__device__ __noinline__ void emit_pairs(EvalShared& sh, u32 a1ok, int s, u32 m0, int op0, u32 m1, int op1, u32 opip,
+__device__ __noinline__ void emit_pairs(EvalShared& sh, const RegVals* R, u32 a1ok, int s, u32 m0, int op0, u32 m1, int op1, u32 opip,
                                         bool SWAP) {
     for (u32 m = m0; m; m &= m - 1) {
         const int j = __ffs((int)m) - 1;
@@ -1187,13 +1198,19 @@ __device__ __noinline__ void emit_pairs(EvalShared& sh, u32 a1ok, int s, u32 m0,
 // are tp -+ A*b, i.e. A*a - tp == -+ A*b; with SWAP they are +-(tp - A*b).  Either way the pair
 // hits iff the sign-free forms agree: ca == t_pm.  Which of the two hit is settled in the rare
 // path, from t_add.
-template <u32 MASK, bool SWAP>
-__device__ __noinline__ void ring_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
+// Broadcast operands per warp vote.  A vote that fires makes every lane repeat the group's tests,
+// so the group is large where hits are rare (the vote and the loop control are shared by more
+// candidates) and small where they are frequent (holes that take the second look: DENSE).
+template <bool DENSE> struct VoteGroup { static constexpr int kRing = DENSE ? 4 : 8, kDiv = DENSE ? 2 : 4; };
+
+template <u32 MASK, bool SWAP, bool DENSE>
+__device__ __noinline__ void ring_pass(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
     constexpr bool kPair = (MASK & 3u) == 3u;
+    constexpr int kRingGroup = VoteGroup<DENSE>::kRing;
     u32 aA[kNA], ca[kNA];                               // A * value, and the sign-free form for the joint +/- test
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
-        aA[j] = sh.rv[j][threadIdx.x] * A;
+        aA[j] = R->lo[j] * A;
         ca[j] = signfree(SWAP ? aA[j] : aA[j] - tp);
     }
     auto t_sub_of = [&](u32 t_add) { return SWAP ? 0u - t_add : 2u * tp - t_add; };
@@ -1223,21 +1240,24 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 
             if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b + e.mul_nt == 0u) << j;
         }
         m_as &= alive; m_mul &= alive;
-        if (m_as | m_mul) emit_ring(sh, a1ok, s, m_as, m_mul, A, tp, opip, MASK, SWAP);
+        if (m_as | m_mul) emit_ring(sh, R, a1ok, s, m_as, m_mul, A, tp, opip, MASK, SWAP);
     };
-    // One warp vote per four broadcast operands (fewer at the end of the run).  The rare path has
+    // One warp vote per kRingGroup broadcast operands (fewer at the end of the run).  The rare path has
     // a single, rolled call site: its code is large, and every copy of it competes with the loops
     // for the instruction cache.
-    for (int s = s0; s < s1; s += 4) {
-        const int n = s1 - s < 4 ? s1 - s : 4;
+    for (int s = s0; s < s1; s += kRingGroup) {
+        const int n = s1 - s < kRingGroup ? s1 - s : kRingGroup;
         bool h[4] = {false, false, false, false};       // independent chains of comparisons
         u32 m[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};       // ... and of minima
-        if (n == 4) {
-            const BcRing e0 = sh.bc_ring[s], e1 = sh.bc_ring[s + 1], e2 = sh.bc_ring[s + 2], e3 = sh.bc_ring[s + 3];
-            scan(e0, h, m);
-            scan(e1, h, m);
-            scan(e2, h, m);
-            scan(e3, h, m);
+        if (n == kRingGroup) {
+#pragma unroll
+            for (int q0 = 0; q0 < kRingGroup; q0 += 4) {
+                const BcRing e0 = sh.bc_ring[s + q0], e1 = sh.bc_ring[s + q0 + 1], e2 = sh.bc_ring[s + q0 + 2], e3 = sh.bc_ring[s + q0 + 3];
+                scan(e0, h, m);
+                scan(e1, h, m);
+                scan(e2, h, m);
+                scan(e3, h, m);
+            }
         } else {
 #pragma unroll 1
             for (int q = 0; q < n; ++q) { const BcRing e0 = sh.bc_ring[s + q]; scan(e0, h, m); }
@@ -1254,18 +1274,18 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 
 // in a run of their own: 0 is skipped (invalid), +-1 gives |quotient| = |dividend| and remainder
 // 0.  There are at most a few such slots per tile, so this is a small rolled routine rather than
 // another instance of the loop below.
-__device__ __noinline__ void div_special(EvalShared& sh, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip, u32 mask) {
+__device__ __noinline__ void div_special(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip, u32 mask) {
     constexpr bool SWAP = false;
     for (int s = s0; s < s1; ++s) {
         if (sh.bc_div[s].ub != 1u) continue;
         u32 mq = 0, mr = 0;
         for (int j = 0; j < kNA; ++j) {
-            if ((mask & 1u) && abs_u32((i32)sh.rv[j][threadIdx.x]) == tabs) mq |= 1u << j;
+            if ((mask & 1u) && abs_u32((i32)R->lo[j]) == tabs) mq |= 1u << j;
             if ((mask & 2u) && tabs == 0u) mr |= 1u << j;
         }
         mq &= alive; mr &= alive;
         const bool any = (mq | mr) != 0;
-        if (__any_sync(0xffffffffu, any) && any) emit_pairs(sh, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
+        if (__any_sync(0xffffffffu, any) && any) emit_pairs(sh, R, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     }
 }
 
@@ -1279,8 +1299,9 @@ __device__ __noinline__ void div_special(EvalShared& sh, u32 alive, u32 a1ok, u3
 // SWAP = false: register operand / broadcast operand; SWAP = true: broadcast / register.
 // SPECIAL (without SWAP only): the slots hold the divisors 0 and +-1: 0 is skipped (invalid),
 // +-1 gives |quotient| = |dividend| and remainder 0.
-template <u32 MASK, bool SWAP, bool SPECIAL>
-__device__ __noinline__ void div_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip) {
+template <u32 MASK, bool SWAP, bool SPECIAL, bool DENSE>
+__device__ __noinline__ void div_pass(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, u32 tabs, int s0, int s1, u32 opip) {
+    constexpr int kDivGroup = VoteGroup<DENSE>::kDiv;
     // ua: |value|.  xa: |value| - tabs as a dividend (register operand / broadcast operand).  With SWAP the
     // register operand is the DIVISOR: low = tabs * |value| (0x80000000 when that is 2^31 or more: never
     // matches), inv = inverse mod 2^32 of the odd part of |value|, kk = its trailing zero bits, cc =
@@ -1288,7 +1309,7 @@ __device__ __noinline__ void div_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 t
     u32 ua[kNA], xa[kNA], low[kNA], inv[kNA], kk[kNA], cc[kNA];
 #pragma unroll
     for (int j = 0; j < kNA; ++j) {
-        ua[j] = abs_u32((i32)sh.rv[j][threadIdx.x]);
+        ua[j] = abs_u32((i32)R->lo[j]);
         xa[j] = ua[j] >= tabs ? ua[j] - tabs : 1u;      // 1 is a multiple of no divisor >= 2
         if (SWAP) {
             low[j] = 0x80000000u; inv[j] = 1u; kk[j] = 0u; cc[j] = 0u;
@@ -1340,18 +1361,25 @@ __device__ __noinline__ void div_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 t
         // register operands that are invalid, or (SWAP) zero divisors, are dropped here
         const u32 keep = SWAP ? alive & nz : alive;
         mq &= keep; mr &= keep;
-        if (mq | mr) emit_pairs(sh, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
+        if (mq | mr) emit_pairs(sh, R, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     };
-    for (int s = s0; s < s1; s += 2) {                  // one warp vote per two broadcast operands; one rare-path site
-        const int n = s1 - s < 2 ? 1 : 2;
-        const BcDiv e0 = sh.bc_div[s];
-        const u32 k0 = need_k ? (sh.bc_meta[s].meta >> 16) & 63u : 0u;
+    for (int s = s0; s < s1; s += kDivGroup) {          // one warp vote per kDivGroup broadcast operands; one rare-path site
+        const int n = s1 - s < kDivGroup ? s1 - s : kDivGroup;
         bool h0 = false, h1 = false, h2 = false, h3 = false;
-        scan(e0, k0, h0, h1, h2, h3);
-        if (n == 2) {
-            const BcDiv e1 = sh.bc_div[s + 1];
-            const u32 k1 = need_k ? (sh.bc_meta[s + 1].meta >> 16) & 63u : 0u;
-            scan(e1, k1, h0, h1, h2, h3);
+        if (n == kDivGroup) {
+#pragma unroll
+            for (int q = 0; q < kDivGroup; ++q) {
+                const BcDiv e = sh.bc_div[s + q];
+                const u32 k = need_k ? (sh.bc_meta[s + q].meta >> 16) & 63u : 0u;
+                scan(e, k, h0, h1, h2, h3);
+            }
+        } else {
+#pragma unroll 1
+            for (int q = 0; q < n; ++q) {
+                const BcDiv e = sh.bc_div[s + q];
+                const u32 k = need_k ? (sh.bc_meta[s + q].meta >> 16) & 63u : 0u;
+                scan(e, k, h0, h1, h2, h3);
+            }
         }
         if (__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) {
 #pragma unroll 1
@@ -1363,10 +1391,10 @@ __device__ __noinline__ void div_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 t
 // min and max of int32-exact operands (exact signed comparison), times the context factor A,
 // against tp.  MASK: bit0 min, bit1 max.  Both are symmetric, so SWAP plays no role.
 template <u32 MASK, bool HAS_A>
-__device__ __noinline__ void minmax_pass(EvalShared& sh, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
+__device__ __noinline__ void minmax_pass(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, u32 A, u32 tp, int s0, int s1, u32 opip) {
     i32 av[kNA];
 #pragma unroll
-    for (int j = 0; j < kNA; ++j) av[j] = (i32)sh.rv[j][threadIdx.x];
+    for (int j = 0; j < kNA; ++j) av[j] = (i32)R->lo[j];
     auto test = [&](i32 b, int j, bool& hmin, bool& hmax) {
         u32 lo = (u32)(av[j] < b ? av[j] : b), hi = (u32)(av[j] < b ? b : av[j]);
         if (HAS_A) { lo *= A; hi *= A; }
@@ -1394,7 +1422,7 @@ __device__ __noinline__ void minmax_pass(EvalShared& sh, u32 alive, u32 a1ok, u3
                 if (MASK & 2u) mmax |= (u32)hmax << j;
             }
             mmin &= alive; mmax &= alive;
-            if (mmin | mmax) { constexpr bool SWAP = false; emit_pairs(sh, a1ok, s, mmin, XP_OP_MIN, mmax, XP_OP_MAX, opip, SWAP); }
+            if (mmin | mmax) { constexpr bool SWAP = false; emit_pairs(sh, R, a1ok, s, mmin, XP_OP_MIN, mmax, XP_OP_MAX, opip, SWAP); }
         }
     }
 }
@@ -1403,13 +1431,13 @@ __device__ __noinline__ void minmax_pass(EvalShared& sh, u32 alive, u32 a1ok, u3
 // compared with tp.  Plain 32-bit division; this form only serves sketches whose hole sits
 // under a multiplication (small searches).
 template <bool SWAP>
-__device__ __noinline__ void div_pass_signed(EvalShared& sh, u32 alive, u32 a1ok, u32 mask, u32 A, u32 tp,
+__device__ __noinline__ void div_pass_signed(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, u32 mask, u32 A, u32 tp,
                                              int s0, int s1, u32 opip) {
     for (int s = s0; s < s1; ++s) {
         const i32 b = (i32)sh.bc_meta[s].lo;
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
-            const i32 a = (i32)sh.rv[j][threadIdx.x];
+            const i32 a = (i32)R->lo[j];
             const i32 n = SWAP ? b : a, d = SWAP ? a : b;
             if (d == 0) continue;
             const i32 q = n / d;                         // magnitudes are below 2^31: no overflow case
@@ -1424,14 +1452,14 @@ __device__ __noinline__ void div_pass_signed(EvalShared& sh, u32 alive, u32 a1ok
 // Any operator on int64 operands (tiles with an operand outside int32): exact, slow, rare.
 // rng 1: the context compares (HoleDev::rng_lo) and the value must lie in [lo, hi] instead;
 // rng 2: every defined value passes.
-__device__ __noinline__ void wide_chunk(EvalShared& sh, u32 alive, u32 a1ok, bool swap, u64 A, u64 tq,
+__device__ __noinline__ void wide_chunk(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, bool swap, u64 A, u64 tq,
                                         int rng, i64 lo, i64 hi, int s0, int s1, int n_ops, const i32* ops) {
     const bool SWAP = swap;
     for (int s = s0; s < s1; ++s) {
         const i64 b = (i64)(((u64)sh.bc_meta[s].hi << 32) | sh.bc_meta[s].lo);
         for (int j = 0; j < kNA; ++j) {
             if (!((alive >> j) & 1u)) continue;
-            const i64 aj = (i64)(((u64)sh.rh[j][threadIdx.x] << 32) | sh.rv[j][threadIdx.x]);
+            const i64 aj = (i64)(((u64)R->hi[j] << 32) | R->lo[j]);
             for (int o = 0; o < n_ops; ++o) {
                 i64 v;
                 if (!apply_op(ops[o], swap ? b : aj, swap ? aj : b, v)) continue;
@@ -1507,11 +1535,11 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
 
 template <bool SWAP>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
-                                          u64 reg_first, u64 pairs, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
+                                          u64 reg_first, u64 pairs, const RegVals* R, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
     const SegDev& seg = sh.mseg[m];
     const MemberState& mbs = sh.mb[m];
     const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
-    const bool tile_wide = (sh.reg_wide | mbs.wide) != 0;
+    const bool tile_wide = (sh.reg_wide | mbs.wide | seg.generic) != 0;
     const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
     // a context that compares: interval test on int32-exact operands (results stay below 2^62 in
     // magnitude, where the interval is exact); wider operands are all passed on to the exact stages
@@ -1544,30 +1572,33 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
+    const bool dense = sh.p1_on != 0;                   // the hole takes the second look: hits are frequent
     auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide || rng) {
-            wide_chunk(sh, alv, a1ok, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
+            wide_chunk(sh, R, alv, a1ok, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
             return;
         }
         switch (mask & 7u) {
-#define XP_RING(M) case M: ring_pass<M, SWAP>(sh, alv, a1ok, A, tp, s0, s1, opip); break;
+#define XP_RING(M) case M: if (dense) ring_pass<M, SWAP, true>(sh, R, alv, a1ok, A, tp, s0, s1, opip); \
+                           else ring_pass<M, SWAP, false>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
             XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
 #undef XP_RING
             default: break;
         }
         if (mask >> kSlotMin) switch ((mask >> kSlotMin) & 3u) {
-#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, alv, a1ok, A, tp, s0, s1, opip); \
-                         else minmax_pass<M, false>(sh, alv, a1ok, A, tp, s0, s1, opip); break;
+#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, R, alv, a1ok, A, tp, s0, s1, opip); \
+                         else minmax_pass<M, false>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
             XP_MM(1u) XP_MM(2u) XP_MM(3u)
 #undef XP_MM
             default: break;
         }
         if (!(mask & 24u)) return;
-        if (A != 1u) { div_pass_signed<SWAP>(sh, alv, a1ok, mask, A, tp, s0, s1, opip); return; }
+        if (A != 1u) { div_pass_signed<SWAP>(sh, R, alv, a1ok, mask, A, tp, s0, s1, opip); return; }
         if (!t_small) return;                            // no int32 quotient or remainder can be the target
         switch (skip_mod ? (mask >> 3) & 1u : (mask >> 3) & 3u) {
-#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, alv, a1ok, tabs, s0, s1, opip, M); \
-                          else div_pass<M, SWAP, false>(sh, alv, a1ok, tabs, s0, s1, opip); break;
+#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, R, alv, a1ok, tabs, s0, s1, opip, M); \
+                          else if (dense) div_pass<M, SWAP, false, true>(sh, R, alv, a1ok, tabs, s0, s1, opip); \
+                          else div_pass<M, SWAP, false, false>(sh, R, alv, a1ok, tabs, s0, s1, opip); break;
             XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
 #undef XP_DIV
             default: break;
@@ -1719,18 +1750,19 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         sh.p1_rng = (hole->rng_okmask >> 1) & 1u;
         sh.p1_lo = hole->rng_lo[1]; sh.p1_hi = hole->rng_hi[1];
     }
-    // this thread's operands: kNA consecutive ranks, into its column of the tile
+    // this thread's operands: kNA consecutive ranks
+    RegVals RV;
     const int mine = n_reg - (int)threadIdx.x * kNA;
     const int n_mine = mine < 0 ? 0 : (mine > kNA ? kNA : mine);
     u32 fits0 = 0;
     u32 alive = fill_reg_operands(g, hole, 0, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA, n_mine,
-                                  &sh.rv[0][threadIdx.x], &sh.rh[0][threadIdx.x], fits0);
+                                  RV.lo, RV.hi, fits0);
     const bool wide_reg = fits0 != alive;
     // second look: the same operands at probe 1; one that is undefined there can be in no match
     u32 a1ok = 0;
     if (second)
         alive &= fill_reg_operands(g, hole, 1, reg_nt, reg_size, reg_first + threadIdx.x * (u64)kNA, n_mine,
-                                   &sh.r1[0][threadIdx.x], nullptr, a1ok);
+                                   RV.p1, nullptr, a1ok);
     __syncthreads();                                    // the members' segments are in place, reg_wide is clear
     if (wide_reg) sh.reg_wide = 1;
     // broadcast operands of member m: tile bc_tile0 of the head (a family's other members have one tile)
@@ -1766,8 +1798,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
             if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, false, my_evals);
-            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, false, my_evals);
+            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
+            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
         }
         drain_queue(sh, plan, sk, hole, reg_first, my_evals);
         return;
@@ -1781,8 +1813,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         const SegDev& seg = sh.mseg[m];
         const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
         if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, true, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, a1ok, alive, true, my_evals);
+        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
+        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
     }
 }
 
@@ -1790,53 +1822,50 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
 #define XP_MIN_CTAS 3
 #endif
 __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanDev plan) {
-    extern __shared__ __align__(16) unsigned char eval_smem[];      // (more than the 48 KB a static array may have)
-    EvalShared& sh = *reinterpret_cast<EvalShared*>(eval_smem);
+    __shared__ EvalShared sh;
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
     if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; sh.filter_tests = 0; sh.tile_cands = 0; }
     if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
     __syncthreads();
     for (;;) {
-        if (threadIdx.x == 0) sh.item = plan.item_base + atomicAdd(plan.ticket, 1ull);
-        __syncthreads();
-        const u64 item = sh.item;
-        if (item >= plan.n_items) break;
-        const u64 t_first = plan.group_first ? plan.group_first[item] : item;
-        const u64 t_last = plan.group_first ? plan.group_first[item + 1] : item + 1;
-        for (u64 t = t_first; t < t_last; ++t) {
+        if (threadIdx.x == 0) {
+            sh.ticket = plan.ticket_base + atomicAdd(plan.ticket, 1ull);
             // many filter hits so far for the hole at hand (this CTA's own counts): second look from now on
-            if (threadIdx.x == 0 && !sh.adapt_second && sh.filter_survivors * kAdaptRate > sh.tile_cands) sh.adapt_second = 1;
-            if (threadIdx.x < 32) {
-                // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
-                int lo = 0, n = plan.n_segs;
-                while (n > 1) {
-                    const int step = (n + 31) / 32;
-                    const int pos = lo + (int)threadIdx.x * step;
-                    const bool le = pos < lo + n && plan.segs[pos].first_ticket <= t;
-                    const u32 mask = __ballot_sync(0xffffffffu, le);          // lane 0 always holds
-                    const int k = 31 - __clz((int)(mask | 1u));
-                    const int nlo = lo + k * step;
-                    n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
-                    lo = nlo;
-                }
-                if (!XP_CHECKED(lo >= 0 && lo < plan.n_segs && plan.segs[lo].first_ticket <= t, kChkSegment)) lo = 0;
-                if (threadIdx.x == 0) sh.seg_index = lo;
-                load_segment(sh, plan, lo);
+            if (!sh.adapt_second && sh.filter_survivors * kAdaptRate > sh.tile_cands) sh.adapt_second = 1;
+        }
+        __syncthreads();
+        const u64 t = sh.ticket;
+        if (t >= plan.n_tickets) break;
+        if (threadIdx.x < 32) {
+            // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
+            int lo = 0, n = plan.n_segs;
+            while (n > 1) {
+                const int step = (n + 31) / 32;
+                const int pos = lo + (int)threadIdx.x * step;
+                const bool le = pos < lo + n && plan.segs[pos].first_ticket <= t;
+                const u32 mask = __ballot_sync(0xffffffffu, le);          // lane 0 always holds
+                const int k = 31 - __clz((int)(mask | 1u));
+                const int nlo = lo + k * step;
+                n = (lo + n - nlo) < step ? (lo + n - nlo) : step;
+                lo = nlo;
             }
-            __syncthreads();
-            if (sh.seg.acc != sh.cur_acc) {
-                flush_acc(sh, plan, my_evals);
-                if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
-                __syncthreads();
-            }
-            const SketchDev* sk = plan.sketches[sh.seg.sketch];
-            const HoleDev* hole = &sk->holes[sh.seg.hole];
-            const u64 local = t - sh.seg.first_ticket;
-            if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
-            else linear_ticket(sh, plan, sk, hole, local, my_evals);
+            if (!XP_CHECKED(lo >= 0 && lo < plan.n_segs && plan.segs[lo].first_ticket <= t, kChkSegment)) lo = 0;
+            if (threadIdx.x == 0) sh.seg_index = lo;
+            load_segment(sh, plan, lo);
+        }
+        __syncthreads();
+        if (sh.seg.acc != sh.cur_acc) {
+            flush_acc(sh, plan, my_evals);
+            if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
             __syncthreads();
         }
+        const SketchDev* sk = plan.sketches[sh.seg.sketch];
+        const HoleDev* hole = &sk->holes[sh.seg.hole];
+        const u64 local = t - sh.seg.first_ticket;
+        if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
+        else linear_ticket(sh, plan, sk, hole, local, my_evals);
+        __syncthreads();
     }
     flush_acc(sh, plan, my_evals);
 }
@@ -1903,12 +1932,22 @@ __global__ void __launch_bounds__(256) surv_scatter_kernel(const PlanDev plan) {
 // that fails at some point of the step leaves the set.
 constexpr int kVArena = 256;                              // program entries a warp stages at once
 constexpr int kVStep = 128;                               // points per step
-struct __align__(16) VerifyWarp {
+constexpr int kVBatchVars = 4;                            // most variables a table may have for this form
+constexpr int kVBatchDepth = 4;                           // deepest operand stack it takes
+// A warp's shared memory: the batch form's arrays and the one-survivor form's share the same bytes
+// (a warp is in one form at a time), which keeps three CTAs resident per SM.
+struct VerifyBatch {
     i32 pvar[kVArena];                                    // >= 0: variable; -1: constant; -2 - op: operator
     i64 pval[kVArena];
-    i32 coords[kMaxVars][kVStep];                         // the step's points, [variable][point]
-    uint4 stack[kVecDepth * 32];                          // operand stacks below the top, per level and lane
-    CandShared cand;                                      // the one-survivor form (boxes, long programs)
+    i32 coords[kVBatchVars][kVStep];                      // the step's points, [variable][point]
+    uint4 stack[kVBatchDepth * 32];                       // operand stacks below the top, per level and lane
+};
+struct VerifySingle {
+    uint4 stack[kVecDepth * 32];
+    CandShared cand;                                      // the one-survivor form (boxes, long or deep programs, many variables)
+};
+struct __align__(16) VerifyWarp {
+    union { VerifyBatch b; VerifySingle s; };
 };
 
 // Length of the program that candidate code of `n` nodes gives in the hole's context; -1 if the
@@ -1934,8 +1973,8 @@ __device__ __noinline__ int stage_compact(VerifyWarp& w, int off, const SketchDe
     u64 mag[kMaxStack + kCandStack + 1];
     auto mag_of = [](i64 v) { return v < 0 ? 0ull - (u64)v : (u64)v; };
     auto emit = [&](i32 var, i64 val) {
-        if (sp > kMaxStack + kCandStack - 1) { depth = kVecDepth + 1; return; }
-        w.pvar[off + len] = var; w.pval[off + len] = val; ++len;
+        if (sp > kMaxStack + kCandStack - 1) { depth = kVBatchDepth + 1; return; }
+        w.b.pvar[off + len] = var; w.b.pval[off + len] = val; ++len;
         u64 m;
         if (var >= -1) {
             if (var >= 0) { const u64 a = mag_of(sk->vmin[var]), b = mag_of(sk->vmax[var]); m = a > b ? a : b; }
@@ -1951,6 +1990,8 @@ __device__ __noinline__ int stage_compact(VerifyWarp& w, int off, const SketchDe
                 case XP_OP_DIV: m = a; break;
                 case XP_OP_MOD: m = a < b ? a : b; break;
                 case XP_OP_MIN: case XP_OP_MAX: m = a > b ? a : b; break;
+                case XP_OP_SHL: m = kSat; break;
+                case XP_OP_SHR: m = a; break;
                 default: m = 1; break;
             }
             mag[sp - 1] = m < kSat ? m : kSat;
@@ -1972,22 +2013,22 @@ __device__ __noinline__ int stage_compact(VerifyWarp& w, int off, const SketchDe
             else emit(in.kind == XP_I_VAR ? in.arg : -1, in.value);
         }
     narrow_out = narrow;
-    if (depth > kVecDepth) return -1;
+    if (depth > kVBatchDepth) return -1;
     if (narrow) {                                         // "push c; x / y" -> one instruction on the top of the stack
         int wr = 0;
         for (int k = 0; k < len; ++k) {
-            const i32 cv = w.pvar[off + k];
+            const i32 cv = w.b.pvar[off + k];
             const bool divmod = cv == -2 - XP_OP_DIV || cv == -2 - XP_OP_MOD;
-            if (divmod && wr > 0 && w.pvar[off + wr - 1] == -1 && w.pval[off + wr - 1] != 0 &&
-                w.pval[off + wr - 1] > -(1ll << 31) && w.pval[off + wr - 1] < (1ll << 31)) {
-                const i32 d = (i32)w.pval[off + wr - 1];
+            if (divmod && wr > 0 && w.b.pvar[off + wr - 1] == -1 && w.b.pval[off + wr - 1] != 0 &&
+                w.b.pval[off + wr - 1] > -(1ll << 31) && w.b.pval[off + wr - 1] < (1ll << 31)) {
+                const i32 d = (i32)w.b.pval[off + wr - 1];
                 const u32 ad = d < 0 ? 0u - (u32)d : (u32)d;
                 const u32 M = ad == 1u ? 0xffffffffu : (u32)((1ull << 32) / ad);
-                w.pvar[off + wr - 1] = -2 - (cv == -2 - XP_OP_DIV ? kOpDivC : kOpModC);
-                w.pval[off + wr - 1] = (i64)(((u64)M << 32) | (u32)d);
+                w.b.pvar[off + wr - 1] = -2 - (cv == -2 - XP_OP_DIV ? kOpDivC : kOpModC);
+                w.b.pval[off + wr - 1] = (i64)(((u64)M << 32) | (u32)d);
                 continue;
             }
-            w.pvar[off + wr] = cv; w.pval[off + wr] = w.pval[off + k]; ++wr;
+            w.b.pvar[off + wr] = cv; w.b.pval[off + wr] = w.b.pval[off + k]; ++wr;
         }
         len = wr;
     }
@@ -2006,18 +2047,18 @@ __device__ __forceinline__ u32 run_staged(VerifyWarp& w, int off, int len, int h
     bool bad = false;
     int below = 0;
     for (int k = 0; k < len; ++k) {
-        const i32 cv = w.pvar[off + k];
+        const i32 cv = w.b.pvar[off + k];
         if (cv >= -1) {
-            w.stack[below * 32 + lane] = t.q;
+            w.b.stack[below * 32 + lane] = t.q;
             ++below;
             if (cv >= 0) {
-                if (sizeof(T) == 4) t.q = *reinterpret_cast<const uint4*>(&w.coords[cv][lane * 4]);
+                if (sizeof(T) == 4) t.q = *reinterpret_cast<const uint4*>(&w.b.coords[cv][lane * 4]);
                 else {
 #pragma unroll
-                    for (int i = 0; i < P; ++i) t.v[i] = (T)w.coords[cv][lane * 4 + half * P + i];
+                    for (int i = 0; i < P; ++i) t.v[i] = (T)w.b.coords[cv][lane * 4 + half * P + i];
                 }
             } else {
-                const T v = (T)w.pval[off + k];
+                const T v = (T)w.b.pval[off + k];
 #pragma unroll
                 for (int i = 0; i < P; ++i) t.v[i] = v;
             }
@@ -2026,8 +2067,8 @@ __device__ __forceinline__ u32 run_staged(VerifyWarp& w, int off, int len, int h
         const int op = -2 - cv;
         Slot a;
         a.q = t.q;
-        if (!(sizeof(T) == 4 && op >= kOpDivC)) { --below; a.q = w.stack[below * 32 + lane]; }
-        vec_op<T, P>(op, w.pval[off + k], a, t, bad);
+        if (!(sizeof(T) == 4 && op >= kOpDivC)) { --below; a.q = w.b.stack[below * 32 + lane]; }
+        vec_op<T, P>(op, w.b.pval[off + k], a, t, bad);
     }
     u32 which = 0;
 #pragma unroll
@@ -2052,7 +2093,7 @@ __device__ __noinline__ void verify_batch(VerifyWarp& w, const SketchDev* sk, co
         for (int idx = lane; idx < kVStep * nv; idx += 32) {      // rows are contiguous: coalesced reads
             const int p = idx / nv, v = idx - p * nv;
             const int src = p < npts ? idx : v;           // points past the end repeat the step's first point
-            w.coords[v][p] = coords[base * nv + src];
+            w.b.coords[v][p] = coords[base * nv + src];
         }
         i64 want[4];
         u32 in_mask = 0;
@@ -2090,7 +2131,7 @@ __device__ __noinline__ void verify_batch(VerifyWarp& w, const SketchDev* sk, co
 // programs that do not fit the arena, contexts that never mention the hole).
 __device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 si, u64 chunk) {
     const int lane = threadIdx.x & 31;
-    CandShared& cand = w.cand;
+    CandShared& cand = w.s.cand;
     int skip = 1;
     i64 np = 0;
     SurvDev* sv = &plan.surv[si];
@@ -2117,8 +2158,8 @@ __device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 
     i64 fail_pid = 0;
     bool ok;
     if (sk->coords != nullptr && hole->spec_table != nullptr && cand.depth >= 1 && cand.depth <= kVecDepth) {
-        ok = cand.narrow ? check_points_vec<i32, 4>(cand, w.stack, sk, hole, first, last, &fail_pid)
-                         : check_points_vec<i64, 2>(cand, w.stack, sk, hole, first, last, &fail_pid);
+        ok = cand.narrow ? check_points_vec<i32, 4>(cand, w.s.stack, sk, hole, first, last, &fail_pid)
+                         : check_points_vec<i64, 2>(cand, w.s.stack, sk, hole, first, last, &fail_pid);
     } else {
         ok = check_points(cand, sk, hole, first, last, evals, &fail_pid);
     }
@@ -2130,7 +2171,7 @@ __device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 
     __syncwarp();                                       // the staged candidate is free for the next item
 }
 
-// Items are (chunk of points, block of 32 survivors in hole order), chunk-major: the first chunk
+// Items are (chunk of points, block of up to 32 survivors in hole order), chunk-major: the first chunk
 // of every survivor is taken before any second chunk, so candidates that fail early cost one
 // chunk.  Each WARP takes items on its own: nothing in this kernel synchronises a CTA, and no
 // warp waits for another.  Within a block the survivors of one hole are handled together when the
@@ -2138,13 +2179,20 @@ __device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 
 // that has already failed is skipped.
 constexpr int kVerifyThreads = 256;
 constexpr int kVerifyWarps = kVerifyThreads / 32;
-__global__ void __launch_bounds__(kVerifyThreads, 2) verify_kernel(const PlanDev plan) {
+__global__ void __launch_bounds__(kVerifyThreads, 3) verify_kernel(const PlanDev plan) {
     extern __shared__ __align__(16) unsigned char verify_smem[];
     VerifyWarp& w = reinterpret_cast<VerifyWarp*>(verify_smem)[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const u32 pushed = *plan.surv_n;
     const u64 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
-    const u64 n_blocks = (n + 31) / 32;
+    // Survivors per item: 32 when there are plenty (the batch form then has a full warp to stage and
+    // share points with); fewer, down to one, when the call has too few survivors to give every warp
+    // of the grid a full block (a search with a few thousand survivors on a large domain spreads
+    // better as one survivor per warp).
+    const u64 warps = (u64)gridDim.x * kVerifyWarps;
+    u32 width = 32;
+    while (width > 1 && n < warps * width) width >>= 1;
+    const u64 n_blocks = (n + width - 1) / width;
     const u64 total = n_blocks * plan.max_chunks;
     constexpr u64 kBatch = 2;                           // items a warp takes per atomic
     u64 next = 0, batch_end = 0;
@@ -2157,8 +2205,8 @@ __global__ void __launch_bounds__(kVerifyThreads, 2) verify_kernel(const PlanDev
         const u64 t = next++;
         if (t >= total) break;
         const u64 chunk = t / n_blocks, block = t % n_blocks;
-        const u64 pos = block * 32 + lane;
-        const bool have = pos < n;
+        const u64 pos = block * width + lane;
+        const bool have = (u32)lane < width && pos < n;
         const u32 si = have ? (plan.surv_sorted ? plan.surv_sorted[pos] : (u32)pos) : 0u;
         const int my_acc = have ? plan.surv[si].acc : -1;
         u32 remaining = __ballot_sync(0xffffffffu, have);
@@ -2170,7 +2218,8 @@ __global__ void __launch_bounds__(kVerifyThreads, 2) verify_kernel(const PlanDev
             const u32 lsi = __shfl_sync(0xffffffffu, si, leader);
             const SketchDev* sk = plan.sketches[plan.surv[lsi].sketch];
             const HoleDev* hole = &sk->holes[plan.surv[lsi].hole];
-            const bool table = sk->domain_kind == XP_DOMAIN_TABLE && sk->coords != nullptr && hole->spec_table != nullptr;
+            const bool table = sk->domain_kind == XP_DOMAIN_TABLE && sk->coords != nullptr && hole->spec_table != nullptr &&
+                               sk->n_vars <= kVBatchVars;
             const i64 first = (i64)chunk * kVerifyChunk;
             const bool mine = (run >> lane) & 1u;
             u32 single = 0;                               // survivors of the run that go one by one
@@ -2344,9 +2393,8 @@ static int resident_ctas(const void* kernel, size_t dynamic_smem = 0) {
 
 static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sketches, u32 max_chunks) {
     PlanDev pd;
-    pd.item_base = 0;
-    pd.n_items = 0;
-    pd.group_first = L.n_groups ? (const u64*)(base + L.groups) : nullptr;
+    pd.ticket_base = 0;
+    pd.n_tickets = 0;
     pd.n_segs = n_segs;
     pd.n_sketches = n_sketches;
     pd.ticket = (u64*)base;
@@ -2367,8 +2415,7 @@ static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sket
     return pd;
 }
 
-// Stages 1 and 2 for the work items [t_begin, t_end) of the plan staged at `base` (an item is a
-// ticket, or a group of tickets when the layout carries groups).  A search is one
+// Stages 1 and 2 for the tickets [t_begin, t_end) of the plan staged at `base`.  A search is one
 // such launch, or several in a row when the host wants to look at a cancel word or a clock in
 // between; `restart` says that the ticket counter has to be set back to zero first (every launch
 // but the first, whose counter the staged copy has just zeroed).
@@ -2378,15 +2425,11 @@ cudaError_t launch_search_part(char* base, const SearchLayout& L, u64 t_begin, u
     cudaError_t e;
     if (restart && (e = cudaMemsetAsync(base, 0, 8, stream)) != cudaSuccess) return e;
     PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
-    pd.item_base = t_begin;
-    pd.n_items = t_end;
-    if ((e = cudaFuncSetAttribute((const void*)eval_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EvalShared))) != cudaSuccess) return e;
-#ifdef XP_CARVEOUT
-    if ((e = cudaFuncSetAttribute((const void*)eval_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, XP_CARVEOUT)) != cudaSuccess) return e;
-#endif
-    u64 ctas = (u64)resident_ctas((const void*)eval_kernel, sizeof(EvalShared));      // persistent CTAs: one wave
+    pd.ticket_base = t_begin;
+    pd.n_tickets = t_end;
+    u64 ctas = (u64)resident_ctas((const void*)eval_kernel, 0);      // persistent CTAs: one wave
     if (ctas > t_end - t_begin) ctas = t_end - t_begin;
-    eval_kernel<<<(unsigned)ctas, kThreads, sizeof(EvalShared), stream>>>(pd);
+    eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
     *n_launches += 1;
     return cudaGetLastError();
 }

@@ -16,10 +16,10 @@ cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most
 // Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
 //   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32), 20: failed-check word (u32; checked
 //      build only)   -- zero at launch
-//   segs, sketches, acc, groups (first ticket of every group of tickets, when the plan is grouped): staged from the host;  [0, head) is what the host copies in
+//   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
 //   hist: survivors per accumulator slot, zero at launch (staged);
 //   surv: the survivor queue (surv_cap entries); sort_off, sorted: its hole order -- written by the kernels only
-struct SearchLayout { size_t segs, sketches, acc, groups, hist, head, surv, sort_off, sorted, total; u32 surv_cap; u64 n_groups; int n_acc; };
+struct SearchLayout { size_t segs, sketches, acc, hist, head, surv, sort_off, sorted, total; u32 surv_cap; int n_acc; };
 
 // The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel;
 // or the same in pieces: eval_kernel over one range of tickets at a time, then the rest.
@@ -33,5 +33,15 @@ constexpr size_t kStaticScratchBytes = 1u << 20;     // fixed scratch of the all
 cudaError_t launch_search_static(const void* stage, const SearchLayout& L, u64 n_tickets, int n_segs, int n_acc,
                                  u32 max_chunks, AccDev* acc_out, cudaStream_t stream);
 cudaError_t launch_int32_peak(int which, u32* out, int blocks, int iters, cudaStream_t stream);
+
+// What the library's other source files may know of a grammar and a loaded sketch (defined in xp_api.cu).
+struct SketchInternals { const SketchDev* d_s; const xp_grammar* g; i64 n_points; int device, n_vars; };
+SketchInternals sketch_internals(const xp_sketch* s);
+u64 grammar_cnt(const xp_grammar* g, int nt, int size);      // trees of nt with exactly `size` nodes
+int grammar_nonterminals(const xp_grammar* g);
+int grammar_ok_size(const xp_grammar* g);                    // counts are exact (< 2^63) up to this size
+cudaError_t device_alloc(void** out, size_t bytes, int* device, size_t* granted);     // the library's device pool
+void device_release(void* ptr, size_t granted, int device);
+xp_status set_error(xp_status st, const char* msg);
 
 }  // namespace xp

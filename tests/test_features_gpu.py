@@ -216,3 +216,43 @@ def test_small_parity_cases_under_the_checked_build():
                        cwd=root, env=env, capture_output=True, text=True, timeout=1500)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-1000:]
     assert " passed" in r.stdout
+
+
+def test_shifts_as_grammar_operators(xp):
+    """<< and >> in productions, contexts and specs: no 32-bit filter loop exists for them, their
+    operand tiles are evaluated exactly; a count outside 0..63 fails the candidate at that point."""
+    vs = [Variable("i", 0, 6), Variable("j", -2, 5)]
+    g = free_grammar(vs, [1, 2, 3, 64], ops=["+", "*", "<<", ">>"])
+    for spec, ctx in [("(i<<2)+j", ""), ("(i+j)>>1", ""), ("i<<j", ""), ("j>>64", ""), ("(i<<3)+(j<<1)", "HOLE<<1"),
+                      ("((i*3)>>1)<4", "(HOLE>>1)<4")]:
+        sk = Sketch(g, [Hole(0, 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))], name=f"shifts: {spec}")
+        for flags in PATHS:
+            check_sketch(xp, sk, flags=flags)
+    wide = [Variable("x", 2 ** 33, 2 ** 33 + 4), Variable("s", 0, 66)]
+    gw = free_grammar(wide, [1, 31], ops=["-", "<<", ">>"])
+    skw = Sketch(gw, [Hole(0, 5, spec_expr=parse_expr("(x>>s)-(1<<31)", wide))], name="wide shifts")
+    for flags in PATHS:
+        check_sketch(xp, skw, flags=flags)
+
+
+def test_constant_only_holes(xp):
+    """Instruction-parameter and buffer-size holes: the hole is filled from constants alone (a
+    nonterminal with constant productions only, size bound 1).  The vector length of an
+    instruction that must cover exactly the elements the source touches (2309 was written where
+    1024 is right), and the row pitch of a staging buffer."""
+    vs = [Variable("e", 0, 4096)]
+    lengths = [16, 64, 256, 1000, 1024, 2048, 2309, 4096]
+    prods = [Production(lhs=0, kind=P_CONST, value=c) for c in lengths]
+    g = Grammar(vs, 1, prods)
+    sk = Sketch(g, [Hole(0, 1, ctx=parse_expr("e<HOLE", vs), spec_expr=parse_expr("e<1024", vs))], name="vector length")
+    res = check_sketch(xp, sk)
+    assert res[0].least_text == "1024" and res[0].match_count == [0, 1] and res[0].cand_count == [0, 8]
+    vs2 = [Variable("r", 0, 32), Variable("c", 0, 48)]
+    prods2 = [Production(lhs=0, kind=P_VAR, var=0), Production(lhs=0, kind=P_VAR, var=1)]
+    prods2 += [Production(lhs=1, kind=P_CONST, value=c) for c in (32, 40, 48, 64, 96)]
+    g2 = Grammar(vs2, 2, prods2)
+    sk2 = Sketch(g2, [Hole(1, 1, ctx=parse_expr("(r*HOLE)+c", vs2), spec_expr=parse_expr("(r*48)+c", vs2))], name="row pitch")
+    res2 = check_sketch(xp, sk2)
+    assert res2[0].least_text == "48" and res2[0].solved
+    sk3 = Sketch(g2, [Hole(1, 1, ctx=parse_expr("(r*HOLE)+c", vs2), spec_expr=parse_expr("(r*50)+c", vs2))], name="no such pitch")
+    assert not check_sketch(xp, sk3)[0].solved
