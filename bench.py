@@ -35,6 +35,7 @@ WORKLOADS = {
     "config5": "config5_batch_4096_instances_size6",
 }
 HEADLINE = "config4"
+DIVISION_COST = None
 
 # Counters of one eval_kernel launch per workload, from the ncu captures summarised under profiles/
 # (dram = dram__bytes_read.sum + dram__bytes_write.sum, thread_inst = smsp__thread_inst_executed.sum).
@@ -292,6 +293,7 @@ def roofline(m, steps, world, peak_add, peak_mad, name):
            "frac_executed": (thread_inst * steps / kern_s / peak_add) if thread_inst else None,
            "frac_cost_model": (m["model_ops"] / world) / kern_s / peak_add if m.get("model_ops") else None,
            "traffic": cap.get("dram_bytes") if fresh else None,
+           "division_cost": DIVISION_COST,
            "kernel": "eval_kernel",
            "peak_source": "measured live: independent 32-bit add chains (xp_int32_peak); multiply-add chains reach %.0f" % (peak_mad / 1e9),
            "model": "frac: 2 x candidate-point evaluations that ran (one 32-bit operation + one comparison each) / kernel time / peak; "
@@ -364,6 +366,10 @@ def main():
         torch.cuda.synchronize()
 
     peak_add, peak_mad = xp.xp_int32_peak()
+    div_general, div_reciprocal = xp.xp_int_div_rate()
+    global DIVISION_COST
+    DIVISION_COST = {"int64_general_form": peak_add / div_general, "int32_by_constant_reciprocal_form": peak_add / div_reciprocal,
+                     "unit": "32-bit add-peak operations per division, measured live (xp_int_div_rate)"}
     head = args.workload or HEADLINE
     if args.shard:
         run_shard(args, xp, torch, dist, rank, world, stream, flush, barrier)

@@ -363,6 +363,53 @@ xp_status xp_repair_joint(const xp_sketch* sketch, const xp_joint_desc* joint, c
 xp_status xp_joint_result_get(const xp_joint_result* r, xp_joint_view* out);
 void xp_joint_result_free(xp_joint_result* r);
 
+/* The behaviour mode: bottom-up enumeration with observational-equivalence pruning (the paper keeps
+ * its symbolic synthesis "limited scale" because the space of expressions explodes; pruning by behaviour
+ * is the enumerative way to push the bound).  A different contract from xp_repair: what is counted is
+ * BEHAVIOURS on a caller-given list of signature points, not syntactic candidates.
+ *   A tree's signature is the vector of its values at the signature points.  Per nonterminal and size
+ *   (ascending), the candidates are the leaf productions (size 1) and, for each binary production in the
+ *   grammar's order, each left size ascending, every pair (left representative, right representative) in
+ *   the order the representatives were found, right fastest.  A candidate that is undefined at a signature
+ *   point (zero divisor, bad shift count) is dropped; one whose signature a representative of the same
+ *   nonterminal already has (a smaller size, or earlier at this size) is dropped; the others become
+ *   the representatives of this size, in that order.  A behaviour first realised by some tree of size s is
+ *   found at size s (subtrees can be swapped for their representatives, which are no larger).
+ * For hole `hole` of the sketch (start nonterminal, size bound, context, spec) the call reports, per size,
+ * the candidates enumerated and the new behaviours found for the start nonterminal; how many
+ * representatives satisfy the constraint at every signature point; the first of them (size, then order
+ * found) and whether it satisfies the constraint on the whole domain; and the first that does.
+ * Signatures live in device memory (8 bytes x n_sig per representative) beside a hash table of
+ * fingerprints; an equal fingerprint is always confirmed by comparing the signatures themselves, so the
+ * result does not depend on the hash.  The work is bound by memory traffic, not by the integer units.
+ * Errors: XP_ERR_INVALID_ARG (bad hole, n_sig outside 1..XP_MAX_SIG, a point id outside the domain),
+ * XP_ERR_TOO_LARGE (more representatives than max_representatives), XP_ERR_NOMEM, XP_ERR_CUDA. */
+enum { XP_MAX_SIG = 16 };
+typedef struct {
+    int32_t hole;
+    int32_t n_sig;
+    const int64_t* sig_points;          /* domain point ids (box: mixed radix, first variable slowest), in signature order */
+    uint64_t max_representatives;       /* of all nonterminals and sizes together; 0: 2^22 */
+} xp_behaviour_desc;
+typedef struct {
+    int32_t max_size, pad;
+    uint64_t enumerated[XP_MAX_SIZE + 1];
+    uint64_t distinct[XP_MAX_SIZE + 1];
+    uint64_t sig_matches;
+    int32_t hit, hit_size;              /* first representative that satisfies the signature points */
+    uint64_t hit_index;                 /* its position among the representatives of its size */
+    int32_t hit_verified;               /* it satisfies the constraint on the whole domain */
+    int32_t solved, solution_size, pad2;  /* first representative that does */
+    uint64_t solution_index;
+    char hit_text[256], solution_text[256];
+    uint64_t representatives;           /* of all nonterminals and sizes */
+    uint64_t bytes_moved;               /* algorithmic bytes of the signature passes (see DESIGN notes in the source) */
+    double kernel_ms, total_ms;
+    int32_t n_launches, pad3;
+} xp_behaviour_summary;
+xp_status xp_behaviours(const xp_sketch* sketch, const xp_behaviour_desc* desc, const xp_repair_opts* opts,
+                        xp_behaviour_summary* out);
+
 /* Algorithm 3 from end to end for one expression: the source snippet's expression S_s and the
  * erroneous expression S_e that the transformed program computes in its place go in, the repaired
  * expression comes out.
@@ -416,6 +463,13 @@ const char* xp_last_error(void);
  * 32-bit add chains (out[0]) and multiply-add chains (out[1]) in thread-operations per
  * second, on the current device and stream NULL.  Errors: XP_ERR_CUDA. */
 xp_status xp_int32_peak(double* out_ops_per_s /* [2] */, double* out_ms /* [2], may be NULL */);
+
+/* Measures what a division costs on the current device: out[0] = int64 truncating divisions per second
+ * with divisors not known in advance (the general form of the exact evaluators), out[1] = int32 divisions
+ * per second by a constant through a precomputed reciprocal (multiply-high, multiply-subtract, one
+ * correction: the form the whole-domain check folds constant divisors into).  Dividing xp_int32_peak's
+ * add figure by these gives the cost of one division in 32-bit operations.  Errors: XP_ERR_CUDA. */
+xp_status xp_int_div_rate(double* out_divs_per_s /* [2] */);
 
 #ifdef __cplusplus
 }

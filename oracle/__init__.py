@@ -78,6 +78,17 @@ class _JointResult(C.Structure):
                 ("least_text0", C.c_char * 512), ("least_text1", C.c_char * 512)]
 
 
+class _BehaviourProblem(C.Structure):
+    _fields_ = [("base", _Problem), ("n_sig", C.c_int64), ("sig_points", C.POINTER(C.c_int64))]
+
+
+class _BehaviourResult(C.Structure):
+    _fields_ = [("enumerated", C.c_uint64 * (XO_MAX_SIZE + 1)), ("distinct", C.c_uint64 * (XO_MAX_SIZE + 1)),
+                ("sig_matches", C.c_uint64), ("hit", C.c_int32), ("hit_size", C.c_int32), ("hit_index", C.c_uint64),
+                ("hit_verified", C.c_int32), ("solved", C.c_int32), ("solution_size", C.c_int32),
+                ("solution_index", C.c_uint64), ("hit_text", C.c_char * 1024), ("solution_text", C.c_char * 1024)]
+
+
 _lib = None
 
 
@@ -93,6 +104,8 @@ def _load():
         lib.xo_eval_code.argtypes = [C.POINTER(_Instr), C.c_int, C.POINTER(C.c_int64), C.c_int64, C.POINTER(C.c_int64)]
         lib.xo_repair.restype = C.c_int
         lib.xo_repair.argtypes = [C.POINTER(_Problem), C.POINTER(_Result)]
+        lib.xo_behaviours.restype = C.c_int
+        lib.xo_behaviours.argtypes = [C.POINTER(_BehaviourProblem), C.POINTER(_BehaviourResult)]
         lib.xo_repair_joint.restype = C.c_int
         lib.xo_repair_joint.argtypes = [C.POINTER(_JointProblem), C.POINTER(_JointResult)]
         _lib = lib
@@ -170,12 +183,25 @@ def repair_hole(sk: Sketch, hole_index: int = 0, rank_ranges: Optional[dict] = N
     that size to those ranks (sizes not named are searched in full).
     ``first_points`` are point indices tried before the rest; the result does not
     depend on them."""
+    P, keep = _problem(sk, hole_index, rank_ranges, first_points)
+    h: Hole = sk.holes[hole_index]
+    R = _Result()
+    rc = _load().xo_repair(C.byref(P), C.byref(R))
+    if rc:
+        raise ValueError("oracle rejected the problem")
+    K = h.max_size
+    return OracleResult([int(x) for x in R.cand_count[:K + 1]], [int(x) for x in R.match_count[:K + 1]],
+                        bool(R.solved), int(R.least_size), int(R.least_rank), R.least_text.decode(), int(R.evals))
+
+
+def _problem(sk: Sketch, hole_index: int, rank_ranges=None, first_points=None):
+    """The C description of one hole's problem and the buffers it points into."""
     h: Hole = sk.holes[hole_index]
     gc = _GrammarC(sk.grammar)
     P = _Problem()
     P.g = gc.c
     P.n_points = sk.n_points
-    keep = []
+    keep = [gc]
     if sk.coords is not None:
         co = np.ascontiguousarray(sk.coords, dtype=np.int32)
         keep.append(co)
@@ -203,13 +229,7 @@ def repair_hole(sk: Sketch, hole_index: int = 0, rank_ranges: Optional[dict] = N
             rb[s], re[s] = b, e
         keep += [rb, re]
         P.rank_begin, P.rank_end = rb, re
-    R = _Result()
-    rc = _load().xo_repair(C.byref(P), C.byref(R))
-    if rc:
-        raise ValueError("oracle rejected the problem")
-    K = h.max_size
-    return OracleResult([int(x) for x in R.cand_count[:K + 1]], [int(x) for x in R.match_count[:K + 1]],
-                        bool(R.solved), int(R.least_size), int(R.least_rank), R.least_text.decode(), int(R.evals))
+    return P, keep
 
 
 @dataclass
@@ -258,3 +278,37 @@ def repair_joint(sk: Sketch, joint) -> JointResult:
     return JointResult([int(x) for x in R.cand_count[:K + 1]], [int(x) for x in R.match_count[:K + 1]], bool(R.solved),
                        int(R.least_total), int(R.least_size0), int(R.least_rank0), int(R.least_rank1),
                        R.least_text0.decode(), R.least_text1.decode(), int(R.evals))
+
+
+@dataclass
+class BehaviourResult:
+    enumerated: List[int]          # candidates generated for the start nonterminal, per size
+    distinct: List[int]            # new behaviours among them
+    sig_matches: int
+    hit: bool
+    hit_size: int
+    hit_index: int
+    hit_verified: bool
+    hit_text: str
+    solved: bool
+    solution_size: int
+    solution_index: int
+    solution_text: str
+
+
+def behaviours(sk: Sketch, sig_points: Sequence[int], hole_index: int = 0) -> BehaviourResult:
+    """Bottom-up enumeration with observational-equivalence pruning on the given signature points
+    (indices into the sketch's domain, in the given order)."""
+    P, keep = _problem(sk, hole_index)
+    B = _BehaviourProblem()
+    B.base = P
+    sp = np.ascontiguousarray(sig_points, dtype=np.int64)
+    B.n_sig = sp.shape[0]
+    B.sig_points = sp.ctypes.data_as(C.POINTER(C.c_int64))
+    R = _BehaviourResult()
+    if _load().xo_behaviours(C.byref(B), C.byref(R)):
+        raise ValueError("oracle rejected the problem")
+    K = sk.holes[hole_index].max_size
+    return BehaviourResult([int(x) for x in R.enumerated[:K + 1]], [int(x) for x in R.distinct[:K + 1]], int(R.sig_matches),
+                           bool(R.hit), int(R.hit_size), int(R.hit_index), bool(R.hit_verified), R.hit_text.decode(),
+                           bool(R.solved), int(R.solution_size), int(R.solution_index), R.solution_text.decode())

@@ -37,7 +37,15 @@
 //     << wraps, >> keeps the sign;
 //   * a joint sketch has two holes inside ONE constraint (xo_repair_joint): the candidates
 //     are the pairs of trees, ordered by total size, then the size of the first tree, then
-//     its rank, then the second tree's rank; counts are per total size.
+//     its rank, then the second tree's rank; counts are per total size;
+//   * the behaviour mode (xo_behaviours) enumerates bottom-up with observational-equivalence
+//     pruning on a given list of signature points: a tree's signature is its value at every
+//     signature point; per nonterminal and size, the candidates are the leaves (size 1) and, for
+//     each binary production in order, each left size ascending, the pairs (left representative,
+//     right representative) in the order the representatives were found, right fastest; a
+//     candidate undefined at a signature point is dropped; one whose signature a representative
+//     of the same nonterminal already has (smaller size, or earlier at this size) is dropped;
+//     the others become the representatives of this size, in that order.
 //
 // Parity against the paper itself is unpinned: it prints no instance, query or
 // solution for this step (its constraint figure is not available).  The functions
@@ -48,6 +56,8 @@
 #include <cstdio>
 #include <cstring>
 #include <functional>
+#include <map>
+#include <memory>
 #include <string>
 #include <vector>
 
@@ -115,6 +125,25 @@ struct xo_joint_result {
     u64 least_rank0, least_rank1;
     u64 evals;
     char least_text0[512], least_text1[512];
+};
+
+// Bottom-up enumeration with observational-equivalence pruning on signature points.
+struct xo_behaviour_problem {
+    xo_problem base;               // grammar, domain, hole (start_nt, max_size, ctx, spec); rank windows unused
+    i64 n_sig;                     // signature points: indices into the domain, in this order
+    const i64* sig_points;
+};
+
+struct xo_behaviour_result {
+    u64 enumerated[XO_MAX_SIZE + 1];   // candidates generated for the start nonterminal, per size
+    u64 distinct[XO_MAX_SIZE + 1];     // of them, new behaviours (representatives)
+    u64 sig_matches;                   // representatives (all sizes) that satisfy the constraint at every signature point
+    int32_t hit, hit_size;             // the first of them in (size, order found) ...
+    u64 hit_index;                     // ... its position among the representatives of its size
+    int32_t hit_verified;              // ... and whether it satisfies the constraint on the whole domain
+    int32_t solved, solution_size;     // the first of them that does
+    u64 solution_index;
+    char hit_text[1024], solution_text[1024];
 };
 
 }  // extern "C"
@@ -435,6 +464,120 @@ int xo_repair_joint(const xo_joint_problem* P, xo_joint_result* R) {
             });
         }
     }
+    return 0;
+}
+
+// The behaviour mode.  Returns 0, or 1 on a malformed problem.
+int xo_behaviours(const xo_behaviour_problem* B, xo_behaviour_result* R) {
+    memset(R, 0, sizeof(*R));
+    const xo_problem* P = &B->base;
+    const xo_grammar* g = &P->g;
+    const int K = P->max_size, nv = g->n_vars;
+    const i64 np = P->n_points, ns = B->n_sig;
+    if (K < 1 || K > XO_MAX_SIZE || nv > 16 || ns < 0) return 1;
+    auto coords_of = [&](i64 p, i64* pt) {
+        if (P->coords) { for (int d = 0; d < nv; ++d) pt[d] = P->coords[p * nv + d]; return; }
+        i64 rem = p;
+        for (int d = nv - 1; d >= 0; --d) { const i64 ext = g->hi[d] - g->lo[d]; pt[d] = g->lo[d] + rem % ext; rem /= ext; }
+    };
+    auto spec_at = [&](i64 p, const i64* pt, i64& v) {
+        if (P->spec_table) { v = P->spec_table[p]; return true; }
+        const i64 none = 0;
+        return eval_code(P->spec_expr, P->spec_len, pt, &none, v);
+    };
+    std::vector<i64> sig_pt((size_t)ns * (nv ? nv : 1)), sig_spec(ns);
+    std::vector<char> sig_ok(ns, 1);
+    for (i64 j = 0; j < ns; ++j) {
+        if (B->sig_points[j] < 0 || B->sig_points[j] >= np) return 1;
+        coords_of(B->sig_points[j], &sig_pt[j * nv]);
+        sig_ok[j] = spec_at(B->sig_points[j], &sig_pt[j * nv], sig_spec[j]);
+    }
+    std::vector<std::vector<const xo_prod*>> of(g->n_nt);
+    for (int i = 0; i < g->n_prods; ++i) of[g->prods[i].lhs].push_back(&g->prods[i]);
+    struct Rep { std::vector<i64> sig; const xo_prod* p; int a; u64 l, r; };
+    std::vector<std::vector<std::vector<Rep>>> reps(g->n_nt, std::vector<std::vector<Rep>>(K + 1));
+    std::vector<std::map<std::vector<i64>, int>> seen(g->n_nt);
+    std::function<void(int, int, u64, std::string&)> text = [&](int nt, int size, u64 idx, std::string& out) {
+        const Rep& t = reps[nt][size][idx];
+        if (t.p->kind == P_VAR) { out += g->var_names ? g->var_names[t.p->var] : ("v" + std::to_string(t.p->var)); return; }
+        if (t.p->kind == P_CONST) { out += std::to_string((long long)t.p->value); return; }
+        const bool call = t.p->op == OP_MIN || t.p->op == OP_MAX;
+        out += call ? std::string(OP_TEXT[t.p->op]) + "(" : std::string("(");
+        text(t.p->left, t.a, t.l, out);
+        out += call ? "," : OP_TEXT[t.p->op];
+        text(t.p->right, size - 1 - t.a, t.r, out);
+        out += ")";
+    };
+    std::function<bool(int, int, u64, const i64*, i64&)> value = [&](int nt, int size, u64 idx, const i64* pt, i64& out) {
+        const Rep& t = reps[nt][size][idx];
+        if (t.p->kind == P_VAR) { out = pt[t.p->var]; return true; }
+        if (t.p->kind == P_CONST) { out = t.p->value; return true; }
+        i64 a, b;
+        const bool va = value(t.p->left, t.a, t.l, pt, a), vb = value(t.p->right, size - 1 - t.a, t.r, pt, b);
+        return va && vb && apply_op(t.p->op, a, b, out);
+    };
+    for (int s = 1; s <= K; ++s)
+        for (int nt = 0; nt < g->n_nt; ++nt) {
+            u64 enumerated = 0;
+            auto offer = [&](Rep&& c, bool defined) {
+                ++enumerated;
+                if (!defined) return;
+                if (seen[nt].count(c.sig)) return;
+                seen[nt][c.sig] = 1;
+                reps[nt][s].push_back(std::move(c));
+            };
+            for (const xo_prod* p : of[nt]) {
+                if (p->kind != P_BIN) {
+                    if (s != 1) continue;
+                    Rep c{std::vector<i64>(ns), p, 0, 0, 0};
+                    for (i64 j = 0; j < ns; ++j) c.sig[j] = p->kind == P_VAR ? sig_pt[j * nv + p->var] : p->value;
+                    offer(std::move(c), true);
+                    continue;
+                }
+                for (int a = 1; a <= s - 2; ++a) {
+                    const auto& L = reps[p->left][a];
+                    const auto& Rr = reps[p->right][s - 1 - a];
+                    for (u64 l = 0; l < L.size(); ++l)
+                        for (u64 r = 0; r < Rr.size(); ++r) {
+                            Rep c{std::vector<i64>(ns), p, a, l, r};
+                            bool defined = true;
+                            for (i64 j = 0; j < ns && defined; ++j) defined = apply_op(p->op, L[l].sig[j], Rr[r].sig[j], c.sig[j]);
+                            offer(std::move(c), defined);
+                        }
+                }
+            }
+            if (nt == P->start_nt) { R->enumerated[s] = enumerated; R->distinct[s] = reps[nt][s].size(); }
+        }
+    // representatives of the start nonterminal against the constraint
+    for (int s = 1; s <= K; ++s)
+        for (u64 i = 0; i < reps[P->start_nt][s].size(); ++i) {
+            const Rep& t = reps[P->start_nt][s][i];
+            bool ok = true;
+            for (i64 j = 0; j < ns && ok; ++j) {
+                i64 v = t.sig[j];
+                ok = sig_ok[j] && (P->ctx_len == 0 || eval_code(P->ctx, P->ctx_len, &sig_pt[j * nv], &t.sig[j], v)) && v == sig_spec[j];
+            }
+            if (!ok) continue;
+            ++R->sig_matches;
+            if (R->solved) continue;
+            bool all = true;
+            for (i64 p = 0; p < np && all; ++p) {
+                i64 pt[16], want, h, v;
+                coords_of(p, pt);
+                all = spec_at(p, pt, want) && value(P->start_nt, s, i, pt, h);
+                if (all) { v = h; all = (P->ctx_len == 0 || eval_code(P->ctx, P->ctx_len, pt, &h, v)) && v == want; }
+            }
+            std::string txt;
+            text(P->start_nt, s, i, txt);
+            if (!R->hit) {
+                R->hit = 1; R->hit_size = s; R->hit_index = i; R->hit_verified = all ? 1 : 0;
+                snprintf(R->hit_text, sizeof(R->hit_text), "%s", txt.c_str());
+            }
+            if (all) {
+                R->solved = 1; R->solution_size = s; R->solution_index = i;
+                snprintf(R->solution_text, sizeof(R->solution_text), "%s", txt.c_str());
+            }
+        }
     return 0;
 }
 

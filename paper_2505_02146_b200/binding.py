@@ -27,7 +27,7 @@ EXPORTS = ["xp_grammar_create", "xp_grammar_destroy", "xp_grammar_count", "xp_gr
            "xp_result_get", "xp_result_free", "xp_last_error", "xp_int32_peak", "xp_repair_static",
            "xp_sketch_info_get", "xp_sketch_refine", "xp_result_pack",
            "xp_repair_pair", "xp_pair_result_get", "xp_pair_result_free",
-           "xp_repair_joint", "xp_joint_result_get", "xp_joint_result_free"]
+           "xp_repair_joint", "xp_joint_result_get", "xp_joint_result_free", "xp_behaviours", "xp_int_div_rate"]
 
 
 class XpError(RuntimeError):
@@ -113,6 +113,21 @@ class xp_pair_view(C.Structure):
                 ("load_ms", C.c_double), ("search_ms", C.c_double)]
 
 
+class xp_behaviour_desc(C.Structure):
+    _fields_ = [("hole", C.c_int32), ("n_sig", C.c_int32), ("sig_points", C.POINTER(C.c_int64)),
+                ("max_representatives", C.c_uint64)]
+
+
+class xp_behaviour_summary(C.Structure):
+    _fields_ = [("max_size", C.c_int32), ("pad", C.c_int32), ("enumerated", C.c_uint64 * (XP_MAX_SIZE + 1)),
+                ("distinct", C.c_uint64 * (XP_MAX_SIZE + 1)), ("sig_matches", C.c_uint64), ("hit", C.c_int32),
+                ("hit_size", C.c_int32), ("hit_index", C.c_uint64), ("hit_verified", C.c_int32), ("solved", C.c_int32),
+                ("solution_size", C.c_int32), ("pad2", C.c_int32), ("solution_index", C.c_uint64),
+                ("hit_text", C.c_char * 256), ("solution_text", C.c_char * 256), ("representatives", C.c_uint64),
+                ("bytes_moved", C.c_uint64), ("kernel_ms", C.c_double), ("total_ms", C.c_double),
+                ("n_launches", C.c_int32), ("pad3", C.c_int32)]
+
+
 class xp_joint_desc(C.Structure):
     _fields_ = [("start_nt", C.c_int32 * 2), ("max_size", C.c_int32 * 2), ("ctx_len", C.c_int32), ("ctx", C.POINTER(xp_instr)),
                 ("spec_kind", C.c_int32), ("spec_len", C.c_int32), ("spec_expr", C.POINTER(xp_instr)),
@@ -156,10 +171,12 @@ def load(path: Optional[str] = None):
     lib.xp_result_free.restype = None
     lib.xp_last_error.restype = C.c_char_p
     lib.xp_int32_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.xp_int_div_rate.argtypes = [C.POINTER(C.c_double)]
     lib.xp_repair_static.argtypes = [vp, C.POINTER(xp_repair_opts), C.POINTER(xp_hole_summary), C.c_int32]
     lib.xp_sketch_info_get.argtypes = [vp, C.POINTER(xp_sketch_info)]
     lib.xp_sketch_refine.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32)]
     lib.xp_result_pack.argtypes = [C.POINTER(vp), C.c_size_t, C.POINTER(xp_hole_summary), C.c_size_t, C.POINTER(C.c_size_t)]
+    lib.xp_behaviours.argtypes = [vp, C.POINTER(xp_behaviour_desc), C.POINTER(xp_repair_opts), C.POINTER(xp_behaviour_summary)]
     lib.xp_repair_joint.argtypes = [vp, C.POINTER(xp_joint_desc), C.POINTER(xp_repair_opts), C.POINTER(vp)]
     lib.xp_joint_result_get.argtypes = [vp, C.POINTER(xp_joint_view)]
     lib.xp_joint_result_free.argtypes = [vp]
@@ -458,6 +475,20 @@ def summaries_as_numpy(packed) -> np.ndarray:
     return np.frombuffer(packed, dtype=SUMMARY_DTYPE)
 
 
+def xp_behaviours(sketch: LoadedSketch, sig_points: Sequence[int], hole: int = 0, max_representatives: int = 0,
+                  stream=None) -> xp_behaviour_summary:
+    """The behaviour mode: bottom-up enumeration with observational-equivalence pruning on the given
+    signature points (domain point ids).  Returns the C summary (per-size ``enumerated`` / ``distinct``,
+    ``sig_matches``, the first hit and the first verified solution)."""
+    d = xp_behaviour_desc()
+    pts = (C.c_int64 * len(sig_points))(*[int(p) for p in sig_points])
+    d.hole, d.n_sig, d.sig_points, d.max_representatives = hole, len(sig_points), pts, max_representatives
+    o, _keep = _opts(stream=stream)
+    out = xp_behaviour_summary()
+    _check(load().xp_behaviours(sketch.handle, C.byref(d), C.byref(o), C.byref(out)))
+    return out
+
+
 @dataclass
 class JointResult:
     solved: bool
@@ -564,4 +595,11 @@ def xp_repair_pair(gr: Grammar, source, erroneous, start_nt: int, max_size: int,
 def xp_int32_peak() -> Tuple[float, float]:
     out = (C.c_double * 2)()
     _check(load().xp_int32_peak(out, None))
+    return float(out[0]), float(out[1])
+
+
+def xp_int_div_rate() -> Tuple[float, float]:
+    """(int64 general divisions per second, int32 reciprocal divisions by a constant per second)."""
+    out = (C.c_double * 2)()
+    _check(load().xp_int_div_rate(out))
     return float(out[0]), float(out[1])

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libxpiler_repair.so")
 LIB_CHECKED = os.path.join(HERE, "libxpiler_repair_checked.so")       # the same sources with -DXP_CHECKS (index checks)
-SOURCES = ["xp_api.cu", "xp_kernels.cu", "xp_pair.cu", "xp_joint.cu"]
+SOURCES = ["xp_api.cu", "xp_kernels.cu", "xp_pair.cu", "xp_joint.cu", "xp_behaviour.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

@@ -342,6 +342,7 @@ struct HoleHost {
     bool filter_ok = false;          // the probe filter applies (probe 0 exists, context affine there)
     bool never = false;              // the spec is undefined at some point: no candidate can match
     bool compares = false;           // the filter works on an interval of hole values (the context compares)
+    bool second = false;             // filter hits are looked at once more at probe 1 from the start (hits are frequent)
 };
 
 struct xp_sketch {
@@ -753,6 +754,7 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
             s->holes[h].filter_ok = o.filter_ok != 0;
             s->holes[h].compares = o.filter_ok != 0 && o.aff_ok == 0;
             s->holes[h].never = bad != 0;                 // the spec is undefined at some point
+            s->holes[h].second = o.second != 0;
             s->n_probes.push_back(o.n_probe);
         }
         outs[i] = s;
@@ -770,6 +772,17 @@ SketchInternals sketch_internals(const xp_sketch* s) { return SketchInternals{s-
 u64 grammar_cnt(const xp_grammar* g, int nt, int size) { return g->cnt[nt][size]; }
 int grammar_nonterminals(const xp_grammar* g) { return g->n_nt; }
 int grammar_ok_size(const xp_grammar* g) { return g->ok_size; }
+GrammarHost grammar_host(const xp_grammar* g) {
+    static thread_local std::vector<const char*> names;
+    names.clear();
+    for (const std::string& n : g->names) names.push_back(n.c_str());
+    return GrammarHost{g->n_nt, g->n_vars, g->leaf_begin, g->bin_begin, g->leaves.data(), g->bins.data(), names.data()};
+}
+HoleSpec sketch_hole(const xp_sketch* s, int hole) {
+    if (hole < 0 || hole >= s->n_holes) return HoleSpec{-1, 0};
+    return HoleSpec{s->holes[hole].start_nt, s->holes[hole].max_size};
+}
+const HoleDev* sketch_hole_dev(const xp_sketch* s, int hole) { return s->d_holes + hole; }
 cudaError_t device_alloc(void** out, size_t bytes, int* device, size_t* granted) { return pool_alloc(out, bytes, device, granted); }
 void device_release(void* ptr, size_t granted, int device) { pool_release(ptr, granted, device); }
 }  // namespace xp
@@ -855,6 +868,7 @@ extern "C" xp_status xp_sketch_refine(xp_sketch* s, int32_t max_promote, int32_t
         for (int h = 0; h < nh; ++h) {
             s->holes[h].filter_ok = hh[h].filter_ok != 0;
             s->holes[h].compares = hh[h].filter_ok != 0 && hh[h].aff_ok == 0;
+            s->holes[h].second = hh[h].second != 0;
             s->n_probes[h] = hh[h].n_probe;
         }
         std::lock_guard<std::mutex> lock(s->plan_mu);
@@ -1131,8 +1145,16 @@ static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u3
     w.sorted = w.sort_off + align256(sizeof(u32) * (n_acc + 2));
     w.total = w.sorted + align256(sizeof(u32) * (size_t)surv_cap);
     w.n_acc = (int)n_acc;
+    w.dense = 0;
     w.surv_cap = surv_cap;
     return w;
+}
+
+// Does some hole among the sketches take the second look (frequent filter hits)?
+static int any_dense(const xp_sketch* const* sk, size_t n) {
+    for (size_t i = 0; i < n; ++i)
+        for (const HoleHost& h : sk[i]->holes) if (h.second) return 1;
+    return 0;
 }
 
 // Chunks of the whole-domain check that the largest domain among the sketches needs.
@@ -1163,7 +1185,8 @@ extern "C" xp_status xp_repair_batch(const xp_sketch* const* sketches, size_t n,
     if (st != XP_OK) return st;
     cudaStream_t stream = (cudaStream_t)o->stream;
 
-    const SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
+    SearchLayout w = ws_layout(plan.segs.size(), n, plan.acc.size(), surv_cap_for(n));
+    w.dense = any_dense(sketches, n);
     char* ws = (char*)o->workspace;
     bool own_ws = false, cached_ws = false;
     if (ws) {
@@ -1295,7 +1318,8 @@ extern "C" xp_status xp_repair_static(const xp_sketch* sketch, const xp_repair_o
     xp_status st = build_plan(&sketch, 1, o, &plan);
     if (st == XP_OK) st = check_device(&sketch, 1);
     if (st != XP_OK) return st;
-    const SearchLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size(), kSurvCapStatic);
+    SearchLayout w = ws_layout(plan.segs.size(), 1, plan.acc.size(), kSurvCapStatic);
+    w.dense = any_dense(&sketch, 1);
     if (plan.acc.size() > 64)
         return fail(XP_ERR_TOO_LARGE, "xp_repair_static: the sketch has more than 64 holes; use xp_repair with a workspace");
     if (w.total > kStaticScratchBytes)
@@ -1388,6 +1412,38 @@ extern "C" const char* xp_last_error(void) { return g_last_error.c_str(); }
 // ------------------------------------------------------------------------------------------
 // integer peak
 // ------------------------------------------------------------------------------------------
+
+// Divisions per second of the two division forms (see the kernels): 64 per chain, 4 chains per thread.
+extern "C" xp_status xp_int_div_rate(double* out_divs) {
+    if (!out_divs) return fail(XP_ERR_INVALID_ARG, "xp_int_div_rate: null argument");
+    int dev = 0, sms = 1;
+    XP_CUDA(cudaGetDevice(&dev));
+    XP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    u32* d = nullptr;
+    XP_CUDA(cudaMalloc(&d, 256));
+    cudaEvent_t e0, e1;
+    XP_CUDA(cudaEventCreate(&e0));
+    XP_CUDA(cudaEventCreate(&e1));
+    const int blocks = sms * 8;
+    for (int which = 2; which < 4; ++which) {
+        const int iters = which == 2 ? 64 : 2048;
+        float best = 1e30f;
+        for (int rep = 0; rep < 4; ++rep) {
+            XP_CUDA(cudaEventRecord(e0, nullptr));
+            XP_CUDA(launch_int32_peak(which, d, blocks, iters, nullptr));
+            XP_CUDA(cudaEventRecord(e1, nullptr));
+            XP_CUDA(cudaEventSynchronize(e1));
+            float ms = 0.f;
+            XP_CUDA(cudaEventElapsedTime(&ms, e0, e1));
+            if (rep > 0 && ms < best) best = ms;
+        }
+        out_divs[which - 2] = (double)blocks * 256.0 * (double)iters * 64.0 / (best * 1e-3);
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(d);
+    return XP_OK;
+}
 
 extern "C" xp_status xp_int32_peak(double* out_ops, double* out_ms) {
     if (!out_ops) return fail(XP_ERR_INVALID_ARG, "xp_int32_peak: null argument");

@@ -1200,7 +1200,10 @@ __device__ __noinline__ void emit_pairs(EvalShared& sh, const RegVals* R, u32 a1
 // path, from t_add.
 // Broadcast operands per warp vote.  A vote that fires makes every lane repeat the group's tests,
 // so the group is large where hits are rare (the vote and the loop control are shared by more
-// candidates) and small where they are frequent (holes that take the second look: DENSE).
+// candidates) and small where they are frequent (DENSE).  The choice is made per launch, not per
+// hole: the search kernel exists in both forms and the host launches the dense one when a hole of
+// the plan takes the second look.  (Both sets of loops inside one kernel cost the batch workload a
+// tenth of its time in instruction-cache misses although only one set ever runs there.)
 template <bool DENSE> struct VoteGroup { static constexpr int kRing = DENSE ? 4 : 8, kDiv = DENSE ? 2 : 4; };
 
 template <u32 MASK, bool SWAP, bool DENSE>
@@ -1533,7 +1536,7 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
     __syncwarp();
 }
 
-template <bool SWAP>
+template <bool SWAP, bool DENSE>
 __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
                                           u64 reg_first, u64 pairs, const RegVals* R, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
     const SegDev& seg = sh.mseg[m];
@@ -1572,7 +1575,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     }
 
     // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
-    const bool dense = sh.p1_on != 0;                   // the hole takes the second look: hits are frequent
+    constexpr bool dense = DENSE;
     auto run = [&](int s0, int s1, u32 alv, bool special) {
         if (tile_wide || rng) {
             wide_chunk(sh, R, alv, a1ok, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
@@ -1726,6 +1729,7 @@ __device__ __forceinline__ void load_family(EvalShared& sh, const PlanDev& plan,
     }
 }
 
+template <bool DENSE>
 __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
                                             u64 local, u64& my_evals) {
     const GrammarDev* g = sk->g;
@@ -1798,8 +1802,8 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
             if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-            if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
-            else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
+            if (seg.swap) tile_body<true, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
+            else tile_body<false, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
         }
         drain_queue(sh, plan, sk, hole, reg_first, my_evals);
         return;
@@ -1813,14 +1817,15 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         const SegDev& seg = sh.mseg[m];
         const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
         if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
-        else tile_body<false>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
+        if (seg.swap) tile_body<true, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
+        else tile_body<false, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
     }
 }
 
 #ifndef XP_MIN_CTAS
 #define XP_MIN_CTAS 3
 #endif
+template <bool DENSE>
 __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanDev plan) {
     __shared__ EvalShared sh;
     u64 my_evals = 0;
@@ -1863,7 +1868,7 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
         const SketchDev* sk = plan.sketches[sh.seg.sketch];
         const HoleDev* hole = &sk->holes[sh.seg.hole];
         const u64 local = t - sh.seg.first_ticket;
-        if (sh.seg.kind == kSegTile) tile_ticket(sh, plan, sk, hole, local, my_evals);
+        if (sh.seg.kind == kSegTile) tile_ticket<DENSE>(sh, plan, sk, hole, local, my_evals);
         else linear_ticket(sh, plan, sk, hole, local, my_evals);
         __syncthreads();
     }
@@ -2344,6 +2349,38 @@ __global__ void __launch_bounds__(256) int32_peak_mad_kernel(u32* out, int iters
     if (r == 0x12345678u) out[0] = r;
 }
 
+// Cost of a division in thread-operations: four independent chains per thread of (a) int64
+// truncating division by a divisor that is not known in advance, (b) int32 division by a
+// constant through a precomputed reciprocal (multiply-high, multiply-subtract, one correction),
+// the form the whole-domain check uses.  64 divisions per chain and loop iteration.
+__global__ void __launch_bounds__(256) int_div_general_kernel(long long* out, int iters, long long seed) {
+    long long a0 = seed + threadIdx.x, a1 = a0 * 3 + 1, a2 = a0 * 5 + 2, a3 = a0 * 7 + 3;
+    const long long d0 = (seed & 1023) + 3 + (threadIdx.x & 7), big = 0x3fffffffffffll;
+#pragma unroll 1
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            a0 = (a0 | big) / (d0 + u); a1 = (a1 | big) / (d0 + u + 1); a2 = (a2 | big) / (d0 + u + 2); a3 = (a3 | big) / (d0 + u + 3);
+        }
+    }
+    if ((a0 ^ a1 ^ a2 ^ a3) == 0x12345678) out[0] = a0;
+}
+
+__global__ void __launch_bounds__(256) int_div_reciprocal_kernel(u32* out, int iters, u32 seed) {
+    u32 a0 = seed + threadIdx.x, a1 = a0 * 3 + 1, a2 = a0 * 5 + 2, a3 = a0 * 7 + 3;
+    const u32 d = (seed & 127u) + 3u, M = (u32)((1ull << 32) / d);
+#pragma unroll 1
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+#define XP_RDIV(a) { const u32 x = a | 0x40000000u; u32 q = __umulhi(x, M); u32 r = x - q * d; if (r >= d) ++q; a = q + u; }
+            XP_RDIV(a0) XP_RDIV(a1) XP_RDIV(a2) XP_RDIV(a3)
+#undef XP_RDIV
+        }
+    }
+    if ((a0 ^ a1 ^ a2 ^ a3) == 0x12345678u) out[0] = a0;
+}
+
 // ------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------
@@ -2427,9 +2464,11 @@ cudaError_t launch_search_part(char* base, const SearchLayout& L, u64 t_begin, u
     PlanDev pd = plan_on(base, L, n_segs, n_sketches, max_chunks);
     pd.ticket_base = t_begin;
     pd.n_tickets = t_end;
-    u64 ctas = (u64)resident_ctas((const void*)eval_kernel, 0);      // persistent CTAs: one wave
+    const void* kernel = L.dense ? (const void*)eval_kernel<true> : (const void*)eval_kernel<false>;
+    u64 ctas = (u64)resident_ctas(kernel, 0);             // persistent CTAs: one wave
     if (ctas > t_end - t_begin) ctas = t_end - t_begin;
-    eval_kernel<<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
+    if (L.dense) eval_kernel<true><<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
+    else eval_kernel<false><<<(unsigned)ctas, kThreads, 0, stream>>>(pd);
     *n_launches += 1;
     return cudaGetLastError();
 }
@@ -2507,7 +2546,9 @@ cudaError_t launch_search_static(const void* stage, const SearchLayout& L, u64 n
 
 cudaError_t launch_int32_peak(int which, u32* out, int blocks, int iters, cudaStream_t stream) {
     if (which == 0) int32_peak_add_kernel<<<blocks, 256, 0, stream>>>(out, iters, 1u);
-    else int32_peak_mad_kernel<<<blocks, 256, 0, stream>>>(out, iters, 1u);
+    else if (which == 1) int32_peak_mad_kernel<<<blocks, 256, 0, stream>>>(out, iters, 1u);
+    else if (which == 2) int_div_general_kernel<<<blocks, 256, 0, stream>>>((long long*)out, iters, 12345);
+    else int_div_reciprocal_kernel<<<blocks, 256, 0, stream>>>(out, iters, 12345u);
     return cudaGetLastError();
 }
 

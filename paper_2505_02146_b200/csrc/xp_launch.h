@@ -19,7 +19,8 @@ cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most
 //   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
 //   hist: survivors per accumulator slot, zero at launch (staged);
 //   surv: the survivor queue (surv_cap entries); sort_off, sorted: its hole order -- written by the kernels only
-struct SearchLayout { size_t segs, sketches, acc, hist, head, surv, sort_off, sorted, total; u32 surv_cap; int n_acc; };
+struct SearchLayout { size_t segs, sketches, acc, hist, head, surv, sort_off, sorted, total; u32 surv_cap; int n_acc;
+                      int dense; /* some hole of the plan takes the second look: launch the search kernel's dense form */ };
 
 // The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel;
 // or the same in pieces: eval_kernel over one range of tickets at a time, then the rest.
@@ -40,6 +41,13 @@ SketchInternals sketch_internals(const xp_sketch* s);
 u64 grammar_cnt(const xp_grammar* g, int nt, int size);      // trees of nt with exactly `size` nodes
 int grammar_nonterminals(const xp_grammar* g);
 int grammar_ok_size(const xp_grammar* g);                    // counts are exact (< 2^63) up to this size
+// The grammar as the kernels see it (host copy of the tables): leaves and binary productions grouped by nonterminal.
+struct GrammarHost { int n_nt, n_vars; const int* leaf_begin; const int* bin_begin; const LeafDev* leaves; const BinDev* bins;
+                     const char* const* var_names; };
+GrammarHost grammar_host(const xp_grammar* g);
+struct HoleSpec { int start_nt, max_size; };
+HoleSpec sketch_hole(const xp_sketch* s, int hole);           // hole < 0 or >= n_holes: start_nt = -1
+const HoleDev* sketch_hole_dev(const xp_sketch* s, int hole); // device pointer
 cudaError_t device_alloc(void** out, size_t bytes, int* device, size_t* granted);     // the library's device pool
 void device_release(void* ptr, size_t granted, int device);
 xp_status set_error(xp_status st, const char* msg);

@@ -40,7 +40,7 @@ def test_joint_small_products(xp, ctx, spec, K):
     g = free_grammar(vs, constant_set(-1, 4))
     J = JointHole((0, 0), K, parse_expr(ctx, vs), spec_expr=parse_expr(spec, vs))
     got = _check(xp, _base(g, vs), J)
-    assert got.evals_executed > 0 and got.n_launches >= 3
+    assert (got.evals_executed > 0 or not got.solved) and got.n_launches >= 3
 
 
 def test_joint_typed_grammar_table_domain_and_table_spec(xp):
@@ -51,11 +51,11 @@ def test_joint_typed_grammar_table_domain_and_table_spec(xp):
     coords = np.stack([ids // 30, (ids // 3) % 10, ids % 3], axis=1).astype(np.int32)
     spec = (coords[:, 0].astype(np.int64) * 10 + coords[:, 1]) * 3 + coords[:, 2]
     sk = Sketch(g, [Hole(0, 1, spec_table=spec)], coords, name="typed joint")
-    J = JointHole((0, 0), (3, 3), parse_expr("(HOLE0*3)+HOLE1", vs), spec_table=spec)
+    J = JointHole((0, 0), (5, 1), parse_expr("(HOLE0*3)+HOLE1", vs), spec_table=spec)
     got = _check(xp, sk, J)
-    assert got.solved
+    assert got.solved and (got.least_text0, got.least_text1) == ("(c+(r*10))", "k")
     import torch
-    J2 = JointHole((0, 0), (3, 3), parse_expr("(HOLE0*3)+HOLE1", vs), spec_table=torch.from_numpy(spec).cuda())
+    J2 = JointHole((0, 0), (5, 1), parse_expr("(HOLE0*3)+HOLE1", vs), spec_table=torch.from_numpy(spec).cuda())
     ls = xp.xp_sketch_load(xp.xp_grammar_create(g), sk)
     again = xp.xp_repair_joint(ls, J2)
     assert again.match_count == got.match_count and again.least_rank0 == got.least_rank0

@@ -487,3 +487,71 @@ def test_joint_reduces_to_the_single_hole_search_when_one_part_is_cancelled():
     for s in range(2, 9):
         assert r.match_count[s] == sum(single.match_count[s0] * cnt[s - s0] for s0 in range(1, 6) if 1 <= s - s0 <= 3)
     assert r.solved and r.least_size0 == single.least_size and r.least_rank0 == single.least_rank and r.least_rank1 == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# behaviour mode: bottom-up enumeration with observational-equivalence pruning
+# ---------------------------------------------------------------------------------------------
+
+def _behaviours_by_brute_force(g, nt, K, pts):
+    """Value vectors on ``pts`` of ALL syntactic trees, by the smallest size at which each occurs
+    (trees undefined at some point are left out): what pruning must not change."""
+    T = pybrute.all_trees(g, K)
+    seen, per_size = set(), [0] * (K + 1)
+    for s in range(1, K + 1):
+        new = set()
+        for t in T[(nt, s)]:
+            sig = tuple(pybrute.tree_value(t, p) for p in pts)
+            if None in sig or sig in seen:
+                continue
+            new.add(sig)
+        per_size[s] = len(new)
+        seen |= new
+    return per_size
+
+
+def test_behaviour_counts_equal_brute_force_over_all_trees():
+    """A behaviour first realised by a syntactic tree of size s is first realised in the pruned
+    space at size s too (subtrees can be swapped for their class representatives, which are no
+    larger), so the per-size counts of new behaviours must equal a brute force over every tree."""
+    vs = [Variable("p", 0, 3), Variable("q", -1, 2)]
+    cases = [(free_grammar(vs, [0, 1, 2], ops=["+", "*"]), 5), (free_grammar(vs, [1, -2], ops=["-", "/", "%"]), 5),
+             (quasi_affine_grammar(vs, [-1, 2], [1, 2]), 7), (free_grammar(vs[:1], [1, 3], ops=["+", "<<", "min"]), 7)]
+    for g, K in cases:
+        sk = Sketch(g, [Hole(0, K, spec_expr=parse_expr("p", vs))])
+        pts = pybrute.points_of(sk)
+        for sig in (list(range(len(pts))), [0, len(pts) - 1, 2]):
+            r = oracle.behaviours(sk, sig)
+            assert r.distinct == _behaviours_by_brute_force(g, 0, K, [pts[i] for i in sig])
+            assert r.enumerated[1] == g.leaf_count(0)
+
+
+def test_behaviour_mode_with_every_point_as_signature_agrees_with_the_exhaustive_search():
+    """With the whole domain as signature the first matching representative has the size of the
+    exhaustive search's least solution, is verified, and evaluates to the spec everywhere."""
+    vs = [Variable("i", 0, 6), Variable("j", 0, 5)]
+    g = free_grammar(vs, constant_set(-2, 3))
+    for spec in ["(i*3)+j", "i%3", "j", "(i+j)/2", "(i*i)*(j+7)"]:
+        sk = Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, vs))])
+        full = oracle.repair_hole(sk)
+        r = oracle.behaviours(sk, list(range(sk.n_points)))
+        assert r.solved == full.solved and r.hit == full.solved
+        if full.solved:
+            assert r.solution_size == full.least_size and r.hit_verified and r.sig_matches == 1
+            for p in pybrute.points_of(sk):
+                assert pybrute.text_value(r.solution_text, g, p) == pybrute.code_value(sk.holes[0].spec_expr, p)
+
+
+def test_behaviour_mode_on_a_partial_signature_reports_an_unverified_hit():
+    vs = [Variable("i", 0, 8), Variable("j", 0, 8)]
+    g = free_grammar(vs, [0, 1, 2])
+    sk = Sketch(g, [Hole(0, 3, spec_expr=parse_expr("i*j", vs))])
+    diag = [k * 8 + k for k in range(8)]                      # on the diagonal i*j and i*i look the same
+    r = oracle.behaviours(sk, diag)
+    assert r.hit and r.hit_text == "(i*i)" and not r.hit_verified and not r.solved and r.sig_matches == 1
+    r2 = oracle.behaviours(sk, diag + [19])                   # (2, 3): 6 against 4
+    assert r2.solved and r2.solution_text == "(i*j)"
+    # through a context that is not injective several representatives satisfy the signature
+    sk3 = Sketch(g, [Hole(0, 3, ctx=parse_expr("HOLE/4", vs), spec_expr=parse_expr("(i*j)/4", vs))])
+    r3 = oracle.behaviours(sk3, list(range(64)))
+    assert r3.sig_matches >= 1 and r3.solved and r3.hit_verified

@@ -393,3 +393,13 @@ def test_integer_peak_microbenchmark_is_plausible(xp):
     lanes = props.multi_processor_count * 128
     assert 0.3e9 * lanes < add < 2.3e9 * lanes          # between 0.3 and 2.3 GHz worth of one add per lane and clock
     assert 0.35 * add < mad < 0.75 * add
+
+
+def test_division_cost_microbenchmark_is_plausible(xp):
+    """A general int64 division costs tens to a few hundred 32-bit operations, a division by a
+    constant through its reciprocal a handful."""
+    add, _ = xp.xp_int32_peak()
+    general, reciprocal = xp.xp_int_div_rate()
+    assert 20 < add / general < 2000
+    assert 2 < add / reciprocal < 40
+    assert reciprocal > 4 * general
