@@ -53,7 +53,7 @@ xp_status set_error(xp_status st, const char* msg) { return fail(st, msg); }    
 // up to kPoolBigKeep bytes in all, and handed out again to a request of the same size.  Slabs
 // and kept blocks are returned to the driver when the process ends.  One pool per device.
 namespace {
-constexpr size_t kPoolSlabBytes = 64ull << 20, kPoolBigBytes = 16ull << 20, kPoolBigKeep = 1ull << 30;
+constexpr size_t kPoolSlabBytes = 64ull << 20, kPoolBigBytes = 16ull << 20, kPoolBigKeep = 24ull << 30;
 struct DevPool {
     std::multimap<size_t, char*> free_blocks;
     std::multimap<size_t, char*> big_blocks;
@@ -122,6 +122,36 @@ void pool_release(void* ptr, size_t bytes, int device) {
 
 struct xp_sketch;
 static xp_status check_device(const xp_sketch* const* sk, size_t n);
+
+// Page-locked host memory for the staged copies of a load (what goes to the device and what comes
+// back), kept by the library from load to load: copies from and to page-locked memory are queued
+// without the extra pass through the driver's own staging buffer that a copy from ordinary memory
+// takes, which for a batch of thousands of sketches was most of the load's time.  One load uses it
+// at a time (a concurrent load falls back to ordinary memory).
+namespace {
+constexpr size_t kPinnedChunk = 64ull << 20, kPinnedMost = 1ull << 30;
+struct PinnedArena {
+    std::mutex mu;
+    std::vector<char*> chunks;
+    size_t chunk = 0, used = 0;
+    void reset() { chunk = 0; used = 0; }
+    char* take(size_t bytes) {
+        const size_t need = (bytes + 255) & ~(size_t)255;
+        if (need > kPinnedChunk) return nullptr;
+        if (chunk < chunks.size() && used + need > kPinnedChunk) { ++chunk; used = 0; }
+        if (chunk >= chunks.size()) {
+            if ((chunks.size() + 1) * kPinnedChunk > kPinnedMost) return nullptr;
+            void* p = nullptr;
+            if (cudaHostAlloc(&p, kPinnedChunk, cudaHostAllocDefault) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+            chunks.push_back((char*)p);
+        }
+        char* out = chunks[chunk] + used;
+        used += need;
+        return out;
+    }
+};
+PinnedArena g_pinned;
+}  // namespace
 
 static const char* const kOpText[] = {"+", "-", "*", "/", "%", "<", "<=", "==", "!=", "min", "max", "&&", "||", "<<", ">>"};
 
@@ -364,6 +394,7 @@ struct xp_sketch {
     size_t off_holes = 0;
     int tab_size_cap = 0, tab_probes_cap = 0;        // most sizes / probes that the subtree tables of a hole cover
     u64 entries_at[kMaxSize + 1] = {0};              // subtree-table entries per size (all nonterminals)
+    u64 big_entries = 0;                             // most entries of a hole's first-probe table of the next size
     // The sketch's part of a launch plan under default options (every size, no rank window, no flag), as
     // if it were the only sketch of the call: built on the first such call and copied, with ticket, sketch
     // and accumulator numbers shifted, into the plan of every later one (a batch of thousands of small
@@ -429,11 +460,15 @@ static u64 table_entries(const xp_grammar* g, int max_size, u64 (*off)[kMaxSize 
 struct LoadState {
     xp_sketch* s = nullptr;
     std::vector<HoleDev> hh;
-    std::vector<char> back;          // holes and flags as the kernels left them
+    std::vector<char> back_own;      // holes and flags as the kernels left them (ordinary memory, when no page-locked
+    char* back = nullptr;            //   memory could be had); back points at whichever holds them
+    size_t back_bytes = 0;
+    PinnedArena* pinned = nullptr;   // page-locked staging memory of this load, or null
     size_t off_holes = 0;
     i64 table_points = 0;            // rows of a table domain (0 for a box)
     u64 entries_at[kMaxSize + 1] = {0};      // subtree-table entries per size (all nonterminals)
     int size_cap = 0, probes_cap = 0;        // over the holes
+    u64 big_entries = 0;                     // most entries of a hole's first-probe table of the next size
 };
 
 // First half of a load: checks the description, lays out and allocates the sketch's device
@@ -500,7 +535,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     const size_t off_holes = off;   off += al(sizeof(HoleDev) * nh + sizeof(u32) * nh);       // holes, then one flag each
     const size_t off_bad = off_holes + sizeof(HoleDev) * nh;
     size_t off_coords = 0;
-    std::vector<size_t> off_spec(nh, 0), off_tabv(nh, 0), off_tabk(nh, 0), off_tabm(nh, 0);
+    std::vector<size_t> off_spec(nh, 0), off_tabv(nh, 0), off_tabk(nh, 0), off_tabm(nh, 0), off_bigv(nh, 0), off_bigk(nh, 0);
     if (copy_coords && coords_bytes <= kPackMax) { off_coords = off; off += al(coords_bytes); }
     for (int h = 0; h < nh; ++h)
         if (d->holes[h].spec_kind == XP_SPEC_TABLE && np > 0 && !d->holes[h].spec_table_on_device && spec_bytes <= kPackMax) {
@@ -529,6 +564,26 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
             off_tabv[h] = off; off += al(sizeof(i64) * entries * probes);
             off_tabk[h] = off; off += al(entries * probes);
             off_tabm[h] = off; off += al(entries);
+        }
+        // one size further at the first probe only (see HoleDev::big_size): the register-side operands of the largest candidates
+        int big = o.tab_size_cap + 1;                     // the next size that has trees at all
+        while (big <= hd.max_size - 2) {
+            bool any = false;
+            for (int nt = 0; nt < g->n_nt; ++nt) any = any || g->cnt[nt][big] > 0;
+            if (any) break;
+            ++big;
+        }
+        if (entries > 0 && o.tab_size_cap >= 1 && big <= hd.max_size - 2) {
+            u64 total = 0;
+            for (int nt = 0; nt < g->n_nt; ++nt) { o.big_off[nt] = total; total += g->cnt[nt][big]; }
+            size_t free_b = 0, total_b = 0;
+            const bool room = cudaMemGetInfo(&free_b, &total_b) == cudaSuccess && (u64)free_b > 3 * total * 9;
+            if (total > 0 && total <= kBigMaxEntries && total * 9 <= kBigBudgetBytes && room) {
+                o.big_size = big; o.big_total = total;
+                off_bigv[h] = off; off += al(sizeof(i64) * total);
+                off_bigk[h] = off; off += al(total);
+                if (total > L->big_entries) L->big_entries = total;
+            }
         }
     }
     size_t arena_granted = 0;
@@ -609,6 +664,10 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
             o.tab_ok = (unsigned char*)(base + off_tabk[h]);
             o.tab_vars = (unsigned char*)(base + off_tabm[h]);
         }
+        if (o.big_size > 0) {
+            o.big_val = (i64*)(base + off_bigv[h]);
+            o.big_ok = (unsigned char*)(base + off_bigk[h]);
+        }
         // variables the context and the spec mention (a caller's spec table may depend on all)
         u32 fv = hd.spec_kind == XP_SPEC_EXPR ? 0u : 0xffffffffu;
         for (int i = 0; i < hd.ctx_len; ++i) if (hd.ctx[i].kind == XP_I_VAR) fv |= 1u << hd.ctx[i].arg;
@@ -623,7 +682,10 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     }
 
     // the staged copy, then the tables too large for it
-    std::vector<char> stg(head, 0);
+    std::vector<char> stg_own;
+    char* stg = L->pinned ? L->pinned->take(head) : nullptr;
+    if (!stg) { stg_own.resize(head); stg = stg_own.data(); }
+    memset(stg, 0, head);
     memcpy(&stg[off_sketch], &hs, sizeof(hs));
     memcpy(&stg[off_holes], hh.data(), sizeof(HoleDev) * nh);
     if (copy_coords && coords_bytes <= kPackMax) memcpy(&stg[off_coords], d->coords, coords_bytes);
@@ -634,7 +696,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
         memset(&stg[s->off_kill[h]], 0xff, sizeof(i64) * kKillSlots);           // no point noted yet (ids -1, counts 0)
     }
     s->load_h2d = grammar_bytes + head;
-    XP_CUDA_S(cudaMemcpyAsync(base, stg.data(), head, cudaMemcpyHostToDevice, nullptr));
+    XP_CUDA_S(cudaMemcpyAsync(base, stg, head, cudaMemcpyHostToDevice, nullptr));
     if (copy_coords && coords_bytes > kPackMax) {
         XP_CUDA_S(cudaMemcpyAsync(base + off_coords, d->coords, coords_bytes, cudaMemcpyHostToDevice, nullptr));
         s->load_h2d += coords_bytes;
@@ -665,7 +727,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     }
     for (int k = 1; k <= kMaxSize; ++k)
         for (int nt = 0; nt < g->n_nt; ++nt) L->entries_at[k] += g->cnt[nt][k];
-    s->tab_size_cap = L->size_cap; s->tab_probes_cap = L->probes_cap;
+    s->tab_size_cap = L->size_cap; s->tab_probes_cap = L->probes_cap; s->big_entries = L->big_entries;
     memcpy(s->entries_at, L->entries_at, sizeof(s->entries_at));
 #undef XP_CUDA_S
     return XP_OK;
@@ -676,6 +738,11 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
     if (!grammars || !descs || !outs || n == 0) return fail(XP_ERR_INVALID_ARG, "xp_sketch_load_batch: null argument");
     for (size_t i = 0; i < n; ++i) outs[i] = nullptr;
     std::vector<LoadState> st(n);
+    std::unique_lock<std::mutex> pin(g_pinned.mu, std::try_to_lock);
+    if (pin.owns_lock()) {
+        g_pinned.reset();
+        for (size_t i = 0; i < n; ++i) st[i].pinned = &g_pinned;
+    }
     char* jobs_dev = nullptr;
     size_t jobs_bytes = 0;
     int jobs_device = 0;
@@ -731,12 +798,20 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
     for (int k = 1; k <= size_cap; ++k)
         for (size_t at = 0; at < n_jobs; at += kPiece)
             XP_CUDA_B(launch_subvalues(d_jobs + at, (int)(n_jobs - at < kPiece ? n_jobs - at : kPiece), k, probes_cap, most_entries[k], nullptr));
+    {
+        u64 big = 0;
+        for (size_t i = 0; i < n; ++i) big = st[i].big_entries > big ? st[i].big_entries : big;
+        for (size_t at = 0; at < n_jobs && big > 0; at += 32768)
+            XP_CUDA_B(launch_bigvalues(d_jobs + at, (int)(n_jobs - at < 32768 ? n_jobs - at : 32768), big, nullptr));
+    }
     // what the kernels decided, per hole
     for (size_t i = 0; i < n; ++i) {
         const int nh = st[i].s->n_holes;
-        st[i].back.resize(sizeof(HoleDev) * nh + sizeof(u32) * nh);
-        XP_CUDA_B(cudaMemcpyAsync(st[i].back.data(), st[i].s->arena + st[i].off_holes, st[i].back.size(), cudaMemcpyDeviceToHost, nullptr));
-        st[i].s->load_d2h = st[i].back.size();
+        st[i].back_bytes = sizeof(HoleDev) * nh + sizeof(u32) * nh;
+        st[i].back = st[i].pinned ? st[i].pinned->take(st[i].back_bytes) : nullptr;
+        if (!st[i].back) { st[i].back_own.resize(st[i].back_bytes); st[i].back = st[i].back_own.data(); }
+        XP_CUDA_B(cudaMemcpyAsync(st[i].back, st[i].s->arena + st[i].off_holes, st[i].back_bytes, cudaMemcpyDeviceToHost, nullptr));
+        st[i].s->load_d2h = st[i].back_bytes;
         st[i].s->load_h2d += sizeof(SketchDev*) + sizeof(LoadJob) * (size_t)nh;       // its lines of the batch's job lists
     }
     XP_CUDA_B(cudaStreamSynchronize(nullptr));
@@ -860,6 +935,7 @@ extern "C" xp_status xp_sketch_refine(xp_sketch* s, int32_t max_promote, int32_t
         if (e == cudaSuccess) e = launch_reprobe((const LoadJob*)jobs_dev, (int)jobs.size(), nullptr);
         for (int k = 1; k <= s->tab_size_cap && e == cudaSuccess; ++k)
             e = launch_subvalues((const LoadJob*)jobs_dev, (int)jobs.size(), k, s->tab_probes_cap, s->entries_at[k], nullptr);
+        if (e == cudaSuccess) e = launch_bigvalues((const LoadJob*)jobs_dev, (int)jobs.size(), s->big_entries, nullptr);
         if (e == cudaSuccess) e = cudaMemcpyAsync(hh.data(), s->arena + s->off_holes, sizeof(HoleDev) * nh, cudaMemcpyDeviceToHost, nullptr);
         const cudaError_t e2 = cudaStreamSynchronize(nullptr);
         pool_release(jobs_dev, jobs_bytes, jobs_device);

@@ -31,6 +31,8 @@ constexpr u64 kStageMaxPoints = 1ull << 26;  // largest box whose points and spe
 constexpr int kProgMax = 64;          // candidate substituted into its context: longest staged program
 constexpr u64 kTabBudgetBytes = 64ull << 20;   // subtree-value tables of one hole, all probes together
 constexpr u64 kTabMaxEntries = 1ull << 22;   // largest (nonterminal, size) subtree-value table per hole
+constexpr u64 kBigMaxEntries = 1ull << 30;   // ... of the one further size that is tabulated at the first probe only
+constexpr u64 kBigBudgetBytes = 12ull << 30; // ... and its bytes (9 per entry), per hole
 constexpr u32 kOpBit = 0x80000000u;  // candidate code word: operator (low bits = XP_OP_*) or leaf index
 constexpr int kMaxFamily = 8;         // tile segments that may share one fill of the register-side operands (a hit's
                                       // queue entry names its member in 3 bits)
@@ -97,6 +99,17 @@ struct HoleDev {
     i32 tab_size_cap, tab_probes_cap, small_search;
     i32 filter_ok;                                // the probe filter applies: probe 0 exists, its context is affine or compares
     i32 tab_max_size, tab_probes;
+    // One size further (big_size = the next size above tab_size_cap that has trees, when operands of that size occur and its trees fit
+    // kBigMaxEntries / kBigBudgetBytes) the values are tabulated at probe 0 ONLY: these are the register-side
+    // operands of the largest candidates (config 4: 5.9e8 subtrees of size 7, 5.3 GB), which every search
+    // would otherwise rebuild from the smaller tables tile by tile -- a third of such a search's time.
+    // The memory of a B200 has room for them; they stay resident with the sketch.  big_on is set by the
+    // load's kernels once the smaller tables exist at probe 0.
+    i32 big_size, big_on;
+    u64 big_off[kMaxNt];                          // first entry of each nonterminal
+    u64 big_total;
+    i64* big_val;                                 // device
+    unsigned char* big_ok;                        // device
     u64 tab_total;
     u64 tab_off[kMaxNt][kMaxSize + 1];
     i64* tab_val;                                 // device

@@ -150,6 +150,7 @@ __device__ __forceinline__ void probe_contexts(HoleDev* hole, int n, int ncand, 
             if (filter_ok && hole->tab_size_cap > 0 && hole->tab_total > 0) probes = n < hole->tab_probes_cap ? n : hole->tab_probes_cap;
             hole->tab_probes = probes;
             hole->tab_max_size = probes > 0 ? hole->tab_size_cap : 0;
+            hole->big_on = 0;                             // (the kernel that fills the big table turns it on)
             // Second look at probe 1 inside the filter: for small searches (its cost is in the operand
             // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
             // probe 0 alone lets many through.
@@ -929,6 +930,11 @@ __device__ __forceinline__ void push_hit(EvalShared& sh, u32 reg_idx, u32 slot, 
 __device__ __noinline__ bool operand_value(const GrammarDev* g, const HoleDev* hole, int pr, int nt, int size, u64 rank, i64& v) {
     const int tmax = hole->tab_max_size;
     const u64 pbase = (u64)pr * hole->tab_total;
+    if (pr == 0 && size == hole->big_size && hole->big_on) {
+        const u64 at = hole->big_off[nt] + rank;
+        v = hole->big_val[at];
+        return hole->big_ok[at] != 0;
+    }
     if (size <= tmax) {
         u64 at = pbase + hole->tab_off[nt][size] + rank;
         if (!XP_CHECKED(pr < hole->tab_probes && hole->tab_off[nt][size] + rank < hole->tab_total && rank < g->cnt[nt][size], kChkTable)) at = 0;
@@ -990,6 +996,11 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
         if (v > -(1ll << 31) && v < (1ll << 31)) fits |= 1u << j;
     };
     int j = 0;
+    if (pr == 0 && size == hole->big_size && hole->big_on) {      // tabulated at the first probe: consecutive entries
+        const u64 at = hole->big_off[nt] + rank;
+        for (; j < n; ++j) if (hole->big_ok[at + j]) put(j, hole->big_val[at + j]);
+        return alive;
+    }
     if (size > tmax && tmax >= 1 && size >= 3) {
         int op, lnt, rnt, a;
         u64 l, r;
@@ -1104,6 +1115,35 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const LoadJob* jobs, int 
         hole->tab_val[at] = v;
         hole->tab_ok[at] = ok ? 1 : 0;
         if (pr == 0) hole->tab_vars[hole->tab_off[nt][size] + idx] = (unsigned char)vars;
+        return;
+    }
+}
+
+// The big table: values at probe 0 of every subtree of size big_size (thread = (nonterminal,
+// rank)), from the smaller sizes' tables by one level of unranking.  The first thread turns the
+// table on for the searches once the launch is under way for a hole whose smaller tables exist
+// (the flag is read by later launches only).
+__global__ void __launch_bounds__(256) bigvalue_kernel(const LoadJob* jobs) {
+    const SketchDev* sk = jobs[blockIdx.y].s;
+    HoleDev* hole = &sk->holes[jobs[blockIdx.y].hole];
+    const int size = hole->big_size;
+    if (size <= 0 || hole->tab_probes < 1 || hole->tab_max_size != hole->tab_size_cap || hole->big_val == nullptr) return;
+    const GrammarDev* g = sk->g;
+    u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx == 0) hole->big_on = 1;
+    if (idx >= hole->big_total) return;
+    const u64 at = idx;
+    for (int nt = 0; nt < g->n_nt; ++nt) {
+        const u64 c = g->cnt[nt][size];
+        if (idx >= c) { idx -= c; continue; }
+        int op, lnt, rnt, a;
+        u64 l, r;
+        unrank_root(g, nt, size, idx, op, lnt, rnt, a, l, r);
+        const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;      // (probe 0: first copy of the tables)
+        i64 v = 0;
+        const bool ok = hole->tab_ok[la] && hole->tab_ok[ra] && apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
+        hole->big_val[at] = v;
+        hole->big_ok[at] = ok ? 1 : 0;
         return;
     }
 }
@@ -2388,6 +2428,12 @@ __global__ void __launch_bounds__(256) int_div_reciprocal_kernel(u32* out, int i
 cudaError_t launch_prepare(const LoadJob* jobs, int n_jobs, cudaStream_t stream) {
     if (n_jobs <= 0) return cudaSuccess;
     prepare_kernel<<<n_jobs, kPrepThreads, 0, stream>>>(jobs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bigvalues(const LoadJob* jobs, int n_jobs, u64 most_entries, cudaStream_t stream) {
+    if (most_entries == 0 || n_jobs <= 0) return cudaSuccess;
+    bigvalue_kernel<<<dim3((unsigned)((most_entries + 255) / 256), (unsigned)n_jobs), 256, 0, stream>>>(jobs);
     return cudaGetLastError();
 }
 

@@ -13,6 +13,7 @@ cudaError_t launch_coord_bounds(SketchDev* const* list, int n_sketches, i64 most
 cudaError_t launch_stage_points(const SketchDev* s, i64 n_points, i32* coords, cudaStream_t stream);
 cudaError_t launch_stage_spec(const SketchDev* s, int hole_index, i64 n_points, i64* spec, u32* bad, cudaStream_t stream);
 cudaError_t launch_subvalues(const LoadJob* jobs, int n_jobs, int size, int most_probes, u64 most_entries, cudaStream_t stream);
+cudaError_t launch_bigvalues(const LoadJob* jobs, int n_jobs, u64 most_entries, cudaStream_t stream);
 // Layout of one call's device scratch (byte offsets from its 256-byte aligned base):
 //   0: eval ticket (u64), 8: verify ticket (u64), 16: survivor pushes (u32), 20: failed-check word (u32; checked
 //      build only)   -- zero at launch
