@@ -135,7 +135,7 @@ def run_reference(args):
     if rank != 0:
         return
     name = args.workload or HEADLINE
-    scale = 1.0 / max(1, args.steps + args.warmup) * 3.0           # the whole run stays within about a minute
+    scale = min(1.0, 3.0 / max(1, args.steps + args.warmup))      # the whole run stays within a minute or two
     for _ in range(args.warmup):
         oracle_sample(name, scale / 8)
     evals, secs, sample = 0, 0.0, ""

@@ -12,6 +12,7 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "xp_dev.h"
@@ -134,8 +135,10 @@ struct PinnedArena {
     std::mutex mu;
     std::vector<char*> chunks;
     size_t chunk = 0, used = 0;
+    std::mutex take_mu;               // (the threads of one batch load share the arena)
     void reset() { chunk = 0; used = 0; }
     char* take(size_t bytes) {
+        std::lock_guard<std::mutex> lock(take_mu);
         const size_t need = (bytes + 255) & ~(size_t)255;
         if (need > kPinnedChunk) return nullptr;
         if (chunk < chunks.size() && used + need > kPinnedChunk) { ++chunk; used = 0; }
@@ -752,10 +755,35 @@ extern "C" xp_status xp_sketch_load_batch(const xp_grammar* const* grammars, con
         pool_release(jobs_dev, jobs_bytes, jobs_device);
     };
     size_t n_jobs = 0;
-    for (size_t i = 0; i < n; ++i) {
-        const xp_status r = load_begin(grammars[i], &descs[i], &st[i]);
-        if (r != XP_OK) { const std::string msg = g_last_error; undo(); return fail(r, "sketch " + std::to_string(i) + ": " + msg); }
-        n_jobs += (size_t)st[i].s->n_holes;
+    {
+        // The host part of a load (checks, layout, staging of the tables, queueing of the copies) is
+        // independent from sketch to sketch: large batches spread it over a few threads, each with
+        // the caller's device current.  Everything is queued on the same stream; the batch's kernels
+        // follow once the threads are done.
+        std::vector<xp_status> status(n, XP_OK);
+        std::vector<std::string> message(n);
+        int dev = 0;
+        cudaGetDevice(&dev);
+        unsigned hw = std::thread::hardware_concurrency();
+        size_t n_threads = n / 128;
+        if (n_threads > 8) n_threads = 8;
+        if (hw > 0 && n_threads > hw) n_threads = hw;
+        auto work = [&](size_t t, size_t step) {
+            if (step > 1) cudaSetDevice(dev);
+            for (size_t i = t; i < n; i += step) {
+                status[i] = load_begin(grammars[i], &descs[i], &st[i]);
+                if (status[i] != XP_OK) message[i] = g_last_error;
+            }
+        };
+        if (n_threads < 2) work(0, 1);
+        else {
+            std::vector<std::thread> pool;
+            for (size_t t = 0; t < n_threads; ++t) pool.emplace_back(work, t, n_threads);
+            for (std::thread& th : pool) th.join();
+        }
+        for (size_t i = 0; i < n; ++i)
+            if (status[i] != XP_OK) { undo(); return fail(status[i], "sketch " + std::to_string(i) + ": " + message[i]); }
+        for (size_t i = 0; i < n; ++i) n_jobs += (size_t)st[i].s->n_holes;
     }
 #define XP_CUDA_B(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { undo(); \
         return fail(e_ == cudaErrorMemoryAllocation ? XP_ERR_NOMEM : XP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } } while (0)

@@ -2239,7 +2239,7 @@ __global__ void __launch_bounds__(kVerifyThreads, 3) verify_kernel(const PlanDev
     while (width > 1 && n < warps * width) width >>= 1;
     const u64 n_blocks = (n + width - 1) / width;
     const u64 total = n_blocks * plan.max_chunks;
-    constexpr u64 kBatch = 2;                           // items a warp takes per atomic
+    const u64 kBatch = width >= 16 ? 2 : 16;            // items a warp takes per atomic (narrow items are light and many)
     u64 next = 0, batch_end = 0;
     for (;;) {
         if (next == batch_end) {
