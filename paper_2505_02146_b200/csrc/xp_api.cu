@@ -1247,7 +1247,8 @@ static SearchLayout ws_layout(size_t n_segs, size_t n_sketches, size_t n_acc, u3
     w.surv = w.head;
     w.sort_off = w.surv + align256(sizeof(SurvDev) * (size_t)surv_cap);
     w.sorted = w.sort_off + align256(sizeof(u32) * (n_acc + 2));
-    w.total = w.sorted + align256(sizeof(u32) * (size_t)surv_cap);
+    w.longs = w.sorted + align256(sizeof(u32) * (size_t)surv_cap);
+    w.total = w.longs + align256(sizeof(u32) * (size_t)surv_cap);
     w.n_acc = (int)n_acc;
     w.dense = 0;
     w.surv_cap = surv_cap;

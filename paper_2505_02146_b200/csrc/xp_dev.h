@@ -220,6 +220,10 @@ struct PlanDev {
     u32* surv_hist;                  // device, n_acc, zero at launch
     u32* surv_off;                   // device, n_acc + 1
     u32* surv_sorted;                // device, surv_cap
+    // Survivors whose check spans more than one chunk of points (queue indices, in no particular order),
+    // listed after the search so that the later chunks are walked for them alone.
+    u32* surv_long;                  // device, surv_cap
+    u32* surv_long_n;                // device counter, zero at launch
 };
 
 }  // namespace xp

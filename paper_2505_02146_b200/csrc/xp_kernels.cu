@@ -1967,6 +1967,18 @@ __global__ void __launch_bounds__(256) surv_scatter_kernel(const PlanDev plan) {
     plan.surv_sorted[plan.surv_off[acc] + atomicAdd(&plan.surv_hist[acc], 1u)] = i;
 }
 
+// One thread per queued survivor: those whose (projected) domain has more than one chunk of points
+// go on the list of long survivors.
+__global__ void __launch_bounds__(256) surv_long_kernel(const PlanDev plan) {
+    const u32 pushed = *plan.surv_n;
+    const u32 n = pushed < plan.surv_cap ? pushed : plan.surv_cap;
+    const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const SurvDev sv = plan.surv[i];
+    const SketchDev* sk = plan.sketches[sv.sketch];
+    if (proj_points(sk, &sk->holes[sv.hole], sv.vars, nullptr) > (i64)kVerifyChunk) plan.surv_long[atomicAdd(plan.surv_long_n, 1u)] = i;
+}
+
 // ---- whole-domain check of several survivors of one hole together ----
 //
 // For table domains.  The warp's lanes each stage one survivor (unranking, substitution into the
@@ -2216,9 +2228,11 @@ __device__ __noinline__ void verify_one(const PlanDev& plan, VerifyWarp& w, u32 
     __syncwarp();                                       // the staged candidate is free for the next item
 }
 
-// Items are (chunk of points, block of up to 32 survivors in hole order), chunk-major: the first chunk
-// of every survivor is taken before any second chunk, so candidates that fail early cost one
-// chunk.  Each WARP takes items on its own: nothing in this kernel synchronises a CTA, and no
+// Items are (chunk of points, block of up to 32 survivors), chunk-major: the first chunk of every
+// survivor (blocks in hole order) is taken before any second chunk, so candidates that fail early
+// cost one chunk; the later chunks exist for the long survivors only (surv_long_kernel), which keeps
+// a call whose largest domain has hundreds of chunks from walking hundreds of empty items for every
+// survivor of a small (or projected) domain.  Each WARP takes items on its own: nothing in this kernel synchronises a CTA, and no
 // warp waits for another.  Within a block the survivors of one hole are handled together when the
 // hole's domain is a table (verify_batch), one after the other otherwise (verify_one).  A survivor
 // that has already failed is skipped.
@@ -2238,8 +2252,11 @@ __global__ void __launch_bounds__(kVerifyThreads, 3) verify_kernel(const PlanDev
     u32 width = 32;
     while (width > 1 && n < warps * width) width >>= 1;
     const u64 n_blocks = (n + width - 1) / width;
-    const u64 total = n_blocks * plan.max_chunks;
-    const u64 kBatch = width >= 16 ? 2 : 16;            // items a warp takes per atomic (narrow items are light and many)
+    // The first chunk is walked for every survivor, the later ones for the long survivors only.
+    const u64 n_long = plan.max_chunks > 1 ? *plan.surv_long_n : 0u;
+    const u64 long_blocks = (n_long + width - 1) / width;
+    const u64 total = n_blocks + long_blocks * (plan.max_chunks - 1);
+    const u64 kBatch = 2;                               // items a warp takes per atomic
     u64 next = 0, batch_end = 0;
     for (;;) {
         if (next == batch_end) {
@@ -2249,10 +2266,12 @@ __global__ void __launch_bounds__(kVerifyThreads, 3) verify_kernel(const PlanDev
         }
         const u64 t = next++;
         if (t >= total) break;
-        const u64 chunk = t / n_blocks, block = t % n_blocks;
+        const bool later = t >= n_blocks;
+        const u64 chunk = later ? 1 + (t - n_blocks) / long_blocks : 0;
+        const u64 block = later ? (t - n_blocks) % long_blocks : t;
         const u64 pos = block * width + lane;
-        const bool have = (u32)lane < width && pos < n;
-        const u32 si = have ? (plan.surv_sorted ? plan.surv_sorted[pos] : (u32)pos) : 0u;
+        const bool have = (u32)lane < width && pos < (later ? n_long : n);
+        const u32 si = !have ? 0u : later ? plan.surv_long[pos] : plan.surv_sorted ? plan.surv_sorted[pos] : (u32)pos;
         const int my_acc = have ? plan.surv[si].acc : -1;
         u32 remaining = __ballot_sync(0xffffffffu, have);
         while (remaining) {
@@ -2495,6 +2514,8 @@ static PlanDev plan_on(char* base, const SearchLayout& L, int n_segs, int n_sket
     pd.surv_hist = order ? (u32*)(base + L.hist) : nullptr;
     pd.surv_off = order ? (u32*)(base + L.sort_off) : nullptr;
     pd.surv_sorted = order ? (u32*)(base + L.sorted) : nullptr;
+    pd.surv_long = (u32*)(base + L.longs);
+    pd.surv_long_n = (u32*)(base + 24);
     return pd;
 }
 
@@ -2531,6 +2552,11 @@ cudaError_t launch_search_end(char* base, const SearchLayout& L, bool any_ticket
             surv_scatter_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
             if ((e = cudaGetLastError()) != cudaSuccess) return e;
             *n_launches += 2;
+        }
+        if (max_chunks > 1) {
+            surv_long_kernel<<<(L.surv_cap + 255) / 256, 256, 0, stream>>>(pd);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            *n_launches += 1;
         }
         const size_t vsmem = sizeof(VerifyWarp) * kVerifyWarps;
         if ((e = cudaFuncSetAttribute((const void*)verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vsmem)) != cudaSuccess) return e;

@@ -20,7 +20,7 @@ cudaError_t launch_bigvalues(const LoadJob* jobs, int n_jobs, u64 most_entries, 
 //   segs, sketches, acc: staged from the host;  [0, head) is what the host copies in
 //   hist: survivors per accumulator slot, zero at launch (staged);
 //   surv: the survivor queue (surv_cap entries); sort_off, sorted: its hole order -- written by the kernels only
-struct SearchLayout { size_t segs, sketches, acc, hist, head, surv, sort_off, sorted, total; u32 surv_cap; int n_acc;
+struct SearchLayout { size_t segs, sketches, acc, hist, head, surv, sort_off, sorted, longs, total; u32 surv_cap; int n_acc;
                       int dense; /* some hole of the plan takes the second look: launch the search kernel's dense form */ };
 
 // The whole search on a staged scratch: eval_kernel, verify_kernel, count_kernel, finish_kernel;
