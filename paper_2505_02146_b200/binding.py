@@ -219,9 +219,16 @@ class Grammar:
             self.handle = None
 
 
-def xp_grammar_create(g) -> Grammar:
-    """``g``: an ``xp_instances.Grammar`` (variables with ranges, productions in canonical order)."""
-    lib = load()
+class GrammarDesc:
+    """A grammar's C descriptor in host memory (``marshal_grammar``), with what it points to kept alive."""
+
+    def __init__(self, desc, model, keep):
+        self.desc, self.model, self._keep = desc, model, keep
+
+
+def marshal_grammar(g) -> GrammarDesc:
+    """Encodes an ``xp_instances.Grammar`` as the C descriptor ``xp_grammar_create`` takes; a caller that
+    creates the same grammar again and again does this once."""
     nv = len(g.variables)
     names = [v.name.encode() for v in g.variables]
     vs = (xp_variable * max(1, nv))()
@@ -231,10 +238,17 @@ def xp_grammar_create(g) -> Grammar:
     for i, p in enumerate(g.productions):
         q = ps[i]
         q.lhs, q.kind, q.var, q.op, q.left, q.right, q.value = p.lhs, p.kind, p.var, p.op, p.left, p.right, p.value
-    desc = xp_grammar_desc(nv, vs, g.n_nonterminals, len(g.productions), ps)
+    return GrammarDesc(xp_grammar_desc(nv, vs, g.n_nonterminals, len(g.productions), ps), g, (names, vs, ps))
+
+
+def xp_grammar_create(g) -> Grammar:
+    """``g``: an ``xp_instances.Grammar`` (variables with ranges, productions in canonical order), or the
+    descriptor ``marshal_grammar`` made of one."""
+    lib = load()
+    d = g if isinstance(g, GrammarDesc) else marshal_grammar(g)
     out = C.c_void_p()
-    _check(lib.xp_grammar_create(C.byref(desc), C.byref(out)))
-    return Grammar(out.value, g)
+    _check(lib.xp_grammar_create(C.byref(d.desc), C.byref(out)))
+    return Grammar(out.value, d.model)
 
 
 def xp_grammar_count(gr: Grammar, nt: int, max_size: int) -> List[int]:
