@@ -578,7 +578,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
         }
         if (entries > 0 && o.tab_size_cap >= 1 && big <= hd.max_size - 2) {
             u64 total = 0;
-            for (int nt = 0; nt < g->n_nt; ++nt) { o.big_off[nt] = total; total += g->cnt[nt][big]; }
+            for (int nt = 0; nt < g->n_nt; ++nt) { o.big_off[nt] = total; total += (g->cnt[nt][big] + 7) & ~7ull; }     // (ranges start at multiples of 8: bigvalue_kernel)
             size_t free_b = 0, total_b = 0;
             const bool room = cudaMemGetInfo(&free_b, &total_b) == cudaSuccess && (u64)free_b > 3 * total * 9;
             if (total > 0 && total <= kBigMaxEntries && total * 9 <= kBigBudgetBytes && room) {

@@ -317,6 +317,8 @@ constexpr u64 kAdaptRate = 4096;                          // filter hits per eva
 constexpr int kWarps = kThreads / 32;
 constexpr int kQueueCap = 3072;                           // filter hits waiting for the exact probe check (all warps)
 constexpr int kWarpQueue = kQueueCap / kWarps;            // ... per warp: every warp keeps and empties its own queue
+ constexpr int kQueueTags = 8;                             // tiles whose hits may wait in a warp's queue at a time
+constexpr u32 kDrainMin = 32;                             // hits a warp lets gather before it checks them (resident families)
 constexpr int kChunkB = 512;                              // broadcast operands between block-wide queue checks
 static_assert(kRegTile <= 2048 && kBcTile <= 1024, "queue entries pack the tile indices in 11 + 10 bits");
 static_assert(32 * 5 <= kWarpQueue / 2, "one replay step of a warp must fit the free half of its queue");
@@ -356,6 +358,8 @@ struct CandShared {
 
 struct MemberState {
     u64 bc_first; i32 lo, hi; u32 n, nspecial; i32 wide;
+    u32 mask, opip;              // the member's operators: bit per operator slot, and (3 bits per slot) each one's index
+                                 // in the segment's list
     i32 mod_possible;            // some operand of the member, as a divisor, exceeds the target's magnitude: only
                                  // then can a remainder equal the target (|n % d| < |d|)
 };
@@ -384,18 +388,32 @@ struct EvalShared {
     MemberState mb[kMaxFamily];
     i32 kept_head;
     i32 reg_wide;                // some register-side operand of the ticket does not fit int32
-    u32 wmember[kWarps];         // member the warp is working on (tags its queue entries)
+    u32 wmember[kWarps];         // member the warp is working on, and (<< 3) the tag of its tile: both go into its queue entries
     u32 wq_n[kWarps], wq_over[kWarps];
     // second look (HoleDev::second): context factor, offset and spec value at probe 1 of the hole at hand
     i32 adapt_second;            // this CTA has seen more than one filter hit per kAdaptRate evaluations for the
                                  // hole it works on: it takes the second look from now on (until it changes hole)
+    // what the loops need of the hole at the first probe (read from the hole once per ticket)
+    u64 h_A, h_tq;               // context factor; spec value minus the context's offset
+    i64 h_rng_lo, h_rng_hi;      // interval of values that satisfy a comparing context
+    i32 h_aff_ok;
     i32 p1_on, p1_rng;           // p1_rng: the context compares at probe 1; the value must lie in [p1_lo, p1_hi]
     u64 p1_A, p1_B, p1_spec;
     i64 p1_lo, p1_hi;
     BcRing bc_ring[kBcTile];
     BcDiv bc_div[kBcTile];
     BcMeta bc_meta[kBcTile];
-    u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21 | member << 24
+    u32 queue[kWarps][kWarpQueue];   // reg index | broadcast slot << 11 | op index << 21 | member << 24 | tile tag << 27
+    // Hits may wait in a warp's queue over several tickets of one resident family, until there are
+    // enough of them to give every lane of the exact check one (a tile of a sparse search leaves a
+    // handful per warp).  An entry names its tile by a tag: wq_first holds the first register-side rank
+    // of the warp's last kQueueTags tiles, wq_tiles counts the warp's tiles, wq_age the tiles since the
+    // queue was last emptied (it is emptied before a tag comes round again).  q_sketch and q_hole name
+    // the hole the waiting hits belong to.
+    u64 wq_first[kWarps][kQueueTags];
+    u32 wq_tiles[kWarps], wq_age[kWarps];
+    i32 q_sketch, q_hole;
+    i32 q_waiting;               // some warp has let hits wait
 };
 
 // Moves the CTA's private results of one (sketch, hole) into the global accumulators.
@@ -818,14 +836,14 @@ __device__ __noinline__ bool check_points(const CandShared& c, const SketchDev* 
 
 // A candidate that passed the probes goes into the global queue for the verification kernel.
 // Returns false if the queue is full: the caller's warp then checks the candidate itself.
-__device__ __forceinline__ bool push_survivor(EvalShared& sh, const PlanDev& plan, u64 rank, u32 vars) {
+__device__ __forceinline__ bool push_survivor(const PlanDev& plan, const SegDev& seg, u64 rank, u32 vars) {
     // (the counter saturates: once the queue is full nothing is added, so it cannot wrap around
     // and hand out a slot twice however many survivors a search has)
     if (*(volatile const u32*)plan.surv_n >= plan.surv_cap) return false;
     const u32 at = atomicAdd(plan.surv_n, 1u);
     if (at >= plan.surv_cap) return false;
     SurvDev r;
-    r.rank = rank; r.sketch = sh.seg.sketch; r.hole = sh.seg.hole; r.size = sh.seg.size; r.acc = sh.seg.acc;
+    r.rank = rank; r.sketch = seg.sketch; r.hole = seg.hole; r.size = seg.size; r.acc = seg.acc;
     r.state = 0; r.vars = vars;
     plan.surv[at] = r;
     if (plan.surv_hist) atomicAdd(&plan.surv_hist[r.acc], 1u);       // (for the hole order the verification walks)
@@ -885,7 +903,7 @@ __device__ __noinline__ void linear_ticket(EvalShared& sh, const PlanDev& plan, 
                 u32 vars = 0;
                 for (int k = 0; k < n; ++k)
                     if (!(code[k] & kOpBit)) { const i32 var = g->leaves[code[k]].var; if (var >= 0) vars |= 1u << var; }
-                pending = !push_survivor(sh, plan, rank, vars);
+                pending = !push_survivor(plan, seg, rank, vars);
             }
         }
         warp_verify_pending(sh, sk, hole, seg.size, pending, rank, my_evals);
@@ -998,6 +1016,20 @@ __device__ __noinline__ u32 fill_reg_operands(const GrammarDev* g, const HoleDev
     int j = 0;
     if (pr == 0 && size == hole->big_size && hole->big_on) {      // tabulated at the first probe: consecutive entries
         const u64 at = hole->big_off[nt] + rank;
+        if (n == kNA && (at & 7ull) == 0) {
+            // the usual case: eight aligned entries, fetched with five independent loads
+            const u64 oks = *reinterpret_cast<const u64*>(hole->big_ok + at);
+            const longlong2* src = reinterpret_cast<const longlong2*>(hole->big_val + at);
+            longlong2 v[kNA / 2];
+#pragma unroll
+            for (int k = 0; k < kNA / 2; ++k) v[k] = src[k];
+#pragma unroll
+            for (int k = 0; k < kNA / 2; ++k) {
+                if ((oks >> (16 * k)) & 0xffull) put(2 * k, v[k].x);
+                if ((oks >> (16 * k + 8)) & 0xffull) put(2 * k + 1, v[k].y);
+            }
+            return alive;
+        }
         for (; j < n; ++j) if (hole->big_ok[at + j]) put(j, hole->big_val[at + j]);
         return alive;
     }
@@ -1119,32 +1151,51 @@ __global__ void __launch_bounds__(256) subvalue_kernel(const LoadJob* jobs, int 
     }
 }
 
-// The big table: values at probe 0 of every subtree of size big_size (thread = (nonterminal,
-// rank)), from the smaller sizes' tables by one level of unranking.  The first thread turns the
-// table on for the searches once the launch is under way for a hole whose smaller tables exist
-// (the flag is read by later launches only).
+// The big table: values at probe 0 of every subtree of size big_size, from the smaller sizes'
+// tables by one level of unranking.  A thread writes 8 consecutive entries of one nonterminal (the
+// nonterminals' ranges start at multiples of 8): the first is unranked, the others follow by
+// advancing the operand ranks like an odometer (right operand fastest).  The first thread turns
+// the table on for the searches once the launch is under way for a hole whose smaller tables
+// exist (the flag is read by later launches only).
+constexpr int kBigPerThread = 8;
 __global__ void __launch_bounds__(256) bigvalue_kernel(const LoadJob* jobs) {
     const SketchDev* sk = jobs[blockIdx.y].s;
     HoleDev* hole = &sk->holes[jobs[blockIdx.y].hole];
     const int size = hole->big_size;
     if (size <= 0 || hole->tab_probes < 1 || hole->tab_max_size != hole->tab_size_cap || hole->big_val == nullptr) return;
     const GrammarDev* g = sk->g;
-    u64 idx = (u64)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx == 0) hole->big_on = 1;
-    if (idx >= hole->big_total) return;
-    const u64 at = idx;
-    for (int nt = 0; nt < g->n_nt; ++nt) {
-        const u64 c = g->cnt[nt][size];
-        if (idx >= c) { idx -= c; continue; }
+    const u64 t = (u64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t == 0) hole->big_on = 1;
+    const u64 at0 = t * (u64)kBigPerThread;
+    if (at0 >= hole->big_total) return;
+    int nt = g->n_nt - 1;                               // the last nonterminal whose range starts at or before at0
+    while (nt > 0 && hole->big_off[nt] > at0) --nt;
+    const u64 c = g->cnt[nt][size], idx = at0 - hole->big_off[nt];
+    if (idx >= c) return;                               // (padding between two nonterminals' ranges)
+    const int n = c - idx < (u64)kBigPerThread ? (int)(c - idx) : kBigPerThread;
+    // (local copies: the stores below cannot change them, which the compiler cannot know of fields of *hole)
+    const i64* __restrict__ tab_val = hole->tab_val;
+    const unsigned char* __restrict__ tab_ok = hole->tab_ok;
+    i64* __restrict__ out_val = hole->big_val + at0;
+    unsigned char* __restrict__ out_ok = hole->big_ok + at0;
+    int j = 0;
+    while (j < n) {
         int op, lnt, rnt, a;
         u64 l, r;
-        unrank_root(g, nt, size, idx, op, lnt, rnt, a, l, r);
-        const u64 la = hole->tab_off[lnt][a] + l, ra = hole->tab_off[rnt][size - 1 - a] + r;      // (probe 0: first copy of the tables)
-        i64 v = 0;
-        const bool ok = hole->tab_ok[la] && hole->tab_ok[ra] && apply_op(op, hole->tab_val[la], hole->tab_val[ra], v);
-        hole->big_val[at] = v;
-        hole->big_ok[at] = ok ? 1 : 0;
-        return;
+        unrank_root(g, nt, size, idx + j, op, lnt, rnt, a, l, r);
+        const u64 cl = g->cnt[lnt][a], cr = g->cnt[rnt][size - 1 - a];
+        const u64 lbase = hole->tab_off[lnt][a], rbase = hole->tab_off[rnt][size - 1 - a];      // (probe 0: first copy of the tables)
+        while (j < n && l < cl) {                       // until this (production, left size) block ends
+            const bool lok = tab_ok[lbase + l] != 0;
+            const i64 lv = tab_val[lbase + l];
+            for (; j < n && r < cr; ++r, ++j) {
+                i64 v = 0;
+                const bool ok = lok && tab_ok[rbase + r] && apply_op(op, lv, tab_val[rbase + r], v);
+                out_val[j] = v;
+                out_ok[j] = ok ? 1 : 0;
+            }
+            if (r == cr) { r = 0; ++l; }
+        }
     }
 }
 
@@ -1518,7 +1569,7 @@ __device__ __noinline__ void wide_chunk(EvalShared& sh, const RegVals* R, u32 al
 // for the remaining probes the candidate is rebuilt by full unranking.  Survivors go to the
 // global queue, or are checked by the warp itself when that is full.  Called by all 32 lanes.
 __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole,
-                                         u64 reg_first, u64& my_evals) {
+                                         u64& my_evals) {
     const GrammarDev* g = sk->g;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncwarp();
@@ -1530,12 +1581,14 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
     while (n_tab < hole->tab_probes && n_tab < hole->n_probe &&
            ((hole->probe_spec_ok & (hole->aff_okmask | hole->rng_okmask)) >> n_tab & 1u)) ++n_tab;
     u32 passes = 0;
+    const int cand_size = sh.mseg[0].size;              // (the members of a family build candidates of one size)
     for (u32 base = 0; base < nq; base += 32) {
         const u32 i = base + lane;
         bool pending = false;
         u64 rank = 0;
         if (i < nq) {
             const u32 e = sh.queue[warp][i];
+            const u64 reg_first = sh.wq_first[warp][(e >> 27) & (u32)(kQueueTags - 1)];
             const SegDev& seg = sh.mseg[(e >> 24) & 7u];
             const u32 opi = (e >> 21) & 7u;
             const u64 rr = reg_first + (e & 2047u);
@@ -1566,37 +1619,93 @@ __device__ __noinline__ void drain_queue(EvalShared& sh, const PlanDev& plan, co
                 ++passes;
                 const u32 vars = sk->project ? operand_vars(g, hole, seg.reg_nt, seg.reg_size, rr) |
                                                operand_vars(g, hole, seg.bc_nt, seg.bc_size, br) : 0xffu;
-                pending = !push_survivor(sh, plan, rank, vars);
+                pending = !push_survivor(plan, seg, rank, vars);      // (the hit's own segment: the ticket at hand may be another's)
             }
         }
-        warp_verify_pending(sh, sk, hole, sh.seg.size, pending, rank, my_evals);
+        warp_verify_pending(sh, sk, hole, cand_size, pending, rank, my_evals);
     }
     warp_tally(&sh.probe_survivors, passes);
-    if (lane == 0) { atomicAdd(&sh.filter_survivors, (u64)nq); sh.wq_n[warp] = 0; }
+    if (lane == 0) { atomicAdd(&sh.filter_survivors, (u64)nq); sh.wq_n[warp] = 0; sh.wq_age[warp] = 0; }
     __syncwarp();
 }
 
-template <bool SWAP, bool DENSE>
-__device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
-                                          u64 reg_first, u64 pairs, const RegVals* R, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
-    const SegDev& seg = sh.mseg[m];
-    const MemberState& mbs = sh.mb[m];
-    const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
-    const bool tile_wide = (sh.reg_wide | mbs.wide | seg.generic) != 0;
-    const u64 A64 = hole->aff_A, tq = (u64)hole->probe_spec[0] - hole->aff_B;
-    // a context that compares: interval test on int32-exact operands (results stay below 2^62 in
-    // magnitude, where the interval is exact); wider operands are all passed on to the exact stages
-    const int rng = hole->aff_ok ? 0 : (tile_wide ? 2 : 1);
-    const i64 rng_lo = hole->rng_lo[0], rng_hi = hole->rng_hi[0];
-    u32 opip = 0, mask = 0;
-    for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * op_slot(seg.op[o])); mask |= 1u << op_slot(seg.op[o]); }
+// The exact check of the hits that wait in the warp's queue, for the hole they belong to.
+__device__ __forceinline__ void drain_waiting(EvalShared& sh, const PlanDev& plan, u64& my_evals) {
+    const SketchDev* qs = plan.sketches[sh.q_sketch];
+    drain_queue(sh, plan, qs, &qs->holes[sh.q_hole], my_evals);
+}
 
+// What a piece of a tile needs beyond the member's and the hole's constants in shared memory.
+constexpr u32 kPieceSpecial = 1u, kPieceWide = 2u, kPieceSkipMod = 4u;
+
+// One piece of a tile: broadcast slots [s0, s1) of member m against the register operands in `alv`.
+// Picks the loops for the member's operators; one copy of this dispatch serves every member and
+// both call sites of a tile.
+template <bool SWAP, bool DENSE>
+__device__ __forceinline__ void run_piece_as(EvalShared& sh, const RegVals* R, u32 alv, u32 a1ok, int m, int s0, int s1, u32 flags) {
+    const SegDev& seg = sh.mseg[m];
+    const u32 mask = sh.mb[m].mask, opip = sh.mb[m].opip;
+    const u64 A64 = sh.h_A, tq = sh.h_tq;
+    const bool tile_wide = (flags & kPieceWide) != 0;
+    const int rng = sh.h_aff_ok ? 0 : (tile_wide ? 2 : 1);
+    if (tile_wide || rng) {
+        wide_chunk(sh, R, alv, a1ok, SWAP, A64, tq, rng, sh.h_rng_lo, sh.h_rng_hi, s0, s1, seg.n_ops, seg.op);
+        return;
+    }
     const u32 A = (u32)A64, tp = (u32)tq;
+    switch (mask & 7u) {
+#define XP_RING(M) case M: ring_pass<M, SWAP, DENSE>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
+        XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
+#undef XP_RING
+        default: break;
+    }
+    if (mask >> kSlotMin) switch ((mask >> kSlotMin) & 3u) {
+#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, R, alv, a1ok, A, tp, s0, s1, opip); \
+                         else minmax_pass<M, false>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
+        XP_MM(1u) XP_MM(2u) XP_MM(3u)
+#undef XP_MM
+        default: break;
+    }
+    if (!(mask & 24u)) return;
+    if (A != 1u) { div_pass_signed<SWAP>(sh, R, alv, a1ok, mask, A, tp, s0, s1, opip); return; }
     // With A == 1 a quotient or remainder of int32 operands can only equal a target of
     // magnitude below 2^31; its magnitude is what the unsigned loops compare with.
     const i64 T = (i64)tq;
-    const bool t_small = T > -(1ll << 31) && T < (1ll << 31);
+    if (!(T > -(1ll << 31) && T < (1ll << 31))) return;    // no int32 quotient or remainder can be the target
     const u32 tabs = (u32)(T < 0 ? -T : T);
+    const bool special = (flags & kPieceSpecial) != 0;
+    switch ((flags & kPieceSkipMod) ? (mask >> 3) & 1u : (mask >> 3) & 3u) {
+#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, R, alv, a1ok, tabs, s0, s1, opip, M); \
+                          else div_pass<M, SWAP, false, DENSE>(sh, R, alv, a1ok, tabs, s0, s1, opip); break;
+        XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
+#undef XP_DIV
+        default: break;
+    }
+}
+
+template <bool DENSE>
+__device__ __noinline__ void run_piece(EvalShared& sh, const RegVals* R, u32 alv, u32 a1ok, int m, int s0, int s1, u32 flags) {
+    if (sh.mseg[m].swap) run_piece_as<true, DENSE>(sh, R, alv, a1ok, m, s0, s1, flags);
+    else run_piece_as<false, DENSE>(sh, R, alv, a1ok, m, s0, s1, flags);
+}
+
+// Member m of the family on the ticket's register operands.
+template <bool DENSE>
+__device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, const SketchDev* sk, const HoleDev* hole, int m,
+                                       u64 reg_first, u64 pairs, const RegVals* R, u32 a1ok, u32 alive, bool drain_at_end, u64& my_evals) {
+    const SegDev& seg = sh.mseg[m];
+    const MemberState& mbs = sh.mb[m];
+    const bool SWAP = seg.swap != 0;
+    const int nb = (int)mbs.n, bc_lo = mbs.lo, bc_hi = mbs.hi;
+    const bool tile_wide = (sh.reg_wide | mbs.wide | seg.generic) != 0;
+    const u64 tq = sh.h_tq;
+    // a context that compares: interval test on int32-exact operands (results stay below 2^62 in
+    // magnitude, where the interval is exact); wider operands are all passed on to the exact stages
+    const int rng = sh.h_aff_ok ? 0 : (tile_wide ? 2 : 1);
+    const u32 mask = mbs.mask;
+    const u32 A = (u32)sh.h_A;
+    const i64 T = (i64)tq;
+    const bool t_small = T > -(1ll << 31) && T < (1ll << 31);
     // A remainder is smaller in magnitude than its divisor: when no divisor of the tile exceeds the
     // target's magnitude no candidate  a % b  can match, and the loops leave the remainders out.
     const bool skip_mod = !SWAP && (mask & 16u) && !mbs.mod_possible && !tile_wide && !rng && A == 1u && t_small;
@@ -1613,40 +1722,7 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         }
         warp_tally(&sh.filter_tests, (u32)__popc(alive) * (u32)(nb + (int)mbs.nspecial) * (u32)tested_ops);
     }
-
-    // One piece of the tile: broadcast slots [s0, s1) against the register operands in `alv`.
-    constexpr bool dense = DENSE;
-    auto run = [&](int s0, int s1, u32 alv, bool special) {
-        if (tile_wide || rng) {
-            wide_chunk(sh, R, alv, a1ok, SWAP, A64, tq, rng, rng_lo, rng_hi, s0, s1, seg.n_ops, seg.op);
-            return;
-        }
-        switch (mask & 7u) {
-#define XP_RING(M) case M: if (dense) ring_pass<M, SWAP, true>(sh, R, alv, a1ok, A, tp, s0, s1, opip); \
-                           else ring_pass<M, SWAP, false>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
-            XP_RING(1u) XP_RING(2u) XP_RING(3u) XP_RING(4u) XP_RING(5u) XP_RING(6u) XP_RING(7u)
-#undef XP_RING
-            default: break;
-        }
-        if (mask >> kSlotMin) switch ((mask >> kSlotMin) & 3u) {
-#define XP_MM(M) case M: if (A != 1u) minmax_pass<M, true>(sh, R, alv, a1ok, A, tp, s0, s1, opip); \
-                         else minmax_pass<M, false>(sh, R, alv, a1ok, A, tp, s0, s1, opip); break;
-            XP_MM(1u) XP_MM(2u) XP_MM(3u)
-#undef XP_MM
-            default: break;
-        }
-        if (!(mask & 24u)) return;
-        if (A != 1u) { div_pass_signed<SWAP>(sh, R, alv, a1ok, mask, A, tp, s0, s1, opip); return; }
-        if (!t_small) return;                            // no int32 quotient or remainder can be the target
-        switch (skip_mod ? (mask >> 3) & 1u : (mask >> 3) & 3u) {
-#define XP_DIV(M) case M: if (special && !SWAP) div_special(sh, R, alv, a1ok, tabs, s0, s1, opip, M); \
-                          else if (dense) div_pass<M, SWAP, false, true>(sh, R, alv, a1ok, tabs, s0, s1, opip); \
-                          else div_pass<M, SWAP, false, false>(sh, R, alv, a1ok, tabs, s0, s1, opip); break;
-            XP_DIV(1u) XP_DIV(2u) XP_DIV(3u)
-#undef XP_DIV
-            default: break;
-        }
-    };
+    const u32 flags = (tile_wide ? kPieceWide : 0u) | (skip_mod ? kPieceSkipMod : 0u);
 
     // The broadcast operands sit in two runs of slots: the general ones from slot 0 up, the
     // ones of magnitude <= 1 (special as divisors) from the last slot down.  Every warp walks
@@ -1660,32 +1736,33 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     const int n_special = (int)mbs.nspecial;
     int chunk = sh.chunk_hint[warp];
     bool shrunk = false;
-    if ((threadIdx.x & 31) == 0) sh.wmember[warp] = (u32)m;
+    if ((threadIdx.x & 31) == 0) sh.wmember[warp] = (u32)m | (((sh.wq_tiles[warp] - 1u) & (u32)(kQueueTags - 1)) << 3);
     __syncwarp();
     u32 q_start = sh.wq_n[warp];                        // queue length when the current chunk began (hits of
                                                         // earlier members of the family may still wait there)
     for (int part = 0; part < 2; ++part) {
         const int lo = part == 0 ? bc_lo : bc_hi - n_special, hi = part == 0 ? bc_lo + nb : bc_hi;
+        const u32 pflags = flags | (part == 1 ? kPieceSpecial : 0u);
         int s0 = lo;
         while (s0 < hi) {
             const int s1 = s0 + chunk < hi ? s0 + chunk : hi;
-            run(s0, s1, alive, part == 1);
+            run_piece<DENSE>(sh, R, alive, a1ok, m, s0, s1, pflags);
             __syncwarp();
             const u32 qn = sh.wq_n[warp];
             const bool overflow = sh.wq_over[warp] != 0;
             __syncwarp();
             if (overflow) {
                 if ((threadIdx.x & 31) == 0) { sh.wq_n[warp] = q_start; sh.wq_over[warp] = 0; }
-                drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+                drain_queue(sh, plan, sk, hole, my_evals);
                 q_start = 0;
                 shrunk = true;
                 if (chunk > 1) { chunk = chunk / 4 > 1 ? chunk / 4 : 1; continue; }
                 for (int j = 0; j < kNA; ++j) {
-                    run(s0, s0 + 1, alive & (1u << j), part == 1);
-                    drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+                    run_piece<DENSE>(sh, R, alive & (1u << j), a1ok, m, s0, s0 + 1, pflags);
+                    drain_queue(sh, plan, sk, hole, my_evals);
                 }
             } else if (qn > (u32)(kWarpQueue / 2)) {
-                drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+                drain_queue(sh, plan, sk, hole, my_evals);
                 q_start = 0;
             } else {
                 q_start = qn;
@@ -1694,12 +1771,12 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
         }
     }
     if ((threadIdx.x & 31) == 0) sh.chunk_hint[warp] = shrunk ? chunk : (chunk * 2 < kChunkB ? chunk * 2 : kChunkB);
-    if (drain_at_end) drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+    if (drain_at_end) drain_queue(sh, plan, sk, hole, my_evals);
 }
 
 // Fills the broadcast side of a tile: operand values at probe 0, with everything the loops
 // need that depends on them alone.  Returns (per thread) whether a value did not fit int32.
-__device__ __forceinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, int m, int n_bc) {
+__device__ __noinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, int m, int n_bc) {
     const SegDev& seg = sh.mseg[m];
     MemberState& mbs = sh.mb[m];
     const u64 bc_first = mbs.bc_first;
@@ -1786,13 +1863,20 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
     const bool resident = keep && sh.kept_head == seg_index;       // this family's broadcast operands are in the tile
     const int reg_nt = sh.seg.reg_nt, reg_size = sh.seg.reg_size;
     const bool second = hole->second != 0 || (hole->second_ok != 0 && sh.adapt_second != 0);
-    load_family(sh, plan, seg_index, family);
+    if (!resident) load_family(sh, plan, seg_index, family);       // (a resident family's segments are still in place)
+    if ((threadIdx.x & 31) == 0) {                      // the tag that this tile's hits carry in the warp's queue
+        const int w = threadIdx.x >> 5;
+        sh.wq_first[w][sh.wq_tiles[w] & (u32)(kQueueTags - 1)] = reg_first;
+        sh.wq_tiles[w] += 1u;
+    }
     if (threadIdx.x == 0) {
         sh.reg_wide = 0;
         sh.p1_on = second ? 1 : 0;
         sh.p1_A = hole->aff_Aj[1]; sh.p1_B = hole->aff_Bj[1]; sh.p1_spec = (u64)hole->probe_spec[1];
         sh.p1_rng = (hole->rng_okmask >> 1) & 1u;
         sh.p1_lo = hole->rng_lo[1]; sh.p1_hi = hole->rng_hi[1];
+        sh.h_A = hole->aff_A; sh.h_tq = (u64)hole->probe_spec[0] - hole->aff_B;
+        sh.h_rng_lo = hole->rng_lo[0]; sh.h_rng_hi = hole->rng_hi[0]; sh.h_aff_ok = hole->aff_ok;
     }
     // this thread's operands: kNA consecutive ranks
     RegVals RV;
@@ -1809,6 +1893,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
                                    RV.p1, nullptr, a1ok);
     __syncthreads();                                    // the members' segments are in place, reg_wide is clear
     if (wide_reg) sh.reg_wide = 1;
+    if (threadIdx.x == 0) { sh.q_sketch = sh.seg.sketch; sh.q_hole = sh.seg.hole; }      // (read at the top of a later ticket)
     // broadcast operands of member m: tile bc_tile0 of the head (a family's other members have one tile)
     auto n_bc_of = [&](int m) {
         const SegDev& seg = sh.mseg[m];
@@ -1823,6 +1908,9 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         mbs.lo = keep ? seg.bc_base : 0;
         mbs.hi = keep ? seg.bc_base + n_bc_of(m) : kBcTile;
         mbs.n = 0; mbs.nspecial = 0; mbs.wide = 0; mbs.mod_possible = 0;
+        u32 opip = 0, mask = 0;
+        for (int o = 0; o < seg.n_ops; ++o) { opip |= (u32)o << (3 * op_slot(seg.op[o])); mask |= 1u << op_slot(seg.op[o]); }
+        mbs.opip = opip; mbs.mask = mask;
     };
     if (keep) {
         // Every member's operands fit the tile side by side.  They are filled once (by the first
@@ -1842,10 +1930,17 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
             if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-            if (seg.swap) tile_body<true, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
-            else tile_body<false, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
+            tile_body<DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
         }
-        drain_queue(sh, plan, sk, hole, reg_first, my_evals);
+        // In the sparse form of the kernel, when the CTA came to this ticket from another one of the same
+        // family (a long run of them is likely), a handful of hits waits for the next (eval_kernel empties the queues before anything
+        // else runs); enough of them, or old ones, are checked now.
+        const int w = threadIdx.x >> 5;
+        __syncwarp();
+        const u32 qn = sh.wq_n[w], age = sh.wq_age[w];
+        __syncwarp();
+        if (DENSE || !resident || qn >= kDrainMin || age + 2u >= (u32)kQueueTags) drain_queue(sh, plan, sk, hole, my_evals);
+        else if ((threadIdx.x & 31) == 0) { sh.wq_age[w] = age + 1u; if (qn) sh.q_waiting = 1; }
         return;
     }
     for (int m = 0; m < family; ++m) {                  // members take turns in the tile
@@ -1857,8 +1952,7 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
         const SegDev& seg = sh.mseg[m];
         const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
         if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
-        if (seg.swap) tile_body<true, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
-        else tile_body<false, DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
+        tile_body<DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, true, my_evals);
     }
 }
 
@@ -1871,7 +1965,11 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
     u64 my_evals = 0;
     if (threadIdx.x <= kMaxSize) { sh.match_count[threadIdx.x] = 0; sh.min_rank[threadIdx.x] = ~0ull; }
     if (threadIdx.x == 0) { sh.cur_acc = -1; sh.kept_head = -1; sh.filter_survivors = 0; sh.probe_survivors = 0; sh.ops_skipped = 0; sh.adapt_second = 0; sh.filter_tests = 0; sh.tile_cands = 0; }
-    if (threadIdx.x < kWarps) { sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0; }
+    if (threadIdx.x < kWarps) {
+        sh.chunk_hint[threadIdx.x] = kChunkB; sh.wq_n[threadIdx.x] = 0; sh.wq_over[threadIdx.x] = 0; sh.wmember[threadIdx.x] = 0;
+        sh.wq_tiles[threadIdx.x] = 0; sh.wq_age[threadIdx.x] = 0;
+    }
+    if (threadIdx.x == 0) { sh.q_sketch = 0; sh.q_hole = 0; sh.q_waiting = 0; }
     __syncthreads();
     for (;;) {
         if (threadIdx.x == 0) {
@@ -1881,7 +1979,10 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
         }
         __syncthreads();
         const u64 t = sh.ticket;
-        if (t >= plan.n_tickets) break;
+        if (t >= plan.n_tickets) {
+            if (!DENSE && sh.q_waiting && sh.wq_n[threadIdx.x >> 5] != 0) drain_waiting(sh, plan, my_evals);
+            break;
+        }
         if (threadIdx.x < 32) {
             // last segment with first_ticket <= t: a 32-way search, one probe per lane and round
             int lo = 0, n = plan.n_segs;
@@ -1900,6 +2001,13 @@ __global__ void __launch_bounds__(kThreads, XP_MIN_CTAS) eval_kernel(const PlanD
             load_segment(sh, plan, lo);
         }
         __syncthreads();
+        // Hits that wait in the warps' queues belong to the family resident in the tile: any ticket but
+        // another one of that family has them checked first (their segments and operands are about to go).
+        if (!DENSE && sh.q_waiting && !(sh.seg.kind == kSegTile && sh.seg.bc_keep != 0 && sh.kept_head == sh.seg_index)) {
+            if (sh.wq_n[threadIdx.x >> 5] != 0) drain_waiting(sh, plan, my_evals);
+            __syncthreads();
+            if (threadIdx.x == 0) sh.q_waiting = 0;
+        }
         if (sh.seg.acc != sh.cur_acc) {
             flush_acc(sh, plan, my_evals);
             if (threadIdx.x == 0) sh.cur_acc = sh.seg.acc;
@@ -2452,7 +2560,7 @@ cudaError_t launch_prepare(const LoadJob* jobs, int n_jobs, cudaStream_t stream)
 
 cudaError_t launch_bigvalues(const LoadJob* jobs, int n_jobs, u64 most_entries, cudaStream_t stream) {
     if (most_entries == 0 || n_jobs <= 0) return cudaSuccess;
-    bigvalue_kernel<<<dim3((unsigned)((most_entries + 255) / 256), (unsigned)n_jobs), 256, 0, stream>>>(jobs);
+    bigvalue_kernel<<<dim3((unsigned)((most_entries / kBigPerThread + 255) / 256 + 1), (unsigned)n_jobs), 256, 0, stream>>>(jobs);
     return cudaGetLastError();
 }
 
