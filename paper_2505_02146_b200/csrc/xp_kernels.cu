@@ -1232,6 +1232,40 @@ __device__ __noinline__ bool probe1_pass(const EvalShared& sh, int op, bool a_ok
 // (a1ok: bit j says that this thread's operand j is known exactly at probe 1)
 #define XP_P1(op, j, s) probe1_pass(sh, op, (a1ok >> (j)) & 1u, (i32)R->p1[j], sh.bc_meta[s].meta, sh.bc_meta[s].pad, SWAP)
 
+// The second look, first cut (dense form of the loops): the hits `m` of operator OP between this
+// thread's operands and broadcast slot s are held against the spec at probe 1 in 32-bit arithmetic,
+// inline.  It is a necessary condition for the exact test of probe1_pass (the low 32 bits of both
+// sides must agree; a zero divisor makes the candidate undefined there), like the filter itself, so
+// the few hits it leaves still go through that test.  Where the spec is small at the first probe and
+// one candidate in a hundred agrees with it there, this keeps the out-of-line routines rare.
+// Operands that are not known exactly at probe 1 are kept.  Returns the bits that remain.
+template <int OP, bool SWAP>
+__device__ __forceinline__ u32 p1_first_cut(const EvalShared& sh, const RegVals* R, u32 a1ok, int s, u32 m) {
+    if (!sh.p1_on || sh.p1_rng) return m;
+    const u32 meta = sh.bc_meta[s].meta;
+    if (!(meta >> 31)) return m;
+    const u32 b1 = sh.bc_meta[s].pad, A1 = (u32)sh.p1_A, t1 = (u32)sh.p1_spec - (u32)sh.p1_B;
+    u32 out = m & ~a1ok;
+    for (u32 k = m & a1ok; k; k &= k - 1) {
+        const int j = __ffs((int)k) - 1;
+        const u32 a1 = R->p1[j];
+        const u32 x = SWAP ? b1 : a1, y = SWAP ? a1 : b1;
+        u32 v;
+        bool ok = true;
+        if (OP == XP_OP_ADD) v = x + y;
+        else if (OP == XP_OP_SUB) v = x - y;
+        else if (OP == XP_OP_MUL) v = x * y;
+        else {                                          // / and %: exact in int32 but for the one quotient that leaves it
+            ok = y != 0u;
+            const i32 d = ok ? (i32)y : 1;
+            if (OP == XP_OP_DIV) v = y == 0xffffffffu ? 0u - x : (u32)((i32)x / d);
+            else v = y == 0xffffffffu ? 0u : (u32)((i32)x % d);
+        }
+        if (ok && v * A1 == t1) out |= 1u << j;
+    }
+    return out;
+}
+
 // The loops below are separate (not inlined) functions on purpose: each copies the thread's
 // register-side operands into registers, derives what it needs of them and runs with a small
 // live set, instead of sharing one large frame with the rest of the kernel.
@@ -1334,6 +1368,11 @@ __device__ __noinline__ void ring_pass(EvalShared& sh, const RegVals* R, u32 ali
             if (MASK & 4u) m_mul |= (u32)(aA[j] * e.mul_b + e.mul_nt == 0u) << j;
         }
         m_as &= alive; m_mul &= alive;
+        if (DENSE) {
+            if (MASK & 3u) m_as = ((MASK & 1u) ? p1_first_cut<XP_OP_ADD, SWAP>(sh, R, a1ok, s, m_as) : 0u) |
+                                  ((MASK & 2u) ? p1_first_cut<XP_OP_SUB, SWAP>(sh, R, a1ok, s, m_as) : 0u);
+            if (MASK & 4u) m_mul = p1_first_cut<XP_OP_MUL, SWAP>(sh, R, a1ok, s, m_mul);
+        }
         if (m_as | m_mul) emit_ring(sh, R, a1ok, s, m_as, m_mul, A, tp, opip, MASK, SWAP);
     };
     // One warp vote per kRingGroup broadcast operands (fewer at the end of the run).  The rare path has
@@ -1455,6 +1494,10 @@ __device__ __noinline__ void div_pass(EvalShared& sh, const RegVals* R, u32 aliv
         // register operands that are invalid, or (SWAP) zero divisors, are dropped here
         const u32 keep = SWAP ? alive & nz : alive;
         mq &= keep; mr &= keep;
+        if (DENSE) {
+            if (MASK & 1u) mq = p1_first_cut<XP_OP_DIV, SWAP>(sh, R, a1ok, s, mq);
+            if (MASK & 2u) mr = p1_first_cut<XP_OP_MOD, SWAP>(sh, R, a1ok, s, mr);
+        }
         if (mq | mr) emit_pairs(sh, R, a1ok, s, mq, XP_OP_DIV, mr, XP_OP_MOD, opip, SWAP);
     };
     for (int s = s0; s < s1; s += kDivGroup) {          // one warp vote per kDivGroup broadcast operands; one rare-path site
