@@ -1817,6 +1817,63 @@ __device__ __forceinline__ void tile_body(EvalShared& sh, const PlanDev& plan, c
     if (drain_at_end) drain_queue(sh, plan, sk, hole, my_evals);
 }
 
+// Members with a handful of broadcast operands and no operator but + and - (the large typed search:
+// `E + v`, `E - v`, `v + E`, `v - E` over 4 variables) have a few dozen candidates per thread and
+// tile: the general walk above, with its chunks, votes and choice of loop, spends far more
+// instructions around them than on them, and most of those from cold code.  This compact routine
+// takes all such members of the family in one call and tests their candidates directly (no votes: a
+// lane with a hit goes to the rare path on its own).  Returns the set of members it has done; a
+// member is left to the general walk when the warp's queue is too full to be sure of room, or ran
+// over (its hits are then forgotten first).
+constexpr u32 kTinyOperands = 16;
+__device__ __forceinline__ bool tiny_member(const EvalShared& sh, int m) {      // (the same for every thread of the CTA)
+    const MemberState& mbs = sh.mb[m];
+    return (mbs.mask & ~3u) == 0u && mbs.n + mbs.nspecial <= kTinyOperands && sh.h_aff_ok != 0 &&
+           (sh.reg_wide | mbs.wide | sh.mseg[m].generic) == 0;
+}
+__device__ __noinline__ u32 tiny_ring(EvalShared& sh, const RegVals* R, u32 alive, u32 a1ok, int family) {
+    const int warp = threadIdx.x >> 5;
+    const u32 A = (u32)sh.h_A, tp = (u32)sh.h_tq;
+    u32 aA[kNA];
+#pragma unroll
+    for (int j = 0; j < kNA; ++j) aA[j] = R->lo[j] * A;
+    u32 done = 0;
+    for (int m = 0; m < family; ++m) {
+        if (!tiny_member(sh, m)) continue;
+        const SegDev& seg = sh.mseg[m];
+        const MemberState& mbs = sh.mb[m];
+        const bool SWAP = seg.swap != 0;
+        const u32 mask = mbs.mask;
+        __syncwarp();
+        const u32 q_start = sh.wq_n[warp];
+        if (q_start > (u32)(kWarpQueue / 2)) continue;
+        if ((threadIdx.x & 31) == 0) sh.wmember[warp] = (u32)m | (((sh.wq_tiles[warp] - 1u) & (u32)(kQueueTags - 1)) << 3);
+        __syncwarp();
+        for (int part = 0; part < 2; ++part) {          // the general operands, then those of magnitude <= 1
+            const int lo = part == 0 ? mbs.lo : mbs.hi - (int)mbs.nspecial, hi = part == 0 ? mbs.lo + (int)mbs.n : mbs.hi;
+            for (int s = lo; s < hi; ++s) {
+                const u32 t_add = sh.bc_ring[s].t_add;  // A*a must equal this for +, and t_sub for - (see ring_pass)
+                const u32 t_sub = SWAP ? 0u - t_add : 2u * tp - t_add;
+                u32 hits = 0;
+#pragma unroll
+                for (int j = 0; j < kNA; ++j)
+                    hits |= (u32)(((mask & 1u) && aA[j] == t_add) || ((mask & 2u) && aA[j] == t_sub)) << j;
+                hits &= alive;
+                if (hits) emit_ring(sh, R, a1ok, s, hits, 0u, A, tp, mbs.opip, mask, SWAP);
+            }
+        }
+        __syncwarp();
+        if (sh.wq_over[warp] != 0) {                    // the queue ran over: this member's hits are forgotten
+            __syncwarp();
+            if ((threadIdx.x & 31) == 0) { sh.wq_n[warp] = q_start; sh.wq_over[warp] = 0; }
+            continue;
+        }
+        warp_tally(&sh.filter_tests, (u32)__popc(alive) * (mbs.n + mbs.nspecial) * (u32)seg.n_ops);
+        done |= 1u << m;
+    }
+    return done;
+}
+
 // Fills the broadcast side of a tile: operand values at probe 0, with everything the loops
 // need that depends on them alone.  Returns (per thread) whether a value did not fit int32.
 __device__ __noinline__ bool fill_bc_operands(EvalShared& sh, const GrammarDev* g, const HoleDev* hole, int m, int n_bc) {
@@ -1968,11 +2025,19 @@ __device__ __noinline__ void tile_ticket(EvalShared& sh, const PlanDev& plan, co
             if (threadIdx.x == 0) sh.kept_head = seg_index;
         }
         __syncthreads();
+        // (sparse form) the members with next to no work per tile first, all in one compact routine
+        const u32 tiny_done = DENSE ? 0u : tiny_ring(sh, &RV, alive, a1ok, family);
+        bool first = true;
         for (int m = 0; m < family; ++m) {
             const SegDev& seg = sh.mseg[m];
-            if (m > 0) __syncthreads();
             const u64 pairs = (u64)n_reg * (u64)n_bc_of(m);
             if (threadIdx.x == 0) sh.tile_cands += pairs * (u64)seg.n_ops;
+            const bool tiny = !DENSE && tiny_member(sh, m);
+            if (!tiny) {                                // (the same for every thread of the CTA)
+                if (!first) __syncthreads();            // keeps the CTA's warps in the same loop from member to member
+                first = false;
+            }
+            if ((tiny_done >> m) & 1u) continue;
             tile_body<DENSE>(sh, plan, sk, hole, m, reg_first, pairs, &RV, a1ok, alive, false, my_evals);
         }
         // In the sparse form of the kernel, when the CTA came to this ticket from another one of the same
