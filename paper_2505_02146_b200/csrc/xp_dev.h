@@ -87,9 +87,10 @@ struct HoleDev {
     // Hits of the filter are checked exactly there (two lookups and one operation per probe); only
     // probes without tables need the candidate unranked in full.
     // second: filter hits are also checked exactly at probe 1 before they are queued (needs tables, a
-    // defined spec and an affine context at probe 1); sample_pass0: how many of the candidates
-    // sampled at load satisfied probe 0 (a high rate makes the second look worth its cost).
-    i32 second, sample_pass0, sample_n;
+    // defined spec and an affine context at probe 1); sample_pass0: how many of the sample_n small
+    // candidates sampled at load satisfied probe 0, sample_big: how many of the kPrepBigSamples random
+    // candidates of the largest size did (a high rate of either makes the second look worth its cost).
+    i32 second, sample_pass0, sample_n, sample_big;
     i32 second_ok;                                // the second look is possible (tables, spec and context at probe 1): a
                                                   // CTA that sees many filter hits for this hole turns it on for itself
     // Set by the host before the load's kernels run: the largest subtree size and the number of

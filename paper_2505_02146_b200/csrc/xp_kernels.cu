@@ -119,11 +119,14 @@ __device__ bool ctx_interval(const HoleDev* hole, const i64* pt, i64 spec, i64& 
     return false;
 }
 
+constexpr int kPrepBigSamples = 8192;                    // random candidates of the largest size, held against the first probe
+
 // The context at every probe (affine in the hole, or a comparison; one thread per probe), and what
 // the rest of the load and the searches go by.  Called by every thread of the CTA once the n
 // probes (ids, coordinates, spec values) are in place; ncand / pass0: how many sampled candidates
-// the probe choice looked at and how many of them satisfied the first probe.
-__device__ __forceinline__ void probe_contexts(HoleDev* hole, int n, int ncand, int pass0) {
+// the probe choice looked at and how many of them satisfied the first probe; big_hits: how many of
+// the kPrepBigSamples candidates of the largest size did.
+__device__ __forceinline__ void probe_contexts(HoleDev* hole, int n, int ncand, int pass0, int big_hits) {
     const int t = threadIdx.x;
     if (t < kMaxProbe) {
         u64 A = 0, B = 0;
@@ -155,7 +158,9 @@ __device__ __forceinline__ void probe_contexts(HoleDev* hole, int n, int ncand, 
             // fills, which large tiles amortise anyway) and wherever the sampled candidates say that
             // probe 0 alone lets many through.
             const bool possible = n >= 2 && probes >= 2 && ((spec_ok & (amask | rmask)) >> 1 & 1u);
-            const bool frequent = ncand > 0 && (u64)pass0 * 256 >= (u64)ncand;
+            // (one in 256 of the small sample, or one in 4096 of the large candidates: the dense form of the
+            // loops wins from about there, see kAdaptRate)
+            const bool frequent = (ncand > 0 && (u64)pass0 * 256 >= (u64)ncand) || (u64)big_hits * 4096 >= (u64)kPrepBigSamples;
             hole->second = possible && (hole->small_search || frequent) ? 1 : 0;
             hole->second_ok = possible ? 1 : 0;
         }
@@ -184,6 +189,7 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
     __shared__ u32 s_count[kProbeSamples];
     __shared__ u64 s_chosen;
     __shared__ int s_best;
+    __shared__ int s_big_hits;
     const int t = threadIdx.x;
     const int ns = s->n_samples;
     const int nv = s->n_vars;
@@ -277,11 +283,38 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
     if (t == 0) {
         hole->n_probe = n;
         if (n == 0) hole->probe_spec_ok = 0;
-        hole->sample_pass0 = pass0;                       // sampled candidates that satisfy the first probe chosen
-        hole->sample_n = ncand;
+        s_big_hits = 0;
     }
     __syncthreads();
-    probe_contexts(hole, n, ncand, pass0);
+    // How often the first probe lets a candidate through is estimated once more on random candidates
+    // of the largest size, where nearly all of a search's work is: the behaviour of expressions of one
+    // to five nodes says little about those of nine.
+    int big_size = hole->max_size;
+    while (big_size > 1 && g->cnt[hole->start_nt][big_size] == 0) --big_size;
+    const bool sample_big = n > 0 && big_size >= 3 && (hole->probe_spec_ok & 1u);
+    if (sample_big) {
+        const u64 cnt = g->cnt[hole->start_nt][big_size];
+        i64 pt0[kMaxVars];
+        for (int d = 0; d < nv; ++d) pt0[d] = hole->probe_pt[0][d];
+        const i64 spec0 = hole->probe_spec[0];
+        for (int c = t; c < kPrepBigSamples; c += kPrepThreads) {
+            u64 x = (u64)(c + 1) * 0x9E3779B97F4A7C15ull;     // (a fixed scramble of the sample's number)
+            x ^= x >> 29; x *= 0xBF58476D1CE4E5B9ull; x ^= x >> 32;
+            u32 code[kMaxSize];
+            const int len = unrank(g, hole->start_nt, big_size, __umul64hi(x, cnt), code);
+            i64 v;
+            if (eval_cand(code, len, g->leaves, pt0, v) && ctx_matches(hole, pt0, v, spec0)) atomicAdd(&s_big_hits, 1);
+        }
+    }
+    __syncthreads();
+    const int big_hits = sample_big ? s_big_hits : 0;
+    if (t == 0) {
+        hole->sample_pass0 = pass0;                       // sampled candidates that satisfy the first probe chosen
+        hole->sample_n = ncand;
+        hole->sample_big = big_hits;
+    }
+    __syncthreads();
+    probe_contexts(hole, n, ncand, pass0, big_hits);
 }
 
 // The probes of a hole replaced by the host (xp_sketch_refine: points that ended whole-domain
@@ -305,7 +338,7 @@ __global__ void __launch_bounds__(32) reprobe_kernel(const LoadJob* jobs) {
     const u32 okmask = __ballot_sync(0xffffffffu, ok);
     if (t == 0) hole->probe_spec_ok = okmask;
     __syncthreads();
-    probe_contexts(hole, n, hole->sample_n, hole->sample_pass0);
+    probe_contexts(hole, n, hole->sample_n, hole->sample_pass0, hole->sample_big);
 }
 
 // ------------------------------------------------------------------------------------------
