@@ -212,7 +212,7 @@ def test_small_parity_cases_under_the_checked_build():
     cases = "config1 or contexts or repeated or min_max or edge or windows or table_domain"
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
                         "tests/test_parity_gpu.py", "tests/test_features_gpu.py", "-k",
-                        f"({cases} or family or refinement or rank_windows) and not checked_build"],
+                        f"({cases} or family or refinement or rank_windows or one_point) and not checked_build"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=1500)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-1000:]
     assert " passed" in r.stdout
@@ -256,3 +256,26 @@ def test_constant_only_holes(xp):
     assert res2[0].least_text == "48" and res2[0].solved
     sk3 = Sketch(g2, [Hole(1, 1, ctx=parse_expr("(r*HOLE)+c", vs2), spec_expr=parse_expr("(r*50)+c", vs2))], name="no such pitch")
     assert not check_sketch(xp, sk3)[0].solved
+
+
+def test_one_point_domain_where_a_large_share_of_the_candidates_match(xp):
+    """A typed grammar of the large search's shape (leaves, E+E, E-E, E*K, E/P, E%P) on a domain of one
+    point: there is one probe, so no second look, and every candidate whose value at that point is
+    the target is a match.  Hits are frequent in every member of a family, the small ones included,
+    the warps' hit queues run over, and the global survivor queue fills up; counts and least
+    solutions must still be exact."""
+    vs = [Variable("a", 3, 4), Variable("b", 5, 6), Variable("c", 2, 3), Variable("d", 7, 8)]
+    prods = [Production(lhs=0, kind=P_VAR, var=i) for i in range(4)]
+    prods += [Production(lhs=1, kind=P_CONST, value=k) for k in (-2, -1, 2, 3, 4, 6)]
+    prods += [Production(lhs=2, kind=P_CONST, value=p) for p in (2, 3, 4, 5)]
+    prods += [Production(lhs=0, kind=P_BIN, op=OP_CODE["+"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["-"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["*"], left=0, right=1),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["/"], left=0, right=2),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["%"], left=0, right=2)]
+    g = Grammar(vs, 3, prods)
+    for spec in ["a+b", "c-c", "(d*3)-1"]:
+        sk = Sketch(g, [Hole(0, 9, spec_expr=parse_expr(spec, vs))], name=f"one point, target {spec}")
+        res = check_sketch(xp, sk)
+        assert res[0].cand_count[1:10:2] == [4, 88, 2640, 94688, 3769920]
+        assert sum(res[0].match_count) > 1000
