@@ -327,7 +327,9 @@ extern "C" xp_status xp_grammar_unrank(const xp_grammar* g, int32_t nt, int32_t 
     return XP_OK;
 }
 
-static xp_status grammar_to_device(xp_grammar* g, size_t* copied) {
+// (staging: page-locked memory of the load at hand, or null; with it the copy is queued on the
+// load's stream like the sketch's own copies and nobody waits for it here)
+static xp_status grammar_to_device(xp_grammar* g, size_t* copied, PinnedArena* staging) {
     *copied = 0;
     std::lock_guard<std::mutex> lock(g->mu);
     if (g->d_g) {
@@ -355,11 +357,16 @@ static xp_status grammar_to_device(xp_grammar* g, size_t* copied) {
     g->d_bytes = granted;
     h.leaves = (const LeafDev*)(block + off_leaves);
     h.bins = (const BinDev*)(block + off_bins);
-    std::vector<char> stage(total, 0);
-    memcpy(&stage[0], &h, sizeof(h));
-    if (!g->leaves.empty()) memcpy(&stage[off_leaves], g->leaves.data(), sizeof(LeafDev) * g->leaves.size());
-    if (!g->bins.empty()) memcpy(&stage[off_bins], g->bins.data(), sizeof(BinDev) * g->bins.size());
-    cudaError_t e = cudaMemcpy(block, stage.data(), total, cudaMemcpyHostToDevice);
+    std::vector<char> stage_own;
+    char* stage = staging ? staging->take(total) : nullptr;
+    const bool queued = stage != nullptr;
+    if (!stage) { stage_own.resize(total); stage = stage_own.data(); }
+    memset(stage, 0, total);
+    memcpy(stage, &h, sizeof(h));
+    if (!g->leaves.empty()) memcpy(stage + off_leaves, g->leaves.data(), sizeof(LeafDev) * g->leaves.size());
+    if (!g->bins.empty()) memcpy(stage + off_bins, g->bins.data(), sizeof(BinDev) * g->bins.size());
+    cudaError_t e = queued ? cudaMemcpyAsync(block, stage, total, cudaMemcpyHostToDevice, nullptr)
+                           : cudaMemcpy(block, stage, total, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { pool_release(block, g->d_bytes, g->d_device); return fail(XP_ERR_CUDA, std::string("cudaMemcpy: ") + cudaGetErrorString(e)); }
     g->d_g = (GrammarDev*)block;
     *copied = total;
@@ -510,7 +517,7 @@ static xp_status load_begin(const xp_grammar* gc, const xp_sketch_desc* d, LoadS
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(XP_ERR_CUDA, "no CUDA device is usable");
     size_t grammar_bytes = 0;
-    xp_status st = grammar_to_device(g, &grammar_bytes);
+    xp_status st = grammar_to_device(g, &grammar_bytes, L->pinned);
     if (st != XP_OK) return st;
 
     xp_sketch* s = new (std::nothrow) xp_sketch;
