@@ -279,3 +279,23 @@ def test_one_point_domain_where_a_large_share_of_the_candidates_match(xp):
         res = check_sketch(xp, sk)
         assert res[0].cand_count[1:10:2] == [4, 88, 2640, 94688, 3769920]
         assert sum(res[0].match_count) > 1000
+
+
+def test_negation_as_zero_minus_operand(xp):
+    """Negation enters a grammar as  E -> Z - E  with  Z -> 0  (the reading taken for a unary minus): a typed
+    production like the others, through the filter and both exact paths."""
+    vs = [Variable("i", 0, 6), Variable("j", -2, 5)]
+    prods = [Production(lhs=0, kind=P_VAR, var=0), Production(lhs=0, kind=P_VAR, var=1)]
+    prods += [Production(lhs=0, kind=P_CONST, value=c) for c in (1, 2, 3)]
+    prods += [Production(lhs=1, kind=P_CONST, value=0)]
+    prods += [Production(lhs=0, kind=P_BIN, op=OP_CODE["+"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["*"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["-"], left=1, right=0)]
+    g = Grammar(vs, 2, prods)
+    for spec, ctx, least in [("0-(i+j)", "", "(0-(i+j))"), ("(0-i)*3", "", None), ("(0-(i*j))+7", "HOLE+7", "(i*(0-j))")]:
+        sk = Sketch(g, [Hole(0, 7 if not ctx else 5, ctx=parse_expr(ctx, vs) if ctx else [], spec_expr=parse_expr(spec, vs))],
+                    name=f"negation: {spec}")
+        for flags in PATHS:
+            res = check_sketch(xp, sk, flags=flags)
+        if least:
+            assert res[0].least_text == least

@@ -555,3 +555,34 @@ def test_behaviour_mode_on_a_partial_signature_reports_an_unverified_hit():
     sk3 = Sketch(g, [Hole(0, 3, ctx=parse_expr("HOLE/4", vs), spec_expr=parse_expr("(i*j)/4", vs))])
     r3 = oracle.behaviours(sk3, list(range(64)))
     assert r3.sig_matches >= 1 and r3.solved and r3.hit_verified
+
+
+def _negation_grammar(vs):
+    """Negation as the production  E -> Z - E  with the one-constant nonterminal  Z -> 0  (the reading
+    taken for a unary minus: it costs two nodes more than its operand, not one)."""
+    from xp_instances.model import OP_CODE, P_BIN, P_CONST, P_VAR, Grammar, Production
+    prods = [Production(lhs=0, kind=P_VAR, var=i) for i in range(len(vs))]
+    prods += [Production(lhs=0, kind=P_CONST, value=c) for c in (1, 2, 3)]
+    prods += [Production(lhs=1, kind=P_CONST, value=0)]
+    prods += [Production(lhs=0, kind=P_BIN, op=OP_CODE["+"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["*"], left=0, right=0),
+              Production(lhs=0, kind=P_BIN, op=OP_CODE["-"], left=1, right=0)]
+    return Grammar(vs, 2, prods)
+
+
+def test_negation_as_zero_minus_operand():
+    """Counts by the closed form (with L leaves: n1 = L, n3 = 2 L^2 + L, n5 = 2 (2 n1 n3) + n3), results
+    equal to brute force, and the least solution of a negated target is the `0 - e` form."""
+    vs = [Variable("i", 0, 5), Variable("j", -2, 3)]
+    g = _negation_grammar(vs)
+    L = 5
+    n3 = 2 * L * L + L
+    assert oracle.counts(g, 0, 5) == [0, L, 0, n3, 0, 4 * L * n3 + n3]
+    for spec, least in [("0-(i+j)", "(0-(i+j))"), ("(0-i)*3", None), ("0-i", "(0-i)")]:
+        sk = Sketch(g, [Hole(0, 5, spec_expr=parse_expr(spec, vs))])
+        got = oracle.repair_hole(sk)
+        cand, match, want, _ = pybrute.repair(sk)
+        assert got.cand_count == cand and got.match_count == match
+        assert (got.solved, got.least_size, got.least_rank, got.least_text) == ((True,) + want if want else (False, 0, 0, ""))
+        if least:
+            assert got.least_text == least
