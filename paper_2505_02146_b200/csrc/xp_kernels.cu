@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_kernel(const LoadJob* jo
     // to five nodes says little about those of nine.
     int big_size = hole->max_size;
     while (big_size > 1 && g->cnt[hole->start_nt][big_size] == 0) --big_size;
-    const bool sample_big = n > 0 && big_size >= 3 && (hole->probe_spec_ok & 1u);
+    const bool sample_big = n > 0 && big_size >= 3 && (hole->probe_spec_ok & 1u) && !hole->small_search;      // (a small search takes the second look anyway)
     if (sample_big) {
         const u64 cnt = g->cnt[hole->start_nt][big_size];
         i64 pt0[kMaxVars];
